@@ -1,0 +1,215 @@
+/*
+ * CPU oracle for the Monarch multiply (Dao et al., arXiv 2204.00595).
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain fp64 statement of
+ * what the hot path computes.  It shares nothing with the CUDA library: no
+ * header, no helper, no table.  Only tests, the smoke check and the CPU
+ * baseline leg of the benchmark may call it.
+ *
+ * Notation (0-indexed; the paper's Section 3.3 uses 1-indexed subscripts):
+ *   n = m*m                                   (Definition 3.1)
+ *   x[t][k*m + i]    token t, viewed as an m x m matrix x_{ki}
+ *   R[k][j][i]       block k of R, output row j, input column i
+ *   L[j][l][k]       block j of L, output row l, input column k
+ *   u[t][k][j]       the paper's intermediate "y_{kj}" of step 1
+ *   y[t][l*m + j]    the paper's "z_{lj}" of steps 2-3, flattened l-major
+ *
+ * Every loop nest below is the formula of the cited passage written out;
+ * there is no blocking, fusion or reordering.  OpenMP only distributes
+ * independent tokens (or independent weight blocks) over host cores.
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+int oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* Step 1 of the multiply (Section 3.3, "Steps to multiply x by a Monarch
+ * matrix", item 1):  u_{kj} = sum_i R_{kji} x_{ki}. */
+static void step1_one_token(const double *x, const double *R, double *u, int m)
+{
+    for (int k = 0; k < m; ++k)
+        for (int j = 0; j < m; ++j) {
+            double acc = 0.0;
+            for (int i = 0; i < m; ++i)
+                acc += R[((size_t)k * m + j) * m + i] * x[(size_t)k * m + i];
+            u[(size_t)k * m + j] = acc;
+        }
+}
+
+/* Steps 2-3 (same passage, items 2 and 3):  z_{lj} = sum_k L_{jlk} u_{kj},
+ * returned flattened with l major and j minor. */
+static void step23_one_token(const double *u, const double *L, double *y, int m)
+{
+    for (int l = 0; l < m; ++l)
+        for (int j = 0; j < m; ++j) {
+            double acc = 0.0;
+            for (int k = 0; k < m; ++k)
+                acc += L[((size_t)j * m + l) * m + k] * u[(size_t)k * m + j];
+            y[(size_t)l * m + j] = acc;
+        }
+}
+
+/* y = M x for T tokens; u_out (T*n doubles) may be NULL. */
+int oracle_fwd(const double *x, const double *L, const double *R, double *y,
+               double *u_out, long T, int m)
+{
+    const size_t n = (size_t)m * m;
+    int fail = 0;
+#pragma omp parallel
+    {
+        double *u = (double *)malloc(n * sizeof(double));
+        if (!u) {
+#pragma omp atomic write
+            fail = 1;
+        }
+#pragma omp barrier
+        if (!fail) {
+#pragma omp for schedule(static)
+            for (long t = 0; t < T; ++t) {
+                step1_one_token(x + (size_t)t * n, R, u, m);
+                step23_one_token(u, L, y + (size_t)t * n, m);
+                if (u_out) memcpy(u_out + (size_t)t * n, u, n * sizeof(double));
+            }
+        }
+        free(u);
+    }
+    return fail;
+}
+
+/* Dense materialisation by the entry formula, Eq. (2):
+ *   M_{l j k i} = L_{j l k} R_{k j i},  row index l*m+j, column index k*m+i
+ * (the index map of Algorithm 1's reshape). Mdense is n x n row-major. */
+void oracle_dense(const double *L, const double *R, double *Mdense, int m)
+{
+    const size_t n = (size_t)m * m;
+    for (int l = 0; l < m; ++l)
+        for (int j = 0; j < m; ++j)
+            for (int k = 0; k < m; ++k)
+                for (int i = 0; i < m; ++i)
+                    Mdense[((size_t)l * m + j) * n + (size_t)k * m + i] =
+                        L[((size_t)j * m + l) * m + k] * R[((size_t)k * m + j) * m + i];
+}
+
+/* Gradients of  f = <dy, M x>  (the paper trains by automatic
+ * differentiation, Section 4; these are the adjoints of steps 1-3):
+ *   du[t][k][j] = sum_l L[j][l][k] dy[t][l*m+j]
+ *   dx[t][k*m+i] = sum_j R[k][j][i] du[t][k][j]
+ *   dL[j][l][k] = sum_t dy[t][l*m+j] u[t][k][j]
+ *   dR[k][j][i] = sum_t du[t][k][j] x[t][k*m+i]
+ * Any of dx, dL, dR may be NULL.  dL and dR are overwritten. */
+int oracle_bwd(const double *x, const double *dy, const double *L, const double *R,
+               double *dx, double *dL, double *dR, long T, int m)
+{
+    const size_t n = (size_t)m * m;
+    double *u = (double *)malloc((size_t)T * n * sizeof(double));
+    double *du = (double *)malloc((size_t)T * n * sizeof(double));
+    if (!u || !du) {
+        free(u);
+        free(du);
+        return 1;
+    }
+#pragma omp parallel for schedule(static)
+    for (long t = 0; t < T; ++t) {
+        const double *xt = x + (size_t)t * n;
+        const double *dyt = dy + (size_t)t * n;
+        double *ut = u + (size_t)t * n;
+        double *dut = du + (size_t)t * n;
+        step1_one_token(xt, R, ut, m);
+        for (int k = 0; k < m; ++k)
+            for (int j = 0; j < m; ++j) {
+                double acc = 0.0;
+                for (int l = 0; l < m; ++l)
+                    acc += L[((size_t)j * m + l) * m + k] * dyt[(size_t)l * m + j];
+                dut[(size_t)k * m + j] = acc;
+            }
+        if (dx) {
+            double *dxt = dx + (size_t)t * n;
+            for (int k = 0; k < m; ++k)
+                for (int i = 0; i < m; ++i) {
+                    double acc = 0.0;
+                    for (int j = 0; j < m; ++j)
+                        acc += R[((size_t)k * m + j) * m + i] * dut[(size_t)k * m + j];
+                    dxt[(size_t)k * m + i] = acc;
+                }
+        }
+    }
+    if (dL) {
+#pragma omp parallel for schedule(static)
+        for (int j = 0; j < m; ++j)
+            for (int l = 0; l < m; ++l)
+                for (int k = 0; k < m; ++k) {
+                    double acc = 0.0;
+                    for (long t = 0; t < T; ++t)
+                        acc += dy[(size_t)t * n + (size_t)l * m + j] *
+                               u[(size_t)t * n + (size_t)k * m + j];
+                    dL[((size_t)j * m + l) * m + k] = acc;
+                }
+    }
+    if (dR) {
+#pragma omp parallel for schedule(static)
+        for (int k = 0; k < m; ++k)
+            for (int j = 0; j < m; ++j)
+                for (int i = 0; i < m; ++i) {
+                    double acc = 0.0;
+                    for (long t = 0; t < T; ++t)
+                        acc += du[(size_t)t * n + (size_t)k * m + j] *
+                               x[(size_t)t * n + (size_t)k * m + i];
+                    dR[((size_t)k * m + j) * m + i] = acc;
+                }
+    }
+    free(u);
+    free(du);
+    return 0;
+}
+
+/* Monarch feed-forward block: the paper replaces the FFN weight matrices by
+ * Monarch matrices (Section 4, end-to-end setting); the block evaluated is
+ *   h = GELU(M1 x + b1),  y = M2 h + b2,  GELU(a) = a/2 (1 + erf(a/sqrt 2)). */
+int oracle_mlp_fwd(const double *x, const double *L1, const double *R1, const double *b1,
+                   const double *L2, const double *R2, const double *b2, double *y,
+                   long T, int m)
+{
+    const size_t n = (size_t)m * m;
+    int fail = 0;
+#pragma omp parallel
+    {
+        double *u = (double *)malloc(n * sizeof(double));
+        double *h = (double *)malloc(n * sizeof(double));
+        if (!u || !h) {
+#pragma omp atomic write
+            fail = 1;
+        }
+#pragma omp barrier
+        if (!fail) {
+#pragma omp for schedule(static)
+            for (long t = 0; t < T; ++t) {
+                step1_one_token(x + (size_t)t * n, R1, u, m);
+                step23_one_token(u, L1, h, m);
+                for (size_t q = 0; q < n; ++q) {
+                    const double a = h[q] + b1[q];
+                    h[q] = 0.5 * a * (1.0 + erf(a / sqrt(2.0)));
+                }
+                step1_one_token(h, R2, u, m);
+                double *yt = y + (size_t)t * n;
+                step23_one_token(u, L2, yt, m);
+                for (size_t q = 0; q < n; ++q) yt[q] += b2[q];
+            }
+        }
+        free(u);
+        free(h);
+    }
+    return fail;
+}

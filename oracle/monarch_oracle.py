@@ -1,0 +1,209 @@
+"""CPU oracle for the Monarch multiply (Dao et al., arXiv 2204.00595).
+
+TEST INFRASTRUCTURE ONLY.  Nothing in the product path may import this
+module: it exists so that tests, the smoke check and the benchmark's CPU
+baseline can compare the CUDA library against a plain fp64 statement of the
+paper's definitions.  It shares no code with the CUDA library.
+
+Two layers:
+
+* ``monarch_oracle.c`` - plain C loops in fp64 over the paper's multiply
+  steps (Section 3.3, steps 1-3), their adjoints, the entry formula Eq. (2)
+  and the Monarch feed-forward block.  Compiled on demand with gcc.
+* numpy routines in this file that restate *Definition 3.1 literally*
+  (explicit permutation and block-diagonal matrices) and Algorithm 1
+  (projection by rank-1 SVDs).  They are the independent routes the C loops
+  are pinned against; they only run at tiny n.
+
+All inputs and outputs are float64, C-contiguous:
+  x, y, dy, dx : [T, n]      L, R : [m, m, m] = [block, out, in]     n = m*m
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import sys
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "monarch_oracle.c")
+_LIB = os.path.join(_HERE, "libmonarch_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle (gcc -O2 -fopenmp) next to its source."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    tmp = _LIB + f".tmp{os.getpid()}"
+    cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c99", "-o", tmp, _SRC, "-lm"]
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        dp = ctypes.POINTER(ctypes.c_double)
+        lib.oracle_num_threads.restype = ctypes.c_int
+        lib.oracle_fwd.restype = ctypes.c_int
+        lib.oracle_fwd.argtypes = [dp, dp, dp, dp, dp, ctypes.c_long, ctypes.c_int]
+        lib.oracle_dense.restype = None
+        lib.oracle_dense.argtypes = [dp, dp, dp, ctypes.c_int]
+        lib.oracle_bwd.restype = ctypes.c_int
+        lib.oracle_bwd.argtypes = [dp] * 7 + [ctypes.c_long, ctypes.c_int]
+        lib.oracle_mlp_fwd.restype = ctypes.c_int
+        lib.oracle_mlp_fwd.argtypes = [dp] * 8 + [ctypes.c_long, ctypes.c_int]
+        _lib = lib
+    return _lib
+
+
+def num_threads() -> int:
+    """Host threads the C loops will use (OpenMP's max threads)."""
+    return int(_load().oracle_num_threads())
+
+
+def _f64(a, shape=None):
+    a = np.ascontiguousarray(a, dtype=np.float64)
+    if shape is not None and tuple(a.shape) != tuple(shape):
+        raise ValueError(f"expected shape {shape}, got {a.shape}")
+    return a
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(ctypes.POINTER(ctypes.c_double))
+
+
+def _m_of(L):
+    m = L.shape[0]
+    if L.shape != (m, m, m):
+        raise ValueError("weights must be [m, m, m]")
+    return m
+
+
+# --------------------------------------------------------------------------
+# C loops: steps 1-3, adjoints, Eq. (2), feed-forward block
+# --------------------------------------------------------------------------
+
+def fwd(x, L, R, return_u: bool = False):
+    """y = M x by the paper's steps 1-3 (Section 3.3).  x: [T, n]."""
+    L = _f64(L); R = _f64(R); m = _m_of(L); n = m * m
+    x = _f64(x); T = x.shape[0]
+    if x.shape != (T, n) or R.shape != L.shape:
+        raise ValueError("shape mismatch")
+    y = np.empty((T, n), dtype=np.float64)
+    u = np.empty((T, n), dtype=np.float64) if return_u else None
+    if _load().oracle_fwd(_p(x), _p(L), _p(R), _p(y), _p(u), T, m):
+        raise MemoryError("oracle_fwd")
+    return (y, u.reshape(T, m, m)) if return_u else y
+
+
+def dense(L, R):
+    """The n x n matrix M by the entry formula Eq. (2)."""
+    L = _f64(L); R = _f64(R); m = _m_of(L); n = m * m
+    M = np.empty((n, n), dtype=np.float64)
+    _load().oracle_dense(_p(L), _p(R), _p(M), m)
+    return M
+
+
+def bwd(x, dy, L, R, want=("dx", "dL", "dR")):
+    """Adjoints of steps 1-3 for f = <dy, Mx>: returns dict with dx, dL, dR."""
+    L = _f64(L); R = _f64(R); m = _m_of(L); n = m * m
+    x = _f64(x); dy = _f64(dy); T = x.shape[0]
+    if x.shape != (T, n) or dy.shape != (T, n):
+        raise ValueError("shape mismatch")
+    out = {}
+    if "dx" in want:
+        out["dx"] = np.empty((T, n), dtype=np.float64)
+    if "dL" in want:
+        out["dL"] = np.empty((m, m, m), dtype=np.float64)
+    if "dR" in want:
+        out["dR"] = np.empty((m, m, m), dtype=np.float64)
+    if _load().oracle_bwd(_p(x), _p(dy), _p(L), _p(R), _p(out.get("dx")),
+                          _p(out.get("dL")), _p(out.get("dR")), T, m):
+        raise MemoryError("oracle_bwd")
+    return out
+
+
+def mlp_fwd(x, L1, R1, b1, L2, R2, b2):
+    """y = M2 GELU(M1 x + b1) + b2 with the erf form of GELU."""
+    L1 = _f64(L1); R1 = _f64(R1); L2 = _f64(L2); R2 = _f64(R2)
+    m = _m_of(L1); n = m * m
+    b1 = _f64(b1, (n,)); b2 = _f64(b2, (n,))
+    x = _f64(x); T = x.shape[0]
+    y = np.empty((T, n), dtype=np.float64)
+    if _load().oracle_mlp_fwd(_p(x), _p(L1), _p(R1), _p(b1), _p(L2), _p(R2), _p(b2),
+                              _p(y), T, m):
+        raise MemoryError("oracle_mlp_fwd")
+    return y
+
+
+# --------------------------------------------------------------------------
+# numpy restatements of the definitions (tiny n only)
+# --------------------------------------------------------------------------
+
+def perm_matrix(m: int) -> np.ndarray:
+    """The permutation P of Definition 3.1 as an n x n 0/1 matrix.
+
+    P maps [x_1..x_n] to [x_1, x_{1+m}, ..., x_{1+(m-1)m}, x_2, ...]: output
+    position a*m+b holds input element b*m+a (0-indexed) - reshape to m x m,
+    transpose, flatten.
+    """
+    n = m * m
+    P = np.zeros((n, n), dtype=np.float64)
+    for a in range(m):
+        for b in range(m):
+            P[a * m + b, b * m + a] = 1.0
+    return P
+
+
+def blockdiag(W) -> np.ndarray:
+    """diag(W_0, ..., W_{m-1}) as a dense n x n matrix."""
+    W = np.asarray(W, dtype=np.float64)
+    m = W.shape[0]
+    n = m * m
+    B = np.zeros((n, n), dtype=np.float64)
+    for b in range(m):
+        B[b * m:(b + 1) * m, b * m:(b + 1) * m] = W[b]
+    return B
+
+
+def dense_from_definition(L, R) -> np.ndarray:
+    """M = P L P^T R with every factor materialised (Definition 3.1)."""
+    m = np.asarray(L).shape[0]
+    P = perm_matrix(m)
+    return P @ blockdiag(L) @ P.T @ blockdiag(R)
+
+
+def project(A, m: int):
+    """Algorithm 1: closest Monarch matrix to a dense A in Frobenius norm.
+
+    A is viewed as A~[l, j, k, i] = A[l*m+j, k*m+i]; every slice
+    A~[:, j, k, :] (an m x m matrix indexed l, i) is replaced by its best
+    rank-1 approximation u v^T, with L[j, :, k] = u and R[k, j, :] = v.
+    The paper fixes only the product u v^T; here both carry sqrt(sigma_1).
+    """
+    A = np.asarray(A, dtype=np.float64)
+    n = m * m
+    if A.shape != (n, n):
+        raise ValueError("A must be n x n with n = m*m")
+    A4 = A.reshape(m, m, m, m)            # [l, j, k, i]
+    L = np.zeros((m, m, m), dtype=np.float64)
+    R = np.zeros((m, m, m), dtype=np.float64)
+    for j in range(m):
+        for k in range(m):
+            S = A4[:, j, k, :]
+            U, s, Vt = np.linalg.svd(S)
+            L[j, :, k] = U[:, 0] * np.sqrt(s[0])
+            R[k, j, :] = Vt[0, :] * np.sqrt(s[0])
+    return L, R
+
+
+if __name__ == "__main__":
+    build(force=True)
+    print("built", _LIB, "threads", num_threads(), file=sys.stderr)

@@ -1,0 +1,104 @@
+"""Seeded synthetic inputs for the Monarch multiply, shared by tests and bench.
+
+This module holds no arithmetic of the method: it only draws Gaussian tensors
+of the benchmark shapes and rounds them to the storage dtype, so that the CUDA
+library and the CPU oracle see bit-identical values.
+
+Recipe: ``numpy.random.default_rng(595000 + config)``; tensors are drawn in the
+fixed order x, L, R, dy, L2, R2, b1, b2 as float32 ``standard_normal * std``
+(only those the config uses), then rounded to nearest-even to the storage
+dtype.  ``N(0, v)`` in the workload descriptions is read as variance v.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass
+
+import numpy as np
+
+
+@dataclass(frozen=True)
+class Config:
+    index: int          # 1-based, as the workloads are numbered
+    name: str
+    dtype: str          # "f32" or "bf16" storage / operand type
+    m: int
+    tokens: int
+    ops: tuple          # subset of ("fwd", "bwd_dx", "bwd_dw", "mlp_fwd")
+    std_x: float
+    std_w: float
+    std_b: float = 0.0
+
+    @property
+    def n(self) -> int:
+        return self.m * self.m
+
+
+CONFIGS = {
+    1: Config(1, "fwd f32 n=256 m=16 T=64", "f32", 16, 64, ("fwd",), 0.25, 0.25),
+    2: Config(2, "fwd bf16 n=1024 m=32 T=16384", "bf16", 32, 16384, ("fwd",),
+              1.0, 1.0 / math.sqrt(32)),
+    3: Config(3, "fwd+bwd bf16 n=4096 m=64 T=8192", "bf16", 64, 8192,
+              ("fwd", "bwd_dx", "bwd_dw"), 1.0, 1.0 / 8.0),
+    4: Config(4, "fwd+bwd bf16 n=16384 m=128 T=4096", "bf16", 128, 4096,
+              ("fwd", "bwd_dx", "bwd_dw"), 1.0, 1.0 / math.sqrt(128)),
+    5: Config(5, "mlp fwd bf16 n=4096 m=64 T=32768", "bf16", 64, 32768,
+              ("mlp_fwd",), 1.0, 1.0 / 8.0, math.sqrt(0.02)),
+}
+
+
+def f32_to_bf16_bits(a: np.ndarray) -> np.ndarray:
+    """Round float32 to bfloat16 (nearest even); returns uint16 bit patterns."""
+    u = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+    rounded = (u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) >> np.uint32(16)
+    return rounded.astype(np.uint16)
+
+
+def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
+    """Exact promotion of bfloat16 bit patterns to float32."""
+    return (np.ascontiguousarray(b, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+def round_to_storage(a: np.ndarray, dtype: str) -> np.ndarray:
+    """float32 array whose values are exactly representable in ``dtype``."""
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    if dtype == "f32":
+        return a
+    if dtype == "bf16":
+        return bf16_bits_to_f32(f32_to_bf16_bits(a)).reshape(a.shape)
+    raise ValueError(dtype)
+
+
+def make_inputs(config: int, tokens: int | None = None, m: int | None = None,
+                dtype: str | None = None, seed: int | None = None) -> dict:
+    """Draw the tensors of workload ``config`` (1..5).
+
+    ``tokens``, ``m`` and ``dtype`` override the workload's values (for small
+    parity cases of the same distribution).  Returns float32 arrays already
+    rounded to the storage dtype, plus the scalars ``m``, ``n``, ``tokens``,
+    ``dtype``.
+    """
+    c = CONFIGS[config]
+    T = c.tokens if tokens is None else int(tokens)
+    mm = c.m if m is None else int(m)
+    dt = c.dtype if dtype is None else dtype
+    std_w = c.std_w if m is None else 1.0 / math.sqrt(mm)
+    n = mm * mm
+    rng = np.random.default_rng(595000 + config if seed is None else seed)
+
+    def draw(shape, std):
+        a = rng.standard_normal(shape, dtype=np.float32) * np.float32(std)
+        return round_to_storage(a, dt)
+
+    out = {"m": mm, "n": n, "tokens": T, "dtype": dt, "config": config}
+    out["x"] = draw((T, n), c.std_x)
+    out["L"] = draw((mm, mm, mm), std_w)
+    out["R"] = draw((mm, mm, mm), std_w)
+    if "bwd_dx" in c.ops or "bwd_dw" in c.ops:
+        out["dy"] = draw((T, n), 1.0)
+    if "mlp_fwd" in c.ops:
+        out["L2"] = draw((mm, mm, mm), std_w)
+        out["R2"] = draw((mm, mm, mm), std_w)
+        out["b1"] = draw((n,), c.std_b)
+        out["b2"] = draw((n,), c.std_b)
+    return out

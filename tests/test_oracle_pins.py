@@ -1,0 +1,328 @@
+"""Pins for the CPU oracle: every check compares the C loops against something
+other than themselves - Definition 3.1 materialised literally, closed forms,
+finite differences, textbook values, and the projection invariant."""
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import monarch_oracle as O
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rand(rng, *shape):
+    return rng.standard_normal(shape)
+
+
+def _read_table(name):
+    rows = []
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                rows.append([float(v) for v in line.split()])
+    return np.array(rows)
+
+
+# ------------------------------------------------------------------ permutation
+
+def test_perm_matches_definition_listing():
+    # Definition 3.1 lists the order of the permuted vector.
+    listed = _read_table("perm_m3.txt")[0].astype(int) - 1
+    P = O.perm_matrix(3)
+    x = np.arange(9, dtype=np.float64)
+    assert np.array_equal(P @ x, x[listed])
+
+
+@pytest.mark.parametrize("m", [2, 3, 4, 8])
+def test_perm_is_symmetric_involution(m):
+    # Section 3.1: "Note that P = P^T"; hence P P = I.
+    P = O.perm_matrix(m)
+    assert np.array_equal(P, P.T)
+    assert np.array_equal(P @ P, np.eye(m * m))
+    x = np.arange(m * m, dtype=np.float64)
+    assert np.array_equal(P @ x, x.reshape(m, m).T.reshape(-1))
+
+
+@pytest.mark.parametrize("m", [2, 3, 4])
+def test_PtLP_is_grid_of_diagonal_blocks(m):
+    # Section 3.1: L' = P^T L P consists of m x m blocks, each diagonal.
+    rng = np.random.default_rng(1)
+    L = _rand(rng, m, m, m)
+    P = O.perm_matrix(m)
+    Lp = P.T @ O.blockdiag(L) @ P
+    for a in range(m):
+        for b in range(m):
+            D = Lp[a * m:(a + 1) * m, b * m:(b + 1) * m]
+            assert np.array_equal(D, np.diag(np.diag(D)))
+            assert np.allclose(np.diag(D), L[:, a, b], rtol=0, atol=0)
+
+
+# ------------------------------------------------------------------ forward
+
+@pytest.mark.parametrize("m", [2, 3, 4, 8])
+def test_three_routes_agree(m):
+    # Definition 3.1 (explicit P, blockdiag), Eq. (2), and steps 1-3.
+    rng = np.random.default_rng(10 + m)
+    n = m * m
+    L, R = _rand(rng, m, m, m), _rand(rng, m, m, m)
+    x = _rand(rng, 5, n)
+    M_def = O.dense_from_definition(L, R)
+    M_eq2 = O.dense(L, R)
+    assert np.allclose(M_def, M_eq2, rtol=1e-13, atol=1e-13)
+    y = O.fwd(x, L, R)
+    assert np.allclose(y, x @ M_def.T, rtol=1e-12, atol=1e-12)
+
+
+def test_eq2_entry_formula_explicit():
+    # M[(l)m+j, (k)m+i] = L[j,l,k] R[k,j,i], spelled with numpy's einsum as a
+    # second statement of Eq. (2).
+    rng = np.random.default_rng(3)
+    m = 4
+    L, R = _rand(rng, m, m, m), _rand(rng, m, m, m)
+    M4 = np.einsum("jlk,kji->ljki", L, R)
+    assert np.allclose(O.dense(L, R), M4.reshape(m * m, m * m), rtol=0, atol=1e-15)
+    assert np.allclose(O.dense_from_definition(L, R), M4.reshape(m * m, m * m), atol=1e-13)
+
+
+@pytest.mark.parametrize("m", [3, 4])
+def test_stage_isolation(m):
+    rng = np.random.default_rng(4)
+    n = m * m
+    W = _rand(rng, m, m, m)
+    I = np.stack([np.eye(m)] * m)
+    x = _rand(rng, 3, n)
+    # L = I: M = P P^T R = blockdiag(R)
+    y = O.fwd(x, I, W)
+    assert np.allclose(y, x @ O.blockdiag(W).T, atol=1e-13)
+    # R = I: M = P L P^T, entries delta_{ji} L[j,l,k]
+    y = O.fwd(x, W, I)
+    P = O.perm_matrix(m)
+    assert np.allclose(y, x @ (P @ O.blockdiag(W) @ P.T).T, atol=1e-13)
+    u_expected = x.reshape(3, m, m)                           # u = x when R = I
+    _, u = O.fwd(x, W, I, return_u=True)
+    assert np.array_equal(u, u_expected)
+
+
+@pytest.mark.parametrize("m", [2, 3, 5])
+def test_kronecker_closed_form(m):
+    # Identical blocks: L_j = A, R_k = B  =>  M = A (x) B  (from Eq. (2)).
+    rng = np.random.default_rng(5)
+    A, B = _rand(rng, m, m), _rand(rng, m, m)
+    L = np.stack([A] * m)
+    R = np.stack([B] * m)
+    x = _rand(rng, 4, m * m)
+    assert np.allclose(O.dense(L, R), np.kron(A, B), atol=1e-14)
+    assert np.allclose(O.fwd(x, L, R), x @ np.kron(A, B).T, atol=1e-12)
+
+
+def _sylvester(m):
+    H = np.array([[1.0]])
+    while H.shape[0] < m:
+        H = np.block([[H, H], [H, -H]])
+    return H
+
+
+def test_hadamard_h4_golden():
+    H4 = _read_table("hadamard_h4.txt")
+    H2 = _sylvester(2)
+    L = np.stack([H2] * 2)
+    R = np.stack([H2] * 2)
+    assert np.array_equal(O.dense(L, R), H4)
+    assert np.array_equal(O.dense_from_definition(L, R), H4)
+
+
+@pytest.mark.parametrize("m", [2, 4, 8, 16])
+def test_hadamard_transform_exact(m):
+    # All blocks H_m  =>  M = H_n in natural (Sylvester) order:
+    # y[a] = sum_b (-1)^{popcount(a & b)} x[b].  Small integers: exact.
+    n = m * m
+    rng = np.random.default_rng(6)
+    x = rng.integers(-3, 4, size=(3, n)).astype(np.float64)
+    Hm = _sylvester(m)
+    y = O.fwd(x, np.stack([Hm] * m), np.stack([Hm] * m))
+    a = np.arange(n)
+    sign = np.array([[(-1) ** bin(p & q).count("1") for q in a] for p in a], dtype=np.float64)
+    assert np.array_equal(y, x @ sign.T)
+
+
+def test_forward_edge_token_counts():
+    rng = np.random.default_rng(7)
+    m = 4
+    L, R = _rand(rng, m, m, m), _rand(rng, m, m, m)
+    M = O.dense_from_definition(L, R)
+    for T in (0, 1, 7):
+        x = _rand(rng, T, m * m)
+        y = O.fwd(x, L, R)
+        assert y.shape == (T, m * m)
+        assert np.allclose(y, x @ M.T, atol=1e-12)
+
+
+def test_parameter_count():
+    # Section 3.2.2: a Monarch matrix has 2 n sqrt(n) parameters.
+    m = 8
+    n = m * m
+    assert 2 * m * m * m == 2 * n * int(math.isqrt(n))
+
+
+# ------------------------------------------------------------------ backward
+
+def _loss(x, dy, L, R):
+    return float(np.sum(dy * (x @ O.dense_from_definition(L, R).T)))
+
+
+def test_gradients_by_finite_differences():
+    rng = np.random.default_rng(8)
+    m, T = 3, 4
+    n = m * m
+    x, dy = _rand(rng, T, n), _rand(rng, T, n)
+    L, R = _rand(rng, m, m, m), _rand(rng, m, m, m)
+    g = O.bwd(x, dy, L, R)
+    h = 1e-6
+
+    def fd(arr, which):
+        out = np.zeros_like(arr)
+        it = np.nditer(arr, flags=["multi_index"])
+        for _ in it:
+            idx = it.multi_index
+            ap, am = arr.copy(), arr.copy()
+            ap[idx] += h
+            am[idx] -= h
+            args_p = {"x": x, "L": L, "R": R}
+            args_m = dict(args_p)
+            args_p[which] = ap
+            args_m[which] = am
+            out[idx] = (_loss(args_p["x"], dy, args_p["L"], args_p["R"])
+                        - _loss(args_m["x"], dy, args_m["L"], args_m["R"])) / (2 * h)
+        return out
+
+    assert np.allclose(g["dx"], fd(x, "x"), rtol=1e-7, atol=1e-7)
+    assert np.allclose(g["dL"], fd(L, "L"), rtol=1e-7, atol=1e-7)
+    assert np.allclose(g["dR"], fd(R, "R"), rtol=1e-7, atol=1e-7)
+
+
+@pytest.mark.parametrize("m", [2, 4, 8])
+def test_gradients_via_dense_chain_rule(m):
+    # dx = M^T dy;  dM = sum_t dy_t x_t^T;  by Eq. (2)
+    # dL[j,l,k] = sum_i dM[l m+j, k m+i] R[k,j,i],  dR[k,j,i] = sum_l dM[..] L[j,l,k].
+    rng = np.random.default_rng(9)
+    n = m * m
+    T = 6
+    x, dy = _rand(rng, T, n), _rand(rng, T, n)
+    L, R = _rand(rng, m, m, m), _rand(rng, m, m, m)
+    g = O.bwd(x, dy, L, R)
+    M = O.dense_from_definition(L, R)
+    assert np.allclose(g["dx"], dy @ M, atol=1e-11)
+    dM4 = (dy.T @ x).reshape(m, m, m, m)                     # [l, j, k, i]
+    assert np.allclose(g["dL"], np.einsum("ljki,kji->jlk", dM4, R), atol=1e-11)
+    assert np.allclose(g["dR"], np.einsum("ljki,jlk->kji", dM4, L), atol=1e-11)
+
+
+def test_adjoint_and_euler_identities():
+    rng = np.random.default_rng(11)
+    m, T = 8, 9
+    n = m * m
+    x, dy = _rand(rng, T, n), _rand(rng, T, n)
+    L, R = _rand(rng, m, m, m), _rand(rng, m, m, m)
+    y = O.fwd(x, L, R)
+    g = O.bwd(x, dy, L, R)
+    s = np.sum(dy * y)
+    assert np.isclose(np.sum(g["dx"] * x), s, rtol=1e-12)     # <M^T dy, x> = <dy, Mx>
+    assert np.isclose(np.sum(g["dL"] * L), s, rtol=1e-12)     # y is linear in L
+    assert np.isclose(np.sum(g["dR"] * R), s, rtol=1e-12)     # and in R
+
+
+def test_bwd_partial_outputs_and_empty():
+    rng = np.random.default_rng(12)
+    m = 4
+    n = m * m
+    x, dy = _rand(rng, 5, n), _rand(rng, 5, n)
+    L, R = _rand(rng, m, m, m), _rand(rng, m, m, m)
+    full = O.bwd(x, dy, L, R)
+    only = O.bwd(x, dy, L, R, want=("dR",))
+    assert set(only) == {"dR"} and np.array_equal(only["dR"], full["dR"])
+    z = O.bwd(x[:0], dy[:0], L, R)
+    assert z["dx"].shape == (0, n) and not z["dL"].any() and not z["dR"].any()
+
+
+# ------------------------------------------------------------------ projection
+
+@pytest.mark.parametrize("m", [2, 3, 4, 6])
+def test_projection_recovers_monarch(m):
+    # Section 3.3: if A is Monarch, Algorithm 1 recovers factors with A = P L P^T R.
+    rng = np.random.default_rng(13)
+    L, R = _rand(rng, m, m, m), _rand(rng, m, m, m)
+    A = O.dense(L, R)
+    L2, R2 = O.project(A, m)
+    assert np.allclose(O.dense(L2, R2), A, atol=1e-12)
+    assert np.allclose(O.dense_from_definition(L2, R2), A, atol=1e-12)
+    for j in range(m):
+        for k in range(m):
+            s = np.linalg.svd(A.reshape(m, m, m, m)[:, j, k, :], compute_uv=False)
+            assert s[1] <= 1e-12 * max(s[0], 1.0)
+
+
+@pytest.mark.parametrize("m", [3, 4])
+def test_projection_residual_is_discarded_spectrum(m):
+    # Proof of Theorem 1: the objective splits over the m*m slices, each solved
+    # by its best rank-1 approximation (Eckart-Young).
+    rng = np.random.default_rng(14)
+    n = m * m
+    A = _rand(rng, n, n)
+    L, R = O.project(A, m)
+    res = np.sum((A - O.dense(L, R)) ** 2)
+    A4 = A.reshape(m, m, m, m)
+    tail = 0.0
+    for j in range(m):
+        for k in range(m):
+            s = np.linalg.svd(A4[:, j, k, :], compute_uv=False)
+            tail += np.sum(s[1:] ** 2)
+    assert np.isclose(res, tail, rtol=1e-10)
+    for _ in range(20):                                       # local optimality
+        Lp = L + 1e-3 * _rand(rng, m, m, m)
+        Rp = R + 1e-3 * _rand(rng, m, m, m)
+        assert np.sum((A - O.dense(Lp, Rp)) ** 2) >= res - 1e-12
+
+
+# ------------------------------------------------------------------ MLP block
+
+def _gelu(a):
+    return np.array([0.5 * v * (1.0 + math.erf(v / math.sqrt(2.0))) for v in a.ravel()]).reshape(a.shape)
+
+
+def test_gelu_textbook_values():
+    tab = _read_table("gelu_values.txt")
+    m = 2
+    n = 4
+    I = np.stack([np.eye(m)] * m)
+    for a, g in tab:
+        x = np.full((1, n), a)
+        h = O.mlp_fwd(x, I, I, np.zeros(n), I, I, np.zeros(n))
+        assert np.allclose(h, g, rtol=1e-14, atol=1e-16)
+
+
+def test_mlp_special_cases():
+    rng = np.random.default_rng(15)
+    m, T = 4, 5
+    n = m * m
+    x = _rand(rng, T, n)
+    b1, b2 = _rand(rng, n), _rand(rng, n)
+    I = np.stack([np.eye(m)] * m)
+    Z = np.zeros((m, m, m))
+    W = [_rand(rng, m, m, m) for _ in range(4)]
+    # second matrix zero: y = b2
+    assert np.allclose(O.mlp_fwd(x, W[0], W[1], b1, Z, W[3], b2), np.broadcast_to(b2, (T, n)))
+    # identities: y = GELU(x + b1) + b2
+    assert np.allclose(O.mlp_fwd(x, I, I, b1, I, I, b2), _gelu(x + b1) + b2, atol=1e-14)
+    # general: composition through the dense matrices of Definition 3.1
+    M1 = O.dense_from_definition(W[0], W[1])
+    M2 = O.dense_from_definition(W[2], W[3])
+    ref = _gelu(x @ M1.T + b1) @ M2.T + b2
+    assert np.allclose(O.mlp_fwd(x, W[0], W[1], b1, W[2], W[3], b2), ref, atol=1e-11)
+    # odd part of GELU: GELU(a) - GELU(-a) = a
+    a = _rand(rng, 1, n)
+    gp = O.mlp_fwd(a, I, I, np.zeros(n), I, I, np.zeros(n))
+    gm = O.mlp_fwd(-a, I, I, np.zeros(n), I, I, np.zeros(n))
+    assert np.allclose(gp - gm, a, atol=1e-14)
