@@ -1,0 +1,353 @@
+#!/usr/bin/env python
+"""Benchmark of the Monarch multiply hot path on B200.
+
+One step = one pass of the hot path over one batch of synthetic tokens of the chosen
+workload (default: workload 3, n=4096, m=64, 8192 tokens per GPU, bf16):
+    monarch_fwd (y) + monarch_bwd_dx (dx) + monarch_bwd_dw (dL, dR).
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+
+Launch for N > 1:  python -m torch.distributed.run --nnodes=1 --nproc-per-node N
+    --master-addr 127.0.0.1 --master-port P bench.py --gpus N --steps K --warmup W
+Tokens are sharded over ranks (fixed tokens per GPU: weak scaling); the only exchange is
+one all-reduce of the packed (dL, dR) gradients per step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=3, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--kernels", default="auto", choices=["auto", "staged", "fused"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+# ----------------------------------------------------------------------------- accounting
+
+def esize(dtype):
+    return 4 if dtype == "f32" else 2
+
+
+def call_flops(call, n, m, T):
+    """Algorithmic FLOPs: 4 n m per token per pass (two block-diagonal stages of 2 n m each)."""
+    return {"fwd": 4, "bwd_dx": 4, "bwd_dw": 4, "mlp_fwd": 8}[call] * n * m * T
+
+
+def call_bytes(call, n, m, T, dtype):
+    """Algorithmic bytes: the token tensors read and written once, plus the weights once."""
+    s = esize(dtype)
+    w = 2 * n * m * s
+    if call in ("fwd", "bwd_dx"):
+        return 2 * T * n * s + w
+    if call == "bwd_dw":
+        return 2 * T * n * s + w + 2 * n * m * 4
+    if call == "mlp_fwd":
+        return 2 * T * n * s + 2 * w + 2 * n * s
+    raise ValueError(call)
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "source": "measured"}
+    except Exception:
+        return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": FALLBACK_BF16_TFLOPS,
+                "source": "fallback"}
+
+
+# ----------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+            "hw_power_brake": getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(0.02)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        return {
+            "sm_mhz": statistics.median(self.samples) if self.samples else None,
+            "sm_max_mhz": self.max_mhz,
+            "reasons": sorted(self.reasons),
+            "samples": len(self.samples),
+        }
+
+
+# ----------------------------------------------------------------------------- CPU oracle timing
+
+def time_oracle(cfg, d, target_s=12.0):
+    """Time the oracle (as it stands) on a bounded token sample of the workload."""
+    from oracle import monarch_oracle as O
+    c = cfg
+    calls = list(c.ops)
+
+    def run(T):
+        t0 = time.perf_counter()
+        if "fwd" in calls:
+            O.fwd(d["x"][:T], d["L"], d["R"])
+        if "bwd_dx" in calls or "bwd_dw" in calls:
+            want = tuple(k for k, op in (("dx", "bwd_dx"), ("dL", "bwd_dw"), ("dR", "bwd_dw"))
+                         if op in calls)
+            O.bwd(d["x"][:T], d["dy"][:T], d["L"], d["R"], want=want)
+        if "mlp_fwd" in calls:
+            O.mlp_fwd(d["x"][:T], d["L"], d["R"], d["b1"], d["L2"], d["R2"], d["b2"])
+        return time.perf_counter() - t0
+
+    T = min(32, c.tokens)
+    dt = run(T)
+    while dt < 0.5 and T < c.tokens:
+        T = min(T * 4, c.tokens)
+        dt = run(T)
+    Ts = int(min(c.tokens, max(T, T * target_s / max(dt, 1e-9))))
+    if Ts != T:
+        dt = run(Ts)
+        T = Ts
+    flops = sum(call_flops(k, c.n, c.m, T) for k in calls)
+    return {"tflops": flops / dt / 1e12, "tokens": T, "seconds": dt, "cores": O.num_threads(),
+            "tokens_per_s": T / dt}
+
+
+# ----------------------------------------------------------------------------- main
+
+def main():
+    args = parse_args()
+    from paper_2204_00595_b200.inputs import CONFIGS, make_inputs
+    cfg = CONFIGS[args.workload]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    calls = list(cfg.ops)
+    n, m, T = cfg.n, cfg.m, cfg.tokens
+    workload = (f"workload {cfg.index}: {'+'.join(calls)} {cfg.dtype} n={n} m={m} "
+                f"tokens/GPU={T}")
+    metric, unit = "monarch_fwd_bwd_tflops", "TFLOP/s"
+    step_flops = sum(call_flops(k, n, m, T) for k in calls)
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        import __graft_entry__ as entry
+        from oracle import monarch_oracle as O
+        O.build()
+        d = make_inputs(cfg.index)
+        times, sample = [], None
+        for i in range(args.warmup + args.steps):
+            r = time_oracle(cfg, d, target_s=max(1.0, min(8.0, 120.0 / (args.warmup + args.steps))))
+            sample = r
+            if i >= args.warmup:
+                times.append(r)
+        tfl = statistics.mean(r["tflops"] for r in times)
+        tps = statistics.mean(r["tokens_per_s"] for r in times)
+        ms = statistics.mean(r["seconds"] for r in times) * 1e3
+        line = {
+            "impl": "reference", "metric": metric, "value": tfl, "unit": unit, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "tokens_per_s": tps,
+            "config": {"workload": workload, "sample_tokens_per_step": sample["tokens"]},
+            "cpu_baseline": {"value": tfl, "unit": unit, "cores": sample["cores"], "kind": "oracle",
+                             "sample": f"{sample['tokens']} tokens of the workload per step"},
+            "e2e": {"value": tfl, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        }
+        print(json.dumps(line))
+        return 0
+
+    import torch
+    import __graft_entry__ as entry
+    entry.build()
+    import paper_2204_00595_b200 as P
+
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    P.monarch_set_impl({"auto": P.IMPL_AUTO, "staged": P.IMPL_STAGED, "fused": P.IMPL_FUSED}[args.kernels])
+
+    code = P.F32 if cfg.dtype == "f32" else P.BF16
+    tdt = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
+    d = make_inputs(cfg.index)              # every rank draws the same recipe, then offsets it
+    from tests.helpers import to_device
+
+    # Two rotating sets of token tensors so that no launch finds its operands in L2 from the
+    # previous step (each set alone already exceeds the 126 MB L2 for workloads 3-5).
+    SETS = 2 if T * n * esize(cfg.dtype) * 4 < (1 << 30) else 1
+    sets = []
+    for s in range(SETS):
+        x = to_device(d["x"], cfg.dtype)
+        if s or rank:
+            x = torch.roll(x, shifts=17 * s + 5 * rank, dims=0).contiguous()
+        e = {"x": x, "y": torch.empty_like(x)}
+        if "dy" in d:
+            e["dy"] = torch.roll(to_device(d["dy"], cfg.dtype), shifts=3 * s + rank, dims=0).contiguous()
+            e["dx"] = torch.empty_like(x)
+        sets.append(e)
+    W = {k: to_device(d[k], cfg.dtype) for k in ("L", "R", "L2", "R2", "b1", "b2") if k in d}
+    grads = torch.zeros(2, m, m, m, dtype=torch.float32, device="cuda")   # packed (dL, dR)
+    op_of = {"fwd": P.OP_FWD, "bwd_dx": P.OP_BWD_DX, "bwd_dw": P.OP_BWD_DW, "mlp_fwd": P.OP_MLP_FWD}
+    ws = P.Workspace(max(P.monarch_workspace_bytes(op_of[k], T, n, m, code) for k in calls))
+    stream = torch.cuda.current_stream()
+
+    ev = {k: [] for k in calls}
+
+    def step(i, timed):
+        e = sets[i % SETS]
+        for k in calls:
+            if timed:
+                a = torch.cuda.Event(enable_timing=True)
+                b = torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+            if k == "fwd":
+                P.monarch_fwd(e["x"], W["L"], W["R"], e["y"], T, n, m, ws)
+            elif k == "bwd_dx":
+                P.monarch_bwd_dx(e["dy"], W["L"], W["R"], e["dx"], T, n, m, ws)
+            elif k == "bwd_dw":
+                P.monarch_bwd_dw(e["x"], e["dy"], W["L"], W["R"], grads[0], grads[1], 0, T, n, m, ws)
+                if dist is not None:
+                    dist.all_reduce(grads)
+            elif k == "mlp_fwd":
+                P.monarch_mlp_fwd(e["x"], W["L"], W["R"], W["b1"], W["L2"], W["R2"], W["b2"],
+                                  e["y"], T, n, m, ws)
+            if timed:
+                b.record(stream)
+                ev[k].append((a, b))
+
+    for i in range(args.warmup):
+        step(i, False)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = P.monarch_launch_count()
+    torch.cuda.synchronize()
+    t_start = torch.cuda.Event(enable_timing=True)
+    t_stop = torch.cuda.Event(enable_timing=True)
+    t_start.record(stream)
+    for i in range(args.steps):
+        step(args.warmup + i, True)
+    t_stop.record(stream)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    total_ms = t_start.elapsed_time(t_stop)
+    clocks = sampler.stop()
+    launches = P.monarch_launch_count() - launches0
+    status = P.monarch_last_device_status(ws)
+    if dist is not None:
+        tmax = torch.tensor([total_ms], device="cuda")
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        total_ms = float(tmax.item())
+    ms_per_step = total_ms / args.steps
+    value = step_flops * world / (ms_per_step * 1e-3) / 1e12
+    tokens_per_s = T * world / (ms_per_step * 1e-3)
+
+    peaks = load_peaks()
+    per_call = {}
+    for k in calls:
+        ts = [a.elapsed_time(b) for a, b in ev[k]]
+        ms = statistics.mean(ts)
+        by = call_bytes(k, n, m, T, cfg.dtype)
+        fl = call_flops(k, n, m, T)
+        roof_ms = max(by / (peaks["hbm_gbs"] * 1e9), fl / (peaks["bf16_tflops"] * 1e12)) * 1e3
+        per_call[k] = {"ms": ms, "ms_min": min(ts), "gbs": by / ms / 1e6, "tflops": fl / ms / 1e9,
+                       "roofline_ms": roof_ms, "roofline_frac": roof_ms / ms,
+                       "impl": P.monarch_impl_name(op_of[k], m, code)}
+    dom = max(calls, key=lambda k: per_call[k]["ms"])
+    roofline = {
+        "bound": "hbm", "kernel": f"{dom} ({per_call[dom]['impl']})",
+        "achieved": per_call[dom]["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+        "frac": per_call[dom]["gbs"] / peaks["hbm_gbs"], "peak_source": peaks["source"],
+        "traffic": None,
+    }
+
+    line = {
+        "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+        "tokens_per_s": tokens_per_s,
+        "config": {"workload": workload, "l2": f"inputs larger than L2; {SETS} rotating buffer sets",
+                   "kernels": args.kernels, "device_status": status},
+        "clocks": clocks, "gpu_launches": int(launches), "roofline": roofline, "calls": per_call,
+    }
+
+    if rank == 0 and not args.no_e2e:
+        line["e2e"] = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        r = time_oracle(cfg, d)
+        line["cpu_baseline"] = {"value": r["tflops"], "unit": unit, "cores": r["cores"],
+                                "kind": "oracle", "tokens_per_s": r["tokens_per_s"],
+                                "sample": f"first {r['tokens']} tokens of the workload, "
+                                          f"{r['seconds']:.1f} s"}
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,135 @@
+/*
+ * libmonarch - the Monarch matrix multiply on NVIDIA B200 (sm_100a), C ABI.
+ *
+ * A Monarch matrix (Dao et al., arXiv 2204.00595, Definition 3.1) of size
+ * n x n, n = m*m, is  M = P L P^T R  with L and R block-diagonal (m blocks of
+ * m x m each) and P the reshape(m,m)-transpose "stride" permutation.  The
+ * calls below multiply a batch of token vectors by M, by M^T, form the
+ * gradients of the blocks, and evaluate a Monarch feed-forward block.
+ *
+ * Conventions shared by every call
+ * --------------------------------
+ *  - All data pointers are DEVICE pointers owned by the caller, 16-byte
+ *    aligned, dense and row-major.  Nothing is allocated, freed or retained
+ *    by the library; outputs must not overlap inputs or the workspace.
+ *  - x, y, dy, dx : [tokens][n]   (token-major; element k*m+i of a row is
+ *    entry (k,i) of the m x m view of the vector used in Section 3.3).
+ *  - L, R : [m][m][m] = [block][output row][input column]; i.e. R[k][j][i] and
+ *    L[j][l][k] in the notation of Section 3.3 steps 1-2 and Algorithm 1.
+ *  - b1, b2 : [n].
+ *  - dtype MONARCH_F32 : every tensor is IEEE float32, fp32 arithmetic.
+ *    dtype MONARCH_BF16: x, y, dy, dx, L, R, b1, b2 are bfloat16; products
+ *    accumulate in fp32; on-chip intermediates (u, du, h) are rounded to
+ *    bfloat16 once because they are tensor-core operands; dL, dR are float32.
+ *  - n must equal m*m and m must be one of 16, 32, 64, 128; otherwise
+ *    MONARCH_ERR_UNSUPPORTED.  tokens >= 0 (0 is a no-op that still defines
+ *    dL/dR when accumulate == 0).
+ *  - `stream` is a cudaStream_t passed as void*.  Calls enqueue work on it
+ *    and return without synchronising.  Argument errors are reported by the
+ *    return value before anything is enqueued.
+ *  - `workspace` is caller-owned device scratch of at least
+ *    monarch_workspace_bytes(op, ...) bytes, 256-byte aligned.  Its first
+ *    MONARCH_STATUS_BYTES bytes hold a device status word that kernels set
+ *    when one of their bounded waits runs out; zero it once with
+ *    monarch_workspace_init and read it with monarch_last_device_status.
+ *    Calls that overlap on the GPU must not share a workspace.
+ *  - Return value: a monarch_status_t.  Nothing throws.
+ */
+#ifndef MONARCH_H_
+#define MONARCH_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { MONARCH_F32 = 0, MONARCH_BF16 = 1 } monarch_dtype_t;
+
+typedef enum {
+    MONARCH_OK = 0,
+    MONARCH_ERR_INVALID_ARG = 1, /* null / misaligned / overlapping pointer, n != m*m, bad enum */
+    MONARCH_ERR_UNSUPPORTED = 2, /* m or dtype not built for this call */
+    MONARCH_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or too small */
+    MONARCH_ERR_CUDA = 4,        /* a CUDA runtime/driver call or a launch failed */
+    MONARCH_ERR_TIMEOUT = 5      /* a kernel gave up on one of its bounded waits */
+} monarch_status_t;
+
+typedef enum {
+    MONARCH_OP_FWD = 0,
+    MONARCH_OP_BWD_DX = 1,
+    MONARCH_OP_BWD_DW = 2,
+    MONARCH_OP_MLP_FWD = 3
+} monarch_op_t;
+
+/* Which kernel family serves a call (process-wide; default AUTO). */
+typedef enum {
+    MONARCH_IMPL_AUTO = 0,   /* fused tensor-core kernels where built, else staged */
+    MONARCH_IMPL_STAGED = 1, /* one block-diagonal stage per launch, CUDA-core FMA, any m */
+    MONARCH_IMPL_FUSED = 2   /* fused tcgen05 kernels only; UNSUPPORTED where none exists */
+} monarch_impl_t;
+
+#define MONARCH_STATUS_BYTES 256
+
+/* y = M x = P L P^T R x  (Definition 3.1; computed as Section 3.3 steps 1-3:
+ * u[k][j] = sum_i R[k][j][i] x[k*m+i];  y[l*m+j] = sum_k L[j][l][k] u[k][j]). */
+int monarch_fwd(const void *x, const void *L, const void *R, void *y,
+                int64_t tokens, int32_t n, int32_t m, int dtype,
+                void *workspace, size_t workspace_bytes, void *stream);
+
+/* dx = M^T dy = R^T P L^T P dy, the adjoint of steps 1-3 (the paper trains by
+ * automatic differentiation, Section 4):
+ * du[k][j] = sum_l L[j][l][k] dy[l*m+j];  dx[k*m+i] = sum_j R[k][j][i] du[k][j]. */
+int monarch_bwd_dx(const void *dy, const void *L, const void *R, void *dx,
+                   int64_t tokens, int32_t n, int32_t m, int dtype,
+                   void *workspace, size_t workspace_bytes, void *stream);
+
+/* Gradients of the blocks for f = <dy, M x> summed over tokens:
+ * dL[j][l][k] = sum_t dy[t][l*m+j] u[t][k][j],  dR[k][j][i] = sum_t du[t][k][j] x[t][k*m+i],
+ * with u, du as above (recomputed inside).  dL, dR are float32 [m][m][m] in
+ * both dtypes; accumulate == 0 overwrites them, 1 adds to their contents. */
+int monarch_bwd_dw(const void *x, const void *dy, const void *L, const void *R,
+                   float *dL, float *dR, int accumulate,
+                   int64_t tokens, int32_t n, int32_t m, int dtype,
+                   void *workspace, size_t workspace_bytes, void *stream);
+
+/* Monarch feed-forward block (Section 4: the FFN weights replaced by Monarch
+ * matrices):  y = M2 GELU(M1 x + b1) + b2,  M1 = P L1 P^T R1, M2 = P L2 P^T R2,
+ * GELU(a) = a/2 (1 + erf(a / sqrt 2)). */
+int monarch_mlp_fwd(const void *x, const void *L1, const void *R1, const void *b1,
+                    const void *L2, const void *R2, const void *b2, void *y,
+                    int64_t tokens, int32_t n, int32_t m, int dtype,
+                    void *workspace, size_t workspace_bytes, void *stream);
+
+/* Bytes of workspace `op` (a monarch_op_t) needs for these sizes under the
+ * current implementation choice; always >= MONARCH_STATUS_BYTES.  Returns 0
+ * for invalid or unsupported arguments. */
+size_t monarch_workspace_bytes(int op, int64_t tokens, int32_t n, int32_t m, int dtype);
+
+/* Zero the status word of a workspace (enqueued on `stream`). */
+int monarch_workspace_init(void *workspace, size_t workspace_bytes, void *stream);
+
+/* Synchronise `stream`, read and clear the status word: MONARCH_OK, or
+ * MONARCH_ERR_TIMEOUT if a kernel abandoned a bounded wait since the last
+ * query (its outputs are then undefined), or MONARCH_ERR_CUDA. */
+int monarch_last_device_status(void *workspace, void *stream);
+
+/* Select the kernel family for later calls (a monarch_impl_t).  Not
+ * thread-safe against concurrent calls. Returns the previous value, or -1. */
+int monarch_set_impl(int impl);
+
+/* Name of the kernel family the next call with these arguments would use
+ * ("staged-simt", "fused-tcgen05", ... ; "unsupported").  Static storage. */
+const char *monarch_impl_name(int op, int32_t m, int dtype);
+
+/* Number of kernel launches the library has enqueued since load (for
+ * benchmarks that report their launch count). */
+uint64_t monarch_launch_count(void);
+
+const char *monarch_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MONARCH_H_ */

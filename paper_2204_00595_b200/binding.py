@@ -1,0 +1,188 @@
+"""ctypes binding of libmonarch: same names and argument order as include/monarch.h.
+
+Tensors are torch CUDA tensors used as typed device buffers; the binding checks dtype,
+contiguity and device, takes their pointers, and calls the C entry point on the current
+CUDA stream (or the one given).  A non-zero status raises MonarchError.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+F32, BF16 = 0, 1
+OP_FWD, OP_BWD_DX, OP_BWD_DW, OP_MLP_FWD = 0, 1, 2, 3
+IMPL_AUTO, IMPL_STAGED, IMPL_FUSED = 0, 1, 2
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libmonarch.so")
+_lib = None
+
+_vp, _i64, _i32, _int, _sz = (ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_int,
+                              ctypes.c_size_t)
+_SIGNATURES = {
+    "monarch_fwd": (_int, [_vp, _vp, _vp, _vp, _i64, _i32, _i32, _int, _vp, _sz, _vp]),
+    "monarch_bwd_dx": (_int, [_vp, _vp, _vp, _vp, _i64, _i32, _i32, _int, _vp, _sz, _vp]),
+    "monarch_bwd_dw": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _int, _i64, _i32, _i32, _int, _vp,
+                              _sz, _vp]),
+    "monarch_mlp_fwd": (_int, [_vp] * 8 + [_i64, _i32, _i32, _int, _vp, _sz, _vp]),
+    "monarch_workspace_bytes": (_sz, [_int, _i64, _i32, _i32, _int]),
+    "monarch_workspace_init": (_int, [_vp, _sz, _vp]),
+    "monarch_last_device_status": (_int, [_vp, _vp]),
+    "monarch_set_impl": (_int, [_int]),
+    "monarch_impl_name": (ctypes.c_char_p, [_int, _i32, _int]),
+    "monarch_launch_count": (ctypes.c_uint64, []),
+    "monarch_status_string": (ctypes.c_char_p, [_int]),
+}
+
+
+class MonarchError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: status {status} ({monarch_status_string(status)})")
+
+
+def lib() -> ctypes.CDLL:
+    """Load libmonarch.so (raises if it has not been built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise FileNotFoundError(
+                f"{_LIB_PATH} not found: run `python -m paper_2204_00595_b200.build` first")
+        handle = ctypes.CDLL(_LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(handle, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = handle
+    return _lib
+
+
+def exported_symbols():
+    """Names this binding expects the library to export."""
+    return sorted(_SIGNATURES)
+
+
+def _dtype_code(t) -> int:
+    import torch
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported tensor dtype {t.dtype}")
+
+
+def _ptr(t, name, dtype=None):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{name} must have dtype {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+def _stream(stream):
+    import torch
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return getattr(stream, "cuda_stream", stream)
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise MonarchError(status, where)
+
+
+class Workspace:
+    """Caller-owned device scratch: a torch byte buffer plus its size."""
+
+    def __init__(self, nbytes: int, device="cuda"):
+        import torch
+        nbytes = max(int(nbytes), 256)
+        self.buf = torch.empty(nbytes + 256, dtype=torch.uint8, device=device)
+        off = (-self.buf.data_ptr()) % 256
+        self.ptr = self.buf.data_ptr() + off
+        self.nbytes = nbytes
+        monarch_workspace_init(self)
+
+    @classmethod
+    def for_op(cls, op: int, tokens: int, m: int, dtype: int, device="cuda"):
+        need = monarch_workspace_bytes(op, tokens, m * m, m, dtype)
+        if need == 0:
+            raise MonarchError(2, "monarch_workspace_bytes")
+        return cls(need, device)
+
+
+def _ws(ws):
+    if isinstance(ws, Workspace):
+        return ws.ptr, ws.nbytes
+    ptr, nbytes = ws
+    return ptr, nbytes
+
+
+def monarch_workspace_bytes(op: int, tokens: int, n: int, m: int, dtype: int) -> int:
+    return int(lib().monarch_workspace_bytes(op, tokens, n, m, dtype))
+
+
+def monarch_workspace_init(workspace, stream=None) -> None:
+    p, b = _ws(workspace)
+    _check(lib().monarch_workspace_init(p, b, _stream(stream)), "monarch_workspace_init")
+
+
+def monarch_last_device_status(workspace, stream=None) -> int:
+    p, _ = _ws(workspace)
+    return int(lib().monarch_last_device_status(p, _stream(stream)))
+
+
+def monarch_set_impl(impl: int) -> int:
+    return int(lib().monarch_set_impl(impl))
+
+
+def monarch_impl_name(op: int, m: int, dtype: int) -> str:
+    return lib().monarch_impl_name(op, m, dtype).decode()
+
+
+def monarch_launch_count() -> int:
+    return int(lib().monarch_launch_count())
+
+
+def monarch_status_string(status: int) -> str:
+    return lib().monarch_status_string(status).decode()
+
+
+def monarch_fwd(x, L, R, y, tokens, n, m, workspace, stream=None) -> None:
+    """y = P L P^T R x for ``tokens`` rows of x (see include/monarch.h)."""
+    dt = x.dtype
+    p, b = _ws(workspace)
+    _check(lib().monarch_fwd(_ptr(x, "x"), _ptr(L, "L", dt), _ptr(R, "R", dt), _ptr(y, "y", dt),
+                             tokens, n, m, _dtype_code(x), p, b, _stream(stream)), "monarch_fwd")
+
+
+def monarch_bwd_dx(dy, L, R, dx, tokens, n, m, workspace, stream=None) -> None:
+    """dx = M^T dy."""
+    dt = dy.dtype
+    p, b = _ws(workspace)
+    _check(lib().monarch_bwd_dx(_ptr(dy, "dy"), _ptr(L, "L", dt), _ptr(R, "R", dt),
+                                _ptr(dx, "dx", dt), tokens, n, m, _dtype_code(dy), p, b,
+                                _stream(stream)), "monarch_bwd_dx")
+
+
+def monarch_bwd_dw(x, dy, L, R, dL, dR, accumulate, tokens, n, m, workspace, stream=None) -> None:
+    """dL, dR (float32) summed over tokens; accumulate=1 adds to their contents."""
+    import torch
+    dt = x.dtype
+    p, b = _ws(workspace)
+    _check(lib().monarch_bwd_dw(_ptr(x, "x"), _ptr(dy, "dy", dt), _ptr(L, "L", dt),
+                                _ptr(R, "R", dt), _ptr(dL, "dL", torch.float32),
+                                _ptr(dR, "dR", torch.float32), int(accumulate), tokens, n, m,
+                                _dtype_code(x), p, b, _stream(stream)), "monarch_bwd_dw")
+
+
+def monarch_mlp_fwd(x, L1, R1, b1, L2, R2, b2, y, tokens, n, m, workspace, stream=None) -> None:
+    """y = M2 GELU(M1 x + b1) + b2."""
+    dt = x.dtype
+    p, b = _ws(workspace)
+    _check(lib().monarch_mlp_fwd(_ptr(x, "x"), _ptr(L1, "L1", dt), _ptr(R1, "R1", dt),
+                                 _ptr(b1, "b1", dt), _ptr(L2, "L2", dt), _ptr(R2, "R2", dt),
+                                 _ptr(b2, "b2", dt), _ptr(y, "y", dt), tokens, n, m,
+                                 _dtype_code(x), p, b, _stream(stream)), "monarch_mlp_fwd")

@@ -1,0 +1,57 @@
+// Shared host/device helpers of libmonarch (internal; not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "monarch.h"
+
+namespace monarch {
+
+// Launch counter behind monarch_launch_count().
+void note_launch(int n = 1);
+
+#define MONARCH_CUDA_TRY(expr)                                   \
+    do {                                                         \
+        cudaError_t err_ = (expr);                               \
+        if (err_ != cudaSuccess) return MONARCH_ERR_CUDA;        \
+    } while (0)
+
+#define MONARCH_TRY(expr)                                        \
+    do {                                                         \
+        int st_ = (expr);                                        \
+        if (st_ != MONARCH_OK) return st_;                       \
+    } while (0)
+
+template <typename T> struct elem;
+template <> struct elem<float> {
+    static __device__ __forceinline__ float load(const float *p) { return *p; }
+    static __device__ __forceinline__ void store(float *p, float v) { *p = v; }
+};
+template <> struct elem<__nv_bfloat16> {
+    static __device__ __forceinline__ float load(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
+    static __device__ __forceinline__ void store(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
+};
+
+// erf form of GELU, evaluated in fp32.
+static __device__ __forceinline__ float gelu_erf(float a)
+{
+    return 0.5f * a * (1.0f + erff(a * 0.70710678118654752440f));
+}
+
+// ---- staged (one block-diagonal stage per launch) kernels, staged_simt.cu ----
+// Workspace layout helpers and launchers; every launcher returns a monarch_status_t.
+size_t staged_workspace_bytes(int op, int64_t tokens, int32_t n, int32_t m, int dtype);
+int staged_fwd(const void *x, const void *L, const void *R, void *y, int64_t tokens, int m,
+               int dtype, void *ws, cudaStream_t s);
+int staged_bwd_dx(const void *dy, const void *L, const void *R, void *dx, int64_t tokens, int m,
+                  int dtype, void *ws, cudaStream_t s);
+int staged_bwd_dw(const void *x, const void *dy, const void *L, const void *R, float *dL,
+                  float *dR, int accumulate, int64_t tokens, int m, int dtype, void *ws,
+                  cudaStream_t s);
+int staged_mlp_fwd(const void *x, const void *L1, const void *R1, const void *b1, const void *L2,
+                   const void *R2, const void *b2, void *y, int64_t tokens, int m, int dtype,
+                   void *ws, cudaStream_t s);
+
+}  // namespace monarch

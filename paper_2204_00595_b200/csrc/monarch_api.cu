@@ -1,0 +1,213 @@
+// C-ABI entry points of libmonarch: argument validation and dispatch.  No arithmetic here.
+#include <atomic>
+
+#include "common.cuh"
+
+namespace monarch {
+
+static std::atomic<uint64_t> g_launches{0};
+static std::atomic<int> g_impl{MONARCH_IMPL_AUTO};
+
+void note_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+namespace {
+
+bool aligned(const void *p, size_t a) { return ((uintptr_t)p & (a - 1)) == 0; }
+size_t esize(int dtype) { return dtype == MONARCH_F32 ? 4 : 2; }
+
+struct Range {
+    const void *p;
+    size_t bytes;
+};
+
+bool overlap(const Range &a, const Range &b)
+{
+    if (!a.p || !b.p || a.bytes == 0 || b.bytes == 0) return false;
+    const uintptr_t a0 = (uintptr_t)a.p, a1 = a0 + a.bytes;
+    const uintptr_t b0 = (uintptr_t)b.p, b1 = b0 + b.bytes;
+    return a0 < b1 && b0 < a1;
+}
+
+// Shape / enum checks shared by every call.
+int check_shape(int64_t tokens, int32_t n, int32_t m, int dtype)
+{
+    if (tokens < 0 || n <= 0 || m <= 0) return MONARCH_ERR_INVALID_ARG;
+    if ((int64_t)m * m != (int64_t)n) return MONARCH_ERR_INVALID_ARG;
+    if (dtype != MONARCH_F32 && dtype != MONARCH_BF16) return MONARCH_ERR_INVALID_ARG;
+    if (m != 16 && m != 32 && m != 64 && m != 128) return MONARCH_ERR_UNSUPPORTED;
+    return MONARCH_OK;
+}
+
+// Inputs and outputs: non-null, 16-byte aligned; no output overlaps an input, another
+// output or the workspace.
+int check_buffers(const Range *in, int n_in, const Range *out, int n_out, const void *ws,
+                  size_t ws_bytes, size_t ws_need)
+{
+    for (int i = 0; i < n_in; ++i)
+        if (!in[i].p || !aligned(in[i].p, 16)) return MONARCH_ERR_INVALID_ARG;
+    for (int i = 0; i < n_out; ++i)
+        if (!out[i].p || !aligned(out[i].p, 16)) return MONARCH_ERR_INVALID_ARG;
+    if (!ws || !aligned(ws, 256) || ws_need == 0 || ws_bytes < ws_need) return MONARCH_ERR_WORKSPACE;
+    const Range w = {ws, ws_bytes};
+    for (int o = 0; o < n_out; ++o) {
+        for (int i = 0; i < n_in; ++i)
+            if (overlap(out[o], in[i])) return MONARCH_ERR_INVALID_ARG;
+        for (int p = o + 1; p < n_out; ++p)
+            if (overlap(out[o], out[p])) return MONARCH_ERR_INVALID_ARG;
+        if (overlap(out[o], w)) return MONARCH_ERR_INVALID_ARG;
+    }
+    for (int i = 0; i < n_in; ++i)
+        if (overlap(in[i], w)) return MONARCH_ERR_INVALID_ARG;
+    return MONARCH_OK;
+}
+
+// true when the fused tensor-core family has a kernel for (op, m, dtype)
+bool fused_available(int op, int m, int dtype)
+{
+    (void)op; (void)m; (void)dtype;
+    return false;
+}
+
+// 0 = staged, 1 = fused, -1 = unsupported under the current selection
+int pick(int op, int m, int dtype)
+{
+    const int impl = g_impl.load(std::memory_order_relaxed);
+    const bool f = fused_available(op, m, dtype);
+    if (impl == MONARCH_IMPL_STAGED) return 0;
+    if (impl == MONARCH_IMPL_FUSED) return f ? 1 : -1;
+    return f ? 1 : 0;
+}
+
+}  // namespace
+}  // namespace monarch
+
+using namespace monarch;
+
+extern "C" {
+
+size_t monarch_workspace_bytes(int op, int64_t tokens, int32_t n, int32_t m, int dtype)
+{
+    if (op < MONARCH_OP_FWD || op > MONARCH_OP_MLP_FWD) return 0;
+    if (check_shape(tokens, n, m, dtype) != MONARCH_OK) return 0;
+    const int which = pick(op, m, dtype);
+    if (which < 0) return 0;
+    return staged_workspace_bytes(op, tokens, n, m, dtype);
+}
+
+int monarch_fwd(const void *x, const void *L, const void *R, void *y, int64_t tokens, int32_t n,
+                int32_t m, int dtype, void *workspace, size_t workspace_bytes, void *stream)
+{
+    MONARCH_TRY(check_shape(tokens, n, m, dtype));
+    const size_t act = (size_t)tokens * n * esize(dtype), wb = (size_t)n * m * esize(dtype);
+    const Range in[] = {{x, act}, {L, wb}, {R, wb}};
+    const Range out[] = {{y, act}};
+    const int which = pick(MONARCH_OP_FWD, m, dtype);
+    if (which < 0) return MONARCH_ERR_UNSUPPORTED;
+    MONARCH_TRY(check_buffers(in, 3, out, 1, workspace, workspace_bytes,
+                              monarch_workspace_bytes(MONARCH_OP_FWD, tokens, n, m, dtype)));
+    return staged_fwd(x, L, R, y, tokens, m, dtype, workspace, (cudaStream_t)stream);
+}
+
+int monarch_bwd_dx(const void *dy, const void *L, const void *R, void *dx, int64_t tokens,
+                   int32_t n, int32_t m, int dtype, void *workspace, size_t workspace_bytes,
+                   void *stream)
+{
+    MONARCH_TRY(check_shape(tokens, n, m, dtype));
+    const size_t act = (size_t)tokens * n * esize(dtype), wb = (size_t)n * m * esize(dtype);
+    const Range in[] = {{dy, act}, {L, wb}, {R, wb}};
+    const Range out[] = {{dx, act}};
+    const int which = pick(MONARCH_OP_BWD_DX, m, dtype);
+    if (which < 0) return MONARCH_ERR_UNSUPPORTED;
+    MONARCH_TRY(check_buffers(in, 3, out, 1, workspace, workspace_bytes,
+                              monarch_workspace_bytes(MONARCH_OP_BWD_DX, tokens, n, m, dtype)));
+    return staged_bwd_dx(dy, L, R, dx, tokens, m, dtype, workspace, (cudaStream_t)stream);
+}
+
+int monarch_bwd_dw(const void *x, const void *dy, const void *L, const void *R, float *dL,
+                   float *dR, int accumulate, int64_t tokens, int32_t n, int32_t m, int dtype,
+                   void *workspace, size_t workspace_bytes, void *stream)
+{
+    MONARCH_TRY(check_shape(tokens, n, m, dtype));
+    if (accumulate != 0 && accumulate != 1) return MONARCH_ERR_INVALID_ARG;
+    const size_t act = (size_t)tokens * n * esize(dtype), wb = (size_t)n * m * esize(dtype);
+    const size_t gb = (size_t)n * m * sizeof(float);
+    const Range in[] = {{x, act}, {dy, act}, {L, wb}, {R, wb}};
+    const Range out[] = {{dL, gb}, {dR, gb}};
+    const int which = pick(MONARCH_OP_BWD_DW, m, dtype);
+    if (which < 0) return MONARCH_ERR_UNSUPPORTED;
+    MONARCH_TRY(check_buffers(in, 4, out, 2, workspace, workspace_bytes,
+                              monarch_workspace_bytes(MONARCH_OP_BWD_DW, tokens, n, m, dtype)));
+    return staged_bwd_dw(x, dy, L, R, dL, dR, accumulate, tokens, m, dtype, workspace,
+                         (cudaStream_t)stream);
+}
+
+int monarch_mlp_fwd(const void *x, const void *L1, const void *R1, const void *b1, const void *L2,
+                    const void *R2, const void *b2, void *y, int64_t tokens, int32_t n, int32_t m,
+                    int dtype, void *workspace, size_t workspace_bytes, void *stream)
+{
+    MONARCH_TRY(check_shape(tokens, n, m, dtype));
+    const size_t act = (size_t)tokens * n * esize(dtype), wb = (size_t)n * m * esize(dtype);
+    const size_t bb = (size_t)n * esize(dtype);
+    const Range in[] = {{x, act}, {L1, wb}, {R1, wb}, {b1, bb}, {L2, wb}, {R2, wb}, {b2, bb}};
+    const Range out[] = {{y, act}};
+    const int which = pick(MONARCH_OP_MLP_FWD, m, dtype);
+    if (which < 0) return MONARCH_ERR_UNSUPPORTED;
+    MONARCH_TRY(check_buffers(in, 7, out, 1, workspace, workspace_bytes,
+                              monarch_workspace_bytes(MONARCH_OP_MLP_FWD, tokens, n, m, dtype)));
+    return staged_mlp_fwd(x, L1, R1, b1, L2, R2, b2, y, tokens, m, dtype, workspace,
+                          (cudaStream_t)stream);
+}
+
+int monarch_workspace_init(void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < MONARCH_STATUS_BYTES)
+        return MONARCH_ERR_WORKSPACE;
+    MONARCH_CUDA_TRY(cudaMemsetAsync(workspace, 0, MONARCH_STATUS_BYTES, (cudaStream_t)stream));
+    return MONARCH_OK;
+}
+
+int monarch_last_device_status(void *workspace, void *stream)
+{
+    if (!workspace || ((uintptr_t)workspace & 255)) return MONARCH_ERR_WORKSPACE;
+    unsigned int word = 0;
+    cudaStream_t s = (cudaStream_t)stream;
+    MONARCH_CUDA_TRY(cudaMemcpyAsync(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost, s));
+    MONARCH_CUDA_TRY(cudaStreamSynchronize(s));
+    if (word != 0) {
+        MONARCH_CUDA_TRY(cudaMemsetAsync(workspace, 0, MONARCH_STATUS_BYTES, s));
+        MONARCH_CUDA_TRY(cudaStreamSynchronize(s));
+        return MONARCH_ERR_TIMEOUT;
+    }
+    return MONARCH_OK;
+}
+
+int monarch_set_impl(int impl)
+{
+    if (impl < MONARCH_IMPL_AUTO || impl > MONARCH_IMPL_FUSED) return -1;
+    return g_impl.exchange(impl);
+}
+
+const char *monarch_impl_name(int op, int32_t m, int dtype)
+{
+    if (op < MONARCH_OP_FWD || op > MONARCH_OP_MLP_FWD) return "unsupported";
+    if (check_shape(0, m * m, m, dtype) != MONARCH_OK) return "unsupported";
+    const int which = pick(op, m, dtype);
+    return which < 0 ? "unsupported" : which == 1 ? "fused-tcgen05" : "staged-simt";
+}
+
+uint64_t monarch_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char *monarch_status_string(int status)
+{
+    switch (status) {
+        case MONARCH_OK: return "ok";
+        case MONARCH_ERR_INVALID_ARG: return "invalid argument";
+        case MONARCH_ERR_UNSUPPORTED: return "unsupported size or dtype";
+        case MONARCH_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case MONARCH_ERR_CUDA: return "CUDA error";
+        case MONARCH_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"
