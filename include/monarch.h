@@ -129,6 +129,32 @@ uint64_t monarch_launch_count(void);
 
 const char *monarch_status_string(int status);
 
+/* Forward pass y = M x for callers that cannot allocate device memory - code running where
+ * cudaMalloc is off limits (a real-time or serving loop whose device memory was fixed at
+ * start-up, a plug-in under a host framework that owns the whole device heap, a process
+ * whose memory budget is already spent) and that has no spare buffer to lend as a workspace.
+ * The paper has no counterpart; this is a convenience of this library.
+ *
+ * Same arguments, layouts and results as monarch_fwd, minus the workspace: the
+ * intermediate between the two stages is kept in an array built into the library
+ * (MONARCH_NOALLOC_SCRATCH_BYTES, resident on every GPU that loads the library until the
+ * process exits).  The call allocates and frees nothing.
+ *
+ *  - Limit: tokens * n * sizeof(element) must not exceed MONARCH_NOALLOC_SCRATCH_BYTES
+ *    (e.g. 1024 tokens of n = 4096 in bf16); larger problems return
+ *    MONARCH_ERR_WORKSPACE and enqueue nothing - split the batch or use monarch_fwd.
+ *  - The first call on each device looks up the device address of the built-in array
+ *    (with that device current).  Make that first call before starting any stream capture.
+ *  - All calls share the one array and it keeps the previous call's contents.  Nothing in
+ *    it has to start at zero (each call overwrites what it later reads), but two calls
+ *    that may run at the same time on one GPU - different streams, or different host
+ *    threads - race on it: serialise them on one stream.
+ *  - Served by the staged kernel family regardless of monarch_set_impl.
+ */
+#define MONARCH_NOALLOC_SCRATCH_BYTES (8u << 20)
+int monarch_fwd_noalloc(const void *x, const void *L, const void *R, void *y,
+                        int64_t tokens, int32_t n, int32_t m, int dtype, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

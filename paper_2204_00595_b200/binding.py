@@ -31,6 +31,7 @@ _SIGNATURES = {
     "monarch_impl_name": (ctypes.c_char_p, [_int, _i32, _int]),
     "monarch_launch_count": (ctypes.c_uint64, []),
     "monarch_status_string": (ctypes.c_char_p, [_int]),
+    "monarch_fwd_noalloc": (_int, [_vp, _vp, _vp, _vp, _i64, _i32, _i32, _int, _vp]),
 }
 
 
@@ -186,3 +187,19 @@ def monarch_mlp_fwd(x, L1, R1, b1, L2, R2, b2, y, tokens, n, m, workspace, strea
                                  _ptr(b1, "b1", dt), _ptr(L2, "L2", dt), _ptr(R2, "R2", dt),
                                  _ptr(b2, "b2", dt), _ptr(y, "y", dt), tokens, n, m,
                                  _dtype_code(x), p, b, _stream(stream)), "monarch_mlp_fwd")
+
+
+NOALLOC_SCRATCH_BYTES = 8 << 20
+
+
+def monarch_fwd_noalloc(x, L, R, y, tokens, n, m, stream=None) -> None:
+    """y = P L P^T R x without a workspace, for callers that cannot allocate device memory.
+
+    The intermediate lives in an array built into the library, so the problem must satisfy
+    tokens * n * element_size <= NOALLOC_SCRATCH_BYTES; calls share that array, so do not
+    let two of them overlap on one GPU (see include/monarch.h).
+    """
+    dt = x.dtype
+    _check(lib().monarch_fwd_noalloc(_ptr(x, "x"), _ptr(L, "L", dt), _ptr(R, "R", dt),
+                                     _ptr(y, "y", dt), tokens, n, m, _dtype_code(x),
+                                     _stream(stream)), "monarch_fwd_noalloc")

@@ -9,6 +9,8 @@
 //
 // This family serves float32 (where tensor cores cannot meet the 1e-5 tolerance) and every
 // size that has no fused tensor-core kernel.  It is arithmetic-bound, not HBM-bound.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace monarch {
@@ -320,3 +322,71 @@ int staged_mlp_fwd(const void *x, const void *L1, const void *R1, const void *b1
 }
 
 }  // namespace monarch
+
+// ------------------------------------------------------------------------------------------
+// Forward pass for callers that cannot allocate device memory.
+//
+// The scratch that monarch_fwd takes from the caller's workspace (the permuted intermediate
+// between the two stages) lives here in a fixed array in the library's device image, so the
+// caller passes only inputs and outputs.  Every GPU that loads the library holds these
+// MONARCH_NOALLOC_SCRATCH_BYTES until the process exits.
+namespace monarch {
+namespace {
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[MONARCH_NOALLOC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_noalloc_mutex;
+void *g_noalloc_ptr[kMaxDevices] = {};   // device address of the array, per device ordinal
+
+// In host code `g_noalloc_scratch` is only a handle, not a device address: the address a
+// kernel can use has to be asked for, once per device, while that device is current.
+int noalloc_scratch_address(void **out)
+{
+    int dev = -1;
+    MONARCH_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return MONARCH_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[dev]) {
+        void *p = nullptr;
+        MONARCH_CUDA_TRY(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+        if (!p) return MONARCH_ERR_CUDA;
+        g_noalloc_ptr[dev] = p;
+    }
+    *out = g_noalloc_ptr[dev];
+    return MONARCH_OK;
+}
+
+bool ranges_overlap(const void *a, size_t ab, const void *b, size_t bb)
+{
+    const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+    return ab && bb && a0 < b0 + bb && b0 < a0 + ab;
+}
+
+}  // namespace
+}  // namespace monarch
+
+extern "C" int monarch_fwd_noalloc(const void *x, const void *L, const void *R, void *y,
+                                   int64_t tokens, int32_t n, int32_t m, int dtype, void *stream)
+{
+    using namespace monarch;
+    if (tokens < 0 || n <= 0 || m <= 0 || (int64_t)m * m != (int64_t)n) return MONARCH_ERR_INVALID_ARG;
+    if (dtype != MONARCH_F32 && dtype != MONARCH_BF16) return MONARCH_ERR_INVALID_ARG;
+    if (m != 16 && m != 32 && m != 64 && m != 128) return MONARCH_ERR_UNSUPPORTED;
+    const void *ptrs[] = {x, L, R, y};
+    for (const void *p : ptrs)
+        if (!p || ((uintptr_t)p & 15)) return MONARCH_ERR_INVALID_ARG;
+    const size_t act = (size_t)tokens * n * esize(dtype), wb = (size_t)n * m * esize(dtype);
+    if (ranges_overlap(y, act, x, act) || ranges_overlap(y, act, L, wb) || ranges_overlap(y, act, R, wb))
+        return MONARCH_ERR_INVALID_ARG;
+    // the intermediate needs one element per input element; it must fit the built-in array
+    if (act > (size_t)MONARCH_NOALLOC_SCRATCH_BYTES) return MONARCH_ERR_WORKSPACE;
+    if (tokens == 0) return MONARCH_OK;
+    void *u = nullptr;
+    MONARCH_TRY(noalloc_scratch_address(&u));
+    cudaStream_t s = (cudaStream_t)stream;
+    // Every element of the intermediate that the second stage reads is written by the first
+    // stage of this same call, so nothing left over from an earlier call is ever consumed.
+    MONARCH_TRY(stage(dtype, false, m, x, R, u, nullptr, 0, tokens, s));
+    return stage(dtype, false, m, u, L, y, nullptr, 0, tokens, s);
+}
