@@ -54,4 +54,12 @@ int staged_mlp_fwd(const void *x, const void *L1, const void *R1, const void *b1
                    const void *R2, const void *b2, void *y, int64_t tokens, int m, int dtype,
                    void *ws, cudaStream_t s);
 
+
+// ---- tensor-core stage chains through the workspace (bf16, m >= 32), tc_stage.cu ----
+int tc_staged_fwd(const void *x, const void *L, const void *R, void *y, int64_t tokens, int m,
+                  void *ws, cudaStream_t s);
+int tc_staged_mlp_fwd(const void *x, const void *L1, const void *R1, const void *b1, const void *L2,
+                      const void *R2, const void *b2, void *y, int64_t tokens, int m, void *ws,
+                      cudaStream_t s);
+
 }  // namespace monarch

@@ -61,6 +61,8 @@ int check_buffers(const Range *in, int n_in, const Range *out, int n_out, const 
     return MONARCH_OK;
 }
 
+enum Family { kSimt = 0, kFused = 1, kTcStaged = 2, kNone = -1 };
+
 // true when the fused tensor-core family has a kernel for (op, m, dtype)
 bool fused_available(int op, int m, int dtype)
 {
@@ -68,14 +70,21 @@ bool fused_available(int op, int m, int dtype)
     return false;
 }
 
-// 0 = staged, 1 = fused, -1 = unsupported under the current selection
+// true when the call can run as a chain of tensor-core stages through the workspace
+bool tc_staged_available(int op, int m, int dtype)
+{
+    return dtype == MONARCH_BF16 && m >= 32 && (op == MONARCH_OP_FWD || op == MONARCH_OP_MLP_FWD);
+}
+
+// kernel family for a call under the current selection
 int pick(int op, int m, int dtype)
 {
     const int impl = g_impl.load(std::memory_order_relaxed);
     const bool f = fused_available(op, m, dtype);
-    if (impl == MONARCH_IMPL_STAGED) return 0;
-    if (impl == MONARCH_IMPL_FUSED) return f ? 1 : -1;
-    return f ? 1 : 0;
+    if (impl == MONARCH_IMPL_STAGED) return kSimt;
+    if (impl == MONARCH_IMPL_FUSED) return f ? kFused : kNone;
+    if (f) return kFused;
+    return tc_staged_available(op, m, dtype) ? kTcStaged : kSimt;
 }
 
 }  // namespace
@@ -105,6 +114,7 @@ int monarch_fwd(const void *x, const void *L, const void *R, void *y, int64_t to
     if (which < 0) return MONARCH_ERR_UNSUPPORTED;
     MONARCH_TRY(check_buffers(in, 3, out, 1, workspace, workspace_bytes,
                               monarch_workspace_bytes(MONARCH_OP_FWD, tokens, n, m, dtype)));
+    if (which == kTcStaged) return tc_staged_fwd(x, L, R, y, tokens, m, workspace, (cudaStream_t)stream);
     return staged_fwd(x, L, R, y, tokens, m, dtype, workspace, (cudaStream_t)stream);
 }
 
@@ -154,6 +164,9 @@ int monarch_mlp_fwd(const void *x, const void *L1, const void *R1, const void *b
     if (which < 0) return MONARCH_ERR_UNSUPPORTED;
     MONARCH_TRY(check_buffers(in, 7, out, 1, workspace, workspace_bytes,
                               monarch_workspace_bytes(MONARCH_OP_MLP_FWD, tokens, n, m, dtype)));
+    if (which == kTcStaged)
+        return tc_staged_mlp_fwd(x, L1, R1, b1, L2, R2, b2, y, tokens, m, workspace,
+                                 (cudaStream_t)stream);
     return staged_mlp_fwd(x, L1, R1, b1, L2, R2, b2, y, tokens, m, dtype, workspace,
                           (cudaStream_t)stream);
 }
@@ -192,7 +205,8 @@ const char *monarch_impl_name(int op, int32_t m, int dtype)
     if (op < MONARCH_OP_FWD || op > MONARCH_OP_MLP_FWD) return "unsupported";
     if (check_shape(0, m * m, m, dtype) != MONARCH_OK) return "unsupported";
     const int which = pick(op, m, dtype);
-    return which < 0 ? "unsupported" : which == 1 ? "fused-tcgen05" : "staged-simt";
+    return which < 0 ? "unsupported" : which == kFused ? "fused-tcgen05"
+         : which == kTcStaged ? "staged-tcgen05" : "staged-simt";
 }
 
 uint64_t monarch_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
