@@ -1,5 +1,6 @@
 // C-ABI entry points of libmonarch: argument validation and dispatch.  No arithmetic here.
 #include <atomic>
+#include <cstdlib>
 
 #include "common.cuh"
 
@@ -66,8 +67,18 @@ enum Family { kSimt = 0, kFused = 1, kTcStaged = 2, kNone = -1 };
 // true when the fused tensor-core family has a kernel for (op, m, dtype)
 bool fused_available(int op, int m, int dtype)
 {
-    (void)op; (void)m; (void)dtype;
-    return false;
+    return dtype == MONARCH_BF16 && m == 64 && op == MONARCH_OP_FWD;
+}
+
+// Development switch: MONARCH_FUSED_MODE=0 runs the fused forward as one launch per stage.
+int fused_mode()
+{
+    static int mode = -1;
+    if (mode < 0) {
+        const char *e = getenv("MONARCH_FUSED_MODE");
+        mode = (e && e[0] == '0') ? 0 : 2;
+    }
+    return mode;
 }
 
 // true when the call can run as a chain of tensor-core stages through the workspace
@@ -100,6 +111,7 @@ size_t monarch_workspace_bytes(int op, int64_t tokens, int32_t n, int32_t m, int
     if (check_shape(tokens, n, m, dtype) != MONARCH_OK) return 0;
     const int which = pick(op, m, dtype);
     if (which < 0) return 0;
+    if (which == kFused) return fused_fwd_m64_workspace_bytes(tokens);
     return staged_workspace_bytes(op, tokens, n, m, dtype);
 }
 
@@ -114,6 +126,8 @@ int monarch_fwd(const void *x, const void *L, const void *R, void *y, int64_t to
     if (which < 0) return MONARCH_ERR_UNSUPPORTED;
     MONARCH_TRY(check_buffers(in, 3, out, 1, workspace, workspace_bytes,
                               monarch_workspace_bytes(MONARCH_OP_FWD, tokens, n, m, dtype)));
+    if (which == kFused)
+        return fused_fwd_m64(x, L, R, y, tokens, workspace, fused_mode(), (cudaStream_t)stream);
     if (which == kTcStaged) return tc_staged_fwd(x, L, R, y, tokens, m, workspace, (cudaStream_t)stream);
     return staged_fwd(x, L, R, y, tokens, m, dtype, workspace, (cudaStream_t)stream);
 }
@@ -175,7 +189,10 @@ int monarch_workspace_init(void *workspace, size_t workspace_bytes, void *stream
 {
     if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < MONARCH_STATUS_BYTES)
         return MONARCH_ERR_WORKSPACE;
-    MONARCH_CUDA_TRY(cudaMemsetAsync(workspace, 0, MONARCH_STATUS_BYTES, (cudaStream_t)stream));
+    // status word plus the dependency counters that follow it (64 KB) where the workspace has them
+    const size_t clear = workspace_bytes < MONARCH_STATUS_BYTES + 65536 ? workspace_bytes
+                                                                         : MONARCH_STATUS_BYTES + 65536;
+    MONARCH_CUDA_TRY(cudaMemsetAsync(workspace, 0, clear, (cudaStream_t)stream));
     return MONARCH_OK;
 }
 
