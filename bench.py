@@ -37,6 +37,8 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=3, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--kernels", default="auto", choices=["auto", "staged", "fused"])
+    ap.add_argument("--calls", default="", help="comma-separated subset of the workload's calls "
+                    "(profiling aid; the default step runs them all)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -180,6 +182,8 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     calls = list(cfg.ops)
+    if args.calls:
+        calls = [k for k in calls if k in args.calls.split(",")]
     n, m, T = cfg.n, cfg.m, cfg.tokens
     workload = (f"workload {cfg.index}: {'+'.join(calls)} {cfg.dtype} n={n} m={m} "
                 f"tokens/GPU={T}")

@@ -64,9 +64,8 @@ int tc_staged_mlp_fwd(const void *x, const void *L1, const void *R1, const void 
 
 
 // ---- fused single-pass forward for m = 64, bf16 (fused_m64.cu) ----
-// mode 2: one launch, both stages dependency-tracked; mode 0: one launch per stage.
 size_t fused_fwd_m64_workspace_bytes(int64_t tokens);
 int fused_fwd_m64(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws,
-                  int mode, cudaStream_t s);
+                  cudaStream_t s);
 
 }  // namespace monarch

@@ -1,28 +1,37 @@
 // Fused Monarch forward for m = 64 (n = 4096), bf16 in/out, fp32 accumulation in TMEM.
 //
-// One persistent launch runs both block-diagonal stages and both permutations.  The work is
-// cut into items that a CTA (one per SM) processes in a fixed interleaved order:
+// One persistent launch runs both block-diagonal stages and both permutations; the
+// intermediate u never leaves the chip's L2.  CTAs (one per SM) specialise; both kinds work on
+// 64-token tiles with tcgen05.mma M = 64, whose accumulators occupy one 16-lane half of every
+// TMEM sub-partition, and both keep two tiles in flight so that one is drained while the next is
+// multiplied:
 //
-//   S1 item (128 tokens, 8 consecutive blocks k of R):
-//       TMA brings x[128 x 64] and R_k[64 x 64] per block into 128B-swizzled K-major tiles;
-//       tcgen05.mma (M=128 tokens, N=64, K=16) accumulates u[t][k][:] in TMEM columns
-//       [64*kb, 64*kb+64).  With all 8 accumulators resident, the thread that owns token t picks
-//       entry j of each block - a register renaming - and writes the 16 bytes
-//       u'[t][j][8g..8g+8) into an L2-resident exchange buffer whose layout,
-//       [64-token tile][j][k/8][t%64][k%8], makes that store fully coalesced (a warp writes 512
-//       contiguous bytes) and is at the same time the canonical no-swizzle K-major operand
-//       layout of stage 2: the inner permutation P^T costs no data movement at all.
-//   S2 item (64 tokens, 16 consecutive blocks j of L):
-//       one 8 KB bulk copy per block fetches u'_j[64 x 64] from L2, TMA fetches L_j;
-//       tcgen05.mma (M=64, N=64) accumulates w[t][j][:]; the 16 accumulators sit in the two
-//       16-lane halves of each TMEM sub-partition, so lanes i and i+16 of a warp hold blocks
-//       j0..j0+7 and j0+8..j0+15 of the same token and together store the 32 contiguous bytes
-//       y[t][l*64 + 16h .. 16h+16) - whole 32-byte sectors, which is what HBM writes need.
+//   S1 CTAs (8 groups g of `a` CTAs): keep the 8 blocks R_{8g..8g+7} resident in shared memory.
+//       Per tile, TMA brings x[64 x 64] per block into a 128B-swizzled K-major ring slot;
+//       4 MMAs (N = 64, K = 16) accumulate u[t][k][:] in TMEM columns [64*kb, 64*kb+64) of lane half
+//       (tile parity).  With all 8 accumulators resident, the thread that owns token t picks
+//       entry j of each block - a register renaming - and writes the 16 bytes u'[t][j][8g..8g+8)
+//       into the exchange buffer, whose layout [tile][j][k/8][t%64][k%8] makes that store
+//       coalesced (16 lanes write 256 contiguous bytes) and is at the same time the canonical
+//       no-swizzle K-major operand layout of stage 2: the inner permutation P^T costs no data
+//       movement at all.
+//   S2 CTAs (4 x 2 groups (hj, hl) of `b` CTAs): keep rows [32hl, 32hl+32) of L_{16hj..16hj+15}
+//       resident.  One 8 KB bulk copy per block fetches u'_j[64 x 64] from L2; 4 MMAs (N = 32)
+//       accumulate w[t][j][32hl..]; blocks 0-7 sit in lane half 0 and blocks 8-15 in lane half 1
+//       of 256 TMEM columns (tile parity picks which 256).  Lanes i and i+16 of a warp then hold
+//       blocks j0..j0+7 and j0+8..j0+15 of the same token and store, in one instruction, the 32
+//       contiguous bytes y[t][l*64 + 16hj .. 16hj+16): whole 32-byte sectors, which is what HBM
+//       writes need (16-byte pieces were measured 5x slower).
 //
-// S2 items of a token tile come `lag` tiles after its S1 items in the schedule and wait (with
-// a bound) on a per-tile counter that S1 epilogues bump after their stores, so u' is consumed
-// from L2 shortly after it is produced.  Warps: 0-3 drain TMEM, 4 issues TMA/bulk loads,
-// 5 issues MMAs; an 8-slot shared-memory ring decouples loads from MMAs across items.
+// An S2 tile waits (bounded) on a per-tile counter that the S1 epilogues bump after their stores;
+// S1 tiles wait on nothing, so the schedule cannot deadlock.  Warps 0-7 drain TMEM (two per
+// sub-partition) into shared-memory staging buffers, warps 13-14 send those out with TMA tensor
+// stores, warps 8-11 issue TMA/bulk loads, warp 12 issues every MMA.  The single-thread
+// roles are latency-bound (one thread sustains about 50 GB/s of TMA issue and one MMA per
+// 50-70 cycles), so loads are shared by four warps, ring slots are handled in groups of four (one
+// full and one empty barrier per group), and the role loops are unrolled with static offsets.
+#include <cstdlib>
+
 #include "tc_common.cuh"
 
 namespace monarch {
@@ -31,56 +40,28 @@ namespace {
 
 constexpr int kM = 64;
 constexpr int kN = kM * kM;
-constexpr int kSlots = 8;
-constexpr int kSlotBytes = 24576;            // 16 KB A + 8 KB B
-constexpr int kSlotB = 16384;                // offset of B inside a slot
-constexpr int kThreads = 192;
-constexpr int kSmemBytes = kSlots * kSlotBytes + 1024;
-constexpr unsigned kS1Arrivals = 8 * 4;      // 8 S1 items x 4 epilogue warps per 128-token tile
-constexpr unsigned kS2Items = 8;             // S2 items per 128-token tile
+constexpr int kEpiWarps = 8, kProdWarps = 4, kStoreWarps = 2;
+constexpr int kMmaWarp = kEpiWarps + kProdWarps, kStoreWarp0 = kMmaWarp + 1;
+constexpr int kThreads = (kEpiWarps + kProdWarps + 1 + kStoreWarps) * 32;
+constexpr int kSlotBytes = 8192;                       // one [64 x 64] bf16 operand tile
+constexpr int kSlots = 12, kQuads = kSlots / 4;        // ring, released and filled in groups of 4
+constexpr int kWBytes = 65536;                         // resident weights: 8 R blocks, or 16 half L blocks
+constexpr int kStageBytes = 8192, kStagesPerHalf = 4;  // output staging ring of each epilogue half
+constexpr int kStages = 2 * kStagesPerHalf;
+constexpr int kSmemBytes = kWBytes + kStages * kStageBytes + kSlots * kSlotBytes + 1024;
+constexpr unsigned kS1Arrivals = 8 * 2;                // 8 S1 groups x 2 epilogue halves per tile
+constexpr unsigned kS2Groups = 8;
 
 struct FwdParams {
-    __nv_bfloat16 *u;          // exchange buffer, [tiles64][64 j][8][64 t][8] bf16
+    __nv_bfloat16 *u;          // exchange buffer, [tiles][64 j][8][64 t][8] bf16
     __nv_bfloat16 *y;
-    unsigned *counters;        // one per 128-token tile, zero between calls
+    unsigned *counters;        // one per 64-token tile, zero between calls
     unsigned *status;
     long long tokens;
-    int tiles;                 // 128-token tiles
-    int mode;                  // 0: S1 items only, 1: S2 items only, 2: both, dependency-tracked
-    int lag;                   // tiles between a tile's S1 and S2 items (mode 2)
+    int tiles;                 // 64-token tiles
+    int a, b;                  // S1 CTAs per R group, S2 CTAs per L group
+    long long *trace;          // optional per-CTA timeline (debug builds), else null
 };
-
-struct Item {
-    int kind;   // 0 = S1, 1 = S2, -1 = none
-    int tile;   // 128-token tile
-    int sub;    // S1: block group g (0..7); S2: half*4 + h
-};
-
-// position in the global item order -> item.  Mode 2 order by tile step u: the 8 S1 items of
-// tile u (while u < tiles), then the 8 S2 items of tile u - lag (once u >= lag).
-__device__ __forceinline__ Item item_at(const FwdParams &p, long long pos)
-{
-    Item it = {-1, 0, 0};
-    if (p.mode == 0 || p.mode == 1) {
-        if (pos < (long long)p.tiles * 8) { it.kind = p.mode; it.tile = (int)(pos >> 3); it.sub = (int)(pos & 7); }
-        return it;
-    }
-    const long long lag = p.lag < p.tiles ? p.lag : p.tiles;
-    const long long a = lag * 8;                          // S1-only prefix
-    const long long b = a + (p.tiles - lag) * 16;         // mixed region
-    const long long c = b + lag * 8;                      // S2-only suffix
-    if (pos < a) { it.kind = 0; it.tile = (int)(pos >> 3); it.sub = (int)(pos & 7); }
-    else if (pos < b) {
-        const long long q = pos - a;
-        const int step = (int)(q >> 4), r = (int)(q & 15);
-        if (r < 8) { it.kind = 0; it.tile = (int)lag + step; it.sub = r; }
-        else { it.kind = 1; it.tile = step; it.sub = r - 8; }
-    } else if (pos < c) {
-        const long long q = pos - b;
-        it.kind = 1; it.tile = (int)(p.tiles - lag + (q >> 3)); it.sub = (int)(q & 7);
-    }
-    return it;
-}
 
 __device__ __forceinline__ unsigned ld_acquire(const unsigned *p)
 {
@@ -99,31 +80,348 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_
         "l"(src), "r"(bytes), "r"(bar)
         : "memory");
 }
+#ifdef MONARCH_TRACE
+#define TRACE(slot) do { if (p.trace && nitem_t < 16) p.trace[((size_t)blockIdx.x * 16 + nitem_t) * 8 + (slot)] = clock64(); } while (0)
+#else
+#define TRACE(slot) do { } while (0)
+#endif
+
+// One try before the bounded wait: the common case in the single-thread role loops, where every
+// extra dependent instruction costs several cycles.
+__device__ __forceinline__ bool wait_fast(uint32_t bar, uint32_t parity, unsigned *status, volatile int *dead,
+                                          unsigned code)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait(bar, parity, status, dead, code);
+}
+
+// Position of a tile's first block in the ring, in slot groups of four; advances without division.
+template <int QUADS_PER_TILE> struct RingBase {
+    int quad = 0;
+    uint32_t phase = 0;
+    __device__ __forceinline__ void next_tile()
+    {
+        quad += QUADS_PER_TILE;
+#pragma unroll
+        for (int i = 0; i < (QUADS_PER_TILE + kQuads - 1) / kQuads; ++i)
+            if (quad >= kQuads) { quad -= kQuads; phase ^= 1; }
+    }
+    // group index and phase of the tile's q-th group
+    __device__ __forceinline__ void at(int q, int &g, uint32_t &ph) const
+    {
+        g = quad + q;
+        ph = phase;
+#pragma unroll
+        for (int i = 0; i < (QUADS_PER_TILE + kQuads - 1) / kQuads; ++i)
+            if (g >= kQuads) { g -= kQuads; ph ^= 1; }
+    }
+};
+
+template <bool S1>
+__device__ __forceinline__ void role_body(const CUtensorMap &tm_x, const CUtensorMap &tm_R, const CUtensorMap &tm_L,
+                                          const CUtensorMap &tm_u, const CUtensorMap &tm_y, const FwdParams &p, uint32_t smem0, uint64_t *bar_full, uint64_t *bar_empty,
+                                          uint64_t *bar_acc_full, uint64_t *bar_acc_empty, uint64_t *bar_w,
+                                          uint64_t *bar_st_full, uint64_t *bar_st_free, volatile int *dep_items, uint32_t tmem_base, volatile int *dead, int grp,
+                                          int first, int step)
+{
+    constexpr int NBLK = S1 ? 8 : 16;
+    constexpr int NQ = NBLK / 4;                     // slot groups per tile
+    constexpr int WBYTES = kWBytes;
+    static_assert(kProdWarps == 4, "one producer warp per slot of a group");
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t stage0 = smem0 + kWBytes;
+    const uint32_t ring0 = stage0 + kStages * kStageBytes;
+    const int hj = grp >> 1, hl = grp & 1;           // S2 only: block group (16 blocks), output-row half
+    const int n_tiles = p.tiles;
+    if (first >= n_tiles) return;
+    const uint32_t full0 = smem_u32(bar_full), empty0 = smem_u32(bar_empty);
+    const uint32_t accf0 = smem_u32(bar_acc_full), acce0 = smem_u32(bar_acc_empty);
+
+    if (warp >= kEpiWarps && warp < kEpiWarps + kProdWarps) {
+        // ------------------------------------------------------------ producers: warp pw loads slot pw of every group
+        const int pw = warp - kEpiWarps;
+        if (lane != 0) return;
+        if (pw == 0) {
+            // resident weights of this CTA's group
+            const uint32_t wbar = smem_u32(bar_w);
+            mbar_expect_tx(wbar, WBYTES);
+            if (S1) {
+                for (int b = 0; b < 8; ++b) tma_load_2d(smem0 + b * 8192, &tm_R, 0, (grp * 8 + b) * kM, wbar);
+            } else {
+                for (int b = 0; b < 16; ++b)
+                    tma_load_2d(smem0 + b * 4096, &tm_L, 0, (hj * 16 + b) * kM + hl * 32, wbar);
+            }
+        }
+        RingBase<NQ> ring;
+        int nitem_p = 0;
+        [[maybe_unused]] int nitem_t = 0;
+        for (int tile = first; tile < n_tiles; tile += step, ++nitem_t, ++nitem_p) {
+            if (pw == 0) TRACE(0);
+            if (!S1) {
+                if (pw == 0) {
+                    // wait until all S1 groups have published their part of u' for this tile
+                    const unsigned *ctr = p.counters + tile;
+                    if (ld_acquire(ctr) < kS1Arrivals) {
+                        const unsigned long long t0 = global_timer_ns();
+                        while (ld_acquire(ctr) < kS1Arrivals) {
+                            if (*dead || global_timer_ns() - t0 > kWaitLimitNs) {
+                                *dead = 1;
+                                atomicCAS(p.status, 0u, (unsigned)kErrPeerWait);
+                                return;
+                            }
+                        }
+                    }
+                    // the last S2 group to get here clears the tile's counter for the next call
+                    const unsigned old = atomicAdd(p.counters + tile, 1u);
+                    if (old + 1 == kS1Arrivals + kS2Groups) atomicExch(p.counters + tile, 0u);
+                    fence_proxy_async_global();
+                    __threadfence_block();
+                    *dep_items = nitem_p + 1;             // monotonic: cannot alias like a parity would
+                } else {
+                    if (*dep_items <= nitem_p) {
+                        const unsigned long long t0 = global_timer_ns();
+                        while (*dep_items <= nitem_p) {
+                            if (*dead || global_timer_ns() - t0 > kWaitLimitNs) {
+                                *dead = 1;
+                                atomicCAS(p.status, 0u, (unsigned)kErrPeerWait);
+                                return;
+                            }
+                        }
+                    }
+                    __threadfence_block();
+                    fence_proxy_async_global();
+                }
+            }
+            if (pw == 0) TRACE(1);
+            const __nv_bfloat16 *usrc = p.u + ((long long)tile * 64 + hj * 16 + pw) * 4096;
+#pragma unroll
+            for (int q = 0; q < NQ; ++q) {
+                int g;
+                uint32_t ph;
+                ring.at(q, g, ph);
+                if (!wait_fast(empty0 + g * 8, ph ^ 1, p.status, dead, kErrSlotWait)) return;
+                const uint32_t full = full0 + g * 8;
+                mbar_expect_tx(full, kSlotBytes);
+                const uint32_t dst = ring0 + (g * 4 + pw) * kSlotBytes;
+                if (S1) tma_load_2d(dst, &tm_x, (grp * 8 + q * 4 + pw) * kM, tile * 64, full);
+                else bulk_load(dst, usrc + (size_t)q * 4 * 4096, 8192, full);
+            }
+            ring.next_tile();
+            if (pw == 0) TRACE(2);
+        }
+    } else if (warp == kMmaWarp) {
+        // ------------------------------------------------------------ MMA issuer (one thread issues every MMA)
+        if (lane != 0) return;
+        if (!mbar_wait(smem_u32(bar_w), 0, p.status, dead, kErrTmaWait)) return;
+        tc_fence_after();
+        RingBase<NQ> ring;
+        uint32_t nitem = 0;
+        [[maybe_unused]] int nitem_t = 0;
+        // descriptor templates: only the 14-bit start-address field changes
+        const uint64_t a_ring = (S1 ? make_smem_desc(0, 16, 1024, kSwizzle128) : make_smem_desc(0, 1024, 128, 0)) |
+                                (uint64_t)(ring0 >> 4);
+        const uint64_t b_res = make_smem_desc(0, 16, 1024, kSwizzle128) | (uint64_t)(smem0 >> 4);
+        constexpr uint32_t idesc = make_idesc_bf16(64, S1 ? 64 : 32, 0, 0);
+        constexpr int AK = S1 ? 2 : 128;             // K-step advance of the A descriptor (>>4 units)
+        for (int tile = first; tile < n_tiles; tile += step, ++nitem_t, ++nitem) {
+            // tiles alternate between two accumulator sets: lane halves (S1) or column halves (S2)
+            const uint32_t buf = nitem & 1, par = (nitem >> 1) & 1;
+            if (!wait_fast(acce0 + buf * 8, par ^ 1, p.status, dead, kErrTmemWait)) return;
+            tc_fence_after();
+            TRACE(3);
+            const uint32_t dbase = S1 ? tmem_base + ((buf * 16) << 16) : tmem_base + buf * 256;
+#pragma unroll
+            for (int q = 0; q < NQ; ++q) {
+                int g;
+                uint32_t ph;
+                ring.at(q, g, ph);
+                if (!wait_fast(full0 + g * 8, ph, p.status, dead, kErrTmaWait)) return;
+                tc_fence_after();
+                const uint64_t aq = a_ring + (uint64_t)(g * 4 * (kSlotBytes >> 4));
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int b = q * 4 + i;
+                    const uint64_t ad = aq + i * (kSlotBytes >> 4);
+                    const uint64_t bd = b_res + b * (S1 ? 512 : 256);
+                    // S2: blocks 0-7 in lanes [0,16) of each sub-partition, 8-15 in lanes [16,32)
+                    const uint32_t d = S1 ? dbase + b * 64 : dbase + ((uint32_t)((b >> 3) * 16) << 16) + (b & 7) * 32;
+                    mma_f16_ss(d, ad, bd, idesc, 0);
+                    mma_f16_ss(d, ad + AK, bd + 2, idesc, 1);
+                    mma_f16_ss(d, ad + 2 * AK, bd + 4, idesc, 1);
+                    mma_f16_ss(d, ad + 3 * AK, bd + 6, idesc, 1);
+                }
+                mma_commit(empty0 + g * 8);
+            }
+            mma_commit(accf0 + buf * 8);
+            ring.next_tile();
+            TRACE(4);
+        }
+    } else if (warp < kEpiWarps) {
+        // ------------------------------------------------------------ epilogue (warps 0-7)
+        // Two halves of four warps (one per TMEM sub-partition) take alternate chunks of a tile.  A chunk
+        // is packed to bf16 into a staging buffer and handed to the half's store thread, which sends it
+        // out with one TMA tensor store: global stores issued by these warps themselves would queue in
+        // front of the tcgen05.mma issue (measured: they halve the MMA rate), bulk stores do not.
+        const int q4 = warp & 3, sub = warp >> 2;      // TMEM sub-partition, epilogue half
+        const uint32_t lane_base = tmem_base + ((uint32_t)(q4 * 32) << 16);
+        const int row = q4 * 16 + (lane & 15);         // token row of this thread within a tile
+        const uint32_t my_stage = stage0 + sub * kStagesPerHalf * kStageBytes;
+        const uint32_t stf0 = smem_u32(bar_st_full) + sub * kStagesPerHalf * 8;
+        const uint32_t stfree0 = smem_u32(bar_st_free) + sub * kStagesPerHalf * 8;
+        uint32_t nitem = 0, nchunk = 0;
+        [[maybe_unused]] int nitem_t = 0;
+        for (int tile = first; tile < n_tiles; tile += step, ++nitem_t, ++nitem) {
+            const uint32_t buf = nitem & 1, par = (nitem >> 1) & 1;
+            if (!wait_fast(accf0 + buf * 8, par, p.status, dead, kErrMmaWait)) return;
+            tc_fence_after();
+            if (threadIdx.x == 0) TRACE(5);
+#pragma unroll 1
+            for (int c = sub; c < 8; c += 2, ++nchunk) {
+                const uint32_t k = nchunk & (kStagesPerHalf - 1);
+                const uint32_t sbuf = my_stage + k * kStageBytes;
+                // the store that last read this staging buffer must be done reading it
+                if (!wait_fast(stfree0 + k * 8, ((nchunk / kStagesPerHalf) & 1) ^ 1, p.status, dead, kErrSlotWait))
+                    return;
+                if (S1) {
+                    // accumulators of this tile live in lane half `buf`; chunk = 8 consecutive j
+                    uint32_t v[8][8];
+#pragma unroll
+                    for (int kb = 0; kb < 8; ++kb) tmem_ld8(lane_base + kb * 64 + c * 8, v[kb]);
+                    tmem_ld_wait();
+                    if ((uint32_t)(lane >> 4) == buf) {
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            const uint32_t o0 = pack_bf16(__uint_as_float(v[0][q]), __uint_as_float(v[1][q]));
+                            const uint32_t o1 = pack_bf16(__uint_as_float(v[2][q]), __uint_as_float(v[3][q]));
+                            const uint32_t o2 = pack_bf16(__uint_as_float(v[4][q]), __uint_as_float(v[5][q]));
+                            const uint32_t o3 = pack_bf16(__uint_as_float(v[6][q]), __uint_as_float(v[7][q]));
+                            // staging [j local 8][t 64][8 k]: the 1 KB slab of u'[tile][j][k/8 = g]
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sbuf + q * 1024 + row * 16),
+                                         "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
+                        }
+                    }
+                } else {
+                    // chunk = 4 consecutive output rows l; lanes i and i+16 hold blocks 0-7 and 8-15
+                    uint32_t v[8][4];
+#pragma unroll
+                    for (int a = 0; a < 8; ++a) tmem_ld4(lane_base + buf * 256 + a * 32 + c * 4, v[a]);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const uint32_t o0 = pack_bf16(__uint_as_float(v[0][q]), __uint_as_float(v[1][q]));
+                        const uint32_t o1 = pack_bf16(__uint_as_float(v[2][q]), __uint_as_float(v[3][q]));
+                        const uint32_t o2 = pack_bf16(__uint_as_float(v[4][q]), __uint_as_float(v[5][q]));
+                        const uint32_t o3 = pack_bf16(__uint_as_float(v[6][q]), __uint_as_float(v[7][q]));
+                        // staging [l local 4][t 64][16 j]
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sbuf + q * 2048 + row * 32 + (lane >> 4) * 16),
+                                     "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
+                    }
+                }
+                if (c + 2 >= 8) {
+                    // last chunk of this half: the tile's accumulators have been read
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(acce0 + buf * 8);
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(stf0 + k * 8);
+            }
+            if (threadIdx.x == 0) { TRACE(6); TRACE(7); }
+        }
+    } else if (warp >= kStoreWarp0) {
+        // ------------------------------------------------------------ store threads (one per epilogue half)
+        const int sub = warp - kStoreWarp0;
+        if (lane != 0) return;
+        const uint32_t my_stage = stage0 + sub * kStagesPerHalf * kStageBytes;
+        const uint32_t stf0 = smem_u32(bar_st_full) + sub * kStagesPerHalf * 8;
+        const uint32_t stfree0 = smem_u32(bar_st_free) + sub * kStagesPerHalf * 8;
+        uint32_t nchunk = 0;
+        int pending = -1;                              // S1: tile whose stores still await publishing
+        for (int tile = first; tile < n_tiles; tile += step) {
+#pragma unroll 1
+            for (int c = sub; c < 8; c += 2, ++nchunk) {
+                const uint32_t k = nchunk & (kStagesPerHalf - 1);
+                const uint32_t sbuf = my_stage + k * kStageBytes;
+                if (!wait_fast(stf0 + k * 8, (nchunk / kStagesPerHalf) & 1, p.status, dead, kErrMmaWait)) return;
+                if (S1) {
+                    // u' as 8-byte words: [tile*64 + j][k/8][128 words]; 8 rows (j) of 1 KB
+                    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(&tm_u),
+                                 "r"(sbuf), "r"(0), "r"(grp), "r"(tile * 64 + c * 8) : "memory");
+                } else {
+                    // y as [l][t][j]: box 16 j x 64 t x 4 l; rows past the last token are clipped
+                    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(&tm_y),
+                                 "r"(sbuf), "r"(hj * 16), "r"(tile * 64), "r"(hl * 32 + c * 4) : "memory");
+                }
+                tma_store_commit();
+                if (nchunk >= kStagesPerHalf - 1) {
+                    // keep three stores in flight (a store's read latency is 1-2 thousand cycles); the
+                    // buffer of the one before them is free again
+                    tma_store_wait_read<kStagesPerHalf - 1>();
+                    mbar_arrive(stfree0 + ((nchunk - (kStagesPerHalf - 1)) & (kStagesPerHalf - 1)) * 8);
+                }
+            }
+            if (S1) {
+                if (pending >= 0) {
+                    // the previous tile's four stores are complete once at most four newer ones are pending
+                    asm volatile("cp.async.bulk.wait_group 4;" ::: "memory");
+                    fence_proxy_async_global();
+                    __threadfence();
+                    atomicAdd(p.counters + pending, 1u);
+                }
+                pending = tile;
+            }
+        }
+        tma_store_wait_all<0>();
+        if (S1 && pending >= 0) {
+            fence_proxy_async_global();
+            __threadfence();
+            atomicAdd(p.counters + pending, 1u);
+        }
+    }
+}
 
 __global__ void __launch_bounds__(kThreads, 1)
 fused_fwd_m64_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_R,
-                     const __grid_constant__ CUtensorMap tm_L, const FwdParams p)
+                     const __grid_constant__ CUtensorMap tm_L, const __grid_constant__ CUtensorMap tm_u,
+                     const __grid_constant__ CUtensorMap tm_y, const FwdParams p)
 {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bar_full[kSlots], bar_empty[kSlots], bar_acc_full, bar_acc_empty;
+    __shared__ __align__(8) uint64_t bar_full[kQuads], bar_empty[kQuads], bar_acc_full[2], bar_acc_empty[2], bar_w,
+        bar_st_full[kStages], bar_st_free[kStages];
     __shared__ uint32_t tmem_base_s;
     __shared__ int dead;
+    __shared__ int dep_items;
 
     const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+
+    // role of this CTA
+    const int n_s1 = 8 * p.a;
+    const bool is_s1 = (int)blockIdx.x < n_s1;
+    const int grp = is_s1 ? (int)blockIdx.x % 8 : ((int)blockIdx.x - n_s1) % 8;
+    const int first = is_s1 ? (int)blockIdx.x / 8 : ((int)blockIdx.x - n_s1) / 8;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kSlots; ++s) {
-            mbar_init(smem_u32(&bar_full[s]), 1);
+        for (int s = 0; s < kQuads; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), kProdWarps);   // four loads, one per producer warp
             mbar_init(smem_u32(&bar_empty[s]), 1);
         }
-        mbar_init(smem_u32(&bar_acc_full), 1);
-        mbar_init(smem_u32(&bar_acc_empty), 4);
+        for (int h = 0; h < 2; ++h) {
+            mbar_init(smem_u32(&bar_acc_full[h]), 1);
+            mbar_init(smem_u32(&bar_acc_empty[h]), kEpiWarps);
+        }
+        mbar_init(smem_u32(&bar_w), 1);
+        for (int k = 0; k < kStages; ++k) {
+            mbar_init(smem_u32(&bar_st_full[k]), 4);    // the four warps of an epilogue half
+            mbar_init(smem_u32(&bar_st_free[k]), 1);
+        }
         fence_mbar_init();
         dead = 0;
-        tma_prefetch_desc(&tm_x);
-        tma_prefetch_desc(&tm_R);
-        tma_prefetch_desc(&tm_L);
+        dep_items = 0;
+        tma_prefetch_desc(is_s1 ? &tm_x : &tm_L);
+        tma_prefetch_desc(is_s1 ? &tm_R : &tm_y);
+        if (is_s1) tma_prefetch_desc(&tm_u);
     }
     if (warp == 0) {
         tmem_alloc(smem_u32(&tmem_base_s), 512);
@@ -133,166 +431,14 @@ fused_fwd_m64_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
-    const long long stride = gridDim.x;
 
-    if (warp == 4) {
-        // ------------------------------------------------------------ producer
-        if (lane == 0) {
-            uint32_t cnt = 0;
-            bool ok = true;
-            for (long long pos = blockIdx.x; ok; pos += stride) {
-                const Item it = item_at(p, pos);
-                if (it.kind < 0) break;
-                if (it.kind == 1 && p.mode == 2) {
-                    // wait until all S1 items of this tile have published their part of u'
-                    const unsigned *ctr = p.counters + it.tile;
-                    const unsigned long long t0 = global_timer_ns();
-                    while (ld_acquire(ctr) < kS1Arrivals) {
-                        if (*(volatile int *)&dead || global_timer_ns() - t0 > kWaitLimitNs) {
-                            dead = 1;
-                            atomicCAS(p.status, 0u, (unsigned)kErrPeerWait);
-                            ok = false;
-                            break;
-                        }
-                    }
-                    if (!ok) break;
-                    fence_proxy_async_global();
-                }
-                const int nblk = it.kind == 0 ? 8 : 16;
-                for (int b = 0; b < nblk; ++b, ++cnt) {
-                    const int s = cnt % kSlots;
-                    if (!mbar_wait(smem_u32(&bar_empty[s]), ((cnt / kSlots) & 1) ^ 1, p.status, &dead,
-                                   kErrSlotWait)) { ok = false; break; }
-                    const uint32_t a = smem0 + s * kSlotBytes, w = a + kSlotB;
-                    const uint32_t full = smem_u32(&bar_full[s]);
-                    if (it.kind == 0) {
-                        const int k = it.sub * 8 + b;
-                        mbar_expect_tx(full, 16384 + 8192);
-                        tma_load_2d(a, &tm_x, k * kM, it.tile * 128, full);
-                        tma_load_2d(w, &tm_R, 0, k * kM, full);
-                    } else {
-                        const int half = it.sub >> 2, h = it.sub & 3;
-                        const int j = h * 16 + b;
-                        const long long tile64 = (long long)it.tile * 2 + half;
-                        mbar_expect_tx(full, 8192 + 8192);
-                        bulk_load(a, p.u + (tile64 * 64 + j) * 4096, 8192, full);
-                        tma_load_2d(w, &tm_L, 0, j * kM, full);
-                    }
-                }
-                if (ok && it.kind == 1 && p.mode == 2) {
-                    // the last S2 item of a tile to get here clears the tile's counter for the next call
-                    const unsigned old = atomicAdd(p.counters + it.tile, 1u);
-                    if (old + 1 == kS1Arrivals + kS2Items) atomicExch(p.counters + it.tile, 0u);
-                }
-            }
-        }
-    } else if (warp == 5) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc1 = make_idesc_bf16(128, 64, 0, 0);
-            constexpr uint32_t idesc2 = make_idesc_bf16(64, 64, 0, 0);
-            uint32_t cnt = 0, nitem = 0;
-            bool ok = true;
-            for (long long pos = blockIdx.x; ok; pos += stride, ++nitem) {
-                const Item it = item_at(p, pos);
-                if (it.kind < 0) break;
-                if (!mbar_wait(smem_u32(&bar_acc_empty), (nitem & 1) ^ 1, p.status, &dead, kErrTmemWait)) break;
-                tc_fence_after();
-                const int nblk = it.kind == 0 ? 8 : 16;
-                for (int b = 0; b < nblk; ++b, ++cnt) {
-                    const int s = cnt % kSlots;
-                    if (!mbar_wait(smem_u32(&bar_full[s]), (cnt / kSlots) & 1, p.status, &dead, kErrTmaWait)) {
-                        ok = false;
-                        break;
-                    }
-                    tc_fence_after();
-                    const uint32_t a = smem0 + s * kSlotBytes, w = a + kSlotB;
-                    if (it.kind == 0) {
-#pragma unroll
-                        for (int ks = 0; ks < 4; ++ks)
-                            mma_f16_ss(tmem_base + b * 64, make_smem_desc(a + ks * 32, 16, 1024, kSwizzle128),
-                                       make_smem_desc(w + ks * 32, 16, 1024, kSwizzle128), idesc1, ks != 0);
-                    } else {
-                        // accumulators 0-7 in lanes [0,16) of each sub-partition, 8-15 in lanes [16,32)
-                        const uint32_t d = tmem_base + ((uint32_t)((b >> 3) * 16) << 16) + (b & 7) * 64;
-#pragma unroll
-                        for (int ks = 0; ks < 4; ++ks)
-                            mma_f16_ss(d, make_smem_desc(a + ks * 2048, 1024, 128, 0),
-                                       make_smem_desc(w + ks * 32, 16, 1024, kSwizzle128), idesc2, ks != 0);
-                    }
-                    mma_commit(smem_u32(&bar_empty[s]));
-                }
-                if (ok) mma_commit(smem_u32(&bar_acc_full));
-            }
-        }
-    } else {
-        // ------------------------------------------------------------ epilogue (warps 0-3)
-        const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
-        uint32_t nitem = 0;
-        for (long long pos = blockIdx.x;; pos += stride, ++nitem) {
-            const Item it = item_at(p, pos);
-            if (it.kind < 0) break;
-            if (!mbar_wait(smem_u32(&bar_acc_full), nitem & 1, p.status, &dead, kErrMmaWait)) break;
-            tc_fence_after();
-            if (it.kind == 0) {
-                const int r = warp * 32 + lane;
-                const long long tile64 = (long long)it.tile * 2 + (r >> 6);
-                uint8_t *dst = reinterpret_cast<uint8_t *>(p.u) + (tile64 * 64) * 8192 + it.sub * 1024 + (r & 63) * 16;
-#pragma unroll 1
-                for (int jc = 0; jc < 8; ++jc) {
-                    uint32_t v[8][8];
-#pragma unroll
-                    for (int kb = 0; kb < 8; ++kb) tmem_ld8(lane_base + kb * 64 + jc * 8, v[kb]);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        uint4 o;
-                        o.x = pack_bf16(__uint_as_float(v[0][q]), __uint_as_float(v[1][q]));
-                        o.y = pack_bf16(__uint_as_float(v[2][q]), __uint_as_float(v[3][q]));
-                        o.z = pack_bf16(__uint_as_float(v[4][q]), __uint_as_float(v[5][q]));
-                        o.w = pack_bf16(__uint_as_float(v[6][q]), __uint_as_float(v[7][q]));
-                        *reinterpret_cast<uint4 *>(dst + (size_t)(jc * 8 + q) * 8192) = o;
-                    }
-                }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty));
-                if (p.mode == 2) {
-                    // publish: the stores above must be visible to other SMs' bulk copies
-                    fence_proxy_async_global();
-                    __threadfence();
-                    __syncwarp();
-                    if (lane == 0) atomicAdd(p.counters + it.tile, 1u);
-                }
-            } else {
-                const int half = it.sub >> 2, h = it.sub & 3;
-                const long long t = (long long)it.tile * 128 + half * 64 + warp * 16 + (lane & 15);
-                uint8_t *dst = reinterpret_cast<uint8_t *>(p.y) + (size_t)t * (kN * 2) + h * 32 + (lane >> 4) * 16;
-                const bool live = t < p.tokens;
-#pragma unroll 1
-                for (int lc = 0; lc < 8; ++lc) {
-                    uint32_t v[8][8];
-#pragma unroll
-                    for (int a = 0; a < 8; ++a) tmem_ld8(lane_base + a * 64 + lc * 8, v[a]);
-                    tmem_ld_wait();
-                    if (live) {
-#pragma unroll
-                        for (int q = 0; q < 8; ++q) {
-                            uint4 o;
-                            o.x = pack_bf16(__uint_as_float(v[0][q]), __uint_as_float(v[1][q]));
-                            o.y = pack_bf16(__uint_as_float(v[2][q]), __uint_as_float(v[3][q]));
-                            o.z = pack_bf16(__uint_as_float(v[4][q]), __uint_as_float(v[5][q]));
-                            o.w = pack_bf16(__uint_as_float(v[6][q]), __uint_as_float(v[7][q]));
-                            *reinterpret_cast<uint4 *>(dst + (lc * 8 + q) * 128) = o;
-                        }
-                    }
-                }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty));
-            }
-        }
-    }
+    if (is_s1)
+        role_body<true>(tm_x, tm_R, tm_L, tm_u, tm_y, p, smem0, bar_full, bar_empty, bar_acc_full, bar_acc_empty, &bar_w,
+                        bar_st_full, bar_st_free, &dep_items, tmem_base, &dead, grp, first, p.a);
+    else
+        role_body<false>(tm_x, tm_R, tm_L, tm_u, tm_y, p, smem0, bar_full, bar_empty, bar_acc_full, bar_acc_empty, &bar_w,
+                         bar_st_full, bar_st_free, &dep_items, tmem_base, &dead, grp, first, p.b);
+
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem_base, 512);
@@ -303,34 +449,37 @@ size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
 }  // namespace
 }  // namespace tc
 
-// Workspace: [status 256 B][tile counters, 64 KB][u' exchange buffer, tokens rounded up to 128].
+// Workspace: [status 256 B][tile counters, 64 KB][u' exchange buffer, tokens rounded up to 64].
 constexpr size_t kFusedCounterBytes = 65536;
 
 size_t fused_fwd_m64_workspace_bytes(int64_t tokens)
 {
-    const size_t tiles = (size_t)((tokens + 127) / 128);
-    return MONARCH_STATUS_BYTES + kFusedCounterBytes + tc::align256(tiles * 128 * (size_t)tc::kN * 2);
+    const size_t tiles = (size_t)((tokens + 63) / 64);
+    return MONARCH_STATUS_BYTES + kFusedCounterBytes + tc::align256(tiles * 64 * (size_t)tc::kN * 2);
 }
 
 int fused_fwd_m64(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws,
-                  int mode, cudaStream_t s)
+                  cudaStream_t s)
 {
     using namespace tc;
     if (tokens == 0) return MONARCH_OK;
-    const long long tiles = (tokens + 127) / 128;
+    const long long tiles = (tokens + 63) / 64;
     if (tiles * 4 > (long long)kFusedCounterBytes) return MONARCH_ERR_UNSUPPORTED;
-    CUtensorMap tm_x, tm_R, tm_L;
-    MONARCH_TRY(encode_tmap_2d(&tm_x, x, (uint64_t)tokens, kN, kN * 2, 128, 64, 128));
+    CUtensorMap tm_x, tm_R, tm_L, tm_u, tm_y;
+    MONARCH_TRY(encode_tmap_2d(&tm_x, x, (uint64_t)tokens, kN, kN * 2, 64, 64, 128));
     MONARCH_TRY(encode_tmap_2d(&tm_R, R, kN, kM, kM * 2, 64, 64, 128));
-    MONARCH_TRY(encode_tmap_2d(&tm_L, L, kN, kM, kM * 2, 64, 64, 128));
-    FwdParams p;
-    p.status = (unsigned *)ws;
-    p.counters = (unsigned *)((char *)ws + MONARCH_STATUS_BYTES);
-    p.u = (__nv_bfloat16 *)((char *)ws + MONARCH_STATUS_BYTES + kFusedCounterBytes);
-    p.y = (__nv_bfloat16 *)y;
-    p.tokens = tokens;
-    p.tiles = (int)tiles;
-    p.lag = 24;
+    MONARCH_TRY(encode_tmap_2d(&tm_L, L, kN, kM, kM * 2, 32, 64, 128));
+    void *u = (char *)ws + MONARCH_STATUS_BYTES + kFusedCounterBytes;
+    {
+        // exchange buffer as 8-byte words [tile*64 + j][k/8][128]; a store moves 8 rows (j) of one k/8
+        const uint64_t dims[3] = {128, 8, (uint64_t)tiles * 64}, strides[2] = {1024, 8192};
+        const uint32_t box[3] = {128, 1, 8};
+        MONARCH_TRY(encode_tmap_nd(&tm_u, u, 8, 3, dims, strides, box));
+        // y as [l][t][j] bf16; a store moves 16 j x 64 t x 4 l
+        const uint64_t ydims[3] = {64, (uint64_t)tokens, 64}, ystrides[2] = {(uint64_t)kN * 2, 128};
+        const uint32_t ybox[3] = {16, 64, 4};
+        MONARCH_TRY(encode_tmap_nd(&tm_y, y, 2, 3, ydims, ystrides, ybox));
+    }
     static int sms = 0;
     if (!sms) {
         int dev = 0;
@@ -339,18 +488,36 @@ int fused_fwd_m64(const void *x, const void *L, const void *R, void *y, int64_t 
         MONARCH_CUDA_TRY(cudaFuncSetAttribute(fused_fwd_m64_kernel,
                                               cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
     }
-    auto launch = [&](int m) -> int {
-        p.mode = m;
-        const long long items = m == 2 ? tiles * 16 : tiles * 8;
-        const unsigned grid = (unsigned)(items < sms ? items : sms);
-        fused_fwd_m64_kernel<<<grid, kThreads, kSmemBytes, s>>>(tm_x, tm_R, tm_L, p);
-        note_launch();
-        MONARCH_CUDA_TRY(cudaGetLastError());
-        return MONARCH_OK;
-    };
-    if (mode == 2) return launch(2);
-    MONARCH_TRY(launch(0));
-    return launch(1);
+    FwdParams p;
+    p.status = (unsigned *)ws;
+    p.counters = (unsigned *)((char *)ws + MONARCH_STATUS_BYTES);
+    p.u = (__nv_bfloat16 *)u;
+    p.y = (__nv_bfloat16 *)y;
+    p.tokens = tokens;
+    p.tiles = (int)tiles;
+    // split the SMs between the stages: 8 R groups x a CTAs + 8 L groups x b CTAs.  Stage 2 issues
+    // twice the MMAs (N = 32) and writes 32-byte pieces, so it gets about 60 % of the SMs.
+    int a = (sms * 2 + 20) / 40;
+    if (a < 1) a = 1;
+    int b = (sms - 8 * a) / 8;
+    if (b < 1) b = 1;
+    if (a > tiles) a = (int)tiles;
+    if (b > tiles) b = (int)tiles;
+    p.a = a;
+    p.b = b;
+    p.trace = nullptr;
+#ifdef MONARCH_TRACE
+    if (const char *e = getenv("MONARCH_TRACE_OFFSET")) p.trace = (long long *)((char *)ws + atoll(e));
+    if (const char *e = getenv("MONARCH_TRACE_PTR")) p.trace = (long long *)strtoull(e, nullptr, 0);
+    if (const char *e = getenv("MONARCH_SPLIT_A")) { p.a = atoi(e); p.b = (sms - 8 * p.a) / 8; }
+    if (const char *e = getenv("MONARCH_SPLIT_B")) p.b = atoi(e);
+    if (p.a > tiles) p.a = (int)tiles;
+    if (p.b > tiles) p.b = (int)tiles;
+#endif
+    fused_fwd_m64_kernel<<<8 * p.a + 8 * p.b, kThreads, kSmemBytes, s>>>(tm_x, tm_R, tm_L, tm_u, tm_y, p);
+    note_launch();
+    MONARCH_CUDA_TRY(cudaGetLastError());
+    return MONARCH_OK;
 }
 
 }  // namespace monarch

@@ -67,18 +67,8 @@ enum Family { kSimt = 0, kFused = 1, kTcStaged = 2, kNone = -1 };
 // true when the fused tensor-core family has a kernel for (op, m, dtype)
 bool fused_available(int op, int m, int dtype)
 {
-    return dtype == MONARCH_BF16 && m == 64 && op == MONARCH_OP_FWD;
-}
-
-// Development switch: MONARCH_FUSED_MODE=0 runs the fused forward as one launch per stage.
-int fused_mode()
-{
-    static int mode = -1;
-    if (mode < 0) {
-        const char *e = getenv("MONARCH_FUSED_MODE");
-        mode = (e && e[0] == '0') ? 0 : 2;
-    }
-    return mode;
+    static const bool off = getenv("MONARCH_NO_FUSED") != nullptr;   // comparison runs: stage chain instead
+    return !off && dtype == MONARCH_BF16 && m == 64 && op == MONARCH_OP_FWD;
 }
 
 // true when the call can run as a chain of tensor-core stages through the workspace
@@ -127,7 +117,7 @@ int monarch_fwd(const void *x, const void *L, const void *R, void *y, int64_t to
     MONARCH_TRY(check_buffers(in, 3, out, 1, workspace, workspace_bytes,
                               monarch_workspace_bytes(MONARCH_OP_FWD, tokens, n, m, dtype)));
     if (which == kFused)
-        return fused_fwd_m64(x, L, R, y, tokens, workspace, fused_mode(), (cudaStream_t)stream);
+        return fused_fwd_m64(x, L, R, y, tokens, workspace, (cudaStream_t)stream);
     if (which == kTcStaged) return tc_staged_fwd(x, L, R, y, tokens, m, workspace, (cudaStream_t)stream);
     return staged_fwd(x, L, R, y, tokens, m, dtype, workspace, (cudaStream_t)stream);
 }

@@ -192,6 +192,13 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8])
                  : "r"(taddr)
                  : "memory");
 }
+__device__ __forceinline__ void tmem_ld4(uint32_t taddr, uint32_t (&r)[4])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(taddr)
+                 : "memory");
+}
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
 {
     asm volatile(
@@ -268,6 +275,11 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 int encode_tmap_2d(CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols,
                    uint64_t row_stride_bytes, uint32_t box_rows, uint32_t box_cols,
                    uint32_t swizzle_bytes);
+
+// General form: `rank` dimensions (innermost first) of `elem_bytes`-wide elements (2 = bf16,
+// 8 = opaque 64-bit words), strides in bytes for dimensions 1..rank-1, no swizzle.
+int encode_tmap_nd(CUtensorMap *out, const void *base, int elem_bytes, int rank, const uint64_t *dims,
+                   const uint64_t *strides_bytes, const uint32_t *box);
 
 }  // namespace tc
 }  // namespace monarch

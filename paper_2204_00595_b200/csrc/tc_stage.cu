@@ -202,22 +202,31 @@ size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
 }  // namespace
 
 // ---- host: tensor-map encoder through the driver entry point (no link-time libcuda) ----
-int encode_tmap_2d(CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols,
-                   uint64_t row_stride_bytes, uint32_t box_rows, uint32_t box_cols,
-                   uint32_t swizzle_bytes)
+typedef CUresult (*tmap_encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                   CUtensorMapFloatOOBfill);
+
+static int tmap_encoder(tmap_encode_fn *out)
 {
-    typedef CUresult (*encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
-                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
-                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-    static encode_fn fn = nullptr;
+    static tmap_encode_fn fn = nullptr;
     if (!fn) {
         void *p = nullptr;
         cudaDriverEntryPointQueryResult q;
         MONARCH_CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q));
         if (!p || q != cudaDriverEntryPointSuccess) return MONARCH_ERR_CUDA;
-        fn = (encode_fn)p;
+        fn = (tmap_encode_fn)p;
     }
+    *out = fn;
+    return MONARCH_OK;
+}
+
+int encode_tmap_2d(CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols,
+                   uint64_t row_stride_bytes, uint32_t box_rows, uint32_t box_cols,
+                   uint32_t swizzle_bytes)
+{
+    tmap_encode_fn fn;
+    MONARCH_TRY(tmap_encoder(&fn));
     const cuuint64_t dims[2] = {cols, rows};
     const cuuint64_t strides[1] = {row_stride_bytes};
     const cuuint32_t box[2] = {box_cols, box_rows};
@@ -229,6 +238,25 @@ int encode_tmap_2d(CUtensorMap *out, const void *base, uint64_t rows, uint64_t c
     const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims,
                           strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? MONARCH_OK : MONARCH_ERR_CUDA;
+}
+
+int encode_tmap_nd(CUtensorMap *out, const void *base, int elem_bytes, int rank, const uint64_t *dims,
+                   const uint64_t *strides_bytes, const uint32_t *box)
+{
+    tmap_encode_fn fn;
+    MONARCH_TRY(tmap_encoder(&fn));
+    if (rank < 1 || rank > 5) return MONARCH_ERR_INVALID_ARG;
+    cuuint64_t d[5], st[4];
+    cuuint32_t b[5], es[5];
+    for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; es[i] = 1; }
+    for (int i = 0; i + 1 < rank; ++i) st[i] = strides_bytes[i];
+    const CUtensorMapDataType dt = elem_bytes == 8 ? CU_TENSOR_MAP_DATA_TYPE_UINT64
+                                 : elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_UINT32
+                                                   : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    const CUresult r = fn(out, dt, (cuuint32_t)rank, const_cast<void *>(base), d, st, b, es,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                          CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? MONARCH_OK : MONARCH_ERR_CUDA;
 }
 
