@@ -68,4 +68,9 @@ size_t fused_fwd_m64_workspace_bytes(int64_t tokens);
 int fused_fwd_m64(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws,
                   cudaStream_t s);
 
+// ---- fused single-pass dx = M^T dy for m = 64, bf16 (fused_m64_bwd.cu) ----
+size_t fused_bwd_dx_m64_workspace_bytes(int64_t tokens);
+int fused_bwd_dx_m64(const void *dy, const void *L, const void *R, void *dx, int64_t tokens, void *ws,
+                     cudaStream_t s);
+
 }  // namespace monarch

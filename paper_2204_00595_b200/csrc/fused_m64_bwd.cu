@@ -1,0 +1,587 @@
+// Fused dx = M^T dy = R^T P L^T P dy for m = 64 (n = 4096), bf16 in/out, fp32 accumulation in TMEM.
+//
+// The mirror image of the fused forward kernel: one persistent launch, CTAs (one per SM) specialise in
+// one of the two adjoint stages, 64-token tiles, tcgen05.mma with M = 64, two tiles in flight per CTA,
+// the intermediate du handed over through an L2-resident exchange buffer that already has the operand
+// layout of the consumer, outputs leaving through shared-memory staging and TMA tensor stores.
+//
+//   B1 CTAs (4 x 2 groups (hj, hk) of `b1` CTAs): du[t][k][j] = sum_l L[j][l][k] dy[t][l*64+j] for blocks
+//       j in [16hj, 16hj+16) and columns k in [32hk, 32hk+32).  The outer permutation sits on the INPUT
+//       side here: block j needs column j of every 64-element row segment.  TMA fetches the 32-byte
+//       pieces dy[t][l][16hj..16hj+16) (whole sectors) as [64 t][16 l][16 j] chunks (32B swizzle, so that
+//       8 rows l of one token spread over all banks); four warps turn each chunk into K-major operand
+//       slices [j][l/8][t][l%8] with ldmatrix.trans / stmatrix (an 8x8 16-bit transpose per instruction
+//       pair) - the only place in the library where the permutation costs a pass over shared memory.  MMAs (N = 32) run K-step by K-step as slices arrive; L_j is used
+//       transposed straight from its row-major tile (MN-major descriptor, 64B swizzle).  The epilogue
+//       writes the 16 bytes du[t][k][8jc..8jc+8) per (t, k) into the exchange buffer
+//       [tile][k][j/8][t%64][j%8].
+//   B2 CTAs (8 groups g of `b2` CTAs): dx[t][k*64+i] = sum_j R[k][j][i] du[t][k][j] for blocks
+//       k in [8g, 8g+8).  One 8 KB bulk copy per block fetches du_k[64 x 64]; R_k is used transposed
+//       from its row-major tile (MN-major, 128B swizzle); the result rows are 128 contiguous bytes per
+//       (t, k), staged with the 128B swizzle and stored as 64 x 64 boxes.
+//
+// Waits are bounded; B1 waits on nothing outside its CTA, B2 on a per-tile counter bumped by B1.
+#include <cstdlib>
+
+#include "tc_common.cuh"
+
+namespace monarch {
+namespace tc {
+namespace {
+
+constexpr int kM = 64;
+constexpr int kN = kM * kM;
+// warps: 0-7 epilogue, 8 control/loads, 9 MMA, 10-11 store threads, 12-15 transposers (B1) / loaders (B2)
+constexpr int kEpiWarps = 8, kCtlWarp = 8, kMmaWarp = 9, kStoreWarp0 = 10, kAuxWarp0 = 12;
+constexpr int kThreads = 16 * 32;
+constexpr int kWBytes = 65536;                 // resident weights
+constexpr int kStageBytes = 8192;
+constexpr int kB1StagesPerHalf = 2, kB2StagesPerHalf = 4;
+constexpr int kRawBytes = 32768;                              // B1: one K-step (16 l) of 16 blocks, as loaded
+constexpr int kBlockSlice = 2048 + 16;                        // B1: one block's K-step operand, padded so that
+constexpr int kSliceBytes = 16 * kBlockSlice;                 //     the 8 rows of an stmatrix hit 8 bank groups
+constexpr int kSlotBytes = 8192, kSlots = 12, kQuads = 3;     // B2 operand ring
+constexpr int kSmemBytes = kWBytes + 65536 + 98304 + 512 + 1024;   // 224.5 KB (+ alignment) covers both kinds
+static_assert(kWBytes + 2 * kB1StagesPerHalf * kStageBytes + 2 * kRawBytes + 2 * kSliceBytes + 1024 <= kSmemBytes, "B1");
+static_assert(kWBytes + 2 * kB2StagesPerHalf * kStageBytes + kSlots * kSlotBytes + 1024 <= kSmemBytes, "B2");
+constexpr unsigned kB1Arrivals = 8 * 2;        // 8 B1 groups x 2 store threads per tile
+constexpr unsigned kB2Groups = 8;
+
+struct BwdParams {
+    __nv_bfloat16 *du;         // exchange buffer [tiles][64 k][8][64 t][8] bf16
+    unsigned *counters;        // one per 64-token tile, zero between calls
+    unsigned *status;
+    long long tokens;
+    int tiles;
+    int b1, b2;                // CTAs per B1 group, per B2 group
+};
+
+struct Bars {
+    uint64_t w;                               // resident weights landed
+    uint64_t acc_full[2], acc_empty[2];       // TMEM accumulator sets
+    uint64_t st_full[8], st_free[8];          // staging buffers (per half: B1 uses 2, B2 uses 4)
+    uint64_t raw_full[2], raw_empty[2];       // B1 raw chunks
+    uint64_t a_full[2], a_empty[2];           // B1 operand slices
+    uint64_t full[kQuads], empty[kQuads];     // B2 operand ring, groups of four slots
+};
+
+__device__ __forceinline__ unsigned ld_acquire(const unsigned *p)
+{
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void fence_proxy_async_global()
+{
+    asm volatile("fence.proxy.async.global;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+        "l"(src), "r"(bytes), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *m, int x, int y, int z, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
+        "l"(m), "r"(bar), "r"(x), "r"(y), "r"(z)
+        : "memory");
+}
+__device__ __forceinline__ bool wait_fast(uint32_t bar, uint32_t parity, unsigned *status, volatile int *dead,
+                                          unsigned code)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait(bar, parity, status, dead, code);
+}
+// bounded spin on a monotonic shared counter
+__device__ __forceinline__ bool wait_count(volatile int *ctr, int need, unsigned *status, volatile int *dead)
+{
+    if (*ctr >= need) return true;
+    const unsigned long long t0 = global_timer_ns();
+    while (*ctr < need) {
+        if (*dead || global_timer_ns() - t0 > kWaitLimitNs) {
+            *dead = 1;
+            atomicCAS(status, 0u, (unsigned)kErrPeerWait);
+            return false;
+        }
+    }
+    return true;
+}
+
+// Store thread shared by both kinds: sends staged chunks out with TMA tensor stores, keeps NST-1 of them
+// in flight, and (B1) publishes a tile once its stores are complete.
+template <bool B1, int NST, typename IssueFn>
+__device__ __forceinline__ void store_thread(const BwdParams &p, Bars *bars, uint32_t stage0, int sub, int first,
+                                             int step, volatile int *dead, IssueFn issue)
+{
+    const uint32_t my_stage = stage0 + sub * NST * kStageBytes;
+    const uint32_t stf0 = smem_u32(bars->st_full) + sub * NST * 8;
+    const uint32_t stfree0 = smem_u32(bars->st_free) + sub * NST * 8;
+    uint32_t nchunk = 0;
+    int pending = -1;
+    for (int tile = first; tile < p.tiles; tile += step) {
+#pragma unroll 1
+        for (int c = sub; c < 8; c += 2, ++nchunk) {
+            const uint32_t k = nchunk & (NST - 1);
+            if (!wait_fast(stf0 + k * 8, (nchunk / NST) & 1, p.status, dead, kErrMmaWait)) return;
+            issue(my_stage + k * kStageBytes, tile, c);
+            tma_store_commit();
+            if (nchunk >= NST - 1) {
+                tma_store_wait_read<NST - 1>();
+                mbar_arrive(stfree0 + ((nchunk - (NST - 1)) & (NST - 1)) * 8);
+            }
+        }
+        if (B1) {
+            if (pending >= 0) {
+                // the previous tile's four stores are complete once at most four newer ones are pending
+                asm volatile("cp.async.bulk.wait_group 4;" ::: "memory");
+                fence_proxy_async_global();
+                __threadfence();
+                atomicAdd(p.counters + pending, 1u);
+            }
+            pending = tile;
+        }
+    }
+    tma_store_wait_all<0>();
+    if (B1 && pending >= 0) {
+        fence_proxy_async_global();
+        __threadfence();
+        atomicAdd(p.counters + pending, 1u);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ B1
+__device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtensorMap &tm_Lt, const CUtensorMap &tm_du,
+                                        const BwdParams &p, uint32_t smem0, Bars *bars, uint32_t tmem_base,
+                                        volatile int *dead, int grp, int first)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int hj = grp >> 1, hk = grp & 1;
+    const int step = p.b1;
+    if (first >= p.tiles) return;
+    const uint32_t stage0 = smem0 + kWBytes;
+    const uint32_t raw0 = stage0 + 2 * kB1StagesPerHalf * kStageBytes;
+    const uint32_t a0 = raw0 + 2 * kRawBytes;
+    const uint32_t rawf = smem_u32(bars->raw_full), rawe = smem_u32(bars->raw_empty);
+    const uint32_t af = smem_u32(bars->a_full), ae = smem_u32(bars->a_empty);
+    const uint32_t accf0 = smem_u32(bars->acc_full), acce0 = smem_u32(bars->acc_empty);
+
+    if (warp == kCtlWarp) {
+        if (lane != 0) return;
+        // resident: columns [32hk, 32hk+32) of the 16 blocks L_j, row-major [l][k] with 64B swizzle
+        const uint32_t wbar = smem_u32(&bars->w);
+        mbar_expect_tx(wbar, kWBytes);
+        for (int b = 0; b < 16; ++b) tma_load_2d(smem0 + b * 4096, &tm_Lt, hk * 32, (hj * 16 + b) * kM, wbar);
+        uint32_t n = 0;
+        for (int tile = first; tile < p.tiles; tile += step) {
+#pragma unroll 1
+            for (int ks = 0; ks < 4; ++ks, ++n) {
+                const uint32_t rb = n & 1;
+                if (!wait_fast(rawe + rb * 8, ((n >> 1) & 1) ^ 1, p.status, dead, kErrSlotWait)) return;
+                mbar_expect_tx(rawf + rb * 8, kRawBytes);
+                tma_load_3d(raw0 + rb * kRawBytes, &tm_dy3, hj * 16, ks * 16, tile * 64, rawf + rb * 8);
+            }
+        }
+    } else if (warp >= kAuxWarp0) {
+        // transposers: raw [64 t][16 l][16 j] (16-byte halves swapped where bit 2 of l is set)
+        //           ->  slices [16 j][2 l/8][64 t][8 l]
+        const int tw = warp - kAuxWarp0;
+        const int mi = lane >> 3, r = lane & 7;      // matrix of the x4 group, row within it
+        const int lo = mi >> 1, jo = mi & 1;
+        uint32_t n = 0;
+        for (int tile = first; tile < p.tiles; tile += step) {
+#pragma unroll 1
+            for (int ks = 0; ks < 4; ++ks, ++n) {
+                const uint32_t rb = n & 1;
+                if (!wait_fast(rawf + rb * 8, (n >> 1) & 1, p.status, dead, kErrTmaWait)) return;
+                if (!wait_fast(ae + rb * 8, ((n >> 1) & 1) ^ 1, p.status, dead, kErrSlotWait)) return;
+                const uint32_t src = raw0 + rb * kRawBytes + (lo * 8 + r) * 32 + ((jo ^ (r >> 2)) * 16);
+                const uint32_t dst = a0 + rb * kSliceBytes + (jo * 8 + r) * kBlockSlice + lo * 1024;
+#pragma unroll 4
+                for (int tt = 0; tt < 16; ++tt) {
+                    const int t = tw * 16 + tt;
+                    uint32_t m0, m1, m2, m3;
+                    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(m0), "=r"(m1), "=r"(m2), "=r"(m3)
+                                 : "r"(src + t * 512)
+                                 : "memory");
+                    asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1, %2, %3, %4};" ::"r"(dst + t * 16),
+                                 "r"(m0), "r"(m1), "r"(m2), "r"(m3)
+                                 : "memory");
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(rawe + rb * 8);
+                    mbar_arrive(af + rb * 8);
+                }
+            }
+        }
+    } else if (warp == kMmaWarp) {
+        if (lane != 0) return;
+        if (!mbar_wait(smem_u32(&bars->w), 0, p.status, dead, kErrTmaWait)) return;
+        tc_fence_after();
+        constexpr uint32_t idesc = make_idesc_bf16(64, 32, 0, 1);          // B = L_j^T: MN-major
+        const uint64_t a_ns = make_smem_desc(0, 1024, 128, 0);
+        const uint64_t b_mn = make_smem_desc(0, 16, 512, kSwizzle64) | (uint64_t)(smem0 >> 4);
+        uint32_t n = 0, nitem = 0;
+        for (int tile = first; tile < p.tiles; tile += step, ++nitem) {
+            const uint32_t buf = nitem & 1, par = (nitem >> 1) & 1;
+            if (!wait_fast(acce0 + buf * 8, par ^ 1, p.status, dead, kErrTmemWait)) return;
+            tc_fence_after();
+            const uint32_t dbase = tmem_base + buf * 256;
+#pragma unroll 1
+            for (int ks = 0; ks < 4; ++ks, ++n) {
+                const uint32_t ab = n & 1;
+                if (!wait_fast(af + ab * 8, (n >> 1) & 1, p.status, dead, kErrTmaWait)) return;
+                tc_fence_after();
+                const uint64_t as = a_ns | (uint64_t)((a0 + ab * kSliceBytes) >> 4);
+                const uint64_t bs = b_mn + ks * 64;                           // 16 rows of 64 B
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const uint32_t d = dbase + ((uint32_t)((j >> 3) * 16) << 16) + (j & 7) * 32;
+                    mma_f16_ss(d, as + j * (kBlockSlice >> 4), bs + j * 256, idesc, ks != 0);
+                }
+                mma_commit(ae + ab * 8);
+            }
+            mma_commit(accf0 + buf * 8);
+        }
+    } else if (warp < kEpiWarps) {
+        const int q4 = warp & 3, sub = warp >> 2;
+        const uint32_t lane_base = tmem_base + ((uint32_t)(q4 * 32) << 16);
+        const int row = q4 * 16 + (lane & 15);
+        constexpr int NST = kB1StagesPerHalf;
+        const uint32_t my_stage = stage0 + sub * NST * kStageBytes;
+        const uint32_t stf0 = smem_u32(bars->st_full) + sub * NST * 8;
+        const uint32_t stfree0 = smem_u32(bars->st_free) + sub * NST * 8;
+        uint32_t nitem = 0, nchunk = 0;
+        for (int tile = first; tile < p.tiles; tile += step, ++nitem) {
+            const uint32_t buf = nitem & 1, par = (nitem >> 1) & 1;
+            if (!wait_fast(accf0 + buf * 8, par, p.status, dead, kErrMmaWait)) return;
+            tc_fence_after();
+#pragma unroll 1
+            for (int c = sub; c < 8; c += 2, ++nchunk) {
+                const uint32_t k = nchunk & (NST - 1);
+                const uint32_t sbuf = my_stage + k * kStageBytes;
+                if (!wait_fast(stfree0 + k * 8, ((nchunk / NST) & 1) ^ 1, p.status, dead, kErrSlotWait)) return;
+                // chunk = 4 consecutive columns k; lanes i and i+16 hold blocks j 0-7 and 8-15
+                uint32_t v[8][4];
+#pragma unroll
+                for (int a = 0; a < 8; ++a) tmem_ld4(lane_base + buf * 256 + a * 32 + c * 4, v[a]);
+                tmem_ld_wait();
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const uint32_t o0 = pack_bf16(__uint_as_float(v[0][q]), __uint_as_float(v[1][q]));
+                    const uint32_t o1 = pack_bf16(__uint_as_float(v[2][q]), __uint_as_float(v[3][q]));
+                    const uint32_t o2 = pack_bf16(__uint_as_float(v[4][q]), __uint_as_float(v[5][q]));
+                    const uint32_t o3 = pack_bf16(__uint_as_float(v[6][q]), __uint_as_float(v[7][q]));
+                    // staging [k local 4][j/8 local 2][t 64][8 j]
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sbuf + q * 2048 + (lane >> 4) * 1024 + row * 16),
+                                 "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
+                }
+                if (c + 2 >= 8) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(acce0 + buf * 8);
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(stf0 + k * 8);
+            }
+        }
+    } else if (warp >= kStoreWarp0 && warp < kStoreWarp0 + 2) {
+        if (lane != 0) return;
+        const int sub = warp - kStoreWarp0;
+        store_thread<true, kB1StagesPerHalf>(p, bars, stage0, sub, first, step, dead,
+            [&](uint32_t sbuf, int tile, int c) {
+                // du as 8-byte words [tile*64 + k][j/8][128]: 4 rows k x 2 j/8 x 1 KB
+                asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(&tm_du),
+                             "r"(sbuf), "r"(0), "r"(2 * hj), "r"(tile * 64 + hk * 32 + c * 4) : "memory");
+            });
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ B2
+__device__ __forceinline__ void b2_body(const CUtensorMap &tm_R, const CUtensorMap &tm_dx, const BwdParams &p,
+                                        uint32_t smem0, Bars *bars, volatile int *dep_items, uint32_t tmem_base,
+                                        volatile int *dead, int grp, int first)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int step = p.b2;
+    if (first >= p.tiles) return;
+    const uint32_t stage0 = smem0 + kWBytes;
+    const uint32_t ring0 = stage0 + 2 * kB2StagesPerHalf * kStageBytes;
+    const uint32_t full0 = smem_u32(bars->full), empty0 = smem_u32(bars->empty);
+    const uint32_t accf0 = smem_u32(bars->acc_full), acce0 = smem_u32(bars->acc_empty);
+
+    if (warp == kCtlWarp) {
+        if (lane != 0) return;
+        // resident: the 8 blocks R_k, row-major [j][i] with 128B swizzle
+        const uint32_t wbar = smem_u32(&bars->w);
+        mbar_expect_tx(wbar, kWBytes);
+        for (int b = 0; b < 8; ++b) tma_load_2d(smem0 + b * 8192, &tm_R, 0, (grp * 8 + b) * kM, wbar);
+        int nitem = 0;
+        for (int tile = first; tile < p.tiles; tile += step, ++nitem) {
+            // wait until all B1 groups have published their part of du for this tile
+            const unsigned *ctr = p.counters + tile;
+            if (ld_acquire(ctr) < kB1Arrivals) {
+                const unsigned long long t0 = global_timer_ns();
+                while (ld_acquire(ctr) < kB1Arrivals) {
+                    if (*dead || global_timer_ns() - t0 > kWaitLimitNs) {
+                        *dead = 1;
+                        atomicCAS(p.status, 0u, (unsigned)kErrPeerWait);
+                        return;
+                    }
+                }
+            }
+            // the last B2 group to get here clears the tile's counter for the next call
+            const unsigned old = atomicAdd(p.counters + tile, 1u);
+            if (old + 1 == kB1Arrivals + kB2Groups) atomicExch(p.counters + tile, 0u);
+            fence_proxy_async_global();
+            __threadfence_block();
+            *dep_items = nitem + 1;
+        }
+    } else if (warp >= kAuxWarp0) {
+        // loaders: warp pw fetches slot pw of every group of four
+        if (lane != 0) return;
+        const int pw = warp - kAuxWarp0;
+        int quad = 0, nitem = 0;
+        uint32_t phase = 0;
+        for (int tile = first; tile < p.tiles; tile += step, ++nitem) {
+            if (!wait_count(dep_items, nitem + 1, p.status, dead)) return;
+            __threadfence_block();
+            fence_proxy_async_global();
+            const __nv_bfloat16 *src = p.du + ((long long)tile * 64 + grp * 8 + pw) * 4096;
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                int g = quad + q;
+                uint32_t ph = phase;
+                if (g >= kQuads) { g -= kQuads; ph ^= 1; }
+                if (!wait_fast(empty0 + g * 8, ph ^ 1, p.status, dead, kErrSlotWait)) return;
+                mbar_expect_tx(full0 + g * 8, kSlotBytes);
+                bulk_load(ring0 + (g * 4 + pw) * kSlotBytes, src + (size_t)q * 4 * 4096, 8192, full0 + g * 8);
+            }
+            quad += 2;
+            if (quad >= kQuads) { quad -= kQuads; phase ^= 1; }
+        }
+    } else if (warp == kMmaWarp) {
+        if (lane != 0) return;
+        if (!mbar_wait(smem_u32(&bars->w), 0, p.status, dead, kErrTmaWait)) return;
+        tc_fence_after();
+        constexpr uint32_t idesc = make_idesc_bf16(64, 64, 0, 1);          // B = R_k^T: MN-major
+        const uint64_t a_ring = make_smem_desc(0, 1024, 128, 0) | (uint64_t)(ring0 >> 4);
+        const uint64_t b_mn = make_smem_desc(0, 16, 1024, kSwizzle128) | (uint64_t)(smem0 >> 4);
+        int quad = 0;
+        uint32_t phase = 0, nitem = 0;
+        for (int tile = first; tile < p.tiles; tile += step, ++nitem) {
+            const uint32_t buf = nitem & 1, par = (nitem >> 1) & 1;
+            if (!wait_fast(acce0 + buf * 8, par ^ 1, p.status, dead, kErrTmemWait)) return;
+            tc_fence_after();
+            const uint32_t dbase = tmem_base + ((buf * 16) << 16);
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                int g = quad + q;
+                uint32_t ph = phase;
+                if (g >= kQuads) { g -= kQuads; ph ^= 1; }
+                if (!wait_fast(full0 + g * 8, ph, p.status, dead, kErrTmaWait)) return;
+                tc_fence_after();
+                const uint64_t aq = a_ring + (uint64_t)(g * 4 * (kSlotBytes >> 4));
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int b = q * 4 + i;
+                    const uint64_t ad = aq + i * (kSlotBytes >> 4);
+                    const uint64_t bd = b_mn + b * 512;
+                    const uint32_t d = dbase + b * 64;
+                    mma_f16_ss(d, ad, bd, idesc, 0);
+                    mma_f16_ss(d, ad + 128, bd + 128, idesc, 1);             // 16 rows of 128 B per K-step
+                    mma_f16_ss(d, ad + 256, bd + 256, idesc, 1);
+                    mma_f16_ss(d, ad + 384, bd + 384, idesc, 1);
+                }
+                mma_commit(empty0 + g * 8);
+            }
+            mma_commit(accf0 + buf * 8);
+            quad += 2;
+            if (quad >= kQuads) { quad -= kQuads; phase ^= 1; }
+        }
+    } else if (warp < kEpiWarps) {
+        const int q4 = warp & 3, sub = warp >> 2;
+        const uint32_t lane_base = tmem_base + ((uint32_t)(q4 * 32) << 16);
+        const int row = q4 * 16 + (lane & 15);
+        constexpr int NST = kB2StagesPerHalf;
+        const uint32_t my_stage = stage0 + sub * NST * kStageBytes;
+        const uint32_t stf0 = smem_u32(bars->st_full) + sub * NST * 8;
+        const uint32_t stfree0 = smem_u32(bars->st_free) + sub * NST * 8;
+        uint32_t nitem = 0, nchunk = 0;
+        for (int tile = first; tile < p.tiles; tile += step, ++nitem) {
+            const uint32_t buf = nitem & 1, par = (nitem >> 1) & 1;
+            if (!wait_fast(accf0 + buf * 8, par, p.status, dead, kErrMmaWait)) return;
+            tc_fence_after();
+            const bool mine = (uint32_t)(lane >> 4) == buf;
+#pragma unroll 1
+            for (int c = sub; c < 8; c += 2, ++nchunk) {
+                const uint32_t k = nchunk & (NST - 1);
+                const uint32_t sbuf = my_stage + k * kStageBytes;
+                if (!wait_fast(stfree0 + k * 8, ((nchunk / NST) & 1) ^ 1, p.status, dead, kErrSlotWait)) return;
+                // chunk = block c: 64 contiguous outputs dx[t][(8g+c)*64 ..] per token
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t v[2][16];
+                    tmem_ld16(lane_base + c * 64 + h * 32, v[0]);
+                    tmem_ld16(lane_base + c * 64 + h * 32 + 16, v[1]);
+                    tmem_ld_wait();
+                    if (mine) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const uint32_t *w = &v[e >> 1][(e & 1) * 8];
+                            const uint32_t o0 = pack_bf16(__uint_as_float(w[0]), __uint_as_float(w[1]));
+                            const uint32_t o1 = pack_bf16(__uint_as_float(w[2]), __uint_as_float(w[3]));
+                            const uint32_t o2 = pack_bf16(__uint_as_float(w[4]), __uint_as_float(w[5]));
+                            const uint32_t o3 = pack_bf16(__uint_as_float(w[6]), __uint_as_float(w[7]));
+                            const int ch = h * 4 + e;                          // 16-byte chunk of the 128-byte row
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sbuf + row * 128 + ((ch ^ (row & 7)) * 16)),
+                                         "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
+                        }
+                    }
+                }
+                if (c + 2 >= 8) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(acce0 + buf * 8);
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(stf0 + k * 8);
+            }
+        }
+    } else if (warp >= kStoreWarp0 && warp < kStoreWarp0 + 2) {
+        if (lane != 0) return;
+        const int sub = warp - kStoreWarp0;
+        store_thread<false, kB2StagesPerHalf>(p, bars, stage0, sub, first, step, dead,
+            [&](uint32_t sbuf, int tile, int c) { tma_store_2d(&tm_dx, sbuf, (grp * 8 + c) * kM, tile * 64); });
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+fused_bwd_dx_m64_kernel(const __grid_constant__ CUtensorMap tm_dy3, const __grid_constant__ CUtensorMap tm_Lt,
+                        const __grid_constant__ CUtensorMap tm_R, const __grid_constant__ CUtensorMap tm_du,
+                        const __grid_constant__ CUtensorMap tm_dx, const BwdParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) Bars bars;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int dead;
+    __shared__ int dep_items;
+
+    const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int warp = threadIdx.x >> 5;
+    const int n_b1 = 8 * p.b1;
+    const bool is_b1 = (int)blockIdx.x < n_b1;
+    const int grp = is_b1 ? (int)blockIdx.x % 8 : ((int)blockIdx.x - n_b1) % 8;
+    const int first = is_b1 ? (int)blockIdx.x / 8 : ((int)blockIdx.x - n_b1) / 8;
+
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bars.w), 1);
+        for (int h = 0; h < 2; ++h) {
+            mbar_init(smem_u32(&bars.acc_full[h]), 1);
+            mbar_init(smem_u32(&bars.acc_empty[h]), kEpiWarps);
+            mbar_init(smem_u32(&bars.raw_full[h]), 1);
+            mbar_init(smem_u32(&bars.raw_empty[h]), 4);      // the four transposer warps
+            mbar_init(smem_u32(&bars.a_full[h]), 4);
+            mbar_init(smem_u32(&bars.a_empty[h]), 1);
+        }
+        for (int k = 0; k < 8; ++k) {
+            mbar_init(smem_u32(&bars.st_full[k]), 4);        // the four warps of an epilogue half
+            mbar_init(smem_u32(&bars.st_free[k]), 1);
+        }
+        for (int q = 0; q < kQuads; ++q) {
+            mbar_init(smem_u32(&bars.full[q]), 4);           // four loads, one per loader warp
+            mbar_init(smem_u32(&bars.empty[q]), 1);
+        }
+        fence_mbar_init();
+        dead = 0;
+        dep_items = 0;
+        if (is_b1) { tma_prefetch_desc(&tm_dy3); tma_prefetch_desc(&tm_Lt); tma_prefetch_desc(&tm_du); }
+        else { tma_prefetch_desc(&tm_R); tma_prefetch_desc(&tm_dx); }
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&tmem_base_s), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+
+    if (is_b1) b1_body(tm_dy3, tm_Lt, tm_du, p, smem0, &bars, tmem_base, &dead, grp, first);
+    else b2_body(tm_R, tm_dx, p, smem0, &bars, &dep_items, tmem_base, &dead, grp, first);
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem_base, 512);
+}
+
+}  // namespace
+}  // namespace tc
+
+constexpr size_t kBwdCounterBytes = 65536;
+
+size_t fused_bwd_dx_m64_workspace_bytes(int64_t tokens)
+{
+    const size_t tiles = (size_t)((tokens + 63) / 64);
+    return MONARCH_STATUS_BYTES + kBwdCounterBytes + ((tiles * 64 * (size_t)tc::kN * 2 + 255) & ~(size_t)255);
+}
+
+int fused_bwd_dx_m64(const void *dy, const void *L, const void *R, void *dx, int64_t tokens, void *ws,
+                     cudaStream_t s)
+{
+    using namespace tc;
+    if (tokens == 0) return MONARCH_OK;
+    const long long tiles = (tokens + 63) / 64;
+    if (tiles * 4 > (long long)kBwdCounterBytes) return MONARCH_ERR_UNSUPPORTED;
+    void *du = (char *)ws + MONARCH_STATUS_BYTES + kBwdCounterBytes;
+    CUtensorMap tm_dy3, tm_Lt, tm_R, tm_du, tm_dx;
+    {
+        // dy as [t][l][j]: a load brings 16 j x 16 l x 64 t (32-byte pieces)
+        const uint64_t dims[3] = {64, 64, (uint64_t)tokens}, strides[2] = {128, (uint64_t)kN * 2};
+        const uint32_t box[3] = {16, 16, 64};
+        MONARCH_TRY(encode_tmap_nd(&tm_dy3, dy, 2, 3, dims, strides, box, 32));
+        // exchange buffer as 8-byte words [tile*64 + k][j/8][128]; a store moves 4 k x 2 j/8 x 1 KB
+        const uint64_t udims[3] = {128, 8, (uint64_t)tiles * 64}, ustrides[2] = {1024, 8192};
+        const uint32_t ubox[3] = {128, 2, 4};
+        MONARCH_TRY(encode_tmap_nd(&tm_du, du, 8, 3, udims, ustrides, ubox));
+    }
+    MONARCH_TRY(encode_tmap_2d(&tm_Lt, L, kN, kM, kM * 2, 64, 32, 64));      // [64 l][32 k] per block, 64B swizzle
+    MONARCH_TRY(encode_tmap_2d(&tm_R, R, kN, kM, kM * 2, 64, 64, 128));
+    MONARCH_TRY(encode_tmap_2d(&tm_dx, dx, (uint64_t)tokens, kN, kN * 2, 64, 64, 128));
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        MONARCH_CUDA_TRY(cudaGetDevice(&dev));
+        MONARCH_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        MONARCH_CUDA_TRY(cudaFuncSetAttribute(fused_bwd_dx_m64_kernel,
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+    }
+    BwdParams p;
+    p.status = (unsigned *)ws;
+    p.counters = (unsigned *)((char *)ws + MONARCH_STATUS_BYTES);
+    p.du = (__nv_bfloat16 *)du;
+    p.tokens = tokens;
+    p.tiles = (int)tiles;
+    // B1 issues twice the MMAs (N = 32) and transposes its input: about 60 % of the SMs
+    int b1 = (sms * 3 + 20) / 40;
+    if (b1 < 1) b1 = 1;
+    int b2 = (sms - 8 * b1) / 8;
+    if (b2 < 1) b2 = 1;
+    if (b1 > tiles) b1 = (int)tiles;
+    if (b2 > tiles) b2 = (int)tiles;
+    p.b1 = b1;
+    p.b2 = b2;
+    fused_bwd_dx_m64_kernel<<<8 * b1 + 8 * b2, kThreads, kSmemBytes, s>>>(tm_dy3, tm_Lt, tm_R, tm_du, tm_dx, p);
+    note_launch();
+    MONARCH_CUDA_TRY(cudaGetLastError());
+    return MONARCH_OK;
+}
+
+}  // namespace monarch

@@ -242,7 +242,7 @@ int encode_tmap_2d(CUtensorMap *out, const void *base, uint64_t rows, uint64_t c
 }
 
 int encode_tmap_nd(CUtensorMap *out, const void *base, int elem_bytes, int rank, const uint64_t *dims,
-                   const uint64_t *strides_bytes, const uint32_t *box)
+                   const uint64_t *strides_bytes, const uint32_t *box, uint32_t swizzle_bytes)
 {
     tmap_encode_fn fn;
     MONARCH_TRY(tmap_encoder(&fn));
@@ -255,7 +255,8 @@ int encode_tmap_nd(CUtensorMap *out, const void *base, int elem_bytes, int rank,
                                  : elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_UINT32
                                                    : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     const CUresult r = fn(out, dt, (cuuint32_t)rank, const_cast<void *>(base), d, st, b, es,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          swizzle_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE,
                           CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? MONARCH_OK : MONARCH_ERR_CUDA;
 }
