@@ -67,10 +67,21 @@ int tc_staged_mlp_fwd(const void *x, const void *L1, const void *R1, const void 
 size_t fused_fwd_m64_workspace_bytes(int64_t tokens);
 int fused_fwd_m64(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws,
                   cudaStream_t s);
+// first stage only: u = P R x in the exchange layout [tile][j][k/8][t%64][k%8] (tokens rounded up to 64)
+int fused_fwd_m64_stage1(const void *x, const void *R, void *u, int64_t tokens, unsigned *status,
+                         cudaStream_t s);
 
 // ---- fused single-pass dx = M^T dy for m = 64, bf16 (fused_m64_bwd.cu) ----
 size_t fused_bwd_dx_m64_workspace_bytes(int64_t tokens);
 int fused_bwd_dx_m64(const void *dy, const void *L, const void *R, void *dx, int64_t tokens, void *ws,
                      cudaStream_t s);
+// first stage only: du as [tile][k][j/8][t%64][j%8] and P dy as [tile][j][l/8][t%64][l%8]
+int fused_bwd_m64_stage1(const void *dy, const void *L, void *du, void *dyp, int64_t tokens,
+                         unsigned *status, cudaStream_t s);
+
+// ---- weight gradients for m = 64, bf16 (fused_m64_bwd_dw.cu) ----
+size_t fused_bwd_dw_m64_workspace_bytes(int64_t tokens);
+int fused_bwd_dw_m64(const void *x, const void *dy, const void *L, const void *R, float *dL, float *dR,
+                     int accumulate, int64_t tokens, void *ws, cudaStream_t s);
 
 }  // namespace monarch

@@ -361,7 +361,7 @@ __device__ __forceinline__ void role_body(const CUtensorMap &tm_x, const CUtenso
                     mbar_arrive(stfree0 + ((nchunk - (kStagesPerHalf - 1)) & (kStagesPerHalf - 1)) * 8);
                 }
             }
-            if (S1) {
+            if (S1 && p.b > 0) {      // no stage-2 CTAs in the launch: nothing to publish to
                 if (pending >= 0) {
                     // the previous tile's four stores are complete once at most four newer ones are pending
                     asm volatile("cp.async.bulk.wait_group 4;" ::: "memory");
@@ -373,7 +373,7 @@ __device__ __forceinline__ void role_body(const CUtensorMap &tm_x, const CUtenso
             }
         }
         tma_store_wait_all<0>();
-        if (S1 && pending >= 0) {
+        if (S1 && p.b > 0 && pending >= 0) {
             fence_proxy_async_global();
             __threadfence();
             atomicAdd(p.counters + pending, 1u);
@@ -458,27 +458,34 @@ size_t fused_fwd_m64_workspace_bytes(int64_t tokens)
     return MONARCH_STATUS_BYTES + kFusedCounterBytes + tc::align256(tiles * 64 * (size_t)tc::kN * 2);
 }
 
-int fused_fwd_m64(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws,
-                  cudaStream_t s)
+namespace {
+// Launch with both stages (y != null) or with stage-1 CTAs only, which leaves P R x in `u` in the
+// exchange layout [tile][j][k/8][t%64][k%8] for another kernel to consume.
+int launch_fwd_m64(const void *x, const void *L, const void *R, void *y, void *u, unsigned *counters,
+                   unsigned *status, int64_t tokens, cudaStream_t s)
 {
     using namespace tc;
-    if (tokens == 0) return MONARCH_OK;
+    const bool both = y != nullptr;
     const long long tiles = (tokens + 63) / 64;
     if (tiles * 4 > (long long)kFusedCounterBytes) return MONARCH_ERR_UNSUPPORTED;
     CUtensorMap tm_x, tm_R, tm_L, tm_u, tm_y;
     MONARCH_TRY(encode_tmap_2d(&tm_x, x, (uint64_t)tokens, kN, kN * 2, 64, 64, 128));
     MONARCH_TRY(encode_tmap_2d(&tm_R, R, kN, kM, kM * 2, 64, 64, 128));
-    MONARCH_TRY(encode_tmap_2d(&tm_L, L, kN, kM, kM * 2, 32, 64, 128));
-    void *u = (char *)ws + MONARCH_STATUS_BYTES + kFusedCounterBytes;
     {
         // exchange buffer as 8-byte words [tile*64 + j][k/8][128]; a store moves 8 rows (j) of one k/8
         const uint64_t dims[3] = {128, 8, (uint64_t)tiles * 64}, strides[2] = {1024, 8192};
         const uint32_t box[3] = {128, 1, 8};
         MONARCH_TRY(encode_tmap_nd(&tm_u, u, 8, 3, dims, strides, box));
+    }
+    if (both) {
+        MONARCH_TRY(encode_tmap_2d(&tm_L, L, kN, kM, kM * 2, 32, 64, 128));
         // y as [l][t][j] bf16; a store moves 16 j x 64 t x 4 l
         const uint64_t ydims[3] = {64, (uint64_t)tokens, 64}, ystrides[2] = {(uint64_t)kN * 2, 128};
         const uint32_t ybox[3] = {16, 64, 4};
         MONARCH_TRY(encode_tmap_nd(&tm_y, y, 2, 3, ydims, ystrides, ybox));
+    } else {
+        tm_L = tm_R;
+        tm_y = tm_u;
     }
     static int sms = 0;
     if (!sms) {
@@ -489,35 +496,52 @@ int fused_fwd_m64(const void *x, const void *L, const void *R, void *y, int64_t 
                                               cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
     }
     FwdParams p;
-    p.status = (unsigned *)ws;
-    p.counters = (unsigned *)((char *)ws + MONARCH_STATUS_BYTES);
+    p.status = status;
+    p.counters = counters;
     p.u = (__nv_bfloat16 *)u;
     p.y = (__nv_bfloat16 *)y;
     p.tokens = tokens;
     p.tiles = (int)tiles;
     // split the SMs between the stages: 8 R groups x a CTAs + 8 L groups x b CTAs.  Stage 2 issues
     // twice the MMAs (N = 32) and writes 32-byte pieces, so it gets about 60 % of the SMs.
-    int a = (sms * 2 + 20) / 40;
+    int a = both ? (sms * 2 + 20) / 40 : sms / 8;
     if (a < 1) a = 1;
-    int b = (sms - 8 * a) / 8;
-    if (b < 1) b = 1;
+    int b = both ? (sms - 8 * a) / 8 : 0;
+    if (both && b < 1) b = 1;
     if (a > tiles) a = (int)tiles;
     if (b > tiles) b = (int)tiles;
     p.a = a;
     p.b = b;
     p.trace = nullptr;
 #ifdef MONARCH_TRACE
-    if (const char *e = getenv("MONARCH_TRACE_OFFSET")) p.trace = (long long *)((char *)ws + atoll(e));
-    if (const char *e = getenv("MONARCH_TRACE_PTR")) p.trace = (long long *)strtoull(e, nullptr, 0);
-    if (const char *e = getenv("MONARCH_SPLIT_A")) { p.a = atoi(e); p.b = (sms - 8 * p.a) / 8; }
-    if (const char *e = getenv("MONARCH_SPLIT_B")) p.b = atoi(e);
-    if (p.a > tiles) p.a = (int)tiles;
-    if (p.b > tiles) p.b = (int)tiles;
+    if (both) {
+        if (const char *e = getenv("MONARCH_TRACE_PTR")) p.trace = (long long *)strtoull(e, nullptr, 0);
+        if (const char *e = getenv("MONARCH_SPLIT_A")) { p.a = atoi(e); p.b = (sms - 8 * p.a) / 8; }
+        if (const char *e = getenv("MONARCH_SPLIT_B")) p.b = atoi(e);
+        if (p.a > tiles) p.a = (int)tiles;
+        if (p.b > tiles) p.b = (int)tiles;
+    }
 #endif
     fused_fwd_m64_kernel<<<8 * p.a + 8 * p.b, kThreads, kSmemBytes, s>>>(tm_x, tm_R, tm_L, tm_u, tm_y, p);
     note_launch();
     MONARCH_CUDA_TRY(cudaGetLastError());
     return MONARCH_OK;
+}
+}  // namespace
+
+int fused_fwd_m64(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws,
+                  cudaStream_t s)
+{
+    if (tokens == 0) return MONARCH_OK;
+    return launch_fwd_m64(x, L, R, y, (char *)ws + MONARCH_STATUS_BYTES + kFusedCounterBytes,
+                          (unsigned *)((char *)ws + MONARCH_STATUS_BYTES), (unsigned *)ws, tokens, s);
+}
+
+int fused_fwd_m64_stage1(const void *x, const void *R, void *u, int64_t tokens, unsigned *status,
+                         cudaStream_t s)
+{
+    if (tokens == 0) return MONARCH_OK;
+    return launch_fwd_m64(x, nullptr, R, nullptr, u, nullptr, status, tokens, s);
 }
 
 }  // namespace monarch

@@ -31,9 +31,10 @@ namespace {
 
 constexpr int kM = 64;
 constexpr int kN = kM * kM;
-// warps: 0-7 epilogue, 8 control/loads, 9 MMA, 10-11 store threads, 12-15 transposers (B1) / loaders (B2)
-constexpr int kEpiWarps = 8, kCtlWarp = 8, kMmaWarp = 9, kStoreWarp0 = 10, kAuxWarp0 = 12;
-constexpr int kThreads = 16 * 32;
+// warps: 0-7 epilogue, 8 control/loads, 9 MMA, 10-11 store threads, 12-15 transposers (B1) / loaders (B2),
+// 16 writes the transposed dy out when a caller wants it (B1)
+constexpr int kEpiWarps = 8, kCtlWarp = 8, kMmaWarp = 9, kStoreWarp0 = 10, kAuxWarp0 = 12, kDypWarp = 16;
+constexpr int kThreads = 17 * 32;
 constexpr int kWBytes = 65536;                 // resident weights
 constexpr int kStageBytes = 8192;
 constexpr int kB1StagesPerHalf = 2, kB2StagesPerHalf = 4;
@@ -49,6 +50,7 @@ constexpr unsigned kB2Groups = 8;
 
 struct BwdParams {
     __nv_bfloat16 *du;         // exchange buffer [tiles][64 k][8][64 t][8] bf16
+    __nv_bfloat16 *dyp;        // optional: P dy in the layout [tiles][64 j][8][64 t][8] (l = 8 * chunk + l%8)
     unsigned *counters;        // one per 64-token tile, zero between calls
     unsigned *status;
     long long tokens;
@@ -133,7 +135,7 @@ __device__ __forceinline__ void store_thread(const BwdParams &p, Bars *bars, uin
                 mbar_arrive(stfree0 + ((nchunk - (NST - 1)) & (NST - 1)) * 8);
             }
         }
-        if (B1) {
+        if (B1 && p.b2 > 0) {     // no B2 CTAs in the launch: nothing to publish to
             if (pending >= 0) {
                 // the previous tile's four stores are complete once at most four newer ones are pending
                 asm volatile("cp.async.bulk.wait_group 4;" ::: "memory");
@@ -145,7 +147,7 @@ __device__ __forceinline__ void store_thread(const BwdParams &p, Bars *bars, uin
         }
     }
     tma_store_wait_all<0>();
-    if (B1 && pending >= 0) {
+    if (B1 && p.b2 > 0 && pending >= 0) {
         fence_proxy_async_global();
         __threadfence();
         atomicAdd(p.counters + pending, 1u);
@@ -184,7 +186,7 @@ __device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtenso
                 tma_load_3d(raw0 + rb * kRawBytes, &tm_dy3, hj * 16, ks * 16, tile * 64, rawf + rb * 8);
             }
         }
-    } else if (warp >= kAuxWarp0) {
+    } else if (warp >= kAuxWarp0 && warp < kAuxWarp0 + 4) {
         // transposers: raw [64 t][16 l][16 j] (16-byte halves swapped where bit 2 of l is set)
         //           ->  slices [16 j][2 l/8][64 t][8 l]
         const int tw = warp - kAuxWarp0;
@@ -219,6 +221,26 @@ __device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtenso
                 }
             }
         }
+    } else if (warp == kDypWarp) {
+        // the operand slices are P dy in 2 KB runs [l/8 2][t 64][8 l] per block j: copy them out
+        if (lane != 0 || p.dyp == nullptr) return;
+        uint32_t n = 0;
+        for (int tile = first; tile < p.tiles; tile += step) {
+            __nv_bfloat16 *dst = p.dyp + ((long long)tile * 64 + hj * 16) * 4096;
+#pragma unroll 1
+            for (int ks = 0; ks < 4; ++ks, ++n) {
+                const uint32_t ab = n & 1;
+                if (!wait_fast(af + ab * 8, (n >> 1) & 1, p.status, dead, kErrTmaWait)) return;
+#pragma unroll 4
+                for (int j = 0; j < 16; ++j)
+                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst + j * 4096 + ks * 1024),
+                                 "r"(a0 + ab * kSliceBytes + j * kBlockSlice), "r"(2048) : "memory");
+                tma_store_commit();
+                tma_store_wait_read<0>();
+                mbar_arrive(ae + ab * 8);
+            }
+        }
+        tma_store_wait_all<0>();
     } else if (warp == kMmaWarp) {
         if (lane != 0) return;
         if (!mbar_wait(smem_u32(&bars->w), 0, p.status, dead, kErrTmaWait)) return;
@@ -343,7 +365,7 @@ __device__ __forceinline__ void b2_body(const CUtensorMap &tm_R, const CUtensorM
             __threadfence_block();
             *dep_items = nitem + 1;
         }
-    } else if (warp >= kAuxWarp0) {
+    } else if (warp >= kAuxWarp0 && warp < kAuxWarp0 + 4) {
         // loaders: warp pw fetches slot pw of every group of four
         if (lane != 0) return;
         const int pw = warp - kAuxWarp0;
@@ -489,7 +511,7 @@ fused_bwd_dx_m64_kernel(const __grid_constant__ CUtensorMap tm_dy3, const __grid
             mbar_init(smem_u32(&bars.raw_full[h]), 1);
             mbar_init(smem_u32(&bars.raw_empty[h]), 4);      // the four transposer warps
             mbar_init(smem_u32(&bars.a_full[h]), 4);
-            mbar_init(smem_u32(&bars.a_empty[h]), 1);
+            mbar_init(smem_u32(&bars.a_empty[h]), p.dyp ? 2 : 1);   // MMA commit (+ the copy out)
         }
         for (int k = 0; k < 8; ++k) {
             mbar_init(smem_u32(&bars.st_full[k]), 4);        // the four warps of an epilogue half
@@ -533,14 +555,17 @@ size_t fused_bwd_dx_m64_workspace_bytes(int64_t tokens)
     return MONARCH_STATUS_BYTES + kBwdCounterBytes + ((tiles * 64 * (size_t)tc::kN * 2 + 255) & ~(size_t)255);
 }
 
-int fused_bwd_dx_m64(const void *dy, const void *L, const void *R, void *dx, int64_t tokens, void *ws,
-                     cudaStream_t s)
+namespace {
+// Launch with both stages (dx != null) or with B1 CTAs only, which leaves du in the exchange layout
+// [tile][k][j/8][t%64][j%8] (and, if `dyp` is given, P dy as [tile][j][l/8][t%64][l%8]) for another
+// kernel to consume.
+int launch_bwd_m64(const void *dy, const void *L, const void *R, void *dx, void *du, void *dyp,
+                   unsigned *counters, unsigned *status, int64_t tokens, cudaStream_t s)
 {
     using namespace tc;
-    if (tokens == 0) return MONARCH_OK;
+    const bool both = dx != nullptr;
     const long long tiles = (tokens + 63) / 64;
     if (tiles * 4 > (long long)kBwdCounterBytes) return MONARCH_ERR_UNSUPPORTED;
-    void *du = (char *)ws + MONARCH_STATUS_BYTES + kBwdCounterBytes;
     CUtensorMap tm_dy3, tm_Lt, tm_R, tm_du, tm_dx;
     {
         // dy as [t][l][j]: a load brings 16 j x 16 l x 64 t (32-byte pieces)
@@ -553,8 +578,13 @@ int fused_bwd_dx_m64(const void *dy, const void *L, const void *R, void *dx, int
         MONARCH_TRY(encode_tmap_nd(&tm_du, du, 8, 3, udims, ustrides, ubox));
     }
     MONARCH_TRY(encode_tmap_2d(&tm_Lt, L, kN, kM, kM * 2, 64, 32, 64));      // [64 l][32 k] per block, 64B swizzle
-    MONARCH_TRY(encode_tmap_2d(&tm_R, R, kN, kM, kM * 2, 64, 64, 128));
-    MONARCH_TRY(encode_tmap_2d(&tm_dx, dx, (uint64_t)tokens, kN, kN * 2, 64, 64, 128));
+    if (both) {
+        MONARCH_TRY(encode_tmap_2d(&tm_R, R, kN, kM, kM * 2, 64, 64, 128));
+        MONARCH_TRY(encode_tmap_2d(&tm_dx, dx, (uint64_t)tokens, kN, kN * 2, 64, 64, 128));
+    } else {
+        tm_R = tm_Lt;
+        tm_dx = tm_du;
+    }
     static int sms = 0;
     if (!sms) {
         int dev = 0;
@@ -564,16 +594,17 @@ int fused_bwd_dx_m64(const void *dy, const void *L, const void *R, void *dx, int
                                               cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
     }
     BwdParams p;
-    p.status = (unsigned *)ws;
-    p.counters = (unsigned *)((char *)ws + MONARCH_STATUS_BYTES);
+    p.status = status;
+    p.counters = counters;
     p.du = (__nv_bfloat16 *)du;
+    p.dyp = (__nv_bfloat16 *)dyp;
     p.tokens = tokens;
     p.tiles = (int)tiles;
     // B1 issues twice the MMAs (N = 32) and transposes its input: about 60 % of the SMs
-    int b1 = (sms * 3 + 20) / 40;
+    int b1 = both ? (sms * 3 + 20) / 40 : sms / 8;
     if (b1 < 1) b1 = 1;
-    int b2 = (sms - 8 * b1) / 8;
-    if (b2 < 1) b2 = 1;
+    int b2 = both ? (sms - 8 * b1) / 8 : 0;
+    if (both && b2 < 1) b2 = 1;
     if (b1 > tiles) b1 = (int)tiles;
     if (b2 > tiles) b2 = (int)tiles;
     p.b1 = b1;
@@ -582,6 +613,22 @@ int fused_bwd_dx_m64(const void *dy, const void *L, const void *R, void *dx, int
     note_launch();
     MONARCH_CUDA_TRY(cudaGetLastError());
     return MONARCH_OK;
+}
+}  // namespace
+
+int fused_bwd_dx_m64(const void *dy, const void *L, const void *R, void *dx, int64_t tokens, void *ws,
+                     cudaStream_t s)
+{
+    if (tokens == 0) return MONARCH_OK;
+    return launch_bwd_m64(dy, L, R, dx, (char *)ws + MONARCH_STATUS_BYTES + kBwdCounterBytes, nullptr,
+                          (unsigned *)((char *)ws + MONARCH_STATUS_BYTES), (unsigned *)ws, tokens, s);
+}
+
+int fused_bwd_m64_stage1(const void *dy, const void *L, void *du, void *dyp, int64_t tokens,
+                         unsigned *status, cudaStream_t s)
+{
+    if (tokens == 0) return MONARCH_OK;
+    return launch_bwd_m64(dy, L, nullptr, nullptr, du, dyp, nullptr, status, tokens, s);
 }
 
 }  // namespace monarch

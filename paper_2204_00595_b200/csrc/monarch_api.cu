@@ -68,7 +68,7 @@ enum Family { kSimt = 0, kFused = 1, kTcStaged = 2, kNone = -1 };
 bool fused_available(int op, int m, int dtype)
 {
     static const bool off = getenv("MONARCH_NO_FUSED") != nullptr;   // comparison runs: stage chain instead
-    return !off && dtype == MONARCH_BF16 && m == 64 && (op == MONARCH_OP_FWD || op == MONARCH_OP_BWD_DX);
+    return !off && dtype == MONARCH_BF16 && m == 64 && op != MONARCH_OP_MLP_FWD;
 }
 
 // true when the call can run as a chain of tensor-core stages through the workspace
@@ -102,8 +102,9 @@ size_t monarch_workspace_bytes(int op, int64_t tokens, int32_t n, int32_t m, int
     const int which = pick(op, m, dtype);
     if (which < 0) return 0;
     if (which == kFused)
-        return op == MONARCH_OP_FWD ? fused_fwd_m64_workspace_bytes(tokens)
-                                    : fused_bwd_dx_m64_workspace_bytes(tokens);
+        return op == MONARCH_OP_FWD      ? fused_fwd_m64_workspace_bytes(tokens)
+               : op == MONARCH_OP_BWD_DX ? fused_bwd_dx_m64_workspace_bytes(tokens)
+                                         : fused_bwd_dw_m64_workspace_bytes(tokens);
     return staged_workspace_bytes(op, tokens, n, m, dtype);
 }
 
@@ -155,6 +156,8 @@ int monarch_bwd_dw(const void *x, const void *dy, const void *L, const void *R, 
     if (which < 0) return MONARCH_ERR_UNSUPPORTED;
     MONARCH_TRY(check_buffers(in, 4, out, 2, workspace, workspace_bytes,
                               monarch_workspace_bytes(MONARCH_OP_BWD_DW, tokens, n, m, dtype)));
+    if (which == kFused)
+        return fused_bwd_dw_m64(x, dy, L, R, dL, dR, accumulate, tokens, workspace, (cudaStream_t)stream);
     return staged_bwd_dw(x, dy, L, R, dL, dR, accumulate, tokens, m, dtype, workspace,
                          (cudaStream_t)stream);
 }
