@@ -338,8 +338,51 @@ def main():
         "clocks": clocks, "gpu_launches": int(launches), "roofline": roofline, "calls": per_call,
     }
 
-    if rank == 0 and not args.no_e2e:
-        line["e2e"] = None
+    if not args.no_e2e:
+        e2e = None
+        if calls == ["fwd", "bwd_dx", "bwd_dw"]:
+            # the same step through the host-buffer entry point: pinned host tensors in, host tensors
+            # out, uploads and downloads inside the timed region (wall clock around blocking calls)
+            del sets, ws
+            torch.cuda.empty_cache()
+            hx = torch.roll(to_device(d["x"], cfg.dtype), 5 * rank, 0).cpu().pin_memory()
+            hdy = torch.roll(to_device(d["dy"], cfg.dtype), rank, 0).cpu().pin_memory()
+            hL, hR = W["L"].cpu().pin_memory(), W["R"].cpu().pin_memory()
+            hy, hdx = torch.empty_like(hx).pin_memory(), torch.empty_like(hx).pin_memory()
+            hg = torch.empty(2, m, m, m, dtype=torch.float32).pin_memory()
+            ctx = P.HostContext(T, n, m, code)
+
+            def host_step():
+                ctx.fwd_bwd(hx, hdy, hL, hR, hy, hdx, hg[0], hg[1], T)
+                if dist is not None:
+                    grads.copy_(hg, non_blocking=True)
+                    dist.all_reduce(grads)
+                    hg.copy_(grads, non_blocking=True)
+                    torch.cuda.synchronize()
+
+            for _ in range(3):
+                host_step()
+            torch.cuda.synchronize()
+            if dist is not None:
+                dist.barrier()
+            k_e2e = max(1, min(args.steps, 10))
+            t0 = time.perf_counter()
+            for _ in range(k_e2e):
+                host_step()
+            torch.cuda.synchronize()
+            dt = (time.perf_counter() - t0) / k_e2e
+            if dist is not None:
+                tmax = torch.tensor([dt], device="cuda")
+                dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+                dt = float(tmax.item())
+            act = T * n * esize(cfg.dtype)
+            wbytes = n * m * esize(cfg.dtype)
+            e2e = {"value": step_flops * world / dt / 1e12, "unit": unit, "ms_per_step": dt * 1e3,
+                   "h2d_bytes_per_step": 2 * act + 2 * wbytes, "d2h_bytes_per_step": 2 * act + 2 * n * m * 4,
+                   "steps": k_e2e, "api": "monarch_host_fwd_bwd (pinned host tensors, chunked 3-stream staging)",
+                   "timer": "host wall clock around blocking calls"}
+            ctx.close()
+        line["e2e"] = e2e
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         r = time_oracle(cfg, d)
         line["cpu_baseline"] = {"value": r["tflops"], "unit": unit, "cores": r["cores"],

@@ -107,7 +107,8 @@ int monarch_mlp_fwd(const void *x, const void *L1, const void *R1, const void *b
  * for invalid or unsupported arguments. */
 size_t monarch_workspace_bytes(int op, int64_t tokens, int32_t n, int32_t m, int dtype);
 
-/* Zero the status word of a workspace (enqueued on `stream`). */
+/* Zero the status word and the tile counters that follow it (enqueued on
+ * `stream`); call once before the first use of a workspace. */
 int monarch_workspace_init(void *workspace, size_t workspace_bytes, void *stream);
 
 /* Synchronise `stream`, read and clear the status word: MONARCH_OK, or
@@ -128,6 +129,41 @@ const char *monarch_impl_name(int op, int32_t m, int dtype);
 uint64_t monarch_launch_count(void);
 
 const char *monarch_status_string(int status);
+
+/* ---- Host-buffer calls ---------------------------------------------------
+ * For callers whose tensors live in HOST memory.  A context owns the device
+ * buffers (three token chunks of x, dy, y, dx, the weights, dL/dR and a
+ * workspace) and three streams; a call uploads chunk c+1, runs the device
+ * entry points above on chunk c and downloads chunk c-1 concurrently, and
+ * returns after everything has arrived.  The arithmetic is exactly that of
+ * monarch_fwd / monarch_bwd_dx / monarch_bwd_dw (Section 3.3 steps 1-3 and
+ * their adjoints); the paper has no counterpart of the staging itself.
+ *
+ * All data pointers of these calls are HOST pointers owned by the caller
+ * (page-locked memory lets the copies overlap; pageable memory is accepted
+ * and serialises them), layouts and dtypes as above.  The calls block until
+ * the outputs are complete and are not re-entrant on one context.
+ *
+ * monarch_host_create: max_tokens bounds later calls; chunk_tokens is the
+ * staging granularity (a multiple of 64; 0 picks a default).  Allocates
+ * device memory with cudaMalloc on the current device; MONARCH_ERR_CUDA if
+ * that fails, MONARCH_ERR_UNSUPPORTED / MONARCH_ERR_INVALID_ARG for bad
+ * shapes.  monarch_host_destroy frees everything (null is a no-op). */
+typedef struct monarch_host_ctx monarch_host_ctx;
+int monarch_host_create(monarch_host_ctx **out, int64_t max_tokens, int32_t n, int32_t m,
+                        int dtype, int64_t chunk_tokens);
+int monarch_host_destroy(monarch_host_ctx *ctx);
+
+/* y = M x on host buffers ([tokens][n] each; L, R [m][m][m]). */
+int monarch_host_fwd(monarch_host_ctx *ctx, const void *x, const void *L, const void *R,
+                     void *y, int64_t tokens);
+
+/* One training step on host buffers: y = M x, dx = M^T dy, and dL, dR (float32,
+ * overwritten) summed over all tokens.  Returns MONARCH_ERR_TIMEOUT if a
+ * kernel reported an abandoned wait. */
+int monarch_host_fwd_bwd(monarch_host_ctx *ctx, const void *x, const void *dy, const void *L,
+                         const void *R, void *y, void *dx, float *dL, float *dR,
+                         int64_t tokens);
 
 /* Forward pass y = M x for callers that cannot allocate device memory - code running where
  * cudaMalloc is off limits (a real-time or serving loop whose device memory was fixed at

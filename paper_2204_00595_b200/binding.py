@@ -32,6 +32,10 @@ _SIGNATURES = {
     "monarch_launch_count": (ctypes.c_uint64, []),
     "monarch_status_string": (ctypes.c_char_p, [_int]),
     "monarch_fwd_noalloc": (_int, [_vp, _vp, _vp, _vp, _i64, _i32, _i32, _int, _vp]),
+    "monarch_host_create": (_int, [ctypes.POINTER(_vp), _i64, _i32, _i32, _int, _i64]),
+    "monarch_host_destroy": (_int, [_vp]),
+    "monarch_host_fwd": (_int, [_vp, _vp, _vp, _vp, _vp, _i64]),
+    "monarch_host_fwd_bwd": (_int, [_vp] * 9 + [_i64]),
 }
 
 
@@ -203,3 +207,45 @@ def monarch_fwd_noalloc(x, L, R, y, tokens, n, m, stream=None) -> None:
     _check(lib().monarch_fwd_noalloc(_ptr(x, "x"), _ptr(L, "L", dt), _ptr(R, "R", dt),
                                      _ptr(y, "y", dt), tokens, n, m, _dtype_code(x),
                                      _stream(stream)), "monarch_fwd_noalloc")
+
+
+def _hptr(t, name, dtype=None):
+    if t.is_cuda:
+        raise ValueError(f"{name} must be a host tensor")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{name} must have dtype {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+class HostContext:
+    """Device staging for the host-buffer calls (monarch_host_*): tensors are CPU tensors, ideally
+    pinned; every call blocks until its outputs have arrived."""
+
+    def __init__(self, max_tokens: int, n: int, m: int, dtype: int, chunk_tokens: int = 0):
+        h = _vp()
+        _check(lib().monarch_host_create(ctypes.byref(h), max_tokens, n, m, dtype, chunk_tokens),
+               "monarch_host_create")
+        self._h, self.n, self.m, self.dtype = h, n, m, dtype
+
+    def close(self):
+        if self._h:
+            lib().monarch_host_destroy(self._h)
+            self._h = None
+
+    __del__ = close
+
+    def fwd(self, x, L, R, y, tokens: int) -> None:
+        dt = x.dtype
+        _check(lib().monarch_host_fwd(self._h, _hptr(x, "x"), _hptr(L, "L", dt), _hptr(R, "R", dt),
+                                      _hptr(y, "y", dt), tokens), "monarch_host_fwd")
+
+    def fwd_bwd(self, x, dy, L, R, y, dx, dL, dR, tokens: int) -> None:
+        import torch
+        dt = x.dtype
+        _check(lib().monarch_host_fwd_bwd(self._h, _hptr(x, "x"), _hptr(dy, "dy", dt),
+                                          _hptr(L, "L", dt), _hptr(R, "R", dt), _hptr(y, "y", dt),
+                                          _hptr(dx, "dx", dt), _hptr(dL, "dL", torch.float32),
+                                          _hptr(dR, "dR", torch.float32), tokens),
+               "monarch_host_fwd_bwd")
