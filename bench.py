@@ -52,7 +52,7 @@ def esize(dtype):
 
 def call_flops(call, n, m, T):
     """Algorithmic FLOPs: 4 n m per token per pass (two block-diagonal stages of 2 n m each)."""
-    return {"fwd": 4, "bwd_dx": 4, "bwd_dw": 4, "mlp_fwd": 8}[call] * n * m * T
+    return {"fwd": 4, "bwd_dx": 4, "bwd_dw": 4, "bwd": 8, "mlp_fwd": 8}[call] * n * m * T
 
 
 def call_bytes(call, n, m, T, dtype):
@@ -63,6 +63,8 @@ def call_bytes(call, n, m, T, dtype):
         return 2 * T * n * s + w
     if call == "bwd_dw":
         return 2 * T * n * s + w + 2 * n * m * 4
+    if call == "bwd":          # read x, dy; write dx, dL, dR
+        return 3 * T * n * s + w + 2 * n * m * 4
     if call == "mlp_fwd":
         return 2 * T * n * s + 2 * w + 2 * n * s
     raise ValueError(call)
@@ -184,6 +186,10 @@ def main():
     calls = list(cfg.ops)
     if args.calls:
         calls = [k for k in calls if k in args.calls.split(",")]
+    elif calls == ["fwd", "bwd_dx", "bwd_dw"]:
+        # default: the backward pass as one call (dx, dL, dR) that reuses the intermediate the forward
+        # call left in its workspace; --calls fwd,bwd_dx,bwd_dw times the three separate entry points
+        calls = ["fwd", "bwd"]
     n, m, T = cfg.n, cfg.m, cfg.tokens
     workload = (f"workload {cfg.index}: {'+'.join(calls)} {cfg.dtype} n={n} m={m} "
                 f"tokens/GPU={T}")
@@ -251,8 +257,10 @@ def main():
         sets.append(e)
     W = {k: to_device(d[k], cfg.dtype) for k in ("L", "R", "L2", "R2", "b1", "b2") if k in d}
     grads = torch.zeros(2, m, m, m, dtype=torch.float32, device="cuda")   # packed (dL, dR)
-    op_of = {"fwd": P.OP_FWD, "bwd_dx": P.OP_BWD_DX, "bwd_dw": P.OP_BWD_DW, "mlp_fwd": P.OP_MLP_FWD}
-    ws = P.Workspace(max(P.monarch_workspace_bytes(op_of[k], T, n, m, code) for k in calls))
+    op_of = {"fwd": P.OP_FWD, "bwd_dx": P.OP_BWD_DX, "bwd_dw": P.OP_BWD_DW, "mlp_fwd": P.OP_MLP_FWD,
+             "bwd": P.OP_BWD}
+    ws = P.Workspace(max(P.monarch_workspace_bytes(op_of[k], T, n, m, code) for k in calls if k != "bwd"))
+    ws_b = P.Workspace(P.monarch_workspace_bytes(P.OP_BWD, T, n, m, code)) if "bwd" in calls else None
     stream = torch.cuda.current_stream()
 
     ev = {k: [] for k in calls}
@@ -270,6 +278,11 @@ def main():
                 P.monarch_bwd_dx(e["dy"], W["L"], W["R"], e["dx"], T, n, m, ws)
             elif k == "bwd_dw":
                 P.monarch_bwd_dw(e["x"], e["dy"], W["L"], W["R"], grads[0], grads[1], 0, T, n, m, ws)
+                if dist is not None:
+                    dist.all_reduce(grads)
+            elif k == "bwd":
+                P.monarch_bwd(e["x"], e["dy"], W["L"], W["R"], e["dx"], grads[0], grads[1], 0, T, n, m,
+                              ws_b, fwd_workspace=ws)
                 if dist is not None:
                     dist.all_reduce(grads)
             elif k == "mlp_fwd":
@@ -340,10 +353,10 @@ def main():
 
     if not args.no_e2e:
         e2e = None
-        if calls == ["fwd", "bwd_dx", "bwd_dw"]:
+        if "fwd" in calls and ("bwd" in calls or "bwd_dw" in calls):
             # the same step through the host-buffer entry point: pinned host tensors in, host tensors
             # out, uploads and downloads inside the timed region (wall clock around blocking calls)
-            del sets, ws
+            del sets, ws, ws_b
             torch.cuda.empty_cache()
             hx = torch.roll(to_device(d["x"], cfg.dtype), 5 * rank, 0).cpu().pin_memory()
             hdy = torch.roll(to_device(d["dy"], cfg.dtype), rank, 0).cpu().pin_memory()

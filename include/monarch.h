@@ -60,7 +60,8 @@ typedef enum {
     MONARCH_OP_FWD = 0,
     MONARCH_OP_BWD_DX = 1,
     MONARCH_OP_BWD_DW = 2,
-    MONARCH_OP_MLP_FWD = 3
+    MONARCH_OP_MLP_FWD = 3,
+    MONARCH_OP_BWD = 4 /* monarch_bwd: dx, dL and dR in one call */
 } monarch_op_t;
 
 /* Which kernel family serves a call (process-wide; default AUTO). */
@@ -93,6 +94,20 @@ int monarch_bwd_dw(const void *x, const void *dy, const void *L, const void *R,
                    float *dL, float *dR, int accumulate,
                    int64_t tokens, int32_t n, int32_t m, int dtype,
                    void *workspace, size_t workspace_bytes, void *stream);
+
+/* The whole backward pass in one call: dx as in monarch_bwd_dx and dL, dR as in
+ * monarch_bwd_dw, sharing du (and reading dy once).  `fwd_workspace` is either
+ * null or the workspace that monarch_fwd used for the SAME x, L, R, tokens, n,
+ * m, dtype, untouched since that call returned its work to the stream: kernel
+ * families that keep u = P^T R x there in a layout they can read back use it
+ * instead of recomputing u (as an autograd function saves its intermediate);
+ * the others ignore it.  The caller vouches for its contents; a stale buffer
+ * gives a wrong dL, not an error.  `workspace` (monarch_workspace_bytes with
+ * MONARCH_OP_BWD) must not be the same buffer as `fwd_workspace`. */
+int monarch_bwd(const void *x, const void *dy, const void *L, const void *R,
+                const void *fwd_workspace, void *dx, float *dL, float *dR, int accumulate,
+                int64_t tokens, int32_t n, int32_t m, int dtype,
+                void *workspace, size_t workspace_bytes, void *stream);
 
 /* Monarch feed-forward block (Section 4: the FFN weights replaced by Monarch
  * matrices):  y = M2 GELU(M1 x + b1) + b2,  M1 = P L1 P^T R1, M2 = P L2 P^T R2,

@@ -10,7 +10,7 @@ import ctypes
 import os
 
 F32, BF16 = 0, 1
-OP_FWD, OP_BWD_DX, OP_BWD_DW, OP_MLP_FWD = 0, 1, 2, 3
+OP_FWD, OP_BWD_DX, OP_BWD_DW, OP_MLP_FWD, OP_BWD = 0, 1, 2, 3, 4
 IMPL_AUTO, IMPL_STAGED, IMPL_FUSED = 0, 1, 2
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libmonarch.so")
@@ -24,6 +24,7 @@ _SIGNATURES = {
     "monarch_bwd_dw": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _int, _i64, _i32, _i32, _int, _vp,
                               _sz, _vp]),
     "monarch_mlp_fwd": (_int, [_vp] * 8 + [_i64, _i32, _i32, _int, _vp, _sz, _vp]),
+    "monarch_bwd": (_int, [_vp] * 8 + [_int, _i64, _i32, _i32, _int, _vp, _sz, _vp]),
     "monarch_workspace_bytes": (_sz, [_int, _i64, _i32, _i32, _int]),
     "monarch_workspace_init": (_int, [_vp, _sz, _vp]),
     "monarch_last_device_status": (_int, [_vp, _vp]),
@@ -181,6 +182,19 @@ def monarch_bwd_dw(x, dy, L, R, dL, dR, accumulate, tokens, n, m, workspace, str
                                 _ptr(R, "R", dt), _ptr(dL, "dL", torch.float32),
                                 _ptr(dR, "dR", torch.float32), int(accumulate), tokens, n, m,
                                 _dtype_code(x), p, b, _stream(stream)), "monarch_bwd_dw")
+
+
+def monarch_bwd(x, dy, L, R, dx, dL, dR, accumulate, tokens, n, m, workspace, fwd_workspace=None,
+                stream=None) -> None:
+    """dx, dL, dR in one call; fwd_workspace = the Workspace monarch_fwd used for the same x, L, R."""
+    import torch
+    dt = x.dtype
+    p, b = _ws(workspace)
+    fp = _ws(fwd_workspace)[0] if fwd_workspace is not None else None
+    _check(lib().monarch_bwd(_ptr(x, "x"), _ptr(dy, "dy", dt), _ptr(L, "L", dt), _ptr(R, "R", dt), fp,
+                             _ptr(dx, "dx", dt), _ptr(dL, "dL", torch.float32),
+                             _ptr(dR, "dR", torch.float32), int(accumulate), tokens, n, m,
+                             _dtype_code(x), p, b, _stream(stream)), "monarch_bwd")
 
 
 def monarch_mlp_fwd(x, L1, R1, b1, L2, R2, b2, y, tokens, n, m, workspace, stream=None) -> None:

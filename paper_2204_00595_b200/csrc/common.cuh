@@ -79,9 +79,20 @@ int fused_bwd_dx_m64(const void *dy, const void *L, const void *R, void *dx, int
 int fused_bwd_m64_stage1(const void *dy, const void *L, void *du, void *dyp, int64_t tokens,
                          unsigned *status, cudaStream_t s);
 
+// both stages, also leaving du (and P dy if dyp != null) behind for the weight gradients
+int fused_bwd_dx_m64_keep(const void *dy, const void *L, const void *R, void *dx, void *du, void *dyp,
+                          unsigned *counters, unsigned *status, int64_t tokens, cudaStream_t s);
+
 // ---- weight gradients for m = 64, bf16 (fused_m64_bwd_dw.cu) ----
 size_t fused_bwd_dw_m64_workspace_bytes(int64_t tokens);
 int fused_bwd_dw_m64(const void *x, const void *dy, const void *L, const void *R, float *dL, float *dR,
                      int accumulate, int64_t tokens, void *ws, cudaStream_t s);
+// dx, dL, dR in one pass; u_saved (optional) = the exchange buffer a fused forward call left behind
+size_t fused_bwd_m64_workspace_bytes(int64_t tokens);
+int fused_bwd_m64(const void *x, const void *dy, const void *L, const void *R, const void *u_saved,
+                  void *dx, float *dL, float *dR, int accumulate, int64_t tokens, void *ws,
+                  cudaStream_t s);
+// where the fused forward keeps u inside its workspace
+const void *fused_fwd_m64_saved_u(const void *fwd_ws);
 
 }  // namespace monarch

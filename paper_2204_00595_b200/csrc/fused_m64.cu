@@ -157,7 +157,7 @@ __device__ __forceinline__ void role_body(const CUtensorMap &tm_x, const CUtenso
         [[maybe_unused]] int nitem_t = 0;
         for (int tile = first; tile < n_tiles; tile += step, ++nitem_t, ++nitem_p) {
             if (pw == 0) TRACE(0);
-            if (!S1) {
+            if (!S1 && p.a > 0) {      // (a launch without stage-1 CTAs finds u' complete)
                 if (pw == 0) {
                     // wait until all S1 groups have published their part of u' for this tile
                     const unsigned *ctr = p.counters + tile;
@@ -465,19 +465,21 @@ int launch_fwd_m64(const void *x, const void *L, const void *R, void *y, void *u
                    unsigned *status, int64_t tokens, cudaStream_t s)
 {
     using namespace tc;
-    const bool both = y != nullptr;
+    const bool both = y != nullptr && x != nullptr;
+    const bool s2_only = x == nullptr;
     const long long tiles = (tokens + 63) / 64;
     if (tiles * 4 > (long long)kFusedCounterBytes) return MONARCH_ERR_UNSUPPORTED;
     CUtensorMap tm_x, tm_R, tm_L, tm_u, tm_y;
-    MONARCH_TRY(encode_tmap_2d(&tm_x, x, (uint64_t)tokens, kN, kN * 2, 64, 64, 128));
     MONARCH_TRY(encode_tmap_2d(&tm_R, R, kN, kM, kM * 2, 64, 64, 128));
+    if (s2_only) tm_x = tm_R;
+    else MONARCH_TRY(encode_tmap_2d(&tm_x, x, (uint64_t)tokens, kN, kN * 2, 64, 64, 128));
     {
         // exchange buffer as 8-byte words [tile*64 + j][k/8][128]; a store moves 8 rows (j) of one k/8
         const uint64_t dims[3] = {128, 8, (uint64_t)tiles * 64}, strides[2] = {1024, 8192};
         const uint32_t box[3] = {128, 1, 8};
         MONARCH_TRY(encode_tmap_nd(&tm_u, u, 8, 3, dims, strides, box));
     }
-    if (both) {
+    if (both || s2_only) {
         MONARCH_TRY(encode_tmap_2d(&tm_L, L, kN, kM, kM * 2, 32, 64, 128));
         // y as [l][t][j] bf16; a store moves 16 j x 64 t x 4 l
         const uint64_t ydims[3] = {64, (uint64_t)tokens, 64}, ystrides[2] = {(uint64_t)kN * 2, 128};
@@ -510,14 +512,17 @@ int launch_fwd_m64(const void *x, const void *L, const void *R, void *y, void *u
     if (both && b < 1) b = 1;
     if (a > tiles) a = (int)tiles;
     if (b > tiles) b = (int)tiles;
+    if (s2_only) { a = 0; b = sms / 8 < tiles ? sms / 8 : (int)tiles; if (b < 1) b = 1; }
     p.a = a;
     p.b = b;
     p.trace = nullptr;
 #ifdef MONARCH_TRACE
-    if (both) {
+    if (both == (getenv("MONARCH_TRACE_S1ONLY") == nullptr)) {
         if (const char *e = getenv("MONARCH_TRACE_PTR")) p.trace = (long long *)strtoull(e, nullptr, 0);
-        if (const char *e = getenv("MONARCH_SPLIT_A")) { p.a = atoi(e); p.b = (sms - 8 * p.a) / 8; }
-        if (const char *e = getenv("MONARCH_SPLIT_B")) p.b = atoi(e);
+        if (both) {
+            if (const char *e = getenv("MONARCH_SPLIT_A")) { p.a = atoi(e); p.b = (sms - 8 * p.a) / 8; }
+            if (const char *e = getenv("MONARCH_SPLIT_B")) p.b = atoi(e);
+        }
         if (p.a > tiles) p.a = (int)tiles;
         if (p.b > tiles) p.b = (int)tiles;
     }
@@ -533,8 +538,19 @@ int fused_fwd_m64(const void *x, const void *L, const void *R, void *y, int64_t 
                   cudaStream_t s)
 {
     if (tokens == 0) return MONARCH_OK;
+    static const bool two = getenv("MONARCH_TWO_LAUNCH") != nullptr;
+    if (two) {
+        void *u = (char *)ws + MONARCH_STATUS_BYTES + kFusedCounterBytes;
+        MONARCH_TRY(launch_fwd_m64(x, nullptr, R, nullptr, u, nullptr, (unsigned *)ws, tokens, s));
+        return launch_fwd_m64(nullptr, L, R, y, u, nullptr, (unsigned *)ws, tokens, s);
+    }
     return launch_fwd_m64(x, L, R, y, (char *)ws + MONARCH_STATUS_BYTES + kFusedCounterBytes,
                           (unsigned *)((char *)ws + MONARCH_STATUS_BYTES), (unsigned *)ws, tokens, s);
+}
+
+const void *fused_fwd_m64_saved_u(const void *fwd_ws)
+{
+    return (const char *)fwd_ws + MONARCH_STATUS_BYTES + kFusedCounterBytes;
 }
 
 int fused_fwd_m64_stage1(const void *x, const void *R, void *u, int64_t tokens, unsigned *status,

@@ -236,8 +236,12 @@ __device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtenso
                     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst + j * 4096 + ks * 1024),
                                  "r"(a0 + ab * kSliceBytes + j * kBlockSlice), "r"(2048) : "memory");
                 tma_store_commit();
-                tma_store_wait_read<0>();
-                mbar_arrive(ae + ab * 8);
+                // one copy stays in flight: the slice before this one has been read out by now (its
+                // buffer is only needed again after the current slice, which is already transposed)
+                if (n >= 1) {
+                    tma_store_wait_read<1>();
+                    mbar_arrive(ae + (ab ^ 1) * 8);
+                }
             }
         }
         tma_store_wait_all<0>();
@@ -622,6 +626,13 @@ int fused_bwd_dx_m64(const void *dy, const void *L, const void *R, void *dx, int
     if (tokens == 0) return MONARCH_OK;
     return launch_bwd_m64(dy, L, R, dx, (char *)ws + MONARCH_STATUS_BYTES + kBwdCounterBytes, nullptr,
                           (unsigned *)((char *)ws + MONARCH_STATUS_BYTES), (unsigned *)ws, tokens, s);
+}
+
+int fused_bwd_dx_m64_keep(const void *dy, const void *L, const void *R, void *dx, void *du, void *dyp,
+                          unsigned *counters, unsigned *status, int64_t tokens, cudaStream_t s)
+{
+    if (tokens == 0) return MONARCH_OK;
+    return launch_bwd_m64(dy, L, R, dx, du, dyp, counters, status, tokens, s);
 }
 
 int fused_bwd_m64_stage1(const void *dy, const void *L, void *du, void *dyp, int64_t tokens,

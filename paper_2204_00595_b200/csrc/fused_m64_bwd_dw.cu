@@ -197,24 +197,13 @@ size_t fused_bwd_dw_m64_workspace_bytes(int64_t tokens)
     return MONARCH_STATUS_BYTES + kDwCounterBytes + 3 * ((tiles * 64 * (size_t)tc::kN * 2 + 255) & ~(size_t)255);
 }
 
-int fused_bwd_dw_m64(const void *x, const void *dy, const void *L, const void *R, float *dL, float *dR,
-                     int accumulate, int64_t tokens, void *ws, cudaStream_t s)
+namespace {
+// dL, dR += token reduction over the three intermediates
+int launch_dw(const void *x, const void *u, const void *du, const void *dyp, float *dL, float *dR,
+              unsigned *status, int64_t tokens, cudaStream_t s)
 {
     using namespace tc;
-    const size_t gbytes = (size_t)kN * 64 * sizeof(float);
-    if (!accumulate) {
-        MONARCH_CUDA_TRY(cudaMemsetAsync(dL, 0, gbytes, s));
-        MONARCH_CUDA_TRY(cudaMemsetAsync(dR, 0, gbytes, s));
-    }
-    if (tokens == 0) return MONARCH_OK;
     const long long tiles = (tokens + 63) / 64;
-    const size_t ex = ((size_t)tiles * 64 * kN * 2 + 255) & ~(size_t)255;
-    unsigned *status = (unsigned *)ws;
-    char *u = (char *)ws + MONARCH_STATUS_BYTES + kDwCounterBytes;
-    char *du = u + ex, *dyp = du + ex;
-    MONARCH_TRY(fused_fwd_m64_stage1(x, R, u, tokens, status, s));
-    MONARCH_TRY(fused_bwd_m64_stage1(dy, L, du, dyp, tokens, status, s));
-
     CUtensorMap tm_x;
     MONARCH_TRY(encode_tmap_2d(&tm_x, x, (uint64_t)tokens, kN, kN * 2, 64, 64, 128));
     static int sms = 0;
@@ -241,6 +230,61 @@ int fused_bwd_dw_m64(const void *x, const void *dy, const void *L, const void *R
     note_launch();
     MONARCH_CUDA_TRY(cudaGetLastError());
     return MONARCH_OK;
+}
+
+size_t exchange_bytes(int64_t tokens)
+{
+    const size_t tiles = (size_t)((tokens + 63) / 64);
+    return (tiles * 64 * (size_t)tc::kN * 2 + 255) & ~(size_t)255;
+}
+
+int zero_grads(float *dL, float *dR, cudaStream_t s)
+{
+    const size_t gbytes = (size_t)tc::kN * 64 * sizeof(float);
+    MONARCH_CUDA_TRY(cudaMemsetAsync(dL, 0, gbytes, s));
+    MONARCH_CUDA_TRY(cudaMemsetAsync(dR, 0, gbytes, s));
+    return MONARCH_OK;
+}
+}  // namespace
+
+int fused_bwd_dw_m64(const void *x, const void *dy, const void *L, const void *R, float *dL, float *dR,
+                     int accumulate, int64_t tokens, void *ws, cudaStream_t s)
+{
+    if (!accumulate) MONARCH_TRY(zero_grads(dL, dR, s));
+    if (tokens == 0) return MONARCH_OK;
+    const size_t ex = exchange_bytes(tokens);
+    unsigned *status = (unsigned *)ws;
+    char *u = (char *)ws + MONARCH_STATUS_BYTES + kDwCounterBytes;
+    char *du = u + ex, *dyp = du + ex;
+    MONARCH_TRY(fused_fwd_m64_stage1(x, R, u, tokens, status, s));
+    MONARCH_TRY(fused_bwd_m64_stage1(dy, L, du, dyp, tokens, status, s));
+    return launch_dw(x, u, du, dyp, dL, dR, status, tokens, s);
+}
+
+// Workspace: [status 256 B][tile counters 64 KB][du][P dy][u], each tokens (rounded up to 64) x 4096 bf16.
+size_t fused_bwd_m64_workspace_bytes(int64_t tokens)
+{
+    return MONARCH_STATUS_BYTES + kDwCounterBytes + 3 * exchange_bytes(tokens);
+}
+
+int fused_bwd_m64(const void *x, const void *dy, const void *L, const void *R, const void *u_saved,
+                  void *dx, float *dL, float *dR, int accumulate, int64_t tokens, void *ws,
+                  cudaStream_t s)
+{
+    if (!accumulate) MONARCH_TRY(zero_grads(dL, dR, s));
+    if (tokens == 0) return MONARCH_OK;
+    const size_t ex = exchange_bytes(tokens);
+    unsigned *status = (unsigned *)ws;
+    unsigned *counters = (unsigned *)((char *)ws + MONARCH_STATUS_BYTES);
+    char *du = (char *)ws + MONARCH_STATUS_BYTES + kDwCounterBytes;
+    char *dyp = du + ex, *u_own = dyp + ex;
+    const void *u = u_saved;
+    if (!u) {
+        MONARCH_TRY(fused_fwd_m64_stage1(x, R, u_own, tokens, status, s));
+        u = u_own;
+    }
+    MONARCH_TRY(fused_bwd_dx_m64_keep(dy, L, R, dx, du, dyp, counters, status, tokens, s));
+    return launch_dw(x, u, du, dyp, dL, dR, status, tokens, s);
 }
 
 }  // namespace monarch

@@ -1,7 +1,7 @@
 // Host-buffer entry points: the caller's tensors live in host memory; the library streams them
 // through the GPU in token chunks so that the upload of chunk c+1, the kernels of chunk c and the
 // download of chunk c-1 overlap on three streams.  All arithmetic is done by the device entry points
-// (monarch_fwd / monarch_bwd_dx / monarch_bwd_dw); nothing is computed on the host.
+// (monarch_fwd / monarch_bwd); nothing is computed on the host.
 #include <cstdlib>
 #include <new>
 
@@ -22,8 +22,8 @@ struct monarch_host_ctx {
     char *x[kBuf] = {}, *dy[kBuf] = {}, *y[kBuf] = {}, *dx[kBuf] = {};
     char *L = nullptr, *R = nullptr;
     float *dL = nullptr, *dR = nullptr;
-    void *ws = nullptr;
-    size_t ws_bytes = 0;
+    void *ws = nullptr, *ws_b = nullptr;      // forward workspace (keeps u for the backward call), backward
+    size_t ws_bytes = 0, ws_b_bytes = 0;
 };
 
 namespace {
@@ -38,7 +38,7 @@ void destroy(monarch_host_ctx *c)
         if (c->out_done[i]) cudaEventDestroy(c->out_done[i]);
     }
     if (c->w_ready) cudaEventDestroy(c->w_ready);
-    cudaFree(c->L); cudaFree(c->R); cudaFree(c->dL); cudaFree(c->dR); cudaFree(c->ws);
+    cudaFree(c->L); cudaFree(c->R); cudaFree(c->dL); cudaFree(c->dR); cudaFree(c->ws); cudaFree(c->ws_b);
     if (c->s_in) cudaStreamDestroy(c->s_in);
     if (c->s_run) cudaStreamDestroy(c->s_run);
     if (c->s_out) cudaStreamDestroy(c->s_out);
@@ -76,11 +76,9 @@ int run(monarch_host_ctx *c, const void *x, const void *dy, const void *L, const
         MONARCH_CUDA_TRY(cudaStreamWaitEvent(c->s_run, c->in_ready[b], 0));
         if (ci >= kBuf) MONARCH_CUDA_TRY(cudaStreamWaitEvent(c->s_run, c->out_done[b], 0));
         MONARCH_TRY(monarch_fwd(c->x[b], c->L, c->R, c->y[b], tn, c->n, c->m, c->dtype, c->ws, c->ws_bytes, c->s_run));
-        if (backward) {
-            MONARCH_TRY(monarch_bwd_dx(c->dy[b], c->L, c->R, c->dx[b], tn, c->n, c->m, c->dtype, c->ws, c->ws_bytes, c->s_run));
-            MONARCH_TRY(monarch_bwd_dw(c->x[b], c->dy[b], c->L, c->R, c->dL, c->dR, ci > 0, tn, c->n, c->m,
-                                       c->dtype, c->ws, c->ws_bytes, c->s_run));
-        }
+        if (backward)
+            MONARCH_TRY(monarch_bwd(c->x[b], c->dy[b], c->L, c->R, c->ws, c->dx[b], c->dL, c->dR, ci > 0, tn,
+                                    c->n, c->m, c->dtype, c->ws_b, c->ws_b_bytes, c->s_run));
         MONARCH_CUDA_TRY(cudaEventRecord(c->out_ready[b], c->s_run));
 
         MONARCH_CUDA_TRY(cudaStreamWaitEvent(c->s_out, c->out_ready[b], 0));
@@ -95,7 +93,8 @@ int run(monarch_host_ctx *c, const void *x, const void *dy, const void *L, const
     }
     MONARCH_CUDA_TRY(cudaStreamSynchronize(c->s_in));
     MONARCH_CUDA_TRY(cudaStreamSynchronize(c->s_out));
-    return monarch_last_device_status(c->ws, c->s_run);
+    MONARCH_TRY(monarch_last_device_status(c->ws, c->s_run));
+    return monarch_last_device_status(c->ws_b, c->s_run);
 }
 
 }  // namespace
@@ -110,16 +109,14 @@ int monarch_host_create(monarch_host_ctx **out, int64_t max_tokens, int32_t n, i
     if (chunk_tokens == 0) chunk_tokens = 2048;
     if (chunk_tokens % 64) return MONARCH_ERR_INVALID_ARG;
     if (chunk_tokens > max_tokens && max_tokens > 0) chunk_tokens = (max_tokens + 63) / 64 * 64;
-    size_t wsb = 0;
-    for (int op = MONARCH_OP_FWD; op <= MONARCH_OP_BWD_DW; ++op) {
-        const size_t b = monarch_workspace_bytes(op, chunk_tokens, n, m, dtype);
-        if (b == 0) return MONARCH_ERR_UNSUPPORTED;
-        if (b > wsb) wsb = b;
-    }
+    const size_t wsb = monarch_workspace_bytes(MONARCH_OP_FWD, chunk_tokens, n, m, dtype);
+    const size_t wsb_b = monarch_workspace_bytes(MONARCH_OP_BWD, chunk_tokens, n, m, dtype);
+    if (wsb == 0 || wsb_b == 0) return MONARCH_ERR_UNSUPPORTED;
     monarch_host_ctx *c = new (std::nothrow) monarch_host_ctx;
     if (!c) return MONARCH_ERR_CUDA;
     c->max_tokens = max_tokens; c->chunk = chunk_tokens; c->n = n; c->m = m; c->dtype = dtype;
     c->ws_bytes = wsb;
+    c->ws_b_bytes = wsb_b;
     const size_t act = (size_t)chunk_tokens * n * esz(dtype), wb = (size_t)n * m * esz(dtype);
     const size_t gb = (size_t)n * m * sizeof(float);
     bool ok = cudaStreamCreateWithFlags(&c->s_in, cudaStreamNonBlocking) == cudaSuccess &&
@@ -135,8 +132,9 @@ int monarch_host_create(monarch_host_ctx **out, int64_t max_tokens, int32_t n, i
     }
     ok = ok && cudaMalloc(&c->L, wb) == cudaSuccess && cudaMalloc(&c->R, wb) == cudaSuccess &&
          cudaMalloc(&c->dL, gb) == cudaSuccess && cudaMalloc(&c->dR, gb) == cudaSuccess &&
-         cudaMalloc(&c->ws, wsb) == cudaSuccess &&
+         cudaMalloc(&c->ws, wsb) == cudaSuccess && cudaMalloc(&c->ws_b, wsb_b) == cudaSuccess &&
          monarch_workspace_init(c->ws, wsb, c->s_run) == MONARCH_OK &&
+         monarch_workspace_init(c->ws_b, wsb_b, c->s_run) == MONARCH_OK &&
          cudaStreamSynchronize(c->s_run) == cudaSuccess;
     if (!ok) {
         destroy(c);

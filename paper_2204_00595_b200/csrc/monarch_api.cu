@@ -68,7 +68,7 @@ enum Family { kSimt = 0, kFused = 1, kTcStaged = 2, kNone = -1 };
 bool fused_available(int op, int m, int dtype)
 {
     static const bool off = getenv("MONARCH_NO_FUSED") != nullptr;   // comparison runs: stage chain instead
-    return !off && dtype == MONARCH_BF16 && m == 64 && op != MONARCH_OP_MLP_FWD;
+    return !off && dtype == MONARCH_BF16 && m == 64 && op != MONARCH_OP_MLP_FWD;   // FWD, BWD_DX, BWD_DW, BWD
 }
 
 // true when the call can run as a chain of tensor-core stages through the workspace
@@ -97,10 +97,16 @@ extern "C" {
 
 size_t monarch_workspace_bytes(int op, int64_t tokens, int32_t n, int32_t m, int dtype)
 {
-    if (op < MONARCH_OP_FWD || op > MONARCH_OP_MLP_FWD) return 0;
+    if (op < MONARCH_OP_FWD || op > MONARCH_OP_BWD) return 0;
     if (check_shape(tokens, n, m, dtype) != MONARCH_OK) return 0;
     const int which = pick(op, m, dtype);
     if (which < 0) return 0;
+    if (op == MONARCH_OP_BWD) {
+        if (which == kFused) return fused_bwd_m64_workspace_bytes(tokens);
+        const size_t a = staged_workspace_bytes(MONARCH_OP_BWD_DX, tokens, n, m, dtype);
+        const size_t b = staged_workspace_bytes(MONARCH_OP_BWD_DW, tokens, n, m, dtype);
+        return a > b ? a : b;
+    }
     if (which == kFused)
         return op == MONARCH_OP_FWD      ? fused_fwd_m64_workspace_bytes(tokens)
                : op == MONARCH_OP_BWD_DX ? fused_bwd_dx_m64_workspace_bytes(tokens)
@@ -162,6 +168,31 @@ int monarch_bwd_dw(const void *x, const void *dy, const void *L, const void *R, 
                          (cudaStream_t)stream);
 }
 
+int monarch_bwd(const void *x, const void *dy, const void *L, const void *R, const void *fwd_workspace,
+                void *dx, float *dL, float *dR, int accumulate, int64_t tokens, int32_t n, int32_t m,
+                int dtype, void *workspace, size_t workspace_bytes, void *stream)
+{
+    MONARCH_TRY(check_shape(tokens, n, m, dtype));
+    if (accumulate != 0 && accumulate != 1) return MONARCH_ERR_INVALID_ARG;
+    if (fwd_workspace != nullptr && fwd_workspace == workspace) return MONARCH_ERR_INVALID_ARG;
+    const size_t act = (size_t)tokens * n * esize(dtype), wb = (size_t)n * m * esize(dtype);
+    const size_t gb = (size_t)n * m * sizeof(float);
+    const Range in[] = {{x, act}, {dy, act}, {L, wb}, {R, wb}};
+    const Range out[] = {{dx, act}, {dL, gb}, {dR, gb}};
+    const int which = pick(MONARCH_OP_BWD, m, dtype);
+    if (which < 0) return MONARCH_ERR_UNSUPPORTED;
+    MONARCH_TRY(check_buffers(in, 4, out, 3, workspace, workspace_bytes,
+                              monarch_workspace_bytes(MONARCH_OP_BWD, tokens, n, m, dtype)));
+    cudaStream_t s = (cudaStream_t)stream;
+    if (which == kFused) {
+        const bool saved = fwd_workspace != nullptr && pick(MONARCH_OP_FWD, m, dtype) == kFused;
+        return fused_bwd_m64(x, dy, L, R, saved ? fused_fwd_m64_saved_u(fwd_workspace) : nullptr, dx, dL,
+                             dR, accumulate, tokens, workspace, s);
+    }
+    MONARCH_TRY(staged_bwd_dx(dy, L, R, dx, tokens, m, dtype, workspace, s));
+    return staged_bwd_dw(x, dy, L, R, dL, dR, accumulate, tokens, m, dtype, workspace, s);
+}
+
 int monarch_mlp_fwd(const void *x, const void *L1, const void *R1, const void *b1, const void *L2,
                     const void *R2, const void *b2, void *y, int64_t tokens, int32_t n, int32_t m,
                     int dtype, void *workspace, size_t workspace_bytes, void *stream)
@@ -216,7 +247,7 @@ int monarch_set_impl(int impl)
 
 const char *monarch_impl_name(int op, int32_t m, int dtype)
 {
-    if (op < MONARCH_OP_FWD || op > MONARCH_OP_MLP_FWD) return "unsupported";
+    if (op < MONARCH_OP_FWD || op > MONARCH_OP_BWD) return "unsupported";
     if (check_shape(0, m * m, m, dtype) != MONARCH_OK) return "unsupported";
     const int which = pick(op, m, dtype);
     return which < 0 ? "unsupported" : which == kFused ? "fused-tcgen05"

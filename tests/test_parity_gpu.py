@@ -113,6 +113,40 @@ def test_fwd_bwd_small(P, impl, m, T, dtype):
     assert_close(to_host64(dR), 2 * ref["dR"], dtype, "dR accumulate")
 
 
+@pytest.mark.parametrize("saved", [False, True])
+@pytest.mark.parametrize("m,T,dtype", [(16, 65, "f32"), (32, 129, "bf16"), (64, 1, "bf16"), (64, 130, "bf16"),
+                                       (64, 257, "bf16"), (128, 70, "bf16")])
+def test_bwd_one_call(P, impl, m, T, dtype, saved):
+    """monarch_bwd = monarch_bwd_dx + monarch_bwd_dw, with or without the forward call's workspace."""
+    import torch
+    code = _code(P, dtype)
+    _skip_if_same_family(P, impl, P.OP_BWD, m, code)
+    n = m * m
+    d = _small_inputs(m, T, dtype, seed=77 * m + T)
+    x, dy, L, R = (to_device(d[k], dtype) for k in ("x", "dy", "L", "R"))
+    yf, y = _guarded((T, n), _tdtype(dtype))
+    dxf, dx = _guarded((T, n), _tdtype(dtype))
+    dLf, dL = _guarded((m, m, m), torch.float32)
+    dRf, dR = _guarded((m, m, m), torch.float32)
+    ws_f = P.Workspace(P.monarch_workspace_bytes(P.OP_FWD, T, n, m, code))
+    ws_b = P.Workspace(P.monarch_workspace_bytes(P.OP_BWD, T, n, m, code))
+    P.monarch_fwd(x, L, R, y, T, n, m, ws_f)
+    P.monarch_bwd(x, dy, L, R, dx, dL, dR, 0, T, n, m, ws_b, fwd_workspace=ws_f if saved else None)
+    torch.cuda.synchronize()
+    assert P.monarch_last_device_status(ws_f) == 0 and P.monarch_last_device_status(ws_b) == 0
+    ref = O.bwd(d["x"], d["dy"], d["L"], d["R"])
+    assert_close(to_host64(y), O.fwd(d["x"], d["L"], d["R"]), dtype, "y")
+    assert_close(to_host64(dx), ref["dx"], dtype, "dx")
+    assert_close(to_host64(dL), ref["dL"], dtype, "dL")
+    assert_close(to_host64(dR), ref["dR"], dtype, "dR")
+    for flat, what in ((yf, "y"), (dxf, "dx"), (dLf, "dL"), (dRf, "dR")):
+        _check_guard(flat, what)
+    P.monarch_bwd(x, dy, L, R, dx, dL, dR, 1, T, n, m, ws_b, fwd_workspace=ws_f if saved else None)
+    torch.cuda.synchronize()
+    assert_close(to_host64(dL), 2 * ref["dL"], dtype, "dL accumulate")
+    assert_close(to_host64(dR), 2 * ref["dR"], dtype, "dR accumulate")
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("m,T", [(16, 5), (32, 129), (64, 257), (128, 66)])
 def test_mlp_small(P, impl, m, T, dtype):
@@ -151,6 +185,13 @@ def test_zero_tokens(P, impl, dtype):
     P.monarch_bwd_dw(x, x.clone(), W, W.clone(), dL, dR, 0, 0, n, m, ws)
     torch.cuda.synchronize()
     assert float(dL.abs().max()) == 0.0 and float(dR.abs().max()) == 0.0
+    for mm in (32, 64):             # the one-call backward defines dL, dR for an empty batch too
+        g = torch.full((2, mm, mm, mm), 5.0, dtype=torch.float32, device="cuda")
+        xx = torch.zeros(1, mm * mm, dtype=td, device="cuda")
+        Wm = torch.zeros(mm, mm, mm, dtype=td, device="cuda")
+        P.monarch_bwd(xx, xx.clone(), Wm, Wm.clone(), xx.clone(), g[0], g[1], 0, 0, mm * mm, mm, ws)
+        torch.cuda.synchronize()
+        assert float(g.abs().max()) == 0.0
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
@@ -247,6 +288,17 @@ def test_workload_fwd_bwd(P, impl, cfg):
     assert abs(float(np.sum(dxh * d["x"])) - s) <= tol
     assert abs(float(np.sum(dLh * d["L"])) - s) <= tol
     assert abs(float(np.sum(dRh * d["R"])) - s) <= tol
+    # the one-call backward on the intermediate the forward call left in its workspace (the launch
+    # configuration the benchmark times)
+    ws_b = P.Workspace(P.monarch_workspace_bytes(P.OP_BWD, T, n, m, code))
+    dx.fill_(float("nan")); dL.fill_(float("nan")); dR.fill_(float("nan"))
+    P.monarch_fwd(x, L, R, y, T, n, m, ws)
+    P.monarch_bwd(x, dy, L, R, dx, dL, dR, 0, T, n, m, ws_b, fwd_workspace=ws)
+    torch.cuda.synchronize()
+    assert P.monarch_last_device_status(ws_b) == 0
+    assert_close(to_host64(dx)[rows], ref["dx"][rows], c.dtype, f"cfg{cfg} dx (one call)")
+    assert_close(to_host64(dL), ref["dL"], c.dtype, f"cfg{cfg} dL (one call)")
+    assert_close(to_host64(dR), ref["dR"], c.dtype, f"cfg{cfg} dR (one call)")
 
 
 def test_workload_mlp(P, impl):
