@@ -222,25 +222,33 @@ __device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtenso
             }
         }
     } else if (warp == kDypWarp) {
-        // the operand slices are P dy in 2 KB runs [l/8 2][t 64][8 l] per block j: copy them out
+        // the operand slices are P dy in 2 KB runs [l/8 2][t 64][8 l] per block j: copy them out.  The two
+        // groups that share these 16 blocks (hk = 0, 1) build identical slices; each writes every other one.
         if (lane != 0 || p.dyp == nullptr) return;
         uint32_t n = 0;
+        int held = -1;                       // buffer whose copy is still in flight
         for (int tile = first; tile < p.tiles; tile += step) {
             __nv_bfloat16 *dst = p.dyp + ((long long)tile * 64 + hj * 16) * 4096;
 #pragma unroll 1
             for (int ks = 0; ks < 4; ++ks, ++n) {
                 const uint32_t ab = n & 1;
                 if (!wait_fast(af + ab * 8, (n >> 1) & 1, p.status, dead, kErrTmaWait)) return;
+                if (held >= 0) {
+                    // the slice before this one has been read out by now (its buffer is only needed
+                    // again after the current slice, which is already transposed)
+                    tma_store_wait_read<0>();
+                    mbar_arrive(ae + held * 8);
+                    held = -1;
+                }
+                if ((ks & 1) == hk) {
 #pragma unroll 4
-                for (int j = 0; j < 16; ++j)
-                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst + j * 4096 + ks * 1024),
-                                 "r"(a0 + ab * kSliceBytes + j * kBlockSlice), "r"(2048) : "memory");
-                tma_store_commit();
-                // one copy stays in flight: the slice before this one has been read out by now (its
-                // buffer is only needed again after the current slice, which is already transposed)
-                if (n >= 1) {
-                    tma_store_wait_read<1>();
-                    mbar_arrive(ae + (ab ^ 1) * 8);
+                    for (int j = 0; j < 16; ++j)
+                        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst + j * 4096 + ks * 1024),
+                                     "r"(a0 + ab * kSliceBytes + j * kBlockSlice), "r"(2048) : "memory");
+                    tma_store_commit();
+                    held = (int)ab;
+                } else {
+                    mbar_arrive(ae + ab * 8);
                 }
             }
         }
