@@ -176,6 +176,18 @@ def time_oracle(cfg, d, target_s=12.0):
 
 # ----------------------------------------------------------------------------- main
 
+# Kernels behind each timed call (bf16, m = 64), and the DRAM traffic one call generated under ncu
+# (profiles/fused_m64_step_workload3_ncu_full.md; captured at workload 3's full size).
+KERNELS_OF = {
+    (64, "bf16", "fwd"): "fused_fwd_m64_kernel (1 launch)",
+    (64, "bf16", "bwd"): "fused_bwd_dx_m64_kernel + fused_bwd_dw_m64_kernel (2 launches, 2 memset nodes)",
+    (64, "bf16", "bwd_dx"): "fused_bwd_dx_m64_kernel (1 launch)",
+    (64, "bf16", "bwd_dw"): "fused_fwd_m64_kernel (stage 1) + fused_bwd_dx_m64_kernel (stage 1) + "
+                            "fused_bwd_dw_m64_kernel (3 launches, 2 memset nodes)",
+}
+NCU_TRAFFIC_MB = {(3, "fwd"): 149.5, (3, "bwd"): 486.5}
+
+
 def main():
     args = parse_args()
     from paper_2204_00595_b200.inputs import CONFIGS, make_inputs
@@ -335,10 +347,13 @@ def main():
                        "impl": P.monarch_impl_name(op_of[k], m, code)}
     dom = max(calls, key=lambda k: per_call[k]["ms"])
     roofline = {
-        "bound": "hbm", "kernel": f"{dom} ({per_call[dom]['impl']})",
+        "bound": "hbm", "kernel": f"{dom}: {KERNELS_OF.get((m, cfg.dtype, dom), per_call[dom]['impl'])}",
         "achieved": per_call[dom]["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
         "frac": per_call[dom]["gbs"] / peaks["hbm_gbs"], "peak_source": peaks["source"],
-        "traffic": None,
+        "traffic": NCU_TRAFFIC_MB.get((cfg.index, dom)),
+        "traffic_unit": "MB per call (dram__bytes_read.sum + dram__bytes_write.sum, summed over the "
+                        "call's kernels; ncu capture summarised under profiles/)",
+        "algorithmic_mb": call_bytes(dom, n, m, T, cfg.dtype) / 1e6,
     }
 
     line = {
