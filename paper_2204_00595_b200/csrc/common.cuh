@@ -67,6 +67,9 @@ int tc_staged_mlp_fwd(const void *x, const void *L1, const void *R1, const void 
 size_t fused_fwd_m64_workspace_bytes(int64_t tokens);
 int fused_fwd_m64(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws,
                   cudaStream_t s);
+// the same with every CTA doing both stages (fused_m64_team.cu); same workspace layout
+int fused_fwd_m64_team(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws,
+                       cudaStream_t s);
 // first stage only: u = P R x in the exchange layout [tile][j][k/8][t%64][k%8] (tokens rounded up to 64)
 int fused_fwd_m64_stage1(const void *x, const void *R, void *u, int64_t tokens, unsigned *status,
                          cudaStream_t s);

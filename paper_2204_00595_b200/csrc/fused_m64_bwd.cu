@@ -56,7 +56,16 @@ struct BwdParams {
     long long tokens;
     int tiles;
     int b1, b2;                // CTAs per B1 group, per B2 group
+    long long *trace;          // optional per-CTA timeline (debug builds), else null
 };
+
+#ifdef MONARCH_TRACE
+#define BTRACE(item, slot, val) do { if (p.trace && (item) < 16) p.trace[((size_t)blockIdx.x * 16 + (item)) * 8 + (slot)] = (val); } while (0)
+#define BCLK() clock64()
+#else
+#define BTRACE(item, slot, val) do { } while (0)
+#define BCLK() 0ll
+#endif
 
 struct Bars {
     uint64_t w;                               // resident weights landed
@@ -178,6 +187,7 @@ __device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtenso
         for (int b = 0; b < 16; ++b) tma_load_2d(smem0 + b * 4096, &tm_Lt, hk * 32, (hj * 16 + b) * kM, wbar);
         uint32_t n = 0;
         for (int tile = first; tile < p.tiles; tile += step) {
+            BTRACE(n >> 2, 0, BCLK());
 #pragma unroll 1
             for (int ks = 0; ks < 4; ++ks, ++n) {
                 const uint32_t rb = n & 1;
@@ -193,12 +203,17 @@ __device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtenso
         const int mi = lane >> 3, r = lane & 7;      // matrix of the x4 group, row within it
         const int lo = mi >> 1, jo = mi & 1;
         uint32_t n = 0;
+        [[maybe_unused]] long long w_raw = 0, w_ae = 0, w_tr = 0;
         for (int tile = first; tile < p.tiles; tile += step) {
 #pragma unroll 1
             for (int ks = 0; ks < 4; ++ks, ++n) {
                 const uint32_t rb = n & 1;
+                [[maybe_unused]] const long long c0 = BCLK();
                 if (!wait_fast(rawf + rb * 8, (n >> 1) & 1, p.status, dead, kErrTmaWait)) return;
+                [[maybe_unused]] const long long c1 = BCLK();
                 if (!wait_fast(ae + rb * 8, ((n >> 1) & 1) ^ 1, p.status, dead, kErrSlotWait)) return;
+                [[maybe_unused]] const long long c2 = BCLK();
+                w_raw += c1 - c0; w_ae += c2 - c1;
                 const uint32_t src = raw0 + rb * kRawBytes + (lo * 8 + r) * 32 + ((jo ^ (r >> 2)) * 16);
                 const uint32_t dst = a0 + rb * kSliceBytes + (jo * 8 + r) * kBlockSlice + lo * 1024;
 #pragma unroll 4
@@ -219,7 +234,12 @@ __device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtenso
                     mbar_arrive(rawe + rb * 8);
                     mbar_arrive(af + rb * 8);
                 }
+                w_tr += BCLK() - c2;
             }
+            if (tw == 0 && lane == 0) {
+                BTRACE((n >> 2) - 1, 1, w_raw); BTRACE((n >> 2) - 1, 2, w_ae); BTRACE((n >> 2) - 1, 3, w_tr);
+            }
+            w_raw = w_ae = w_tr = 0;
         }
     } else if (warp == kDypWarp) {
         // the operand slices are P dy in 2 KB runs [l/8 2][t 64][8 l] per block j: copy them out.  The two
@@ -261,6 +281,7 @@ __device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtenso
         const uint64_t a_ns = make_smem_desc(0, 1024, 128, 0);
         const uint64_t b_mn = make_smem_desc(0, 16, 512, kSwizzle64) | (uint64_t)(smem0 >> 4);
         uint32_t n = 0, nitem = 0;
+        [[maybe_unused]] long long w_af = 0;
         for (int tile = first; tile < p.tiles; tile += step, ++nitem) {
             const uint32_t buf = nitem & 1, par = (nitem >> 1) & 1;
             if (!wait_fast(acce0 + buf * 8, par ^ 1, p.status, dead, kErrTmemWait)) return;
@@ -269,8 +290,10 @@ __device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtenso
 #pragma unroll 1
             for (int ks = 0; ks < 4; ++ks, ++n) {
                 const uint32_t ab = n & 1;
+                [[maybe_unused]] const long long c0 = BCLK();
                 if (!wait_fast(af + ab * 8, (n >> 1) & 1, p.status, dead, kErrTmaWait)) return;
                 tc_fence_after();
+                w_af += BCLK() - c0;
                 const uint64_t as = a_ns | (uint64_t)((a0 + ab * kSliceBytes) >> 4);
                 const uint64_t bs = b_mn + ks * 64;                           // 16 rows of 64 B
 #pragma unroll
@@ -281,6 +304,8 @@ __device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtenso
                 mma_commit(ae + ab * 8);
             }
             mma_commit(accf0 + buf * 8);
+            BTRACE(nitem, 4, w_af); BTRACE(nitem, 5, BCLK());
+            w_af = 0;
         }
     } else if (warp < kEpiWarps) {
         const int q4 = warp & 3, sub = warp >> 2;
@@ -294,6 +319,7 @@ __device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtenso
         for (int tile = first; tile < p.tiles; tile += step, ++nitem) {
             const uint32_t buf = nitem & 1, par = (nitem >> 1) & 1;
             if (!wait_fast(accf0 + buf * 8, par, p.status, dead, kErrMmaWait)) return;
+            if (threadIdx.x == 0) BTRACE(nitem, 6, BCLK());
             tc_fence_after();
 #pragma unroll 1
             for (int c = sub; c < 8; c += 2, ++nchunk) {
@@ -324,6 +350,7 @@ __device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtenso
                 __syncwarp();
                 if (lane == 0) mbar_arrive(stf0 + k * 8);
             }
+            if (threadIdx.x == 0) BTRACE(nitem, 7, BCLK());
         }
     } else if (warp >= kStoreWarp0 && warp < kStoreWarp0 + 2) {
         if (lane != 0) return;
@@ -621,6 +648,10 @@ int launch_bwd_m64(const void *dy, const void *L, const void *R, void *dx, void 
     if (b2 > tiles) b2 = (int)tiles;
     p.b1 = b1;
     p.b2 = b2;
+    p.trace = nullptr;
+#ifdef MONARCH_TRACE
+    if (const char *e = getenv("MONARCH_TRACE_PTR_BWD")) p.trace = (long long *)strtoull(e, nullptr, 0);
+#endif
     fused_bwd_dx_m64_kernel<<<8 * b1 + 8 * b2, kThreads, kSmemBytes, s>>>(tm_dy3, tm_Lt, tm_R, tm_du, tm_dx, p);
     note_launch();
     MONARCH_CUDA_TRY(cudaGetLastError());
