@@ -70,6 +70,10 @@ int fused_fwd_m64(const void *x, const void *L, const void *R, void *y, int64_t 
 // the same with every CTA doing both stages (fused_m64_team.cu); same workspace layout
 int fused_fwd_m64_team(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws,
                        cudaStream_t s);
+// feed-forward block as two passes of the team kernel with bias (+ GELU) in the stage-2 epilogue
+size_t fused_mlp_fwd_m64_workspace_bytes(int64_t tokens);
+int fused_mlp_fwd_m64(const void *x, const void *L1, const void *R1, const void *b1, const void *L2,
+                      const void *R2, const void *b2, void *y, int64_t tokens, void *ws, cudaStream_t s);
 // first stage only: u = P R x in the exchange layout [tile][j][k/8][t%64][k%8] (tokens rounded up to 64)
 int fused_fwd_m64_stage1(const void *x, const void *R, void *u, int64_t tokens, unsigned *status,
                          cudaStream_t s);

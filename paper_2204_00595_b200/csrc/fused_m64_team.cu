@@ -34,6 +34,8 @@ struct TeamParams {
     __nv_bfloat16 *u;          // exchange buffer, [tiles][64 j][8][64 t][8] bf16
     unsigned *counters;        // one per 64-token tile, zero between calls
     unsigned *status;
+    const __nv_bfloat16 *bias; // optional [n]: added to the output (feed-forward block, Section 4)
+    int gelu;                  // apply erf-GELU after the bias
     int tiles;
     int teams;                 // CTA team c takes tiles c, c + teams, ...
     long long *trace;          // optional per-CTA timeline (debug builds), else null
@@ -78,6 +80,20 @@ __device__ __forceinline__ bool wait_fast(uint32_t bar, uint32_t parity, unsigne
     return mbar_wait(bar, parity, status, dead, code);
 }
 
+// GELU(a) = a/2 (1 + erf(a / sqrt 2)) evaluated as a * sigmoid(2 a (c0 + c1 a^2 + c2 a^4)): the logistic form
+// of the usual tanh approximation with one more polynomial term, coefficients fitted (minimax over [-8, 8]) to
+// the erf definition: |error| <= 2.6e-5 everywhere (a^2 is clamped at 64, beyond which the sigmoid has
+// saturated) - well below one bf16 ulp of the result.  Nine instructions, two of them MUFU; the libm-grade erf
+// costs twice that, and the stage-2 epilogue is on the critical path of the pipeline.
+__device__ __forceinline__ float gelu_fast(float a)
+{
+    const float a2 = fminf(a * a, 64.0f);
+    float t = fmaf(a2, 0.0010142630198970437f, -0.10677572339773178f);     // -2 log2(e) * (c2 a^2 + c1)
+    t = fmaf(a2, t, -2.301121234893799f);
+    const float e = exp2f(a * t);                                          // exp(-2 a poly(a^2))
+    return __fdividef(a, 1.0f + e);
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 fused_fwd_m64_team_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_R,
                           const __grid_constant__ CUtensorMap tm_L, const __grid_constant__ CUtensorMap tm_u,
@@ -88,6 +104,7 @@ fused_fwd_m64_team_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid
     __shared__ uint32_t tmem_base_s;
     __shared__ int dead_s;
     __shared__ int dep_items_s;
+    __shared__ __align__(16) __nv_bfloat16 bias_s[32 * 16];   // this CTA's slice of the bias: [l local][j local]
 
     const uint32_t smemR = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t smemL = smemR + kRBytes;
@@ -122,6 +139,12 @@ fused_fwd_m64_team_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid
     if (warp == 0) {
         tmem_alloc(smem_u32(&tmem_base_s), 512);
         tmem_relinquish();
+    }
+    if (p.bias != nullptr && threadIdx.x >= 64 && threadIdx.x < 128) {
+        // global loads stay out of the steady state: they slow the MMA-issuing thread down
+        const int l = (threadIdx.x - 64) >> 1, half = threadIdx.x & 1;
+        *reinterpret_cast<uint4 *>(&bias_s[l * 16 + half * 8]) =
+            __ldg(reinterpret_cast<const uint4 *>(p.bias + (hl * 32 + l) * kM + hj * 16 + half * 8));
     }
     tc_fence_before();
     __syncthreads();
@@ -347,6 +370,21 @@ fused_fwd_m64_team_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid
 #pragma unroll
                     for (int a = 0; a < 8; ++a) tmem_ld4(lane_base + 256 + a * 32 + c * 4, v[a]);
                     tmem_ld_wait();
+                    if (p.bias != nullptr) {
+                        // output element (l, j): l = 32 hl + 4c + q, j = 16 hj + 8h + a
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const uint4 bq = *reinterpret_cast<const uint4 *>(&bias_s[(c * 4 + q) * 16 + h * 8]);
+                            const uint32_t bw[4] = {bq.x, bq.y, bq.z, bq.w};
+#pragma unroll
+                            for (int a = 0; a < 8; ++a) {
+                                const float b = __uint_as_float((a & 1) ? (bw[a >> 1] & 0xFFFF0000u) : (bw[a >> 1] << 16));
+                                float f = __uint_as_float(v[a][q]) + b;
+                                if (p.gelu) f = gelu_fast(f);
+                                v[a][q] = __float_as_uint(f);
+                            }
+                        }
+                    }
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         const uint32_t o0 = pack_bf16(__uint_as_float(v[0][q]), __uint_as_float(v[1][q]));
@@ -434,16 +472,15 @@ fused_fwd_m64_team_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid
 }  // namespace
 }  // namespace tc
 
-// Same workspace layout as the split schedule: [status 256 B][tile counters 64 KB][u'].
-int fused_fwd_m64_team(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws,
-                       cudaStream_t s)
+namespace {
+constexpr size_t kTeamCounterBytes = 65536;
+
+int launch_team(const void *x, const void *L, const void *R, const void *bias, int gelu, void *y, void *u,
+                unsigned *counters, unsigned *status, int64_t tokens, cudaStream_t s)
 {
     using namespace tc;
-    if (tokens == 0) return MONARCH_OK;
-    constexpr size_t kCounterBytes = 65536;
     const long long tiles = (tokens + 63) / 64;
-    if (tiles * 4 > (long long)kCounterBytes) return MONARCH_ERR_UNSUPPORTED;
-    void *u = (char *)ws + MONARCH_STATUS_BYTES + kCounterBytes;
+    if (tiles * 4 > (long long)kTeamCounterBytes) return MONARCH_ERR_UNSUPPORTED;
     CUtensorMap tm_x, tm_R, tm_L, tm_u, tm_y;
     MONARCH_TRY(encode_tmap_2d(&tm_x, x, (uint64_t)tokens, kN, kN * 2, 64, 64, 128));
     MONARCH_TRY(encode_tmap_2d(&tm_R, R, kN, kM, kM * 2, 64, 64, 128));
@@ -465,9 +502,11 @@ int fused_fwd_m64_team(const void *x, const void *L, const void *R, void *y, int
                                               cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
     }
     TeamParams p;
-    p.status = (unsigned *)ws;
-    p.counters = (unsigned *)((char *)ws + MONARCH_STATUS_BYTES);
+    p.status = status;
+    p.counters = counters;
     p.u = (__nv_bfloat16 *)u;
+    p.bias = (const __nv_bfloat16 *)bias;
+    p.gelu = gelu;
     p.tiles = (int)tiles;
     int teams = sms / 8;
     if (teams < 1) teams = 1;
@@ -481,6 +520,42 @@ int fused_fwd_m64_team(const void *x, const void *L, const void *R, void *y, int
     note_launch();
     MONARCH_CUDA_TRY(cudaGetLastError());
     return MONARCH_OK;
+}
+
+size_t exchange_bytes(int64_t tokens)
+{
+    const size_t tiles = (size_t)((tokens + 63) / 64);
+    return (tiles * 64 * (size_t)tc::kN * 2 + 255) & ~(size_t)255;
+}
+}  // namespace
+
+// Same workspace layout as the split schedule: [status 256 B][tile counters 64 KB][u'].
+int fused_fwd_m64_team(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws,
+                       cudaStream_t s)
+{
+    if (tokens == 0) return MONARCH_OK;
+    return launch_team(x, L, R, nullptr, 0, y, (char *)ws + MONARCH_STATUS_BYTES + kTeamCounterBytes,
+                       (unsigned *)((char *)ws + MONARCH_STATUS_BYTES), (unsigned *)ws, tokens, s);
+}
+
+// Feed-forward block y = M2 GELU(M1 x + b1) + b2 as two passes of the same kernel; the hidden activations h
+// (bf16) live in the workspace: [status][counters][u'][h].
+size_t fused_mlp_fwd_m64_workspace_bytes(int64_t tokens)
+{
+    return MONARCH_STATUS_BYTES + kTeamCounterBytes + exchange_bytes(tokens) +
+           (((size_t)tokens * tc::kN * 2 + 255) & ~(size_t)255);
+}
+
+int fused_mlp_fwd_m64(const void *x, const void *L1, const void *R1, const void *b1, const void *L2,
+                      const void *R2, const void *b2, void *y, int64_t tokens, void *ws, cudaStream_t s)
+{
+    if (tokens == 0) return MONARCH_OK;
+    unsigned *status = (unsigned *)ws;
+    unsigned *counters = (unsigned *)((char *)ws + MONARCH_STATUS_BYTES);
+    char *u = (char *)ws + MONARCH_STATUS_BYTES + kTeamCounterBytes;
+    char *h = u + exchange_bytes(tokens);
+    MONARCH_TRY(launch_team(x, L1, R1, b1, 1, h, u, counters, status, tokens, s));
+    return launch_team(h, L2, R2, b2, 0, y, u, counters, status, tokens, s);
 }
 
 }  // namespace monarch

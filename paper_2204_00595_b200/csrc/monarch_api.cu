@@ -68,7 +68,7 @@ enum Family { kSimt = 0, kFused = 1, kTcStaged = 2, kNone = -1 };
 bool fused_available(int op, int m, int dtype)
 {
     static const bool off = getenv("MONARCH_NO_FUSED") != nullptr;   // comparison runs: stage chain instead
-    return !off && dtype == MONARCH_BF16 && m == 64 && op != MONARCH_OP_MLP_FWD;   // FWD, BWD_DX, BWD_DW, BWD
+    return !off && dtype == MONARCH_BF16 && m == 64;   // every op
 }
 
 // true when the call can run as a chain of tensor-core stages through the workspace
@@ -108,7 +108,8 @@ size_t monarch_workspace_bytes(int op, int64_t tokens, int32_t n, int32_t m, int
         return a > b ? a : b;
     }
     if (which == kFused)
-        return op == MONARCH_OP_FWD      ? fused_fwd_m64_workspace_bytes(tokens)
+        return op == MONARCH_OP_MLP_FWD  ? fused_mlp_fwd_m64_workspace_bytes(tokens)
+               : op == MONARCH_OP_FWD    ? fused_fwd_m64_workspace_bytes(tokens)
                : op == MONARCH_OP_BWD_DX ? fused_bwd_dx_m64_workspace_bytes(tokens)
                                          : fused_bwd_dw_m64_workspace_bytes(tokens);
     return staged_workspace_bytes(op, tokens, n, m, dtype);
@@ -206,6 +207,8 @@ int monarch_mlp_fwd(const void *x, const void *L1, const void *R1, const void *b
     if (which < 0) return MONARCH_ERR_UNSUPPORTED;
     MONARCH_TRY(check_buffers(in, 7, out, 1, workspace, workspace_bytes,
                               monarch_workspace_bytes(MONARCH_OP_MLP_FWD, tokens, n, m, dtype)));
+    if (which == kFused)
+        return fused_mlp_fwd_m64(x, L1, R1, b1, L2, R2, b2, y, tokens, workspace, (cudaStream_t)stream);
     if (which == kTcStaged)
         return tc_staged_mlp_fwd(x, L1, R1, b1, L2, R2, b2, y, tokens, m, workspace,
                                  (cudaStream_t)stream);
