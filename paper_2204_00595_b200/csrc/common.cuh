@@ -90,6 +90,11 @@ int fused_bwd_m64_stage1(const void *dy, const void *L, void *du, void *dyp, int
 int fused_bwd_dx_m64_keep(const void *dy, const void *L, const void *R, void *dx, void *du, void *dyp,
                           unsigned *counters, unsigned *status, int64_t tokens, cudaStream_t s);
 
+// dx, dL +=, dR += in one launch; u = P R x in the forward exchange layout, du / dyp = scratch exchange buffers
+int fused_bwd_all_m64(const void *x, const void *dy, const void *L, const void *R, const void *u, void *dx,
+                      void *du, void *dyp, float *dL, float *dR, unsigned *counters, unsigned *status,
+                      int64_t tokens, cudaStream_t s);
+
 // ---- weight gradients for m = 64, bf16 (fused_m64_bwd_dw.cu) ----
 size_t fused_bwd_dw_m64_workspace_bytes(int64_t tokens);
 int fused_bwd_dw_m64(const void *x, const void *dy, const void *L, const void *R, float *dL, float *dR,

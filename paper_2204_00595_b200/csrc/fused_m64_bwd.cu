@@ -21,6 +21,7 @@
 //       (t, k), staged with the 128B swizzle and stored as 64 x 64 boxes.
 //
 // Waits are bounded; B1 waits on nothing outside its CTA, B2 on a per-tile counter bumped by B1.
+#include <cstdio>
 #include <cstdlib>
 
 #include "tc_common.cuh"
@@ -56,6 +57,10 @@ struct BwdParams {
     long long tokens;
     int tiles;
     int b1, b2;                // CTAs per B1 group, per B2 group
+    int b3;                    // all-in-one kernel: CTAs per group of the dL kind (0 elsewhere)
+    unsigned need, reset_at;   // a tile is ready at `need` arrivals; the consumer that brings it to `reset_at` clears it
+    const __nv_bfloat16 *u;    // all-in-one kernel: u' = P R x, [tiles][64 j][8][64 t][8] (forward exchange layout)
+    float *dL, *dR;            // all-in-one kernel: gradients (added to)
     long long *trace;          // optional per-CTA timeline (debug builds), else null
 };
 
@@ -73,7 +78,7 @@ struct Bars {
     uint64_t st_full[8], st_free[8];          // staging buffers (per half: B1 uses 2, B2 uses 4)
     uint64_t raw_full[2], raw_empty[2];       // B1 raw chunks
     uint64_t a_full[2], a_empty[2];           // B1 operand slices
-    uint64_t full[kQuads], empty[kQuads];     // B2 operand ring, groups of four slots
+    uint64_t full[4], empty[4];               // operand rings: groups of four slots (B2, dL kind) or pairs (B2R)
 };
 
 __device__ __forceinline__ unsigned ld_acquire(const unsigned *p)
@@ -271,6 +276,14 @@ __device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtenso
                     mbar_arrive(ae + ab * 8);
                 }
             }
+            if (p.b3 > 0) {
+                // another kind of CTA of this launch reads P dy back: publish the tile once the copies are complete
+                tma_store_wait_all<0>();
+                if (held >= 0) { mbar_arrive(ae + held * 8); held = -1; }
+                fence_proxy_async_global();
+                __threadfence();
+                atomicAdd(p.counters + tile, 1u);
+            }
         }
         tma_store_wait_all<0>();
     } else if (warp == kMmaWarp) {
@@ -387,9 +400,9 @@ __device__ __forceinline__ void b2_body(const CUtensorMap &tm_R, const CUtensorM
         for (int tile = first; tile < p.tiles; tile += step, ++nitem) {
             // wait until all B1 groups have published their part of du for this tile
             const unsigned *ctr = p.counters + tile;
-            if (ld_acquire(ctr) < kB1Arrivals) {
+            if (ld_acquire(ctr) < p.need) {
                 const unsigned long long t0 = global_timer_ns();
-                while (ld_acquire(ctr) < kB1Arrivals) {
+                while (ld_acquire(ctr) < p.need) {
                     if (*dead || global_timer_ns() - t0 > kWaitLimitNs) {
                         *dead = 1;
                         atomicCAS(p.status, 0u, (unsigned)kErrPeerWait);
@@ -399,7 +412,7 @@ __device__ __forceinline__ void b2_body(const CUtensorMap &tm_R, const CUtensorM
             }
             // the last B2 group to get here clears the tile's counter for the next call
             const unsigned old = atomicAdd(p.counters + tile, 1u);
-            if (old + 1 == kB1Arrivals + kB2Groups) atomicExch(p.counters + tile, 0u);
+            if (old + 1 == p.reset_at) atomicExch(p.counters + tile, 0u);
             fence_proxy_async_global();
             __threadfence_block();
             *dep_items = nitem + 1;
@@ -556,7 +569,7 @@ fused_bwd_dx_m64_kernel(const __grid_constant__ CUtensorMap tm_dy3, const __grid
             mbar_init(smem_u32(&bars.st_full[k]), 4);        // the four warps of an epilogue half
             mbar_init(smem_u32(&bars.st_free[k]), 1);
         }
-        for (int q = 0; q < kQuads; ++q) {
+        for (int q = 0; q < 4; ++q) {
             mbar_init(smem_u32(&bars.full[q]), 4);           // four loads, one per loader warp
             mbar_init(smem_u32(&bars.empty[q]), 1);
         }
@@ -577,6 +590,368 @@ fused_bwd_dx_m64_kernel(const __grid_constant__ CUtensorMap tm_dy3, const __grid
 
     if (is_b1) b1_body(tm_dy3, tm_Lt, tm_du, p, smem0, &bars, tmem_base, &dead, grp, first);
     else b2_body(tm_R, tm_dx, p, smem0, &bars, &dep_items, tmem_base, &dead, grp, first);
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem_base, 512);
+}
+
+
+// ------------------------------------------------------------------------------------------------ all-in-one kernel
+// dx, dL and dR in one launch: B1 CTAs as above (writing du and P dy to their L2-resident exchange buffers),
+// "B2R" CTAs that turn the du slabs of 8 blocks k into dx AND into dR (the same 8 KB of shared memory is the
+// K-major A operand of dx = du R and, read token-major, the A operand of dR += du^T x), and "WL" CTAs that
+// reduce dL += (P dy)^T u' for 16 blocks j.  Every consumer waits on the tile's counter, so du and P dy are read
+// back from L2 a few thousand cycles after they were written.
+
+__device__ __forceinline__ bool wait_tile(const BwdParams &p, int tile, volatile int *dead)
+{
+    const unsigned *ctr = p.counters + tile;
+    if (ld_acquire(ctr) < p.need) {
+        const unsigned long long t0 = global_timer_ns();
+        while (ld_acquire(ctr) < p.need) {
+            if (*dead || global_timer_ns() - t0 > kWaitLimitNs) {
+                *dead = 1;
+                atomicCAS(p.status, 0u, (unsigned)kErrPeerWait);
+                return false;
+            }
+        }
+    }
+    const unsigned old = atomicAdd(p.counters + tile, 1u);
+    if (old + 1 == p.reset_at) atomicExch(p.counters + tile, 0u);
+    fence_proxy_async_global();
+    __threadfence_block();
+    return true;
+}
+
+__device__ __forceinline__ void red_add_v4(float *p, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(__uint_as_float(a)),
+                 "f"(__uint_as_float(b)), "f"(__uint_as_float(c)), "f"(__uint_as_float(d))
+                 : "memory");
+}
+
+constexpr int kRSlotBytes = 16384;               // B2R / WL ring slot: two 8 KB operands of one block
+
+__device__ __forceinline__ void b2r_body(const CUtensorMap &tm_R, const CUtensorMap &tm_x, const CUtensorMap &tm_dx,
+                                         const BwdParams &p, uint32_t smem0, Bars *bars, volatile int *dep_items,
+                                         uint32_t tmem_base, volatile int *dead, int grp, int first)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int step = p.b2;
+    if (first >= p.tiles) return;
+    constexpr int NST = 2;                                             // staging buffers per epilogue half
+    const uint32_t stage0 = smem0 + kWBytes;
+    const uint32_t ring0 = stage0 + 2 * NST * kStageBytes;              // 8 slots x 16 KB, handed over in pairs
+    const uint32_t full0 = smem_u32(bars->full), empty0 = smem_u32(bars->empty);
+    const uint32_t dxf = smem_u32(&bars->acc_full[0]), dxe = smem_u32(&bars->acc_empty[0]);
+    const uint32_t drf = smem_u32(&bars->acc_full[1]);
+
+    if (warp == kCtlWarp) {
+        if (lane != 0) return;
+        const uint32_t wbar = smem_u32(&bars->w);
+        mbar_expect_tx(wbar, kWBytes);
+        for (int b = 0; b < 8; ++b) tma_load_2d(smem0 + b * 8192, &tm_R, 0, (grp * 8 + b) * kM, wbar);
+        int nitem = 0;
+        for (int tile = first; tile < p.tiles; tile += step, ++nitem) {
+            if (!wait_tile(p, tile, dead)) return;
+            *dep_items = nitem + 1;
+        }
+    } else if (warp >= kAuxWarp0 && warp < kAuxWarp0 + 2) {
+        // loaders: warp pw fills slot pw of every pair with (du slab, x tile) of block 2g + pw
+        if (lane != 0) return;
+        const int pw = warp - kAuxWarp0;
+        int nitem = 0;
+        for (int tile = first; tile < p.tiles; tile += step, ++nitem) {
+            if (!wait_count(dep_items, nitem + 1, p.status, dead)) return;
+            __threadfence_block();
+            fence_proxy_async_global();
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                const int b = g * 2 + pw;
+                if (!wait_fast(empty0 + g * 8, (nitem & 1) ^ 1, p.status, dead, kErrSlotWait)) return;
+                mbar_expect_tx(full0 + g * 8, kRSlotBytes);
+                const uint32_t slot = ring0 + b * kRSlotBytes;
+                bulk_load(slot, p.du + ((long long)tile * 64 + grp * 8 + b) * 4096, 8192, full0 + g * 8);
+                tma_load_2d(slot + 8192, &tm_x, (grp * 8 + b) * kM, tile * 64, full0 + g * 8);
+            }
+        }
+    } else if (warp == kMmaWarp) {
+        if (lane != 0) return;
+        if (!mbar_wait(smem_u32(&bars->w), 0, p.status, dead, kErrTmaWait)) return;
+        tc_fence_after();
+        constexpr uint32_t idesc_dx = make_idesc_bf16(64, 64, 0, 1);       // A = du (K = j), B = R_k^T
+        constexpr uint32_t idesc_dr = make_idesc_bf16(64, 64, 1, 1);       // A = du^T (K = t), B = x (K = t)
+        const uint64_t a_dx = make_smem_desc(0, 1024, 128, 0) | (uint64_t)(ring0 >> 4);
+        const uint64_t b_dx = make_smem_desc(0, 16, 1024, kSwizzle128) | (uint64_t)(smem0 >> 4);
+        const uint64_t a_dr = make_smem_desc(0, 128, 1024, 0) | (uint64_t)(ring0 >> 4);
+        const uint64_t b_dr = make_smem_desc(0, 16, 1024, kSwizzle128) | (uint64_t)((ring0 + 8192) >> 4);
+        uint32_t nitem = 0;
+        for (int tile = first; tile < p.tiles; tile += step, ++nitem) {
+            // dx of this tile: the single accumulator set must have been drained
+            if (!wait_fast(dxe, (nitem & 1) ^ 1, p.status, dead, kErrTmemWait)) return;
+            tc_fence_after();
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                if (!wait_fast(full0 + g * 8, nitem & 1, p.status, dead, kErrTmaWait)) return;
+                tc_fence_after();
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const int b = g * 2 + i;
+                    const uint64_t ad = a_dx + (uint64_t)(b * (kRSlotBytes >> 4));
+                    const uint64_t bd = b_dx + b * 512;
+                    const uint32_t d = tmem_base + b * 64;
+                    mma_f16_ss(d, ad, bd, idesc_dx, 0);
+                    mma_f16_ss(d, ad + 128, bd + 128, idesc_dx, 1);
+                    mma_f16_ss(d, ad + 256, bd + 256, idesc_dx, 1);
+                    mma_f16_ss(d, ad + 384, bd + 384, idesc_dx, 1);
+                }
+            }
+            mma_commit(dxf);
+            // dR += du^T x while the epilogue drains dx; each pair of slots is released after its last use
+            const uint32_t acc = nitem != 0;
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const int b = g * 2 + i;
+                    const uint64_t ad = a_dr + (uint64_t)(b * (kRSlotBytes >> 4));
+                    const uint64_t bd = b_dr + (uint64_t)(b * (kRSlotBytes >> 4));
+                    const uint32_t d = tmem_base + ((uint32_t)16 << 16) + b * 64;
+                    mma_f16_ss(d, ad, bd, idesc_dr, acc);
+                    mma_f16_ss(d, ad + 16, bd + 128, idesc_dr, 1);
+                    mma_f16_ss(d, ad + 32, bd + 256, idesc_dr, 1);
+                    mma_f16_ss(d, ad + 48, bd + 384, idesc_dr, 1);
+                }
+                mma_commit(empty0 + g * 8);
+            }
+        }
+        mma_commit(drf);
+    } else if (warp < kEpiWarps) {
+        const int q4 = warp & 3, sub = warp >> 2;
+        const uint32_t lane_base = tmem_base + ((uint32_t)(q4 * 32) << 16);
+        const int row = q4 * 16 + (lane & 15);
+        const uint32_t my_stage = stage0 + sub * NST * kStageBytes;
+        const uint32_t stf0 = smem_u32(bars->st_full) + sub * NST * 8;
+        const uint32_t stfree0 = smem_u32(bars->st_free) + sub * NST * 8;
+        const bool mine = lane < 16;                                       // dx lives in the first 16 lanes of each quarter
+        uint32_t nitem = 0, nchunk = 0;
+        for (int tile = first; tile < p.tiles; tile += step, ++nitem) {
+            if (!wait_fast(dxf, nitem & 1, p.status, dead, kErrMmaWait)) return;
+            tc_fence_after();
+#pragma unroll 1
+            for (int c = sub; c < 8; c += 2, ++nchunk) {
+                const uint32_t k = nchunk & (NST - 1);
+                const uint32_t sbuf = my_stage + k * kStageBytes;
+                if (!wait_fast(stfree0 + k * 8, ((nchunk / NST) & 1) ^ 1, p.status, dead, kErrSlotWait)) return;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t v[2][16];
+                    tmem_ld16(lane_base + c * 64 + h * 32, v[0]);
+                    tmem_ld16(lane_base + c * 64 + h * 32 + 16, v[1]);
+                    tmem_ld_wait();
+                    if (mine) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const uint32_t *w = &v[e >> 1][(e & 1) * 8];
+                            const uint32_t o0 = pack_bf16(__uint_as_float(w[0]), __uint_as_float(w[1]));
+                            const uint32_t o1 = pack_bf16(__uint_as_float(w[2]), __uint_as_float(w[3]));
+                            const uint32_t o2 = pack_bf16(__uint_as_float(w[4]), __uint_as_float(w[5]));
+                            const uint32_t o3 = pack_bf16(__uint_as_float(w[6]), __uint_as_float(w[7]));
+                            const int ch = h * 4 + e;
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sbuf + row * 128 + ((ch ^ (row & 7)) * 16)),
+                                         "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
+                        }
+                    }
+                }
+                if (c + 2 >= 8) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(dxe);
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(stf0 + k * 8);
+            }
+        }
+        // dR partial sums of this CTA's tiles: lanes 16-31 of each quarter hold row 16 q4 + lane - 16 of block b
+        if (!mbar_wait(drf, 0, p.status, dead, kErrMmaWait)) return;
+        tc_fence_after();
+        float *out = p.dR + (long long)(grp * 8) * 4096 + row * 64;
+#pragma unroll 1
+        for (int b = sub * 4; b < sub * 4 + 4; ++b) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                uint32_t v[2][16];
+                tmem_ld16(lane_base + b * 64 + h * 32, v[0]);
+                tmem_ld16(lane_base + b * 64 + h * 32 + 16, v[1]);
+                tmem_ld_wait();
+                if (!mine) {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const uint32_t *w = &v[e >> 2][(e & 3) * 4];
+                        red_add_v4(out + b * 4096 + h * 32 + e * 4, w[0], w[1], w[2], w[3]);
+                    }
+                }
+            }
+        }
+    } else if (warp >= kStoreWarp0 && warp < kStoreWarp0 + 2) {
+        if (lane != 0) return;
+        const int sub = warp - kStoreWarp0;
+        store_thread<false, NST>(p, bars, stage0, sub, first, step, dead,
+            [&](uint32_t sbuf, int tile, int c) { tma_store_2d(&tm_dx, sbuf, (grp * 8 + c) * kM, tile * 64); });
+    }
+}
+
+__device__ __forceinline__ void wl_body(const BwdParams &p, uint32_t ring0, Bars *bars, volatile int *dep_items,
+                                        uint32_t tmem_base, volatile int *dead, int grp, int first)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int step = p.b3, blk0 = grp * 16;
+    if (first >= p.tiles) return;
+    const uint32_t full0 = smem_u32(bars->full), empty0 = smem_u32(bars->empty);
+    const uint32_t accf = smem_u32(&bars->acc_full[0]);
+
+    if (warp == kCtlWarp) {
+        if (lane != 0) return;
+        int nitem = 0;
+        for (int tile = first; tile < p.tiles; tile += step, ++nitem) {
+            if (!wait_tile(p, tile, dead)) return;
+            *dep_items = nitem + 1;
+        }
+    } else if (warp >= kAuxWarp0 && warp < kAuxWarp0 + 4) {
+        // loader pw fetches slot pw of every group of four: (P dy slab, u' slab) of block blk0 + 4q + pw
+        if (lane != 0) return;
+        const int pw = warp - kAuxWarp0;
+        int g = 0, nitem = 0;
+        uint32_t ph = 0;
+        for (int tile = first; tile < p.tiles; tile += step, ++nitem) {
+            if (!wait_count(dep_items, nitem + 1, p.status, dead)) return;
+            __threadfence_block();
+            fence_proxy_async_global();
+#pragma unroll 1
+            for (int q = 0; q < 4; ++q) {
+                if (!wait_fast(empty0 + g * 8, ph ^ 1, p.status, dead, kErrSlotWait)) return;
+                const uint32_t slot = ring0 + (g * 4 + pw) * kRSlotBytes;
+                const long long run = ((long long)tile * 64 + blk0 + q * 4 + pw) * 4096;
+                mbar_expect_tx(full0 + g * 8, kRSlotBytes);
+                bulk_load(slot, p.dyp + run, 8192, full0 + g * 8);
+                bulk_load(slot + 8192, p.u + run, 8192, full0 + g * 8);
+                if (++g == kQuads) { g = 0; ph ^= 1; }
+            }
+        }
+    } else if (warp == kMmaWarp) {
+        if (lane != 0) return;
+        constexpr uint32_t idesc = make_idesc_bf16(64, 64, 1, 1);          // both operands token-major
+        const uint64_t d_run = make_smem_desc(0, 128, 1024, 0);
+        const uint64_t a_base = d_run | (uint64_t)(ring0 >> 4);
+        const uint64_t b_base = d_run | (uint64_t)((ring0 + 8192) >> 4);
+        int g = 0;
+        uint32_t ph = 0;
+        for (int tile = first; tile < p.tiles; tile += step) {
+            const uint32_t acc = tile != first;
+#pragma unroll 1
+            for (int q = 0; q < 4; ++q) {
+                if (!wait_fast(full0 + g * 8, ph, p.status, dead, kErrTmaWait)) return;
+                tc_fence_after();
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int b = q * 4 + i;
+                    const uint32_t d = tmem_base + ((uint32_t)((b >> 3) * 16) << 16) + (b & 7) * 64;
+                    const uint64_t ad = a_base + (uint64_t)((g * 4 + i) * (kRSlotBytes >> 4));
+                    const uint64_t bd = b_base + (uint64_t)((g * 4 + i) * (kRSlotBytes >> 4));
+                    mma_f16_ss(d, ad, bd, idesc, acc);
+                    mma_f16_ss(d, ad + 16, bd + 16, idesc, 1);
+                    mma_f16_ss(d, ad + 32, bd + 32, idesc, 1);
+                    mma_f16_ss(d, ad + 48, bd + 48, idesc, 1);
+                }
+                mma_commit(empty0 + g * 8);
+                if (++g == kQuads) { g = 0; ph ^= 1; }
+            }
+        }
+        mma_commit(accf);
+    } else if (warp < kEpiWarps) {
+        const int q4 = warp & 3, sub = warp >> 2;
+        if (!mbar_wait(accf, 0, p.status, dead, kErrMmaWait)) return;
+        tc_fence_after();
+        const uint32_t lane_base = tmem_base + ((uint32_t)(q4 * 32) << 16);
+        const int row = q4 * 16 + (lane & 15);
+        float *out = p.dL + (long long)(blk0 + (lane >> 4) * 8) * 4096 + row * 64;
+#pragma unroll 1
+        for (int b = sub * 4; b < sub * 4 + 4; ++b) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                uint32_t v[2][16];
+                tmem_ld16(lane_base + b * 64 + h * 32, v[0]);
+                tmem_ld16(lane_base + b * 64 + h * 32 + 16, v[1]);
+                tmem_ld_wait();
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const uint32_t *w = &v[e >> 2][(e & 3) * 4];
+                    red_add_v4(out + b * 4096 + h * 32 + e * 4, w[0], w[1], w[2], w[3]);
+                }
+            }
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+fused_bwd_all_m64_kernel(const __grid_constant__ CUtensorMap tm_dy3, const __grid_constant__ CUtensorMap tm_Lt,
+                         const __grid_constant__ CUtensorMap tm_R, const __grid_constant__ CUtensorMap tm_du,
+                         const __grid_constant__ CUtensorMap tm_dx, const __grid_constant__ CUtensorMap tm_x,
+                         const BwdParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) Bars bars;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int dead;
+    __shared__ int dep_items;
+
+    const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int warp = threadIdx.x >> 5;
+    const int n_b1 = 8 * p.b1, n_b2 = 8 * p.b2;
+    const int bid = (int)blockIdx.x;
+    const int kind = bid < n_b1 ? 0 : bid < n_b1 + n_b2 ? 1 : 2;
+    const int idx = kind == 0 ? bid : kind == 1 ? bid - n_b1 : bid - n_b1 - n_b2;
+    const int grp = kind == 2 ? idx % 4 : idx % 8;
+    const int first = kind == 2 ? idx / 4 : idx / 8;
+
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bars.w), 1);
+        for (int h = 0; h < 2; ++h) {
+            mbar_init(smem_u32(&bars.acc_full[h]), 1);
+            mbar_init(smem_u32(&bars.acc_empty[h]), kEpiWarps);
+            mbar_init(smem_u32(&bars.raw_full[h]), 1);
+            mbar_init(smem_u32(&bars.raw_empty[h]), 4);
+            mbar_init(smem_u32(&bars.a_full[h]), 4);
+            mbar_init(smem_u32(&bars.a_empty[h]), 2);        // MMA commit + the copy out of P dy
+        }
+        for (int k = 0; k < 8; ++k) {
+            mbar_init(smem_u32(&bars.st_full[k]), 4);
+            mbar_init(smem_u32(&bars.st_free[k]), 1);
+        }
+        for (int q = 0; q < 4; ++q) {
+            mbar_init(smem_u32(&bars.full[q]), kind == 1 ? 2 : 4);   // loads per group: a pair (B2R) or four (WL)
+            mbar_init(smem_u32(&bars.empty[q]), 1);
+        }
+        fence_mbar_init();
+        dead = 0;
+        dep_items = 0;
+        if (kind == 0) { tma_prefetch_desc(&tm_dy3); tma_prefetch_desc(&tm_Lt); tma_prefetch_desc(&tm_du); }
+        else if (kind == 1) { tma_prefetch_desc(&tm_R); tma_prefetch_desc(&tm_dx); tma_prefetch_desc(&tm_x); }
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&tmem_base_s), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+
+    if (kind == 0) b1_body(tm_dy3, tm_Lt, tm_du, p, smem0, &bars, tmem_base, &dead, grp, first);
+    else if (kind == 1) b2r_body(tm_R, tm_x, tm_dx, p, smem0, &bars, &dep_items, tmem_base, &dead, grp, first);
+    else wl_body(p, smem0, &bars, &dep_items, tmem_base, &dead, grp, first);
 
     tc_fence_before();
     __syncthreads();
@@ -648,6 +1023,11 @@ int launch_bwd_m64(const void *dy, const void *L, const void *R, void *dx, void 
     if (b2 > tiles) b2 = (int)tiles;
     p.b1 = b1;
     p.b2 = b2;
+    p.b3 = 0;
+    p.need = kB1Arrivals;
+    p.reset_at = kB1Arrivals + kB2Groups;
+    p.u = nullptr;
+    p.dL = p.dR = nullptr;
     p.trace = nullptr;
 #ifdef MONARCH_TRACE
     if (const char *e = getenv("MONARCH_TRACE_PTR_BWD")) p.trace = (long long *)strtoull(e, nullptr, 0);
@@ -658,6 +1038,70 @@ int launch_bwd_m64(const void *dy, const void *L, const void *R, void *dx, void 
     return MONARCH_OK;
 }
 }  // namespace
+
+// dx, dL += , dR += in one launch (see the all-in-one kernel); u = u' in the forward exchange layout
+int fused_bwd_all_m64(const void *x, const void *dy, const void *L, const void *R, const void *u, void *dx,
+                      void *du, void *dyp, float *dL, float *dR, unsigned *counters, unsigned *status,
+                      int64_t tokens, cudaStream_t s)
+{
+    using namespace tc;
+    if (tokens == 0) return MONARCH_OK;
+    const long long tiles = (tokens + 63) / 64;
+    if (tiles * 4 > (long long)kBwdCounterBytes) return MONARCH_ERR_UNSUPPORTED;
+    CUtensorMap tm_dy3, tm_Lt, tm_R, tm_du, tm_dx, tm_x;
+    {
+        const uint64_t dims[3] = {64, 64, (uint64_t)tokens}, strides[2] = {128, (uint64_t)kN * 2};
+        const uint32_t box[3] = {16, 16, 64};
+        MONARCH_TRY(encode_tmap_nd(&tm_dy3, dy, 2, 3, dims, strides, box, 32));
+        const uint64_t udims[3] = {128, 8, (uint64_t)tiles * 64}, ustrides[2] = {1024, 8192};
+        const uint32_t ubox[3] = {128, 2, 4};
+        MONARCH_TRY(encode_tmap_nd(&tm_du, du, 8, 3, udims, ustrides, ubox));
+    }
+    MONARCH_TRY(encode_tmap_2d(&tm_Lt, L, kN, kM, kM * 2, 64, 32, 64));
+    MONARCH_TRY(encode_tmap_2d(&tm_R, R, kN, kM, kM * 2, 64, 64, 128));
+    MONARCH_TRY(encode_tmap_2d(&tm_dx, dx, (uint64_t)tokens, kN, kN * 2, 64, 64, 128));
+    MONARCH_TRY(encode_tmap_2d(&tm_x, x, (uint64_t)tokens, kN, kN * 2, 64, 64, 128));
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        MONARCH_CUDA_TRY(cudaGetDevice(&dev));
+        MONARCH_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        MONARCH_CUDA_TRY(cudaFuncSetAttribute(fused_bwd_all_m64_kernel,
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+    }
+    BwdParams p;
+    p.status = status;
+    p.counters = counters;
+    p.du = (__nv_bfloat16 *)du;
+    p.dyp = (__nv_bfloat16 *)dyp;
+    p.u = (const __nv_bfloat16 *)u;
+    p.dL = dL;
+    p.dR = dR;
+    p.tokens = tokens;
+    p.tiles = (int)tiles;
+    // SM split by measured cost per tile and group (B1 ~10 k cycles, B2R ~6 k, WL ~6 k with 4 groups only);
+    // 8/6/6 CTAs per group was the best of a sweep on 148 SMs
+    int b1 = (sms * 8) / 144, b2 = (sms * 6) / 144, b3 = (sms * 6) / 144;
+    if (const char *e = getenv("MONARCH_BWD_SPLIT3")) sscanf(e, "%d,%d,%d", &b1, &b2, &b3);
+    if (b1 < 1) b1 = 1;
+    if (b2 < 1) b2 = 1;
+    if (b3 < 1) b3 = 1;
+    if (b1 > tiles) b1 = (int)tiles;
+    if (b2 > tiles) b2 = (int)tiles;
+    if (b3 > tiles) b3 = (int)tiles;
+    if (8 * b1 + 8 * b2 + 4 * b3 > sms) return MONARCH_ERR_UNSUPPORTED;   // all CTAs must be co-resident
+    p.b1 = b1;
+    p.b2 = b2;
+    p.b3 = b3;
+    p.need = kB1Arrivals + 8;                   // du from 16 store threads + P dy from 8 copy threads
+    p.reset_at = p.need + 8 + 4;                // + 8 B2R groups + 4 WL groups
+    p.trace = nullptr;
+    fused_bwd_all_m64_kernel<<<8 * b1 + 8 * b2 + 4 * b3, kThreads, kSmemBytes, s>>>(tm_dy3, tm_Lt, tm_R, tm_du, tm_dx,
+                                                                                 tm_x, p);
+    note_launch();
+    MONARCH_CUDA_TRY(cudaGetLastError());
+    return MONARCH_OK;
+}
 
 int fused_bwd_dx_m64(const void *dy, const void *L, const void *R, void *dx, int64_t tokens, void *ws,
                      cudaStream_t s)

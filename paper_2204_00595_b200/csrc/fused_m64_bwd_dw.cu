@@ -15,6 +15,8 @@
 // tile and never leaves TMEM until its tiles are done, then adds its partial sums to the output with
 // vector reductions in L2.  Summation order across CTAs is not fixed, so results can differ in the last
 // fp32 bits from run to run.
+#include <cstdlib>
+
 #include "tc_common.cuh"
 
 namespace monarch {
@@ -283,6 +285,8 @@ int fused_bwd_m64(const void *x, const void *dy, const void *L, const void *R, c
         MONARCH_TRY(fused_fwd_m64_stage1(x, R, u_own, tokens, status, s));
         u = u_own;
     }
+    static const bool split = getenv("MONARCH_BWD_SPLIT") != nullptr;     // comparison runs: two kernels
+    if (!split) return fused_bwd_all_m64(x, dy, L, R, u, dx, du, dyp, dL, dR, counters, status, tokens, s);
     MONARCH_TRY(fused_bwd_dx_m64_keep(dy, L, R, dx, du, dyp, counters, status, tokens, s));
     return launch_dw(x, u, du, dyp, dL, dR, status, tokens, s);
 }
