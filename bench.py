@@ -179,13 +179,14 @@ def time_oracle(cfg, d, target_s=12.0):
 # Kernels behind each timed call (bf16, m = 64), and the DRAM traffic one call generated under ncu
 # (profiles/fused_m64_step_workload3_ncu_full.md; captured at workload 3's full size).
 KERNELS_OF = {
-    (64, "bf16", "fwd"): "fused_fwd_m64_kernel (1 launch)",
-    (64, "bf16", "bwd"): "fused_bwd_dx_m64_kernel + fused_bwd_dw_m64_kernel (2 launches, 2 memset nodes)",
+    (64, "bf16", "fwd"): "fused_fwd_m64_team_kernel (1 launch)",
+    (64, "bf16", "bwd"): "fused_bwd_all_m64_kernel (1 launch, 2 memset nodes)",
+    (64, "bf16", "mlp_fwd"): "fused_fwd_m64_team_kernel (2 launches)",
     (64, "bf16", "bwd_dx"): "fused_bwd_dx_m64_kernel (1 launch)",
-    (64, "bf16", "bwd_dw"): "fused_fwd_m64_kernel (stage 1) + fused_bwd_dx_m64_kernel (stage 1) + "
+    (64, "bf16", "bwd_dw"): "fused_fwd_m64_kernel (stage 1 only) + fused_bwd_dx_m64_kernel (stage 1 only) + "
                             "fused_bwd_dw_m64_kernel (3 launches, 2 memset nodes)",
 }
-NCU_TRAFFIC_MB = {(3, "fwd"): 149.5, (3, "bwd"): 486.5}
+NCU_TRAFFIC_MB = {(3, "fwd"): 150.1, (3, "bwd"): 378.8}
 
 
 def main():

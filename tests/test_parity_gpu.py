@@ -189,7 +189,8 @@ def test_zero_tokens(P, impl, dtype):
         g = torch.full((2, mm, mm, mm), 5.0, dtype=torch.float32, device="cuda")
         xx = torch.zeros(1, mm * mm, dtype=td, device="cuda")
         Wm = torch.zeros(mm, mm, mm, dtype=td, device="cuda")
-        P.monarch_bwd(xx, xx.clone(), Wm, Wm.clone(), xx.clone(), g[0], g[1], 0, 0, mm * mm, mm, ws)
+        wsb = P.Workspace(max(P.monarch_workspace_bytes(P.OP_BWD, 0, mm * mm, mm, code), 256))
+        P.monarch_bwd(xx, xx.clone(), Wm, Wm.clone(), xx.clone(), g[0], g[1], 0, 0, mm * mm, mm, wsb)
         torch.cuda.synchronize()
         assert float(g.abs().max()) == 0.0
 
