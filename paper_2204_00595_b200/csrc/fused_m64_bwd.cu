@@ -1,26 +1,24 @@
-// Fused dx = M^T dy = R^T P L^T P dy for m = 64 (n = 4096), bf16 in/out, fp32 accumulation in TMEM.
+// Fused backward kernels for m = 64 (n = 4096), bf16 in/out, fp32 accumulation in TMEM:
+// dx = M^T dy = R^T P L^T P dy, and the all-in-one launch that also forms dL and dR.
 //
-// The mirror image of the fused forward kernel: one persistent launch, CTAs (one per SM) specialise in
-// one of the two adjoint stages, 64-token tiles, tcgen05.mma with M = 64, two tiles in flight per CTA,
-// the intermediate du handed over through an L2-resident exchange buffer that already has the operand
-// layout of the consumer, outputs leaving through shared-memory staging and TMA tensor stores.
+// The mirror image of the fused forward kernel: persistent launches, CTAs (one per SM) specialise, 64-token
+// tiles, tcgen05.mma with M = 64, the intermediate du handed over through an L2-resident exchange buffer that
+// already has the operand layout of the consumer, outputs staged in shared memory and written by the TMA unit.
 //
-//   B1 CTAs (4 x 2 groups (hj, hk) of `b1` CTAs): du[t][k][j] = sum_l L[j][l][k] dy[t][l*64+j] for blocks
-//       j in [16hj, 16hj+16) and columns k in [32hk, 32hk+32).  The outer permutation sits on the INPUT
-//       side here: block j needs column j of every 64-element row segment.  TMA fetches the 32-byte
-//       pieces dy[t][l][16hj..16hj+16) (whole sectors) as [64 t][16 l][16 j] chunks (32B swizzle, so that
-//       8 rows l of one token spread over all banks); four warps turn each chunk into K-major operand
-//       slices [j][l/8][t][l%8] with ldmatrix.trans / stmatrix (an 8x8 16-bit transpose per instruction
-//       pair) - the only place in the library where the permutation costs a pass over shared memory.  MMAs (N = 32) run K-step by K-step as slices arrive; L_j is used
-//       transposed straight from its row-major tile (MN-major descriptor, 64B swizzle).  The epilogue
-//       writes the 16 bytes du[t][k][8jc..8jc+8) per (t, k) into the exchange buffer
-//       [tile][k][j/8][t%64][j%8].
+//   B1 CTAs (8 groups g of `b1` CTAs): du[t][k][j] = sum_l L[j][l][k] dy[t][l*64+j] for blocks j in [8g, 8g+8)
+//       and all 64 columns k.  The outer permutation sits on the INPUT side here: block j needs column j of
+//       every 64-element row segment.  TMA gathers the 16-byte pieces dy[t][l][8g..8g+8) as [64 t][16 l][8 j]
+//       chunks; four warps turn each chunk into operand slices [j][l/8][t][l%8] with ldmatrix.trans / stmatrix
+//       (an 8x8 16-bit transpose per instruction pair) - the only place in the library where the permutation
+//       costs a pass over shared memory.  MMAs run in the transposed orientation D[k][t] (A = L_j^T from its
+//       row-major tile, B = the slice), so that a thread of the epilogue finds the 8 blocks of its row side by
+//       side and writes the 16 bytes du[t][k][8g..8g+8) of the exchange buffer [tile][k][j/8][t%64][j%8].
 //   B2 CTAs (8 groups g of `b2` CTAs): dx[t][k*64+i] = sum_j R[k][j][i] du[t][k][j] for blocks
 //       k in [8g, 8g+8).  One 8 KB bulk copy per block fetches du_k[64 x 64]; R_k is used transposed
 //       from its row-major tile (MN-major, 128B swizzle); the result rows are 128 contiguous bytes per
 //       (t, k), staged with the 128B swizzle and stored as 64 x 64 boxes.
 //
-// Waits are bounded; B1 waits on nothing outside its CTA, B2 on a per-tile counter bumped by B1.
+// Waits are bounded; B1 waits on nothing outside its CTA, the other kinds on a per-tile counter bumped by B1.
 #include <cstdio>
 #include <cstdlib>
 
@@ -38,15 +36,17 @@ constexpr int kEpiWarps = 8, kCtlWarp = 8, kMmaWarp = 9, kStoreWarp0 = 10, kAuxW
 constexpr int kThreads = 17 * 32;
 constexpr int kWBytes = 65536;                 // resident weights
 constexpr int kStageBytes = 8192;
-constexpr int kB1StagesPerHalf = 2, kB2StagesPerHalf = 4;
-constexpr int kRawBytes = 32768;                              // B1: one K-step (16 l) of 16 blocks, as loaded
+constexpr int kB2StagesPerHalf = 4;
+constexpr int kRawBytes = 16384, kRawBufs = 3;                // B1: one K-step (16 l) of 8 blocks, as loaded
 constexpr int kBlockSlice = 2048 + 16;                        // B1: one block's K-step operand, padded so that
-constexpr int kSliceBytes = 16 * kBlockSlice;                 //     the 8 rows of an stmatrix hit 8 bank groups
+constexpr int kSliceBytes = 8 * kBlockSlice;                  //     the 8 rows of an stmatrix hit 8 bank groups
+constexpr int kOutRow = 1024 + 16;                            // B1: staged output row (64 tokens x 16 B), padded
+constexpr int kOutBytes = 16 * kOutRow;                       //     one buffer per 16 rows k (TMEM quarter)
 constexpr int kSlotBytes = 8192, kSlots = 12, kQuads = 3;     // B2 operand ring
 constexpr int kSmemBytes = kWBytes + 65536 + 98304 + 512 + 1024;   // 224.5 KB (+ alignment) covers both kinds
-static_assert(kWBytes + 2 * kB1StagesPerHalf * kStageBytes + 2 * kRawBytes + 2 * kSliceBytes + 1024 <= kSmemBytes, "B1");
+static_assert(kWBytes + kRawBufs * kRawBytes + 2 * kSliceBytes + 4 * kOutBytes + 1024 <= kSmemBytes, "B1");
 static_assert(kWBytes + 2 * kB2StagesPerHalf * kStageBytes + kSlots * kSlotBytes + 1024 <= kSmemBytes, "B2");
-constexpr unsigned kB1Arrivals = 8 * 2;        // 8 B1 groups x 2 store threads per tile
+constexpr unsigned kB1Arrivals = 8;            // 8 B1 groups x 1 store thread per tile
 constexpr unsigned kB2Groups = 8;
 
 struct BwdParams {
@@ -59,6 +59,7 @@ struct BwdParams {
     int b1, b2;                // CTAs per B1 group, per B2 group
     int b3;                    // all-in-one kernel: CTAs per group of the dL kind (0 elsewhere)
     unsigned need, reset_at;   // a tile is ready at `need` arrivals; the consumer that brings it to `reset_at` clears it
+    const __nv_bfloat16 *dy;   // natural dy (for L2 prefetch hints only; the data path goes through TMA)
     const __nv_bfloat16 *u;    // all-in-one kernel: u' = P R x, [tiles][64 j][8][64 t][8] (forward exchange layout)
     float *dL, *dR;            // all-in-one kernel: gradients (added to)
     long long *trace;          // optional per-CTA timeline (debug builds), else null
@@ -76,7 +77,7 @@ struct Bars {
     uint64_t w;                               // resident weights landed
     uint64_t acc_full[2], acc_empty[2];       // TMEM accumulator sets
     uint64_t st_full[8], st_free[8];          // staging buffers (per half: B1 uses 2, B2 uses 4)
-    uint64_t raw_full[2], raw_empty[2];       // B1 raw chunks
+    uint64_t raw_full[4], raw_empty[4];       // B1 raw chunks
     uint64_t a_full[2], a_empty[2];           // B1 operand slices
     uint64_t full[4], empty[4];               // operand rings: groups of four slots (B2, dL kind) or pairs (B2R)
 };
@@ -169,67 +170,73 @@ __device__ __forceinline__ void store_thread(const BwdParams &p, Bars *bars, uin
 }
 
 // ------------------------------------------------------------------------------------------------ B1
-__device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtensorMap &tm_Lt, const CUtensorMap &tm_du,
-                                        const BwdParams &p, uint32_t smem0, Bars *bars, uint32_t tmem_base,
-                                        volatile int *dead, int grp, int first)
+// du^T_j = L_j^T (P dy)_j^T for the 8 blocks j of group g and all 64 columns k, in the "transposed" orientation
+// D[k][t] (M = k, N = tokens): A = L_j^T straight from the resident row-major tile (MN-major, 128B swizzle),
+// B = the transposed slice [l/8][t][l%8] (K-major, no swizzle).  A thread of the epilogue owns one row k and
+// finds the 8 blocks j of its group side by side in TMEM, which is exactly the 16-byte piece
+// du[t][k][8g..8g+8) of the exchange layout - no second group has to contribute to it.
+__device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtensorMap &tm_Lt, const BwdParams &p,
+                                        uint32_t smem0, Bars *bars, uint32_t tmem_base, volatile int *dead, int grp,
+                                        int first)
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int hj = grp >> 1, hk = grp & 1;
     const int step = p.b1;
     if (first >= p.tiles) return;
-    const uint32_t stage0 = smem0 + kWBytes;
-    const uint32_t raw0 = stage0 + 2 * kB1StagesPerHalf * kStageBytes;
-    const uint32_t a0 = raw0 + 2 * kRawBytes;
+    const uint32_t raw0 = smem0 + kWBytes;
+    const uint32_t a0 = raw0 + kRawBufs * kRawBytes;
+    const uint32_t out0 = a0 + 2 * kSliceBytes;
     const uint32_t rawf = smem_u32(bars->raw_full), rawe = smem_u32(bars->raw_empty);
     const uint32_t af = smem_u32(bars->a_full), ae = smem_u32(bars->a_empty);
     const uint32_t accf0 = smem_u32(bars->acc_full), acce0 = smem_u32(bars->acc_empty);
+    const uint32_t stf0 = smem_u32(bars->st_full), stfree0 = smem_u32(bars->st_free);
 
     if (warp == kCtlWarp) {
         if (lane != 0) return;
-        // resident: columns [32hk, 32hk+32) of the 16 blocks L_j, row-major [l][k] with 64B swizzle
+        // resident: the 8 blocks L_j of the group, row-major [l][k] with 128B swizzle
         const uint32_t wbar = smem_u32(&bars->w);
         mbar_expect_tx(wbar, kWBytes);
-        for (int b = 0; b < 16; ++b) tma_load_2d(smem0 + b * 4096, &tm_Lt, hk * 32, (hj * 16 + b) * kM, wbar);
-        uint32_t n = 0;
+        for (int b = 0; b < 8; ++b) tma_load_2d(smem0 + b * 8192, &tm_Lt, 0, (grp * 8 + b) * kM, wbar);
+        // gather: the 16-byte pieces dy[t][l][8g..8g+8) of one K-step (16 l) as [64 t][16 l][8 j]
+        int rb = 0;
+        uint32_t ph = 0;
         for (int tile = first; tile < p.tiles; tile += step) {
-            BTRACE(n >> 2, 0, BCLK());
 #pragma unroll 1
-            for (int ks = 0; ks < 4; ++ks, ++n) {
-                const uint32_t rb = n & 1;
-                if (!wait_fast(rawe + rb * 8, ((n >> 1) & 1) ^ 1, p.status, dead, kErrSlotWait)) return;
+            for (int ks = 0; ks < 4; ++ks) {
+                if (!wait_fast(rawe + rb * 8, ph ^ 1, p.status, dead, kErrSlotWait)) return;
                 mbar_expect_tx(rawf + rb * 8, kRawBytes);
-                tma_load_3d(raw0 + rb * kRawBytes, &tm_dy3, hj * 16, ks * 16, tile * 64, rawf + rb * 8);
+                tma_load_3d(raw0 + rb * kRawBytes, &tm_dy3, grp * 8, ks * 16, tile * 64, rawf + rb * 8);
+                if (++rb == kRawBufs) { rb = 0; ph ^= 1; }
             }
         }
     } else if (warp >= kAuxWarp0 && warp < kAuxWarp0 + 4) {
-        // transposers: raw [64 t][16 l][16 j] (16-byte halves swapped where bit 2 of l is set)
-        //           ->  slices [16 j][2 l/8][64 t][8 l]
+        // transposers: raw [64 t][16 l][8 j]  ->  slices [8 j][2 l/8][64 t][8 l]; one ldmatrix.x4.trans /
+        // stmatrix.x4 pair turns the 16 l x 8 j of two tokens
         const int tw = warp - kAuxWarp0;
         const int mi = lane >> 3, r = lane & 7;      // matrix of the x4 group, row within it
-        const int lo = mi >> 1, jo = mi & 1;
-        uint32_t n = 0;
+        const int lo = mi & 1, tt = mi >> 1;
+        int rb = 0;
+        uint32_t ph = 0, n = 0;
         [[maybe_unused]] long long w_raw = 0, w_ae = 0, w_tr = 0;
         for (int tile = first; tile < p.tiles; tile += step) {
 #pragma unroll 1
             for (int ks = 0; ks < 4; ++ks, ++n) {
-                const uint32_t rb = n & 1;
+                const uint32_t ab = n & 1;
                 [[maybe_unused]] const long long c0 = BCLK();
-                if (!wait_fast(rawf + rb * 8, (n >> 1) & 1, p.status, dead, kErrTmaWait)) return;
+                if (!wait_fast(rawf + rb * 8, ph, p.status, dead, kErrTmaWait)) return;
                 [[maybe_unused]] const long long c1 = BCLK();
-                if (!wait_fast(ae + rb * 8, ((n >> 1) & 1) ^ 1, p.status, dead, kErrSlotWait)) return;
+                if (!wait_fast(ae + ab * 8, ((n >> 1) & 1) ^ 1, p.status, dead, kErrSlotWait)) return;
                 [[maybe_unused]] const long long c2 = BCLK();
                 w_raw += c1 - c0; w_ae += c2 - c1;
-                const uint32_t src = raw0 + rb * kRawBytes + (lo * 8 + r) * 32 + ((jo ^ (r >> 2)) * 16);
-                const uint32_t dst = a0 + rb * kSliceBytes + (jo * 8 + r) * kBlockSlice + lo * 1024;
-#pragma unroll 4
-                for (int tt = 0; tt < 16; ++tt) {
-                    const int t = tw * 16 + tt;
+                const uint32_t src = raw0 + rb * kRawBytes + (tw * 16 + tt) * 256 + (lo * 8 + r) * 16;
+                const uint32_t dst = a0 + ab * kSliceBytes + r * kBlockSlice + lo * 1024 + (tw * 16 + tt) * 16;
+#pragma unroll
+                for (int it = 0; it < 8; ++it) {
                     uint32_t m0, m1, m2, m3;
                     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
                                  : "=r"(m0), "=r"(m1), "=r"(m2), "=r"(m3)
-                                 : "r"(src + t * 512)
+                                 : "r"(src + it * 512)
                                  : "memory");
-                    asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1, %2, %3, %4};" ::"r"(dst + t * 16),
+                    asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1, %2, %3, %4};" ::"r"(dst + it * 32),
                                  "r"(m0), "r"(m1), "r"(m2), "r"(m3)
                                  : "memory");
                 }
@@ -237,8 +244,9 @@ __device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtenso
                 __syncwarp();
                 if (lane == 0) {
                     mbar_arrive(rawe + rb * 8);
-                    mbar_arrive(af + rb * 8);
+                    mbar_arrive(af + ab * 8);
                 }
+                if (++rb == kRawBufs) { rb = 0; ph ^= 1; }
                 w_tr += BCLK() - c2;
             }
             if (tw == 0 && lane == 0) {
@@ -247,13 +255,13 @@ __device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtenso
             w_raw = w_ae = w_tr = 0;
         }
     } else if (warp == kDypWarp) {
-        // the operand slices are P dy in 2 KB runs [l/8 2][t 64][8 l] per block j: copy them out.  The two
-        // groups that share these 16 blocks (hk = 0, 1) build identical slices; each writes every other one.
-        if (lane != 0 || p.dyp == nullptr) return;
+        // the operand slices are P dy in 2 KB runs [l/8 2][t 64][8 l] per block j: copy them out, one lane per
+        // block (a bulk copy costs its issuing thread 100+ cycles)
         uint32_t n = 0;
-        int held = -1;                       // buffer whose copy is still in flight
+        int held = -1;                       // buffer whose copy may still be reading shared memory
+        const bool want = p.dyp != nullptr;
         for (int tile = first; tile < p.tiles; tile += step) {
-            __nv_bfloat16 *dst = p.dyp + ((long long)tile * 64 + hj * 16) * 4096;
+            __nv_bfloat16 *dst = p.dyp + ((long long)tile * 64 + grp * 8) * 4096;
 #pragma unroll 1
             for (int ks = 0; ks < 4; ++ks, ++n) {
                 const uint32_t ab = n & 1;
@@ -262,27 +270,32 @@ __device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtenso
                     // the slice before this one has been read out by now (its buffer is only needed
                     // again after the current slice, which is already transposed)
                     tma_store_wait_read<0>();
-                    mbar_arrive(ae + held * 8);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(ae + held * 8);
                     held = -1;
                 }
-                if ((ks & 1) == hk) {
-#pragma unroll 4
-                    for (int j = 0; j < 16; ++j)
-                        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst + j * 4096 + ks * 1024),
-                                     "r"(a0 + ab * kSliceBytes + j * kBlockSlice), "r"(2048) : "memory");
+                if (want) {
+                    if (lane < 8)
+                        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst + lane * 4096 + ks * 1024),
+                                     "r"(a0 + ab * kSliceBytes + lane * kBlockSlice), "r"(2048) : "memory");
                     tma_store_commit();
                     held = (int)ab;
-                } else {
+                } else if (lane == 0) {
                     mbar_arrive(ae + ab * 8);
                 }
             }
-            if (p.b3 > 0) {
+            if (want && p.b3 > 0) {
                 // another kind of CTA of this launch reads P dy back: publish the tile once the copies are complete
                 tma_store_wait_all<0>();
-                if (held >= 0) { mbar_arrive(ae + held * 8); held = -1; }
+                __syncwarp();
+                if (lane == 0 && held >= 0) mbar_arrive(ae + held * 8);
+                held = -1;
                 fence_proxy_async_global();
-                __threadfence();
-                atomicAdd(p.counters + tile, 1u);
+                __syncwarp();
+                if (lane == 0) {
+                    __threadfence();
+                    atomicAdd(p.counters + tile, 1u);
+                }
             }
         }
         tma_store_wait_all<0>();
@@ -290,16 +303,18 @@ __device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtenso
         if (lane != 0) return;
         if (!mbar_wait(smem_u32(&bars->w), 0, p.status, dead, kErrTmaWait)) return;
         tc_fence_after();
-        constexpr uint32_t idesc = make_idesc_bf16(64, 32, 0, 1);          // B = L_j^T: MN-major
-        const uint64_t a_ns = make_smem_desc(0, 1024, 128, 0);
-        const uint64_t b_mn = make_smem_desc(0, 16, 512, kSwizzle64) | (uint64_t)(smem0 >> 4);
+        constexpr uint32_t idesc = make_idesc_bf16(64, 64, 1, 0);          // A = L_j^T: MN-major; B = slice: K-major
+        const uint64_t a_mn = make_smem_desc(0, 16, 1024, kSwizzle128) | (uint64_t)(smem0 >> 4);
+        const uint64_t b_ns = make_smem_desc(0, 1024, 128, 0);
         uint32_t n = 0, nitem = 0;
-        [[maybe_unused]] long long w_af = 0;
         for (int tile = first; tile < p.tiles; tile += step, ++nitem) {
             const uint32_t buf = nitem & 1, par = (nitem >> 1) & 1;
+            [[maybe_unused]] const long long m0 = BCLK();
             if (!wait_fast(acce0 + buf * 8, par ^ 1, p.status, dead, kErrTmemWait)) return;
             tc_fence_after();
-            const uint32_t dbase = tmem_base + buf * 256;
+            [[maybe_unused]] long long w_af = 0;
+            BTRACE(nitem, 0, BCLK() - m0);
+            const uint32_t dbase = tmem_base + ((buf * 16) << 16);
 #pragma unroll 1
             for (int ks = 0; ks < 4; ++ks, ++n) {
                 const uint32_t ab = n & 1;
@@ -307,73 +322,89 @@ __device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtenso
                 if (!wait_fast(af + ab * 8, (n >> 1) & 1, p.status, dead, kErrTmaWait)) return;
                 tc_fence_after();
                 w_af += BCLK() - c0;
-                const uint64_t as = a_ns | (uint64_t)((a0 + ab * kSliceBytes) >> 4);
-                const uint64_t bs = b_mn + ks * 64;                           // 16 rows of 64 B
+                const uint64_t as = a_mn + ks * 128;                          // 16 rows l of 128 B
+                const uint64_t bs = b_ns | (uint64_t)((a0 + ab * kSliceBytes) >> 4);
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const uint32_t d = dbase + ((uint32_t)((j >> 3) * 16) << 16) + (j & 7) * 32;
-                    mma_f16_ss(d, as + j * (kBlockSlice >> 4), bs + j * 256, idesc, ks != 0);
-                }
+                for (int j = 0; j < 8; ++j)
+                    mma_f16_ss(dbase + j * 64, as + j * 512, bs + j * (kBlockSlice >> 4), idesc, ks != 0);
                 mma_commit(ae + ab * 8);
             }
             mma_commit(accf0 + buf * 8);
             BTRACE(nitem, 4, w_af); BTRACE(nitem, 5, BCLK());
-            w_af = 0;
         }
     } else if (warp < kEpiWarps) {
+        // lane -> row k = 16 q4 + lane % 16 of the tile in lane half `buf`; the two warps of a quarter take
+        // 32 tokens each and fill one staging buffer [16 k][64 t][16 B] (rows padded against bank conflicts)
         const int q4 = warp & 3, sub = warp >> 2;
         const uint32_t lane_base = tmem_base + ((uint32_t)(q4 * 32) << 16);
-        const int row = q4 * 16 + (lane & 15);
-        constexpr int NST = kB1StagesPerHalf;
-        const uint32_t my_stage = stage0 + sub * NST * kStageBytes;
-        const uint32_t stf0 = smem_u32(bars->st_full) + sub * NST * 8;
-        const uint32_t stfree0 = smem_u32(bars->st_free) + sub * NST * 8;
-        uint32_t nitem = 0, nchunk = 0;
+        const uint32_t obuf = out0 + q4 * kOutBytes + (lane & 15) * kOutRow;
+        uint32_t nitem = 0;
         for (int tile = first; tile < p.tiles; tile += step, ++nitem) {
             const uint32_t buf = nitem & 1, par = (nitem >> 1) & 1;
             if (!wait_fast(accf0 + buf * 8, par, p.status, dead, kErrMmaWait)) return;
-            if (threadIdx.x == 0) BTRACE(nitem, 6, BCLK());
             tc_fence_after();
+            [[maybe_unused]] const long long e0 = BCLK();
+            if (!wait_fast(stfree0 + q4 * 8, (nitem & 1) ^ 1, p.status, dead, kErrSlotWait)) return;
+            if (threadIdx.x == 0) BTRACE(nitem, 6, BCLK() - e0);
+            const bool mine = (uint32_t)(lane >> 4) == buf;
 #pragma unroll 1
-            for (int c = sub; c < 8; c += 2, ++nchunk) {
-                const uint32_t k = nchunk & (NST - 1);
-                const uint32_t sbuf = my_stage + k * kStageBytes;
-                if (!wait_fast(stfree0 + k * 8, ((nchunk / NST) & 1) ^ 1, p.status, dead, kErrSlotWait)) return;
-                // chunk = 4 consecutive columns k; lanes i and i+16 hold blocks j 0-7 and 8-15
-                uint32_t v[8][4];
+            for (int c = 0; c < 4; ++c) {
+                const int t0 = sub * 32 + c * 8;
+                uint32_t v[8][8];
 #pragma unroll
-                for (int a = 0; a < 8; ++a) tmem_ld4(lane_base + buf * 256 + a * 32 + c * 4, v[a]);
+                for (int b = 0; b < 8; ++b) tmem_ld8(lane_base + b * 64 + t0, v[b]);
                 tmem_ld_wait();
+                if (mine) {
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const uint32_t o0 = pack_bf16(__uint_as_float(v[0][q]), __uint_as_float(v[1][q]));
-                    const uint32_t o1 = pack_bf16(__uint_as_float(v[2][q]), __uint_as_float(v[3][q]));
-                    const uint32_t o2 = pack_bf16(__uint_as_float(v[4][q]), __uint_as_float(v[5][q]));
-                    const uint32_t o3 = pack_bf16(__uint_as_float(v[6][q]), __uint_as_float(v[7][q]));
-                    // staging [k local 4][j/8 local 2][t 64][8 j]
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sbuf + q * 2048 + (lane >> 4) * 1024 + row * 16),
-                                 "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
+                    for (int t = 0; t < 8; ++t) {
+                        const uint32_t o0 = pack_bf16(__uint_as_float(v[0][t]), __uint_as_float(v[1][t]));
+                        const uint32_t o1 = pack_bf16(__uint_as_float(v[2][t]), __uint_as_float(v[3][t]));
+                        const uint32_t o2 = pack_bf16(__uint_as_float(v[4][t]), __uint_as_float(v[5][t]));
+                        const uint32_t o3 = pack_bf16(__uint_as_float(v[6][t]), __uint_as_float(v[7][t]));
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(obuf + (t0 + t) * 16),
+                                     "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
+                    }
                 }
-                if (c + 2 >= 8) {
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(acce0 + buf * 8);
-                }
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(stf0 + k * 8);
             }
-            if (threadIdx.x == 0) BTRACE(nitem, 7, BCLK());
+            tc_fence_before();
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(acce0 + buf * 8);
+                mbar_arrive(stf0 + q4 * 8);
+            }
+            if (threadIdx.x == 0) BTRACE(nitem, 7, BCLK() - e0);
         }
-    } else if (warp >= kStoreWarp0 && warp < kStoreWarp0 + 2) {
-        if (lane != 0) return;
-        const int sub = warp - kStoreWarp0;
-        store_thread<true, kB1StagesPerHalf>(p, bars, stage0, sub, first, step, dead,
-            [&](uint32_t sbuf, int tile, int c) {
-                // du as 8-byte words [tile*64 + k][j/8][128]: 4 rows k x 2 j/8 x 1 KB
-                asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(&tm_du),
-                             "r"(sbuf), "r"(0), "r"(2 * hj), "r"(tile * 64 + hk * 32 + c * 4) : "memory");
-            });
+    } else if (warp == kStoreWarp0) {
+        // copy the staged rows out: 1 KB per (k, group) into du[tile][k][j/8 = g][t][j%8].  A bulk copy costs
+        // its issuing thread 100+ cycles, so 16 lanes issue one row each per staging buffer.
+        uint32_t nitem = 0;
+        for (int tile = first; tile < p.tiles; tile += step, ++nitem) {
+            __nv_bfloat16 *dst = p.du + (((long long)tile * 64) * 8 + grp) * 512;
+#pragma unroll 1
+            for (int q4 = 0; q4 < 4; ++q4) {
+                if (!wait_fast(stf0 + q4 * 8, nitem & 1, p.status, dead, kErrMmaWait)) return;
+                if (lane < 16)
+                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst + (long long)(q4 * 16 + lane) * 4096),
+                                 "r"(out0 + q4 * kOutBytes + lane * kOutRow), "r"(1024) : "memory");
+            }
+            tma_store_commit();
+            tma_store_wait_read<0>();
+            __syncwarp();
+            if (lane == 0)
+                for (int q4 = 0; q4 < 4; ++q4) mbar_arrive(stfree0 + q4 * 8);
+            if (p.b2 > 0) {
+                // publish the tile (nothing to publish to in a launch without consumers)
+                tma_store_wait_all<0>();
+                fence_proxy_async_global();
+                __syncwarp();
+                if (lane == 0) {
+                    __threadfence();
+                    atomicAdd(p.counters + tile, 1u);
+                }
+            }
+        }
+        tma_store_wait_all<0>();
     }
 }
 
@@ -560,13 +591,16 @@ fused_bwd_dx_m64_kernel(const __grid_constant__ CUtensorMap tm_dy3, const __grid
         for (int h = 0; h < 2; ++h) {
             mbar_init(smem_u32(&bars.acc_full[h]), 1);
             mbar_init(smem_u32(&bars.acc_empty[h]), kEpiWarps);
+            mbar_init(smem_u32(&bars.a_full[h]), 4);
+            mbar_init(smem_u32(&bars.a_empty[h]), 2);        // MMA commit + the copy-out thread
+        }
+        for (int h = 0; h < 4; ++h) {
             mbar_init(smem_u32(&bars.raw_full[h]), 1);
             mbar_init(smem_u32(&bars.raw_empty[h]), 4);      // the four transposer warps
-            mbar_init(smem_u32(&bars.a_full[h]), 4);
-            mbar_init(smem_u32(&bars.a_empty[h]), p.dyp ? 2 : 1);   // MMA commit (+ the copy out)
         }
         for (int k = 0; k < 8; ++k) {
-            mbar_init(smem_u32(&bars.st_full[k]), 4);        // the four warps of an epilogue half
+            // B1: the two warps of a TMEM quarter; B2: the four warps of an epilogue half
+            mbar_init(smem_u32(&bars.st_full[k]), is_b1 ? 2 : 4);
             mbar_init(smem_u32(&bars.st_free[k]), 1);
         }
         for (int q = 0; q < 4; ++q) {
@@ -576,7 +610,7 @@ fused_bwd_dx_m64_kernel(const __grid_constant__ CUtensorMap tm_dy3, const __grid
         fence_mbar_init();
         dead = 0;
         dep_items = 0;
-        if (is_b1) { tma_prefetch_desc(&tm_dy3); tma_prefetch_desc(&tm_Lt); tma_prefetch_desc(&tm_du); }
+        if (is_b1) { tma_prefetch_desc(&tm_dy3); tma_prefetch_desc(&tm_Lt); }
         else { tma_prefetch_desc(&tm_R); tma_prefetch_desc(&tm_dx); }
     }
     if (warp == 0) {
@@ -588,7 +622,7 @@ fused_bwd_dx_m64_kernel(const __grid_constant__ CUtensorMap tm_dy3, const __grid
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
 
-    if (is_b1) b1_body(tm_dy3, tm_Lt, tm_du, p, smem0, &bars, tmem_base, &dead, grp, first);
+    if (is_b1) b1_body(tm_dy3, tm_Lt, p, smem0, &bars, tmem_base, &dead, grp, first);
     else b2_body(tm_R, tm_dx, p, smem0, &bars, &dep_items, tmem_base, &dead, grp, first);
 
     tc_fence_before();
@@ -921,13 +955,15 @@ fused_bwd_all_m64_kernel(const __grid_constant__ CUtensorMap tm_dy3, const __gri
         for (int h = 0; h < 2; ++h) {
             mbar_init(smem_u32(&bars.acc_full[h]), 1);
             mbar_init(smem_u32(&bars.acc_empty[h]), kEpiWarps);
+            mbar_init(smem_u32(&bars.a_full[h]), 4);
+            mbar_init(smem_u32(&bars.a_empty[h]), 2);        // MMA commit + the copy-out thread
+        }
+        for (int h = 0; h < 4; ++h) {
             mbar_init(smem_u32(&bars.raw_full[h]), 1);
             mbar_init(smem_u32(&bars.raw_empty[h]), 4);
-            mbar_init(smem_u32(&bars.a_full[h]), 4);
-            mbar_init(smem_u32(&bars.a_empty[h]), 2);        // MMA commit + the copy out of P dy
         }
         for (int k = 0; k < 8; ++k) {
-            mbar_init(smem_u32(&bars.st_full[k]), 4);
+            mbar_init(smem_u32(&bars.st_full[k]), kind == 0 ? 2 : 4);
             mbar_init(smem_u32(&bars.st_free[k]), 1);
         }
         for (int q = 0; q < 4; ++q) {
@@ -937,7 +973,7 @@ fused_bwd_all_m64_kernel(const __grid_constant__ CUtensorMap tm_dy3, const __gri
         fence_mbar_init();
         dead = 0;
         dep_items = 0;
-        if (kind == 0) { tma_prefetch_desc(&tm_dy3); tma_prefetch_desc(&tm_Lt); tma_prefetch_desc(&tm_du); }
+        if (kind == 0) { tma_prefetch_desc(&tm_dy3); tma_prefetch_desc(&tm_Lt); }
         else if (kind == 1) { tma_prefetch_desc(&tm_R); tma_prefetch_desc(&tm_dx); tma_prefetch_desc(&tm_x); }
     }
     if (warp == 0) {
@@ -949,7 +985,7 @@ fused_bwd_all_m64_kernel(const __grid_constant__ CUtensorMap tm_dy3, const __gri
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
 
-    if (kind == 0) b1_body(tm_dy3, tm_Lt, tm_du, p, smem0, &bars, tmem_base, &dead, grp, first);
+    if (kind == 0) b1_body(tm_dy3, tm_Lt, p, smem0, &bars, tmem_base, &dead, grp, first);
     else if (kind == 1) b2r_body(tm_R, tm_x, tm_dx, p, smem0, &bars, &dep_items, tmem_base, &dead, grp, first);
     else wl_body(p, smem0, &bars, &dep_items, tmem_base, &dead, grp, first);
 
@@ -982,16 +1018,16 @@ int launch_bwd_m64(const void *dy, const void *L, const void *R, void *dx, void 
     if (tiles * 4 > (long long)kBwdCounterBytes) return MONARCH_ERR_UNSUPPORTED;
     CUtensorMap tm_dy3, tm_Lt, tm_R, tm_du, tm_dx;
     {
-        // dy as [t][l][j]: a load brings 16 j x 16 l x 64 t (32-byte pieces)
+        // dy as [t][l][j]: a load brings 8 j x 16 l x 64 t (16-byte pieces)
         const uint64_t dims[3] = {64, 64, (uint64_t)tokens}, strides[2] = {128, (uint64_t)kN * 2};
-        const uint32_t box[3] = {16, 16, 64};
-        MONARCH_TRY(encode_tmap_nd(&tm_dy3, dy, 2, 3, dims, strides, box, 32));
+        const uint32_t box[3] = {8, 16, 64};
+        MONARCH_TRY(encode_tmap_nd(&tm_dy3, dy, 2, 3, dims, strides, box));
         // exchange buffer as 8-byte words [tile*64 + k][j/8][128]; a store moves 4 k x 2 j/8 x 1 KB
         const uint64_t udims[3] = {128, 8, (uint64_t)tiles * 64}, ustrides[2] = {1024, 8192};
         const uint32_t ubox[3] = {128, 2, 4};
         MONARCH_TRY(encode_tmap_nd(&tm_du, du, 8, 3, udims, ustrides, ubox));
     }
-    MONARCH_TRY(encode_tmap_2d(&tm_Lt, L, kN, kM, kM * 2, 64, 32, 64));      // [64 l][32 k] per block, 64B swizzle
+    MONARCH_TRY(encode_tmap_2d(&tm_Lt, L, kN, kM, kM * 2, 64, 64, 128));     // [64 l][64 k] per block, 128B swizzle
     if (both) {
         MONARCH_TRY(encode_tmap_2d(&tm_R, R, kN, kM, kM * 2, 64, 64, 128));
         MONARCH_TRY(encode_tmap_2d(&tm_dx, dx, (uint64_t)tokens, kN, kN * 2, 64, 64, 128));
@@ -1012,9 +1048,10 @@ int launch_bwd_m64(const void *dy, const void *L, const void *R, void *dx, void 
     p.counters = counters;
     p.du = (__nv_bfloat16 *)du;
     p.dyp = (__nv_bfloat16 *)dyp;
+    p.dy = (const __nv_bfloat16 *)dy;
     p.tokens = tokens;
     p.tiles = (int)tiles;
-    // B1 issues twice the MMAs (N = 32) and transposes its input: about 60 % of the SMs
+    // B1 gathers narrow rows and transposes its input: about 60 % of the SMs
     int b1 = both ? (sms * 3 + 20) / 40 : sms / 8;
     if (b1 < 1) b1 = 1;
     int b2 = both ? (sms - 8 * b1) / 8 : 0;
@@ -1051,13 +1088,13 @@ int fused_bwd_all_m64(const void *x, const void *dy, const void *L, const void *
     CUtensorMap tm_dy3, tm_Lt, tm_R, tm_du, tm_dx, tm_x;
     {
         const uint64_t dims[3] = {64, 64, (uint64_t)tokens}, strides[2] = {128, (uint64_t)kN * 2};
-        const uint32_t box[3] = {16, 16, 64};
-        MONARCH_TRY(encode_tmap_nd(&tm_dy3, dy, 2, 3, dims, strides, box, 32));
+        const uint32_t box[3] = {8, 16, 64};
+        MONARCH_TRY(encode_tmap_nd(&tm_dy3, dy, 2, 3, dims, strides, box));
         const uint64_t udims[3] = {128, 8, (uint64_t)tiles * 64}, ustrides[2] = {1024, 8192};
         const uint32_t ubox[3] = {128, 2, 4};
         MONARCH_TRY(encode_tmap_nd(&tm_du, du, 8, 3, udims, ustrides, ubox));
     }
-    MONARCH_TRY(encode_tmap_2d(&tm_Lt, L, kN, kM, kM * 2, 64, 32, 64));
+    MONARCH_TRY(encode_tmap_2d(&tm_Lt, L, kN, kM, kM * 2, 64, 64, 128));
     MONARCH_TRY(encode_tmap_2d(&tm_R, R, kN, kM, kM * 2, 64, 64, 128));
     MONARCH_TRY(encode_tmap_2d(&tm_dx, dx, (uint64_t)tokens, kN, kN * 2, 64, 64, 128));
     MONARCH_TRY(encode_tmap_2d(&tm_x, x, (uint64_t)tokens, kN, kN * 2, 64, 64, 128));
@@ -1074,6 +1111,7 @@ int fused_bwd_all_m64(const void *x, const void *dy, const void *L, const void *
     p.counters = counters;
     p.du = (__nv_bfloat16 *)du;
     p.dyp = (__nv_bfloat16 *)dyp;
+    p.dy = (const __nv_bfloat16 *)dy;
     p.u = (const __nv_bfloat16 *)u;
     p.dL = dL;
     p.dR = dR;
@@ -1093,7 +1131,7 @@ int fused_bwd_all_m64(const void *x, const void *dy, const void *L, const void *
     p.b1 = b1;
     p.b2 = b2;
     p.b3 = b3;
-    p.need = kB1Arrivals + 8;                   // du from 16 store threads + P dy from 8 copy threads
+    p.need = kB1Arrivals + 8;                   // du from 8 store threads + P dy from 8 copy threads
     p.reset_at = p.need + 8 + 4;                // + 8 B2R groups + 4 WL groups
     p.trace = nullptr;
     fused_bwd_all_m64_kernel<<<8 * b1 + 8 * b2 + 4 * b3, kThreads, kSmemBytes, s>>>(tm_dy3, tm_Lt, tm_R, tm_du, tm_dx,
