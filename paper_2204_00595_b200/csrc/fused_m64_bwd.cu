@@ -46,7 +46,7 @@ constexpr int kSlotBytes = 8192, kSlots = 12, kQuads = 3;     // B2 operand ring
 constexpr int kSmemBytes = kWBytes + 65536 + 98304 + 512 + 1024;   // 224.5 KB (+ alignment) covers both kinds
 static_assert(kWBytes + kRawBufs * kRawBytes + 2 * kSliceBytes + 4 * kOutBytes + 1024 <= kSmemBytes, "B1");
 static_assert(kWBytes + 2 * kB2StagesPerHalf * kStageBytes + kSlots * kSlotBytes + 1024 <= kSmemBytes, "B2");
-constexpr unsigned kB1Arrivals = 8;            // 8 B1 groups x 1 store thread per tile
+constexpr unsigned kB1Arrivals = 8 * 2;        // 8 B1 groups x 2 store warps per tile
 constexpr unsigned kB2Groups = 8;
 
 struct BwdParams {
@@ -255,50 +255,38 @@ __device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtenso
             w_raw = w_ae = w_tr = 0;
         }
     } else if (warp == kDypWarp) {
-        // the operand slices are P dy in 2 KB runs [l/8 2][t 64][8 l] per block j: copy them out, one lane per
-        // block (a bulk copy costs its issuing thread 100+ cycles)
+        // the operand slices are P dy in 2 KB runs [l/8 2][t 64][8 l] per block j: copy them out with plain
+        // coalesced stores (512 contiguous bytes per warp instruction; the TMA unit is busy gathering)
         uint32_t n = 0;
-        int held = -1;                       // buffer whose copy may still be reading shared memory
         const bool want = p.dyp != nullptr;
         for (int tile = first; tile < p.tiles; tile += step) {
-            __nv_bfloat16 *dst = p.dyp + ((long long)tile * 64 + grp * 8) * 4096;
+            char *dst = reinterpret_cast<char *>(p.dyp + ((long long)tile * 64 + grp * 8) * 4096) + lane * 16;
 #pragma unroll 1
             for (int ks = 0; ks < 4; ++ks, ++n) {
                 const uint32_t ab = n & 1;
                 if (!wait_fast(af + ab * 8, (n >> 1) & 1, p.status, dead, kErrTmaWait)) return;
-                if (held >= 0) {
-                    // the slice before this one has been read out by now (its buffer is only needed
-                    // again after the current slice, which is already transposed)
-                    tma_store_wait_read<0>();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(ae + held * 8);
-                    held = -1;
-                }
                 if (want) {
-                    if (lane < 8)
-                        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst + lane * 4096 + ks * 1024),
-                                     "r"(a0 + ab * kSliceBytes + lane * kBlockSlice), "r"(2048) : "memory");
-                    tma_store_commit();
-                    held = (int)ab;
-                } else if (lane == 0) {
-                    mbar_arrive(ae + ab * 8);
+                    const uint32_t src = a0 + ab * kSliceBytes + lane * 16;
+#pragma unroll 4
+                    for (int i = 0; i < 32; ++i) {
+                        const int j = i >> 2, off = (i & 3) * 512;
+                        uint4 v;
+                        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                     : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                                     : "r"(src + j * kBlockSlice + off));
+                        *reinterpret_cast<uint4 *>(dst + (long long)j * 8192 + ks * 2048 + off) = v;
+                    }
+                    __syncwarp();
                 }
+                if (lane == 0) mbar_arrive(ae + ab * 8);
             }
             if (want && p.b3 > 0) {
-                // another kind of CTA of this launch reads P dy back: publish the tile once the copies are complete
-                tma_store_wait_all<0>();
+                // another kind of CTA of this launch reads P dy back: publish the tile
+                __threadfence();
                 __syncwarp();
-                if (lane == 0 && held >= 0) mbar_arrive(ae + held * 8);
-                held = -1;
-                fence_proxy_async_global();
-                __syncwarp();
-                if (lane == 0) {
-                    __threadfence();
-                    atomicAdd(p.counters + tile, 1u);
-                }
+                if (lane == 0) atomicAdd(p.counters + tile, 1u);
             }
         }
-        tma_store_wait_all<0>();
     } else if (warp == kMmaWarp) {
         if (lane != 0) return;
         if (!mbar_wait(smem_u32(&bars->w), 0, p.status, dead, kErrTmaWait)) return;
@@ -375,36 +363,38 @@ __device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtenso
             }
             if (threadIdx.x == 0) BTRACE(nitem, 7, BCLK() - e0);
         }
-    } else if (warp == kStoreWarp0) {
-        // copy the staged rows out: 1 KB per (k, group) into du[tile][k][j/8 = g][t][j%8].  A bulk copy costs
-        // its issuing thread 100+ cycles, so 16 lanes issue one row each per staging buffer.
+    } else if (warp == kStoreWarp0 || warp == kStoreWarp0 + 1) {
+        // copy the staged rows out: 1 KB per (k, group) into du[tile][k][j/8 = g][t][j%8].  Plain coalesced
+        // stores (a warp writes 512 contiguous bytes), two quarters per warp: the TMA unit of a B1 SM is busy
+        // gathering narrow rows, and bulk copies queued behind those gathers released the staging buffers
+        // thousands of cycles late.
+        const int sw = warp - kStoreWarp0;
         uint32_t nitem = 0;
         for (int tile = first; tile < p.tiles; tile += step, ++nitem) {
-            __nv_bfloat16 *dst = p.du + (((long long)tile * 64) * 8 + grp) * 512;
+            char *dst = reinterpret_cast<char *>(p.du + (((long long)tile * 64) * 8 + grp) * 512);
 #pragma unroll 1
-            for (int q4 = 0; q4 < 4; ++q4) {
+            for (int qq = 0; qq < 2; ++qq) {
+                const int q4 = sw * 2 + qq;
                 if (!wait_fast(stf0 + q4 * 8, nitem & 1, p.status, dead, kErrMmaWait)) return;
-                if (lane < 16)
-                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst + (long long)(q4 * 16 + lane) * 4096),
-                                 "r"(out0 + q4 * kOutBytes + lane * kOutRow), "r"(1024) : "memory");
-            }
-            tma_store_commit();
-            tma_store_wait_read<0>();
-            __syncwarp();
-            if (lane == 0)
-                for (int q4 = 0; q4 < 4; ++q4) mbar_arrive(stfree0 + q4 * 8);
-            if (p.b2 > 0) {
-                // publish the tile (nothing to publish to in a launch without consumers)
-                tma_store_wait_all<0>();
-                fence_proxy_async_global();
-                __syncwarp();
-                if (lane == 0) {
-                    __threadfence();
-                    atomicAdd(p.counters + tile, 1u);
+#pragma unroll 4
+                for (int i = 0; i < 32; ++i) {
+                    const int r = i >> 1, off = (i & 1) * 512 + lane * 16;      // row k = 16 q4 + r, byte offset in it
+                    uint4 v;
+                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                                 : "r"(out0 + q4 * kOutBytes + r * kOutRow + off));
+                    *reinterpret_cast<uint4 *>(dst + (long long)(q4 * 16 + r) * 8192 + off) = v;
                 }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(stfree0 + q4 * 8);
+            }
+            if (p.b2 > 0) {
+                // publish this warp's half of the tile (nothing to publish to in a launch without consumers)
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) atomicAdd(p.counters + tile, 1u);
             }
         }
-        tma_store_wait_all<0>();
     }
 }
 
@@ -1131,7 +1121,7 @@ int fused_bwd_all_m64(const void *x, const void *dy, const void *L, const void *
     p.b1 = b1;
     p.b2 = b2;
     p.b3 = b3;
-    p.need = kB1Arrivals + 8;                   // du from 8 store threads + P dy from 8 copy threads
+    p.need = kB1Arrivals + 8;                   // du from 16 store warps + P dy from 8 copy warps
     p.reset_at = p.need + 8 + 4;                // + 8 B2R groups + 4 WL groups
     p.trace = nullptr;
     fused_bwd_all_m64_kernel<<<8 * b1 + 8 * b2 + 4 * b3, kThreads, kSmemBytes, s>>>(tm_dy3, tm_Lt, tm_R, tm_du, tm_dx,
