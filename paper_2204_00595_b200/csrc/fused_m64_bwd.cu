@@ -1041,10 +1041,12 @@ int launch_bwd_m64(const void *dy, const void *L, const void *R, void *dx, void 
     p.dy = (const __nv_bfloat16 *)dy;
     p.tokens = tokens;
     p.tiles = (int)tiles;
-    // B1 gathers narrow rows and transposes its input: about 60 % of the SMs
-    int b1 = both ? (sms * 3 + 20) / 40 : sms / 8;
+    // B1 gathers narrow rows (its TMA unit handles about one 16-byte row per 1.2 cycles) and transposes its
+    // input: two thirds of the SMs (12 + 6 CTAs per group was the best of a sweep on 148 SMs)
+    int b1 = both ? (sms * 12) / 148 : sms / 8;
     if (b1 < 1) b1 = 1;
     int b2 = both ? (sms - 8 * b1) / 8 : 0;
+    if (const char *e = getenv("MONARCH_BWD_SPLIT2")) { if (both) sscanf(e, "%d,%d", &b1, &b2); }
     if (both && b2 < 1) b2 = 1;
     if (b1 > tiles) b1 = (int)tiles;
     if (b2 > tiles) b2 = (int)tiles;
