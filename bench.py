@@ -186,7 +186,7 @@ KERNELS_OF = {
     (64, "bf16", "bwd_dw"): "fused_fwd_m64_kernel (stage 1 only) + fused_bwd_dx_m64_kernel (stage 1 only) + "
                             "fused_bwd_dw_m64_kernel (3 launches, 2 memset nodes)",
 }
-NCU_TRAFFIC_MB = {(3, "fwd"): 150.1, (3, "bwd"): 378.8}
+NCU_TRAFFIC_MB = {(3, "fwd"): 150.0, (3, "bwd"): 365.6}
 
 
 def main():
