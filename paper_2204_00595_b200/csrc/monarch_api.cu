@@ -74,7 +74,9 @@ bool fused_available(int op, int m, int dtype)
 // true when the call can run as a chain of tensor-core stages through the workspace
 bool tc_staged_available(int op, int m, int dtype)
 {
-    return dtype == MONARCH_BF16 && m >= 32 && (op == MONARCH_OP_FWD || op == MONARCH_OP_MLP_FWD);
+    if (dtype != MONARCH_BF16 || m < 32) return false;
+    if (op == MONARCH_OP_FWD || op == MONARCH_OP_MLP_FWD || op == MONARCH_OP_BWD_DX) return true;
+    return m == 128;      // dL, dR: the token-reduction kernel is built for 128 x 128 blocks
 }
 
 // kernel family for a call under the current selection
@@ -101,6 +103,8 @@ size_t monarch_workspace_bytes(int op, int64_t tokens, int32_t n, int32_t m, int
     if (check_shape(tokens, n, m, dtype) != MONARCH_OK) return 0;
     const int which = pick(op, m, dtype);
     if (which < 0) return 0;
+    if (which == kTcStaged && op != MONARCH_OP_FWD && op != MONARCH_OP_MLP_FWD)
+        return tc_staged_bwd_workspace_bytes(tokens, m);
     if (op == MONARCH_OP_BWD) {
         if (which == kFused) return fused_bwd_m64_workspace_bytes(tokens);
         const size_t a = staged_workspace_bytes(MONARCH_OP_BWD_DX, tokens, n, m, dtype);
@@ -146,6 +150,9 @@ int monarch_bwd_dx(const void *dy, const void *L, const void *R, void *dx, int64
                               monarch_workspace_bytes(MONARCH_OP_BWD_DX, tokens, n, m, dtype)));
     if (which == kFused)
         return fused_bwd_dx_m64(dy, L, R, dx, tokens, workspace, (cudaStream_t)stream);
+    if (which == kTcStaged)
+        return tc_staged_bwd(nullptr, dy, L, R, dx, nullptr, nullptr, 0, 1, 0, tokens, m, workspace,
+                             (cudaStream_t)stream);
     return staged_bwd_dx(dy, L, R, dx, tokens, m, dtype, workspace, (cudaStream_t)stream);
 }
 
@@ -165,6 +172,9 @@ int monarch_bwd_dw(const void *x, const void *dy, const void *L, const void *R, 
                               monarch_workspace_bytes(MONARCH_OP_BWD_DW, tokens, n, m, dtype)));
     if (which == kFused)
         return fused_bwd_dw_m64(x, dy, L, R, dL, dR, accumulate, tokens, workspace, (cudaStream_t)stream);
+    if (which == kTcStaged)
+        return tc_staged_bwd(x, dy, L, R, nullptr, dL, dR, accumulate, 0, 1, tokens, m, workspace,
+                             (cudaStream_t)stream);
     return staged_bwd_dw(x, dy, L, R, dL, dR, accumulate, tokens, m, dtype, workspace,
                          (cudaStream_t)stream);
 }
@@ -190,6 +200,8 @@ int monarch_bwd(const void *x, const void *dy, const void *L, const void *R, con
         return fused_bwd_m64(x, dy, L, R, saved ? fused_fwd_m64_saved_u(fwd_workspace) : nullptr, dx, dL,
                              dR, accumulate, tokens, workspace, s);
     }
+    if (which == kTcStaged)
+        return tc_staged_bwd(x, dy, L, R, dx, dL, dR, accumulate, 1, 1, tokens, m, workspace, s);
     MONARCH_TRY(staged_bwd_dx(dy, L, R, dx, tokens, m, dtype, workspace, s));
     return staged_bwd_dw(x, dy, L, R, dL, dR, accumulate, tokens, m, dtype, workspace, s);
 }

@@ -1,0 +1,284 @@
+// Backward pass as a chain of tensor-core launches for the block sizes that have no fused kernel (bf16):
+//     z  = P dy                          (stride permutation, a pure data movement)
+//     du = P blockdiag(L^T) z            (one stage of tc_stage.cu with transposed blocks; natural du[t][k][j])
+//     dx = blockdiag(R^T) du             (the same stage kernel without its output permutation)
+//     u' = P blockdiag(R) x              (forward stage 1)
+//     dR[k] = sum_t du_k^T x_k,  dL[j] = sum_t z_j^T u'_j      (token reductions on tcgen05, m = 128)
+// These are the adjoints of Section 3.3 steps 1-3 written with G(W) = P blockdiag(W):
+// M^T = R^T P L^T P = blockdiag(R^T) G(L^T) P.  Everything between two launches goes through the caller's
+// workspace; this family trades HBM traffic for reach.
+#include "tc_common.cuh"
+
+namespace monarch {
+namespace tc {
+namespace {
+
+// z[t][a*m + b] = v[t][b*m + a]: a transpose of every token's m x m view, 32 x 32 tiles through shared memory
+__global__ void __launch_bounds__(256) permute_kernel(const __nv_bfloat16 *__restrict__ v, __nv_bfloat16 *__restrict__ z,
+                                                      int m, long long tokens)
+{
+    __shared__ __nv_bfloat16 tile[32][34];
+    const long long t = blockIdx.z;
+    const int a0 = blockIdx.y * 32, b0 = blockIdx.x * 32;
+    const __nv_bfloat16 *src = v + t * (long long)m * m;
+    __nv_bfloat16 *dst = z + t * (long long)m * m;
+    for (int r = threadIdx.y; r < 32; r += 8) tile[r][threadIdx.x] = src[(long long)(b0 + r) * m + a0 + threadIdx.x];
+    __syncthreads();
+    for (int r = threadIdx.y; r < 32; r += 8) dst[(long long)(a0 + r) * m + b0 + threadIdx.x] = tile[threadIdx.x][r];
+}
+
+// Wt[b][c][e] = W[b][e][c] for every block
+__global__ void __launch_bounds__(256) transpose_blocks_kernel(const __nv_bfloat16 *__restrict__ W,
+                                                               __nv_bfloat16 *__restrict__ Wt, int m)
+{
+    __shared__ __nv_bfloat16 tile[32][34];
+    const int b = blockIdx.z;
+    const int e0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+    const __nv_bfloat16 *src = W + (long long)b * m * m;
+    __nv_bfloat16 *dst = Wt + (long long)b * m * m;
+    for (int r = threadIdx.y; r < 32; r += 8) tile[r][threadIdx.x] = src[(long long)(e0 + r) * m + c0 + threadIdx.x];
+    __syncthreads();
+    for (int r = threadIdx.y; r < 32; r += 8) dst[(long long)(c0 + r) * m + e0 + threadIdx.x] = tile[threadIdx.x][r];
+}
+
+// ---------------------------------------------------------------------------------------------- token reduction
+// out[b][r][c] += sum_t A[t][b*128 + r] * B[t][b*128 + c] for 128 x 128 blocks: both operands are read
+// token-major (MN-major descriptors over 64-token x 64-column TMA boxes, 128B swizzle), a CTA owns 4 blocks
+// (4 accumulators of 128 lanes x 128 columns fill TMEM) and a slice of the token tiles, and adds its partial
+// sums to the output with vector reductions in L2 at the end.
+constexpr int kWM = 128;
+constexpr int kWSlotBytes = 32768;             // A tile 16 KB + B tile 16 KB (two 64-column halves each)
+constexpr int kWSlots = 6;
+constexpr int kWSmem = kWSlots * kWSlotBytes + 1024;
+constexpr int kWThreads = 6 * 32;              // warps 0-3 epilogue, 4 loader, 5 MMA
+
+struct WgradParams {
+    float *out;
+    unsigned *status;
+    int tiles, slices;
+};
+
+__device__ __forceinline__ bool wait_fast(uint32_t bar, uint32_t parity, unsigned *status, volatile int *dead,
+                                          unsigned code)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait(bar, parity, status, dead, code);
+}
+
+__global__ void __launch_bounds__(kWThreads, 1)
+tc_wgrad128_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const WgradParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bar_full[kWSlots], bar_empty[kWSlots], bar_acc;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int dead;
+
+    const uint32_t ring0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int blk0 = blockIdx.x * 4, first = blockIdx.y, step = p.slices;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kWSlots; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 1);
+            mbar_init(smem_u32(&bar_empty[s]), 1);
+        }
+        mbar_init(smem_u32(&bar_acc), 1);
+        fence_mbar_init();
+        dead = 0;
+        tma_prefetch_desc(&tm_a);
+        tma_prefetch_desc(&tm_b);
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&tmem_base_s), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+    const uint32_t full0 = smem_u32(bar_full), empty0 = smem_u32(bar_empty), acc = smem_u32(&bar_acc);
+
+    if (first < p.tiles) {
+        if (warp == 4) {
+            if (lane == 0) {
+                int slot = 0;
+                uint32_t ph = 0;
+                for (int tile = first; tile < p.tiles && !dead; tile += step) {
+#pragma unroll 1
+                    for (int b = 0; b < 4; ++b) {
+                        if (!wait_fast(empty0 + slot * 8, ph ^ 1, p.status, &dead, kErrSlotWait)) break;
+                        const uint32_t dst = ring0 + slot * kWSlotBytes, full = full0 + slot * 8;
+                        const int col = (blk0 + b) * kWM;
+                        mbar_expect_tx(full, kWSlotBytes);
+                        tma_load_2d(dst, &tm_a, col, tile * 64, full);
+                        tma_load_2d(dst + 8192, &tm_a, col + 64, tile * 64, full);
+                        tma_load_2d(dst + 16384, &tm_b, col, tile * 64, full);
+                        tma_load_2d(dst + 24576, &tm_b, col + 64, tile * 64, full);
+                        if (++slot == kWSlots) { slot = 0; ph ^= 1; }
+                    }
+                }
+            }
+        } else if (warp == 5) {
+            if (lane == 0) {
+                constexpr uint32_t idesc = make_idesc_bf16(128, 128, 1, 1);
+                // two 64-column swizzle atoms 8 KB apart along M (N); 8-token groups 1 KB apart along K
+                const uint64_t desc = make_smem_desc(0, 8192, 1024, kSwizzle128);
+                int slot = 0;
+                uint32_t ph = 0;
+                bool ok = true;
+                for (int tile = first; ok && tile < p.tiles; tile += step) {
+                    const uint32_t accum = tile != first;
+#pragma unroll 1
+                    for (int b = 0; b < 4; ++b) {
+                        if (!wait_fast(full0 + slot * 8, ph, p.status, &dead, kErrTmaWait)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint64_t ad = desc | (uint64_t)((ring0 + slot * kWSlotBytes) >> 4);
+                        const uint64_t bd = ad + (16384 >> 4);
+                        const uint32_t d = tmem_base + b * 128;
+                        mma_f16_ss(d, ad, bd, idesc, accum);
+                        mma_f16_ss(d, ad + 128, bd + 128, idesc, 1);          // 16 tokens = 2 KB further
+                        mma_f16_ss(d, ad + 256, bd + 256, idesc, 1);
+                        mma_f16_ss(d, ad + 384, bd + 384, idesc, 1);
+                        mma_commit(empty0 + slot * 8);
+                        if (++slot == kWSlots) { slot = 0; ph ^= 1; }
+                    }
+                }
+                if (ok) mma_commit(acc);
+            }
+        } else if (warp < 4) {
+            if (mbar_wait(acc, 0, p.status, &dead, kErrMmaWait)) {
+                tc_fence_after();
+                const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+                const int row = warp * 32 + lane;
+#pragma unroll 1
+                for (int b = 0; b < 4; ++b) {
+                    float *out = p.out + ((long long)(blk0 + b) * kWM + row) * kWM;
+#pragma unroll 1
+                    for (int c = 0; c < kWM; c += 16) {
+                        uint32_t v[16];
+                        tmem_ld16(lane_base + b * 128 + c, v);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(out + c + e * 4),
+                                         "f"(__uint_as_float(v[e * 4])), "f"(__uint_as_float(v[e * 4 + 1])),
+                                         "f"(__uint_as_float(v[e * 4 + 2])), "f"(__uint_as_float(v[e * 4 + 3]))
+                                         : "memory");
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem_base, 512);
+}
+
+int launch_wgrad128(const void *A, const void *B, float *out, int64_t tokens, unsigned *status, cudaStream_t s)
+{
+    if (tokens == 0) return MONARCH_OK;
+    const int n = kWM * kWM;
+    CUtensorMap tm_a, tm_b;
+    MONARCH_TRY(encode_tmap_2d(&tm_a, A, (uint64_t)tokens, n, (uint64_t)n * 2, 64, 64, 128));
+    MONARCH_TRY(encode_tmap_2d(&tm_b, B, (uint64_t)tokens, n, (uint64_t)n * 2, 64, 64, 128));
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        MONARCH_CUDA_TRY(cudaGetDevice(&dev));
+        MONARCH_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        MONARCH_CUDA_TRY(cudaFuncSetAttribute(tc_wgrad128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmem));
+    }
+    WgradParams p;
+    p.out = out;
+    p.status = status;
+    p.tiles = (int)((tokens + 63) / 64);
+    int slices = sms / 32;
+    if (slices < 1) slices = 1;
+    if (slices > p.tiles) slices = p.tiles;
+    p.slices = slices;
+    tc_wgrad128_kernel<<<dim3(32, slices), kWThreads, kWSmem, s>>>(tm_a, tm_b, p);
+    note_launch();
+    MONARCH_CUDA_TRY(cudaGetLastError());
+    return MONARCH_OK;
+}
+
+int permute(const void *v, void *z, int m, int64_t tokens, cudaStream_t s)
+{
+    if (tokens == 0) return MONARCH_OK;
+    // grid.z carries the token index: at most 65535 per launch
+    const __nv_bfloat16 *src = (const __nv_bfloat16 *)v;
+    __nv_bfloat16 *dst = (__nv_bfloat16 *)z;
+    for (int64_t t0 = 0; t0 < tokens; t0 += 65535) {
+        const int64_t nt = tokens - t0 < 65535 ? tokens - t0 : 65535;
+        permute_kernel<<<dim3(m / 32, m / 32, (unsigned)nt), dim3(32, 8), 0, s>>>(src + t0 * m * m, dst + t0 * m * m, m, nt);
+        note_launch();
+    }
+    MONARCH_CUDA_TRY(cudaGetLastError());
+    return MONARCH_OK;
+}
+
+int transpose_blocks(const void *W, void *Wt, int m, cudaStream_t s)
+{
+    transpose_blocks_kernel<<<dim3(m / 32, m / 32, m), dim3(32, 8), 0, s>>>((const __nv_bfloat16 *)W, (__nv_bfloat16 *)Wt, m);
+    note_launch();
+    MONARCH_CUDA_TRY(cudaGetLastError());
+    return MONARCH_OK;
+}
+
+size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
+
+struct Layout {
+    char *z, *du, *u, *Lt, *Rt;
+};
+Layout carve(void *ws, int64_t tokens, int m)
+{
+    const size_t act = align256((size_t)tokens * m * m * 2), wb = align256((size_t)m * m * m * 2);
+    Layout l;
+    l.z = (char *)ws + MONARCH_STATUS_BYTES;
+    l.du = l.z + act;
+    l.u = l.du + act;
+    l.Lt = l.u + act;
+    l.Rt = l.Lt + wb;
+    return l;
+}
+
+}  // namespace
+}  // namespace tc
+
+// Workspace: [status][z][du][u'][L^T][R^T]
+size_t tc_staged_bwd_workspace_bytes(int64_t tokens, int m)
+{
+    const size_t act = tc::align256((size_t)tokens * m * m * 2), wb = tc::align256((size_t)m * m * m * 2);
+    return MONARCH_STATUS_BYTES + 3 * act + 2 * wb;
+}
+
+// want_dx / want_dw select the outputs; dW needs m = 128 (the token-reduction kernel's block size)
+int tc_staged_bwd(const void *x, const void *dy, const void *L, const void *R, void *dx, float *dL, float *dR,
+                  int accumulate, int want_dx, int want_dw, int64_t tokens, int m, void *ws, cudaStream_t s)
+{
+    using namespace tc;
+    if (want_dw && m != 128) return MONARCH_ERR_UNSUPPORTED;
+    unsigned *status = (unsigned *)ws;
+    const Layout l = carve(ws, tokens, m);
+    if (want_dw && !accumulate) {
+        const size_t gb = (size_t)m * m * m * sizeof(float);
+        MONARCH_CUDA_TRY(cudaMemsetAsync(dL, 0, gb, s));
+        MONARCH_CUDA_TRY(cudaMemsetAsync(dR, 0, gb, s));
+    }
+    if (tokens == 0) return MONARCH_OK;
+    MONARCH_TRY(transpose_blocks(L, l.Lt, m, s));
+    MONARCH_TRY(permute(dy, l.z, m, tokens, s));
+    MONARCH_TRY(tc_stage(m, l.z, l.Lt, l.du, nullptr, 0, tokens, status, s));             // du[t][k][j]
+    if (want_dx) {
+        MONARCH_TRY(transpose_blocks(R, l.Rt, m, s));
+        MONARCH_TRY(tc_stage(m, l.du, l.Rt, dx, nullptr, 0, tokens, status, s, 1));       // dx, no permutation
+    }
+    if (want_dw) {
+        MONARCH_TRY(tc_stage(m, x, R, l.u, nullptr, 0, tokens, status, s));               // u'[t][j][k]
+        MONARCH_TRY(launch_wgrad128(l.du, x, dR, tokens, status, s));
+        MONARCH_TRY(launch_wgrad128(l.z, l.u, dL, tokens, status, s));
+    }
+    return MONARCH_OK;
+}
+
+}  // namespace monarch

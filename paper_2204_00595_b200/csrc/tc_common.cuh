@@ -281,5 +281,10 @@ int encode_tmap_2d(CUtensorMap *out, const void *base, uint64_t rows, uint64_t c
 int encode_tmap_nd(CUtensorMap *out, const void *base, int elem_bytes, int rank, const uint64_t *dims,
                    const uint64_t *strides_bytes, const uint32_t *box, uint32_t swizzle_bytes = 0);
 
+// One block-diagonal stage on the tensor cores (tc_stage.cu): out = P blockdiag(W) in, or with `natural`
+// blockdiag(W) in; optional bias / GELU on the permuted form.
+int tc_stage(int m, const void *in, const void *W, void *out, const void *bias, int gelu, int64_t tokens,
+             unsigned *status, cudaStream_t s, int natural = 0);
+
 }  // namespace tc
 }  // namespace monarch

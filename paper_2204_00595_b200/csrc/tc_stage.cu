@@ -1,7 +1,7 @@
 // One block-diagonal stage on the tcgen05 tensor cores (bf16 in, fp32 accumulate in TMEM):
 //   out[t][e*m + b] = act( sum_c W[b][e][c] * in[t][b*m + c] + bias[e*m + b] )
 // i.e. multiply every length-m segment of a token row by its block, then scatter with the
-// stride permutation P.  Two launches give the forward pass (M = (P L)(P R)), four the
+// stride permutation P (or, with `natural` set, leave the result in place: out[t][b*m + e]).  Two launches give the forward pass (M = (P L)(P R)), four the
 // feed-forward block.  The intermediate goes through the caller's workspace, so this family
 // is bounded by twice the HBM traffic of the fused kernels; it serves the sizes and calls
 // that have no fused kernel.
@@ -42,7 +42,7 @@ template <int M>
 __global__ void __launch_bounds__(128)
 tc_stage_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_constant__ CUtensorMap tm_w,
                 __nv_bfloat16 *__restrict__ out, const __nv_bfloat16 *__restrict__ bias, int gelu,
-                long long tokens, unsigned *status)
+                int natural, long long tokens, unsigned *status)
 {
     using C = StageCfg<M>;
     constexpr int n = M * M;
@@ -130,7 +130,18 @@ tc_stage_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_constant
 #pragma unroll
             for (int b = 0; b < C::NB; ++b) tmem_ld8(lane_base + b * C::NJ + ec * 8, v[b]);
             tmem_ld_wait();
-            if (t < tokens) {
+            if (t < tokens && natural) {
+                // no permutation: the 8 results of block b are contiguous, out[t][(b0+b)*m + e0 + 8 ec ..]
+#pragma unroll
+                for (int b = 0; b < C::NB; ++b) {
+                    uint4 o;
+                    o.x = pack_bf16(__uint_as_float(v[b][0]), __uint_as_float(v[b][1]));
+                    o.y = pack_bf16(__uint_as_float(v[b][2]), __uint_as_float(v[b][3]));
+                    o.z = pack_bf16(__uint_as_float(v[b][4]), __uint_as_float(v[b][5]));
+                    o.w = pack_bf16(__uint_as_float(v[b][6]), __uint_as_float(v[b][7]));
+                    *reinterpret_cast<uint4 *>(out + (size_t)t * n + (b0 + b) * M + e0 + ec * 8) = o;
+                }
+            } else if (t < tokens) {
 #pragma unroll
                 for (int q = 0; q < 8; ++q) {
                     const int col = (e0 + ec * 8 + q) * M + b0;
@@ -166,7 +177,7 @@ tc_stage_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_constant
 }
 
 template <int M>
-int launch_tc_stage(const void *in, const void *W, void *out, const void *bias, int gelu,
+int launch_tc_stage(const void *in, const void *W, void *out, const void *bias, int gelu, int natural,
                     int64_t tokens, unsigned *status, cudaStream_t s)
 {
     using C = StageCfg<M>;
@@ -180,26 +191,26 @@ int launch_tc_stage(const void *in, const void *W, void *out, const void *bias, 
     MONARCH_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
     dim3 grid((unsigned)((tokens + C::TOK - 1) / C::TOK), M / C::NB, M / C::NJ);
     kern<<<grid, 128, C::SMEM_BYTES, s>>>(tm_in, tm_w, (__nv_bfloat16 *)out,
-                                          (const __nv_bfloat16 *)bias, gelu, tokens, status);
+                                          (const __nv_bfloat16 *)bias, gelu, natural, tokens, status);
     note_launch();
     MONARCH_CUDA_TRY(cudaGetLastError());
     return MONARCH_OK;
 }
 
-int tc_stage(int m, const void *in, const void *W, void *out, const void *bias, int gelu,
-             int64_t tokens, unsigned *status, cudaStream_t s)
-{
-    switch (m) {
-        case 32:  return launch_tc_stage<32>(in, W, out, bias, gelu, tokens, status, s);
-        case 64:  return launch_tc_stage<64>(in, W, out, bias, gelu, tokens, status, s);
-        case 128: return launch_tc_stage<128>(in, W, out, bias, gelu, tokens, status, s);
-    }
-    return MONARCH_ERR_UNSUPPORTED;
-}
-
 size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
 
 }  // namespace
+
+int tc_stage(int m, const void *in, const void *W, void *out, const void *bias, int gelu,
+             int64_t tokens, unsigned *status, cudaStream_t s, int natural)
+{
+    switch (m) {
+        case 32:  return launch_tc_stage<32>(in, W, out, bias, gelu, natural, tokens, status, s);
+        case 64:  return launch_tc_stage<64>(in, W, out, bias, gelu, natural, tokens, status, s);
+        case 128: return launch_tc_stage<128>(in, W, out, bias, gelu, natural, tokens, status, s);
+    }
+    return MONARCH_ERR_UNSUPPORTED;
+}
 
 // ---- host: tensor-map encoder through the driver entry point (no link-time libcuda) ----
 typedef CUresult (*tmap_encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
