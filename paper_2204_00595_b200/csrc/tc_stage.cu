@@ -6,13 +6,13 @@
 // is bounded by twice the HBM traffic of the fused kernels; it serves the sizes and calls
 // that have no fused kernel.
 //
-// CTA = 128 tokens x 8 consecutive blocks x NJ output rows.  TMA brings each block's token
+// CTA = 128 tokens x 16 consecutive blocks x 32 output rows.  TMA brings each block's token
 // tile [128 x m] and weight rows [NJ x m] into 128-byte (64-byte for m = 32) swizzled
 // K-major tiles through a 4-slot ring; one thread issues the MMAs (M = 128 tokens, N = NJ,
 // K = 16 per instruction), block b accumulating into TMEM columns [b*NJ, (b+1)*NJ).  With all
-// eight accumulators resident, the thread that owns a token (a TMEM lane) picks element e of
-// each of the 8 blocks - a register renaming, not a data movement - packs them to bf16 and
-// writes the 16 contiguous bytes out[t][e*m + b0 .. b0+7].
+// sixteen accumulators resident, the thread that owns a token (a TMEM lane) picks element e of
+// each of the 16 blocks - a register renaming, not a data movement - packs them to bf16 and
+// writes the 32 contiguous bytes out[t][e*m + b0 .. b0+15].
 #include "tc_common.cuh"
 
 namespace monarch {
@@ -22,8 +22,9 @@ namespace {
 template <int M> struct StageCfg {
     static constexpr int KC = M < 64 ? M : 64;          // K elements per swizzled chunk
     static constexpr int NKC = M / KC;
-    static constexpr int NJ = M < 64 ? M : 64;          // output rows per CTA
-    static constexpr int NB = 8;                        // blocks per CTA
+    static constexpr int NJ = 32;                       // output rows per CTA
+    static constexpr int NB = 16;                       // blocks per CTA: the permuted output leaves in 32-byte
+                                                        // pieces (16-byte pieces reach only ~1 TB/s)
     static constexpr int TOK = 128;
     static constexpr int SWZ_BYTES = KC * 2;            // 64 or 128
     static constexpr uint32_t LAYOUT = SWZ_BYTES == 128 ? kSwizzle128 : kSwizzle64;
@@ -33,7 +34,7 @@ template <int M> struct StageCfg {
     static constexpr int B_BYTES = B_CHUNK * NKC;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int STAGES = 4;
-    static constexpr int TMEM_COLS = NB * NJ;           // 256 or 512 (power of two)
+    static constexpr int TMEM_COLS = NB * NJ;           // 512
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;
     static_assert(A_BYTES % 1024 == 0 && B_BYTES % 1024 == 0, "swizzle atoms need 1 KB alignment");
 };
@@ -124,49 +125,69 @@ tc_stage_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_constant
     tc_fence_after();
     const long long t = t0 + threadIdx.x;
     const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
-    if (have) {
-        for (int ec = 0; ec < C::NJ / 8; ++ec) {
-            uint32_t v[C::NB][8];
+    if (have && natural) {
+        // no permutation: the NJ results of block b are contiguous, out[t][(b0+b)*m + e0 ..]
+        for (int b = 0; b < C::NB; ++b) {
 #pragma unroll
-            for (int b = 0; b < C::NB; ++b) tmem_ld8(lane_base + b * C::NJ + ec * 8, v[b]);
-            tmem_ld_wait();
-            if (t < tokens && natural) {
-                // no permutation: the 8 results of block b are contiguous, out[t][(b0+b)*m + e0 + 8 ec ..]
-#pragma unroll
-                for (int b = 0; b < C::NB; ++b) {
-                    uint4 o;
-                    o.x = pack_bf16(__uint_as_float(v[b][0]), __uint_as_float(v[b][1]));
-                    o.y = pack_bf16(__uint_as_float(v[b][2]), __uint_as_float(v[b][3]));
-                    o.z = pack_bf16(__uint_as_float(v[b][4]), __uint_as_float(v[b][5]));
-                    o.w = pack_bf16(__uint_as_float(v[b][6]), __uint_as_float(v[b][7]));
-                    *reinterpret_cast<uint4 *>(out + (size_t)t * n + (b0 + b) * M + e0 + ec * 8) = o;
+            for (int ec = 0; ec < C::NJ / 16; ++ec) {
+                uint32_t v[16];
+                tmem_ld16(lane_base + b * C::NJ + ec * 16, v);
+                tmem_ld_wait();
+                if (t < tokens) {
+                    uint4 o0, o1;
+                    o0.x = pack_bf16(__uint_as_float(v[0]), __uint_as_float(v[1]));
+                    o0.y = pack_bf16(__uint_as_float(v[2]), __uint_as_float(v[3]));
+                    o0.z = pack_bf16(__uint_as_float(v[4]), __uint_as_float(v[5]));
+                    o0.w = pack_bf16(__uint_as_float(v[6]), __uint_as_float(v[7]));
+                    o1.x = pack_bf16(__uint_as_float(v[8]), __uint_as_float(v[9]));
+                    o1.y = pack_bf16(__uint_as_float(v[10]), __uint_as_float(v[11]));
+                    o1.z = pack_bf16(__uint_as_float(v[12]), __uint_as_float(v[13]));
+                    o1.w = pack_bf16(__uint_as_float(v[14]), __uint_as_float(v[15]));
+                    uint4 *dst = reinterpret_cast<uint4 *>(out + (size_t)t * n + (b0 + b) * M + e0 + ec * 16);
+                    dst[0] = o0;
+                    dst[1] = o1;
                 }
-            } else if (t < tokens) {
+            }
+        }
+    } else if (have) {
+        for (int ec = 0; ec < C::NJ / 4; ++ec) {
+            uint32_t v[C::NB][4];
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const int col = (e0 + ec * 8 + q) * M + b0;
-                    float f[8];
+            for (int b = 0; b < C::NB; ++b) tmem_ld4(lane_base + b * C::NJ + ec * 4, v[b]);
+            tmem_ld_wait();
+            if (t < tokens) {
 #pragma unroll
-                    for (int b = 0; b < 8; ++b) f[b] = __uint_as_float(v[b][q]);
+                for (int q = 0; q < 4; ++q) {
+                    const int col = (e0 + ec * 4 + q) * M + b0;
+                    float f[16];
+#pragma unroll
+                    for (int b = 0; b < 16; ++b) f[b] = __uint_as_float(v[b][q]);
                     if (bias) {
-                        const uint4 bv = *reinterpret_cast<const uint4 *>(bias + col);
-                        const uint32_t bw[4] = {bv.x, bv.y, bv.z, bv.w};
+                        const uint4 bv0 = *reinterpret_cast<const uint4 *>(bias + col);
+                        const uint4 bv1 = *reinterpret_cast<const uint4 *>(bias + col + 8);
+                        const uint32_t bw[8] = {bv0.x, bv0.y, bv0.z, bv0.w, bv1.x, bv1.y, bv1.z, bv1.w};
 #pragma unroll
-                        for (int b = 0; b < 4; ++b) {
+                        for (int b = 0; b < 8; ++b) {
                             f[2 * b] += __uint_as_float(bw[b] << 16);
                             f[2 * b + 1] += __uint_as_float(bw[b] & 0xFFFF0000u);
                         }
                     }
                     if (gelu) {
 #pragma unroll
-                        for (int b = 0; b < 8; ++b) f[b] = gelu_erf(f[b]);
+                        for (int b = 0; b < 16; ++b) f[b] = gelu_erf(f[b]);
                     }
-                    uint4 o;
-                    o.x = pack_bf16(f[0], f[1]);
-                    o.y = pack_bf16(f[2], f[3]);
-                    o.z = pack_bf16(f[4], f[5]);
-                    o.w = pack_bf16(f[6], f[7]);
-                    *reinterpret_cast<uint4 *>(out + (size_t)t * n + col) = o;
+                    uint4 o0, o1;
+                    o0.x = pack_bf16(f[0], f[1]);
+                    o0.y = pack_bf16(f[2], f[3]);
+                    o0.z = pack_bf16(f[4], f[5]);
+                    o0.w = pack_bf16(f[6], f[7]);
+                    o1.x = pack_bf16(f[8], f[9]);
+                    o1.y = pack_bf16(f[10], f[11]);
+                    o1.z = pack_bf16(f[12], f[13]);
+                    o1.w = pack_bf16(f[14], f[15]);
+                    uint4 *dst = reinterpret_cast<uint4 *>(out + (size_t)t * n + col);
+                    dst[0] = o0;
+                    dst[1] = o1;
                 }
             }
         }
