@@ -276,15 +276,14 @@ def main():
     ws_b = P.Workspace(P.monarch_workspace_bytes(P.OP_BWD, T, n, m, code)) if "bwd" in calls else None
     stream = torch.cuda.current_stream()
 
-    ev = {k: [] for k in calls}
+    # One boundary event between consecutive calls (pre-created: nothing but the records sits between two
+    # launches): call k of a timed step runs between marks[j] and marks[j+1].
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps * len(calls) + 1)]
+    nmark = [0]
 
     def step(i, timed):
         e = sets[i % SETS]
         for k in calls:
-            if timed:
-                a = torch.cuda.Event(enable_timing=True)
-                b = torch.cuda.Event(enable_timing=True)
-                a.record(stream)
             if k == "fwd":
                 P.monarch_fwd(e["x"], W["L"], W["R"], e["y"], T, n, m, ws)
             elif k == "bwd_dx":
@@ -302,8 +301,8 @@ def main():
                 P.monarch_mlp_fwd(e["x"], W["L"], W["R"], W["b1"], W["L2"], W["R2"], W["b2"],
                                   e["y"], T, n, m, ws)
             if timed:
-                b.record(stream)
-                ev[k].append((a, b))
+                nmark[0] += 1
+                marks[nmark[0]].record(stream)
 
     for i in range(args.warmup):
         step(i, False)
@@ -317,6 +316,7 @@ def main():
     t_start = torch.cuda.Event(enable_timing=True)
     t_stop = torch.cuda.Event(enable_timing=True)
     t_start.record(stream)
+    marks[0].record(stream)
     for i in range(args.steps):
         step(args.warmup + i, True)
     t_stop.record(stream)
@@ -337,8 +337,8 @@ def main():
 
     peaks = load_peaks()
     per_call = {}
-    for k in calls:
-        ts = [a.elapsed_time(b) for a, b in ev[k]]
+    for ci, k in enumerate(calls):
+        ts = [marks[st * len(calls) + ci].elapsed_time(marks[st * len(calls) + ci + 1]) for st in range(args.steps)]
         ms = statistics.mean(ts)
         by = call_bytes(k, n, m, T, cfg.dtype)
         fl = call_flops(k, n, m, T)

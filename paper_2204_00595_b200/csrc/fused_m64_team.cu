@@ -20,9 +20,9 @@ namespace {
 
 constexpr int kM = 64;
 constexpr int kN = kM * kM;
-// warps: 0-7 epilogue (two halves of four), 8-9 operand loaders, 10 MMA, 11-12 store threads
-constexpr int kEpiWarps = 8, kLoadWarp0 = 8, kMmaWarp = 10, kStoreWarp0 = 11;
-constexpr int kThreads = 13 * 32;
+// warps: 0-7 epilogue (two halves of four), 8-9 operand loaders, 10 MMA, 11-12 store threads, 13 L2 prefetch
+constexpr int kEpiWarps = 8, kLoadWarp0 = 8, kMmaWarp = 10, kStoreWarp0 = 11, kPrefetchWarp = 13;
+constexpr int kThreads = 14 * 32;
 constexpr int kRBytes = 65536, kLBytes = 65536;
 constexpr int kStageBytes = 8192, kStagesPerHalf = 2;
 constexpr int kSlotBytes = 8192, kPairs = 4;                   // ring of 8 slots, handed over in pairs
@@ -34,6 +34,8 @@ struct TeamParams {
     __nv_bfloat16 *u;          // exchange buffer, [tiles][64 j][8][64 t][8] bf16
     unsigned *counters;        // one per 64-token tile, zero between calls
     unsigned *status;
+    const __nv_bfloat16 *x;    // input (for L2 prefetch hints only; the data path goes through TMA)
+    long long tokens;
     const __nv_bfloat16 *bias; // optional [n]: added to the output (feed-forward block, Section 4)
     int gelu;                  // apply erf-GELU after the bias
     int tiles;
@@ -464,6 +466,24 @@ fused_fwd_m64_team_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid
         }
     }
 
+    else if (nt > 0 && warp == kPrefetchWarp) {
+        // ------------------------------------------------------------ L2 prefetch hints for the next x tiles
+        // The operand ring holds less than one tile, so an x tile is requested only ~2 k cycles before the MMAs
+        // want it - less than a trip to DRAM.  One tile ahead, ask L2 for this CTA's 8 KB row segments.
+        for (int it = 0; it + 1 < nt; ++it) {
+            const int tile = team + (it + 1) * p.teams;
+            const char *base = reinterpret_cast<const char *>(p.x) + ((long long)tile * 64 * kN + grp * 8 * kM) * 2;
+#pragma unroll 1
+            for (int i = 0; i < 16; ++i) {
+                const int t = i * 4 + (lane >> 3);
+                if ((long long)tile * 64 + t < p.tokens)
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(base + (long long)t * (kN * 2) + (lane & 7) * 128));
+            }
+            // pace: one tile of hints per tile of stage-1 MMAs
+            if (!wait_fast(s1f, it & 1, p.status, dead, kErrMmaWait)) break;
+        }
+    }
+
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem_base, 512);
@@ -505,6 +525,8 @@ int launch_team(const void *x, const void *L, const void *R, const void *bias, i
     p.status = status;
     p.counters = counters;
     p.u = (__nv_bfloat16 *)u;
+    p.x = (const __nv_bfloat16 *)x;
+    p.tokens = tokens;
     p.bias = (const __nv_bfloat16 *)bias;
     p.gelu = gelu;
     p.tiles = (int)tiles;
