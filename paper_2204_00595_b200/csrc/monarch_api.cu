@@ -68,7 +68,8 @@ enum Family { kSimt = 0, kFused = 1, kTcStaged = 2, kNone = -1 };
 bool fused_available(int op, int m, int dtype)
 {
     static const bool off = getenv("MONARCH_NO_FUSED") != nullptr;   // comparison runs: stage chain instead
-    return !off && dtype == MONARCH_BF16 && m == 64;   // every op
+    if (off || dtype != MONARCH_BF16) return false;
+    return m == 64 || (m == 32 && op == MONARCH_OP_FWD);   // m = 64: every op; m = 32: forward
 }
 
 // true when the call can run as a chain of tensor-core stages through the workspace
@@ -112,7 +113,8 @@ size_t monarch_workspace_bytes(int op, int64_t tokens, int32_t n, int32_t m, int
         return a > b ? a : b;
     }
     if (which == kFused)
-        return op == MONARCH_OP_MLP_FWD  ? fused_mlp_fwd_m64_workspace_bytes(tokens)
+        return m == 32                   ? (size_t)MONARCH_STATUS_BYTES
+               : op == MONARCH_OP_MLP_FWD ? fused_mlp_fwd_m64_workspace_bytes(tokens)
                : op == MONARCH_OP_FWD    ? fused_fwd_m64_workspace_bytes(tokens)
                : op == MONARCH_OP_BWD_DX ? fused_bwd_dx_m64_workspace_bytes(tokens)
                                          : fused_bwd_dw_m64_workspace_bytes(tokens);
@@ -131,7 +133,8 @@ int monarch_fwd(const void *x, const void *L, const void *R, void *y, int64_t to
     MONARCH_TRY(check_buffers(in, 3, out, 1, workspace, workspace_bytes,
                               monarch_workspace_bytes(MONARCH_OP_FWD, tokens, n, m, dtype)));
     if (which == kFused)
-        return fused_fwd_m64(x, L, R, y, tokens, workspace, (cudaStream_t)stream);
+        return m == 32 ? fused_fwd_m32(x, L, R, y, tokens, workspace, (cudaStream_t)stream)
+                       : fused_fwd_m64(x, L, R, y, tokens, workspace, (cudaStream_t)stream);
     if (which == kTcStaged) return tc_staged_fwd(x, L, R, y, tokens, m, workspace, (cudaStream_t)stream);
     return staged_fwd(x, L, R, y, tokens, m, dtype, workspace, (cudaStream_t)stream);
 }
