@@ -4,11 +4,11 @@
 // nothing is exchanged between SMs (Section 3.3 steps 1-3 with the permutations done on chip, as the method
 // is meant to run): a persistent CTA per SM takes whole tiles.
 //   stage 1: x arrives as 64 x 64 TMA boxes (two blocks k side by side, 128B swizzle), R_k pairs as 64 x 32 boxes;
-//            M = 64, N = 32 MMAs accumulate 16 blocks at a time into one 16-lane half of TMEM ("plane 0", 512
-//            columns); the epilogue packs 8 blocks' results for one (t, j) into 16 bytes and writes them into
+//            M = 64, N = 32 MMAs accumulate 16 blocks at a time into one 16-lane half of TMEM (a "plane" of 512
+//            columns; the two halves of a stage go to the two planes); the epilogue packs 8 blocks' results for one (t, j) into 16 bytes and writes them into
 //            the shared-memory buffer U[j][k/8][t][k%8] - the P^T of step 2 is which columns are packed together,
 //            and U[j] is, as it lies, the K-major A operand of stage 2.
-//   stage 2: A = U[j], B = L_j (streamed as pairs), 16 blocks j at a time into the other half of TMEM ("plane 1");
+//   stage 2: A = U[j], B = L_j (streamed as pairs), again 16 blocks j per plane;
 //            the epilogue packs 16 blocks into the 32 bytes y[t][l*32 + 16s .. +16) (the final P), staged and
 //            stored with 3-D TMA boxes.
 // One thread issues all MMAs in the order S1a S1b S2a S2b per tile (a = blocks 0-15, b = 16-31); stage 1 of
@@ -38,12 +38,21 @@ constexpr int kSmemBytes = kUBytes + kXSlots * kXSlotBytes + kLSlots * kLSlotByt
 struct P32 {
     unsigned *status;
     int tiles;
+    long long *trace;            // optional per-CTA timeline (debug builds), else null
 };
 
+#ifdef MONARCH_TRACE
+#define T32(item, slot, val) do { if (p.trace && (item) < 16) p.trace[((size_t)blockIdx.x * 16 + (item)) * 8 + (slot)] = (val); } while (0)
+#define C32() clock64()
+#else
+#define T32(item, slot, val) do { } while (0)
+#define C32() 0ll
+#endif
+
 struct Bars {
-    uint64_t xfull[kXSlots], xempty[kXSlots];
-    uint64_t lfull[kLSlots], lempty[kLSlots];
-    uint64_t p0_full, p0_empty, p1_full, p1_empty;
+    uint64_t xfull[2], xempty[2];                     // ring slots are handed over in groups of two
+    uint64_t lfull[2], lempty[2];
+    uint64_t pl_full[2], pl_empty[2];                 // the two accumulator planes (16-lane halves of TMEM)
     uint64_t st_full[2 * kStagesPerHalf], st_free[2 * kStagesPerHalf];
 };
 
@@ -71,18 +80,16 @@ fused_fwd_m32_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     volatile int *dead = &dead_s;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kXSlots; ++s) {
-            mbar_init(smem_u32(&bars.xfull[s]), 1);
-            mbar_init(smem_u32(&bars.xempty[s]), 1);
+        for (int g = 0; g < 2; ++g) {
+            mbar_init(smem_u32(&bars.xfull[g]), 2);          // one (x, R) pair from each of the two loaders
+            mbar_init(smem_u32(&bars.xempty[g]), 1);
+            mbar_init(smem_u32(&bars.lfull[g]), 1);
+            mbar_init(smem_u32(&bars.lempty[g]), 1);
         }
-        for (int s = 0; s < kLSlots; ++s) {
-            mbar_init(smem_u32(&bars.lfull[s]), 1);
-            mbar_init(smem_u32(&bars.lempty[s]), 1);
+        for (int h = 0; h < 2; ++h) {
+            mbar_init(smem_u32(&bars.pl_full[h]), 1);
+            mbar_init(smem_u32(&bars.pl_empty[h]), kEpiWarps);
         }
-        mbar_init(smem_u32(&bars.p0_full), 1);
-        mbar_init(smem_u32(&bars.p0_empty), kEpiWarps);
-        mbar_init(smem_u32(&bars.p1_full), 1);
-        mbar_init(smem_u32(&bars.p1_empty), kEpiWarps);
         for (int k = 0; k < 2 * kStagesPerHalf; ++k) {
             mbar_init(smem_u32(&bars.st_full[k]), 4);
             mbar_init(smem_u32(&bars.st_free[k]), 1);
@@ -103,8 +110,7 @@ fused_fwd_m32_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     const int first = (int)blockIdx.x, step = (int)gridDim.x;
     const uint32_t xf0 = smem_u32(bars.xfull), xe0 = smem_u32(bars.xempty);
     const uint32_t lf0 = smem_u32(bars.lfull), le0 = smem_u32(bars.lempty);
-    const uint32_t p0f = smem_u32(&bars.p0_full), p0e = smem_u32(&bars.p0_empty);
-    const uint32_t p1f = smem_u32(&bars.p1_full), p1e = smem_u32(&bars.p1_empty);
+    const uint32_t plf0 = smem_u32(bars.pl_full), ple0 = smem_u32(bars.pl_empty);
 
     if (first >= p.tiles) {
         // nothing to do
@@ -112,14 +118,15 @@ fused_fwd_m32_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         // ------------------------------------------------------------ (x, R) loaders: warp pw takes pairs pw, pw+2, ...
         if (lane == 0) {
             const int pw = warp - kXWarp0;
-            uint32_t n = pw;                               // use count of the ring: pair index over all tiles
+            uint32_t ng = 0;                               // group use count: pairs (2 ng, 2 ng + 1) of the stream
             for (int tile = first; tile < p.tiles; tile += step) {
                 bool ok = true;
 #pragma unroll 1
-                for (int pr = pw; pr < 16; pr += 2, n += 2) {
-                    const uint32_t s = n & (kXSlots - 1), ph = (n / kXSlots) & 1;
-                    if (!wait_fast(xe0 + s * 8, ph ^ 1, p.status, dead, kErrSlotWait)) { ok = false; break; }
-                    const uint32_t dst = xring0 + s * kXSlotBytes, full = xf0 + s * 8;
+                for (int G = 0; G < 8; ++G, ++ng) {
+                    const uint32_t g = ng & 1, ph = (ng >> 1) & 1;
+                    const int pr = G * 2 + pw;
+                    if (!wait_fast(xe0 + g * 8, ph ^ 1, p.status, dead, kErrSlotWait)) { ok = false; break; }
+                    const uint32_t dst = xring0 + (g * 2 + pw) * kXSlotBytes, full = xf0 + g * 8;
                     mbar_expect_tx(full, kXSlotBytes);
                     tma_load_2d(dst, &tm_x, pr * 64, tile * 64, full);            // blocks 2pr, 2pr+1: 64 columns
                     tma_load_2d(dst + 8192, &tm_R, 0, pr * 64, full);             // R rows of both blocks
@@ -130,15 +137,16 @@ fused_fwd_m32_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     } else if (warp == kLWarp) {
         // ------------------------------------------------------------ L loader
         if (lane == 0) {
-            uint32_t n = 0;
+            uint32_t ng = 0;
             for (int tile = first; tile < p.tiles; tile += step) {
                 bool ok = true;
 #pragma unroll 1
-                for (int pr = 0; pr < 16; ++pr, ++n) {
-                    const uint32_t s = n & (kLSlots - 1), ph = (n / kLSlots) & 1;
-                    if (!wait_fast(le0 + s * 8, ph ^ 1, p.status, dead, kErrSlotWait)) { ok = false; break; }
-                    mbar_expect_tx(lf0 + s * 8, kLSlotBytes);
-                    tma_load_2d(lring0 + s * kLSlotBytes, &tm_L, 0, pr * 64, lf0 + s * 8);
+                for (int G = 0; G < 8; ++G, ++ng) {
+                    const uint32_t g = ng & 1, ph = (ng >> 1) & 1;
+                    if (!wait_fast(le0 + g * 8, ph ^ 1, p.status, dead, kErrSlotWait)) { ok = false; break; }
+                    mbar_expect_tx(lf0 + g * 8, 2 * kLSlotBytes);
+                    tma_load_2d(lring0 + (g * 2) * kLSlotBytes, &tm_L, 0, (G * 2) * 64, lf0 + g * 8);
+                    tma_load_2d(lring0 + (g * 2 + 1) * kLSlotBytes, &tm_L, 0, (G * 2 + 1) * 64, lf0 + g * 8);
                 }
                 if (!ok) break;
             }
@@ -150,69 +158,84 @@ fused_fwd_m32_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
             const uint64_t d_x = make_smem_desc(0, 16, 1024, kSwizzle128);   // x pair tile: 128-byte rows
             const uint64_t d_w = make_smem_desc(0, 16, 512, kSwizzle64);     // weight tiles: 64-byte rows
             const uint64_t d_u = make_smem_desc(0, 1024, 128, 0);            // U[j]: k chunks 1 KB apart
-            const uint32_t plane0 = tmem_base, plane1 = tmem_base + ((uint32_t)16 << 16);
-            // ring use counts; sub-items issued per stage; completions of p0_empty / p1_empty already waited for
-            uint32_t nx = 0, nl = 0, k0 = 0, m1 = 0, c0 = 0, c1 = 0;
+            // ring use counts; per plane: sub-items issued so far, completions of its `empty` barrier waited for
+            uint32_t nx = 0, nl = 0, issued[2] = {0, 0}, c[2] = {0, 0};
             bool ok = true;
-            // wait until the epilogue has drained `target` sub-items of a plane (completion c has parity c & 1)
-            auto drained = [&](uint32_t bar, uint32_t &c, uint32_t target) {
-                while (ok && c < target) {
-                    if (!wait_fast(bar, c & 1, p.status, dead, kErrTmemWait)) ok = false;
-                    ++c;
+            // wait until the epilogue has drained `target` sub-items of plane P (completion n has parity n & 1)
+            auto drained = [&](int P, uint32_t target) {
+                while (ok && c[P] < target) {
+                    if (!wait_fast(ple0 + P * 8, c[P] & 1, p.status, dead, kErrTmemWait)) ok = false;
+                    ++c[P];
                 }
                 tc_fence_after();
             };
+            [[maybe_unused]] int ntile = -1;
             for (int tile = first; ok && tile < p.tiles; tile += step) {
-                // ---- stage 1, two halves of 16 blocks through plane 0
+                ++ntile;
+                // sub-items S1a S1b S2a S2b alternate between the two planes, so a half never waits for the
+                // epilogue of the half before it; only stage 2 waits - for all of U
 #pragma unroll 1
-                for (int h = 0; h < 2 && ok; ++h, ++k0) {
-                    drained(p0e, c0, k0);                  // the previous stage-1 half has left plane 0
+                for (int q = 0; q < 4 && ok; ++q) {
+                    const int P = q & 1, h = q & 1;
+                    const uint32_t plane = tmem_base + ((uint32_t)(P * 16) << 16);
+                    [[maybe_unused]] const long long t_a = C32();
+                    if (q == 2) drained(1, issued[1]);     // S1b's epilogue: U is complete
+                    drained(P, issued[P]);                 // this plane has been read out
                     if (!ok) break;
-#pragma unroll 1
-                    for (int pr = 0; pr < 8; ++pr, ++nx) {
-                        const uint32_t s = nx & (kXSlots - 1), ph = (nx / kXSlots) & 1;
-                        if (!wait_fast(xf0 + s * 8, ph, p.status, dead, kErrTmaWait)) { ok = false; break; }
-                        tc_fence_after();
-                        const uint32_t slot = xring0 + s * kXSlotBytes;
-                        const uint64_t ax = d_x | (uint64_t)(slot >> 4);
-                        const uint64_t bw = d_w | (uint64_t)((slot + 8192) >> 4);
+                    [[maybe_unused]] const long long t_b = C32();
+                    [[maybe_unused]] long long wsum = 0;
+                    if (q < 2) {
+                        // four groups per half and two in the ring: group G sits in ring position G & 1
 #pragma unroll
-                        for (int i = 0; i < 2; ++i) {
-                            const uint32_t d = plane0 + (pr * 2 + i) * 32;
-                            // block 2pr+i: columns [32 i, 32 i + 32) of the pair tile, rows [32 i, +32) of the R pair
-                            mma_f16_ss(d, ax + i * 4, bw + i * 128, idesc, 0);
-                            mma_f16_ss(d, ax + i * 4 + 2, bw + i * 128 + 2, idesc, 1);
+                        for (int G = 0; G < 4; ++G, ++nx) {
+                            const uint32_t g = G & 1, ph = (nx >> 1) & 1;
+                            [[maybe_unused]] const long long w0 = C32();
+                            if (!wait_fast(xf0 + g * 8, ph, p.status, dead, kErrTmaWait)) { ok = false; break; }
+                            tc_fence_after();
+                            wsum += C32() - w0;
+#pragma unroll
+                            for (int e = 0; e < 2; ++e) {
+                                const uint32_t slot = xring0 + (g * 2 + e) * kXSlotBytes;
+                                const uint64_t ax = d_x | (uint64_t)(slot >> 4);
+                                const uint64_t bw = d_w | (uint64_t)((slot + 8192) >> 4);
+#pragma unroll
+                                for (int i = 0; i < 2; ++i) {
+                                    const uint32_t d = plane + ((G * 2 + e) * 2 + i) * 32;
+                                    // block 2pr+i: columns [32 i, +32) of the pair tile, rows [32 i, +32) of the R pair
+                                    mma_f16_ss(d, ax + i * 4, bw + i * 128, idesc, 0);
+                                    mma_f16_ss(d, ax + i * 4 + 2, bw + i * 128 + 2, idesc, 1);
+                                }
+                            }
+                            mma_commit(xe0 + g * 8);
                         }
-                        mma_commit(xe0 + s * 8);
+                    } else {
+#pragma unroll
+                        for (int G = 0; G < 4; ++G, ++nl) {
+                            const uint32_t g = G & 1, ph = (nl >> 1) & 1;
+                            [[maybe_unused]] const long long w0 = C32();
+                            if (!wait_fast(lf0 + g * 8, ph, p.status, dead, kErrTmaWait)) { ok = false; break; }
+                            tc_fence_after();
+                            wsum += C32() - w0;
+#pragma unroll
+                            for (int e = 0; e < 2; ++e) {
+                                const uint64_t bl = d_w | (uint64_t)((lring0 + (g * 2 + e) * kLSlotBytes) >> 4);
+#pragma unroll
+                                for (int i = 0; i < 2; ++i) {
+                                    const int jb = (G * 2 + e) * 2 + i;
+                                    const uint32_t d = plane + jb * 32;
+                                    const uint64_t au = d_u | (uint64_t)((U0 + (h * 16 + jb) * 4096) >> 4);
+                                    mma_f16_ss(d, au, bl + i * 128, idesc, 0);
+                                    mma_f16_ss(d, au + 128, bl + i * 128 + 2, idesc, 1);
+                                }
+                            }
+                            mma_commit(le0 + g * 8);
+                        }
                     }
                     if (!ok) break;
-                    mma_commit(p0f);
-                }
-                if (!ok) break;
-                // ---- stage 2 needs all of U: both stage-1 epilogues of this tile must be done
-                drained(p0e, c0, k0);
-#pragma unroll 1
-                for (int h = 0; h < 2 && ok; ++h, ++m1) {
-                    drained(p1e, c1, m1);                  // the previous stage-2 half has left plane 1
-                    if (!ok) break;
-#pragma unroll 1
-                    for (int pr = 0; pr < 8; ++pr, ++nl) {
-                        const uint32_t s = nl & (kLSlots - 1), ph = (nl / kLSlots) & 1;
-                        if (!wait_fast(lf0 + s * 8, ph, p.status, dead, kErrTmaWait)) { ok = false; break; }
-                        tc_fence_after();
-                        const uint64_t bl = d_w | (uint64_t)((lring0 + s * kLSlotBytes) >> 4);
-#pragma unroll
-                        for (int i = 0; i < 2; ++i) {
-                            const int j = h * 16 + pr * 2 + i;
-                            const uint32_t d = plane1 + (pr * 2 + i) * 32;
-                            const uint64_t au = d_u | (uint64_t)((U0 + j * 4096) >> 4);
-                            mma_f16_ss(d, au, bl + i * 128, idesc, 0);
-                            mma_f16_ss(d, au + 128, bl + i * 128 + 2, idesc, 1);
-                        }
-                        mma_commit(le0 + s * 8);
-                    }
-                    if (!ok) break;
-                    mma_commit(p1f);
+                    mma_commit(plf0 + P * 8);
+                    T32(ntile * 4 + q, 0, t_a); T32(ntile * 4 + q, 1, t_b - t_a); T32(ntile * 4 + q, 2, wsum);
+                    T32(ntile * 4 + q, 3, C32());
+                    ++issued[P];
                 }
             }
         }
@@ -224,13 +247,14 @@ fused_fwd_m32_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         const uint32_t my_stage = stage0 + sub * kStagesPerHalf * kStageBytes;
         const uint32_t stf0 = smem_u32(bars.st_full) + sub * kStagesPerHalf * 8;
         const uint32_t stfree0 = smem_u32(bars.st_free) + sub * kStagesPerHalf * 8;
-        uint32_t n0 = 0, n1 = 0, nchunk = 0;
+        uint32_t np[2] = {0, 0}, nchunk = 0;          // sub-items seen per plane
         bool ok = true;
         for (int tile = first; ok && tile < p.tiles; tile += step) {
-            // ---- stage 1 halves: plane 0 (lanes 0-15 of every quarter) -> U
+            // ---- stage 1 halves: half h sits in plane h (lanes 16 h .. 16 h + 15 of every quarter) -> U
 #pragma unroll 1
-            for (int h = 0; h < 2 && ok; ++h, ++n0) {
-                if (!wait_fast(p0f, n0 & 1, p.status, dead, kErrMmaWait)) { ok = false; break; }
+            for (int h = 0; h < 2 && ok; ++h) {
+                if (!wait_fast(plf0 + h * 8, np[h] & 1, p.status, dead, kErrMmaWait)) { ok = false; break; }
+                ++np[h];
                 tc_fence_after();
                 // this warp: rows j in [16 sub, 16 sub + 16), in two chunks of 8; blocks k of this half in two
                 // groups of 8 -> U chunk index 2h + g
@@ -242,7 +266,7 @@ fused_fwd_m32_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
 #pragma unroll
                         for (int kb = 0; kb < 8; ++kb) tmem_ld8(lane_base + (g * 8 + kb) * 32 + sub * 16 + jc * 8, v[kb]);
                         tmem_ld_wait();
-                        if (hl == 0) {
+                        if (hl == h) {
 #pragma unroll
                             for (int q = 0; q < 8; ++q) {
                                 const uint32_t o0 = pack_bf16(__uint_as_float(v[0][q]), __uint_as_float(v[1][q]));
@@ -259,12 +283,13 @@ fused_fwd_m32_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
                 tc_fence_before();
                 fence_proxy_async_smem();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(p0e);
+                if (lane == 0) mbar_arrive(ple0 + h * 8);
             }
-            // ---- stage 2 halves: plane 1 (lanes 16-31 of every quarter) -> y
+            // ---- stage 2 halves: half h in plane h -> y
 #pragma unroll 1
-            for (int h = 0; h < 2 && ok; ++h, ++n1) {
-                if (!wait_fast(p1f, n1 & 1, p.status, dead, kErrMmaWait)) { ok = false; break; }
+            for (int h = 0; h < 2 && ok; ++h) {
+                if (!wait_fast(plf0 + h * 8, np[h] & 1, p.status, dead, kErrMmaWait)) { ok = false; break; }
+                ++np[h];
                 tc_fence_after();
 #pragma unroll 1
                 for (int c = sub; c < 8; c += 2, ++nchunk) {
@@ -276,7 +301,7 @@ fused_fwd_m32_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
 #pragma unroll
                     for (int a = 0; a < 16; ++a) tmem_ld4(lane_base + a * 32 + c * 4, v[a]);
                     tmem_ld_wait();
-                    if (hl == 1) {
+                    if (hl == h) {
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
 #pragma unroll
@@ -294,7 +319,7 @@ fused_fwd_m32_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
                     if (c + 2 >= 8) {
                         tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) mbar_arrive(p1e);
+                        if (lane == 0) mbar_arrive(ple0 + h * 8);
                     }
                     fence_proxy_async_smem();
                     __syncwarp();
@@ -371,6 +396,10 @@ int fused_fwd_m32(const void *x, const void *L, const void *R, void *y, int64_t 
     P32 p;
     p.status = (unsigned *)ws;
     p.tiles = (int)tiles;
+    p.trace = nullptr;
+#ifdef MONARCH_TRACE
+    if (const char *e = getenv("MONARCH_TRACE_PTR")) p.trace = (long long *)strtoull(e, nullptr, 0);
+#endif
     const int grid = tiles < sms ? (int)tiles : sms;
     fused_fwd_m32_kernel<<<grid, kThreads, kSmemBytes, s>>>(tm_x, tm_R, tm_L, tm_y, p);
     note_launch();
