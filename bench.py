@@ -182,6 +182,7 @@ KERNELS_OF = {
     (64, "bf16", "fwd"): "fused_fwd_m64_team_kernel (1 launch)",
     (64, "bf16", "bwd"): "fused_bwd_all_m64_kernel (1 launch, 2 memset nodes)",
     (64, "bf16", "mlp_fwd"): "fused_fwd_m64_team_kernel (2 launches)",
+    (32, "bf16", "fwd"): "fused_fwd_m32_kernel (1 launch)",
     (64, "bf16", "bwd_dx"): "fused_bwd_dx_m64_kernel (1 launch)",
     (64, "bf16", "bwd_dw"): "fused_fwd_m64_kernel (stage 1 only) + fused_bwd_dx_m64_kernel (stage 1 only) + "
                             "fused_bwd_dw_m64_kernel (3 launches, 2 memset nodes)",

@@ -108,6 +108,7 @@ fused_fwd_m64_team_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid
     __shared__ int dep_items_s;
     __shared__ __align__(16) __nv_bfloat16 bias_s[32 * 16];   // this CTA's slice of the bias: [l local][j local]
 
+    [[maybe_unused]] const long long t_entry = TCLK();
     const uint32_t smemR = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t smemL = smemR + kRBytes;
     const uint32_t stage0 = smemL + kLBytes;
@@ -152,6 +153,7 @@ fused_fwd_m64_team_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
+    if (threadIdx.x == 0) { TTRACE(15, 0, t_entry); TTRACE(15, 1, TCLK()); }
 
     // number of tiles of this team; step `it` does S1(tile it) then S2(tile it-1)
     const int nt = team < p.tiles ? (p.tiles - team + p.teams - 1) / p.teams : 0;
@@ -484,9 +486,12 @@ fused_fwd_m64_team_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid
         }
     }
 
+    if (threadIdx.x == 0) TTRACE(15, 2, TCLK());
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) TTRACE(15, 3, TCLK());
     if (warp == 0) tmem_dealloc(tmem_base, 512);
+    if (threadIdx.x == 0) TTRACE(15, 4, TCLK());
 }
 
 }  // namespace
