@@ -7,7 +7,8 @@
  * calls below multiply a batch of token vectors by M, by M^T, form the
  * gradients of the blocks, and evaluate a Monarch feed-forward block.
  *
- * Conventions shared by every call
+ * Conventions shared by every call (the monarch_host_* calls at the end of
+ * this file take HOST pointers and own their device memory; they say so)
  * --------------------------------
  *  - All data pointers are DEVICE pointers owned by the caller, 16-byte
  *    aligned, dense and row-major.  Nothing is allocated, freed or retained
@@ -33,6 +34,10 @@
  *    when one of their bounded waits runs out; zero it once with
  *    monarch_workspace_init and read it with monarch_last_device_status.
  *    Calls that overlap on the GPU must not share a workspace.
+ *  - Weight gradients of the tensor-core families are summed with fp32
+ *    reductions whose order across thread blocks is not fixed: dL, dR can
+ *    differ in the last fp32 bits from run to run (the CUDA-core family,
+ *    MONARCH_IMPL_STAGED, sums in a fixed order).
  *  - Return value: a monarch_status_t.  Nothing throws.
  */
 #ifndef MONARCH_H_
