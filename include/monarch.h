@@ -133,7 +133,9 @@ int monarch_workspace_init(void *workspace, size_t workspace_bytes, void *stream
 
 /* Synchronise `stream`, read and clear the status word: MONARCH_OK, or
  * MONARCH_ERR_TIMEOUT if a kernel abandoned a bounded wait since the last
- * query (its outputs are then undefined), or MONARCH_ERR_CUDA. */
+ * query (its outputs are then undefined, and the tile counters in the
+ * workspace may be left non-zero: call monarch_workspace_init again before
+ * reusing it), or MONARCH_ERR_CUDA. */
 int monarch_last_device_status(void *workspace, void *stream);
 
 /* Select the kernel family for later calls (a monarch_impl_t).  Not

@@ -538,16 +538,20 @@ int fused_fwd_m64(const void *x, const void *L, const void *R, void *y, int64_t 
                   cudaStream_t s)
 {
     if (tokens == 0) return MONARCH_OK;
-    static const bool two = getenv("MONARCH_TWO_LAUNCH") != nullptr;       // comparison runs only
-    static const bool split = getenv("MONARCH_FWD_SPLIT") != nullptr;      // comparison runs only
-    if (!two && !split) return fused_fwd_m64_team(x, L, R, y, tokens, ws, s);
+#ifdef MONARCH_TRACE
+    // debug builds: comparison runs of the split schedule, as one launch or as one launch per stage
+    static const bool two = getenv("MONARCH_TWO_LAUNCH") != nullptr;
+    static const bool split = getenv("MONARCH_FWD_SPLIT") != nullptr;
     if (two) {
         void *u = (char *)ws + MONARCH_STATUS_BYTES + kFusedCounterBytes;
         MONARCH_TRY(launch_fwd_m64(x, nullptr, R, nullptr, u, nullptr, (unsigned *)ws, tokens, s));
         return launch_fwd_m64(nullptr, L, R, y, u, nullptr, (unsigned *)ws, tokens, s);
     }
-    return launch_fwd_m64(x, L, R, y, (char *)ws + MONARCH_STATUS_BYTES + kFusedCounterBytes,
-                          (unsigned *)((char *)ws + MONARCH_STATUS_BYTES), (unsigned *)ws, tokens, s);
+    if (split)
+        return launch_fwd_m64(x, L, R, y, (char *)ws + MONARCH_STATUS_BYTES + kFusedCounterBytes,
+                              (unsigned *)((char *)ws + MONARCH_STATUS_BYTES), (unsigned *)ws, tokens, s);
+#endif
+    return fused_fwd_m64_team(x, L, R, y, tokens, ws, s);
 }
 
 const void *fused_fwd_m64_saved_u(const void *fwd_ws)

@@ -1046,7 +1046,9 @@ int launch_bwd_m64(const void *dy, const void *L, const void *R, void *dx, void 
     int b1 = both ? (sms * 12) / 148 : sms / 8;
     if (b1 < 1) b1 = 1;
     int b2 = both ? (sms - 8 * b1) / 8 : 0;
+#ifdef MONARCH_TRACE
     if (const char *e = getenv("MONARCH_BWD_SPLIT2")) { if (both) sscanf(e, "%d,%d", &b1, &b2); }
+#endif
     if (both && b2 < 1) b2 = 1;
     if (b1 > tiles) b1 = (int)tiles;
     if (b2 > tiles) b2 = (int)tiles;
@@ -1112,7 +1114,9 @@ int fused_bwd_all_m64(const void *x, const void *dy, const void *L, const void *
     // SM split by measured cost per tile and group (B1 ~10 k cycles, B2R ~6 k, WL ~6 k with 4 groups only);
     // 8/6/6 CTAs per group was the best of a sweep on 148 SMs
     int b1 = (sms * 8) / 144, b2 = (sms * 6) / 144, b3 = (sms * 6) / 144;
+#ifdef MONARCH_TRACE
     if (const char *e = getenv("MONARCH_BWD_SPLIT3")) sscanf(e, "%d,%d,%d", &b1, &b2, &b3);
+#endif
     if (b1 < 1) b1 = 1;
     if (b2 < 1) b2 = 1;
     if (b3 < 1) b3 = 1;

@@ -285,10 +285,15 @@ int fused_bwd_m64(const void *x, const void *dy, const void *L, const void *R, c
         MONARCH_TRY(fused_fwd_m64_stage1(x, R, u_own, tokens, status, s));
         u = u_own;
     }
-    static const bool split = getenv("MONARCH_BWD_SPLIT") != nullptr;     // comparison runs: two kernels
-    if (!split) return fused_bwd_all_m64(x, dy, L, R, u, dx, du, dyp, dL, dR, counters, status, tokens, s);
-    MONARCH_TRY(fused_bwd_dx_m64_keep(dy, L, R, dx, du, dyp, counters, status, tokens, s));
-    return launch_dw(x, u, du, dyp, dL, dR, status, tokens, s);
+#ifdef MONARCH_TRACE
+    // debug builds: the two-kernel form (backward kernel, then the token reduction), for comparison
+    static const bool split = getenv("MONARCH_BWD_SPLIT") != nullptr;
+    if (split) {
+        MONARCH_TRY(fused_bwd_dx_m64_keep(dy, L, R, dx, du, dyp, counters, status, tokens, s));
+        return launch_dw(x, u, du, dyp, dL, dR, status, tokens, s);
+    }
+#endif
+    return fused_bwd_all_m64(x, dy, L, R, u, dx, du, dyp, dL, dR, counters, status, tokens, s);
 }
 
 }  // namespace monarch

@@ -67,7 +67,11 @@ enum Family { kSimt = 0, kFused = 1, kTcStaged = 2, kNone = -1 };
 // true when the fused tensor-core family has a kernel for (op, m, dtype)
 bool fused_available(int op, int m, int dtype)
 {
-    static const bool off = getenv("MONARCH_NO_FUSED") != nullptr;   // comparison runs: stage chain instead
+#ifdef MONARCH_TRACE
+    static const bool off = getenv("MONARCH_NO_FUSED") != nullptr;   // debug builds: stage chain, for comparison
+#else
+    constexpr bool off = false;
+#endif
     if (off || dtype != MONARCH_BF16) return false;
     return m == 64 || (m == 32 && op == MONARCH_OP_FWD);   // m = 64: every op; m = 32: forward
 }
