@@ -147,6 +147,53 @@ def test_bwd_one_call(P, impl, m, T, dtype, saved):
     assert_close(to_host64(dR), 2 * ref["dR"], dtype, "dR accumulate")
 
 
+# Token counts around the persistent kernels' schedule boundaries: 18 teams of 8 CTAs (m = 64: one, two and
+# "two and a bit" tiles per team), 148 CTAs (m = 32), each with a ragged last tile.
+@pytest.mark.parametrize("m,T", [(64, 64 * 18 - 1), (64, 64 * 18 + 1), (64, 64 * 36 + 5), (64, 64 * 40 - 63),
+                                 (32, 64 * 148 - 1), (32, 64 * 148 + 1), (32, 64 * 300 + 3)])
+def test_schedule_boundaries(P, m, T):
+    import torch
+    dtype = "bf16"
+    code = P.BF16
+    n = m * m
+    d = _small_inputs(m, T, dtype, seed=4242 + T)
+    x, dy, L, R, L2, R2, b1, b2 = (to_device(d[k], dtype) for k in ("x", "dy", "L", "R", "L2", "R2", "b1", "b2"))
+    rows = _sample_tokens(T, 96, 11) if T > 96 else np.arange(T)
+    rows = np.unique(np.concatenate([rows, np.arange(T - 70, T)]))          # always include the ragged tail
+    yf, y = _guarded((T, n), torch.bfloat16)
+    ws = P.Workspace(max(P.monarch_workspace_bytes(P.OP_FWD, T, n, m, code), 256))
+    P.monarch_fwd(x, L, R, y, T, n, m, ws)
+    torch.cuda.synchronize()
+    assert P.monarch_last_device_status(ws) == 0
+    yh = to_host64(y)
+    assert np.isfinite(yh).all()
+    assert_close(yh[rows], O.fwd(d["x"][rows], d["L"], d["R"]), dtype, "y")
+    _check_guard(yf, "y")
+    if m != 64:
+        return
+    dxf, dx = _guarded((T, n), torch.bfloat16)
+    dL = torch.full((m, m, m), float("nan"), dtype=torch.float32, device="cuda")
+    dR = torch.full_like(dL, float("nan"))
+    ws_b = P.Workspace(P.monarch_workspace_bytes(P.OP_BWD, T, n, m, code))
+    P.monarch_bwd(x, dy, L, R, dx, dL, dR, 0, T, n, m, ws_b, fwd_workspace=ws)
+    torch.cuda.synchronize()
+    assert P.monarch_last_device_status(ws_b) == 0
+    ref = O.bwd(d["x"], d["dy"], d["L"], d["R"])
+    dxh = to_host64(dx)
+    assert np.isfinite(dxh).all()
+    assert_close(dxh[rows], ref["dx"][rows], dtype, "dx")
+    assert_close(to_host64(dL), ref["dL"], dtype, "dL")
+    assert_close(to_host64(dR), ref["dR"], dtype, "dR")
+    _check_guard(dxf, "dx")
+    ws_m = P.Workspace(P.monarch_workspace_bytes(P.OP_MLP_FWD, T, n, m, code))
+    P.monarch_mlp_fwd(x, L, R, b1, L2, R2, b2, y, T, n, m, ws_m)
+    torch.cuda.synchronize()
+    assert P.monarch_last_device_status(ws_m) == 0
+    ref_m = O.mlp_fwd(d["x"][rows], d["L"], d["R"], d["b1"], d["L2"], d["R2"], d["b2"])
+    assert_close(to_host64(y)[rows], ref_m, dtype, "mlp y")
+    _check_guard(yf, "mlp y")
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("m,T", [(16, 5), (32, 129), (64, 257), (128, 66)])
 def test_mlp_small(P, impl, m, T, dtype):
