@@ -194,6 +194,40 @@ def test_schedule_boundaries(P, m, T):
     _check_guard(yf, "mlp y")
 
 
+def test_workspace_reuse_across_sizes(P):
+    """One workspace, many calls of different sizes: the per-tile dependency counters must be back at zero after
+    every call, whatever mix of calls and token counts came before."""
+    import torch
+    m, n, dtype, code = 64, 4096, "bf16", P.BF16
+    Tmax = 1300
+    d = _small_inputs(m, Tmax, dtype, seed=99)
+    L, R = to_device(d["L"], dtype), to_device(d["R"], dtype)
+    ws = P.Workspace(max(P.monarch_workspace_bytes(op, Tmax, n, m, code)
+                         for op in (P.OP_FWD, P.OP_BWD_DX, P.OP_BWD_DW, P.OP_BWD, P.OP_MLP_FWD)))
+    ws_f = P.Workspace(P.monarch_workspace_bytes(P.OP_FWD, Tmax, n, m, code))
+    for T in (257, 64, 1300, 130, 1153, 1):
+        x, dy = to_device(d["x"][:T], dtype), to_device(d["dy"][:T], dtype)
+        y, dx = torch.empty_like(x), torch.empty_like(x)
+        dL = torch.empty(m, m, m, dtype=torch.float32, device="cuda")
+        dR = torch.empty_like(dL)
+        ref_y = O.fwd(d["x"][:T], d["L"], d["R"])
+        ref = O.bwd(d["x"][:T], d["dy"][:T], d["L"], d["R"])
+        P.monarch_fwd(x, L, R, y, T, n, m, ws)
+        assert_close(to_host64(y), ref_y, dtype, f"y T={T}")
+        P.monarch_bwd_dx(dy, L, R, dx, T, n, m, ws)
+        assert_close(to_host64(dx), ref["dx"], dtype, f"dx T={T}")
+        P.monarch_bwd_dw(x, dy, L, R, dL, dR, 0, T, n, m, ws)
+        assert_close(to_host64(dL), ref["dL"], dtype, f"dL T={T}")
+        assert_close(to_host64(dR), ref["dR"], dtype, f"dR T={T}")
+        P.monarch_fwd(x, L, R, y, T, n, m, ws_f)
+        P.monarch_bwd(x, dy, L, R, dx, dL, dR, 0, T, n, m, ws, fwd_workspace=ws_f)
+        assert_close(to_host64(dx), ref["dx"], dtype, f"dx one call T={T}")
+        assert_close(to_host64(dL), ref["dL"], dtype, f"dL one call T={T}")
+        assert_close(to_host64(dR), ref["dR"], dtype, f"dR one call T={T}")
+        torch.cuda.synchronize()
+        assert P.monarch_last_device_status(ws) == 0 and P.monarch_last_device_status(ws_f) == 0
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("m,T", [(16, 5), (32, 129), (64, 257), (128, 66)])
 def test_mlp_small(P, impl, m, T, dtype):
