@@ -143,7 +143,7 @@ int monarch_last_device_status(void *workspace, void *stream);
 int monarch_set_impl(int impl);
 
 /* Name of the kernel family the next call with these arguments would use
- * ("staged-simt", "fused-tcgen05", ... ; "unsupported").  Static storage. */
+ * ("staged-simt", "fused-simt", "staged-tcgen05", "fused-tcgen05"; "unsupported").  Static storage. */
 const char *monarch_impl_name(int op, int32_t m, int dtype);
 
 /* Number of kernel launches the library has enqueued since load (for

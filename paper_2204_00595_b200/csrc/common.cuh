@@ -68,6 +68,9 @@ size_t tc_staged_bwd_workspace_bytes(int64_t tokens, int m);
 int tc_staged_bwd(const void *x, const void *dy, const void *L, const void *R, void *dx, float *dL, float *dR,
                   int accumulate, int want_dx, int want_dw, int64_t tokens, int m, void *ws, cudaStream_t s);
 
+// ---- forward for m = 16 in one launch on the CUDA cores, both dtypes (fused_m16.cu); no workspace use ----
+int fused_fwd_m16(const void *x, const void *L, const void *R, void *y, int64_t tokens, int dtype, cudaStream_t s);
+
 // ---- fused forward for m = 32, bf16: both stages inside one CTA (fused_m32.cu); workspace = status word only ----
 int fused_fwd_m32(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws, cudaStream_t s);
 

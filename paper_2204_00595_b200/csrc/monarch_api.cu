@@ -140,6 +140,9 @@ int monarch_fwd(const void *x, const void *L, const void *R, void *y, int64_t to
         return m == 32 ? fused_fwd_m32(x, L, R, y, tokens, workspace, (cudaStream_t)stream)
                        : fused_fwd_m64(x, L, R, y, tokens, workspace, (cudaStream_t)stream);
     if (which == kTcStaged) return tc_staged_fwd(x, L, R, y, tokens, m, workspace, (cudaStream_t)stream);
+    // the automatic choice runs m = 16 in one launch; MONARCH_IMPL_STAGED keeps the two-launch chain
+    if (m == 16 && g_impl.load(std::memory_order_relaxed) == MONARCH_IMPL_AUTO)
+        return fused_fwd_m16(x, L, R, y, tokens, dtype, (cudaStream_t)stream);
     return staged_fwd(x, L, R, y, tokens, m, dtype, workspace, (cudaStream_t)stream);
 }
 
@@ -272,6 +275,9 @@ const char *monarch_impl_name(int op, int32_t m, int dtype)
     if (op < MONARCH_OP_FWD || op > MONARCH_OP_BWD) return "unsupported";
     if (check_shape(0, m * m, m, dtype) != MONARCH_OK) return "unsupported";
     const int which = pick(op, m, dtype);
+    if (which == kSimt && op == MONARCH_OP_FWD && m == 16 &&
+        g_impl.load(std::memory_order_relaxed) == MONARCH_IMPL_AUTO)
+        return "fused-simt";
     return which < 0 ? "unsupported" : which == kFused ? "fused-tcgen05"
          : which == kTcStaged ? "staged-tcgen05" : "staged-simt";
 }
