@@ -176,8 +176,8 @@ def time_oracle(cfg, d, target_s=12.0):
 
 # ----------------------------------------------------------------------------- main
 
-# Kernels behind each timed call (bf16, m = 64), and the DRAM traffic one call generated under ncu
-# (profiles/fused_m64_step_workload3_ncu_full.md; captured at workload 3's full size).
+# Kernels behind each timed call, and the DRAM traffic one call generated under ncu (dram__bytes_read.sum +
+# dram__bytes_write.sum of the call's kernels, captured at workload 3's full size with this script).
 KERNELS_OF = {
     (64, "bf16", "fwd"): "fused_fwd_m64_team_kernel (1 launch)",
     (64, "bf16", "bwd"): "fused_bwd_all_m64_kernel (1 launch, 2 memset nodes)",
@@ -354,7 +354,7 @@ def main():
         "frac": per_call[dom]["gbs"] / peaks["hbm_gbs"], "peak_source": peaks["source"],
         "traffic": NCU_TRAFFIC_MB.get((cfg.index, dom)),
         "traffic_unit": "MB per call (dram__bytes_read.sum + dram__bytes_write.sum, summed over the "
-                        "call's kernels; ncu capture summarised under profiles/)",
+                        "call's kernels, from an ncu capture of this workload at full size)",
         "algorithmic_mb": call_bytes(dom, n, m, T, cfg.dtype) / 1e6,
     }
 
