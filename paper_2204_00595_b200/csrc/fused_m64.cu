@@ -1,4 +1,6 @@
-// Fused Monarch forward for m = 64 (n = 4096), bf16 in/out, fp32 accumulation in TMEM.
+// Fused Monarch forward for m = 64 (n = 4096), bf16 in/out, fp32 accumulation in TMEM: the SPLIT schedule.
+// (The forward call itself uses the team schedule of fused_m64_team.cu, where every CTA does both stages; this
+// kernel serves the stage-1-only launch inside monarch_bwd_dw, and debug builds can select it for comparison.)
 //
 // One persistent launch runs both block-diagonal stages and both permutations; the
 // intermediate u never leaves the chip's L2.  CTAs (one per SM) specialise; both kinds work on
@@ -10,18 +12,16 @@
 //       Per tile, TMA brings x[64 x 64] per block into a 128B-swizzled K-major ring slot;
 //       4 MMAs (N = 64, K = 16) accumulate u[t][k][:] in TMEM columns [64*kb, 64*kb+64) of lane half
 //       (tile parity).  With all 8 accumulators resident, the thread that owns token t picks
-//       entry j of each block - a register renaming - and writes the 16 bytes u'[t][j][8g..8g+8)
-//       into the exchange buffer, whose layout [tile][j][k/8][t%64][k%8] makes that store
-//       coalesced (16 lanes write 256 contiguous bytes) and is at the same time the canonical
-//       no-swizzle K-major operand layout of stage 2: the inner permutation P^T costs no data
-//       movement at all.
+//       entry j of each block - a register renaming - and packs the 16 bytes u'[t][j][8g..8g+8)
+//       of the exchange buffer, whose layout [tile][j][k/8][t%64][k%8] is the canonical no-swizzle
+//       K-major operand layout of stage 2: the inner permutation P^T costs no data movement at all.
 //   S2 CTAs (4 x 2 groups (hj, hl) of `b` CTAs): keep rows [32hl, 32hl+32) of L_{16hj..16hj+15}
 //       resident.  One 8 KB bulk copy per block fetches u'_j[64 x 64] from L2; 4 MMAs (N = 32)
 //       accumulate w[t][j][32hl..]; blocks 0-7 sit in lane half 0 and blocks 8-15 in lane half 1
 //       of 256 TMEM columns (tile parity picks which 256).  Lanes i and i+16 of a warp then hold
-//       blocks j0..j0+7 and j0+8..j0+15 of the same token and store, in one instruction, the 32
-//       contiguous bytes y[t][l*64 + 16hj .. 16hj+16): whole 32-byte sectors, which is what HBM
-//       writes need (16-byte pieces were measured 5x slower).
+//       blocks j0..j0+7 and j0+8..j0+15 of the same token and together form the 32 contiguous
+//       bytes y[t][l*64 + 16hj .. 16hj+16): whole 32-byte sectors, which is what HBM writes need
+//       (16-byte pieces were measured 5x slower).
 //
 // An S2 tile waits (bounded) on a per-tile counter that the S1 epilogues bump after their stores;
 // S1 tiles wait on nothing, so the schedule cannot deadlock.  Warps 0-7 drain TMEM (two per
