@@ -31,19 +31,20 @@ namespace {
 constexpr int kM = 64;
 constexpr int kN = kM * kM;
 // warps: 0-7 epilogue, 8 control/loads, 9 MMA, 10-11 store threads, 12-15 transposers (B1) / loaders (B2),
-// 16 writes the transposed dy out when a caller wants it (B1)
+// 16-17 write the transposed dy out when a caller wants it (B1)
 constexpr int kEpiWarps = 8, kCtlWarp = 8, kMmaWarp = 9, kStoreWarp0 = 10, kAuxWarp0 = 12, kDypWarp = 16;
-constexpr int kThreads = 17 * 32;
+constexpr int kDypWarps = 2;
+constexpr int kThreads = (kDypWarp + kDypWarps) * 32;
 constexpr int kWBytes = 65536;                 // resident weights
 constexpr int kStageBytes = 8192;
 constexpr int kB2StagesPerHalf = 4;
-constexpr int kRawBytes = 16384, kRawBufs = 3;                // B1: one K-step (16 l) of 8 blocks, as loaded
+constexpr int kRawBytes = 16384, kRawBufs = 4;                // B1: one K-step (16 l) of 8 blocks, as loaded
 constexpr int kBlockSlice = 2048 + 16;                        // B1: one block's K-step operand, padded so that
 constexpr int kSliceBytes = 8 * kBlockSlice;                  //     the 8 rows of an stmatrix hit 8 bank groups
 constexpr int kOutRow = 1024 + 16;                            // B1: staged output row (64 tokens x 16 B), padded
 constexpr int kOutBytes = 16 * kOutRow;                       //     one buffer per 16 rows k (TMEM quarter)
 constexpr int kSlotBytes = 8192, kSlots = 12, kQuads = 3;     // B2 operand ring
-constexpr int kSmemBytes = kWBytes + 65536 + 98304 + 512 + 1024;   // 224.5 KB (+ alignment) covers both kinds
+constexpr int kSmemBytes = kWBytes + 65536 + 98304 + 1280 + 1024;  // 226.25 KB incl. alignment: B1 is the largest kind
 static_assert(kWBytes + kRawBufs * kRawBytes + 2 * kSliceBytes + 4 * kOutBytes + 1024 <= kSmemBytes, "B1");
 static_assert(kWBytes + 2 * kB2StagesPerHalf * kStageBytes + kSlots * kSlotBytes + 1024 <= kSmemBytes, "B2");
 constexpr unsigned kB1Arrivals = 8 * 2;        // 8 B1 groups x 2 store warps per tile
@@ -254,9 +255,11 @@ __device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtenso
             }
             w_raw = w_ae = w_tr = 0;
         }
-    } else if (warp == kDypWarp) {
+    } else if (warp >= kDypWarp) {
         // the operand slices are P dy in 2 KB runs [l/8 2][t 64][8 l] per block j: copy them out with plain
-        // coalesced stores (512 contiguous bytes per warp instruction; the TMA unit is busy gathering)
+        // coalesced stores (512 contiguous bytes per warp instruction; the TMA unit is busy gathering).  Each of
+        // the copy warps takes half of the blocks; a slice buffer is free again when the MMAs and both have read it.
+        const int dw = warp - kDypWarp;
         uint32_t n = 0;
         const bool want = p.dyp != nullptr;
         for (int tile = first; tile < p.tiles; tile += step) {
@@ -268,7 +271,7 @@ __device__ __forceinline__ void b1_body(const CUtensorMap &tm_dy3, const CUtenso
                 if (want) {
                     const uint32_t src = a0 + ab * kSliceBytes + lane * 16;
 #pragma unroll 4
-                    for (int i = 0; i < 32; ++i) {
+                    for (int i = dw * 16; i < dw * 16 + 16; ++i) {
                         const int j = i >> 2, off = (i & 3) * 512;
                         uint4 v;
                         asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
@@ -582,7 +585,7 @@ fused_bwd_dx_m64_kernel(const __grid_constant__ CUtensorMap tm_dy3, const __grid
             mbar_init(smem_u32(&bars.acc_full[h]), 1);
             mbar_init(smem_u32(&bars.acc_empty[h]), kEpiWarps);
             mbar_init(smem_u32(&bars.a_full[h]), 4);
-            mbar_init(smem_u32(&bars.a_empty[h]), 2);        // MMA commit + the copy-out thread
+            mbar_init(smem_u32(&bars.a_empty[h]), 1 + kDypWarps);   // MMA commit + the copy-out warps
         }
         for (int h = 0; h < 4; ++h) {
             mbar_init(smem_u32(&bars.raw_full[h]), 1);
@@ -946,7 +949,7 @@ fused_bwd_all_m64_kernel(const __grid_constant__ CUtensorMap tm_dy3, const __gri
             mbar_init(smem_u32(&bars.acc_full[h]), 1);
             mbar_init(smem_u32(&bars.acc_empty[h]), kEpiWarps);
             mbar_init(smem_u32(&bars.a_full[h]), 4);
-            mbar_init(smem_u32(&bars.a_empty[h]), 2);        // MMA commit + the copy-out thread
+            mbar_init(smem_u32(&bars.a_empty[h]), 1 + kDypWarps);   // MMA commit + the copy-out warps
         }
         for (int h = 0; h < 4; ++h) {
             mbar_init(smem_u32(&bars.raw_full[h]), 1);
@@ -1111,9 +1114,9 @@ int fused_bwd_all_m64(const void *x, const void *dy, const void *L, const void *
     p.dR = dR;
     p.tokens = tokens;
     p.tiles = (int)tiles;
-    // SM split by measured cost per tile and group (B1 ~10 k cycles, B2R ~6 k, WL ~6 k with 4 groups only);
-    // 8/6/6 CTAs per group was the best of a sweep on 148 SMs
-    int b1 = (sms * 8) / 144, b2 = (sms * 6) / 144, b3 = (sms * 6) / 144;
+    // SM split: 8/7/6 CTAs per group (8 B1 groups, 8 B2R groups, 4 WL groups: 144 CTAs) was the best of a sweep
+    // on 148 SMs; one CTA per group less of any kind costs 2-10 %
+    int b1 = (sms * 8) / 144, b2 = (sms * 7) / 144, b3 = (sms * 6) / 144;
 #ifdef MONARCH_TRACE
     if (const char *e = getenv("MONARCH_BWD_SPLIT3")) sscanf(e, "%d,%d,%d", &b1, &b2, &b3);
 #endif
@@ -1127,9 +1130,12 @@ int fused_bwd_all_m64(const void *x, const void *dy, const void *L, const void *
     p.b1 = b1;
     p.b2 = b2;
     p.b3 = b3;
-    p.need = kB1Arrivals + 8;                   // du from 16 store warps + P dy from 8 copy warps
+    p.need = kB1Arrivals + 8 * kDypWarps;       // du from 16 store warps + P dy from 16 copy warps
     p.reset_at = p.need + 8 + 4;                // + 8 B2R groups + 4 WL groups
     p.trace = nullptr;
+#ifdef MONARCH_TRACE
+    if (const char *e = getenv("MONARCH_TRACE_PTR_BWD")) p.trace = (long long *)strtoull(e, nullptr, 0);
+#endif
     fused_bwd_all_m64_kernel<<<8 * b1 + 8 * b2 + 4 * b3, kThreads, kSmemBytes, s>>>(tm_dy3, tm_Lt, tm_R, tm_du, tm_dx,
                                                                                  tm_x, p);
     note_launch();
