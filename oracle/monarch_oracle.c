@@ -213,3 +213,66 @@ int oracle_mlp_fwd(const double *x, const double *L1, const double *R1, const do
     }
     return fail;
 }
+
+/* Gradients of  f = <dy, y>  for the feed-forward block above (the paper
+ * trains it by automatic differentiation, Section 4; this is the chain rule
+ * through  a = M1 x + b1,  h = GELU(a),  y = M2 h + b2):
+ *   db2 = sum_t dy[t]
+ *   (dh, dL2, dR2) = adjoints of  y = M2 h  (oracle_bwd with input h)
+ *   da = dh * GELU'(a),   GELU'(a) = (1 + erf(a/sqrt 2))/2 + a exp(-a^2/2)/sqrt(2 pi)
+ *   db1 = sum_t da[t]
+ *   (dx, dL1, dR1) = adjoints of  a = M1 x  (oracle_bwd with output gradient da)
+ * All outputs are overwritten.  Any output may be NULL. */
+int oracle_mlp_bwd(const double *x, const double *dy, const double *L1, const double *R1,
+                   const double *b1, const double *L2, const double *R2, double *dx,
+                   double *dL1, double *dR1, double *db1, double *dL2, double *dR2, double *db2,
+                   long T, int m)
+{
+    const size_t n = (size_t)m * m;
+    double *a = (double *)malloc((size_t)T * n * sizeof(double));
+    double *h = (double *)malloc((size_t)T * n * sizeof(double));
+    double *dh = (double *)malloc((size_t)T * n * sizeof(double));
+    int fail = !a || !h || !dh;
+    if (!fail) fail = oracle_fwd(x, L1, R1, a, NULL, T, m);
+    if (!fail) {
+#pragma omp parallel for schedule(static)
+        for (long t = 0; t < T; ++t)
+            for (size_t q = 0; q < n; ++q) {
+                const double v = a[(size_t)t * n + q] + b1[q];
+                a[(size_t)t * n + q] = v;
+                h[(size_t)t * n + q] = 0.5 * v * (1.0 + erf(v / sqrt(2.0)));
+            }
+        fail = oracle_bwd(h, dy, L2, R2, dh, dL2, dR2, T, m);
+    }
+    if (!fail) {
+        const double inv_sqrt_2pi = 1.0 / sqrt(2.0 * acos(-1.0));
+#pragma omp parallel for schedule(static)
+        for (long t = 0; t < T; ++t)
+            for (size_t q = 0; q < n; ++q) {
+                const double v = a[(size_t)t * n + q];
+                const double g = 0.5 * (1.0 + erf(v / sqrt(2.0))) + v * exp(-0.5 * v * v) * inv_sqrt_2pi;
+                dh[(size_t)t * n + q] *= g;                 /* now da */
+            }
+        if (db1) {
+#pragma omp parallel for schedule(static)
+            for (size_t q = 0; q < n; ++q) {
+                double acc = 0.0;
+                for (long t = 0; t < T; ++t) acc += dh[(size_t)t * n + q];
+                db1[q] = acc;
+            }
+        }
+        if (db2) {
+#pragma omp parallel for schedule(static)
+            for (size_t q = 0; q < n; ++q) {
+                double acc = 0.0;
+                for (long t = 0; t < T; ++t) acc += dy[(size_t)t * n + q];
+                db2[q] = acc;
+            }
+        }
+        fail = oracle_bwd(x, dh, L1, R1, dx, dL1, dR1, T, m);
+    }
+    free(a);
+    free(h);
+    free(dh);
+    return fail;
+}

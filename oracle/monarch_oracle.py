@@ -9,7 +9,8 @@ Two layers:
 
 * ``monarch_oracle.c`` - plain C loops in fp64 over the paper's multiply
   steps (Section 3.3, steps 1-3), their adjoints, the entry formula Eq. (2)
-  and the Monarch feed-forward block.  Compiled on demand with gcc.
+  and the Monarch feed-forward block with its gradients.  Compiled on demand
+  with gcc.
 * numpy routines in this file that restate *Definition 3.1 literally*
   (explicit permutation and block-diagonal matrices) and Algorithm 1
   (projection by rank-1 SVDs).  They are the independent routes the C loops
@@ -59,6 +60,8 @@ def _load():
         lib.oracle_bwd.argtypes = [dp] * 7 + [ctypes.c_long, ctypes.c_int]
         lib.oracle_mlp_fwd.restype = ctypes.c_int
         lib.oracle_mlp_fwd.argtypes = [dp] * 8 + [ctypes.c_long, ctypes.c_int]
+        lib.oracle_mlp_bwd.restype = ctypes.c_int
+        lib.oracle_mlp_bwd.argtypes = [dp] * 14 + [ctypes.c_long, ctypes.c_int]
         _lib = lib
     return _lib
 
@@ -141,6 +144,29 @@ def mlp_fwd(x, L1, R1, b1, L2, R2, b2):
                               _p(y), T, m):
         raise MemoryError("oracle_mlp_fwd")
     return y
+
+
+def mlp_bwd(x, dy, L1, R1, b1, L2, R2):
+    """Gradients of <dy, y> for y = M2 GELU(M1 x + b1) + b2 (chain rule through the block).
+
+    Returns dict with dx [T, n], dL1, dR1, dL2, dR2 [m, m, m], db1, db2 [n].
+    """
+    L1 = _f64(L1); R1 = _f64(R1); L2 = _f64(L2); R2 = _f64(R2)
+    m = _m_of(L1); n = m * m
+    b1 = _f64(b1, (n,))
+    x = _f64(x); dy = _f64(dy); T = x.shape[0]
+    if x.shape != (T, n) or dy.shape != (T, n):
+        raise ValueError("shape mismatch")
+    out = {"dx": np.empty((T, n))}
+    for k in ("dL1", "dR1", "dL2", "dR2"):
+        out[k] = np.empty((m, m, m))
+    out["db1"] = np.empty(n)
+    out["db2"] = np.empty(n)
+    if _load().oracle_mlp_bwd(_p(x), _p(dy), _p(L1), _p(R1), _p(b1), _p(L2), _p(R2), _p(out["dx"]),
+                              _p(out["dL1"]), _p(out["dR1"]), _p(out["db1"]), _p(out["dL2"]),
+                              _p(out["dR2"]), _p(out["db2"]), T, m):
+        raise MemoryError("oracle_mlp_bwd")
+    return out
 
 
 # --------------------------------------------------------------------------

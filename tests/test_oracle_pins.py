@@ -326,3 +326,88 @@ def test_mlp_special_cases():
     gp = O.mlp_fwd(a, I, I, np.zeros(n), I, I, np.zeros(n))
     gm = O.mlp_fwd(-a, I, I, np.zeros(n), I, I, np.zeros(n))
     assert np.allclose(gp - gm, a, atol=1e-14)
+
+
+def _mlp_args(rng, m, T):
+    n = m * m
+    x, dy = _rand(rng, T, n), _rand(rng, T, n)
+    W = [_rand(rng, m, m, m) / math.sqrt(m) for _ in range(4)]
+    b1, b2 = 0.3 * _rand(rng, n), 0.3 * _rand(rng, n)
+    return x, dy, W, b1, b2
+
+
+@pytest.mark.parametrize("m", [2, 4])
+def test_mlp_gradients_by_finite_differences(m):
+    # f = <dy, y(x, L1, R1, b1, L2, R2, b2)>; central differences of the pinned forward.
+    rng = np.random.default_rng(21)
+    x, dy, W, b1, b2 = _mlp_args(rng, m, 3)
+    g = O.mlp_bwd(x, dy, W[0], W[1], b1, W[2], W[3])
+    args = {"x": x, "L1": W[0], "R1": W[1], "b1": b1, "L2": W[2], "R2": W[3], "b2": b2}
+
+    def f():
+        return np.sum(dy * O.mlp_fwd(args["x"], args["L1"], args["R1"], args["b1"], args["L2"],
+                                     args["R2"], args["b2"]))
+
+    h = 1e-6
+    for name, key in [("x", "dx"), ("L1", "dL1"), ("R1", "dR1"), ("b1", "db1"), ("L2", "dL2"),
+                      ("R2", "dR2"), ("b2", "db2")]:
+        v = args[name]
+        num = np.zeros_like(v)
+        it = np.nditer(v, flags=["multi_index"])
+        for _ in it:
+            idx = it.multi_index
+            keep = v[idx]
+            v[idx] = keep + h
+            fp = f()
+            v[idx] = keep - h
+            fm = f()
+            v[idx] = keep
+            num[idx] = (fp - fm) / (2 * h)
+        assert np.allclose(g[key], num, rtol=1e-6, atol=1e-7), name
+
+
+def test_mlp_gradients_special_cases():
+    rng = np.random.default_rng(22)
+    m, T = 4, 6
+    n = m * m
+    x, dy, W, b1, b2 = _mlp_args(rng, m, T)
+    I = np.stack([np.eye(m)] * m)
+    # identities: y = GELU(x + b1) + b2, so dx = dy * GELU'(x + b1) with the derivative taken
+    # numerically from the textbook-pinned GELU, and db1 = sum_t dx, db2 = sum_t dy.
+    g = O.mlp_bwd(x, dy, I, I, b1, I, I)
+    e = 1e-6
+    dgelu = (_gelu(x + b1 + e) - _gelu(x + b1 - e)) / (2 * e)
+    assert np.allclose(g["dx"], dy * dgelu, atol=1e-8)
+    assert np.allclose(g["db1"], (dy * dgelu).sum(0), atol=1e-8)
+    assert np.allclose(g["db2"], dy.sum(0), atol=1e-12)
+    # GELU'(0) = 1/2: zero first layer and zero bias give da = dh / 2, dx = 0
+    Z = np.zeros((m, m, m))
+    g = O.mlp_bwd(x, dy, Z, Z, np.zeros(n), W[2], W[3])
+    M2 = O.dense_from_definition(W[2], W[3])
+    assert np.allclose(g["db1"], 0.5 * (dy @ M2).sum(0), atol=1e-11)
+    assert not g["dx"].any() and not g["dL2"].any() and not g["dR2"].any()
+    # general: chain rule through the dense matrices of Definition 3.1
+    M1 = O.dense_from_definition(W[0], W[1])
+    a = x @ M1.T + b1
+    dgelu = (_gelu(a + e) - _gelu(a - e)) / (2 * e)
+    da = (dy @ M2) * dgelu
+    g = O.mlp_bwd(x, dy, W[0], W[1], b1, W[2], W[3])
+    assert np.allclose(g["dx"], da @ M1, atol=1e-7)
+    # second layer: the plain Monarch adjoints with input h; Euler identity <dL2, L2> = <dy, y - b2>
+    y = O.mlp_fwd(x, W[0], W[1], b1, W[2], W[3], b2)
+    s = np.sum(dy * (y - b2))
+    assert np.isclose(np.sum(g["dL2"] * W[2]), s, rtol=1e-12)
+    assert np.isclose(np.sum(g["dR2"] * W[3]), s, rtol=1e-12)
+    # first layer: <dL1, L1> = <dR1, R1> = <da, a - b1>
+    s1 = np.sum(da * (a - b1))
+    assert np.isclose(np.sum(g["dL1"] * W[0]), s1, rtol=1e-6)
+    assert np.isclose(np.sum(g["dR1"] * W[1]), s1, rtol=1e-6)
+
+
+def test_mlp_bwd_empty():
+    rng = np.random.default_rng(23)
+    m = 4
+    x, dy, W, b1, b2 = _mlp_args(rng, m, 2)
+    g = O.mlp_bwd(x[:0], dy[:0], W[0], W[1], b1, W[2], W[3])
+    assert g["dx"].shape == (0, m * m)
+    assert not any(g[k].any() for k in ("dL1", "dR1", "db1", "dL2", "dR2", "db2"))
