@@ -52,7 +52,7 @@ def esize(dtype):
 
 def call_flops(call, n, m, T):
     """Algorithmic FLOPs: 4 n m per token per pass (two block-diagonal stages of 2 n m each)."""
-    return {"fwd": 4, "bwd_dx": 4, "bwd_dw": 4, "bwd": 8, "mlp_fwd": 8}[call] * n * m * T
+    return {"fwd": 4, "bwd_dx": 4, "bwd_dw": 4, "bwd": 8, "mlp_fwd": 8, "mlp_bwd": 16}[call] * n * m * T
 
 
 def call_bytes(call, n, m, T, dtype):
@@ -67,6 +67,8 @@ def call_bytes(call, n, m, T, dtype):
         return 3 * T * n * s + w + 2 * n * m * 4
     if call == "mlp_fwd":
         return 2 * T * n * s + 2 * w + 2 * n * s
+    if call == "mlp_bwd":      # read x, dy; write dx and the six parameter gradients
+        return 3 * T * n * s + 2 * w + n * s + 4 * n * m * 4 + 2 * n * 4
     raise ValueError(call)
 
 
@@ -142,11 +144,12 @@ class ClockSampler:
 
 # ----------------------------------------------------------------------------- CPU oracle timing
 
-def time_oracle(cfg, d, target_s=12.0):
+def time_oracle(cfg, d, target_s=12.0, calls=None):
     """Time the oracle (as it stands) on a bounded token sample of the workload."""
     from oracle import monarch_oracle as O
     c = cfg
-    calls = list(c.ops)
+    calls = list(c.ops) if calls is None else [k for k in calls if k != "bwd"] + (
+        ["bwd_dx", "bwd_dw"] if "bwd" in calls else [])
 
     def run(T):
         t0 = time.perf_counter()
@@ -158,6 +161,8 @@ def time_oracle(cfg, d, target_s=12.0):
             O.bwd(d["x"][:T], d["dy"][:T], d["L"], d["R"], want=want)
         if "mlp_fwd" in calls:
             O.mlp_fwd(d["x"][:T], d["L"], d["R"], d["b1"], d["L2"], d["R2"], d["b2"])
+        if "mlp_bwd" in calls:
+            O.mlp_bwd(d["x"][:T], d["dy"][:T], d["L"], d["R"], d["b1"], d["L2"], d["R2"])
         return time.perf_counter() - t0
 
     T = min(32, c.tokens)
@@ -182,6 +187,8 @@ KERNELS_OF = {
     (64, "bf16", "fwd"): "fused_fwd_m64_team_kernel (1 launch)",
     (64, "bf16", "bwd"): "fused_bwd_all_m64_kernel (1 launch, 2 memset nodes)",
     (64, "bf16", "mlp_fwd"): "fused_fwd_m64_team_kernel (2 launches)",
+    (64, "bf16", "mlp_bwd"): "fused_fwd_m64_team_kernel + mlp_act_kernel + fused_fwd_m64_kernel (stage 1 only) + "
+                             "2 x fused_bwd_all_m64_kernel + mlp_dact_kernel + merge_status_kernel (7 launches)",
     (32, "bf16", "fwd"): "fused_fwd_m32_kernel (1 launch)",
     (64, "bf16", "bwd_dx"): "fused_bwd_dx_m64_kernel (1 launch)",
     (64, "bf16", "bwd_dw"): "fused_fwd_m64_kernel (stage 1 only) + fused_bwd_dx_m64_kernel (stage 1 only) + "
@@ -199,7 +206,9 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     calls = list(cfg.ops)
     if args.calls:
-        calls = [k for k in calls if k in args.calls.split(",")]
+        # the backward of the feed-forward block is an optional extra call of the workload that has the block
+        extra = ["mlp_bwd"] if "mlp_fwd" in calls else []
+        calls = [k for k in calls + extra if k in args.calls.split(",")]
     elif calls == ["fwd", "bwd_dx", "bwd_dw"]:
         # default: the backward pass as one call (dx, dL, dR) that reuses the intermediate the forward
         # call left in its workspace; --calls fwd,bwd_dx,bwd_dw times the three separate entry points
@@ -216,10 +225,11 @@ def main():
         import __graft_entry__ as entry
         from oracle import monarch_oracle as O
         O.build()
-        d = make_inputs(cfg.index)
+        d = make_inputs(cfg.index, with_dy="mlp_bwd" in calls)
         times, sample = [], None
         for i in range(args.warmup + args.steps):
-            r = time_oracle(cfg, d, target_s=max(1.0, min(8.0, 120.0 / (args.warmup + args.steps))))
+            r = time_oracle(cfg, d, target_s=max(1.0, min(8.0, 120.0 / (args.warmup + args.steps))),
+                            calls=calls)
             sample = r
             if i >= args.warmup:
                 times.append(r)
@@ -253,7 +263,7 @@ def main():
 
     code = P.F32 if cfg.dtype == "f32" else P.BF16
     tdt = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
-    d = make_inputs(cfg.index)              # every rank draws the same recipe, then offsets it
+    d = make_inputs(cfg.index, with_dy="mlp_bwd" in calls)   # every rank draws the same recipe, then offsets it
     from tests.helpers import to_device
 
     # Two rotating sets of token tensors so that no launch finds its operands in L2 from the
@@ -271,9 +281,12 @@ def main():
         sets.append(e)
     W = {k: to_device(d[k], cfg.dtype) for k in ("L", "R", "L2", "R2", "b1", "b2") if k in d}
     grads = torch.zeros(2, m, m, m, dtype=torch.float32, device="cuda")   # packed (dL, dR)
+    mlp_grads = [torch.zeros(m, m, m, dtype=torch.float32, device="cuda") for _ in range(4)] + \
+                [torch.zeros(n, dtype=torch.float32, device="cuda") for _ in range(2)]   # dL1 dR1 dL2 dR2 db1 db2
     op_of = {"fwd": P.OP_FWD, "bwd_dx": P.OP_BWD_DX, "bwd_dw": P.OP_BWD_DW, "mlp_fwd": P.OP_MLP_FWD,
-             "bwd": P.OP_BWD}
-    ws = P.Workspace(max(P.monarch_workspace_bytes(op_of[k], T, n, m, code) for k in calls if k != "bwd"))
+             "bwd": P.OP_BWD, "mlp_bwd": P.OP_MLP_BWD}
+    ws = P.Workspace(max([P.monarch_workspace_bytes(op_of[k], T, n, m, code) for k in calls if k != "bwd"]
+                         + [256]))
     ws_b = P.Workspace(P.monarch_workspace_bytes(P.OP_BWD, T, n, m, code)) if "bwd" in calls else None
     stream = torch.cuda.current_stream()
 
@@ -301,6 +314,13 @@ def main():
             elif k == "mlp_fwd":
                 P.monarch_mlp_fwd(e["x"], W["L"], W["R"], W["b1"], W["L2"], W["R2"], W["b2"],
                                   e["y"], T, n, m, ws)
+            elif k == "mlp_bwd":
+                g = mlp_grads
+                P.monarch_mlp_bwd(e["x"], e["dy"], W["L"], W["R"], W["b1"], W["L2"], W["R2"], e["dx"],
+                                  g[0], g[1], g[4], g[2], g[3], g[5], 0, T, n, m, ws)
+                if dist is not None:
+                    for t in g:
+                        dist.all_reduce(t)
             if timed:
                 nmark[0] += 1
                 marks[nmark[0]].record(stream)
@@ -414,7 +434,7 @@ def main():
             ctx.close()
         line["e2e"] = e2e
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        r = time_oracle(cfg, d)
+        r = time_oracle(cfg, d, calls=calls)
         line["cpu_baseline"] = {"value": r["tflops"], "unit": unit, "cores": r["cores"],
                                 "kind": "oracle", "tokens_per_s": r["tokens_per_s"],
                                 "sample": f"first {r['tokens']} tokens of the workload, "

@@ -66,7 +66,8 @@ typedef enum {
     MONARCH_OP_BWD_DX = 1,
     MONARCH_OP_BWD_DW = 2,
     MONARCH_OP_MLP_FWD = 3,
-    MONARCH_OP_BWD = 4 /* monarch_bwd: dx, dL and dR in one call */
+    MONARCH_OP_BWD = 4, /* monarch_bwd: dx, dL and dR in one call */
+    MONARCH_OP_MLP_BWD = 5
 } monarch_op_t;
 
 /* Which kernel family serves a call (process-wide; default AUTO). */
@@ -120,6 +121,25 @@ int monarch_bwd(const void *x, const void *dy, const void *L, const void *R,
 int monarch_mlp_fwd(const void *x, const void *L1, const void *R1, const void *b1,
                     const void *L2, const void *R2, const void *b2, void *y,
                     int64_t tokens, int32_t n, int32_t m, int dtype,
+                    void *workspace, size_t workspace_bytes, void *stream);
+
+/* Gradients of f = <dy, y> for the feed-forward block above (Section 4 trains
+ * it by automatic differentiation; this is that chain rule):
+ *   a = M1 x + b1,  h = GELU(a)                       (recomputed inside)
+ *   dh = M2^T dy,   dL2, dR2 = block gradients of M2 with input h,   db2 = sum_t dy[t]
+ *   da = dh * GELU'(a),  GELU'(a) = (1 + erf(a/sqrt 2))/2 + a exp(-a^2/2)/sqrt(2 pi)
+ *   dx = M1^T da,   dL1, dR1 = block gradients of M1 with input x,   db1 = sum_t da[t]
+ * x, dy, dx: [tokens][n] in the storage dtype; b1: [n] storage dtype (b2 does
+ * not enter the gradients).  dL1, dR1, dL2, dR2: float32 [m][m][m]; db1, db2:
+ * float32 [n]; accumulate == 0 overwrites all six, 1 adds to their contents.
+ * a, h and da are rounded to the storage dtype once each (they are tensor-core
+ * operands).  The sums over tokens use atomic adds: their order, hence the
+ * last bits, may vary from run to run.  Workspace: monarch_workspace_bytes
+ * with MONARCH_OP_MLP_BWD. */
+int monarch_mlp_bwd(const void *x, const void *dy, const void *L1, const void *R1, const void *b1,
+                    const void *L2, const void *R2, void *dx,
+                    float *dL1, float *dR1, float *db1, float *dL2, float *dR2, float *db2,
+                    int accumulate, int64_t tokens, int32_t n, int32_t m, int dtype,
                     void *workspace, size_t workspace_bytes, void *stream);
 
 /* Bytes of workspace `op` (a monarch_op_t) needs for these sizes under the

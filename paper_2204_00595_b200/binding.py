@@ -10,7 +10,7 @@ import ctypes
 import os
 
 F32, BF16 = 0, 1
-OP_FWD, OP_BWD_DX, OP_BWD_DW, OP_MLP_FWD, OP_BWD = 0, 1, 2, 3, 4
+OP_FWD, OP_BWD_DX, OP_BWD_DW, OP_MLP_FWD, OP_BWD, OP_MLP_BWD = 0, 1, 2, 3, 4, 5
 IMPL_AUTO, IMPL_STAGED, IMPL_FUSED = 0, 1, 2
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libmonarch.so")
@@ -25,6 +25,7 @@ _SIGNATURES = {
                               _sz, _vp]),
     "monarch_mlp_fwd": (_int, [_vp] * 8 + [_i64, _i32, _i32, _int, _vp, _sz, _vp]),
     "monarch_bwd": (_int, [_vp] * 8 + [_int, _i64, _i32, _i32, _int, _vp, _sz, _vp]),
+    "monarch_mlp_bwd": (_int, [_vp] * 14 + [_int, _i64, _i32, _i32, _int, _vp, _sz, _vp]),
     "monarch_workspace_bytes": (_sz, [_int, _i64, _i32, _i32, _int]),
     "monarch_workspace_init": (_int, [_vp, _sz, _vp]),
     "monarch_last_device_status": (_int, [_vp, _vp]),
@@ -205,6 +206,20 @@ def monarch_mlp_fwd(x, L1, R1, b1, L2, R2, b2, y, tokens, n, m, workspace, strea
                                  _ptr(b1, "b1", dt), _ptr(L2, "L2", dt), _ptr(R2, "R2", dt),
                                  _ptr(b2, "b2", dt), _ptr(y, "y", dt), tokens, n, m,
                                  _dtype_code(x), p, b, _stream(stream)), "monarch_mlp_fwd")
+
+
+def monarch_mlp_bwd(x, dy, L1, R1, b1, L2, R2, dx, dL1, dR1, db1, dL2, dR2, db2, accumulate, tokens, n, m,
+                    workspace, stream=None) -> None:
+    """Gradients of <dy, y> for y = M2 GELU(M1 x + b1) + b2; weight and bias gradients are float32."""
+    import torch
+    dt, f32 = x.dtype, torch.float32
+    p, b = _ws(workspace)
+    _check(lib().monarch_mlp_bwd(_ptr(x, "x"), _ptr(dy, "dy", dt), _ptr(L1, "L1", dt), _ptr(R1, "R1", dt),
+                                 _ptr(b1, "b1", dt), _ptr(L2, "L2", dt), _ptr(R2, "R2", dt),
+                                 _ptr(dx, "dx", dt), _ptr(dL1, "dL1", f32), _ptr(dR1, "dR1", f32),
+                                 _ptr(db1, "db1", f32), _ptr(dL2, "dL2", f32), _ptr(dR2, "dR2", f32),
+                                 _ptr(db2, "db2", f32), int(accumulate), tokens, n, m, _dtype_code(x),
+                                 p, b, _stream(stream)), "monarch_mlp_bwd")
 
 
 NOALLOC_SCRATCH_BYTES = 8 << 20

@@ -85,6 +85,9 @@ int fused_fwd_m64_team(const void *x, const void *L, const void *R, void *y, int
 size_t fused_mlp_fwd_m64_workspace_bytes(int64_t tokens);
 int fused_mlp_fwd_m64(const void *x, const void *L1, const void *R1, const void *b1, const void *L2,
                       const void *R2, const void *b2, void *y, int64_t tokens, void *ws, cudaStream_t s);
+// one pass y = act(M x + bias), act = GELU or identity; workspace layout of fused_fwd_m64 (u stays behind)
+int fused_fwd_bias_m64(const void *x, const void *L, const void *R, const void *bias, int gelu, void *y,
+                       int64_t tokens, void *ws, cudaStream_t s);
 // first stage only: u = P R x in the exchange layout [tile][j][k/8][t%64][k%8] (tokens rounded up to 64)
 int fused_fwd_m64_stage1(const void *x, const void *R, void *u, int64_t tokens, unsigned *status,
                          cudaStream_t s);
@@ -117,5 +120,14 @@ int fused_bwd_m64(const void *x, const void *dy, const void *L, const void *R, c
                   cudaStream_t s);
 // where the fused forward keeps u inside its workspace
 const void *fused_fwd_m64_saved_u(const void *fwd_ws);
+
+// ---- elementwise steps of the feed-forward block's backward pass (mlp_bwd.cu) ----
+// h = GELU(a (+ b1)); b1 may be null when a already holds the bias
+int mlp_act(const void *a, const void *b1, void *h, int64_t tokens, int n, int dtype, cudaStream_t s);
+// dh <- dh * GELU'(a (+ b1)) in place, db1 += column sums of the result, db2 += column sums of dy
+int mlp_dact(void *dh, const void *a, const void *b1, const void *dy, float *db1, float *db2, int64_t tokens, int n,
+             int dtype, cudaStream_t s);
+// fold the status word of an inner workspace into the outer one and clear it
+int merge_status(unsigned *outer, unsigned *inner, cudaStream_t s);
 
 }  // namespace monarch

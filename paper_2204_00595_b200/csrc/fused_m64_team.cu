@@ -565,6 +565,15 @@ int fused_fwd_m64_team(const void *x, const void *L, const void *R, void *y, int
                        (unsigned *)((char *)ws + MONARCH_STATUS_BYTES), (unsigned *)ws, tokens, s);
 }
 
+// One pass with the bias (and optionally GELU) applied in the stage-2 epilogue: y = act(M x + bias).
+int fused_fwd_bias_m64(const void *x, const void *L, const void *R, const void *bias, int gelu, void *y,
+                       int64_t tokens, void *ws, cudaStream_t s)
+{
+    if (tokens == 0) return MONARCH_OK;
+    return launch_team(x, L, R, bias, gelu, y, (char *)ws + MONARCH_STATUS_BYTES + kTeamCounterBytes,
+                       (unsigned *)((char *)ws + MONARCH_STATUS_BYTES), (unsigned *)ws, tokens, s);
+}
+
 // Feed-forward block y = M2 GELU(M1 x + b1) + b2 as two passes of the same kernel; the hidden activations h
 // (bf16) live in the workspace: [status][counters][u'][h].
 size_t fused_mlp_fwd_m64_workspace_bytes(int64_t tokens)

@@ -95,6 +95,27 @@ int pick(int op, int m, int dtype)
     return tc_staged_available(op, m, dtype) ? kTcStaged : kSimt;
 }
 
+// Workspace of monarch_mlp_bwd: [backward workspace (status word first)][forward workspace][a][h][dh]
+struct MlpBwdLayout {
+    size_t ws_b, ws_f, act, off_f, off_a, off_h, off_dh, total;
+};
+
+size_t round256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+MlpBwdLayout mlp_bwd_layout(int64_t tokens, int32_t n, int32_t m, int dtype)
+{
+    MlpBwdLayout l;
+    l.ws_b = round256(monarch_workspace_bytes(MONARCH_OP_BWD, tokens, n, m, dtype));
+    l.ws_f = round256(monarch_workspace_bytes(MONARCH_OP_FWD, tokens, n, m, dtype));
+    l.act = round256((size_t)tokens * n * esize(dtype));
+    l.off_f = l.ws_b;
+    l.off_a = l.off_f + l.ws_f;
+    l.off_h = l.off_a + l.act;
+    l.off_dh = l.off_h + l.act;
+    l.total = l.off_dh + l.act;
+    return l;
+}
+
 }  // namespace
 }  // namespace monarch
 
@@ -104,8 +125,12 @@ extern "C" {
 
 size_t monarch_workspace_bytes(int op, int64_t tokens, int32_t n, int32_t m, int dtype)
 {
-    if (op < MONARCH_OP_FWD || op > MONARCH_OP_BWD) return 0;
+    if (op < MONARCH_OP_FWD || op > MONARCH_OP_MLP_BWD) return 0;
     if (check_shape(tokens, n, m, dtype) != MONARCH_OK) return 0;
+    if (op == MONARCH_OP_MLP_BWD) {
+        const MlpBwdLayout lay = mlp_bwd_layout(tokens, n, m, dtype);
+        return lay.ws_b == 0 || lay.ws_f == 0 ? 0 : lay.total;
+    }
     const int which = pick(op, m, dtype);
     if (which < 0) return 0;
     if (which == kTcStaged && op != MONARCH_OP_FWD && op != MONARCH_OP_MLP_FWD)
@@ -238,6 +263,50 @@ int monarch_mlp_fwd(const void *x, const void *L1, const void *R1, const void *b
                           (cudaStream_t)stream);
 }
 
+int monarch_mlp_bwd(const void *x, const void *dy, const void *L1, const void *R1, const void *b1,
+                    const void *L2, const void *R2, void *dx, float *dL1, float *dR1, float *db1,
+                    float *dL2, float *dR2, float *db2, int accumulate, int64_t tokens, int32_t n,
+                    int32_t m, int dtype, void *workspace, size_t workspace_bytes, void *stream)
+{
+    MONARCH_TRY(check_shape(tokens, n, m, dtype));
+    if (accumulate != 0 && accumulate != 1) return MONARCH_ERR_INVALID_ARG;
+    const size_t act = (size_t)tokens * n * esize(dtype), wb = (size_t)n * m * esize(dtype);
+    const size_t bb = (size_t)n * esize(dtype), gb = (size_t)n * m * sizeof(float);
+    const size_t gbias = (size_t)n * sizeof(float);
+    const Range in[] = {{x, act}, {dy, act}, {L1, wb}, {R1, wb}, {b1, bb}, {L2, wb}, {R2, wb}};
+    const Range out[] = {{dx, act}, {dL1, gb}, {dR1, gb}, {db1, gbias}, {dL2, gb}, {dR2, gb}, {db2, gbias}};
+    const MlpBwdLayout lay = mlp_bwd_layout(tokens, n, m, dtype);
+    if (lay.ws_b == 0 || lay.ws_f == 0) return MONARCH_ERR_UNSUPPORTED;
+    MONARCH_TRY(check_buffers(in, 7, out, 7, workspace, workspace_bytes, lay.total));
+    cudaStream_t s = (cudaStream_t)stream;
+    if (!accumulate) {
+        MONARCH_CUDA_TRY(cudaMemsetAsync(db1, 0, gbias, s));
+        MONARCH_CUDA_TRY(cudaMemsetAsync(db2, 0, gbias, s));
+    }
+    char *ws = (char *)workspace;
+    void *ws_b = ws, *ws_f = ws + lay.off_f;
+    void *a = ws + lay.off_a, *h = ws + lay.off_h, *dh = ws + lay.off_dh;
+    // the inner forward workspace starts with its own status word and tile counters
+    MONARCH_TRY(monarch_workspace_init(ws_f, lay.ws_f, stream));
+    // a = M1 x + b1: the fused m = 64 forward adds the bias in its epilogue, the others leave it to the
+    // elementwise kernels (a then holds M1 x)
+    const bool bias_in_a = pick(MONARCH_OP_FWD, m, dtype) == kFused && m == 64;
+    if (bias_in_a)
+        MONARCH_TRY(fused_fwd_bias_m64(x, L1, R1, b1, 0, a, tokens, ws_f, s));
+    else
+        MONARCH_TRY(monarch_fwd(x, L1, R1, a, tokens, n, m, dtype, ws_f, lay.ws_f, stream));
+    const void *b1_late = bias_in_a ? nullptr : b1;
+    MONARCH_TRY(mlp_act(a, b1_late, h, tokens, n, dtype, s));
+    // second matrix: dh = M2^T dy and its block gradients, input h
+    MONARCH_TRY(monarch_bwd(h, dy, L2, R2, nullptr, dh, dL2, dR2, accumulate, tokens, n, m, dtype, ws_b,
+                            lay.ws_b, stream));
+    MONARCH_TRY(mlp_dact(dh, a, b1_late, dy, db1, db2, tokens, n, dtype, s));
+    // first matrix: dx = M1^T da and its block gradients; u = P^T R1 x is still in the forward workspace
+    MONARCH_TRY(monarch_bwd(x, dh, L1, R1, ws_f, dx, dL1, dR1, accumulate, tokens, n, m, dtype, ws_b, lay.ws_b,
+                            stream));
+    return merge_status((unsigned *)ws_b, (unsigned *)ws_f, s);
+}
+
 int monarch_workspace_init(void *workspace, size_t workspace_bytes, void *stream)
 {
     if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < MONARCH_STATUS_BYTES)
@@ -272,8 +341,9 @@ int monarch_set_impl(int impl)
 
 const char *monarch_impl_name(int op, int32_t m, int dtype)
 {
-    if (op < MONARCH_OP_FWD || op > MONARCH_OP_BWD) return "unsupported";
+    if (op < MONARCH_OP_FWD || op > MONARCH_OP_MLP_BWD) return "unsupported";
     if (check_shape(0, m * m, m, dtype) != MONARCH_OK) return "unsupported";
+    if (op == MONARCH_OP_MLP_BWD) op = MONARCH_OP_BWD;      // its Monarch passes are monarch_bwd's
     const int which = pick(op, m, dtype);
     if (which == kSimt && op == MONARCH_OP_FWD && m == 16 &&
         g_impl.load(std::memory_order_relaxed) == MONARCH_IMPL_AUTO)

@@ -70,13 +70,14 @@ def round_to_storage(a: np.ndarray, dtype: str) -> np.ndarray:
 
 
 def make_inputs(config: int, tokens: int | None = None, m: int | None = None,
-                dtype: str | None = None, seed: int | None = None) -> dict:
+                dtype: str | None = None, seed: int | None = None, with_dy: bool = False) -> dict:
     """Draw the tensors of workload ``config`` (1..5).
 
     ``tokens``, ``m`` and ``dtype`` override the workload's values (for small
     parity cases of the same distribution).  Returns float32 arrays already
     rounded to the storage dtype, plus the scalars ``m``, ``n``, ``tokens``,
-    ``dtype``.
+    ``dtype``.  ``with_dy`` adds an output gradient ``dy`` to workloads that
+    do not list a backward call (for the backward of the feed-forward block).
     """
     c = CONFIGS[config]
     T = c.tokens if tokens is None else int(tokens)
@@ -101,4 +102,6 @@ def make_inputs(config: int, tokens: int | None = None, m: int | None = None,
         out["R2"] = draw((mm, mm, mm), std_w)
         out["b1"] = draw((n,), c.std_b)
         out["b2"] = draw((n,), c.std_b)
+    if with_dy and "dy" not in out:
+        out["dy"] = draw((T, n), 1.0)      # drawn last: the tensors above do not depend on the flag
     return out

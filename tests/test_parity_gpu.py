@@ -247,6 +247,77 @@ def test_mlp_small(P, impl, m, T, dtype):
     _check_guard(yf, "mlp y")
 
 
+MLP_GRADS = ("dL1", "dR1", "db1", "dL2", "dR2", "db2")
+
+
+def _mlp_bwd_buffers(m, T, dtype):
+    import torch
+    n = m * m
+    bufs = {"dx": _guarded((T, n), _tdtype(dtype))}
+    for k in MLP_GRADS:
+        bufs[k] = _guarded((n,) if k.startswith("db") else (m, m, m), torch.float32)
+    return bufs
+
+
+def _call_mlp_bwd(P, t, bufs, accumulate, T, n, m, ws):
+    P.monarch_mlp_bwd(t["x"], t["dy"], t["L"], t["R"], t["b1"], t["L2"], t["R2"], bufs["dx"][1],
+                      *(bufs[k][1] for k in MLP_GRADS), accumulate, T, n, m, ws)
+
+
+def _assert_mlp_grads(bufs, ref, dtype, what, factor=1.0):
+    for k in MLP_GRADS:
+        got, want = to_host64(bufs[k][1]), factor * ref[k]
+        if k.startswith("db"):                 # one problem instance: the whole bias vector
+            got, want = got[None, :], want[None, :]
+        assert_close(got, want, dtype, f"{what} {k}")
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("m,T", [(16, 5), (32, 129), (64, 64), (64, 257), (128, 66)])
+def test_mlp_bwd_small(P, impl, m, T, dtype):
+    import torch
+    code = _code(P, dtype)
+    _skip_if_same_family(P, impl, P.OP_MLP_BWD, m, code)
+    n = m * m
+    d = _small_inputs(m, T, dtype, seed=91 * m + T)
+    t = {k: to_device(d[k], dtype) for k in ("x", "dy", "L", "R", "b1", "L2", "R2")}
+    bufs = _mlp_bwd_buffers(m, T, dtype)
+    ws = P.Workspace(P.monarch_workspace_bytes(P.OP_MLP_BWD, T, n, m, code))
+    _call_mlp_bwd(P, t, bufs, 0, T, n, m, ws)
+    torch.cuda.synchronize()
+    assert P.monarch_last_device_status(ws) == 0
+    ref = O.mlp_bwd(d["x"], d["dy"], d["L"], d["R"], d["b1"], d["L2"], d["R2"])
+    assert_close(to_host64(bufs["dx"][1]), ref["dx"], dtype, "mlp dx")
+    _assert_mlp_grads(bufs, ref, dtype, "mlp")
+    for k, (flat, _) in bufs.items():
+        _check_guard(flat, f"mlp {k}")
+    # accumulate = 1 adds to the previous contents of the six parameter gradients
+    _call_mlp_bwd(P, t, bufs, 1, T, n, m, ws)
+    torch.cuda.synchronize()
+    assert P.monarch_last_device_status(ws) == 0
+    assert_close(to_host64(bufs["dx"][1]), ref["dx"], dtype, "mlp dx (second call)")
+    _assert_mlp_grads(bufs, ref, dtype, "mlp accumulate", factor=2.0)
+
+
+def test_mlp_bwd_zero_tokens(P, impl):
+    import torch
+    m, n = 64, 4096
+    t = {k: torch.zeros(s, dtype=torch.bfloat16, device="cuda")
+         for k, s in (("x", (1, n)), ("dy", (1, n)), ("L", (m, m, m)), ("R", (m, m, m)), ("b1", (n,)),
+                      ("L2", (m, m, m)), ("R2", (m, m, m)))}
+    bufs = _mlp_bwd_buffers(m, 1, "bf16")
+    for k in MLP_GRADS:
+        bufs[k][1].fill_(5.0)
+    ws = P.Workspace(P.monarch_workspace_bytes(P.OP_MLP_BWD, 0, n, m, P.BF16))
+    _call_mlp_bwd(P, t, bufs, 1, 0, n, m, ws)
+    torch.cuda.synchronize()
+    assert all(float(bufs[k][1].min()) == 5.0 for k in MLP_GRADS)
+    _call_mlp_bwd(P, t, bufs, 0, 0, n, m, ws)
+    torch.cuda.synchronize()
+    assert all(float(bufs[k][1].abs().max()) == 0.0 for k in MLP_GRADS)
+    assert P.monarch_last_device_status(ws) == 0
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_zero_tokens(P, impl, dtype):
     import torch
@@ -401,3 +472,52 @@ def test_workload_mlp(P, impl):
     yh = to_host64(y[torch.from_numpy(rows).cuda()])
     assert bool(torch.isfinite(y.float()).all())
     assert_close(yh, ref, c.dtype, "cfg5 mlp y")
+
+
+def test_workload_mlp_bwd(P, impl):
+    """Backward of the feed-forward block on workload 5's tensors: every gradient against the oracle on a
+    ragged slice of the tokens, then the full token count with dx on sampled rows, db2 against its
+    definition and the Euler identities of the two bilinear maps evaluated on the device results."""
+    import torch
+    c = CONFIGS[5]
+    code = _code(P, c.dtype)
+    _skip_if_same_family(P, impl, P.OP_MLP_BWD, c.m, code)
+    d = make_inputs(5, with_dy=True)
+    m, n, T = c.m, c.n, c.tokens
+    t = {k: to_device(d[k], c.dtype) for k in ("x", "dy", "L", "R", "b1", "L2", "R2", "b2")}
+    ws = P.Workspace(P.monarch_workspace_bytes(P.OP_MLP_BWD, T, n, m, code))
+    # (1) a slice the oracle finishes in seconds: 17 tiles and a ragged tail
+    Ts = 1100
+    ts = {k: (v[:Ts].contiguous() if k in ("x", "dy") else v) for k, v in t.items()}
+    bufs = _mlp_bwd_buffers(m, Ts, c.dtype)
+    _call_mlp_bwd(P, ts, bufs, 0, Ts, n, m, ws)
+    torch.cuda.synchronize()
+    assert P.monarch_last_device_status(ws) == 0
+    ref = O.mlp_bwd(d["x"][:Ts], d["dy"][:Ts], d["L"], d["R"], d["b1"], d["L2"], d["R2"])
+    assert_close(to_host64(bufs["dx"][1]), ref["dx"], c.dtype, "cfg5 slice dx")
+    _assert_mlp_grads(bufs, ref, c.dtype, "cfg5 slice")
+    # (2) all tokens
+    bufs = _mlp_bwd_buffers(m, T, c.dtype)
+    _call_mlp_bwd(P, t, bufs, 0, T, n, m, ws)
+    torch.cuda.synchronize()
+    assert P.monarch_last_device_status(ws) == 0
+    rows = _sample_tokens(T, 256, 55)
+    ref = O.mlp_bwd(d["x"][rows], d["dy"][rows], d["L"], d["R"], d["b1"], d["L2"], d["R2"])
+    dxh = to_host64(bufs["dx"][1])
+    assert np.isfinite(dxh).all()
+    assert_close(dxh[rows], ref["dx"], c.dtype, "cfg5 dx")
+    g = {k: to_host64(bufs[k][1]) for k in MLP_GRADS}
+    assert_close(g["db2"][None, :], d["dy"].astype(np.float64).sum(0)[None, :], c.dtype, "cfg5 db2")
+    # y - b2 is bilinear in (L2, R2) and a - b1 in (L1, R1):
+    #   <dL2, L2> = <dR2, R2> = <dy, y - b2>,   <dL1, L1> = <dR1, R1> = <dx, x>
+    y = torch.empty_like(t["x"])
+    ws_f = P.Workspace(P.monarch_workspace_bytes(P.OP_MLP_FWD, T, n, m, code))
+    P.monarch_mlp_fwd(t["x"], t["L"], t["R"], t["b1"], t["L2"], t["R2"], t["b2"], y, T, n, m, ws_f)
+    torch.cuda.synchronize()
+    s2 = float(np.sum(d["dy"].astype(np.float64) * (to_host64(y) - d["b2"].astype(np.float64))))
+    tol = 2e-2 * float(np.sqrt(T * n))
+    assert abs(float(np.sum(g["dL2"] * d["L2"])) - s2) <= tol
+    assert abs(float(np.sum(g["dR2"] * d["R2"])) - s2) <= tol
+    s1 = float(np.sum(dxh * d["x"]))
+    assert abs(float(np.sum(g["dL1"] * d["L"])) - s1) <= tol
+    assert abs(float(np.sum(g["dR1"] * d["R"])) - s1) <= tol
