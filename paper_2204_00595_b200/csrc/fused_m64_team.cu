@@ -82,20 +82,6 @@ __device__ __forceinline__ bool wait_fast(uint32_t bar, uint32_t parity, unsigne
     return mbar_wait(bar, parity, status, dead, code);
 }
 
-// GELU(a) = a/2 (1 + erf(a / sqrt 2)) evaluated as a * sigmoid(2 a (c0 + c1 a^2 + c2 a^4)): the logistic form
-// of the usual tanh approximation with one more polynomial term, coefficients fitted (minimax over [-8, 8]) to
-// the erf definition: |error| <= 2.6e-5 everywhere (a^2 is clamped at 64, beyond which the sigmoid has
-// saturated) - well below one bf16 ulp of the result.  Nine instructions, two of them MUFU; the libm-grade erf
-// costs twice that, and the stage-2 epilogue is on the critical path of the pipeline.
-__device__ __forceinline__ float gelu_fast(float a)
-{
-    const float a2 = fminf(a * a, 64.0f);
-    float t = fmaf(a2, 0.0010142630198970437f, -0.10677572339773178f);     // -2 log2(e) * (c2 a^2 + c1)
-    t = fmaf(a2, t, -2.301121234893799f);
-    const float e = exp2f(a * t);                                          // exp(-2 a poly(a^2))
-    return __fdividef(a, 1.0f + e);
-}
-
 __global__ void __launch_bounds__(kThreads, 1)
 fused_fwd_m64_team_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_R,
                           const __grid_constant__ CUtensorMap tm_L, const __grid_constant__ CUtensorMap tm_u,

@@ -55,24 +55,44 @@ __device__ __forceinline__ float gelu_erf_grad(float a)
     return cdf + a * 0.39894228040143267794f * expf(-0.5f * a * a);
 }
 
+// fp32 tensors get the libm-grade forms; bf16 results are rounded to 8 bits of mantissa, so the cheaper forms
+// (error <= 5.1e-5) change nothing there and keep both kernels bound by memory rather than by erff / expf
+template <typename T> struct act_math;
+template <> struct act_math<float> {
+    static __device__ __forceinline__ float gelu(float a) { return gelu_erf(a); }
+    static __device__ __forceinline__ float grad(float a) { return gelu_erf_grad(a); }
+};
+template <> struct act_math<__nv_bfloat16> {
+    static __device__ __forceinline__ float gelu(float a) { return gelu_fast(a); }
+    static __device__ __forceinline__ float grad(float a) { return gelu_fast_grad(a); }
+};
+
 // h[t][q] = GELU(a[t][q] (+ b1[q])); n is a multiple of the vector width
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
 mlp_act_kernel(const T *__restrict__ a, const T *__restrict__ b1, T *__restrict__ h, long long vecs, int n)
 {
-    constexpr int V = vec16<T>::kElems;
-    for (long long i = (long long)blockIdx.x * kThreads + threadIdx.x; i < vecs; i += (long long)gridDim.x * kThreads) {
-        float v[V];
-        vec16<T>::load(a + i * V, v);
-        if (b1 != nullptr) {
-            float b[V];
-            vec16<T>::load(b1 + (int)((i * V) % n), b);
+    constexpr int V = vec16<T>::kElems, U = 4;          // U independent 16-byte loads in flight per thread
+    const long long stride = (long long)gridDim.x * kThreads;
+    for (long long i0 = (long long)blockIdx.x * kThreads + threadIdx.x; i0 < vecs; i0 += U * stride) {
+        float v[U][V];
 #pragma unroll
-            for (int e = 0; e < V; ++e) v[e] += b[e];
+        for (int u = 0; u < U; ++u)
+            if (i0 + u * stride < vecs) vec16<T>::load(a + (i0 + u * stride) * V, v[u]);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long long i = i0 + u * stride;
+            if (i >= vecs) break;
+            if (b1 != nullptr) {
+                float b[V];
+                vec16<T>::load(b1 + (int)((i * V) % n), b);
+#pragma unroll
+                for (int e = 0; e < V; ++e) v[u][e] += b[e];
+            }
+#pragma unroll
+            for (int e = 0; e < V; ++e) v[u][e] = act_math<T>::gelu(v[u][e]);
+            vec16<T>::store(h + i * V, v[u]);
         }
-#pragma unroll
-        for (int e = 0; e < V; ++e) v[e] = gelu_erf(v[e]);
-        vec16<T>::store(h + i * V, v);
     }
 }
 
@@ -101,7 +121,7 @@ mlp_dact_kernel(T *__restrict__ dh, const T *__restrict__ a, const T *__restrict
         vec16<T>::load(dy + off, yv);
 #pragma unroll
         for (int e = 0; e < V; ++e) {
-            g[e] *= gelu_erf_grad(av[e] + bias[e]);
+            g[e] *= act_math<T>::grad(av[e] + bias[e]);
             s1[e] += g[e];
             s2[e] += yv[e];
         }
