@@ -276,3 +276,54 @@ int oracle_mlp_bwd(const double *x, const double *dy, const double *L1, const do
     free(dh);
     return fail;
 }
+
+/* General (rectangular) Monarch multiply, Appendix "General Monarch Matrix
+ * Parametrization": M = L R with
+ *   R = diag(R_0 .. R_{q-1}),  R_k of size b x b1      (n1 = q b1 inputs, n2 = q b)
+ *   L of size n3 x n2 (n3 = r b), a grid of r x q blocks S_{l,k}, each a
+ *   b x b diagonal matrix (the case b2 = b3 = b of the rectangular definition,
+ *   the one its block-diagonalisation theorem covers).
+ * With i = (i1, i0)_b the theorem's blocks are  R'_{i0}[i1][j1] = S_{i1,j1}[i0][i0];
+ * they are stored as  Lp[j][l][k] = S_{l,k}[j][j]  (b blocks of r x q).  Then
+ *   u[k*b + j] = sum_i R[k][j][i] x[k*b1 + i]         (block-diagonal product)
+ *   y[l*b + j] = sum_k Lp[j][l][k] u[k*b + j]         (row l*b+j of L has its
+ *                                                      nonzeros in columns k*b+j)
+ * q = b1 = b = r = m gives Definition 3.1's square case. */
+int oracle_rect_fwd(const double *x, const double *Lp, const double *R, double *y,
+                    long T, int q, int b1, int b, int r)
+{
+    const size_t n1 = (size_t)q * b1, n2 = (size_t)q * b, n3 = (size_t)r * b;
+    int fail = 0;
+#pragma omp parallel
+    {
+        double *u = (double *)malloc((n2 ? n2 : 1) * sizeof(double));
+        if (!u) {
+#pragma omp atomic write
+            fail = 1;
+        }
+#pragma omp barrier
+        if (!fail) {
+#pragma omp for schedule(static)
+            for (long t = 0; t < T; ++t) {
+                const double *xt = x + (size_t)t * n1;
+                double *yt = y + (size_t)t * n3;
+                for (int k = 0; k < q; ++k)
+                    for (int j = 0; j < b; ++j) {
+                        double acc = 0.0;
+                        for (int i = 0; i < b1; ++i)
+                            acc += R[((size_t)k * b + j) * b1 + i] * xt[(size_t)k * b1 + i];
+                        u[(size_t)k * b + j] = acc;
+                    }
+                for (int l = 0; l < r; ++l)
+                    for (int j = 0; j < b; ++j) {
+                        double acc = 0.0;
+                        for (int k = 0; k < q; ++k)
+                            acc += Lp[((size_t)j * r + l) * q + k] * u[(size_t)k * b + j];
+                        yt[(size_t)l * b + j] = acc;
+                    }
+            }
+        }
+        free(u);
+    }
+    return fail;
+}

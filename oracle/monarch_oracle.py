@@ -60,6 +60,8 @@ def _load():
         lib.oracle_bwd.argtypes = [dp] * 7 + [ctypes.c_long, ctypes.c_int]
         lib.oracle_mlp_fwd.restype = ctypes.c_int
         lib.oracle_mlp_fwd.argtypes = [dp] * 8 + [ctypes.c_long, ctypes.c_int]
+        lib.oracle_rect_fwd.restype = ctypes.c_int
+        lib.oracle_rect_fwd.argtypes = [dp] * 4 + [ctypes.c_long] + [ctypes.c_int] * 4
         lib.oracle_mlp_bwd.restype = ctypes.c_int
         lib.oracle_mlp_bwd.argtypes = [dp] * 14 + [ctypes.c_long, ctypes.c_int]
         _lib = lib
@@ -169,6 +171,26 @@ def mlp_bwd(x, dy, L1, R1, b1, L2, R2):
     return out
 
 
+def rect_fwd(x, Lp, R):
+    """y = L R x for the general (rectangular) Monarch class of the appendix.
+
+    R: [q, b, b1] (q blocks of b x b1), Lp: [b, r, q] with Lp[j, l, k] = S_{l,k}[j, j] (the diagonal
+    blocks of L gathered into the b blocks of its block-diagonal form), x: [T, q*b1] -> y: [T, r*b].
+    """
+    Lp = _f64(Lp); R = _f64(R)
+    q, b, b1 = R.shape
+    if Lp.ndim != 3 or Lp.shape[0] != b or Lp.shape[2] != q:
+        raise ValueError("Lp must be [b, r, q] for R of shape [q, b, b1]")
+    r = Lp.shape[1]
+    x = _f64(x); T = x.shape[0]
+    if x.shape != (T, q * b1):
+        raise ValueError("x must be [T, q*b1]")
+    y = np.empty((T, r * b), dtype=np.float64)
+    if _load().oracle_rect_fwd(_p(x), _p(Lp), _p(R), _p(y), T, q, b1, b, r):
+        raise MemoryError("oracle_rect_fwd")
+    return y
+
+
 # --------------------------------------------------------------------------
 # numpy restatements of the definitions (tiny n only)
 # --------------------------------------------------------------------------
@@ -204,6 +226,38 @@ def dense_from_definition(L, R) -> np.ndarray:
     m = np.asarray(L).shape[0]
     P = perm_matrix(m)
     return P @ blockdiag(L) @ P.T @ blockdiag(R)
+
+
+def sigma(b: int, n: int, i: int) -> int:
+    """The appendix's permutation sigma_(b,n): i = (i1, i0)_b  ->  (i0, i1)_{n/b} = i0 * (n/b) + i1."""
+    i1, i0 = divmod(i, b)
+    return i0 * (n // b) + i1
+
+
+def perm_matrix_general(b: int, n: int) -> np.ndarray:
+    """P_(b,n) as used in the appendix's block-diagonalisation proofs: R'[sigma(i), sigma(j)] = L[i, j]
+    for R' = P L P^T, i.e. P has its ones at (sigma(i), i).  (The prose "reshape b x n/b, transpose,
+    flatten" describes the transpose of this matrix; the two coincide when b = n/b.)"""
+    P = np.zeros((n, n), dtype=np.float64)
+    for i in range(n):
+        P[sigma(b, n, i), i] = 1.0
+    return P
+
+
+def rect_factors_from_definition(Lp, R):
+    """The two factors of the rectangular definition as dense matrices: R = diag(R_k) (n2 x n1) and L
+    (n3 x n2) whose (l, k) block is the diagonal matrix S_{l,k} with S_{l,k}[j, j] = Lp[j, l, k]."""
+    Lp = np.asarray(Lp, dtype=np.float64); R = np.asarray(R, dtype=np.float64)
+    q, b, b1 = R.shape
+    r = Lp.shape[1]
+    Rd = np.zeros((q * b, q * b1))
+    for k in range(q):
+        Rd[k * b:(k + 1) * b, k * b1:(k + 1) * b1] = R[k]
+    Ld = np.zeros((r * b, q * b))
+    for l in range(r):
+        for k in range(q):
+            Ld[l * b:(l + 1) * b, k * b:(k + 1) * b] = np.diag(Lp[:, l, k])
+    return Ld, Rd
 
 
 def project(A, m: int):

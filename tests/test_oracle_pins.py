@@ -411,3 +411,66 @@ def test_mlp_bwd_empty():
     g = O.mlp_bwd(x[:0], dy[:0], W[0], W[1], b1, W[2], W[3])
     assert g["dx"].shape == (0, m * m)
     assert not any(g[k].any() for k in ("dL1", "dR1", "db1", "dL2", "dR2", "db2"))
+
+
+# ------------------------------------------------------------------ general / rectangular class
+
+RECT = [(2, 3, 4, 5), (4, 2, 3, 2), (3, 3, 3, 3), (1, 4, 2, 3), (5, 1, 2, 4), (2, 6, 1, 3)]   # (q, b1, b, r)
+
+
+@pytest.mark.parametrize("q,b1,b,r", RECT)
+def test_rect_matches_definition(q, b1, b, r):
+    # y = L R x with both factors materialised from the appendix's definitions
+    rng = np.random.default_rng(31)
+    R, Lp = _rand(rng, q, b, b1), _rand(rng, b, r, q)
+    x = _rand(rng, 4, q * b1)
+    Ld, Rd = O.rect_factors_from_definition(Lp, R)
+    assert np.allclose(O.rect_fwd(x, Lp, R), x @ (Ld @ Rd).T, atol=1e-12)
+    # parameter counts stated with the definitions: n1*b2 for R, n2*n3/b for L (b2 = b3 = b)
+    assert np.count_nonzero(Rd) == q * b1 * b and np.count_nonzero(Ld) == (q * b) * (r * b) // b
+
+
+@pytest.mark.parametrize("q,b1,b,r", RECT)
+def test_rect_block_diagonalisation_theorem(q, b1, b, r):
+    # P_(b,n3) L P_(b,n2)^T is block diagonal with b blocks of size r x q, block j = Lp[j]
+    rng = np.random.default_rng(32)
+    R, Lp = _rand(rng, q, b, b1), _rand(rng, b, r, q)
+    Ld, _ = O.rect_factors_from_definition(Lp, R)
+    n2, n3 = q * b, r * b
+    Rp = O.perm_matrix_general(b, n3) @ Ld @ O.perm_matrix_general(b, n2).T
+    ref = np.zeros((n3, n2))
+    for j in range(b):
+        ref[j * r:(j + 1) * r, j * q:(j + 1) * q] = Lp[j]
+    assert np.array_equal(Rp, ref)
+
+
+@pytest.mark.parametrize("b,n", [(2, 6), (3, 12), (4, 16), (1, 5), (5, 5)])
+def test_general_permutation_inverse(b, n):
+    # sigma_(b,n)^-1 = sigma_(n/b,n), hence P_(b,n)^T = P_(n/b,n)
+    assert all(O.sigma(n // b, n, O.sigma(b, n, i)) == i for i in range(n))
+    assert np.array_equal(O.perm_matrix_general(b, n).T, O.perm_matrix_general(n // b, n))
+
+
+@pytest.mark.parametrize("m", [2, 3, 5])
+def test_rect_reduces_to_square(m):
+    rng = np.random.default_rng(33)
+    L, R = _rand(rng, m, m, m), _rand(rng, m, m, m)
+    x = _rand(rng, 3, m * m)
+    assert np.allclose(O.rect_fwd(x, L, R), O.fwd(x, L, R), atol=1e-13)
+    assert np.allclose(O.rect_fwd(x, L, R), x @ O.dense_from_definition(L, R).T, atol=1e-12)
+    assert np.array_equal(O.perm_matrix_general(m, m * m), O.perm_matrix(m))
+
+
+def test_rect_kronecker_closed_form():
+    # every R_k = B (b x b1) and every diagonal-block pattern equal (Lp[j] = A, r x q): M = A kron B
+    rng = np.random.default_rng(34)
+    q, b1, b, r = 3, 4, 2, 5
+    A, B = _rand(rng, r, q), _rand(rng, b, b1)
+    x = _rand(rng, 6, q * b1)
+    y = O.rect_fwd(x, np.stack([A] * b), np.stack([B] * q))
+    assert np.allclose(y, x @ np.kron(A, B).T, atol=1e-12)
+    # identity blocks on a square instance give the identity matrix (the class contains I)
+    n = 12
+    y = O.rect_fwd(x, np.stack([np.eye(3)] * 4), np.stack([np.eye(4)] * 3))
+    assert np.allclose(y, x)
+    assert y.shape == (6, n)
