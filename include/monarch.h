@@ -142,6 +142,27 @@ int monarch_mlp_bwd(const void *x, const void *dy, const void *L1, const void *R
                     int accumulate, int64_t tokens, int32_t n, int32_t m, int dtype,
                     void *workspace, size_t workspace_bytes, void *stream);
 
+/* General (rectangular) Monarch multiply of the appendix "General Monarch
+ * Matrix Parametrization":  y = L R x  with
+ *   R = diag(R_0 .. R_{q-1}), R_k of size b x b1   (n1 = q*b1 inputs, n2 = q*b),
+ *   L of size n3 x n2 (n3 = r*b): an r x q grid of b x b diagonal blocks S_{l,k}
+ * (the case b2 = b3 = b of the rectangular definition, the one its
+ * block-diagonalisation theorem covers; q = b1 = b = r = m is Definition 3.1).
+ * Steps:  u[t][k*b + j] = sum_i R[k][j][i] x[t][k*b1 + i]
+ *         y[t][l*b + j] = sum_k L[j][l][k] u[t][k*b + j].
+ * x: [tokens][q*b1], y: [tokens][r*b], row-major, storage dtype;
+ * R: [q][b][b1];  L: [b][r][q] with L[j][l][k] = S_{l,k}[j][j], i.e. the b
+ * blocks (r x q) of the block-diagonal form P L P^T of that theorem.
+ * u is rounded to the storage dtype once (fp32 accumulation throughout).
+ * All four sizes must be in [1, 16384] and every row (q*b1, q*b, r*b) at most
+ * 2^24 elements; MONARCH_ERR_UNSUPPORTED otherwise.  Workspace:
+ * monarch_rect_workspace_bytes (0 for invalid arguments). */
+int monarch_rect_fwd(const void *x, const void *L, const void *R, void *y, int64_t tokens,
+                     int32_t q, int32_t b1, int32_t b, int32_t r, int dtype,
+                     void *workspace, size_t workspace_bytes, void *stream);
+size_t monarch_rect_workspace_bytes(int64_t tokens, int32_t q, int32_t b1, int32_t b, int32_t r,
+                                    int dtype);
+
 /* Bytes of workspace `op` (a monarch_op_t) needs for these sizes under the
  * current implementation choice; always >= MONARCH_STATUS_BYTES.  Returns 0
  * for invalid or unsupported arguments. */

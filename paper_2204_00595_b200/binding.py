@@ -26,6 +26,8 @@ _SIGNATURES = {
     "monarch_mlp_fwd": (_int, [_vp] * 8 + [_i64, _i32, _i32, _int, _vp, _sz, _vp]),
     "monarch_bwd": (_int, [_vp] * 8 + [_int, _i64, _i32, _i32, _int, _vp, _sz, _vp]),
     "monarch_mlp_bwd": (_int, [_vp] * 14 + [_int, _i64, _i32, _i32, _int, _vp, _sz, _vp]),
+    "monarch_rect_fwd": (_int, [_vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32, _int, _vp, _sz, _vp]),
+    "monarch_rect_workspace_bytes": (_sz, [_i64, _i32, _i32, _i32, _i32, _int]),
     "monarch_workspace_bytes": (_sz, [_int, _i64, _i32, _i32, _int]),
     "monarch_workspace_init": (_int, [_vp, _sz, _vp]),
     "monarch_last_device_status": (_int, [_vp, _vp]),
@@ -220,6 +222,18 @@ def monarch_mlp_bwd(x, dy, L1, R1, b1, L2, R2, dx, dL1, dR1, db1, dL2, dR2, db2,
                                  _ptr(db1, "db1", f32), _ptr(dL2, "dL2", f32), _ptr(dR2, "dR2", f32),
                                  _ptr(db2, "db2", f32), int(accumulate), tokens, n, m, _dtype_code(x),
                                  p, b, _stream(stream)), "monarch_mlp_bwd")
+
+
+def monarch_rect_workspace_bytes(tokens: int, q: int, b1: int, b: int, r: int, dtype: int) -> int:
+    return int(lib().monarch_rect_workspace_bytes(tokens, q, b1, b, r, dtype))
+
+
+def monarch_rect_fwd(x, L, R, y, tokens, q, b1, b, r, workspace, stream=None) -> None:
+    """General (rectangular) Monarch multiply: x [tokens, q*b1], R [q, b, b1], L [b, r, q] -> y [tokens, r*b]."""
+    dt = x.dtype
+    p, nb = _ws(workspace)
+    _check(lib().monarch_rect_fwd(_ptr(x, "x"), _ptr(L, "L", dt), _ptr(R, "R", dt), _ptr(y, "y", dt), tokens,
+                                  q, b1, b, r, _dtype_code(x), p, nb, _stream(stream)), "monarch_rect_fwd")
 
 
 NOALLOC_SCRATCH_BYTES = 8 << 20

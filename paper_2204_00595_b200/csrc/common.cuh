@@ -143,6 +143,11 @@ int fused_bwd_m64(const void *x, const void *dy, const void *L, const void *R, c
 // where the fused forward keeps u inside its workspace
 const void *fused_fwd_m64_saved_u(const void *fwd_ws);
 
+// ---- general (rectangular) Monarch multiply on the CUDA cores (rect_simt.cu); workspace = [status][u] ----
+size_t rect_workspace_bytes(int64_t tokens, int q, int b, int dtype);
+int rect_fwd_simt(const void *x, const void *Lp, const void *R, void *y, int64_t tokens, int q, int b1, int b, int r,
+                  int dtype, void *ws, cudaStream_t s);
+
 // ---- elementwise steps of the feed-forward block's backward pass (mlp_bwd.cu) ----
 // h = GELU(a (+ b1)); b1 may be null when a already holds the bias
 int mlp_act(const void *a, const void *b1, void *h, int64_t tokens, int n, int dtype, cudaStream_t s);

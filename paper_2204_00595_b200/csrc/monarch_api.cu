@@ -39,6 +39,17 @@ int check_shape(int64_t tokens, int32_t n, int32_t m, int dtype)
     return MONARCH_OK;
 }
 
+// Sizes of the general (rectangular) multiply.
+int check_rect(int64_t tokens, int32_t q, int32_t b1, int32_t b, int32_t r, int dtype)
+{
+    if (tokens < 0 || q <= 0 || b1 <= 0 || b <= 0 || r <= 0) return MONARCH_ERR_INVALID_ARG;
+    if (dtype != MONARCH_F32 && dtype != MONARCH_BF16) return MONARCH_ERR_INVALID_ARG;
+    const int64_t lim = 16384, row = (int64_t)1 << 24;
+    if (q > lim || b1 > lim || b > lim || r > lim) return MONARCH_ERR_UNSUPPORTED;
+    if ((int64_t)q * b1 > row || (int64_t)q * b > row || (int64_t)r * b > row) return MONARCH_ERR_UNSUPPORTED;
+    return MONARCH_OK;
+}
+
 // Inputs and outputs: non-null, 16-byte aligned; no output overlaps an input, another
 // output or the workspace.
 int check_buffers(const Range *in, int n_in, const Range *out, int n_out, const void *ws,
@@ -305,6 +316,24 @@ int monarch_mlp_bwd(const void *x, const void *dy, const void *L1, const void *R
     MONARCH_TRY(monarch_bwd(x, dh, L1, R1, ws_f, dx, dL1, dR1, accumulate, tokens, n, m, dtype, ws_b, lay.ws_b,
                             stream));
     return merge_status((unsigned *)ws_b, (unsigned *)ws_f, s);
+}
+
+size_t monarch_rect_workspace_bytes(int64_t tokens, int32_t q, int32_t b1, int32_t b, int32_t r, int dtype)
+{
+    if (check_rect(tokens, q, b1, b, r, dtype) != MONARCH_OK) return 0;
+    return rect_workspace_bytes(tokens, q, b, dtype);
+}
+
+int monarch_rect_fwd(const void *x, const void *L, const void *R, void *y, int64_t tokens, int32_t q,
+                     int32_t b1, int32_t b, int32_t r, int dtype, void *workspace,
+                     size_t workspace_bytes, void *stream)
+{
+    MONARCH_TRY(check_rect(tokens, q, b1, b, r, dtype));
+    const size_t es = esize(dtype);
+    const Range in[] = {{x, (size_t)tokens * q * b1 * es}, {L, (size_t)b * r * q * es}, {R, (size_t)q * b * b1 * es}};
+    const Range out[] = {{y, (size_t)tokens * r * b * es}};
+    MONARCH_TRY(check_buffers(in, 3, out, 1, workspace, workspace_bytes, rect_workspace_bytes(tokens, q, b, dtype)));
+    return rect_fwd_simt(x, L, R, y, tokens, q, b1, b, r, dtype, workspace, (cudaStream_t)stream);
 }
 
 int monarch_workspace_init(void *workspace, size_t workspace_bytes, void *stream)

@@ -388,6 +388,73 @@ def test_workspace_too_small_is_reported(P):
     assert e.value.status == 3 or P.monarch_workspace_bytes(P.OP_FWD, T, n, m, P.F32) <= 256
 
 
+# ----------------------------------------------------------------- general (rectangular) class
+
+RECT_CASES = [
+    # (q, b1, b, r, T): odd sizes, one-element blocks, tall and wide, several tiles and ragged tails
+    (2, 3, 4, 5, 7), (5, 1, 2, 4, 65), (1, 4, 2, 3, 3), (3, 20, 17, 6, 130), (7, 5, 33, 9, 70),
+    (4, 64, 64, 4, 257), (4, 96, 32, 16, 129), (16, 16, 16, 16, 100), (32, 32, 32, 32, 65),
+    (4, 256, 256, 4, 200), (256, 4, 4, 256, 131), (8, 48, 80, 24, 90),
+]
+
+
+def _rect_inputs(q, b1, b, r, T, dtype, seed):
+    rng = np.random.default_rng(seed)
+
+    def draw(shape, std):
+        return round_to_storage(rng.standard_normal(shape, dtype=np.float32) * np.float32(std), dtype)
+
+    return {"x": draw((T, q * b1), 1.0), "R": draw((q, b, b1), 1.0 / np.sqrt(b1)),
+            "L": draw((b, r, q), 1.0 / np.sqrt(q))}
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("q,b1,b,r,T", RECT_CASES)
+def test_rect_fwd(P, q, b1, b, r, T, dtype):
+    import torch
+    code = _code(P, dtype)
+    d = _rect_inputs(q, b1, b, r, T, dtype, seed=q * 1000003 + b1 * 1009 + b * 31 + r)
+    x, L, R = (to_device(d[k], dtype) for k in ("x", "L", "R"))
+    yf, y = _guarded((T, r * b), _tdtype(dtype))
+    ws = P.Workspace(P.monarch_rect_workspace_bytes(T, q, b1, b, r, code))
+    P.monarch_rect_fwd(x, L, R, y, T, q, b1, b, r, ws)
+    torch.cuda.synchronize()
+    assert P.monarch_last_device_status(ws) == 0
+    assert_close(to_host64(y), O.rect_fwd(d["x"], d["L"], d["R"]), dtype, "rect y")
+    _check_guard(yf, "rect y")
+
+
+def test_rect_square_case_equals_monarch_fwd(P):
+    """q = b1 = b = r = m is Definition 3.1: both entry points see the same tensors."""
+    import torch
+    m, T = 32, 130
+    n = m * m
+    d = _small_inputs(m, T, "f32", seed=5)
+    x, L, R = (to_device(d[k], "f32") for k in ("x", "L", "R"))
+    y1, y2 = torch.empty_like(x), torch.empty_like(x)
+    ws = P.Workspace(max(P.monarch_workspace_bytes(P.OP_FWD, T, n, m, P.F32),
+                         P.monarch_rect_workspace_bytes(T, m, m, m, m, P.F32)))
+    P.monarch_fwd(x, L, R, y1, T, n, m, ws)
+    P.monarch_rect_fwd(x, L, R, y2, T, m, m, m, m, ws)
+    torch.cuda.synchronize()
+    assert_close(to_host64(y2), to_host64(y1), "f32", "rect vs square")
+    assert_close(to_host64(y2), O.fwd(d["x"], d["L"], d["R"]), "f32", "rect vs oracle")
+
+
+def test_rect_arguments(P):
+    import torch
+    x = torch.zeros(4, 64, device="cuda")
+    ws = P.Workspace(1 << 16)
+    assert P.monarch_rect_workspace_bytes(4, 0, 8, 8, 8, P.F32) == 0
+    assert P.monarch_rect_workspace_bytes(4, 8, 8, 8, 1 << 20, P.F32) == 0
+    with pytest.raises(P.MonarchError):
+        P.monarch_rect_fwd(x, x, x, x.clone(), 4, 8, 8, 8, -1, ws)
+    y = torch.full((1, 8), 3.0, device="cuda")
+    P.monarch_rect_fwd(x, x, x, y, 0, 2, 4, 4, 2, ws)            # zero tokens: nothing written
+    torch.cuda.synchronize()
+    assert float(y.min()) == 3.0
+
+
 # ----------------------------------------------------------------- the five workloads
 
 def _sample_tokens(T, count, seed):
