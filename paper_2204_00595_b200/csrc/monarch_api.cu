@@ -333,7 +333,14 @@ int monarch_rect_fwd(const void *x, const void *L, const void *R, void *y, int64
     const Range in[] = {{x, (size_t)tokens * q * b1 * es}, {L, (size_t)b * r * q * es}, {R, (size_t)q * b * b1 * es}};
     const Range out[] = {{y, (size_t)tokens * r * b * es}};
     MONARCH_TRY(check_buffers(in, 3, out, 1, workspace, workspace_bytes, rect_workspace_bytes(tokens, q, b, dtype)));
-    return rect_fwd_simt(x, L, R, y, tokens, q, b1, b, r, dtype, workspace, (cudaStream_t)stream);
+    cudaStream_t s = (cudaStream_t)stream;
+    // large bf16 blocks: stage 1 (nearly all the FLOPs when q is small) on the tensor cores
+    const bool tc1 = g_impl.load(std::memory_order_relaxed) != MONARCH_IMPL_STAGED &&
+                     rect_stage1_tc_available(q, b1, b, dtype);
+    if (tc1)
+        MONARCH_TRY(rect_stage1_tc(x, R, (char *)workspace + MONARCH_STATUS_BYTES, tokens, q, b1, b,
+                                   (unsigned *)workspace, s));
+    return rect_fwd_simt(x, L, R, y, tokens, q, b1, b, r, dtype, workspace, tc1, s);
 }
 
 int monarch_workspace_init(void *workspace, size_t workspace_bytes, void *stream)

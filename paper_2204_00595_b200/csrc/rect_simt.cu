@@ -133,16 +133,16 @@ size_t rect_workspace_bytes(int64_t tokens, int q, int b, int dtype)
 }
 
 int rect_fwd_simt(const void *x, const void *Lp, const void *R, void *y, int64_t tokens, int q, int b1, int b, int r,
-                  int dtype, void *ws, cudaStream_t s)
+                  int dtype, void *ws, int stage1_done, cudaStream_t s)
 {
     void *u = (char *)ws + MONARCH_STATUS_BYTES;
     const BlockProduct s1 = {tokens, q, b, b1, q * b1, q * b, b1, 1, b, 1};
     const BlockProduct s2 = {tokens, b, r, q, q * b, r * b, 1, b, 1, b};
     if (dtype == MONARCH_F32) {
-        MONARCH_TRY(block_product<float>(x, R, u, s1, s));
+        if (!stage1_done) MONARCH_TRY(block_product<float>(x, R, u, s1, s));
         return block_product<float>(u, Lp, y, s2, s);
     }
-    MONARCH_TRY(block_product<__nv_bfloat16>(x, R, u, s1, s));
+    if (!stage1_done) MONARCH_TRY(block_product<__nv_bfloat16>(x, R, u, s1, s));
     return block_product<__nv_bfloat16>(u, Lp, y, s2, s);
 }
 

@@ -1,0 +1,231 @@
+// Stage 1 of the general (rectangular) Monarch multiply on the tensor cores, bf16:
+//   u[t][k*b + j] = sum_i R[k][j][i] x[t][k*b1 + i]      (appendix: R = diag(R_0 .. R_{q-1}), R_k of size b x b1)
+// i.e. q independent GEMMs  U_k [T x b] = X_k [T x b1] R_k^T  whose operands are both K-major as stored.  With few,
+// large blocks (q = 4 blocks of 1024 x 1024 for n = 4096) this stage holds nearly all the FLOPs of the multiply
+// and is bound by the tensor pipe, not by HBM.
+//
+// Persistent kernel, one CTA per SM, 128-token x NT-column output tiles (NT = 128 or 64):
+//   warp 4 lane 0   TMA loads of the x tile (128 x 64) and the R_k tile (NT x 64), 128-byte swizzle, ring of kStages
+//   warp 5 lane 0   tcgen05.mma M = 128, N = NT, K = 16, four per 64-wide K chunk, accumulators in TMEM,
+//                   two accumulator buffers so that the epilogue of one tile overlaps the MMAs of the next
+//   warps 0-3       epilogue: TMEM -> registers -> bf16 -> swizzled staging tile -> one TMA store per 64 columns
+// Rows past the last token are zero-filled on load and clipped on store by the tensor maps.
+#include "tc_common.cuh"
+
+namespace monarch {
+namespace tc {
+namespace {
+
+constexpr int kTokTile = 128, kKChunk = 64;
+constexpr int kStages = 5;
+constexpr int kThreads = 6 * 32;
+
+struct RectParams {
+    unsigned *status;
+    int q, b1, b;
+    int mtiles, ntiles_per_block;     // output tiles: mtiles x (q * ntiles_per_block)
+};
+
+template <int NT> struct RectSmem {
+    static constexpr int kABytes = kTokTile * kKChunk * 2, kBBytes = NT * kKChunk * 2;
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kStagingBytes = kTokTile * 128;                       // 64 columns of bf16
+    static constexpr int kBytes = kStages * kStageBytes + (NT / 64) * kStagingBytes + 1024;
+};
+
+struct RectBars {
+    uint64_t full[kStages], empty[kStages];
+    uint64_t acc_full[2], acc_empty[2];
+};
+
+template <int NT>
+__global__ void __launch_bounds__(kThreads, 1)
+rect_stage1_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_R,
+                   const __grid_constant__ CUtensorMap tm_u, const RectParams p)
+{
+    using S = RectSmem<NT>;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) RectBars bars;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int dead_s;
+
+    const uint32_t ring0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t staging0 = ring0 + kStages * S::kStageBytes;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    volatile int *dead = &dead_s;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(smem_u32(&bars.full[s]), 1);
+            mbar_init(smem_u32(&bars.empty[s]), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(smem_u32(&bars.acc_full[a]), 1);
+            mbar_init(smem_u32(&bars.acc_empty[a]), 4);
+        }
+        fence_mbar_init();
+        dead_s = 0;
+        tma_prefetch_desc(&tm_x); tma_prefetch_desc(&tm_R); tma_prefetch_desc(&tm_u);
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&tmem_base_s), 2 * NT);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+
+    const int ntiles = p.q * p.ntiles_per_block;
+    const long long total = (long long)p.mtiles * ntiles;
+    const int kchunks = p.b1 / kKChunk;
+    const uint32_t full0 = smem_u32(bars.full), empty0 = smem_u32(bars.empty);
+    const uint32_t accf0 = smem_u32(bars.acc_full), acce0 = smem_u32(bars.acc_empty);
+
+    if (warp == 4) {
+        // ------------------------------------------------------------ loader
+        if (lane == 0) {
+            uint32_t n = 0;                                   // chunks loaded so far
+            bool ok = true;
+            for (long long tile = blockIdx.x; ok && tile < total; tile += gridDim.x) {
+                const int mt = (int)(tile / ntiles), nt = (int)(tile % ntiles);
+                const int k = nt / p.ntiles_per_block, n0 = (nt % p.ntiles_per_block) * NT;
+                for (int c = 0; c < kchunks; ++c, ++n) {
+                    const uint32_t s = n % kStages;
+                    if (!mbar_wait(empty0 + s * 8, ((n / kStages) & 1) ^ 1, p.status, dead, kErrSlotWait)) { ok = false; break; }
+                    mbar_expect_tx(full0 + s * 8, S::kStageBytes);
+                    tma_load_2d(ring0 + s * S::kStageBytes, &tm_x, k * p.b1 + c * kKChunk, mt * kTokTile, full0 + s * 8);
+                    tma_load_2d(ring0 + s * S::kStageBytes + S::kABytes, &tm_R, c * kKChunk, k * p.b + n0, full0 + s * 8);
+                }
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc_bf16(kTokTile, NT, 0, 0);
+            uint32_t n = 0, it = 0;
+            bool ok = true;
+            for (long long tile = blockIdx.x; ok && tile < total; tile += gridDim.x, ++it) {
+                const uint32_t buf = it & 1;
+                if (!mbar_wait(acce0 + buf * 8, ((it >> 1) & 1) ^ 1, p.status, dead, kErrTmemWait)) break;
+                tc_fence_after();
+                const uint32_t d = tmem_base + buf * NT;
+                for (int c = 0; c < kchunks; ++c, ++n) {
+                    const uint32_t s = n % kStages;
+                    if (!mbar_wait(full0 + s * 8, (n / kStages) & 1, p.status, dead, kErrTmaWait)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = ring0 + s * S::kStageBytes;
+                    const uint64_t ad = make_smem_desc(a_addr, 16, 1024, kSwizzle128);
+                    const uint64_t bd = make_smem_desc(a_addr + S::kABytes, 16, 1024, kSwizzle128);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        mma_f16_ss(d, ad + 2 * kk, bd + 2 * kk, idesc, (c | kk) != 0);
+                    mma_commit(empty0 + s * 8);
+                }
+                if (!ok) break;
+                mma_commit(accf0 + buf * 8);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 0-3 = TMEM lanes 32w..32w+31)
+        const int row = warp * 32 + lane;
+        uint32_t it = 0;
+        for (long long tile = blockIdx.x; tile < total; tile += gridDim.x, ++it) {
+            const int mt = (int)(tile / ntiles), nt = (int)(tile % ntiles);
+            const int k = nt / p.ntiles_per_block, n0 = (nt % p.ntiles_per_block) * NT;
+            const uint32_t buf = it & 1;
+            if (!mbar_wait(accf0 + buf * 8, (it >> 1) & 1, p.status, dead, kErrMmaWait)) break;
+            tc_fence_after();
+            // the staging tiles are free once the previous tile's stores have read them
+            if (threadIdx.x == 0) tma_store_wait_read<0>();
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+#pragma unroll
+            for (int h = 0; h < NT / 64; ++h) {
+                const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + buf * NT + h * 64;
+                uint32_t v[4][16];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) tmem_ld16(taddr + i * 16, v[i]);
+                tmem_ld_wait();
+                const uint32_t dst = staging0 + h * S::kStagingBytes + row * 128;
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const uint32_t *w = &v[c >> 1][(c & 1) * 8];
+                    const uint32_t o0 = pack_bf16(__uint_as_float(w[0]), __uint_as_float(w[1]));
+                    const uint32_t o1 = pack_bf16(__uint_as_float(w[2]), __uint_as_float(w[3]));
+                    const uint32_t o2 = pack_bf16(__uint_as_float(w[4]), __uint_as_float(w[5]));
+                    const uint32_t o3 = pack_bf16(__uint_as_float(w[6]), __uint_as_float(w[7]));
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((c ^ (row & 7)) << 4)),
+                                 "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
+                }
+            }
+            // accumulator buffer drained: hand it back to the MMA warp
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acce0 + buf * 8);
+            fence_proxy_async_smem();
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (threadIdx.x == 0) {
+#pragma unroll
+                for (int h = 0; h < NT / 64; ++h)
+                    tma_store_2d(&tm_u, staging0 + h * S::kStagingBytes, k * p.b + n0 + h * 64, mt * kTokTile);
+                tma_store_commit();
+            }
+        }
+        if (threadIdx.x == 0) tma_store_wait_all<0>();
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem_base, 2 * NT);
+}
+
+template <int NT>
+int launch(const void *x, const void *R, void *u, int64_t tokens, int q, int b1, int b, unsigned *status, cudaStream_t s)
+{
+    using S = RectSmem<NT>;
+    CUtensorMap tm_x, tm_R, tm_u;
+    MONARCH_TRY(encode_tmap_2d(&tm_x, x, (uint64_t)tokens, (uint64_t)q * b1, (uint64_t)q * b1 * 2, kTokTile, kKChunk, 128));
+    MONARCH_TRY(encode_tmap_2d(&tm_R, R, (uint64_t)q * b, (uint64_t)b1, (uint64_t)b1 * 2, NT, kKChunk, 128));
+    MONARCH_TRY(encode_tmap_2d(&tm_u, u, (uint64_t)tokens, (uint64_t)q * b, (uint64_t)q * b * 2, kTokTile, 64, 128));
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        MONARCH_CUDA_TRY(cudaGetDevice(&dev));
+        MONARCH_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    }
+    static bool attr = false;
+    if (!attr) {
+        MONARCH_CUDA_TRY(cudaFuncSetAttribute(rect_stage1_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kBytes));
+        attr = true;
+    }
+    RectParams p;
+    p.status = status;
+    p.q = q; p.b1 = b1; p.b = b;
+    p.mtiles = (int)((tokens + kTokTile - 1) / kTokTile);
+    p.ntiles_per_block = b / NT;
+    const long long total = (long long)p.mtiles * q * p.ntiles_per_block;
+    const int grid = (int)(total < sms ? total : sms);
+    rect_stage1_kernel<NT><<<grid, kThreads, S::kBytes, s>>>(tm_x, tm_R, tm_u, p);
+    note_launch();
+    MONARCH_CUDA_TRY(cudaGetLastError());
+    return MONARCH_OK;
+}
+
+}  // namespace
+}  // namespace tc
+
+bool rect_stage1_tc_available(int q, int b1, int b, int dtype)
+{
+    (void)q;
+    return dtype == MONARCH_BF16 && b1 % 64 == 0 && b % 64 == 0;
+}
+
+int rect_stage1_tc(const void *x, const void *R, void *u, int64_t tokens, int q, int b1, int b, unsigned *status,
+                   cudaStream_t s)
+{
+    if (tokens == 0) return MONARCH_OK;
+    return b % 128 == 0 ? tc::launch<128>(x, R, u, tokens, q, b1, b, status, s)
+                        : tc::launch<64>(x, R, u, tokens, q, b1, b, status, s);
+}
+
+}  // namespace monarch
