@@ -104,6 +104,187 @@ block_product_small_kernel(const T *__restrict__ in, const T *__restrict__ W, T 
     }
 }
 
+// Stage 2 when L's blocks are at most 4 x 4 (R has up to four large blocks): a pure streaming pass.  One thread
+// owns two neighbouring columns j, keeps their two r x q blocks in registers and walks a slab of tokens; a warp
+// reads and writes whole 128-byte lines (bf16) of every slice u[t][k*b + .] and y[t][l*b + .].
+template <typename T> struct pair_io;
+template <> struct pair_io<float> {
+    static __device__ __forceinline__ float2 load(const float *p) { return *reinterpret_cast<const float2 *>(p); }
+    static __device__ __forceinline__ void store(float *p, float2 v) { *reinterpret_cast<float2 *>(p) = v; }
+};
+template <> struct pair_io<__nv_bfloat16> {
+    static __device__ __forceinline__ float2 load(const __nv_bfloat16 *p)
+    {
+        const uint32_t w = *reinterpret_cast<const uint32_t *>(p);
+        return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u));
+    }
+    static __device__ __forceinline__ void store(__nv_bfloat16 *p, float2 v)
+    {
+        *reinterpret_cast<__nv_bfloat162 *>(p) = __floats2bfloat162_rn(v.x, v.y);
+    }
+};
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+stage2_small4_kernel(const T *__restrict__ u, const T *__restrict__ Lp, T *__restrict__ y, long long tokens, int q,
+                     int b, int r, int tokens_per_slab)
+{
+    const int j = (blockIdx.x * 256 + threadIdx.x) * 2;
+    if (j >= b) return;
+    float w[2][4][4];
+#pragma unroll
+    for (int jj = 0; jj < 2; ++jj)
+#pragma unroll
+        for (int l = 0; l < 4; ++l)
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                w[jj][l][k] = (l < r && k < q) ? elem<T>::load(Lp + ((size_t)(j + jj) * r + l) * q + k) : 0.0f;
+    const long long t0 = (long long)blockIdx.y * tokens_per_slab;
+    const long long t1 = t0 + tokens_per_slab < tokens ? t0 + tokens_per_slab : tokens;
+    constexpr int U = 2;                          // tokens per batch: all their loads are issued before any use
+    for (long long tb = t0; tb < t1; tb += U) {
+        float2 v[U][4];
+#pragma unroll
+        for (int tt = 0; tt < U; ++tt) {
+            const T *src = u + (size_t)(tb + tt) * q * b + j;
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                v[tt][k] = (k < q && tb + tt < t1) ? pair_io<T>::load(src + (size_t)k * b) : make_float2(0.0f, 0.0f);
+        }
+#pragma unroll
+        for (int tt = 0; tt < U; ++tt) {
+            if (tb + tt >= t1) break;
+            T *dst = y + (size_t)(tb + tt) * r * b + j;
+#pragma unroll
+            for (int l = 0; l < 4; ++l) {
+                if (l >= r) break;
+                float2 o = make_float2(0.0f, 0.0f);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    o.x = fmaf(w[0][l][k], v[tt][k].x, o.x);
+                    o.y = fmaf(w[1][l][k], v[tt][k].y, o.y);
+                }
+                pair_io<T>::store(dst + (size_t)l * b, o);
+            }
+        }
+    }
+}
+
+// The same for bf16 with 16-byte accesses: a CTA owns up to 256 columns j and keeps their blocks in shared memory
+// (fp32); a thread owns 8 neighbouring columns and two tokens per step, so a warp reads 512
+// contiguous bytes of every slice u[t][k*b + .] and eight 16-byte loads per thread are in flight - the pass is
+// bound by memory latency, not by arithmetic.
+constexpr int kS2Cols = 256;
+
+__device__ __forceinline__ float4 lds128(const float4 *p)
+{
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "r"((uint32_t)__cvta_generic_to_shared(p)));
+    return v;
+}
+__device__ __forceinline__ uint32_t pack2(float lo, float hi)
+{
+    const __nv_bfloat162 h2 = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&h2);
+}
+__device__ __forceinline__ float bf_at(const uint4 &v, int e)
+{
+    const uint32_t w = e < 2 ? v.x : e < 4 ? v.y : e < 6 ? v.z : v.w;
+    return (e & 1) ? __uint_as_float(w & 0xFFFF0000u) : __uint_as_float(w << 16);
+}
+
+__global__ void __launch_bounds__(256, 2)
+stage2_small4_bf16_kernel(const __nv_bfloat16 *__restrict__ u, const __nv_bfloat16 *__restrict__ Lp,
+                          __nv_bfloat16 *__restrict__ y, long long tokens, int q, int b, int r, int tokens_per_slab)
+{
+    __shared__ float4 ws[4][4][2][32];            // [l][k][half][lane]: columns 8 lane + 4 half + (0..3)
+    const int j0 = blockIdx.x * kS2Cols;
+    for (int i = threadIdx.x; i < 16 * kS2Cols; i += 256) {
+        const int jl = i >> 4, l = (i >> 2) & 3, k = i & 3;
+        float v = 0.0f;
+        if (j0 + jl < b && l < r && k < q) v = __bfloat162float(Lp[((size_t)(j0 + jl) * r + l) * q + k]);
+        reinterpret_cast<float *>(&ws[l][k][(jl >> 2) & 1][jl >> 3])[jl & 3] = v;
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31, jg = lane * 8, tr = threadIdx.x >> 5;   // 32 threads per token row, 8 rows
+    if (j0 + jg >= b) return;
+    const long long t0 = (long long)blockIdx.y * tokens_per_slab;
+    const long long t1 = t0 + tokens_per_slab < tokens ? t0 + tokens_per_slab : tokens;
+    for (long long tb = t0 + tr; tb < t1; tb += 16) {
+        const bool two = tb + 8 < t1;
+        uint4 v[2][4];
+#pragma unroll
+        for (int tt = 0; tt < 2; ++tt) {
+            const __nv_bfloat16 *src = u + (size_t)(tb + tt * 8) * q * b + j0 + jg;
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                v[tt][k] = (k < q && (tt == 0 || two)) ? *reinterpret_cast<const uint4 *>(src + (size_t)k * b)
+                                                       : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int l = 0; l < 4; ++l) {
+            if (l >= r) break;
+            float acc[2][8];
+#pragma unroll
+            for (int tt = 0; tt < 2; ++tt)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[tt][e] = 0.0f;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                // volatile: re-read per step instead of keeping all 128 weights live across the token loop
+                const float4 wa = lds128(&ws[l][k][0][lane]), wb = lds128(&ws[l][k][1][lane]);
+                const float wv[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+#pragma unroll
+                for (int tt = 0; tt < 2; ++tt)
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) acc[tt][e] = fmaf(wv[e], bf_at(v[tt][k], e), acc[tt][e]);
+            }
+#pragma unroll
+            for (int tt = 0; tt < 2; ++tt) {
+                if (tt == 1 && !two) break;
+                const uint4 o = make_uint4(pack2(acc[tt][0], acc[tt][1]), pack2(acc[tt][2], acc[tt][3]),
+                                           pack2(acc[tt][4], acc[tt][5]), pack2(acc[tt][6], acc[tt][7]));
+                *reinterpret_cast<uint4 *>(y + (size_t)(tb + tt * 8) * r * b + (size_t)l * b + j0 + jg) = o;
+            }
+        }
+    }
+}
+
+template <typename T>
+int stage2_small4(const void *u, const void *Lp, void *y, long long tokens, int q, int b, int r, cudaStream_t s)
+{
+    const int bx = (b / 2 + 255) / 256;
+    long long slabs = (148 * 8 + bx - 1) / bx;
+    if (slabs > (tokens + 3) / 4) slabs = (tokens + 3) / 4;
+    const int per = (int)((tokens + slabs - 1) / slabs);
+    slabs = (tokens + per - 1) / per;
+    if (slabs > 65535) return MONARCH_ERR_UNSUPPORTED;
+    if constexpr (sizeof(T) == 2) {
+        if (b % 8 == 0) {          // 16-byte accesses need rows and slices that start on 16-byte boundaries
+            const int cx = (b + kS2Cols - 1) / kS2Cols;
+            long long sl = (148 * 6 + cx - 1) / cx;
+            if (sl > (tokens + 15) / 16) sl = (tokens + 15) / 16;
+            const int pt = (int)((tokens + sl - 1) / sl);
+            sl = (tokens + pt - 1) / pt;
+            if (sl > 65535) return MONARCH_ERR_UNSUPPORTED;
+            stage2_small4_bf16_kernel<<<dim3((unsigned)cx, (unsigned)sl), 256, 0, s>>>(
+                (const __nv_bfloat16 *)u, (const __nv_bfloat16 *)Lp, (__nv_bfloat16 *)y, tokens, q, b, r, pt);
+            note_launch();
+            MONARCH_CUDA_TRY(cudaGetLastError());
+            return MONARCH_OK;
+        }
+    }
+    {
+        stage2_small4_kernel<T><<<dim3((unsigned)bx, (unsigned)slabs), 256, 0, s>>>((const T *)u, (const T *)Lp, (T *)y,
+                                                                                  tokens, q, b, r, per);
+    }
+    note_launch();
+    MONARCH_CUDA_TRY(cudaGetLastError());
+    return MONARCH_OK;
+}
+
 template <typename T>
 int block_product(const void *in, const void *W, void *out, const BlockProduct &p, cudaStream_t s)
 {
@@ -138,12 +319,14 @@ int rect_fwd_simt(const void *x, const void *Lp, const void *R, void *y, int64_t
     void *u = (char *)ws + MONARCH_STATUS_BYTES;
     const BlockProduct s1 = {tokens, q, b, b1, q * b1, q * b, b1, 1, b, 1};
     const BlockProduct s2 = {tokens, b, r, q, q * b, r * b, 1, b, 1, b};
+    const bool small4 = q <= 4 && r <= 4 && b % 2 == 0 && tokens > 0;
     if (dtype == MONARCH_F32) {
         if (!stage1_done) MONARCH_TRY(block_product<float>(x, R, u, s1, s));
-        return block_product<float>(u, Lp, y, s2, s);
+        return small4 ? stage2_small4<float>(u, Lp, y, tokens, q, b, r, s) : block_product<float>(u, Lp, y, s2, s);
     }
     if (!stage1_done) MONARCH_TRY(block_product<__nv_bfloat16>(x, R, u, s1, s));
-    return block_product<__nv_bfloat16>(u, Lp, y, s2, s);
+    return small4 ? stage2_small4<__nv_bfloat16>(u, Lp, y, tokens, q, b, r, s)
+                  : block_product<__nv_bfloat16>(u, Lp, y, s2, s);
 }
 
 }  // namespace monarch

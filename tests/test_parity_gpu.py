@@ -394,7 +394,7 @@ RECT_CASES = [
     # (q, b1, b, r, T): odd sizes, one-element blocks, tall and wide, several tiles and ragged tails
     (2, 3, 4, 5, 7), (5, 1, 2, 4, 65), (1, 4, 2, 3, 3), (3, 20, 17, 6, 130), (7, 5, 33, 9, 70),
     (4, 64, 64, 4, 257), (4, 96, 32, 16, 129), (16, 16, 16, 16, 100), (32, 32, 32, 32, 65),
-    (4, 256, 256, 4, 200), (256, 4, 4, 256, 131), (8, 48, 80, 24, 90),
+    (4, 256, 256, 4, 200), (256, 4, 4, 256, 131), (8, 48, 80, 24, 90), (3, 5, 7, 2, 33), (2, 8, 6, 4, 50),
     # bf16 with b1 and b multiples of 64: stage 1 on the tensor cores (128- and 64-wide output tiles, K = 64..1024)
     (2, 128, 192, 3, 300), (3, 64, 128, 5, 1), (4, 1024, 1024, 4, 140), (1, 320, 448, 2, 513), (6, 192, 64, 7, 128),
 ]
