@@ -35,7 +35,8 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=3, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--workload", type=int, default=3, choices=[1, 2, 3, 4, 5, 6],
+                    help="1-5: the square workloads; 6: the general (rectangular) class, forward only")
     ap.add_argument("--kernels", default="auto", choices=["auto", "staged", "fused"])
     ap.add_argument("--calls", default="", help="comma-separated subset of the workload's calls "
                     "(profiling aid; the default step runs them all)")
@@ -197,8 +198,132 @@ KERNELS_OF = {
 NCU_TRAFFIC_MB = {(3, "fwd"): 150.0, (3, "bwd"): 365.6}
 
 
+def main_rect(args):
+    """Workload 6: forward of the general Monarch class (appendix), q = 4 blocks of 1024 x 1024, one GPU or
+    token-sharded replicas; bound by the tensor pipe (stage 1 holds nearly all the FLOPs)."""
+    from paper_2204_00595_b200.inputs import RECT_WORKLOAD, make_rect_inputs
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    c = RECT_WORKLOAD
+    q, b1, b, r, T = c["q"], c["b1"], c["b"], c["r"], c["tokens"]
+    flops = 2 * T * (q * b * b1 + b * r * q)
+    nbytes = T * (q * b1 + r * b) * 2 + (q * b * b1 + b * r * q) * 2
+    workload = f"workload 6: rect_fwd bf16 q={q} b1={b1} b={b} r={r} tokens/GPU={T}"
+    metric, unit = "monarch_rect_fwd_tflops", "TFLOP/s"
+
+    def time_oracle_rect(d, target_s):
+        from oracle import monarch_oracle as O
+        Ts, dt = 8, 0.0
+        while True:
+            t0 = time.perf_counter()
+            O.rect_fwd(d["x"][:Ts], d["L"], d["R"])
+            dt = time.perf_counter() - t0
+            if dt >= target_s / 4 or Ts >= T:
+                break
+            Ts = min(T, Ts * 4)
+        return {"tflops": flops * Ts / T / dt / 1e12, "tokens": Ts, "seconds": dt, "cores": O.num_threads()}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        from oracle import monarch_oracle as O
+        O.build()
+        d = make_rect_inputs()
+        rs = [time_oracle_rect(d, 8.0) for _ in range(args.warmup + args.steps)][args.warmup:]
+        tfl = statistics.mean(x["tflops"] for x in rs)
+        print(json.dumps({
+            "impl": "reference", "metric": metric, "value": tfl, "unit": unit, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": statistics.mean(x["seconds"] for x in rs) * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": workload, "sample_tokens_per_step": rs[-1]["tokens"]},
+            "cpu_baseline": {"value": tfl, "unit": unit, "cores": rs[-1]["cores"], "kind": "oracle",
+                             "sample": f"{rs[-1]['tokens']} tokens of the workload per step"},
+            "e2e": {"value": tfl, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+        return 0
+
+    import torch
+    import __graft_entry__ as entry
+    entry.build()
+    import paper_2204_00595_b200 as P
+    from tests.helpers import to_device
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    P.monarch_set_impl({"auto": P.IMPL_AUTO, "staged": P.IMPL_STAGED, "fused": P.IMPL_AUTO}[args.kernels])
+    d = make_rect_inputs()
+    R, L = to_device(d["R"], "bf16"), to_device(d["L"], "bf16")
+    sets = []
+    for s in range(2):                          # two rotating sets, each larger than L2 with its output
+        x = torch.roll(to_device(d["x"], "bf16"), shifts=17 * s + 5 * rank, dims=0).contiguous()
+        sets.append((x, torch.empty(T, r * b, dtype=torch.bfloat16, device="cuda")))
+    ws = P.Workspace(P.monarch_rect_workspace_bytes(T, q, b1, b, r, P.BF16))
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        x, y = sets[i % 2]
+        P.monarch_rect_fwd(x, L, R, y, T, q, b1, b, r, ws)
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = P.monarch_launch_count()
+    t_start, t_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t_start.record(stream)
+    for i in range(args.steps):
+        step(args.warmup + i)
+    t_stop.record(stream)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    total_ms = t_start.elapsed_time(t_stop)
+    clocks = sampler.stop()
+    launches = P.monarch_launch_count() - launches0
+    status = P.monarch_last_device_status(ws)
+    if dist is not None:
+        tmax = torch.tensor([total_ms], device="cuda")
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        total_ms = float(tmax.item())
+    ms = total_ms / args.steps
+    peaks = load_peaks()
+    tfl = flops / (ms * 1e-3) / 1e12
+    line = {
+        "metric": metric, "value": tfl * world, "unit": unit, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "tokens_per_s": T * world / (ms * 1e-3),
+        "config": {"workload": workload, "l2": "inputs larger than L2; 2 rotating buffer sets",
+                   "kernels": args.kernels, "device_status": status},
+        "clocks": clocks, "gpu_launches": int(launches),
+        "roofline": {"bound": "tensor", "kernel": "rect_fwd: rect_stage1_kernel<128> (tcgen05) + "
+                                                  "stage2_small4_bf16_kernel (2 launches)",
+                     "achieved": tfl, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                     "frac": tfl / peaks["bf16_tflops"], "peak_source": peaks["source"], "traffic": None,
+                     "algorithmic_mb": nbytes / 1e6,
+                     "hbm_time_ms": nbytes / (peaks["hbm_gbs"] * 1e9) * 1e3},
+        "e2e": None,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        rr = time_oracle_rect(d, 12.0)
+        line["cpu_baseline"] = {"value": rr["tflops"], "unit": unit, "cores": rr["cores"], "kind": "oracle",
+                                "sample": f"first {rr['tokens']} tokens of the workload, {rr['seconds']:.1f} s"}
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
 def main():
     args = parse_args()
+    if args.workload == 6:
+        return main_rect(args)
     from paper_2204_00595_b200.inputs import CONFIGS, make_inputs
     cfg = CONFIGS[args.workload]
     rank = int(os.environ.get("RANK", "0"))

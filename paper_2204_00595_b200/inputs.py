@@ -105,3 +105,28 @@ def make_inputs(config: int, tokens: int | None = None, m: int | None = None,
     if with_dy and "dy" not in out:
         out["dy"] = draw((T, n), 1.0)      # drawn last: the tensors above do not depend on the flag
     return out
+
+
+# General (rectangular) Monarch class of the paper's appendix: R has q blocks of b x b1, L has b blocks of
+# r x q.  One measured case with the block count the paper's experiments use (four blocks).
+RECT_WORKLOAD = {"q": 4, "b1": 1024, "b": 1024, "r": 4, "tokens": 8192, "dtype": "bf16"}
+
+
+def make_rect_inputs(tokens: int | None = None, seed: int = 595006, **sizes) -> dict:
+    """Seeded tensors x [T, q*b1], R [q, b, b1], L [b, r, q] of the general class (unit-variance
+    activations, weights scaled so that u and y keep unit variance), rounded to the storage dtype."""
+    cfg = dict(RECT_WORKLOAD)
+    cfg.update(sizes)
+    if tokens is not None:
+        cfg["tokens"] = int(tokens)
+    q, b1, b, r, T, dt = cfg["q"], cfg["b1"], cfg["b"], cfg["r"], cfg["tokens"], cfg["dtype"]
+    rng = np.random.default_rng(seed)
+
+    def draw(shape, std):
+        return round_to_storage(rng.standard_normal(shape, dtype=np.float32) * np.float32(std), dt)
+
+    out = dict(cfg)
+    out["x"] = draw((T, q * b1), 1.0)
+    out["R"] = draw((q, b, b1), 1.0 / math.sqrt(b1))
+    out["L"] = draw((b, r, q), 1.0 / math.sqrt(q))
+    return out

@@ -445,6 +445,31 @@ def test_rect_square_case_equals_monarch_fwd(P):
     assert_close(to_host64(y2), O.fwd(d["x"], d["L"], d["R"]), "f32", "rect vs oracle")
 
 
+def test_workload_rect(P, impl):
+    """The measured case of the general class (four 1024 x 1024 blocks, 8192 tokens) at full size: sampled
+    token rows against the oracle, and the stage-2-is-identity special case on all rows."""
+    import torch
+    from paper_2204_00595_b200.inputs import make_rect_inputs
+    d = make_rect_inputs()
+    q, b1, b, r, T = d["q"], d["b1"], d["b"], d["r"], d["tokens"]
+    x, L, R = (to_device(d[k], "bf16") for k in ("x", "L", "R"))
+    y = torch.full((T, r * b), float("nan"), dtype=torch.bfloat16, device="cuda")
+    ws = P.Workspace(P.monarch_rect_workspace_bytes(T, q, b1, b, r, P.BF16))
+    P.monarch_rect_fwd(x, L, R, y, T, q, b1, b, r, ws)
+    torch.cuda.synchronize()
+    assert P.monarch_last_device_status(ws) == 0
+    assert bool(torch.isfinite(y.float()).all())
+    rows = _sample_tokens(T, 96, 6)
+    ref = O.rect_fwd(d["x"][rows], d["L"], d["R"])
+    assert_close(to_host64(y[torch.from_numpy(rows).cuda()]), ref, "bf16", "rect workload y")
+    # L's blocks = identity (r = q): y = u = blockdiag(R) x, one bf16 rounding more than a plain block product
+    Li = to_device(np.broadcast_to(np.eye(q, dtype=np.float32), (b, q, q)).copy(), "bf16")
+    P.monarch_rect_fwd(x, Li, R, y, T, q, b1, b, r, ws)
+    torch.cuda.synchronize()
+    ref = np.einsum("kji,tki->tkj", d["R"].astype(np.float64), d["x"][rows].astype(np.float64).reshape(-1, q, b1))
+    assert_close(to_host64(y[torch.from_numpy(rows).cuda()]), ref.reshape(len(rows), q * b), "bf16", "rect identity L")
+
+
 def test_rect_arguments(P):
     import torch
     x = torch.zeros(4, 64, device="cuda")
