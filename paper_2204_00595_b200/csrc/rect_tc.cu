@@ -4,11 +4,13 @@
 // large blocks (q = 4 blocks of 1024 x 1024 for n = 4096) this stage holds nearly all the FLOPs of the multiply
 // and is bound by the tensor pipe, not by HBM.
 //
-// Persistent kernel, one CTA per SM, 128-token x NT-column output tiles (NT = 128 or 64):
+// Persistent kernel, one CTA per SM, 128-token x NT-column output tiles (NT = 256, 128 or 64, the widest that
+// divides b: a 128 x 256 x 16 MMA keeps the tensor pipe busy for longer than it takes one thread to issue it):
 //   warp 4 lane 0   TMA loads of the x tile (128 x 64) and the R_k tile (NT x 64), 128-byte swizzle, ring of kStages
 //   warp 5 lane 0   tcgen05.mma M = 128, N = NT, K = 16, four per 64-wide K chunk, accumulators in TMEM,
 //                   two accumulator buffers so that the epilogue of one tile overlaps the MMAs of the next
-//   warps 0-3       epilogue: TMEM -> registers -> bf16 -> swizzled staging tile -> one TMA store per 64 columns
+//   warps 0-3       epilogue: TMEM -> registers -> bf16 -> swizzled staging tile (two, alternating) -> one TMA
+//                   store per 64 columns
 // Rows past the last token are zero-filled on load and clipped on store by the tensor maps.
 #include "tc_common.cuh"
 
@@ -17,7 +19,6 @@ namespace tc {
 namespace {
 
 constexpr int kTokTile = 128, kKChunk = 64;
-constexpr int kStages = 5;
 constexpr int kThreads = 6 * 32;
 
 struct RectParams {
@@ -26,15 +27,17 @@ struct RectParams {
     int mtiles, ntiles_per_block;     // output tiles: mtiles x (q * ntiles_per_block)
 };
 
+constexpr int kMaxStages = 5;
 template <int NT> struct RectSmem {
+    static constexpr int kStages = NT == 256 ? 4 : kMaxStages;
     static constexpr int kABytes = kTokTile * kKChunk * 2, kBBytes = NT * kKChunk * 2;
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kStagingBytes = kTokTile * 128;                       // 64 columns of bf16
-    static constexpr int kBytes = kStages * kStageBytes + (NT / 64) * kStagingBytes + 1024;
+    static constexpr int kBytes = kStages * kStageBytes + 2 * kStagingBytes + 1024;
 };
 
 struct RectBars {
-    uint64_t full[kStages], empty[kStages];
+    uint64_t full[kMaxStages], empty[kMaxStages];
     uint64_t acc_full[2], acc_empty[2];
 };
 
@@ -44,6 +47,7 @@ rect_stage1_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
                    const __grid_constant__ CUtensorMap tm_u, const RectParams p)
 {
     using S = RectSmem<NT>;
+    constexpr int kStages = S::kStages;
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) RectBars bars;
     __shared__ uint32_t tmem_base_s;
@@ -129,24 +133,31 @@ rect_stage1_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     } else {
         // ------------------------------------------------------------ epilogue (warps 0-3 = TMEM lanes 32w..32w+31)
         const int row = warp * 32 + lane;
-        uint32_t it = 0;
+        uint32_t it = 0, nchunk = 0;                                   // 64-column chunks stored so far
         for (long long tile = blockIdx.x; tile < total; tile += gridDim.x, ++it) {
             const int mt = (int)(tile / ntiles), nt = (int)(tile % ntiles);
             const int k = nt / p.ntiles_per_block, n0 = (nt % p.ntiles_per_block) * NT;
             const uint32_t buf = it & 1;
             if (!mbar_wait(accf0 + buf * 8, (it >> 1) & 1, p.status, dead, kErrMmaWait)) break;
             tc_fence_after();
-            // the staging tiles are free once the previous tile's stores have read them
-            if (threadIdx.x == 0) tma_store_wait_read<0>();
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-#pragma unroll
-            for (int h = 0; h < NT / 64; ++h) {
+#pragma unroll 1
+            for (int h = 0; h < NT / 64; ++h, ++nchunk) {
+                const uint32_t stg = staging0 + (nchunk & 1) * S::kStagingBytes;
+                // this staging tile is free once the store issued two chunks ago has read it
+                if (threadIdx.x == 0) tma_store_wait_read<1>();
+                asm volatile("bar.sync 1, 128;" ::: "memory");
                 const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + buf * NT + h * 64;
                 uint32_t v[4][16];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) tmem_ld16(taddr + i * 16, v[i]);
                 tmem_ld_wait();
-                const uint32_t dst = staging0 + h * S::kStagingBytes + row * 128;
+                if (h == NT / 64 - 1) {
+                    // accumulator buffer drained: hand it back to the MMA warp
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(acce0 + buf * 8);
+                }
+                const uint32_t dst = stg + row * 128;
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
                     const uint32_t *w = &v[c >> 1][(c & 1) * 8];
@@ -157,18 +168,12 @@ rect_stage1_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
                     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((c ^ (row & 7)) << 4)),
                                  "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
                 }
-            }
-            // accumulator buffer drained: hand it back to the MMA warp
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(acce0 + buf * 8);
-            fence_proxy_async_smem();
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (threadIdx.x == 0) {
-#pragma unroll
-                for (int h = 0; h < NT / 64; ++h)
-                    tma_store_2d(&tm_u, staging0 + h * S::kStagingBytes, k * p.b + n0 + h * 64, mt * kTokTile);
-                tma_store_commit();
+                fence_proxy_async_smem();
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (threadIdx.x == 0) {
+                    tma_store_2d(&tm_u, stg, k * p.b + n0 + h * 64, mt * kTokTile);
+                    tma_store_commit();
+                }
             }
         }
         if (threadIdx.x == 0) tma_store_wait_all<0>();
@@ -224,6 +229,7 @@ int rect_stage1_tc(const void *x, const void *R, void *u, int64_t tokens, int q,
                    cudaStream_t s)
 {
     if (tokens == 0) return MONARCH_OK;
+    if (b % 256 == 0) return tc::launch<256>(x, R, u, tokens, q, b1, b, status, s);
     return b % 128 == 0 ? tc::launch<128>(x, R, u, tokens, q, b1, b, status, s)
                         : tc::launch<64>(x, R, u, tokens, q, b1, b, status, s);
 }
