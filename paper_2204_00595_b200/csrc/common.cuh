@@ -145,13 +145,18 @@ const void *fused_fwd_m64_saved_u(const void *fwd_ws);
 
 // ---- general (rectangular) Monarch multiply on the CUDA cores (rect_simt.cu); workspace = [status][u] ----
 size_t rect_workspace_bytes(int64_t tokens, int q, int b, int dtype);
-// stage1_done != 0: u is already in the workspace, run stage 2 only
-int rect_fwd_simt(const void *x, const void *Lp, const void *R, void *y, int64_t tokens, int q, int b1, int b, int r,
-                  int dtype, void *ws, int stage1_done, cudaStream_t s);
+int rect_stage1_simt(const void *x, const void *R, void *u, int64_t tokens, int q, int b1, int b, int dtype,
+                     cudaStream_t s);
+int rect_stage2_simt(const void *u, const void *Lp, void *y, int64_t tokens, int q, int b, int r, int dtype,
+                     cudaStream_t s);
 // stage 1 on the tensor cores (rect_tc.cu): bf16, b1 and b multiples of 64
 bool rect_stage1_tc_available(int q, int b1, int b, int dtype);
 int rect_stage1_tc(const void *x, const void *R, void *u, int64_t tokens, int q, int b1, int b, unsigned *status,
                    cudaStream_t s);
+// stage 2 as a TMA-fed streaming pass (rect_tc.cu): bf16, q and r at most 4, b a multiple of 8 and at least 256
+bool rect_stage2_stream_available(int q, int b, int r, int dtype);
+int rect_stage2_stream(const void *u, const void *Lp, void *y, int64_t tokens, int q, int b, int r, unsigned *status,
+                       cudaStream_t s);
 
 // ---- elementwise steps of the feed-forward block's backward pass (mlp_bwd.cu) ----
 // h = GELU(a (+ b1)); b1 may be null when a already holds the bias

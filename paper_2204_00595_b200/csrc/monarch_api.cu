@@ -334,13 +334,17 @@ int monarch_rect_fwd(const void *x, const void *L, const void *R, void *y, int64
     const Range out[] = {{y, (size_t)tokens * r * b * es}};
     MONARCH_TRY(check_buffers(in, 3, out, 1, workspace, workspace_bytes, rect_workspace_bytes(tokens, q, b, dtype)));
     cudaStream_t s = (cudaStream_t)stream;
+    void *u = (char *)workspace + MONARCH_STATUS_BYTES;
+    unsigned *status = (unsigned *)workspace;
+    const bool fast = g_impl.load(std::memory_order_relaxed) != MONARCH_IMPL_STAGED;
     // large bf16 blocks: stage 1 (nearly all the FLOPs when q is small) on the tensor cores
-    const bool tc1 = g_impl.load(std::memory_order_relaxed) != MONARCH_IMPL_STAGED &&
-                     rect_stage1_tc_available(q, b1, b, dtype);
-    if (tc1)
-        MONARCH_TRY(rect_stage1_tc(x, R, (char *)workspace + MONARCH_STATUS_BYTES, tokens, q, b1, b,
-                                   (unsigned *)workspace, s));
-    return rect_fwd_simt(x, L, R, y, tokens, q, b1, b, r, dtype, workspace, tc1, s);
+    if (fast && rect_stage1_tc_available(q, b1, b, dtype))
+        MONARCH_TRY(rect_stage1_tc(x, R, u, tokens, q, b1, b, status, s));
+    else
+        MONARCH_TRY(rect_stage1_simt(x, R, u, tokens, q, b1, b, dtype, s));
+    if (fast && rect_stage2_stream_available(q, b, r, dtype))
+        return rect_stage2_stream(u, L, y, tokens, q, b, r, status, s);
+    return rect_stage2_simt(u, L, y, tokens, q, b, r, dtype, s);
 }
 
 int monarch_workspace_init(void *workspace, size_t workspace_bytes, void *stream)

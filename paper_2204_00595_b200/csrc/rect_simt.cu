@@ -313,18 +313,20 @@ size_t rect_workspace_bytes(int64_t tokens, int q, int b, int dtype)
     return MONARCH_STATUS_BYTES + (((size_t)tokens * q * b * es + 255) & ~(size_t)255);
 }
 
-int rect_fwd_simt(const void *x, const void *Lp, const void *R, void *y, int64_t tokens, int q, int b1, int b, int r,
-                  int dtype, void *ws, int stage1_done, cudaStream_t s)
+int rect_stage1_simt(const void *x, const void *R, void *u, int64_t tokens, int q, int b1, int b, int dtype,
+                     cudaStream_t s)
 {
-    void *u = (char *)ws + MONARCH_STATUS_BYTES;
     const BlockProduct s1 = {tokens, q, b, b1, q * b1, q * b, b1, 1, b, 1};
+    return dtype == MONARCH_F32 ? block_product<float>(x, R, u, s1, s) : block_product<__nv_bfloat16>(x, R, u, s1, s);
+}
+
+int rect_stage2_simt(const void *u, const void *Lp, void *y, int64_t tokens, int q, int b, int r, int dtype,
+                     cudaStream_t s)
+{
     const BlockProduct s2 = {tokens, b, r, q, q * b, r * b, 1, b, 1, b};
     const bool small4 = q <= 4 && r <= 4 && b % 2 == 0 && tokens > 0;
-    if (dtype == MONARCH_F32) {
-        if (!stage1_done) MONARCH_TRY(block_product<float>(x, R, u, s1, s));
+    if (dtype == MONARCH_F32)
         return small4 ? stage2_small4<float>(u, Lp, y, tokens, q, b, r, s) : block_product<float>(u, Lp, y, s2, s);
-    }
-    if (!stage1_done) MONARCH_TRY(block_product<__nv_bfloat16>(x, R, u, s1, s));
     return small4 ? stage2_small4<__nv_bfloat16>(u, Lp, y, tokens, q, b, r, s)
                   : block_product<__nv_bfloat16>(u, Lp, y, s2, s);
 }

@@ -216,6 +216,125 @@ int launch(const void *x, const void *R, void *u, int64_t tokens, int q, int b1,
     return MONARCH_OK;
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Stage 2 when L's blocks are at most 4 x 4:  y[t][l*b + j] = sum_k Lp[j][l][k] u[t][k*b + j]  as a streaming pass.
+// A CTA owns 256 columns j and a slab of tokens; TMA brings 16-token tiles of the q slices u[t][k*b + j0 ..] into a
+// three-stage ring (no thread holds a load in flight, so the pass is not limited by registers x occupancy), the
+// blocks sit in shared memory as fp32, and each thread turns 8 columns of two tokens into r x 8 outputs per step,
+// written back with 16-byte stores (a warp writes 512 contiguous bytes of a slice y[t][l*b + .]).
+constexpr int kS2Cols = 256, kS2Tok = 16, kS2Stages = 3, kS2Threads = 256;
+constexpr int kS2SliceBytes = kS2Tok * kS2Cols * 2;                 // one k slice of a tile
+constexpr int kS2SmemBytes = kS2Stages * 4 * kS2SliceBytes + 128;     // two CTAs per SM with the 16 KB of blocks
+
+__device__ __forceinline__ float4 lds128f(uint32_t addr)
+{
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint4 lds128u(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ float bf_elem(const uint4 &v, int e)
+{
+    const uint32_t w = e < 2 ? v.x : e < 4 ? v.y : e < 6 ? v.z : v.w;
+    return (e & 1) ? __uint_as_float(w & 0xFFFF0000u) : __uint_as_float(w << 16);
+}
+
+__global__ void __launch_bounds__(kS2Threads, 2)
+rect_stage2_stream_kernel(const __grid_constant__ CUtensorMap tm_u, const __nv_bfloat16 *__restrict__ Lp,
+                          __nv_bfloat16 *__restrict__ y, unsigned *status, long long tokens, int q, int b, int r,
+                          int tokens_per_slab)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ float4 ws[4][4][2][32];            // [l][k][half][lane]: columns 8 lane + 4 half + (0..3)
+    __shared__ __align__(8) uint64_t full[kS2Stages];
+    __shared__ int dead_s;
+    const uint32_t ring0 = (smem_u32(smem_raw) + 127u) & ~127u;
+    const int j0 = blockIdx.x * kS2Cols;
+    volatile int *dead = &dead_s;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kS2Stages; ++s) mbar_init(smem_u32(&full[s]), 1);
+        fence_mbar_init();
+        dead_s = 0;
+        tma_prefetch_desc(&tm_u);
+    }
+    for (int i = threadIdx.x; i < 16 * kS2Cols; i += kS2Threads) {
+        const int jl = i >> 4, l = (i >> 2) & 3, k = i & 3;
+        float v = 0.0f;
+        if (j0 + jl < b && l < r && k < q) v = __bfloat162float(Lp[((size_t)(j0 + jl) * r + l) * q + k]);
+        reinterpret_cast<float *>(&ws[l][k][(jl >> 2) & 1][jl >> 3])[jl & 3] = v;
+    }
+    __syncthreads();
+
+    const long long t0 = (long long)blockIdx.y * tokens_per_slab;
+    const long long t1 = t0 + tokens_per_slab < tokens ? t0 + tokens_per_slab : tokens;
+    const int ntiles = t1 > t0 ? (int)((t1 - t0 + kS2Tok - 1) / kS2Tok) : 0;
+    const uint32_t full0 = smem_u32(full);
+    const uint32_t stage_bytes = (uint32_t)q * kS2SliceBytes;
+
+    auto issue = [&](int tile) {
+        const uint32_t s = tile % kS2Stages;
+        mbar_expect_tx(full0 + s * 8, stage_bytes);
+        for (int k = 0; k < q; ++k)
+            tma_load_2d(ring0 + s * 4 * kS2SliceBytes + k * kS2SliceBytes, &tm_u, k * b + j0,
+                        (int)(t0 + (long long)tile * kS2Tok), full0 + s * 8);
+    };
+    if (threadIdx.x == 0)
+        for (int tile = 0; tile < kS2Stages - 1 && tile < ntiles; ++tile) issue(tile);
+
+    const int lane = threadIdx.x & 31, tr = threadIdx.x >> 5;             // 32 threads per token row, rows tr, tr + 8
+    const bool active = j0 + lane * 8 < b;
+    const uint32_t ws0 = smem_u32(ws);
+    for (int tile = 0; tile < ntiles; ++tile) {
+        // the stage this load goes to was read in the previous step, which ended with a CTA barrier
+        if (threadIdx.x == 0 && tile + kS2Stages - 1 < ntiles) issue(tile + kS2Stages - 1);
+        const uint32_t s = tile % kS2Stages;
+        if (!mbar_wait(full0 + s * 8, (tile / kS2Stages) & 1, status, dead, kErrTmaWait)) break;
+        const long long ta = t0 + (long long)tile * kS2Tok + tr, tb = ta + 8;
+        if (active && ta < t1) {
+            const bool two = tb < t1;
+            const uint32_t src = ring0 + s * 4 * kS2SliceBytes + lane * 16;
+            uint4 v[2][4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                v[0][k] = k < q ? lds128u(src + k * kS2SliceBytes + tr * (kS2Cols * 2)) : make_uint4(0u, 0u, 0u, 0u);
+                v[1][k] = k < q ? lds128u(src + k * kS2SliceBytes + (tr + 8) * (kS2Cols * 2)) : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll 1
+            for (int l = 0; l < r; ++l) {
+                float acc[2][8];
+#pragma unroll
+                for (int tt = 0; tt < 2; ++tt)
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) acc[tt][e] = 0.0f;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const float4 wa = lds128f(ws0 + ((l * 4 + k) * 2 + 0) * 512 + lane * 16);
+                    const float4 wb = lds128f(ws0 + ((l * 4 + k) * 2 + 1) * 512 + lane * 16);
+                    const float wv[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+#pragma unroll
+                    for (int tt = 0; tt < 2; ++tt)
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) acc[tt][e] = fmaf(wv[e], bf_elem(v[tt][k], e), acc[tt][e]);
+                }
+#pragma unroll
+                for (int tt = 0; tt < 2; ++tt) {
+                    if (tt == 1 && !two) break;
+                    const uint4 o = make_uint4(pack_bf16(acc[tt][0], acc[tt][1]), pack_bf16(acc[tt][2], acc[tt][3]),
+                                               pack_bf16(acc[tt][4], acc[tt][5]), pack_bf16(acc[tt][6], acc[tt][7]));
+                    *reinterpret_cast<uint4 *>(y + (size_t)(tt ? tb : ta) * r * b + (size_t)l * b + j0 + lane * 8) = o;
+                }
+            }
+        }
+        __syncthreads();
+    }
+}
+
 }  // namespace
 }  // namespace tc
 
@@ -223,6 +342,40 @@ bool rect_stage1_tc_available(int q, int b1, int b, int dtype)
 {
     (void)q;
     return dtype == MONARCH_BF16 && b1 % 64 == 0 && b % 64 == 0;
+}
+
+bool rect_stage2_stream_available(int q, int b, int r, int dtype)
+{
+    return dtype == MONARCH_BF16 && q <= 4 && r <= 4 && b % 8 == 0 && b >= 256;     // a 256-column box fits a slice
+}
+
+int rect_stage2_stream(const void *u, const void *Lp, void *y, int64_t tokens, int q, int b, int r, unsigned *status,
+                       cudaStream_t s)
+{
+    using namespace tc;
+    if (tokens == 0) return MONARCH_OK;
+    CUtensorMap tm_u;
+    MONARCH_TRY(encode_tmap_2d(&tm_u, u, (uint64_t)tokens, (uint64_t)q * b, (uint64_t)q * b * 2, kS2Tok, kS2Cols, 0));
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        MONARCH_CUDA_TRY(cudaGetDevice(&dev));
+        MONARCH_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        MONARCH_CUDA_TRY(cudaFuncSetAttribute(rect_stage2_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              kS2SmemBytes));
+    }
+    const int cx = (b + kS2Cols - 1) / kS2Cols;
+    long long slabs = (2LL * sms + cx - 1) / cx;                     // two CTAs per SM, one wave
+    if (slabs > (tokens + kS2Tok - 1) / kS2Tok) slabs = (tokens + kS2Tok - 1) / kS2Tok;
+    long long per = (tokens + slabs - 1) / slabs;
+    per = (per + kS2Tok - 1) / kS2Tok * kS2Tok;
+    slabs = (tokens + per - 1) / per;
+    if (slabs > 65535) return MONARCH_ERR_UNSUPPORTED;
+    rect_stage2_stream_kernel<<<dim3((unsigned)cx, (unsigned)slabs), kS2Threads, kS2SmemBytes, s>>>(
+        tm_u, (const __nv_bfloat16 *)Lp, (__nv_bfloat16 *)y, status, tokens, q, b, r, (int)per);
+    note_launch();
+    MONARCH_CUDA_TRY(cudaGetLastError());
+    return MONARCH_OK;
 }
 
 int rect_stage1_tc(const void *x, const void *R, void *u, int64_t tokens, int q, int b1, int b, unsigned *status,
