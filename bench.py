@@ -5,6 +5,8 @@ One step = one pass of the hot path over one batch of synthetic tokens of the ch
 workload (default: workload 3, n=4096, m=64, 8192 tokens per GPU, bf16):
     monarch_fwd (y) + monarch_bwd_dx (dx) + monarch_bwd_dw (dL, dR).
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+`--workload 5 --calls mlp_fwd,mlp_bwd` adds the backward of the feed-forward block; `--workload 6` times the
+forward of the general (rectangular) Monarch class.
 
 Launch for N > 1:  python -m torch.distributed.run --nnodes=1 --nproc-per-node N
     --master-addr 127.0.0.1 --master-port P bench.py --gpus N --steps K --warmup W

@@ -266,6 +266,8 @@ class HostContext:
     """Device staging for the host-buffer calls (monarch_host_*): tensors are CPU tensors, ideally
     pinned; every call blocks until its outputs have arrived."""
 
+    _h = None          # so that close() is safe when construction raised
+
     def __init__(self, max_tokens: int, n: int, m: int, dtype: int, chunk_tokens: int = 0):
         h = _vp()
         _check(lib().monarch_host_create(ctypes.byref(h), max_tokens, n, m, dtype, chunk_tokens),
