@@ -163,6 +163,25 @@ int monarch_rect_fwd(const void *x, const void *L, const void *R, void *y, int64
 size_t monarch_rect_workspace_bytes(int64_t tokens, int32_t q, int32_t b1, int32_t b, int32_t r,
                                     int dtype);
 
+/* Dense materialisation by the entry formula, Eq. (2):
+ *   M[l*m+j][k*m+i] = L[j][l][k] * R[k][j][i],   M: [n][n] row-major, storage dtype
+ * (the product is formed in fp32 and rounded once). */
+int monarch_dense(const void *L, const void *R, void *M, int32_t n, int32_t m, int dtype,
+                  void *stream);
+
+/* Projection of a dense matrix onto the Monarch class, Algorithm 1: with
+ * A~[l][j][k][i] = A[l*m+j][k*m+i], every m x m slice A~[:, j, k, :] is replaced
+ * by its best rank-1 approximation sigma_1 u_1 v_1^T (Theorem 1: this minimises
+ * ||A - M||_F over Monarch M), stored as L[j][:, k] = sqrt(sigma_1) u_1 and
+ * R[k][j][:] = sqrt(sigma_1) v_1.  The paper fixes only the product u v^T; the
+ * sign of the pair is arbitrary, and where sigma_1 = sigma_2 the slice's
+ * approximation itself is not unique.  A: [n][n] row-major; L, R: [m][m][m];
+ * all in the storage dtype, arithmetic in fp32 (one-sided Jacobi per slice).
+ * `rotation_count` is null or a device counter to which the number of plane
+ * rotations performed is added (for FLOP accounting). */
+int monarch_project(const void *A, void *L, void *R, int32_t n, int32_t m, int dtype,
+                    unsigned long long *rotation_count, void *stream);
+
 /* Bytes of workspace `op` (a monarch_op_t) needs for these sizes under the
  * current implementation choice; always >= MONARCH_STATUS_BYTES.  Returns 0
  * for invalid or unsupported arguments. */

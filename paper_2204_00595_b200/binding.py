@@ -28,6 +28,8 @@ _SIGNATURES = {
     "monarch_mlp_bwd": (_int, [_vp] * 14 + [_int, _i64, _i32, _i32, _int, _vp, _sz, _vp]),
     "monarch_rect_fwd": (_int, [_vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32, _int, _vp, _sz, _vp]),
     "monarch_rect_workspace_bytes": (_sz, [_i64, _i32, _i32, _i32, _i32, _int]),
+    "monarch_dense": (_int, [_vp, _vp, _vp, _i32, _i32, _int, _vp]),
+    "monarch_project": (_int, [_vp, _vp, _vp, _i32, _i32, _int, _vp, _vp]),
     "monarch_workspace_bytes": (_sz, [_int, _i64, _i32, _i32, _int]),
     "monarch_workspace_init": (_int, [_vp, _sz, _vp]),
     "monarch_last_device_status": (_int, [_vp, _vp]),
@@ -234,6 +236,23 @@ def monarch_rect_fwd(x, L, R, y, tokens, q, b1, b, r, workspace, stream=None) ->
     p, nb = _ws(workspace)
     _check(lib().monarch_rect_fwd(_ptr(x, "x"), _ptr(L, "L", dt), _ptr(R, "R", dt), _ptr(y, "y", dt), tokens,
                                   q, b1, b, r, _dtype_code(x), p, nb, _stream(stream)), "monarch_rect_fwd")
+
+
+def monarch_dense(L, R, M, n, m, stream=None) -> None:
+    """M[l*m+j, k*m+i] = L[j, l, k] * R[k, j, i] (Eq. 2); M is [n, n] in the dtype of L."""
+    dt = L.dtype
+    _check(lib().monarch_dense(_ptr(L, "L"), _ptr(R, "R", dt), _ptr(M, "M", dt), n, m, _dtype_code(L),
+                               _stream(stream)), "monarch_dense")
+
+
+def monarch_project(A, L, R, n, m, rotation_count=None, stream=None) -> None:
+    """Algorithm 1: factors L, R of the Monarch matrix closest to the dense A in Frobenius norm.
+    rotation_count: optional one-element int64 CUDA tensor, incremented by the number of Jacobi rotations."""
+    import torch
+    dt = A.dtype
+    rc = _ptr(rotation_count, "rotation_count", torch.int64) if rotation_count is not None else None
+    _check(lib().monarch_project(_ptr(A, "A"), _ptr(L, "L", dt), _ptr(R, "R", dt), n, m, _dtype_code(A), rc,
+                                 _stream(stream)), "monarch_project")
 
 
 NOALLOC_SCRATCH_BYTES = 8 << 20

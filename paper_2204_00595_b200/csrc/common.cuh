@@ -158,6 +158,10 @@ bool rect_stage2_stream_available(int q, int b, int r, int dtype);
 int rect_stage2_stream(const void *u, const void *Lp, void *y, int64_t tokens, int q, int b, int r, unsigned *status,
                        cudaStream_t s);
 
+// ---- dense <-> Monarch factors (project.cu): Eq. (2) and Algorithm 1 ----
+int dense_from_factors(const void *L, const void *R, void *M, int m, int dtype, cudaStream_t s);
+int project_to_factors(const void *A, void *L, void *R, int m, int dtype, unsigned long long *rotations, cudaStream_t s);
+
 // ---- elementwise steps of the feed-forward block's backward pass (mlp_bwd.cu) ----
 // h = GELU(a (+ b1)); b1 may be null when a already holds the bias
 int mlp_act(const void *a, const void *b1, void *h, int64_t tokens, int n, int dtype, cudaStream_t s);

@@ -347,6 +347,32 @@ int monarch_rect_fwd(const void *x, const void *L, const void *R, void *y, int64
     return rect_stage2_simt(u, L, y, tokens, q, b, r, dtype, s);
 }
 
+int monarch_dense(const void *L, const void *R, void *M, int32_t n, int32_t m, int dtype, void *stream)
+{
+    MONARCH_TRY(check_shape(0, n, m, dtype));
+    const size_t wb = (size_t)n * m * esize(dtype), mb = (size_t)n * n * esize(dtype);
+    const Range in[] = {{L, wb}, {R, wb}};
+    const Range out = {M, mb};
+    for (const Range &r : in)
+        if (!r.p || !aligned(r.p, 16) || overlap(out, r)) return MONARCH_ERR_INVALID_ARG;
+    if (!M || !aligned(M, 16)) return MONARCH_ERR_INVALID_ARG;
+    return dense_from_factors(L, R, M, m, dtype, (cudaStream_t)stream);
+}
+
+int monarch_project(const void *A, void *L, void *R, int32_t n, int32_t m, int dtype,
+                    unsigned long long *rotation_count, void *stream)
+{
+    MONARCH_TRY(check_shape(0, n, m, dtype));
+    const size_t wb = (size_t)n * m * esize(dtype), mb = (size_t)n * n * esize(dtype);
+    const Range in = {A, mb};
+    const Range out[] = {{L, wb}, {R, wb}};
+    if (!A || !aligned(A, 16)) return MONARCH_ERR_INVALID_ARG;
+    for (const Range &r : out)
+        if (!r.p || !aligned(r.p, 16) || overlap(r, in)) return MONARCH_ERR_INVALID_ARG;
+    if (overlap(out[0], out[1])) return MONARCH_ERR_INVALID_ARG;
+    return project_to_factors(A, L, R, m, dtype, rotation_count, (cudaStream_t)stream);
+}
+
 int monarch_workspace_init(void *workspace, size_t workspace_bytes, void *stream)
 {
     if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < MONARCH_STATUS_BYTES)

@@ -484,6 +484,84 @@ def test_rect_arguments(P):
     assert float(y.min()) == 3.0
 
 
+# ----------------------------------------------------------------- dense <-> factors (Eq. 2, Algorithm 1)
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("m", [16, 32, 64])
+def test_dense_from_factors(P, m, dtype):
+    import torch
+    n = m * m
+    d = _small_inputs(m, 1, dtype, seed=40 + m)
+    L, R = to_device(d["L"], dtype), to_device(d["R"], dtype)
+    Mf, M = _guarded((n, n), _tdtype(dtype))
+    P.monarch_dense(L, R, M, n, m)
+    torch.cuda.synchronize()
+    assert_close(to_host64(M), O.dense(d["L"], d["R"]), dtype, "dense")
+    _check_guard(Mf, "dense")
+
+
+def _project_gpu(P, A32, m, dtype):
+    import torch
+    n = m * m
+    A = to_device(A32, dtype)
+    Lf, L = _guarded((m, m, m), _tdtype(dtype))
+    Rf, R = _guarded((m, m, m), _tdtype(dtype))
+    rot = torch.zeros(1, dtype=torch.int64, device="cuda")
+    P.monarch_project(A, L, R, n, m, rotation_count=rot)
+    torch.cuda.synchronize()
+    _check_guard(Lf, "project L")
+    _check_guard(Rf, "project R")
+    assert int(rot.item()) > 0
+    return to_host64(L), to_host64(R)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("m", [16, 32, 64])
+def test_project_recovers_monarch_and_planted(P, m, dtype):
+    """Section 3.3: a Monarch input is recovered; with small noise added the slices keep a clear leading
+    singular value, so the rank-1 pieces are well conditioned and must match the oracle's (numpy SVD)."""
+    rng = np.random.default_rng(600 + m)
+    d = _small_inputs(m, 1, dtype, seed=50 + m)
+    A = O.dense(d["L"], d["R"])
+    A32 = round_to_storage(A.astype(np.float32), dtype)
+    Lg, Rg = _project_gpu(P, A32, m, dtype)
+    assert_close(O.dense(Lg, Rg), A32.astype(np.float64), dtype, "project(monarch)", scale=2.0)
+    noisy = round_to_storage((A + 0.02 / m * rng.standard_normal(A.shape)).astype(np.float32), dtype)
+    Lg, Rg = _project_gpu(P, noisy, m, dtype)
+    Lo, Ro = O.project(noisy.astype(np.float64), m)
+    assert_close(O.dense(Lg, Rg), O.dense(Lo, Ro), dtype, "project(planted)", scale=2.0)
+
+
+@pytest.mark.parametrize("m", [16, 64])
+def test_project_generic_is_optimal(P, m):
+    """Theorem 1: the residual of the projection equals the discarded spectrum of the slices - a criterion
+    that does not depend on the gap between the first two singular values."""
+    rng = np.random.default_rng(700 + m)
+    n = m * m
+    A32 = rng.standard_normal((n, n), dtype=np.float32)
+    Lg, Rg = _project_gpu(P, A32, m, "f32")
+    A = A32.astype(np.float64)
+    res = float(np.sum((A - O.dense(Lg, Rg)) ** 2))
+    sv = np.linalg.svd(A.reshape(m, m, m, m).transpose(1, 2, 0, 3).reshape(m * m, m, m), compute_uv=False)
+    tail = float(np.sum(sv[:, 1:] ** 2))
+    assert tail * (1 - 1e-9) <= res <= tail * (1 + 1e-5)
+
+
+def test_project_m128_sampled_slices(P):
+    rng = np.random.default_rng(728)
+    m = 128
+    n = m * m
+    A32 = rng.standard_normal((n, n), dtype=np.float32)
+    Lg, Rg = _project_gpu(P, A32, m, "f32")
+    A4 = A32.reshape(m, m, m, m)                           # [l, j, k, i]
+    for j, k in [(0, 0), (5, 127), (127, 3), (64, 64), (17, 90)]:
+        S = A4[:, j, k, :].astype(np.float64)
+        sv = np.linalg.svd(S, compute_uv=False)
+        res = float(np.sum((S - np.outer(Lg[j, :, k], Rg[k, j, :])) ** 2))
+        tail = float(np.sum(sv[1:] ** 2))
+        assert tail * (1 - 1e-9) <= res <= tail * (1 + 1e-5)
+
+
 # ----------------------------------------------------------------- the five workloads
 
 def _sample_tokens(T, count, seed):
