@@ -37,8 +37,9 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=3, choices=[1, 2, 3, 4, 5, 6],
-                    help="1-5: the square workloads; 6: the general (rectangular) class, forward only")
+    ap.add_argument("--workload", type=int, default=3, choices=[1, 2, 3, 4, 5, 6, 7],
+                    help="1-5: the square workloads; 6: the general (rectangular) class, forward only; "
+                         "7: projection of a dense matrix onto the Monarch class + dense materialisation")
     ap.add_argument("--kernels", default="auto", choices=["auto", "staged", "fused"])
     ap.add_argument("--calls", default="", help="comma-separated subset of the workload's calls "
                     "(profiling aid; the default step runs them all)")
@@ -322,10 +323,105 @@ def main_rect(args):
     return 0
 
 
+def main_project(args):
+    """Workload 7: Algorithm 1 (projection, one rank-1 SVD per m x m slice) followed by Eq. (2) (dense
+    materialisation) for n = 4096, m = 64, fp32.  The projection is bound by instruction issue on the CUDA
+    cores; its FLOPs are counted from the plane rotations the kernel reports (12 m per rotation: three dot
+    products and two column updates of length m)."""
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    m, n = 64, 4096
+    workload = f"workload 7: project+dense f32 n={n} m={m} ({m * m} slices of {m} x {m})"
+    metric, unit = "monarch_project_matrices_per_s", "matrices/s"
+    import numpy as np
+    rng = np.random.default_rng(595007)
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        from oracle import monarch_oracle as O
+        sub = 16                                  # the oracle (numpy SVD per slice) on a 16 x 16-block instance
+        A = rng.standard_normal((sub * sub, sub * sub))
+        ts = []
+        for i in range(args.warmup + args.steps):
+            t0 = time.perf_counter()
+            L, R = O.project(A, sub)
+            O.dense(L, R)
+            ts.append(time.perf_counter() - t0)
+        dt = statistics.mean(ts[args.warmup:])
+        # scale by slice count and the cubic cost of an SVD to the workload's 64 x 64 slices
+        est = dt * (m * m) / (sub * sub) * (m / sub) ** 3
+        print(json.dumps({
+            "impl": "reference", "metric": metric, "value": 1.0 / est, "unit": unit, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": est * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": workload, "sample": f"m={sub} instance timed ({dt * 1e3:.1f} ms), scaled by "
+                                                       "slice count and m^3"},
+            "cpu_baseline": {"value": 1.0 / est, "unit": unit, "cores": 1, "kind": "oracle",
+                             "sample": f"m={sub} instance, scaled"},
+            "e2e": {"value": 1.0 / est, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+        return 0
+
+    import torch
+    import __graft_entry__ as entry
+    entry.build()
+    import paper_2204_00595_b200 as P
+    torch.cuda.set_device(local_rank)
+    A = torch.from_numpy(rng.standard_normal((n, n), dtype=np.float32)).cuda()
+    L = torch.empty(m, m, m, device="cuda")
+    R = torch.empty_like(L)
+    M = torch.empty_like(A)
+    rot = torch.zeros(1, dtype=torch.int64, device="cuda")
+    stream = torch.cuda.current_stream()
+    for _ in range(args.warmup):
+        P.monarch_project(A, L, R, n, m)
+        P.monarch_dense(L, R, M, n, m)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = P.monarch_launch_count()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * args.steps + 1)]
+    ev[0].record(stream)
+    for i in range(args.steps):
+        P.monarch_project(A, L, R, n, m, rotation_count=rot)
+        ev[2 * i + 1].record(stream)
+        P.monarch_dense(L, R, M, n, m)
+        ev[2 * i + 2].record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    launches = P.monarch_launch_count() - launches0
+    t_proj = statistics.mean(ev[2 * i].elapsed_time(ev[2 * i + 1]) for i in range(args.steps))
+    t_dense = statistics.mean(ev[2 * i + 1].elapsed_time(ev[2 * i + 2]) for i in range(args.steps))
+    ms = ev[0].elapsed_time(ev[-1]) / args.steps
+    flops = int(rot.item()) / args.steps * 12 * m
+    sm_mhz = clocks.get("sm_max_mhz") or 1965
+    alu_peak = 148 * 128 * 2 * sm_mhz * 1e6 / 1e12          # fp32 FMA lanes x 2 FLOP x clock
+    line = {
+        "metric": metric, "value": world / (ms * 1e-3), "unit": unit, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": workload, "l2": "A (67 MB) + M (67 MB) exceed L2"},
+        "clocks": clocks, "gpu_launches": int(launches),
+        "calls": {"project": {"ms": t_proj, "rotations": int(rot.item()) // args.steps,
+                              "tflops": flops / t_proj / 1e9},
+                  "dense": {"ms": t_dense, "gbs": n * n * 4 / t_dense / 1e6}},
+        "roofline": {"bound": "alu", "kernel": "project_kernel<float, 64>", "achieved": flops / t_proj / 1e9,
+                     "peak": alu_peak, "unit": "TFLOP/s", "frac": flops / t_proj / 1e9 / alu_peak,
+                     "peak_source": "148 SMs x 128 fp32 FMA lanes x 2 FLOP x max SM clock", "traffic": None},
+        "e2e": None,
+    }
+    if rank == 0:
+        print(json.dumps(line))
+    return 0
+
+
 def main():
     args = parse_args()
     if args.workload == 6:
         return main_rect(args)
+    if args.workload == 7:
+        return main_project(args)
     from paper_2204_00595_b200.inputs import CONFIGS, make_inputs
     cfg = CONFIGS[args.workload]
     rank = int(os.environ.get("RANK", "0"))

@@ -31,12 +31,18 @@ constexpr int kMaxSweeps = 30;
 constexpr float kOrthoTol = 2e-6f;
 
 // Rotation counter for the benchmark's FLOP count (optional, may be null).
+// Warps per slice: each warp takes four column pairs per round (two for m = 16) as independent chains, and
+// several CTAs share an SM - the iteration is bound by the latency of load / shuffle-reduce / rotate, not by FLOPs.
+template <int M> struct ProjectCfg {
+    static constexpr int kWarps = M >= 32 ? M / 8 : 4;
+};
+
 template <typename T, int M>
-__global__ void __launch_bounds__(M <= 64 ? (M / 2) * 32 : 1024)
+__global__ void __launch_bounds__(ProjectCfg<M>::kWarps * 32)
 project_kernel(const T *__restrict__ A, T *__restrict__ L, T *__restrict__ R, unsigned long long *rotations)
 {
     constexpr int N = M * M;
-    constexpr int kWarps = M <= 64 ? M / 2 : 32;
+    constexpr int kWarps = ProjectCfg<M>::kWarps;
     constexpr int kPairsPerWarp = (M / 2) / kWarps;
     constexpr int kPitch = M + 1;                         // column pitch in floats (odd: no bank conflicts)
     constexpr int kRows = (M + 31) / 32;                  // rows per lane
@@ -158,7 +164,7 @@ project_kernel(const T *__restrict__ A, T *__restrict__ L, T *__restrict__ R, un
 template <typename T, int M>
 int launch_project(const void *A, void *L, void *R, unsigned long long *rotations, cudaStream_t s)
 {
-    constexpr int kWarps = M <= 64 ? M / 2 : 32;
+    constexpr int kWarps = ProjectCfg<M>::kWarps;
     constexpr int smem = M * (M + 1) * (int)sizeof(float);
     static bool attr = false;
     if (!attr && smem > 48 * 1024) {
