@@ -31,21 +31,27 @@ constexpr int kMaxSweeps = 30;
 constexpr float kOrthoTol = 2e-6f;
 
 // Rotation counter for the benchmark's FLOP count (optional, may be null).
-// Warps per slice: each warp takes four column pairs per round (two for m = 16) as independent chains, and
-// several CTAs share an SM - the iteration is bound by the latency of load / shuffle-reduce / rotate, not by FLOPs.
+// A column pair is handled by G lanes (m/G rows each): G = 8 for m <= 64, so that a warp rotates four pairs at once
+// - with 64-element columns a whole warp per pair would spend most of its instructions on shuffle and scalar work
+// replicated over 32 lanes - and G = 32 for m = 128, where the strided rows of four different columns would
+// collide in the shared-memory banks.  Several CTAs share an SM.
 template <int M> struct ProjectCfg {
-    static constexpr int kWarps = M >= 32 ? M / 8 : 4;
+    static constexpr int kG = M >= 128 ? 32 : 8;
+    static constexpr int kPairsPerPass = 32 / kG;                       // pairs a warp rotates at once
+    static constexpr int kWarps = M >= 128 ? 32 : (M / 8 < 2 ? 2 : M / 8);
+    static constexpr int kPasses = (M / 2) / (kWarps * kPairsPerPass);  // passes per round
 };
 
 template <typename T, int M>
 __global__ void __launch_bounds__(ProjectCfg<M>::kWarps * 32)
 project_kernel(const T *__restrict__ A, T *__restrict__ L, T *__restrict__ R, unsigned long long *rotations)
 {
+    using C = ProjectCfg<M>;
     constexpr int N = M * M;
-    constexpr int kWarps = ProjectCfg<M>::kWarps;
-    constexpr int kPairsPerWarp = (M / 2) / kWarps;
+    constexpr int kWarps = C::kWarps, G = C::kG;
+    static_assert(kWarps * C::kPairsPerPass * C::kPasses == M / 2, "a round covers every column once");
     constexpr int kPitch = M + 1;                         // column pitch in floats (odd: no bank conflicts)
-    constexpr int kRows = (M + 31) / 32;                  // rows per lane
+    constexpr int kRows = M / G;                          // rows per lane
     extern __shared__ float cols[];                       // cols[i * kPitch + l] = S[l][i]
     __shared__ float red_val[32];
     __shared__ int red_idx[32];
@@ -55,6 +61,7 @@ project_kernel(const T *__restrict__ A, T *__restrict__ L, T *__restrict__ R, un
 
     const int j = blockIdx.x / M, k = blockIdx.x % M;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int grp = lane / G, sub = lane % G;
     const T *slice = A + (size_t)j * N + (size_t)k * M;   // element (l, i) at slice[l * M * N + i]
 
     for (int e = threadIdx.x; e < M * M; e += kWarps * 32) {
@@ -68,57 +75,53 @@ project_kernel(const T *__restrict__ A, T *__restrict__ L, T *__restrict__ R, un
         int rotated = 0;
         for (int rr = 0; rr < M - 1; ++rr) {
 #pragma unroll
-            for (int pp = 0; pp < kPairsPerWarp; ++pp) {
+            for (int pass = 0; pass < C::kPasses; ++pass) {
                 // round-robin tournament: column M-1 stays, the others move round a circle of M-1 seats
-                const int p = warp * kPairsPerWarp + pp;
-                int ca, cb;
-                if (p == 0) {
-                    ca = M - 1;
-                    cb = rr;
-                } else {
-                    ca = (rr + p) % (M - 1);
-                    cb = (rr - p + (M - 1)) % (M - 1);
-                }
-                float *a = cols + ca * kPitch, *b = cols + cb * kPitch;
+                const int p = (warp * C::kPasses + pass) * C::kPairsPerPass + grp;
+                int ca = rr + p, cb = rr - p + (M - 1);
+                if (ca >= M - 1) ca -= M - 1;
+                if (cb >= M - 1) cb -= M - 1;
+                if (p == 0) ca = M - 1;
+                float *a = cols + ca * kPitch + sub, *b = cols + cb * kPitch + sub;
                 float av[kRows], bv[kRows];
                 float aa = 0.0f, bb = 0.0f, ab = 0.0f;
 #pragma unroll
                 for (int q = 0; q < kRows; ++q) {
-                    const int l = lane + 32 * q;
-                    av[q] = l < M ? a[l] : 0.0f;
-                    bv[q] = l < M ? b[l] : 0.0f;
+                    av[q] = a[G * q];
+                    bv[q] = b[G * q];
                     aa = fmaf(av[q], av[q], aa);
                     bb = fmaf(bv[q], bv[q], bb);
                     ab = fmaf(av[q], bv[q], ab);
                 }
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
+                for (int o = G / 2; o > 0; o >>= 1) {
                     aa += __shfl_xor_sync(0xffffffffu, aa, o);
                     bb += __shfl_xor_sync(0xffffffffu, bb, o);
                     ab += __shfl_xor_sync(0xffffffffu, ab, o);
                 }
-                // rotate unless the two columns are already orthogonal to working precision
-                if (fabsf(ab) > kOrthoTol * sqrtf(aa * bb) && ab != 0.0f) {
-                    const float zeta = (bb - aa) / (2.0f * ab);
-                    const float t = copysignf(1.0f, zeta) / (fabsf(zeta) + sqrtf(1.0f + zeta * zeta));
-                    const float c = rsqrtf(1.0f + t * t), s = c * t;
+                // rotate unless the two columns are already orthogonal to working precision.  The angle only has to
+                // be roughly right (orthogonality is re-tested every sweep, and the factors are formed from a
+                // re-normalised column), so the fast reciprocal / square-root forms are enough.
+                if (ab * ab > (kOrthoTol * kOrthoTol) * (aa * bb)) {
+                    // clamped: columns that are pure rounding noise (rank-deficient slices) give huge ratios
+                    const float zeta = fmaxf(fminf(__fdividef(bb - aa, 2.0f * ab), 1e15f), -1e15f);
+                    const float w = fmaf(zeta, zeta, 1.0f);
+                    const float t = copysignf(__fdividef(1.0f, fabsf(zeta) + w * rsqrtf(w)), zeta);
+                    const float c = rsqrtf(fmaf(t, t, 1.0f)), s = c * t;
 #pragma unroll
                     for (int q = 0; q < kRows; ++q) {
-                        const int l = lane + 32 * q;
-                        if (l < M) {
-                            a[l] = c * av[q] - s * bv[q];
-                            b[l] = s * av[q] + c * bv[q];
-                        }
+                        a[G * q] = c * av[q] - s * bv[q];
+                        b[G * q] = s * av[q] + c * bv[q];
                     }
                     rotated = 1;
-                    ++my_rot;
+                    if (sub == 0) ++my_rot;
                 }
             }
             __syncthreads();
         }
         if (!__syncthreads_or(rotated)) break;
     }
-    if (rotations != nullptr && lane == 0 && my_rot) atomicAdd(rotations, (unsigned long long)my_rot);
+    if (rotations != nullptr && my_rot) atomicAdd(rotations, (unsigned long long)my_rot);
 
     // the column of largest norm carries sigma_1 u_1
     float best = -1.0f;
