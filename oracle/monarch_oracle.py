@@ -260,6 +260,45 @@ def rect_factors_from_definition(Lp, R):
     return Ld, Rd
 
 
+def cplx_dense_from_definition(L, R) -> np.ndarray:
+    """Definition 3.1 with complex factors: M = P L P^T R as a dense complex n x n matrix."""
+    L = np.asarray(L, dtype=np.complex128); R = np.asarray(R, dtype=np.complex128)
+    m = L.shape[0]
+    n = m * m
+    P = perm_matrix(m)
+    Ld = np.zeros((n, n), dtype=np.complex128)
+    Rd = np.zeros((n, n), dtype=np.complex128)
+    for b in range(m):
+        Ld[b * m:(b + 1) * m, b * m:(b + 1) * m] = L[b]
+        Rd[b * m:(b + 1) * m, b * m:(b + 1) * m] = R[b]
+    return P @ Ld @ P.T @ Rd
+
+
+def cplx_fwd(x, L, R, adjoint: bool = False) -> np.ndarray:
+    """Complex Monarch multiply by the paper's steps 1-3 in complex128 (x: [T, n], L, R: [m, m, m]);
+    adjoint=True applies M^H = R^H P L^H P (the second factor of the MM* products of Section 3.2)."""
+    x = np.asarray(x, dtype=np.complex128); L = np.asarray(L, dtype=np.complex128)
+    R = np.asarray(R, dtype=np.complex128)
+    m = L.shape[0]
+    T = x.shape[0]
+    if not adjoint:
+        u = np.einsum("kji,tki->tkj", R, x.reshape(T, m, m))           # step 1
+        return np.einsum("jlk,tkj->tlj", L, u).reshape(T, m * m)       # steps 2-3
+    du = np.einsum("jlk,tlj->tkj", L.conj(), x.reshape(T, m, m))       # adjoint of steps 2-3
+    return np.einsum("kji,tkj->tki", R.conj(), du).reshape(T, m * m)   # adjoint of step 1
+
+
+def dft_factors(m: int):
+    """Complex Monarch factors with M = F_n P (F_n the n-point DFT matrix, omega = exp(-2 pi i / n)): the
+    Cooley-Tukey split f = f1 m + f0, s = s1 m + s0 gives L_j = F_m and R_k = diag(omega_n^{j k}) F_m."""
+    n = m * m
+    a = np.arange(m)
+    Fm = np.exp(-2j * np.pi * np.outer(a, a) / m)
+    L = np.stack([Fm] * m)
+    R = np.stack([np.exp(-2j * np.pi * a * k / n)[:, None] * Fm for k in range(m)])
+    return L, R
+
+
 def project(A, m: int):
     """Algorithm 1: closest Monarch matrix to a dense A in Frobenius norm.
 

@@ -474,3 +474,42 @@ def test_rect_kronecker_closed_form():
     y = O.rect_fwd(x, np.stack([np.eye(3)] * 4), np.stack([np.eye(4)] * 3))
     assert np.allclose(y, x)
     assert y.shape == (6, n)
+
+
+# ------------------------------------------------------------------ complex factors (Section 3.2: FFT, MM*)
+
+def _crand(rng, *shape):
+    return rng.standard_normal(shape) + 1j * rng.standard_normal(shape)
+
+
+@pytest.mark.parametrize("m", [2, 3, 4])
+def test_cplx_routes_agree_and_reduce_to_real(m):
+    rng = np.random.default_rng(41)
+    n = m * m
+    L, R, x = _crand(rng, m, m, m), _crand(rng, m, m, m), _crand(rng, 5, n)
+    M = O.cplx_dense_from_definition(L, R)
+    assert np.allclose(O.cplx_fwd(x, L, R), x @ M.T, atol=1e-12)
+    assert np.allclose(O.cplx_fwd(x, L, R, adjoint=True), x @ M.conj(), atol=1e-12)      # rows of x times M^H^T
+    # real data through the complex route equals the (pinned) real oracle
+    assert np.allclose(O.cplx_fwd(x.real, L.real, R.real).real, O.fwd(x.real, L.real, R.real), atol=1e-12)
+    assert np.allclose(O.cplx_fwd(x.real, L.real, R.real, adjoint=True).real,
+                       O.bwd(x.real, x.real, L.real, R.real, want=("dx",))["dx"], atol=1e-12)
+    # <M x, y> = <x, M^H y>
+    y = _crand(rng, 5, n)
+    lhs = np.sum(O.cplx_fwd(x, L, R) * y.conj())
+    rhs = np.sum(x * O.cplx_fwd(y, L, R, adjoint=True).conj())
+    assert np.isclose(lhs, rhs, rtol=1e-12)
+
+
+@pytest.mark.parametrize("m", [2, 4, 8])
+def test_dft_is_monarch(m):
+    # Section 3.2: the DFT matrix (times the stated permutation) is a Monarch matrix; numpy.fft is the pin
+    rng = np.random.default_rng(42)
+    n = m * m
+    L, R = O.dft_factors(m)
+    x = _crand(rng, 3, n)
+    xp = x.reshape(3, m, m).transpose(0, 2, 1).reshape(3, n)              # P x
+    assert np.allclose(O.cplx_fwd(xp, L, R), np.fft.fft(x, axis=1), atol=1e-10)
+    # F_n F_n^H = n I: the MM* product of the DFT factors with themselves
+    z = O.cplx_fwd(O.cplx_fwd(x, L, R, adjoint=True), L, R)
+    assert np.allclose(z, n * x, atol=1e-9)
