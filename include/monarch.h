@@ -67,7 +67,8 @@ typedef enum {
     MONARCH_OP_BWD_DW = 2,
     MONARCH_OP_MLP_FWD = 3,
     MONARCH_OP_BWD = 4, /* monarch_bwd: dx, dL and dR in one call */
-    MONARCH_OP_MLP_BWD = 5
+    MONARCH_OP_MLP_BWD = 5,
+    MONARCH_OP_CPLX = 6 /* monarch_cplx_fwd, either direction */
 } monarch_op_t;
 
 /* Which kernel family serves a call (process-wide; default AUTO). */
@@ -162,6 +163,20 @@ int monarch_rect_fwd(const void *x, const void *L, const void *R, void *y, int64
                      void *workspace, size_t workspace_bytes, void *stream);
 size_t monarch_rect_workspace_bytes(int64_t tokens, int32_t q, int32_t b1, int32_t b, int32_t r,
                                     int dtype);
+
+/* Complex Monarch multiply (Section 3.2: the DFT and the MM* products need
+ * complex factors):  y = M x  (adjoint == 0)  or  y = M^H x  (adjoint == 1),
+ * M = P L P^T R with complex blocks, M^H = R^H P L^H P.  An MM* product
+ * M1 M2^H x is two calls.  Complex tensors are PLANAR in the storage dtype:
+ * x, y: [2][tokens][n] (real plane, then imaginary plane); L, R: [2][m][m][m].
+ * The call runs four real Monarch multiplies over both planes at once
+ * (M(Lr,Rr), M(Li,Ri), M(Lr,Ri), M(Li,Rr) applied to [xr; xi]) and combines
+ * them:  Re M = M(Lr,Rr) - M(Li,Ri),  Im M = M(Lr,Ri) + M(Li,Rr); each of the
+ * four results is rounded to the storage dtype before the combination.
+ * Workspace: monarch_workspace_bytes with MONARCH_OP_CPLX. */
+int monarch_cplx_fwd(const void *x, const void *L, const void *R, void *y, int adjoint,
+                     int64_t tokens, int32_t n, int32_t m, int dtype,
+                     void *workspace, size_t workspace_bytes, void *stream);
 
 /* Dense materialisation by the entry formula, Eq. (2):
  *   M[l*m+j][k*m+i] = L[j][l][k] * R[k][j][i],   M: [n][n] row-major, storage dtype

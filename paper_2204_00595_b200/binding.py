@@ -10,7 +10,7 @@ import ctypes
 import os
 
 F32, BF16 = 0, 1
-OP_FWD, OP_BWD_DX, OP_BWD_DW, OP_MLP_FWD, OP_BWD, OP_MLP_BWD = 0, 1, 2, 3, 4, 5
+OP_FWD, OP_BWD_DX, OP_BWD_DW, OP_MLP_FWD, OP_BWD, OP_MLP_BWD, OP_CPLX = 0, 1, 2, 3, 4, 5, 6
 IMPL_AUTO, IMPL_STAGED, IMPL_FUSED = 0, 1, 2
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libmonarch.so")
@@ -28,6 +28,7 @@ _SIGNATURES = {
     "monarch_mlp_bwd": (_int, [_vp] * 14 + [_int, _i64, _i32, _i32, _int, _vp, _sz, _vp]),
     "monarch_rect_fwd": (_int, [_vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32, _int, _vp, _sz, _vp]),
     "monarch_rect_workspace_bytes": (_sz, [_i64, _i32, _i32, _i32, _i32, _int]),
+    "monarch_cplx_fwd": (_int, [_vp, _vp, _vp, _vp, _int, _i64, _i32, _i32, _int, _vp, _sz, _vp]),
     "monarch_dense": (_int, [_vp, _vp, _vp, _i32, _i32, _int, _vp]),
     "monarch_project": (_int, [_vp, _vp, _vp, _i32, _i32, _int, _vp, _vp]),
     "monarch_workspace_bytes": (_sz, [_int, _i64, _i32, _i32, _int]),
@@ -236,6 +237,14 @@ def monarch_rect_fwd(x, L, R, y, tokens, q, b1, b, r, workspace, stream=None) ->
     p, nb = _ws(workspace)
     _check(lib().monarch_rect_fwd(_ptr(x, "x"), _ptr(L, "L", dt), _ptr(R, "R", dt), _ptr(y, "y", dt), tokens,
                                   q, b1, b, r, _dtype_code(x), p, nb, _stream(stream)), "monarch_rect_fwd")
+
+
+def monarch_cplx_fwd(x, L, R, y, adjoint, tokens, n, m, workspace, stream=None) -> None:
+    """Complex multiply on planar tensors: x, y [2, tokens, n]; L, R [2, m, m, m]; adjoint=1 applies M^H."""
+    dt = x.dtype
+    p, b = _ws(workspace)
+    _check(lib().monarch_cplx_fwd(_ptr(x, "x"), _ptr(L, "L", dt), _ptr(R, "R", dt), _ptr(y, "y", dt), int(adjoint),
+                                  tokens, n, m, _dtype_code(x), p, b, _stream(stream)), "monarch_cplx_fwd")
 
 
 def monarch_dense(L, R, M, n, m, stream=None) -> None:

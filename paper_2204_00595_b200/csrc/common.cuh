@@ -168,6 +168,9 @@ int mlp_act(const void *a, const void *b1, void *h, int64_t tokens, int n, int d
 // dh <- dh * GELU'(a (+ b1)) in place, db1 += column sums of the result, db2 += column sums of dy
 int mlp_dact(void *dh, const void *a, const void *b1, const void *dy, float *db1, float *db2, int64_t tokens, int n,
              int dtype, cudaStream_t s);
+// combination step of the complex multiply (planar tensors, plane_elems = tokens * n)
+int cplx_combine(const void *A, const void *B, const void *C, const void *D, void *y, int64_t plane_elems, int adjoint,
+                 int dtype, cudaStream_t s);
 // fold the status word of an inner workspace into the outer one and clear it
 int merge_status(unsigned *outer, unsigned *inner, cudaStream_t s);
 

@@ -136,6 +136,33 @@ mlp_dact_kernel(T *__restrict__ dh, const T *__restrict__ a, const T *__restrict
     }
 }
 
+// Combination step of the complex multiply: with A, B, C, D = M(Lr,Rr), M(Li,Ri), M(Lr,Ri), M(Li,Rr) applied to
+// the stacked planes [xr; xi] (each [2][plane] elements),
+//   y_re = A[0] - B[0] + sgn (C[1] + D[1]),   y_im = A[1] - B[1] - sgn (C[0] + D[0]),
+// sgn = -1 for y = M x and +1 for y = M^H x.
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+cplx_combine_kernel(const T *__restrict__ A, const T *__restrict__ B, const T *__restrict__ C, const T *__restrict__ D,
+                    T *__restrict__ y, long long plane_vecs, float sgn)
+{
+    constexpr int V = vec16<T>::kElems;
+    for (long long i = (long long)blockIdx.x * kThreads + threadIdx.x; i < plane_vecs; i += (long long)gridDim.x * kThreads) {
+        float a0[V], a1[V], b0[V], b1[V], c0[V], c1[V], d0[V], d1[V], re[V], im[V];
+        const long long o0 = i * V, o1 = (plane_vecs + i) * V;
+        vec16<T>::load(A + o0, a0); vec16<T>::load(A + o1, a1);
+        vec16<T>::load(B + o0, b0); vec16<T>::load(B + o1, b1);
+        vec16<T>::load(C + o0, c0); vec16<T>::load(C + o1, c1);
+        vec16<T>::load(D + o0, d0); vec16<T>::load(D + o1, d1);
+#pragma unroll
+        for (int e = 0; e < V; ++e) {
+            re[e] = (a0[e] - b0[e]) + sgn * (c1[e] + d1[e]);
+            im[e] = (a1[e] - b1[e]) - sgn * (c0[e] + d0[e]);
+        }
+        vec16<T>::store(y + o0, re);
+        vec16<T>::store(y + o1, im);
+    }
+}
+
 __global__ void merge_status_kernel(unsigned *outer, unsigned *inner)
 {
     const unsigned v = *inner;
@@ -189,6 +216,26 @@ int mlp_dact(void *dh, const void *a, const void *b1, const void *dy, float *db1
 {
     return dtype == MONARCH_F32 ? dact_t<float>(dh, a, b1, dy, db1, db2, tokens, n, s)
                                 : dact_t<__nv_bfloat16>(dh, a, b1, dy, db1, db2, tokens, n, s);
+}
+
+int cplx_combine(const void *A, const void *B, const void *C, const void *D, void *y, int64_t plane_elems, int adjoint,
+                 int dtype, cudaStream_t s)
+{
+    if (plane_elems == 0) return MONARCH_OK;
+    const float sgn = adjoint ? 1.0f : -1.0f;
+    const long long vecs = plane_elems / (dtype == MONARCH_F32 ? 4 : 8);
+    long long blocks = (vecs + kThreads - 1) / kThreads;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (dtype == MONARCH_F32)
+        cplx_combine_kernel<float><<<(unsigned)blocks, kThreads, 0, s>>>((const float *)A, (const float *)B, (const float *)C,
+                                                                        (const float *)D, (float *)y, vecs, sgn);
+    else
+        cplx_combine_kernel<__nv_bfloat16><<<(unsigned)blocks, kThreads, 0, s>>>(
+            (const __nv_bfloat16 *)A, (const __nv_bfloat16 *)B, (const __nv_bfloat16 *)C, (const __nv_bfloat16 *)D,
+            (__nv_bfloat16 *)y, vecs, sgn);
+    note_launch();
+    MONARCH_CUDA_TRY(cudaGetLastError());
+    return MONARCH_OK;
 }
 
 int merge_status(unsigned *outer, unsigned *inner, cudaStream_t s)

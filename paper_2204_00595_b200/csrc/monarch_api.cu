@@ -136,8 +136,15 @@ extern "C" {
 
 size_t monarch_workspace_bytes(int op, int64_t tokens, int32_t n, int32_t m, int dtype)
 {
-    if (op < MONARCH_OP_FWD || op > MONARCH_OP_MLP_BWD) return 0;
+    if (op < MONARCH_OP_FWD || op > MONARCH_OP_CPLX) return 0;
     if (check_shape(tokens, n, m, dtype) != MONARCH_OK) return 0;
+    if (op == MONARCH_OP_CPLX) {
+        // [inner workspace for 2 * tokens rows][four results of 2 * tokens rows]
+        const size_t f = monarch_workspace_bytes(MONARCH_OP_FWD, 2 * tokens, n, m, dtype);
+        const size_t b = monarch_workspace_bytes(MONARCH_OP_BWD_DX, 2 * tokens, n, m, dtype);
+        if (f == 0 || b == 0) return 0;
+        return round256(f > b ? f : b) + 4 * round256((size_t)2 * tokens * n * esize(dtype));
+    }
     if (op == MONARCH_OP_MLP_BWD) {
         const MlpBwdLayout lay = mlp_bwd_layout(tokens, n, m, dtype);
         return lay.ws_b == 0 || lay.ws_f == 0 ? 0 : lay.total;
@@ -347,6 +354,33 @@ int monarch_rect_fwd(const void *x, const void *L, const void *R, void *y, int64
     return rect_stage2_simt(u, L, y, tokens, q, b, r, dtype, s);
 }
 
+int monarch_cplx_fwd(const void *x, const void *L, const void *R, void *y, int adjoint, int64_t tokens,
+                     int32_t n, int32_t m, int dtype, void *workspace, size_t workspace_bytes, void *stream)
+{
+    MONARCH_TRY(check_shape(tokens, n, m, dtype));
+    if (adjoint != 0 && adjoint != 1) return MONARCH_ERR_INVALID_ARG;
+    const size_t es = esize(dtype), plane = (size_t)tokens * n * es, wplane = (size_t)n * m * es;
+    const Range in[] = {{x, 2 * plane}, {L, 2 * wplane}, {R, 2 * wplane}};
+    const Range out[] = {{y, 2 * plane}};
+    const size_t need = monarch_workspace_bytes(MONARCH_OP_CPLX, tokens, n, m, dtype);
+    MONARCH_TRY(check_buffers(in, 3, out, 1, workspace, workspace_bytes, need));
+    const size_t res = round256(2 * plane);
+    const size_t inner = need - 4 * res;
+    char *ws = (char *)workspace;
+    void *part[4] = {ws + inner, ws + inner + res, ws + inner + 2 * res, ws + inner + 3 * res};
+    const char *Lr = (const char *)L, *Li = Lr + wplane, *Rr = (const char *)R, *Ri = Rr + wplane;
+    const char *lsel[4] = {Lr, Li, Lr, Li}, *rsel[4] = {Rr, Ri, Ri, Rr};   // A, B, C, D
+    for (int c = 0; c < 4; ++c) {
+        // both planes at once: [xr; xi] is 2 * tokens rows
+        if (adjoint)
+            MONARCH_TRY(monarch_bwd_dx(x, lsel[c], rsel[c], part[c], 2 * tokens, n, m, dtype, ws, inner, stream));
+        else
+            MONARCH_TRY(monarch_fwd(x, lsel[c], rsel[c], part[c], 2 * tokens, n, m, dtype, ws, inner, stream));
+    }
+    return cplx_combine(part[0], part[1], part[2], part[3], y, (int64_t)tokens * n, adjoint, dtype,
+                        (cudaStream_t)stream);
+}
+
 int monarch_dense(const void *L, const void *R, void *M, int32_t n, int32_t m, int dtype, void *stream)
 {
     MONARCH_TRY(check_shape(0, n, m, dtype));
@@ -407,9 +441,10 @@ int monarch_set_impl(int impl)
 
 const char *monarch_impl_name(int op, int32_t m, int dtype)
 {
-    if (op < MONARCH_OP_FWD || op > MONARCH_OP_MLP_BWD) return "unsupported";
+    if (op < MONARCH_OP_FWD || op > MONARCH_OP_CPLX) return "unsupported";
     if (check_shape(0, m * m, m, dtype) != MONARCH_OK) return "unsupported";
     if (op == MONARCH_OP_MLP_BWD) op = MONARCH_OP_BWD;      // its Monarch passes are monarch_bwd's
+    if (op == MONARCH_OP_CPLX) op = MONARCH_OP_FWD;         // four real forward (or dx) passes
     const int which = pick(op, m, dtype);
     if (which == kSimt && op == MONARCH_OP_FWD && m == 16 &&
         g_impl.load(std::memory_order_relaxed) == MONARCH_IMPL_AUTO)

@@ -484,6 +484,65 @@ def test_rect_arguments(P):
     assert float(y.min()) == 3.0
 
 
+# ----------------------------------------------------------------- complex factors (planar tensors)
+
+def _planar(z, dtype):
+    """complex array -> float32 [2, ...] planes rounded to the storage dtype (and the complex value they hold)."""
+    planes = np.stack([round_to_storage(z.real.astype(np.float32), dtype),
+                       round_to_storage(z.imag.astype(np.float32), dtype)])
+    return planes, planes[0].astype(np.float64) + 1j * planes[1].astype(np.float64)
+
+
+@pytest.mark.parametrize("adjoint", [0, 1])
+@pytest.mark.parametrize("m,T,dtype", [(16, 37, "f32"), (32, 130, "f32"), (32, 65, "bf16"), (64, 129, "bf16"),
+                                       (128, 70, "bf16")])
+def test_cplx_fwd(P, impl, m, T, dtype, adjoint):
+    import torch
+    code = _code(P, dtype)
+    _skip_if_same_family(P, impl, P.OP_CPLX, m, code)
+    n = m * m
+    rng = np.random.default_rng(800 + m + T)
+    xp, xc = _planar(rng.standard_normal((T, n)) + 1j * rng.standard_normal((T, n)), dtype)
+    s = 1.0 / np.sqrt(2 * m)
+    Lp, Lc = _planar(s * (rng.standard_normal((m, m, m)) + 1j * rng.standard_normal((m, m, m))), dtype)
+    Rp, Rc = _planar(s * (rng.standard_normal((m, m, m)) + 1j * rng.standard_normal((m, m, m))), dtype)
+    x, L, R = to_device(xp, dtype), to_device(Lp, dtype), to_device(Rp, dtype)
+    yf, y = _guarded((2, T, n), _tdtype(dtype))
+    ws = P.Workspace(P.monarch_workspace_bytes(P.OP_CPLX, T, n, m, code))
+    P.monarch_cplx_fwd(x, L, R, y, adjoint, T, n, m, ws)
+    torch.cuda.synchronize()
+    assert P.monarch_last_device_status(ws) == 0
+    ref = O.cplx_fwd(xc, Lc, Rc, adjoint=bool(adjoint))
+    yh = to_host64(y)
+    # a problem instance is a token's complex row: compare re and im side by side
+    assert_close(np.concatenate([yh[0], yh[1]], axis=1), np.concatenate([ref.real, ref.imag], axis=1), dtype,
+                 f"complex y adjoint={adjoint}", scale=1.5 if dtype == "bf16" else 1.0)
+    _check_guard(yf, "complex y")
+
+
+def test_cplx_dft_closed_form(P):
+    """Section 3.2: with the Cooley-Tukey factors the multiply is the DFT of the permuted input; numpy.fft is
+    the reference, independent of the oracle's loops."""
+    import torch
+    m, T = 16, 33
+    n = m * m
+    rng = np.random.default_rng(816)
+    Lc, Rc = O.dft_factors(m)
+    Lp, _ = _planar(Lc, "f32")
+    Rp, _ = _planar(Rc, "f32")
+    xp, xc = _planar(rng.standard_normal((T, n)) + 1j * rng.standard_normal((T, n)), "f32")
+    xperm = xc.reshape(T, m, m).transpose(0, 2, 1).reshape(T, n)                   # P x
+    xpp, _ = _planar(xperm, "f32")
+    y = torch.empty(2, T, n, device="cuda")
+    ws = P.Workspace(P.monarch_workspace_bytes(P.OP_CPLX, T, n, m, P.F32))
+    P.monarch_cplx_fwd(to_device(xpp, "f32"), to_device(Lp, "f32"), to_device(Rp, "f32"), y, 0, T, n, m, ws)
+    torch.cuda.synchronize()
+    ref = np.fft.fft(xc, axis=1)
+    yh = to_host64(y)
+    assert_close(np.concatenate([yh[0], yh[1]], axis=1), np.concatenate([ref.real, ref.imag], axis=1), "f32",
+                 "DFT", scale=3.0)          # the factors themselves are rounded to fp32 (1e-7 each, n terms)
+
+
 # ----------------------------------------------------------------- dense <-> factors (Eq. 2, Algorithm 1)
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
