@@ -37,9 +37,10 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=3, choices=[1, 2, 3, 4, 5, 6, 7],
+    ap.add_argument("--workload", type=int, default=3, choices=[1, 2, 3, 4, 5, 6, 7, 8],
                     help="1-5: the square workloads; 6: the general (rectangular) class, forward only; "
-                         "7: projection of a dense matrix onto the Monarch class + dense materialisation")
+                         "7: projection of a dense matrix onto the Monarch class + dense materialisation; "
+                         "8: complex multiply (planar), y = M x then z = M^H y")
     ap.add_argument("--kernels", default="auto", choices=["auto", "staged", "fused"])
     ap.add_argument("--calls", default="", help="comma-separated subset of the workload's calls "
                     "(profiling aid; the default step runs them all)")
@@ -416,8 +417,132 @@ def main_project(args):
     return 0
 
 
+def main_cplx(args):
+    """Workload 8: complex Monarch multiply on planar bf16 tensors, n = 4096, m = 64, 8192 tokens: y = M x followed by
+    z = M^H y (the two halves of an MM* product).  Algorithmic work per call: 16 n m FLOP per token (a complex
+    multiply-add is four real ones) and 2 x 2 n s bytes (two planes in, two out)."""
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    import numpy as np
+    m, n, T = 64, 4096, 8192
+    flops = 2 * 16 * n * m * T
+    nbytes = 2 * (4 * T * n * 2 + 4 * n * m * 2)
+    workload = f"workload 8: cplx_fwd + adjoint bf16 (planar) n={n} m={m} tokens/GPU={T}"
+    metric, unit = "monarch_cplx_tflops", "TFLOP/s"
+    rng = np.random.default_rng(595008)
+
+    def draw(shape, std):
+        from paper_2204_00595_b200.inputs import round_to_storage
+        return round_to_storage(rng.standard_normal(shape, dtype=np.float32) * np.float32(std), "bf16")
+
+    x = draw((2, T, n), 1.0)
+    L, R = draw((2, m, m, m), 1.0 / np.sqrt(2 * m)), draw((2, m, m, m), 1.0 / np.sqrt(2 * m))
+
+    def time_oracle_cplx(target_s):
+        from oracle import monarch_oracle as O
+        Lc, Rc = L[0] + 1j * L[1], R[0] + 1j * R[1]
+        Ts = 8
+        while True:
+            xc = x[0, :Ts] + 1j * x[1, :Ts]
+            t0 = time.perf_counter()
+            O.cplx_fwd(O.cplx_fwd(xc, Lc, Rc), Lc, Rc, adjoint=True)
+            dt = time.perf_counter() - t0
+            if dt >= target_s / 4 or Ts >= T:
+                break
+            Ts = min(T, Ts * 4)
+        return {"tflops": flops * Ts / T / dt / 1e12, "tokens": Ts, "seconds": dt, "cores": os.cpu_count()}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        rs = [time_oracle_cplx(8.0) for _ in range(args.warmup + args.steps)][args.warmup:]
+        tfl = statistics.mean(r["tflops"] for r in rs)
+        print(json.dumps({
+            "impl": "reference", "metric": metric, "value": tfl, "unit": unit, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": statistics.mean(r["seconds"] for r in rs) * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "c128", "data": "synthetic",
+            "config": {"workload": workload, "sample_tokens_per_step": rs[-1]["tokens"]},
+            "cpu_baseline": {"value": tfl, "unit": unit, "cores": rs[-1]["cores"], "kind": "oracle",
+                             "sample": f"{rs[-1]['tokens']} tokens of the workload per step (numpy einsum)"},
+            "e2e": {"value": tfl, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+        return 0
+
+    import torch
+    import __graft_entry__ as entry
+    entry.build()
+    import paper_2204_00595_b200 as P
+    from tests.helpers import to_device
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dx, dL, dR = to_device(x, "bf16"), to_device(L, "bf16"), to_device(R, "bf16")
+    y, z = torch.empty_like(dx), torch.empty_like(dx)
+    ws = P.Workspace(P.monarch_workspace_bytes(P.OP_CPLX, T, n, m, P.BF16))
+    stream = torch.cuda.current_stream()
+
+    def step():
+        P.monarch_cplx_fwd(dx, dL, dR, y, 0, T, n, m, ws)
+        P.monarch_cplx_fwd(y, dL, dR, z, 1, T, n, m, ws)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = P.monarch_launch_count()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0.record(stream)
+    for _ in range(args.steps):
+        step()
+    t1.record(stream)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    total_ms = t0.elapsed_time(t1)
+    clocks = sampler.stop()
+    launches = P.monarch_launch_count() - launches0
+    status = P.monarch_last_device_status(ws)
+    if dist is not None:
+        tmax = torch.tensor([total_ms], device="cuda")
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        total_ms = float(tmax.item())
+    ms = total_ms / args.steps
+    peaks = load_peaks()
+    line = {
+        "metric": metric, "value": flops * world / (ms * 1e-3) / 1e12, "unit": unit, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "tokens_per_s": T * world / (ms * 1e-3),
+        "config": {"workload": workload, "l2": "each call streams > 1 GB of planes and partial results",
+                   "device_status": status},
+        "clocks": clocks, "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "kernel": "per call: 4 x fused_fwd_m64_team_kernel (or fused_bwd_dx_m64_kernel) "
+                                               "on 2 x tokens rows + cplx_combine_kernel",
+                     "achieved": nbytes / ms / 1e6, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": nbytes / ms / 1e6 / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": None,
+                     "algorithmic_mb": nbytes / 1e6},
+        "e2e": None,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        rr = time_oracle_cplx(12.0)
+        line["cpu_baseline"] = {"value": rr["tflops"], "unit": unit, "cores": rr["cores"], "kind": "oracle",
+                                "sample": f"first {rr['tokens']} tokens of the workload, {rr['seconds']:.1f} s"}
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
 def main():
     args = parse_args()
+    if args.workload == 8:
+        return main_cplx(args)
     if args.workload == 6:
         return main_rect(args)
     if args.workload == 7:
