@@ -1,7 +1,7 @@
 // Elementwise kernels that sit between the Monarch passes of the composite calls: the combination step of the
-// complex multiply (at the end of this file) and the steps of the feed-forward block's backward pass (Section 4: the block is trained by the chain
-// rule through a = M1 x + b1, h = GELU(a), y = M2 h + b2).  The two Monarch backward passes are the ordinary
-// monarch_bwd kernels; this file holds what sits between them:
+// complex multiply (further down) and the steps of the feed-forward block's backward pass (Section 4: the block
+// is trained by the chain rule through a = M1 x + b1, h = GELU(a), y = M2 h + b2).  The two Monarch backward
+// passes are the ordinary monarch_bwd kernels; this file holds what sits between them:
 //   mlp_act:   h = GELU(a)                                   (a recomputed by a forward pass of M1)
 //   mlp_dact:  da = dh * GELU'(a),  db1 += sum_t da,  db2 += sum_t dy
 // Both are pure streaming kernels (16-byte accesses, one pass over their operands).
