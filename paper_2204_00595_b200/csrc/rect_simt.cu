@@ -285,6 +285,77 @@ int stage2_small4(const void *u, const void *Lp, void *y, long long tokens, int 
     return MONARCH_OK;
 }
 
+// Stage 2 when L's blocks are at most 16 x 16:  y[t][l*b + j] = sum_k Lp[j][l][k] u[t][k*b + j].  A CTA owns 64
+// columns j and keeps their blocks in shared memory as ws[l][k][j] (so that neighbouring threads read neighbouring
+// words); a thread owns one column and walks a slab of tokens two at a time, so that every weight it reads is used
+// twice.  The thread-per-(token, block) kernel above re-reads a block's q*r weights from global memory for every
+// token, one 2-byte load each.
+constexpr int kS2mCols = 64, kS2mLanes = 4;
+
+template <typename T>
+__global__ void __launch_bounds__(kS2mCols * kS2mLanes)
+stage2_medium_kernel(const T *__restrict__ u, const T *__restrict__ Lp, T *__restrict__ y, long long tokens, int q, int b,
+                     int r, int tokens_per_slab)
+{
+    extern __shared__ unsigned char s2m_raw[];
+    T *ws = reinterpret_cast<T *>(s2m_raw);                       // [r][q][64]
+    const int j0 = blockIdx.x * kS2mCols;
+    for (int i = threadIdx.x; i < r * q * kS2mCols; i += kS2mCols * kS2mLanes) {
+        const int jl = i / (r * q), lk = i % (r * q);               // global order: [j][l][k]
+        ws[lk * kS2mCols + jl] = j0 + jl < b ? Lp[((size_t)(j0 + jl)) * r * q + lk] : T(0.0f);
+    }
+    __syncthreads();
+    const int jl = threadIdx.x % kS2mCols, tl = threadIdx.x / kS2mCols;
+    if (j0 + jl >= b) return;
+    const long long t0 = (long long)blockIdx.y * tokens_per_slab;
+    const long long t1 = t0 + tokens_per_slab < tokens ? t0 + tokens_per_slab : tokens;
+    for (long long ta = t0 + tl; ta < t1; ta += 2 * kS2mLanes) {
+        const long long tb = ta + kS2mLanes;
+        const bool two = tb < t1;
+        float va[16], vb[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            va[k] = k < q ? elem<T>::load(u + (size_t)ta * q * b + (size_t)k * b + j0 + jl) : 0.0f;
+            vb[k] = (k < q && two) ? elem<T>::load(u + (size_t)tb * q * b + (size_t)k * b + j0 + jl) : 0.0f;
+        }
+        for (int l = 0; l < r; ++l) {
+            float xa = 0.0f, xb = 0.0f;
+#pragma unroll
+            for (int k = 0; k < 16; ++k)
+                if (k < q) {
+                    const float w = elem<T>::load(ws + (l * q + k) * kS2mCols + jl);
+                    xa = fmaf(w, va[k], xa);
+                    xb = fmaf(w, vb[k], xb);
+                }
+            elem<T>::store(y + (size_t)ta * r * b + (size_t)l * b + j0 + jl, xa);
+            if (two) elem<T>::store(y + (size_t)tb * r * b + (size_t)l * b + j0 + jl, xb);
+        }
+    }
+}
+
+template <typename T>
+int stage2_medium(const void *u, const void *Lp, void *y, long long tokens, int q, int b, int r, cudaStream_t s)
+{
+    const int cx = (b + kS2mCols - 1) / kS2mCols;
+    long long slabs = (148 * 8 + cx - 1) / cx;
+    if (slabs > (tokens + 7) / 8) slabs = (tokens + 7) / 8;
+    const int per = (int)((tokens + slabs - 1) / slabs);
+    slabs = (tokens + per - 1) / per;
+    if (slabs > 65535) return MONARCH_ERR_UNSUPPORTED;
+    const int smem = r * q * kS2mCols * (int)sizeof(T);           // at most 64 KB (fp32, 16 x 16)
+    static bool attr = false;
+    if (!attr) {
+        MONARCH_CUDA_TRY(cudaFuncSetAttribute(stage2_medium_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              16 * 16 * kS2mCols * (int)sizeof(T)));
+        attr = true;
+    }
+    stage2_medium_kernel<T><<<dim3((unsigned)cx, (unsigned)slabs), kS2mCols * kS2mLanes, smem, s>>>(
+        (const T *)u, (const T *)Lp, (T *)y, tokens, q, b, r, per);
+    note_launch();
+    MONARCH_CUDA_TRY(cudaGetLastError());
+    return MONARCH_OK;
+}
+
 template <typename T>
 int block_product(const void *in, const void *W, void *out, const BlockProduct &p, cudaStream_t s)
 {
@@ -325,10 +396,14 @@ int rect_stage2_simt(const void *u, const void *Lp, void *y, int64_t tokens, int
 {
     const BlockProduct s2 = {tokens, b, r, q, q * b, r * b, 1, b, 1, b};
     const bool small4 = q <= 4 && r <= 4 && b % 2 == 0 && tokens > 0;
+    const bool medium = !small4 && q <= 16 && r <= 16 && b >= 32 && tokens > 0;
     if (dtype == MONARCH_F32)
-        return small4 ? stage2_small4<float>(u, Lp, y, tokens, q, b, r, s) : block_product<float>(u, Lp, y, s2, s);
-    return small4 ? stage2_small4<__nv_bfloat16>(u, Lp, y, tokens, q, b, r, s)
-                  : block_product<__nv_bfloat16>(u, Lp, y, s2, s);
+        return small4   ? stage2_small4<float>(u, Lp, y, tokens, q, b, r, s)
+               : medium ? stage2_medium<float>(u, Lp, y, tokens, q, b, r, s)
+                        : block_product<float>(u, Lp, y, s2, s);
+    return small4   ? stage2_small4<__nv_bfloat16>(u, Lp, y, tokens, q, b, r, s)
+           : medium ? stage2_medium<__nv_bfloat16>(u, Lp, y, tokens, q, b, r, s)
+                    : block_product<__nv_bfloat16>(u, Lp, y, s2, s);
 }
 
 }  // namespace monarch

@@ -397,6 +397,8 @@ RECT_CASES = [
     (4, 256, 256, 4, 200), (256, 4, 4, 256, 131), (8, 48, 80, 24, 90), (3, 5, 7, 2, 33), (2, 8, 6, 4, 50),
     # bf16 with b1 and b multiples of 64: stage 1 on the tensor cores (128- and 64-wide output tiles, K = 64..1024)
     (2, 128, 192, 3, 300), (3, 64, 128, 5, 1), (4, 1024, 1024, 4, 140), (1, 320, 448, 2, 513), (6, 192, 64, 7, 128),
+    # L's blocks between 4 x 4 and 16 x 16: the shared-memory stage-2 kernel
+    (16, 256, 256, 16, 70), (12, 8, 64, 5, 40), (5, 64, 128, 16, 33),
 ]
 
 
