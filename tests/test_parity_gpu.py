@@ -399,6 +399,8 @@ RECT_CASES = [
     (2, 128, 192, 3, 300), (3, 64, 128, 5, 1), (4, 1024, 1024, 4, 140), (1, 320, 448, 2, 513), (6, 192, 64, 7, 128),
     # L's blocks between 4 x 4 and 16 x 16: the shared-memory stage-2 kernel
     (16, 256, 256, 16, 70), (12, 8, 64, 5, 40), (5, 64, 128, 16, 33),
+    # the TMA-fed stage 2 at its edges: one token, a ragged tile, many slabs
+    (2, 64, 256, 3, 1), (4, 64, 256, 4, 17), (3, 64, 512, 4, 20011),
 ]
 
 
