@@ -327,3 +327,74 @@ int oracle_rect_fwd(const double *x, const double *Lp, const double *R, double *
     }
     return fail;
 }
+
+/* Gradients of  f = <dy, L R x>  for the general (rectangular) class above - the
+ * adjoints of its two steps (the paper trains these layers by automatic
+ * differentiation, Section 4):
+ *   du[k*b + j]   = sum_l Lp[j][l][k] dy[l*b + j]
+ *   dx[k*b1 + i]  = sum_j R[k][j][i]  du[k*b + j]
+ *   dLp[j][l][k]  = sum_t dy[t][l*b + j] u[t][k*b + j]
+ *   dR[k][j][i]   = sum_t du[t][k*b + j] x[t][k*b1 + i]
+ * Any of dx, dLp, dR may be NULL; dLp and dR are overwritten. */
+int oracle_rect_bwd(const double *x, const double *dy, const double *Lp, const double *R,
+                    double *dx, double *dLp, double *dR, long T, int q, int b1, int b, int r)
+{
+    const size_t n1 = (size_t)q * b1, n2 = (size_t)q * b, n3 = (size_t)r * b;
+    double *u = (double *)malloc(((size_t)T * n2 + 1) * sizeof(double));
+    double *du = (double *)malloc(((size_t)T * n2 + 1) * sizeof(double));
+    if (!u || !du) {
+        free(u);
+        free(du);
+        return 1;
+    }
+#pragma omp parallel for schedule(static)
+    for (long t = 0; t < T; ++t) {
+        const double *xt = x + (size_t)t * n1, *dyt = dy + (size_t)t * n3;
+        double *ut = u + (size_t)t * n2, *dut = du + (size_t)t * n2;
+        for (int k = 0; k < q; ++k)
+            for (int j = 0; j < b; ++j) {
+                double acc = 0.0, dacc = 0.0;
+                for (int i = 0; i < b1; ++i)
+                    acc += R[((size_t)k * b + j) * b1 + i] * xt[(size_t)k * b1 + i];
+                for (int l = 0; l < r; ++l)
+                    dacc += Lp[((size_t)j * r + l) * q + k] * dyt[(size_t)l * b + j];
+                ut[(size_t)k * b + j] = acc;
+                dut[(size_t)k * b + j] = dacc;
+            }
+        if (dx) {
+            double *dxt = dx + (size_t)t * n1;
+            for (int k = 0; k < q; ++k)
+                for (int i = 0; i < b1; ++i) {
+                    double acc = 0.0;
+                    for (int j = 0; j < b; ++j)
+                        acc += R[((size_t)k * b + j) * b1 + i] * dut[(size_t)k * b + j];
+                    dxt[(size_t)k * b1 + i] = acc;
+                }
+        }
+    }
+    if (dLp) {
+#pragma omp parallel for schedule(static)
+        for (int j = 0; j < b; ++j)
+            for (int l = 0; l < r; ++l)
+                for (int k = 0; k < q; ++k) {
+                    double acc = 0.0;
+                    for (long t = 0; t < T; ++t)
+                        acc += dy[(size_t)t * n3 + (size_t)l * b + j] * u[(size_t)t * n2 + (size_t)k * b + j];
+                    dLp[((size_t)j * r + l) * q + k] = acc;
+                }
+    }
+    if (dR) {
+#pragma omp parallel for schedule(static)
+        for (int k = 0; k < q; ++k)
+            for (int j = 0; j < b; ++j)
+                for (int i = 0; i < b1; ++i) {
+                    double acc = 0.0;
+                    for (long t = 0; t < T; ++t)
+                        acc += du[(size_t)t * n2 + (size_t)k * b + j] * x[(size_t)t * n1 + (size_t)k * b1 + i];
+                    dR[((size_t)k * b + j) * b1 + i] = acc;
+                }
+    }
+    free(u);
+    free(du);
+    return 0;
+}

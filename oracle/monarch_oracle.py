@@ -62,6 +62,8 @@ def _load():
         lib.oracle_mlp_fwd.argtypes = [dp] * 8 + [ctypes.c_long, ctypes.c_int]
         lib.oracle_rect_fwd.restype = ctypes.c_int
         lib.oracle_rect_fwd.argtypes = [dp] * 4 + [ctypes.c_long] + [ctypes.c_int] * 4
+        lib.oracle_rect_bwd.restype = ctypes.c_int
+        lib.oracle_rect_bwd.argtypes = [dp] * 7 + [ctypes.c_long] + [ctypes.c_int] * 4
         lib.oracle_mlp_bwd.restype = ctypes.c_int
         lib.oracle_mlp_bwd.argtypes = [dp] * 14 + [ctypes.c_long, ctypes.c_int]
         _lib = lib
@@ -189,6 +191,21 @@ def rect_fwd(x, Lp, R):
     if _load().oracle_rect_fwd(_p(x), _p(Lp), _p(R), _p(y), T, q, b1, b, r):
         raise MemoryError("oracle_rect_fwd")
     return y
+
+
+def rect_bwd(x, dy, Lp, R):
+    """Gradients of <dy, L R x> for the general (rectangular) class: dict with dx, dL (like Lp), dR."""
+    Lp = _f64(Lp); R = _f64(R)
+    q, b, b1 = R.shape
+    r = Lp.shape[1]
+    x = _f64(x); dy = _f64(dy); T = x.shape[0]
+    if x.shape != (T, q * b1) or dy.shape != (T, r * b) or Lp.shape != (b, r, q):
+        raise ValueError("shape mismatch")
+    out = {"dx": np.empty((T, q * b1)), "dL": np.empty((b, r, q)), "dR": np.empty((q, b, b1))}
+    if _load().oracle_rect_bwd(_p(x), _p(dy), _p(Lp), _p(R), _p(out["dx"]), _p(out["dL"]), _p(out["dR"]),
+                               T, q, b1, b, r):
+        raise MemoryError("oracle_rect_bwd")
+    return out
 
 
 # --------------------------------------------------------------------------

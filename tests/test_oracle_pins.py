@@ -513,3 +513,46 @@ def test_dft_is_monarch(m):
     # F_n F_n^H = n I: the MM* product of the DFT factors with themselves
     z = O.cplx_fwd(O.cplx_fwd(x, L, R, adjoint=True), L, R)
     assert np.allclose(z, n * x, atol=1e-9)
+
+
+@pytest.mark.parametrize("q,b1,b,r", [(2, 3, 4, 5), (4, 2, 3, 2), (3, 3, 3, 3), (1, 4, 2, 3)])
+def test_rect_gradients(q, b1, b, r):
+    rng = np.random.default_rng(35)
+    T = 4
+    R, Lp = _rand(rng, q, b, b1), _rand(rng, b, r, q)
+    x, dy = _rand(rng, T, q * b1), _rand(rng, T, r * b)
+    g = O.rect_bwd(x, dy, Lp, R)
+    # dx = M^T dy with M from the definitions' dense factors
+    Ld, Rd = O.rect_factors_from_definition(Lp, R)
+    assert np.allclose(g["dx"], dy @ (Ld @ Rd), atol=1e-12)
+    # central differences of f = <dy, L R x> in the parameters
+    args = {"L": Lp, "R": R}
+    h = 1e-6
+    for name, key in (("L", "dL"), ("R", "dR")):
+        v = args[name]
+        num = np.zeros_like(v)
+        it = np.nditer(v, flags=["multi_index"])
+        for _ in it:
+            idx = it.multi_index
+            keep = v[idx]
+            v[idx] = keep + h
+            fp = np.sum(dy * O.rect_fwd(x, args["L"], args["R"]))
+            v[idx] = keep - h
+            fm = np.sum(dy * O.rect_fwd(x, args["L"], args["R"]))
+            v[idx] = keep
+            num[idx] = (fp - fm) / (2 * h)
+        assert np.allclose(g[key], num, rtol=1e-7, atol=1e-7), name
+    # Euler identities (y is bilinear in the two factors) and the adjoint identity
+    s = np.sum(dy * O.rect_fwd(x, Lp, R))
+    assert np.isclose(np.sum(g["dL"] * Lp), s, rtol=1e-12) and np.isclose(np.sum(g["dR"] * R), s, rtol=1e-12)
+    assert np.isclose(np.sum(g["dx"] * x), s, rtol=1e-12)
+
+
+def test_rect_gradients_reduce_to_square():
+    rng = np.random.default_rng(36)
+    m, T = 4, 5
+    L, R = _rand(rng, m, m, m), _rand(rng, m, m, m)
+    x, dy = _rand(rng, T, m * m), _rand(rng, T, m * m)
+    g, ref = O.rect_bwd(x, dy, L, R), O.bwd(x, dy, L, R)
+    for k in ("dx", "dL", "dR"):
+        assert np.allclose(g[k], ref[k], atol=1e-12), k
