@@ -164,6 +164,23 @@ int monarch_rect_fwd(const void *x, const void *L, const void *R, void *y, int64
 size_t monarch_rect_workspace_bytes(int64_t tokens, int32_t q, int32_t b1, int32_t b, int32_t r,
                                     int dtype);
 
+/* Gradients of f = <dy, L R x> for the general class (adjoints of the two steps
+ * above; the paper trains these layers by automatic differentiation):
+ *   du[t][k*b + j]  = sum_l L[j][l][k] dy[t][l*b + j]
+ *   dx[t][k*b1 + i] = sum_j R[k][j][i] du[t][k*b + j]
+ *   dL[j][l][k] = sum_t dy[t][l*b + j] u[t][k*b + j],  dR[k][j][i] = sum_t du[t][k*b + j] x[t][k*b1 + i]
+ * with u recomputed inside.  x, dx: [tokens][q*b1]; dy: [tokens][r*b]; dL:
+ * float32 [b][r][q]; dR: float32 [q][b][b1]; accumulate == 0 overwrites the two
+ * weight gradients, 1 adds to them.  u and du are rounded to the storage dtype
+ * once; the sums over tokens use atomic adds (last bits may vary run to run).
+ * Workspace: monarch_rect_bwd_workspace_bytes. */
+int monarch_rect_bwd(const void *x, const void *dy, const void *L, const void *R,
+                     void *dx, float *dL, float *dR, int accumulate, int64_t tokens,
+                     int32_t q, int32_t b1, int32_t b, int32_t r, int dtype,
+                     void *workspace, size_t workspace_bytes, void *stream);
+size_t monarch_rect_bwd_workspace_bytes(int64_t tokens, int32_t q, int32_t b1, int32_t b,
+                                        int32_t r, int dtype);
+
 /* Complex Monarch multiply (Section 3.2: the DFT and the MM* products need
  * complex factors):  y = M x  (adjoint == 0)  or  y = M^H x  (adjoint == 1),
  * M = P L P^T R with complex blocks, M^H = R^H P L^H P.  An MM* product

@@ -145,18 +145,21 @@ const void *fused_fwd_m64_saved_u(const void *fwd_ws);
 
 // ---- general (rectangular) Monarch multiply on the CUDA cores (rect_simt.cu); workspace = [status][u] ----
 size_t rect_workspace_bytes(int64_t tokens, int q, int b, int dtype);
-int rect_stage1_simt(const void *x, const void *R, void *u, int64_t tokens, int q, int b1, int b, int dtype,
+// wt = 1 reads the blocks transposed (the adjoint passes of the backward call)
+int rect_stage1_simt(const void *x, const void *R, void *u, int64_t tokens, int q, int b1, int b, int dtype, int wt,
                      cudaStream_t s);
-int rect_stage2_simt(const void *u, const void *Lp, void *y, int64_t tokens, int q, int b, int r, int dtype,
+int rect_stage2_simt(const void *u, const void *Lp, void *y, int64_t tokens, int q, int b, int r, int dtype, int wt,
                      cudaStream_t s);
+int rect_wgrad_simt(const void *x, const void *dy, const void *u, const void *du, float *dL, float *dR, int64_t tokens,
+                    int q, int b1, int b, int r, int dtype, cudaStream_t s);
 // stage 1 on the tensor cores (rect_tc.cu): bf16, b1 and b multiples of 64
 bool rect_stage1_tc_available(int q, int b1, int b, int dtype);
 int rect_stage1_tc(const void *x, const void *R, void *u, int64_t tokens, int q, int b1, int b, unsigned *status,
                    cudaStream_t s);
 // stage 2 as a TMA-fed streaming pass (rect_tc.cu): bf16, q and r at most 4, b a multiple of 8 and at least 256
 bool rect_stage2_stream_available(int q, int b, int r, int dtype);
-int rect_stage2_stream(const void *u, const void *Lp, void *y, int64_t tokens, int q, int b, int r, unsigned *status,
-                       cudaStream_t s);
+int rect_stage2_stream(const void *u, const void *Lp, void *y, int64_t tokens, int q, int b, int r, int wt,
+                       unsigned *status, cudaStream_t s);
 
 // ---- dense <-> Monarch factors (project.cu): Eq. (2) and Algorithm 1 ----
 int dense_from_factors(const void *L, const void *R, void *M, int m, int dtype, cudaStream_t s);

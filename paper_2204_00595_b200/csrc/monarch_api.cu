@@ -348,10 +348,53 @@ int monarch_rect_fwd(const void *x, const void *L, const void *R, void *y, int64
     if (fast && rect_stage1_tc_available(q, b1, b, dtype))
         MONARCH_TRY(rect_stage1_tc(x, R, u, tokens, q, b1, b, status, s));
     else
-        MONARCH_TRY(rect_stage1_simt(x, R, u, tokens, q, b1, b, dtype, s));
+        MONARCH_TRY(rect_stage1_simt(x, R, u, tokens, q, b1, b, dtype, 0, s));
     if (fast && rect_stage2_stream_available(q, b, r, dtype))
-        return rect_stage2_stream(u, L, y, tokens, q, b, r, status, s);
-    return rect_stage2_simt(u, L, y, tokens, q, b, r, dtype, s);
+        return rect_stage2_stream(u, L, y, tokens, q, b, r, 0, status, s);
+    return rect_stage2_simt(u, L, y, tokens, q, b, r, dtype, 0, s);
+}
+
+size_t monarch_rect_bwd_workspace_bytes(int64_t tokens, int32_t q, int32_t b1, int32_t b, int32_t r, int dtype)
+{
+    if (check_rect(tokens, q, b1, b, r, dtype) != MONARCH_OK) return 0;
+    return MONARCH_STATUS_BYTES + 2 * round256((size_t)tokens * q * b * esize(dtype));      // [status][u][du]
+}
+
+int monarch_rect_bwd(const void *x, const void *dy, const void *L, const void *R, void *dx, float *dL, float *dR,
+                     int accumulate, int64_t tokens, int32_t q, int32_t b1, int32_t b, int32_t r, int dtype,
+                     void *workspace, size_t workspace_bytes, void *stream)
+{
+    MONARCH_TRY(check_rect(tokens, q, b1, b, r, dtype));
+    if (accumulate != 0 && accumulate != 1) return MONARCH_ERR_INVALID_ARG;
+    const size_t es = esize(dtype);
+    const size_t lb = (size_t)b * r * q, rb = (size_t)q * b * b1;
+    const Range in[] = {{x, (size_t)tokens * q * b1 * es}, {dy, (size_t)tokens * r * b * es}, {L, lb * es}, {R, rb * es}};
+    const Range out[] = {{dx, (size_t)tokens * q * b1 * es}, {dL, lb * sizeof(float)}, {dR, rb * sizeof(float)}};
+    MONARCH_TRY(check_buffers(in, 4, out, 3, workspace, workspace_bytes,
+                              monarch_rect_bwd_workspace_bytes(tokens, q, b1, b, r, dtype)));
+    cudaStream_t s = (cudaStream_t)stream;
+    if (!accumulate) {
+        MONARCH_CUDA_TRY(cudaMemsetAsync(dL, 0, lb * sizeof(float), s));
+        MONARCH_CUDA_TRY(cudaMemsetAsync(dR, 0, rb * sizeof(float), s));
+    }
+    if (tokens == 0) return MONARCH_OK;
+    unsigned *status = (unsigned *)workspace;
+    char *u = (char *)workspace + MONARCH_STATUS_BYTES;
+    char *du = u + round256((size_t)tokens * q * b * es);
+    const bool fast = g_impl.load(std::memory_order_relaxed) != MONARCH_IMPL_STAGED;
+    // u = blockdiag(R) x (recomputed: the forward call keeps nothing)
+    if (fast && rect_stage1_tc_available(q, b1, b, dtype))
+        MONARCH_TRY(rect_stage1_tc(x, R, u, tokens, q, b1, b, status, s));
+    else
+        MONARCH_TRY(rect_stage1_simt(x, R, u, tokens, q, b1, b, dtype, 0, s));
+    // du = L^T dy: stage 2 with the roles of q and r exchanged and the blocks read transposed
+    if (fast && rect_stage2_stream_available(r, b, q, dtype))
+        MONARCH_TRY(rect_stage2_stream(dy, L, du, tokens, r, b, q, 1, status, s));
+    else
+        MONARCH_TRY(rect_stage2_simt(dy, L, du, tokens, r, b, q, dtype, 1, s));
+    // dx = blockdiag(R)^T du: stage 1 with the roles of b1 and b exchanged and the blocks read transposed
+    MONARCH_TRY(rect_stage1_simt(du, R, dx, tokens, q, b, b1, dtype, 1, s));
+    return rect_wgrad_simt(x, dy, u, du, dL, dR, tokens, q, b1, b, r, dtype, s);
 }
 
 int monarch_cplx_fwd(const void *x, const void *L, const void *R, void *y, int adjoint, int64_t tokens,

@@ -17,6 +17,7 @@ struct BlockProduct {
     int nb, o, k;              // blocks, outputs and inputs per block
     int in_row, out_row;       // elements per token row
     int ibs, ies, obs, oes;    // block / element strides inside a row
+    int wt;                    // 0: W[blk][o][i];  1: the block is stored transposed, W[blk][i][o] (adjoint passes)
 };
 
 constexpr int kTT = 64, kOT = 64, kKC = 16;
@@ -46,7 +47,8 @@ block_product_tiled_kernel(const T *__restrict__ in, const T *__restrict__ W, T 
             float va = 0.0f, vb = 0.0f;
             if (t < p.tokens && k0 + kk < p.k)
                 va = elem<T>::load(in + (size_t)t * p.in_row + (size_t)blk * p.ibs + (size_t)(k0 + kk) * p.ies);
-            if (o0 + row < p.o && k0 + kk < p.k) vb = elem<T>::load(wb + (size_t)(o0 + row) * p.k + k0 + kk);
+            if (o0 + row < p.o && k0 + kk < p.k)
+                vb = elem<T>::load(wb + (p.wt ? (size_t)(k0 + kk) * p.o + o0 + row : (size_t)(o0 + row) * p.k + k0 + kk));
             As[kk][row] = va;
             Bs[kk][row] = vb;
         }
@@ -98,7 +100,7 @@ block_product_small_kernel(const T *__restrict__ in, const T *__restrict__ W, T 
             float acc = 0.0f;
 #pragma unroll
             for (int i = 0; i < kSmallMax; ++i)
-                if (i < p.k) acc = fmaf(elem<T>::load(wb + o * p.k + i), v[i], acc);
+                if (i < p.k) acc = fmaf(elem<T>::load(wb + (p.wt ? i * p.o + o : o * p.k + i)), v[i], acc);
             elem<T>::store(dst + (size_t)o * p.oes, acc);
         }
     }
@@ -127,7 +129,7 @@ template <> struct pair_io<__nv_bfloat16> {
 template <typename T>
 __global__ void __launch_bounds__(256)
 stage2_small4_kernel(const T *__restrict__ u, const T *__restrict__ Lp, T *__restrict__ y, long long tokens, int q,
-                     int b, int r, int tokens_per_slab)
+                     int b, int r, int tokens_per_slab, int wt)
 {
     const int j = (blockIdx.x * 256 + threadIdx.x) * 2;
     if (j >= b) return;
@@ -138,7 +140,8 @@ stage2_small4_kernel(const T *__restrict__ u, const T *__restrict__ Lp, T *__res
         for (int l = 0; l < 4; ++l)
 #pragma unroll
             for (int k = 0; k < 4; ++k)
-                w[jj][l][k] = (l < r && k < q) ? elem<T>::load(Lp + ((size_t)(j + jj) * r + l) * q + k) : 0.0f;
+                w[jj][l][k] = (l < r && k < q)
+                                  ? elem<T>::load(Lp + (size_t)(j + jj) * r * q + (wt ? k * r + l : l * q + k)) : 0.0f;
     const long long t0 = (long long)blockIdx.y * tokens_per_slab;
     const long long t1 = t0 + tokens_per_slab < tokens ? t0 + tokens_per_slab : tokens;
     constexpr int U = 2;                          // tokens per batch: all their loads are issued before any use
@@ -197,14 +200,14 @@ __device__ __forceinline__ float bf_at(const uint4 &v, int e)
 
 __global__ void __launch_bounds__(256, 2)
 stage2_small4_bf16_kernel(const __nv_bfloat16 *__restrict__ u, const __nv_bfloat16 *__restrict__ Lp,
-                          __nv_bfloat16 *__restrict__ y, long long tokens, int q, int b, int r, int tokens_per_slab)
+                          __nv_bfloat16 *__restrict__ y, long long tokens, int q, int b, int r, int tokens_per_slab, int wt)
 {
     __shared__ float4 ws[4][4][2][32];            // [l][k][half][lane]: columns 8 lane + 4 half + (0..3)
     const int j0 = blockIdx.x * kS2Cols;
     for (int i = threadIdx.x; i < 16 * kS2Cols; i += 256) {
         const int jl = i >> 4, l = (i >> 2) & 3, k = i & 3;
         float v = 0.0f;
-        if (j0 + jl < b && l < r && k < q) v = __bfloat162float(Lp[((size_t)(j0 + jl) * r + l) * q + k]);
+        if (j0 + jl < b && l < r && k < q) v = __bfloat162float(Lp[(size_t)(j0 + jl) * r * q + (wt ? k * r + l : l * q + k)]);
         reinterpret_cast<float *>(&ws[l][k][(jl >> 2) & 1][jl >> 3])[jl & 3] = v;
     }
     __syncthreads();
@@ -253,7 +256,7 @@ stage2_small4_bf16_kernel(const __nv_bfloat16 *__restrict__ u, const __nv_bfloat
 }
 
 template <typename T>
-int stage2_small4(const void *u, const void *Lp, void *y, long long tokens, int q, int b, int r, cudaStream_t s)
+int stage2_small4(const void *u, const void *Lp, void *y, long long tokens, int q, int b, int r, int wt, cudaStream_t s)
 {
     const int bx = (b / 2 + 255) / 256;
     long long slabs = (148 * 8 + bx - 1) / bx;
@@ -270,7 +273,7 @@ int stage2_small4(const void *u, const void *Lp, void *y, long long tokens, int 
             sl = (tokens + pt - 1) / pt;
             if (sl > 65535) return MONARCH_ERR_UNSUPPORTED;
             stage2_small4_bf16_kernel<<<dim3((unsigned)cx, (unsigned)sl), 256, 0, s>>>(
-                (const __nv_bfloat16 *)u, (const __nv_bfloat16 *)Lp, (__nv_bfloat16 *)y, tokens, q, b, r, pt);
+                (const __nv_bfloat16 *)u, (const __nv_bfloat16 *)Lp, (__nv_bfloat16 *)y, tokens, q, b, r, pt, wt);
             note_launch();
             MONARCH_CUDA_TRY(cudaGetLastError());
             return MONARCH_OK;
@@ -278,7 +281,7 @@ int stage2_small4(const void *u, const void *Lp, void *y, long long tokens, int 
     }
     {
         stage2_small4_kernel<T><<<dim3((unsigned)bx, (unsigned)slabs), 256, 0, s>>>((const T *)u, (const T *)Lp, (T *)y,
-                                                                                  tokens, q, b, r, per);
+                                                                                  tokens, q, b, r, per, wt);
     }
     note_launch();
     MONARCH_CUDA_TRY(cudaGetLastError());
@@ -295,14 +298,15 @@ constexpr int kS2mCols = 64, kS2mLanes = 4;
 template <typename T>
 __global__ void __launch_bounds__(kS2mCols * kS2mLanes)
 stage2_medium_kernel(const T *__restrict__ u, const T *__restrict__ Lp, T *__restrict__ y, long long tokens, int q, int b,
-                     int r, int tokens_per_slab)
+                     int r, int tokens_per_slab, int wt)
 {
     extern __shared__ unsigned char s2m_raw[];
     T *ws = reinterpret_cast<T *>(s2m_raw);                       // [r][q][64]
     const int j0 = blockIdx.x * kS2mCols;
     for (int i = threadIdx.x; i < r * q * kS2mCols; i += kS2mCols * kS2mLanes) {
-        const int jl = i / (r * q), lk = i % (r * q);               // global order: [j][l][k]
-        ws[lk * kS2mCols + jl] = j0 + jl < b ? Lp[((size_t)(j0 + jl)) * r * q + lk] : T(0.0f);
+        const int jl = i / (r * q), lk = i % (r * q);               // lk = l * q + k; stored [j][l][k], or [j][k][l] if wt
+        const int src = wt ? (lk % q) * r + lk / q : lk;
+        ws[lk * kS2mCols + jl] = j0 + jl < b ? Lp[((size_t)(j0 + jl)) * r * q + src] : T(0.0f);
     }
     __syncthreads();
     const int jl = threadIdx.x % kS2mCols, tl = threadIdx.x / kS2mCols;
@@ -334,7 +338,7 @@ stage2_medium_kernel(const T *__restrict__ u, const T *__restrict__ Lp, T *__res
 }
 
 template <typename T>
-int stage2_medium(const void *u, const void *Lp, void *y, long long tokens, int q, int b, int r, cudaStream_t s)
+int stage2_medium(const void *u, const void *Lp, void *y, long long tokens, int q, int b, int r, int wt, cudaStream_t s)
 {
     const int cx = (b + kS2mCols - 1) / kS2mCols;
     long long slabs = (148 * 8 + cx - 1) / cx;
@@ -350,7 +354,7 @@ int stage2_medium(const void *u, const void *Lp, void *y, long long tokens, int 
         attr = true;
     }
     stage2_medium_kernel<T><<<dim3((unsigned)cx, (unsigned)slabs), kS2mCols * kS2mLanes, smem, s>>>(
-        (const T *)u, (const T *)Lp, (T *)y, tokens, q, b, r, per);
+        (const T *)u, (const T *)Lp, (T *)y, tokens, q, b, r, per, wt);
     note_launch();
     MONARCH_CUDA_TRY(cudaGetLastError());
     return MONARCH_OK;
@@ -384,26 +388,172 @@ size_t rect_workspace_bytes(int64_t tokens, int q, int b, int dtype)
     return MONARCH_STATUS_BYTES + (((size_t)tokens * q * b * es + 255) & ~(size_t)255);
 }
 
-int rect_stage1_simt(const void *x, const void *R, void *u, int64_t tokens, int q, int b1, int b, int dtype,
+// wt = 0: u = blockdiag(R) x.  wt = 1: the adjoint, dx = blockdiag(R)^T du (pass du as x; b1 and b swap roles).
+int rect_stage1_simt(const void *x, const void *R, void *u, int64_t tokens, int q, int b1, int b, int dtype, int wt,
                      cudaStream_t s)
 {
-    const BlockProduct s1 = {tokens, q, b, b1, q * b1, q * b, b1, 1, b, 1};
+    const BlockProduct s1 = {tokens, q, b, b1, q * b1, q * b, b1, 1, b, 1, wt};
     return dtype == MONARCH_F32 ? block_product<float>(x, R, u, s1, s) : block_product<__nv_bfloat16>(x, R, u, s1, s);
 }
 
-int rect_stage2_simt(const void *u, const void *Lp, void *y, int64_t tokens, int q, int b, int r, int dtype,
+// wt = 0: y[t][l*b + j] = sum_k Lp[j][l][k] u[t][k*b + j] (q slices in, r out).  wt = 1: the adjoint,
+// du[t][k*b + j] = sum_l Lp[j][l][k] dy[t][l*b + j]: call with q = r of the forward, r = q of the forward.
+int rect_stage2_simt(const void *u, const void *Lp, void *y, int64_t tokens, int q, int b, int r, int dtype, int wt,
                      cudaStream_t s)
 {
-    const BlockProduct s2 = {tokens, b, r, q, q * b, r * b, 1, b, 1, b};
+    const BlockProduct s2 = {tokens, b, r, q, q * b, r * b, 1, b, 1, b, wt};
     const bool small4 = q <= 4 && r <= 4 && b % 2 == 0 && tokens > 0;
     const bool medium = !small4 && q <= 16 && r <= 16 && b >= 32 && tokens > 0;
     if (dtype == MONARCH_F32)
-        return small4   ? stage2_small4<float>(u, Lp, y, tokens, q, b, r, s)
-               : medium ? stage2_medium<float>(u, Lp, y, tokens, q, b, r, s)
+        return small4   ? stage2_small4<float>(u, Lp, y, tokens, q, b, r, wt, s)
+               : medium ? stage2_medium<float>(u, Lp, y, tokens, q, b, r, wt, s)
                         : block_product<float>(u, Lp, y, s2, s);
-    return small4   ? stage2_small4<__nv_bfloat16>(u, Lp, y, tokens, q, b, r, s)
-           : medium ? stage2_medium<__nv_bfloat16>(u, Lp, y, tokens, q, b, r, s)
+    return small4   ? stage2_small4<__nv_bfloat16>(u, Lp, y, tokens, q, b, r, wt, s)
+           : medium ? stage2_medium<__nv_bfloat16>(u, Lp, y, tokens, q, b, r, wt, s)
                     : block_product<__nv_bfloat16>(u, Lp, y, s2, s);
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Token reductions of the backward pass:  out[blk][o][i] (+)= sum_t A[t][blk*abs + o*aes] * B[t][blk*bbs + i*bes]
+//   dL[j][l][k] = sum_t dy[t][l*b + j] u[t][k*b + j]      (blk = j: strides 1 / b)
+//   dR[k][j][i] = sum_t du[t][k*b + j] x[t][k*b1 + i]     (blk = k: strides b / 1 and b1 / 1)
+// fp32 partial sums per token slab, added to the fp32 output with atomics (summation order may vary run to run).
+namespace {
+
+struct TokenReduce {
+    long long tokens;
+    int nb, o, k;
+    int a_row, b_row;
+    int abs_, aes, bbs, bes;
+    int tokens_per_slab;
+};
+
+// large blocks: a CTA owns a 64 x 64 tile of one block's gradient and a slab of tokens (tokens are the GEMM's K)
+template <typename T>
+__global__ void __launch_bounds__(256)
+token_reduce_tiled_kernel(const T *__restrict__ A, const T *__restrict__ B, float *__restrict__ out, const TokenReduce p)
+{
+    __shared__ float As[kKC][kTT + 4];
+    __shared__ float Bs[kKC][kOT + 4];
+    const int otiles = (p.o + 63) / 64, ktiles = (p.k + 63) / 64;
+    const int blk = blockIdx.x / (otiles * ktiles), rem = blockIdx.x % (otiles * ktiles);
+    const int o0 = (rem / ktiles) * 64, k0 = (rem % ktiles) * 64;
+    const long long t0 = (long long)blockIdx.y * p.tokens_per_slab;
+    const long long t1 = t0 + p.tokens_per_slab < p.tokens ? t0 + p.tokens_per_slab : p.tokens;
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    float acc[4][4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) acc[a][c] = 0.0f;
+    for (long long tb = t0; tb < t1; tb += kKC) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int idx = threadIdx.x + e * 256;           // 16 tokens x 64 columns
+            const int tt = idx >> 6, c = idx & 63;
+            const long long t = tb + tt;
+            float va = 0.0f, vb = 0.0f;
+            if (t < t1 && o0 + c < p.o)
+                va = elem<T>::load(A + (size_t)t * p.a_row + (size_t)blk * p.abs_ + (size_t)(o0 + c) * p.aes);
+            if (t < t1 && k0 + c < p.k)
+                vb = elem<T>::load(B + (size_t)t * p.b_row + (size_t)blk * p.bbs + (size_t)(k0 + c) * p.bes);
+            As[tt][c] = va;
+            Bs[tt][c] = vb;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int tt = 0; tt < kKC; ++tt) {
+            float a[4], c[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                a[e] = As[tt][ty * 4 + e];
+                c[e] = Bs[tt][tx * 4 + e];
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+#pragma unroll
+                for (int f = 0; f < 4; ++f) acc[e][f] = fmaf(a[e], c[f], acc[e][f]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+#pragma unroll
+        for (int f = 0; f < 4; ++f) {
+            const int o = o0 + ty * 4 + e, k = k0 + tx * 4 + f;
+            if (o < p.o && k < p.k) atomicAdd(out + ((size_t)blk * p.o + o) * p.k + k, acc[e][f]);
+        }
+}
+
+// blocks of at most 16 x 16: one thread per (block, output row), block index fastest
+template <typename T>
+__global__ void __launch_bounds__(256)
+token_reduce_small_kernel(const T *__restrict__ A, const T *__restrict__ B, float *__restrict__ out, const TokenReduce p)
+{
+    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (idx >= (long long)p.nb * p.o) return;
+    const int o = (int)(idx / p.nb), blk = (int)(idx % p.nb);
+    const long long t0 = (long long)blockIdx.y * p.tokens_per_slab;
+    const long long t1 = t0 + p.tokens_per_slab < p.tokens ? t0 + p.tokens_per_slab : p.tokens;
+    float acc[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) acc[i] = 0.0f;
+    for (long long t = t0; t < t1; ++t) {
+        const float a = elem<T>::load(A + (size_t)t * p.a_row + (size_t)blk * p.abs_ + (size_t)o * p.aes);
+        const T *brow = B + (size_t)t * p.b_row + (size_t)blk * p.bbs;
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+            if (i < p.k) acc[i] = fmaf(a, elem<T>::load(brow + (size_t)i * p.bes), acc[i]);
+    }
+    if (t1 > t0) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+            if (i < p.k) atomicAdd(out + ((size_t)blk * p.o + o) * p.k + i, acc[i]);
+    }
+}
+
+template <typename T>
+int token_reduce(const void *A, const void *B, float *out, TokenReduce p, cudaStream_t s)
+{
+    if (p.tokens == 0 || p.nb == 0) return MONARCH_OK;
+    if (p.o <= 16 && p.k <= 16) {
+        const long long bx = ((long long)p.nb * p.o + 255) / 256;
+        long long slabs = (148 * 8 + bx - 1) / bx;
+        if (slabs > (p.tokens + 31) / 32) slabs = (p.tokens + 31) / 32;
+        p.tokens_per_slab = (int)((p.tokens + slabs - 1) / slabs);
+        slabs = (p.tokens + p.tokens_per_slab - 1) / p.tokens_per_slab;
+        if (bx > 0x7fffffffLL || slabs > 65535) return MONARCH_ERR_UNSUPPORTED;
+        token_reduce_small_kernel<T><<<dim3((unsigned)bx, (unsigned)slabs), 256, 0, s>>>((const T *)A, (const T *)B, out, p);
+    } else {
+        const long long bx = (long long)p.nb * ((p.o + 63) / 64) * ((p.k + 63) / 64);
+        long long slabs = (148 * 4 + bx - 1) / bx;
+        if (slabs > (p.tokens + 255) / 256) slabs = (p.tokens + 255) / 256;
+        if (slabs < 1) slabs = 1;
+        p.tokens_per_slab = (int)((p.tokens + slabs - 1) / slabs);
+        p.tokens_per_slab = (p.tokens_per_slab + kKC - 1) / kKC * kKC;
+        slabs = (p.tokens + p.tokens_per_slab - 1) / p.tokens_per_slab;
+        if (bx > 0x7fffffffLL || slabs > 65535) return MONARCH_ERR_UNSUPPORTED;
+        token_reduce_tiled_kernel<T><<<dim3((unsigned)bx, (unsigned)slabs), 256, 0, s>>>((const T *)A, (const T *)B, out, p);
+    }
+    note_launch();
+    MONARCH_CUDA_TRY(cudaGetLastError());
+    return MONARCH_OK;
+}
+
+}  // namespace
+
+// dL += sum_t dy (x) u  and  dR += sum_t du (x) x  (the caller zeroes them first when not accumulating)
+int rect_wgrad_simt(const void *x, const void *dy, const void *u, const void *du, float *dL, float *dR, int64_t tokens,
+                    int q, int b1, int b, int r, int dtype, cudaStream_t s)
+{
+    const TokenReduce gl = {tokens, b, r, q, r * b, q * b, 1, b, 1, b, 0};
+    const TokenReduce gr = {tokens, q, b, b1, q * b, q * b1, b, 1, b1, 1, 0};
+    if (dtype == MONARCH_F32) {
+        MONARCH_TRY(token_reduce<float>(dy, u, dL, gl, s));
+        return token_reduce<float>(du, x, dR, gr, s);
+    }
+    MONARCH_TRY(token_reduce<__nv_bfloat16>(dy, u, dL, gl, s));
+    return token_reduce<__nv_bfloat16>(du, x, dR, gr, s);
 }
 
 }  // namespace monarch

@@ -247,7 +247,7 @@ __device__ __forceinline__ float bf_elem(const uint4 &v, int e)
 __global__ void __launch_bounds__(kS2Threads, 2)
 rect_stage2_stream_kernel(const __grid_constant__ CUtensorMap tm_u, const __nv_bfloat16 *__restrict__ Lp,
                           __nv_bfloat16 *__restrict__ y, unsigned *status, long long tokens, int q, int b, int r,
-                          int tokens_per_slab)
+                          int tokens_per_slab, int wt)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ float4 ws[4][4][2][32];            // [l][k][half][lane]: columns 8 lane + 4 half + (0..3)
@@ -266,7 +266,8 @@ rect_stage2_stream_kernel(const __grid_constant__ CUtensorMap tm_u, const __nv_b
     for (int i = threadIdx.x; i < 16 * kS2Cols; i += kS2Threads) {
         const int jl = i >> 4, l = (i >> 2) & 3, k = i & 3;
         float v = 0.0f;
-        if (j0 + jl < b && l < r && k < q) v = __bfloat162float(Lp[((size_t)(j0 + jl) * r + l) * q + k]);
+        // wt: the blocks are stored [j][k][l] (the adjoint pass reads L's blocks transposed)
+        if (j0 + jl < b && l < r && k < q) v = __bfloat162float(Lp[(size_t)(j0 + jl) * r * q + (wt ? k * r + l : l * q + k)]);
         reinterpret_cast<float *>(&ws[l][k][(jl >> 2) & 1][jl >> 3])[jl & 3] = v;
     }
     __syncthreads();
@@ -349,8 +350,8 @@ bool rect_stage2_stream_available(int q, int b, int r, int dtype)
     return dtype == MONARCH_BF16 && q <= 4 && r <= 4 && b % 8 == 0 && b >= 256;     // a 256-column box fits a slice
 }
 
-int rect_stage2_stream(const void *u, const void *Lp, void *y, int64_t tokens, int q, int b, int r, unsigned *status,
-                       cudaStream_t s)
+int rect_stage2_stream(const void *u, const void *Lp, void *y, int64_t tokens, int q, int b, int r, int wt,
+                       unsigned *status, cudaStream_t s)
 {
     using namespace tc;
     if (tokens == 0) return MONARCH_OK;
@@ -372,7 +373,7 @@ int rect_stage2_stream(const void *u, const void *Lp, void *y, int64_t tokens, i
     slabs = (tokens + per - 1) / per;
     if (slabs > 65535) return MONARCH_ERR_UNSUPPORTED;
     rect_stage2_stream_kernel<<<dim3((unsigned)cx, (unsigned)slabs), kS2Threads, kS2SmemBytes, s>>>(
-        tm_u, (const __nv_bfloat16 *)Lp, (__nv_bfloat16 *)y, status, tokens, q, b, r, (int)per);
+        tm_u, (const __nv_bfloat16 *)Lp, (__nv_bfloat16 *)y, status, tokens, q, b, r, (int)per, wt);
     note_launch();
     MONARCH_CUDA_TRY(cudaGetLastError());
     return MONARCH_OK;

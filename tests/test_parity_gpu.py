@@ -432,6 +432,41 @@ def test_rect_fwd(P, impl, q, b1, b, r, T, dtype):
     _check_guard(yf, "rect y")
 
 
+RECT_BWD_CASES = [
+    (2, 3, 4, 5, 7), (5, 1, 2, 4, 65), (3, 20, 17, 6, 130), (7, 5, 33, 9, 70), (4, 64, 64, 4, 257),
+    (4, 96, 32, 16, 129), (16, 16, 16, 16, 100), (4, 256, 256, 4, 200), (256, 4, 4, 256, 131), (8, 48, 80, 24, 90),
+    (2, 128, 192, 3, 300), (4, 64, 256, 4, 17), (3, 64, 512, 4, 1500),
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("q,b1,b,r,T", RECT_BWD_CASES)
+def test_rect_bwd(P, q, b1, b, r, T, dtype):
+    import torch
+    code = _code(P, dtype)
+    d = _rect_inputs(q, b1, b, r, T, dtype, seed=7 + q * 1000003 + b1 * 1009 + b * 31 + r)
+    rng = np.random.default_rng(T + q)
+    d["dy"] = round_to_storage(rng.standard_normal((T, r * b), dtype=np.float32), dtype)
+    x, dy, L, R = (to_device(d[k], dtype) for k in ("x", "dy", "L", "R"))
+    dxf, dx = _guarded((T, q * b1), _tdtype(dtype))
+    dLf, dL = _guarded((b, r, q), torch.float32)
+    dRf, dR = _guarded((q, b, b1), torch.float32)
+    ws = P.Workspace(P.monarch_rect_bwd_workspace_bytes(T, q, b1, b, r, code))
+    P.monarch_rect_bwd(x, dy, L, R, dx, dL, dR, 0, T, q, b1, b, r, ws)
+    torch.cuda.synchronize()
+    assert P.monarch_last_device_status(ws) == 0
+    ref = O.rect_bwd(d["x"], d["dy"], d["L"], d["R"])
+    assert_close(to_host64(dx), ref["dx"], dtype, "rect dx")
+    assert_close(to_host64(dL), ref["dL"], dtype, "rect dL")
+    assert_close(to_host64(dR), ref["dR"], dtype, "rect dR")
+    for flat, what in ((dxf, "dx"), (dLf, "dL"), (dRf, "dR")):
+        _check_guard(flat, f"rect {what}")
+    P.monarch_rect_bwd(x, dy, L, R, dx, dL, dR, 1, T, q, b1, b, r, ws)
+    torch.cuda.synchronize()
+    assert_close(to_host64(dL), 2 * ref["dL"], dtype, "rect dL accumulate")
+    assert_close(to_host64(dR), 2 * ref["dR"], dtype, "rect dR accumulate")
+
+
 def test_rect_square_case_equals_monarch_fwd(P):
     """q = b1 = b = r = m is Definition 3.1: both entry points see the same tensors."""
     import torch
