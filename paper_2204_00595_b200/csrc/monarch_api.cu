@@ -393,7 +393,10 @@ int monarch_rect_bwd(const void *x, const void *dy, const void *L, const void *R
     else
         MONARCH_TRY(rect_stage2_simt(dy, L, du, tokens, r, b, q, dtype, 1, s));
     // dx = blockdiag(R)^T du: stage 1 with the roles of b1 and b exchanged and the blocks read transposed
-    MONARCH_TRY(rect_stage1_simt(du, R, dx, tokens, q, b, b1, dtype, 1, s));
+    if (fast && rect_stage1_tc_available(q, b1, b, dtype))
+        MONARCH_TRY(rect_stage1_adjoint_tc(du, R, dx, tokens, q, b1, b, status, s));
+    else
+        MONARCH_TRY(rect_stage1_simt(du, R, dx, tokens, q, b, b1, dtype, 1, s));
     return rect_wgrad_simt(x, dy, u, du, dL, dR, tokens, q, b1, b, r, dtype, s);
 }
 

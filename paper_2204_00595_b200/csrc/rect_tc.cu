@@ -12,6 +12,9 @@
 //   warps 0-3       epilogue: TMEM -> registers -> bf16 -> swizzled staging tile (two, alternating) -> one TMA
 //                   store per 64 columns
 // Rows past the last token are zero-filled on load and clipped on store by the tensor maps.
+// The same kernel with BT = true computes the adjoint  dx[t][k*b1 + i] = sum_j R[k][j][i] du[t][k*b + j]:  the
+// contraction then runs over the rows of R_k, so the B operand is MN-major (64 x 64 boxes of R_k, 128-byte swizzle,
+// atoms 8 KB apart along N, 16 rows of K = 2 KB).
 #include "tc_common.cuh"
 
 namespace monarch {
@@ -23,7 +26,7 @@ constexpr int kThreads = 6 * 32;
 
 struct RectParams {
     unsigned *status;
-    int q, b1, b;
+    int q, kdim, ndim;                // blocks, contraction length and outputs per block
     int mtiles, ntiles_per_block;     // output tiles: mtiles x (q * ntiles_per_block)
 };
 
@@ -41,7 +44,7 @@ struct RectBars {
     uint64_t acc_full[2], acc_empty[2];
 };
 
-template <int NT>
+template <int NT, bool BT>
 __global__ void __launch_bounds__(kThreads, 1)
 rect_stage1_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_R,
                    const __grid_constant__ CUtensorMap tm_u, const RectParams p)
@@ -82,7 +85,7 @@ rect_stage1_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
 
     const int ntiles = p.q * p.ntiles_per_block;
     const long long total = (long long)p.mtiles * ntiles;
-    const int kchunks = p.b1 / kKChunk;
+    const int kchunks = p.kdim / kKChunk;
     const uint32_t full0 = smem_u32(bars.full), empty0 = smem_u32(bars.empty);
     const uint32_t accf0 = smem_u32(bars.acc_full), acce0 = smem_u32(bars.acc_empty);
 
@@ -98,15 +101,22 @@ rect_stage1_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
                     const uint32_t s = n % kStages;
                     if (!mbar_wait(empty0 + s * 8, ((n / kStages) & 1) ^ 1, p.status, dead, kErrSlotWait)) { ok = false; break; }
                     mbar_expect_tx(full0 + s * 8, S::kStageBytes);
-                    tma_load_2d(ring0 + s * S::kStageBytes, &tm_x, k * p.b1 + c * kKChunk, mt * kTokTile, full0 + s * 8);
-                    tma_load_2d(ring0 + s * S::kStageBytes + S::kABytes, &tm_R, c * kKChunk, k * p.b + n0, full0 + s * 8);
+                    tma_load_2d(ring0 + s * S::kStageBytes, &tm_x, k * p.kdim + c * kKChunk, mt * kTokTile, full0 + s * 8);
+                    if constexpr (!BT) {
+                        tma_load_2d(ring0 + s * S::kStageBytes + S::kABytes, &tm_R, c * kKChunk, k * p.ndim + n0, full0 + s * 8);
+                    } else {
+#pragma unroll
+                        for (int a = 0; a < NT / 64; ++a)      // 64 (K rows) x 64 (N columns) boxes of R_k
+                            tma_load_2d(ring0 + s * S::kStageBytes + S::kABytes + a * 8192, &tm_R, n0 + a * 64,
+                                        k * p.kdim + c * kKChunk, full0 + s * 8);
+                    }
                 }
             }
         }
     } else if (warp == 5) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc_bf16(kTokTile, NT, 0, 0);
+            constexpr uint32_t idesc = make_idesc_bf16(kTokTile, NT, 0, BT ? 1 : 0);
             uint32_t n = 0, it = 0;
             bool ok = true;
             for (long long tile = blockIdx.x; ok && tile < total; tile += gridDim.x, ++it) {
@@ -120,10 +130,12 @@ rect_stage1_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
                     tc_fence_after();
                     const uint32_t a_addr = ring0 + s * S::kStageBytes;
                     const uint64_t ad = make_smem_desc(a_addr, 16, 1024, kSwizzle128);
-                    const uint64_t bd = make_smem_desc(a_addr + S::kABytes, 16, 1024, kSwizzle128);
+                    const uint64_t bd = BT ? make_smem_desc(a_addr + S::kABytes, 8192, 1024, kSwizzle128)
+                                           : make_smem_desc(a_addr + S::kABytes, 16, 1024, kSwizzle128);
+                    constexpr uint32_t bstep = BT ? 128 : 2;          // 16 of K: 2 KB of rows, or 32 bytes along a row
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
-                        mma_f16_ss(d, ad + 2 * kk, bd + 2 * kk, idesc, (c | kk) != 0);
+                        mma_f16_ss(d, ad + 2 * kk, bd + bstep * kk, idesc, (c | kk) != 0);
                     mma_commit(empty0 + s * 8);
                 }
                 if (!ok) break;
@@ -171,7 +183,7 @@ rect_stage1_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
                 fence_proxy_async_smem();
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 if (threadIdx.x == 0) {
-                    tma_store_2d(&tm_u, stg, k * p.b + n0 + h * 64, mt * kTokTile);
+                    tma_store_2d(&tm_u, stg, k * p.ndim + n0 + h * 64, mt * kTokTile);
                     tma_store_commit();
                 }
             }
@@ -184,14 +196,19 @@ rect_stage1_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     if (warp == 0) tmem_dealloc(tmem_base, 2 * NT);
 }
 
-template <int NT>
-int launch(const void *x, const void *R, void *u, int64_t tokens, int q, int b1, int b, unsigned *status, cudaStream_t s)
+// in: [tokens][q * kdim], W: [q][b][b1] (kdim = b1, ndim = b) or, with BT, contracted over its rows (kdim = b, ndim = b1)
+template <int NT, bool BT>
+int launch(const void *in, const void *W, void *out, int64_t tokens, int q, int kdim, int ndim, unsigned *status,
+           cudaStream_t s)
 {
     using S = RectSmem<NT>;
     CUtensorMap tm_x, tm_R, tm_u;
-    MONARCH_TRY(encode_tmap_2d(&tm_x, x, (uint64_t)tokens, (uint64_t)q * b1, (uint64_t)q * b1 * 2, kTokTile, kKChunk, 128));
-    MONARCH_TRY(encode_tmap_2d(&tm_R, R, (uint64_t)q * b, (uint64_t)b1, (uint64_t)b1 * 2, NT, kKChunk, 128));
-    MONARCH_TRY(encode_tmap_2d(&tm_u, u, (uint64_t)tokens, (uint64_t)q * b, (uint64_t)q * b * 2, kTokTile, 64, 128));
+    MONARCH_TRY(encode_tmap_2d(&tm_x, in, (uint64_t)tokens, (uint64_t)q * kdim, (uint64_t)q * kdim * 2, kTokTile, kKChunk, 128));
+    if (BT)
+        MONARCH_TRY(encode_tmap_2d(&tm_R, W, (uint64_t)q * kdim, (uint64_t)ndim, (uint64_t)ndim * 2, 64, 64, 128));
+    else
+        MONARCH_TRY(encode_tmap_2d(&tm_R, W, (uint64_t)q * ndim, (uint64_t)kdim, (uint64_t)kdim * 2, NT, kKChunk, 128));
+    MONARCH_TRY(encode_tmap_2d(&tm_u, out, (uint64_t)tokens, (uint64_t)q * ndim, (uint64_t)q * ndim * 2, kTokTile, 64, 128));
     static int sms = 0;
     if (!sms) {
         int dev = 0;
@@ -200,17 +217,17 @@ int launch(const void *x, const void *R, void *u, int64_t tokens, int q, int b1,
     }
     static bool attr = false;
     if (!attr) {
-        MONARCH_CUDA_TRY(cudaFuncSetAttribute(rect_stage1_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kBytes));
+        MONARCH_CUDA_TRY(cudaFuncSetAttribute(rect_stage1_kernel<NT, BT>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kBytes));
         attr = true;
     }
     RectParams p;
     p.status = status;
-    p.q = q; p.b1 = b1; p.b = b;
+    p.q = q; p.kdim = kdim; p.ndim = ndim;
     p.mtiles = (int)((tokens + kTokTile - 1) / kTokTile);
-    p.ntiles_per_block = b / NT;
+    p.ntiles_per_block = ndim / NT;
     const long long total = (long long)p.mtiles * q * p.ntiles_per_block;
     const int grid = (int)(total < sms ? total : sms);
-    rect_stage1_kernel<NT><<<grid, kThreads, S::kBytes, s>>>(tm_x, tm_R, tm_u, p);
+    rect_stage1_kernel<NT, BT><<<grid, kThreads, S::kBytes, s>>>(tm_x, tm_R, tm_u, p);
     note_launch();
     MONARCH_CUDA_TRY(cudaGetLastError());
     return MONARCH_OK;
@@ -383,9 +400,19 @@ int rect_stage1_tc(const void *x, const void *R, void *u, int64_t tokens, int q,
                    cudaStream_t s)
 {
     if (tokens == 0) return MONARCH_OK;
-    if (b % 256 == 0) return tc::launch<256>(x, R, u, tokens, q, b1, b, status, s);
-    return b % 128 == 0 ? tc::launch<128>(x, R, u, tokens, q, b1, b, status, s)
-                        : tc::launch<64>(x, R, u, tokens, q, b1, b, status, s);
+    if (b % 256 == 0) return tc::launch<256, false>(x, R, u, tokens, q, b1, b, status, s);
+    return b % 128 == 0 ? tc::launch<128, false>(x, R, u, tokens, q, b1, b, status, s)
+                        : tc::launch<64, false>(x, R, u, tokens, q, b1, b, status, s);
+}
+
+// adjoint of stage 1 on the tensor cores: dx[t][k*b1 + i] = sum_j R[k][j][i] du[t][k*b + j]
+int rect_stage1_adjoint_tc(const void *du, const void *R, void *dx, int64_t tokens, int q, int b1, int b,
+                           unsigned *status, cudaStream_t s)
+{
+    if (tokens == 0) return MONARCH_OK;
+    if (b1 % 256 == 0) return tc::launch<256, true>(du, R, dx, tokens, q, b, b1, status, s);
+    return b1 % 128 == 0 ? tc::launch<128, true>(du, R, dx, tokens, q, b, b1, status, s)
+                         : tc::launch<64, true>(du, R, dx, tokens, q, b, b1, status, s);
 }
 
 }  // namespace monarch
