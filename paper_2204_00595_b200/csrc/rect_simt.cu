@@ -512,6 +512,68 @@ token_reduce_small_kernel(const T *__restrict__ A, const T *__restrict__ B, floa
     }
 }
 
+// dL[j][l][k] += sum_t dy[t][l*b + j] u[t][k*b + j] for blocks of at most 4 x 4: one thread owns two neighbouring
+// columns j and their 2 x 16 partial sums, walks a slab of tokens with 4-byte loads (a warp reads whole 128-byte
+// lines of every slice), and adds its sums to the output once.
+template <typename T>
+__global__ void __launch_bounds__(256)
+dl_small4_kernel(const T *__restrict__ dy, const T *__restrict__ u, float *__restrict__ dL, long long tokens, int q, int b,
+                 int r, int tokens_per_slab)
+{
+    const int j = (blockIdx.x * 256 + threadIdx.x) * 2;
+    if (j >= b) return;
+    float acc[2][4][4];
+#pragma unroll
+    for (int jj = 0; jj < 2; ++jj)
+#pragma unroll
+        for (int l = 0; l < 4; ++l)
+#pragma unroll
+            for (int k = 0; k < 4; ++k) acc[jj][l][k] = 0.0f;
+    const long long t0 = (long long)blockIdx.y * tokens_per_slab;
+    const long long t1 = t0 + tokens_per_slab < tokens ? t0 + tokens_per_slab : tokens;
+#pragma unroll 2
+    for (long long t = t0; t < t1; ++t) {
+        float2 g[4], v[4];
+#pragma unroll
+        for (int l = 0; l < 4; ++l)
+            g[l] = l < r ? pair_io<T>::load(dy + (size_t)t * r * b + (size_t)l * b + j) : make_float2(0.0f, 0.0f);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            v[k] = k < q ? pair_io<T>::load(u + (size_t)t * q * b + (size_t)k * b + j) : make_float2(0.0f, 0.0f);
+#pragma unroll
+        for (int l = 0; l < 4; ++l)
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                acc[0][l][k] = fmaf(g[l].x, v[k].x, acc[0][l][k]);
+                acc[1][l][k] = fmaf(g[l].y, v[k].y, acc[1][l][k]);
+            }
+    }
+    if (t1 > t0) {
+#pragma unroll
+        for (int jj = 0; jj < 2; ++jj)
+#pragma unroll
+            for (int l = 0; l < 4; ++l)
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    if (l < r && k < q) atomicAdd(dL + ((size_t)(j + jj) * r + l) * q + k, acc[jj][l][k]);
+    }
+}
+
+template <typename T>
+int dl_small4(const void *dy, const void *u, float *dL, long long tokens, int q, int b, int r, cudaStream_t s)
+{
+    const int bx = (b / 2 + 255) / 256;
+    long long slabs = (148 * 4 + bx - 1) / bx;
+    if (slabs > (tokens + 31) / 32) slabs = (tokens + 31) / 32;
+    const int per = (int)((tokens + slabs - 1) / slabs);
+    slabs = (tokens + per - 1) / per;
+    if (slabs > 65535) return MONARCH_ERR_UNSUPPORTED;
+    dl_small4_kernel<T><<<dim3((unsigned)bx, (unsigned)slabs), 256, 0, s>>>((const T *)dy, (const T *)u, dL, tokens, q, b, r, per);
+    note_launch();
+    MONARCH_CUDA_TRY(cudaGetLastError());
+    return MONARCH_OK;
+}
+
 template <typename T>
 int token_reduce(const void *A, const void *B, float *out, TokenReduce p, cudaStream_t s)
 {
@@ -544,16 +606,18 @@ int token_reduce(const void *A, const void *B, float *out, TokenReduce p, cudaSt
 
 // dL += sum_t dy (x) u  and  dR += sum_t du (x) x  (the caller zeroes them first when not accumulating)
 int rect_wgrad_simt(const void *x, const void *dy, const void *u, const void *du, float *dL, float *dR, int64_t tokens,
-                    int q, int b1, int b, int r, int dtype, cudaStream_t s)
+                    int q, int b1, int b, int r, int dtype, int want_dR, cudaStream_t s)
 {
     const TokenReduce gl = {tokens, b, r, q, r * b, q * b, 1, b, 1, b, 0};
     const TokenReduce gr = {tokens, q, b, b1, q * b, q * b1, b, 1, b1, 1, 0};
+    const bool small4 = q <= 4 && r <= 4 && b % 2 == 0 && tokens > 0;
     if (dtype == MONARCH_F32) {
-        MONARCH_TRY(token_reduce<float>(dy, u, dL, gl, s));
-        return token_reduce<float>(du, x, dR, gr, s);
+        MONARCH_TRY(small4 ? dl_small4<float>(dy, u, dL, tokens, q, b, r, s) : token_reduce<float>(dy, u, dL, gl, s));
+        return want_dR ? token_reduce<float>(du, x, dR, gr, s) : MONARCH_OK;
     }
-    MONARCH_TRY(token_reduce<__nv_bfloat16>(dy, u, dL, gl, s));
-    return token_reduce<__nv_bfloat16>(du, x, dR, gr, s);
+    MONARCH_TRY(small4 ? dl_small4<__nv_bfloat16>(dy, u, dL, tokens, q, b, r, s)
+                       : token_reduce<__nv_bfloat16>(dy, u, dL, gl, s));
+    return want_dR ? token_reduce<__nv_bfloat16>(du, x, dR, gr, s) : MONARCH_OK;
 }
 
 }  // namespace monarch

@@ -353,6 +353,154 @@ rect_stage2_stream_kernel(const __grid_constant__ CUtensorMap tm_u, const __nv_b
     }
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// dR[k][j][i] += sum_t du[t][k*b + j] x[t][k*b1 + i]: per block a GEMM whose contraction runs over the tokens, so both
+// operands are read token-major (MN-major descriptors over 64-token x 64-column boxes, 128-byte swizzle).  A CTA owns
+// a 128 (j) x NT (i) tile of one block's gradient and a slice of the token chunks; its fp32 partial sums go to the
+// output with vector reductions in L2.
+constexpr int kWgStages = 4;
+struct WgParams {
+    float *out;
+    unsigned *status;
+    int q, b, b1, chunks, slices;
+    int jtiles, itiles;
+};
+
+template <int NT>
+__global__ void __launch_bounds__(kThreads, 1)
+rect_wgrad_kernel(const __grid_constant__ CUtensorMap tm_du, const __grid_constant__ CUtensorMap tm_x, const WgParams p)
+{
+    constexpr int kABytes = 2 * 8192, kBBytes = (NT / 64) * 8192, kStageBytes = kABytes + kBBytes;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bar_full[kWgStages], bar_empty[kWgStages], bar_acc;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int dead_s;
+    const uint32_t ring0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    volatile int *dead = &dead_s;
+    int tile = blockIdx.x;
+    const int it = tile % p.itiles; tile /= p.itiles;
+    const int jt = tile % p.jtiles;
+    const int k = tile / p.jtiles;
+    const int j0 = jt * 128, i0 = it * NT;
+    const int first = blockIdx.y;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kWgStages; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 1);
+            mbar_init(smem_u32(&bar_empty[s]), 1);
+        }
+        mbar_init(smem_u32(&bar_acc), 1);
+        fence_mbar_init();
+        dead_s = 0;
+        tma_prefetch_desc(&tm_du);
+        tma_prefetch_desc(&tm_x);
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&tmem_base_s), NT);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+    const uint32_t full0 = smem_u32(bar_full), empty0 = smem_u32(bar_empty), acc = smem_u32(&bar_acc);
+
+    if (first < p.chunks) {
+        if (warp == 4) {
+            if (lane == 0) {
+                uint32_t n = 0;
+                for (int c = first; c < p.chunks; c += p.slices, ++n) {
+                    const uint32_t s = n % kWgStages;
+                    if (!mbar_wait(empty0 + s * 8, ((n / kWgStages) & 1) ^ 1, p.status, dead, kErrSlotWait)) break;
+                    const uint32_t dst = ring0 + s * kStageBytes, full = full0 + s * 8;
+                    mbar_expect_tx(full, kStageBytes);
+                    tma_load_2d(dst, &tm_du, k * p.b + j0, c * 64, full);
+                    tma_load_2d(dst + 8192, &tm_du, k * p.b + j0 + 64, c * 64, full);
+#pragma unroll
+                    for (int a = 0; a < NT / 64; ++a)
+                        tma_load_2d(dst + kABytes + a * 8192, &tm_x, k * p.b1 + i0 + a * 64, c * 64, full);
+                }
+            }
+        } else if (warp == 5) {
+            if (lane == 0) {
+                constexpr uint32_t idesc = make_idesc_bf16(128, NT, 1, 1);
+                // 64-column swizzle atoms 8 KB apart along M (N); 8-token groups 1 KB apart along K
+                const uint64_t desc = make_smem_desc(0, 8192, 1024, kSwizzle128);
+                uint32_t n = 0;
+                bool ok = true;
+                for (int c = first; c < p.chunks; c += p.slices, ++n) {
+                    const uint32_t s = n % kWgStages;
+                    if (!mbar_wait(full0 + s * 8, (n / kWgStages) & 1, p.status, dead, kErrTmaWait)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t ad = desc | (uint64_t)((ring0 + s * kStageBytes) >> 4);
+                    const uint64_t bd = ad + (kABytes >> 4);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)                      // 16 tokens = 2 KB further
+                        mma_f16_ss(tmem_base, ad + 128 * kk, bd + 128 * kk, idesc, (n | kk) != 0);
+                    mma_commit(empty0 + s * 8);
+                }
+                if (ok) mma_commit(acc);
+            }
+        } else {
+            if (mbar_wait(acc, 0, p.status, dead, kErrMmaWait)) {
+                tc_fence_after();
+                const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+                float *out = p.out + ((size_t)k * p.b + j0 + warp * 32 + lane) * p.b1 + i0;
+#pragma unroll 1
+                for (int c = 0; c < NT; c += 16) {
+                    uint32_t v[16];
+                    tmem_ld16(lane_base + c, v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(out + c + e * 4),
+                                     "f"(__uint_as_float(v[e * 4])), "f"(__uint_as_float(v[e * 4 + 1])),
+                                     "f"(__uint_as_float(v[e * 4 + 2])), "f"(__uint_as_float(v[e * 4 + 3]))
+                                     : "memory");
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem_base, NT);
+}
+
+template <int NT>
+int launch_wgrad(const void *du, const void *x, float *dR, int64_t tokens, int q, int b1, int b, unsigned *status,
+                 cudaStream_t s)
+{
+    constexpr int smem = kWgStages * (2 * 8192 + (NT / 64) * 8192) + 1024;
+    CUtensorMap tm_du, tm_x;
+    MONARCH_TRY(encode_tmap_2d(&tm_du, du, (uint64_t)tokens, (uint64_t)q * b, (uint64_t)q * b * 2, 64, 64, 128));
+    MONARCH_TRY(encode_tmap_2d(&tm_x, x, (uint64_t)tokens, (uint64_t)q * b1, (uint64_t)q * b1 * 2, 64, 64, 128));
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        MONARCH_CUDA_TRY(cudaGetDevice(&dev));
+        MONARCH_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        MONARCH_CUDA_TRY(cudaFuncSetAttribute(rect_wgrad_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    }
+    WgParams p;
+    p.out = dR;
+    p.status = status;
+    p.q = q; p.b = b; p.b1 = b1;
+    p.chunks = (int)((tokens + 63) / 64);
+    p.jtiles = b / 128;
+    p.itiles = b1 / NT;
+    const long long tiles = (long long)q * p.jtiles * p.itiles;
+    long long slices = sms / tiles;
+    if (slices < 1) slices = 1;
+    if (slices > p.chunks) slices = p.chunks;
+    if (tiles > 0x7fffffffLL || slices > 65535) return MONARCH_ERR_UNSUPPORTED;
+    p.slices = (int)slices;
+    rect_wgrad_kernel<NT><<<dim3((unsigned)tiles, (unsigned)slices), kThreads, smem, s>>>(tm_du, tm_x, p);
+    note_launch();
+    MONARCH_CUDA_TRY(cudaGetLastError());
+    return MONARCH_OK;
+}
+
 }  // namespace
 }  // namespace tc
 
@@ -403,6 +551,22 @@ int rect_stage1_tc(const void *x, const void *R, void *u, int64_t tokens, int q,
     if (b % 256 == 0) return tc::launch<256, false>(x, R, u, tokens, q, b1, b, status, s);
     return b % 128 == 0 ? tc::launch<128, false>(x, R, u, tokens, q, b1, b, status, s)
                         : tc::launch<64, false>(x, R, u, tokens, q, b1, b, status, s);
+}
+
+// dR on the tensor cores: bf16, b a multiple of 128 (the 128 TMEM lanes), b1 a multiple of 64
+bool rect_wgrad_R_tc_available(int q, int b1, int b, int dtype)
+{
+    (void)q;
+    return dtype == MONARCH_BF16 && b % 128 == 0 && b1 % 64 == 0;
+}
+
+int rect_wgrad_R_tc(const void *du, const void *x, float *dR, int64_t tokens, int q, int b1, int b, unsigned *status,
+                    cudaStream_t s)
+{
+    if (tokens == 0) return MONARCH_OK;
+    if (b1 % 256 == 0) return tc::launch_wgrad<256>(du, x, dR, tokens, q, b1, b, status, s);
+    return b1 % 128 == 0 ? tc::launch_wgrad<128>(du, x, dR, tokens, q, b1, b, status, s)
+                         : tc::launch_wgrad<64>(du, x, dR, tokens, q, b1, b, status, s);
 }
 
 // adjoint of stage 1 on the tensor cores: dx[t][k*b1 + i] = sum_j R[k][j][i] du[t][k*b + j]

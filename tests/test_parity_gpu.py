@@ -435,8 +435,17 @@ def test_rect_fwd(P, impl, q, b1, b, r, T, dtype):
 RECT_BWD_CASES = [
     (2, 3, 4, 5, 7), (5, 1, 2, 4, 65), (3, 20, 17, 6, 130), (7, 5, 33, 9, 70), (4, 64, 64, 4, 257),
     (4, 96, 32, 16, 129), (16, 16, 16, 16, 100), (4, 256, 256, 4, 200), (256, 4, 4, 256, 131), (8, 48, 80, 24, 90),
-    (2, 128, 192, 3, 300), (4, 64, 256, 4, 17), (3, 64, 512, 4, 1500),
+    (2, 128, 192, 3, 300), (4, 64, 256, 4, 17), (3, 64, 512, 4, 1500), (2, 192, 128, 3, 300), (4, 1024, 1024, 4, 140),
+    (1, 128, 384, 2, 77),
 ]
+
+
+def _instances(a):
+    """Gradient tensor -> the problem instances the normwise error is taken over: its blocks, or the whole tensor
+    when a block has fewer than 64 entries (a 2 x 1 block is a componentwise comparison, which sums with
+    cancellation do not pass even in exact fp32 arithmetic)."""
+    a = np.asarray(a)
+    return a if a[0].size >= 64 else a.reshape(1, -1)
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
@@ -457,14 +466,14 @@ def test_rect_bwd(P, q, b1, b, r, T, dtype):
     assert P.monarch_last_device_status(ws) == 0
     ref = O.rect_bwd(d["x"], d["dy"], d["L"], d["R"])
     assert_close(to_host64(dx), ref["dx"], dtype, "rect dx")
-    assert_close(to_host64(dL), ref["dL"], dtype, "rect dL")
-    assert_close(to_host64(dR), ref["dR"], dtype, "rect dR")
+    assert_close(_instances(to_host64(dL)), _instances(ref["dL"]), dtype, "rect dL")
+    assert_close(_instances(to_host64(dR)), _instances(ref["dR"]), dtype, "rect dR")
     for flat, what in ((dxf, "dx"), (dLf, "dL"), (dRf, "dR")):
         _check_guard(flat, f"rect {what}")
     P.monarch_rect_bwd(x, dy, L, R, dx, dL, dR, 1, T, q, b1, b, r, ws)
     torch.cuda.synchronize()
-    assert_close(to_host64(dL), 2 * ref["dL"], dtype, "rect dL accumulate")
-    assert_close(to_host64(dR), 2 * ref["dR"], dtype, "rect dR accumulate")
+    assert_close(_instances(to_host64(dL)), _instances(2 * ref["dL"]), dtype, "rect dL accumulate")
+    assert_close(_instances(to_host64(dR)), _instances(2 * ref["dR"]), dtype, "rect dR accumulate")
 
 
 def test_rect_square_case_equals_monarch_fwd(P):
