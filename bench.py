@@ -211,9 +211,12 @@ def main_rect(args):
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     c = RECT_WORKLOAD
     q, b1, b, r, T = c["q"], c["b1"], c["b"], c["r"], c["tokens"]
-    flops = 2 * T * (q * b * b1 + b * r * q)
+    with_bwd = "rect_bwd" in args.calls.split(",")
+    fwd_flops = 2 * T * (q * b * b1 + b * r * q)
+    flops = fwd_flops * (3 if with_bwd else 1)           # backward: dx and the two weight gradients, 2x the forward
     nbytes = T * (q * b1 + r * b) * 2 + (q * b * b1 + b * r * q) * 2
-    workload = f"workload 6: rect_fwd bf16 q={q} b1={b1} b={b} r={r} tokens/GPU={T}"
+    workload = (f"workload 6: rect_fwd{'+rect_bwd' if with_bwd else ''} bf16 q={q} b1={b1} b={b} r={r} "
+                f"tokens/GPU={T}")
     metric, unit = "monarch_rect_fwd_tflops", "TFLOP/s"
 
     def time_oracle_rect(d, target_s):
@@ -263,12 +266,29 @@ def main_rect(args):
     for s in range(2):                          # two rotating sets, each larger than L2 with its output
         x = torch.roll(to_device(d["x"], "bf16"), shifts=17 * s + 5 * rank, dims=0).contiguous()
         sets.append((x, torch.empty(T, r * b, dtype=torch.bfloat16, device="cuda")))
-    ws = P.Workspace(P.monarch_rect_workspace_bytes(T, q, b1, b, r, P.BF16))
+    ws = P.Workspace(max(P.monarch_rect_workspace_bytes(T, q, b1, b, r, P.BF16),
+                         P.monarch_rect_bwd_workspace_bytes(T, q, b1, b, r, P.BF16)))
     stream = torch.cuda.current_stream()
+    if with_bwd:
+        dy = torch.randn(T, r * b, device="cuda", generator=torch.Generator("cuda").manual_seed(595006)).bfloat16()
+        dxs = [torch.empty_like(sets[0][0]) for _ in range(2)]
+        gL = torch.zeros(b, r, q, dtype=torch.float32, device="cuda")
+        gR = torch.zeros(q, b, b1, dtype=torch.float32, device="cuda")
+    mid = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    nmid = [0]
 
-    def step(i):
+    def step(i, timed=False):
         x, y = sets[i % 2]
         P.monarch_rect_fwd(x, L, R, y, T, q, b1, b, r, ws)
+        if timed and with_bwd:                   # boundary between the two calls of a step
+            mid[nmid[0]].record(stream)
+            nmid[0] += 1
+        if with_bwd:
+            P.monarch_rect_bwd(x, dy, L, R, dxs[i % 2], gL, gR, 0, T, q, b1, b, r, ws)
+            if dist is not None:
+                dist.all_reduce(gL)
+                dist.all_reduce(gR)
 
     for i in range(args.warmup):
         step(i)
@@ -282,7 +302,9 @@ def main_rect(args):
     torch.cuda.synchronize()
     t_start.record(stream)
     for i in range(args.steps):
-        step(args.warmup + i)
+        if with_bwd:
+            starts[i].record(stream)
+        step(args.warmup + i, True)
     t_stop.record(stream)
     torch.cuda.synchronize()
     if dist is not None:
@@ -296,6 +318,7 @@ def main_rect(args):
         dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
         total_ms = float(tmax.item())
     ms = total_ms / args.steps
+    fwd_ms = statistics.mean(starts[i].elapsed_time(mid[i]) for i in range(args.steps)) if with_bwd else ms
     peaks = load_peaks()
     tfl = flops / (ms * 1e-3) / 1e12
     line = {
@@ -305,8 +328,12 @@ def main_rect(args):
         "config": {"workload": workload, "l2": "inputs larger than L2; 2 rotating buffer sets",
                    "kernels": args.kernels, "device_status": status},
         "clocks": clocks, "gpu_launches": int(launches),
-        "roofline": {"bound": "tensor", "kernel": "rect_fwd: rect_stage1_kernel<128> (tcgen05) + "
-                                                  "stage2_small4_bf16_kernel (2 launches)",
+        "calls": {"rect_fwd": {"ms": fwd_ms, "tflops": fwd_flops / fwd_ms / 1e9},
+                  **({"rect_bwd": {"ms": ms - fwd_ms, "tflops": 2 * fwd_flops / (ms - fwd_ms) / 1e9}} if with_bwd else {})},
+        "roofline": {"bound": "tensor", "kernel": "rect_fwd: rect_stage1_kernel<256> (tcgen05) + "
+                                                  "rect_stage2_stream_kernel (2 launches)"
+                                                  + ("; rect_bwd: stage 1, adjoint stage 2, adjoint stage 1 (tcgen05), "
+                                                     "rect_wgrad_kernel (tcgen05), dl_small4_kernel" if with_bwd else ""),
                      "achieved": tfl, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                      "frac": tfl / peaks["bf16_tflops"], "peak_source": peaks["source"], "traffic": None,
                      "algorithmic_mb": nbytes / 1e6,
