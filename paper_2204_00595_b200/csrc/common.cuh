@@ -150,15 +150,18 @@ int rect_stage1_simt(const void *x, const void *R, void *u, int64_t tokens, int 
                      cudaStream_t s);
 int rect_stage2_simt(const void *u, const void *Lp, void *y, int64_t tokens, int q, int b, int r, int dtype, int wt,
                      cudaStream_t s);
-// want_dR = 0 leaves dR to the tensor-core kernel
+// want_dL / want_dR = 0: that gradient comes from the streaming pass / the tensor-core kernel
 int rect_wgrad_simt(const void *x, const void *dy, const void *u, const void *du, float *dL, float *dR, int64_t tokens,
-                    int q, int b1, int b, int r, int dtype, int want_dR, cudaStream_t s);
+                    int q, int b1, int b, int r, int dtype, int want_dL, int want_dR, cudaStream_t s);
 // stage 1 on the tensor cores (rect_tc.cu): bf16, b1 and b multiples of 64
 bool rect_stage1_tc_available(int q, int b1, int b, int dtype);
 int rect_stage1_tc(const void *x, const void *R, void *u, int64_t tokens, int q, int b1, int b, unsigned *status,
                    cudaStream_t s);
 int rect_stage1_adjoint_tc(const void *du, const void *R, void *dx, int64_t tokens, int q, int b1, int b,
                            unsigned *status, cudaStream_t s);
+// dL for blocks up to 4 x 4 as a TMA-fed streaming pass (rect_tc.cu): sizes as rect_stage2_stream_available
+int rect_dl_stream(const void *dy, const void *u, float *dL, int64_t tokens, int q, int b, int r, unsigned *status,
+                   cudaStream_t s);
 bool rect_wgrad_R_tc_available(int q, int b1, int b, int dtype);
 int rect_wgrad_R_tc(const void *du, const void *x, float *dR, int64_t tokens, int q, int b1, int b, unsigned *status,
                     cudaStream_t s);

@@ -399,7 +399,9 @@ int monarch_rect_bwd(const void *x, const void *dy, const void *L, const void *R
         MONARCH_TRY(rect_stage1_simt(du, R, dx, tokens, q, b, b1, dtype, 1, s));
     const bool tc_dR = fast && rect_wgrad_R_tc_available(q, b1, b, dtype);
     if (tc_dR) MONARCH_TRY(rect_wgrad_R_tc(du, x, dR, tokens, q, b1, b, status, s));
-    return rect_wgrad_simt(x, dy, u, du, dL, dR, tokens, q, b1, b, r, dtype, !tc_dR, s);
+    const bool stream_dL = fast && rect_stage2_stream_available(q, b, r, dtype);
+    if (stream_dL) MONARCH_TRY(rect_dl_stream(dy, u, dL, tokens, q, b, r, status, s));
+    return rect_wgrad_simt(x, dy, u, du, dL, dR, tokens, q, b1, b, r, dtype, !stream_dL, !tc_dR, s);
 }
 
 int monarch_cplx_fwd(const void *x, const void *L, const void *R, void *y, int adjoint, int64_t tokens,

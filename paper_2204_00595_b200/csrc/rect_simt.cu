@@ -606,17 +606,19 @@ int token_reduce(const void *A, const void *B, float *out, TokenReduce p, cudaSt
 
 // dL += sum_t dy (x) u  and  dR += sum_t du (x) x  (the caller zeroes them first when not accumulating)
 int rect_wgrad_simt(const void *x, const void *dy, const void *u, const void *du, float *dL, float *dR, int64_t tokens,
-                    int q, int b1, int b, int r, int dtype, int want_dR, cudaStream_t s)
+                    int q, int b1, int b, int r, int dtype, int want_dL, int want_dR, cudaStream_t s)
 {
     const TokenReduce gl = {tokens, b, r, q, r * b, q * b, 1, b, 1, b, 0};
     const TokenReduce gr = {tokens, q, b, b1, q * b, q * b1, b, 1, b1, 1, 0};
     const bool small4 = q <= 4 && r <= 4 && b % 2 == 0 && tokens > 0;
     if (dtype == MONARCH_F32) {
-        MONARCH_TRY(small4 ? dl_small4<float>(dy, u, dL, tokens, q, b, r, s) : token_reduce<float>(dy, u, dL, gl, s));
+        if (want_dL)
+            MONARCH_TRY(small4 ? dl_small4<float>(dy, u, dL, tokens, q, b, r, s) : token_reduce<float>(dy, u, dL, gl, s));
         return want_dR ? token_reduce<float>(du, x, dR, gr, s) : MONARCH_OK;
     }
-    MONARCH_TRY(small4 ? dl_small4<__nv_bfloat16>(dy, u, dL, tokens, q, b, r, s)
-                       : token_reduce<__nv_bfloat16>(dy, u, dL, gl, s));
+    if (want_dL)
+        MONARCH_TRY(small4 ? dl_small4<__nv_bfloat16>(dy, u, dL, tokens, q, b, r, s)
+                           : token_reduce<__nv_bfloat16>(dy, u, dL, gl, s));
     return want_dR ? token_reduce<__nv_bfloat16>(du, x, dR, gr, s) : MONARCH_OK;
 }
 

@@ -354,6 +354,112 @@ rect_stage2_stream_kernel(const __grid_constant__ CUtensorMap tm_u, const __nv_b
 }
 
 // ---------------------------------------------------------------------------------------------------------
+// dL[j][l][k] += sum_t dy[t][l*b + j] u[t][k*b + j] for blocks of at most 4 x 4, as a streaming pass like the one
+// above: TMA brings 16-token tiles of the r slices of dy and the q slices of u into a three-stage ring; a thread owns
+// 8 columns and keeps their r x q x 8 partial sums in registers (one CTA per SM), adding them to dL at the end.
+__global__ void __launch_bounds__(kS2Threads, 1)
+rect_dl_stream_kernel(const __grid_constant__ CUtensorMap tm_dy, const __grid_constant__ CUtensorMap tm_u,
+                      float *__restrict__ dL, unsigned *status, long long tokens, int q, int b, int r, int tokens_per_slab)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full[kS2Stages];
+    __shared__ int dead_s;
+    const uint32_t ring0 = (smem_u32(smem_raw) + 127u) & ~127u;
+    const int j0 = blockIdx.x * kS2Cols;
+    volatile int *dead = &dead_s;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kS2Stages; ++s) mbar_init(smem_u32(&full[s]), 1);
+        fence_mbar_init();
+        dead_s = 0;
+        tma_prefetch_desc(&tm_dy);
+        tma_prefetch_desc(&tm_u);
+    }
+    __syncthreads();
+    const long long t0 = (long long)blockIdx.y * tokens_per_slab;
+    const long long t1 = t0 + tokens_per_slab < tokens ? t0 + tokens_per_slab : tokens;
+    const int ntiles = t1 > t0 ? (int)((t1 - t0 + kS2Tok - 1) / kS2Tok) : 0;
+    const uint32_t full0 = smem_u32(full);
+    const uint32_t stage_bytes = (uint32_t)(q + r) * kS2SliceBytes;
+    auto issue = [&](int tile) {
+        const uint32_t s = tile % kS2Stages;
+        const int row = (int)(t0 + (long long)tile * kS2Tok);
+        mbar_expect_tx(full0 + s * 8, stage_bytes);
+        for (int l = 0; l < r; ++l)
+            tma_load_2d(ring0 + (s * 8 + l) * kS2SliceBytes, &tm_dy, l * b + j0, row, full0 + s * 8);
+        for (int k = 0; k < q; ++k)
+            tma_load_2d(ring0 + (s * 8 + 4 + k) * kS2SliceBytes, &tm_u, k * b + j0, row, full0 + s * 8);
+    };
+    if (threadIdx.x == 0)
+        for (int tile = 0; tile < kS2Stages - 1 && tile < ntiles; ++tile) issue(tile);
+
+    const int lane = threadIdx.x & 31, tr = threadIdx.x >> 5;
+    const bool active = j0 + lane * 8 < b;
+    float gsum[4][4][8];
+#pragma unroll
+    for (int l = 0; l < 4; ++l)
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) gsum[l][k][e] = 0.0f;
+    for (int tile = 0; tile < ntiles; ++tile) {
+        if (threadIdx.x == 0 && tile + kS2Stages - 1 < ntiles) issue(tile + kS2Stages - 1);
+        const uint32_t s = tile % kS2Stages;
+        if (!mbar_wait(full0 + s * 8, (tile / kS2Stages) & 1, status, dead, kErrTmaWait)) break;
+        const long long ta = t0 + (long long)tile * kS2Tok + tr;
+        if (active) {
+            const uint32_t src = ring0 + s * 8 * kS2SliceBytes + lane * 16;
+#pragma unroll
+            for (int tt = 0; tt < 2; ++tt) {
+                if (ta + 8 * tt >= t1) break;                     // rows of the next slab, or past the last token
+                const uint32_t rowoff = (tr + 8 * tt) * (kS2Cols * 2);
+                float gf[4][8];
+#pragma unroll
+                for (int l = 0; l < 4; ++l) {
+                    const uint4 g = l < r ? lds128u(src + l * kS2SliceBytes + rowoff) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) gf[l][e] = bf_elem(g, e);
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    if (k >= q) break;
+                    const uint4 uv = lds128u(src + (4 + k) * kS2SliceBytes + rowoff);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const float uf = bf_elem(uv, e);
+#pragma unroll
+                        for (int l = 0; l < 4; ++l) gsum[l][k][e] = fmaf(gf[l][e], uf, gsum[l][k][e]);
+                    }
+                }
+            }
+        }
+        __syncthreads();
+    }
+    // the eight token rows of a lane hold partial sums of the same entries: add them up through the (now idle) ring
+    // before going to memory - one atomic per entry and CTA instead of eight
+    float *red = reinterpret_cast<float *>(smem_raw + (ring0 - smem_u32(smem_raw)));     // [tr][128 entries][32 lanes]
+#pragma unroll
+    for (int l = 0; l < 4; ++l)
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) red[(tr * 128 + (l * 4 + k) * 8 + e) * 32 + lane] = gsum[l][k][e];
+    __syncthreads();
+    if (ntiles > 0) {
+        for (int i = threadIdx.x; i < 128 * 32; i += kS2Threads) {
+            const int ent = i >> 5, ln = i & 31;                    // entry (l, k, e) of lane ln's columns
+            const int l = ent >> 5, k = (ent >> 3) & 3, e = ent & 7;
+            const int j = j0 + ln * 8 + e;
+            if (j < b && l < r && k < q) {
+                float sum = 0.0f;
+#pragma unroll
+                for (int w = 0; w < 8; ++w) sum += red[(w * 128 + ent) * 32 + ln];
+                atomicAdd(dL + ((size_t)j * r + l) * q + k, sum);
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------------
 // dR[k][j][i] += sum_t du[t][k*b + j] x[t][k*b1 + i]: per block a GEMM whose contraction runs over the tokens, so both
 // operands are read token-major (MN-major descriptors over 64-token x 64-column boxes, 128-byte swizzle).  A CTA owns
 // a 128 (j) x NT (i) tile of one block's gradient and a slice of the token chunks; its fp32 partial sums go to the
@@ -551,6 +657,37 @@ int rect_stage1_tc(const void *x, const void *R, void *u, int64_t tokens, int q,
     if (b % 256 == 0) return tc::launch<256, false>(x, R, u, tokens, q, b1, b, status, s);
     return b % 128 == 0 ? tc::launch<128, false>(x, R, u, tokens, q, b1, b, status, s)
                         : tc::launch<64, false>(x, R, u, tokens, q, b1, b, status, s);
+}
+
+// dL as a TMA-fed streaming pass: same sizes as the streaming stage 2
+int rect_dl_stream(const void *dy, const void *u, float *dL, int64_t tokens, int q, int b, int r, unsigned *status,
+                   cudaStream_t s)
+{
+    using namespace tc;
+    if (tokens == 0) return MONARCH_OK;
+    CUtensorMap tm_dy, tm_u;
+    MONARCH_TRY(encode_tmap_2d(&tm_dy, dy, (uint64_t)tokens, (uint64_t)r * b, (uint64_t)r * b * 2, kS2Tok, kS2Cols, 0));
+    MONARCH_TRY(encode_tmap_2d(&tm_u, u, (uint64_t)tokens, (uint64_t)q * b, (uint64_t)q * b * 2, kS2Tok, kS2Cols, 0));
+    constexpr int smem = kS2Stages * 8 * kS2SliceBytes + 128;
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        MONARCH_CUDA_TRY(cudaGetDevice(&dev));
+        MONARCH_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        MONARCH_CUDA_TRY(cudaFuncSetAttribute(rect_dl_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    }
+    const int cx = (b + kS2Cols - 1) / kS2Cols;
+    long long slabs = (sms + cx - 1) / cx;                            // one CTA per SM, one wave
+    if (slabs > (tokens + kS2Tok - 1) / kS2Tok) slabs = (tokens + kS2Tok - 1) / kS2Tok;
+    long long per = (tokens + slabs - 1) / slabs;
+    per = (per + kS2Tok - 1) / kS2Tok * kS2Tok;
+    slabs = (tokens + per - 1) / per;
+    if (slabs > 65535) return MONARCH_ERR_UNSUPPORTED;
+    rect_dl_stream_kernel<<<dim3((unsigned)cx, (unsigned)slabs), kS2Threads, smem, s>>>(tm_dy, tm_u, dL, status, tokens, q,
+                                                                                      b, r, (int)per);
+    note_launch();
+    MONARCH_CUDA_TRY(cudaGetLastError());
+    return MONARCH_OK;
 }
 
 // dR on the tensor cores: bf16, b a multiple of 128 (the 128 TMEM lanes), b1 a multiple of 64
