@@ -85,6 +85,9 @@ int tc_staged_mlp_fwd(const void *x, const void *L1, const void *R1, const void 
                       cudaStream_t s);
 
 
+// m = 128 through the GEMM kernels of the general class plus permutation passes (tc_bwd.cu)
+int gemm_permute_fwd_m128(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws, cudaStream_t s);
+
 // ---- backward as a chain of tensor-core launches (bf16; dx for m >= 32, dL/dR for m = 128), tc_bwd.cu ----
 size_t tc_staged_bwd_workspace_bytes(int64_t tokens, int m);
 int tc_staged_bwd(const void *x, const void *dy, const void *L, const void *R, void *dx, float *dL, float *dR,

@@ -153,6 +153,8 @@ size_t monarch_workspace_bytes(int op, int64_t tokens, int32_t n, int32_t m, int
     if (which < 0) return 0;
     if (which == kTcStaged && op != MONARCH_OP_FWD && op != MONARCH_OP_MLP_FWD)
         return tc_staged_bwd_workspace_bytes(tokens, m);
+    if (which == kTcStaged && op == MONARCH_OP_FWD && m == 128)       // GEMM and permutation passes alternate
+        return MONARCH_STATUS_BYTES + 2 * round256((size_t)tokens * n * esize(dtype));
     if (op == MONARCH_OP_BWD) {
         if (which == kFused) return fused_bwd_m64_workspace_bytes(tokens);
         const size_t a = staged_workspace_bytes(MONARCH_OP_BWD_DX, tokens, n, m, dtype);

@@ -27,6 +27,36 @@ __global__ void __launch_bounds__(256) permute_kernel(const __nv_bfloat16 *__res
     for (int r = threadIdx.y; r < 32; r += 8) dst[(long long)(a0 + r) * m + b0 + threadIdx.x] = tile[threadIdx.x][r];
 }
 
+// The same with 16-byte global accesses: one CTA per token; the m x m view goes to shared memory as it is stored
+// (pitch m/2 + 1 words) and leaves as rows of the transpose, each thread gathering the 8 elements of one 16-byte piece.
+__global__ void __launch_bounds__(256) permute_vec_kernel(const __nv_bfloat16 *__restrict__ v, __nv_bfloat16 *__restrict__ z,
+                                                          int m)
+{
+    extern __shared__ uint32_t ptile[];                        // [m][m/2 + 1] words
+    const int pitch = m / 2 + 1, chunks = m * m / 8, cpr = m / 8;
+    const __nv_bfloat16 *src = v + (size_t)blockIdx.x * m * m;
+    __nv_bfloat16 *dst = z + (size_t)blockIdx.x * m * m;
+    for (int c = threadIdx.x; c < chunks; c += 256) {
+        const int row = c / cpr, c8 = c % cpr;
+        const uint4 q = *reinterpret_cast<const uint4 *>(src + (size_t)c * 8);
+        uint32_t *d = ptile + row * pitch + c8 * 4;
+        d[0] = q.x; d[1] = q.y; d[2] = q.z; d[3] = q.w;
+    }
+    __syncthreads();
+    const unsigned short *h = reinterpret_cast<const unsigned short *>(ptile);
+    for (int c = threadIdx.x; c < chunks; c += 256) {
+        const int row = c / cpr, c8 = c % cpr;                 // output row = input column
+        uint32_t w[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const uint32_t lo = h[(size_t)(c8 * 8 + 2 * e) * pitch * 2 + row];
+            const uint32_t hi = h[(size_t)(c8 * 8 + 2 * e + 1) * pitch * 2 + row];
+            w[e] = lo | (hi << 16);
+        }
+        *reinterpret_cast<uint4 *>(dst + (size_t)c * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
 // Wt[b][c][e] = W[b][e][c] for every block
 __global__ void __launch_bounds__(256) transpose_blocks_kernel(const __nv_bfloat16 *__restrict__ W,
                                                                __nv_bfloat16 *__restrict__ Wt, int m)
@@ -205,6 +235,13 @@ int launch_wgrad128(const void *A, const void *B, float *out, int64_t tokens, un
 int permute(const void *v, void *z, int m, int64_t tokens, cudaStream_t s)
 {
     if (tokens == 0) return MONARCH_OK;
+    if (m % 8 == 0 && m <= 128 && tokens <= 0x7fffffffLL) {
+        const int smem = m * (m / 2 + 1) * 4;
+        permute_vec_kernel<<<(unsigned)tokens, 256, smem, s>>>((const __nv_bfloat16 *)v, (__nv_bfloat16 *)z, m);
+        note_launch();
+        MONARCH_CUDA_TRY(cudaGetLastError());
+        return MONARCH_OK;
+    }
     // grid.z carries the token index: at most 65535 per launch
     const __nv_bfloat16 *src = (const __nv_bfloat16 *)v;
     __nv_bfloat16 *dst = (__nv_bfloat16 *)z;
@@ -245,11 +282,54 @@ Layout carve(void *ws, int64_t tokens, int m)
 }  // namespace
 }  // namespace tc
 
-// Workspace: [status][z][du][u'][L^T][R^T]
+// Workspace: [status][z][du][u'][L^T][R^T]; for m = 128 the two weight areas hold a fourth token buffer instead
 size_t tc_staged_bwd_workspace_bytes(int64_t tokens, int m)
 {
     const size_t act = tc::align256((size_t)tokens * m * m * 2), wb = tc::align256((size_t)m * m * m * 2);
-    return MONARCH_STATUS_BYTES + 3 * act + 2 * wb;
+    return MONARCH_STATUS_BYTES + 3 * act + (m == 128 ? (act > 2 * wb ? act : 2 * wb) : 2 * wb);
+}
+
+// m = 128: every block product is a GEMM of the general class's kernels (rect_tc.cu: 128 x 128 blocks are large
+// enough for 128-wide MMAs and the kernel runs at the HBM limit), the stride permutation a pass of its own:
+//   forward  u = blockdiag(R) x, u' = P u, w = blockdiag(L) u', y = P w
+//   backward z = P dy, du' = blockdiag(L)^T z, du = P du', dx = blockdiag(R)^T du,
+//            dR = sum_t du (x) x, dL = sum_t z (x) u'  (u' recomputed)
+int gemm_permute_fwd_m128(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws, cudaStream_t s)
+{
+    constexpr int m = 128;
+    unsigned *status = (unsigned *)ws;
+    const size_t act = tc::align256((size_t)tokens * m * m * 2);
+    char *a = (char *)ws + MONARCH_STATUS_BYTES, *b = a + act;
+    MONARCH_TRY(rect_stage1_tc(x, R, a, tokens, m, m, m, status, s));
+    MONARCH_TRY(tc::permute(a, b, m, tokens, s));
+    MONARCH_TRY(rect_stage1_tc(b, L, a, tokens, m, m, m, status, s));
+    return tc::permute(a, y, m, tokens, s);
+}
+
+int gemm_permute_bwd_m128(const void *x, const void *dy, const void *L, const void *R, void *dx, float *dL, float *dR,
+                          int accumulate, int want_dx, int want_dw, int64_t tokens, void *ws, cudaStream_t s)
+{
+    constexpr int m = 128;
+    unsigned *status = (unsigned *)ws;
+    const size_t act = tc::align256((size_t)tokens * m * m * 2);
+    char *z = (char *)ws + MONARCH_STATUS_BYTES, *dup = z + act, *du = dup + act, *up = du + act;
+    if (want_dw && !accumulate) {
+        const size_t gb = (size_t)m * m * m * sizeof(float);
+        MONARCH_CUDA_TRY(cudaMemsetAsync(dL, 0, gb, s));
+        MONARCH_CUDA_TRY(cudaMemsetAsync(dR, 0, gb, s));
+    }
+    if (tokens == 0) return MONARCH_OK;
+    MONARCH_TRY(tc::permute(dy, z, m, tokens, s));
+    MONARCH_TRY(rect_stage1_adjoint_tc(z, L, dup, tokens, m, m, m, status, s));            // du'[t][j][k]
+    MONARCH_TRY(tc::permute(dup, du, m, tokens, s));                                       // du[t][k][j]
+    if (want_dx) MONARCH_TRY(rect_stage1_adjoint_tc(du, R, dx, tokens, m, m, m, status, s));
+    if (want_dw) {
+        MONARCH_TRY(rect_stage1_tc(x, R, dup, tokens, m, m, m, status, s));                // u (du' is dead)
+        MONARCH_TRY(tc::permute(dup, up, m, tokens, s));                                   // u'[t][j][k]
+        MONARCH_TRY(rect_wgrad_R_tc(du, x, dR, tokens, m, m, m, status, s));
+        MONARCH_TRY(rect_wgrad_R_tc(z, up, dL, tokens, m, m, m, status, s));
+    }
+    return MONARCH_OK;
 }
 
 // want_dx / want_dw select the outputs; dW needs m = 128 (the token-reduction kernel's block size)
@@ -258,6 +338,7 @@ int tc_staged_bwd(const void *x, const void *dy, const void *L, const void *R, v
 {
     using namespace tc;
     if (want_dw && m != 128) return MONARCH_ERR_UNSUPPORTED;
+    if (m == 128) return gemm_permute_bwd_m128(x, dy, L, R, dx, dL, dR, accumulate, want_dx, want_dw, tokens, ws, s);
     unsigned *status = (unsigned *)ws;
     const Layout l = carve(ws, tokens, m);
     if (want_dw && !accumulate) {

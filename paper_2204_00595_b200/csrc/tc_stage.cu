@@ -300,6 +300,7 @@ int encode_tmap_nd(CUtensorMap *out, const void *base, int elem_bytes, int rank,
 int tc_staged_fwd(const void *x, const void *L, const void *R, void *y, int64_t tokens, int m,
                   void *ws, cudaStream_t s)
 {
+    if (m == 128) return gemm_permute_fwd_m128(x, L, R, y, tokens, ws, s);   // workspace: two token buffers
     unsigned *status = (unsigned *)ws;
     void *u = (char *)ws + MONARCH_STATUS_BYTES;
     MONARCH_TRY(tc::tc_stage(m, x, R, u, nullptr, 0, tokens, status, s));
