@@ -43,9 +43,13 @@ __global__ void __launch_bounds__(256) permute_vec_kernel(const __nv_bfloat16 *_
         d[0] = q.x; d[1] = q.y; d[2] = q.z; d[3] = q.w;
     }
     __syncthreads();
+    // a warp takes a patch of 8 output rows x 4 pieces: its loads of one source row hit 4 x 4 distinct banks, and
+    // every output row gets 64 contiguous bytes
     const unsigned short *h = reinterpret_cast<const unsigned short *>(ptile);
-    for (int c = threadIdx.x; c < chunks; c += 256) {
-        const int row = c / cpr, c8 = c % cpr;                 // output row = input column
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int pcols = cpr / 4, patches = (m / 8) * pcols;
+    for (int pidx = warp; pidx < patches; pidx += 8) {
+        const int row = (pidx / pcols) * 8 + (lane >> 2), c8 = (pidx % pcols) * 4 + (lane & 3);   // output row = input column
         uint32_t w[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
@@ -53,7 +57,7 @@ __global__ void __launch_bounds__(256) permute_vec_kernel(const __nv_bfloat16 *_
             const uint32_t hi = h[(size_t)(c8 * 8 + 2 * e + 1) * pitch * 2 + row];
             w[e] = lo | (hi << 16);
         }
-        *reinterpret_cast<uint4 *>(dst + (size_t)c * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+        *reinterpret_cast<uint4 *>(dst + ((size_t)row * cpr + c8) * 8) = make_uint4(w[0], w[1], w[2], w[3]);
     }
 }
 
@@ -235,7 +239,7 @@ int launch_wgrad128(const void *A, const void *B, float *out, int64_t tokens, un
 int permute(const void *v, void *z, int m, int64_t tokens, cudaStream_t s)
 {
     if (tokens == 0) return MONARCH_OK;
-    if (m % 8 == 0 && m <= 128 && tokens <= 0x7fffffffLL) {
+    if (m % 32 == 0 && m <= 128 && tokens <= 0x7fffffffLL) {
         const int smem = m * (m / 2 + 1) * 4;
         permute_vec_kernel<<<(unsigned)tokens, 256, smem, s>>>((const __nv_bfloat16 *)v, (__nv_bfloat16 *)z, m);
         note_launch();
