@@ -266,8 +266,8 @@ def main_rect(args):
     for s in range(2):                          # two rotating sets, each larger than L2 with its output
         x = torch.roll(to_device(d["x"], "bf16"), shifts=17 * s + 5 * rank, dims=0).contiguous()
         sets.append((x, torch.empty(T, r * b, dtype=torch.bfloat16, device="cuda")))
-    ws = P.Workspace(max(P.monarch_rect_workspace_bytes(T, q, b1, b, r, P.BF16),
-                         P.monarch_rect_bwd_workspace_bytes(T, q, b1, b, r, P.BF16)))
+    ws = P.Workspace(P.monarch_rect_workspace_bytes(T, q, b1, b, r, P.BF16))
+    ws_b = P.Workspace(P.monarch_rect_bwd_workspace_bytes(T, q, b1, b, r, P.BF16))
     stream = torch.cuda.current_stream()
     if with_bwd:
         dy = torch.randn(T, r * b, device="cuda", generator=torch.Generator("cuda").manual_seed(595006)).bfloat16()
@@ -285,7 +285,7 @@ def main_rect(args):
             mid[nmid[0]].record(stream)
             nmid[0] += 1
         if with_bwd:
-            P.monarch_rect_bwd(x, dy, L, R, dxs[i % 2], gL, gR, 0, T, q, b1, b, r, ws)
+            P.monarch_rect_bwd(x, dy, L, R, dxs[i % 2], gL, gR, 0, T, q, b1, b, r, ws_b, fwd_workspace=ws)
             if dist is not None:
                 dist.all_reduce(gL)
                 dist.all_reduce(gR)

@@ -169,12 +169,16 @@ size_t monarch_rect_workspace_bytes(int64_t tokens, int32_t q, int32_t b1, int32
  *   du[t][k*b + j]  = sum_l L[j][l][k] dy[t][l*b + j]
  *   dx[t][k*b1 + i] = sum_j R[k][j][i] du[t][k*b + j]
  *   dL[j][l][k] = sum_t dy[t][l*b + j] u[t][k*b + j],  dR[k][j][i] = sum_t du[t][k*b + j] x[t][k*b1 + i]
- * with u recomputed inside.  x, dx: [tokens][q*b1]; dy: [tokens][r*b]; dL:
+ * `fwd_workspace` is null (u is recomputed inside) or the workspace that
+ * monarch_rect_fwd used for the SAME x, R and sizes, untouched since: u is then
+ * read from there (the caller vouches for its contents, as for monarch_bwd).
+ * x, dx: [tokens][q*b1]; dy: [tokens][r*b]; dL:
  * float32 [b][r][q]; dR: float32 [q][b][b1]; accumulate == 0 overwrites the two
  * weight gradients, 1 adds to them.  u and du are rounded to the storage dtype
  * once; the sums over tokens use atomic adds (last bits may vary run to run).
  * Workspace: monarch_rect_bwd_workspace_bytes. */
 int monarch_rect_bwd(const void *x, const void *dy, const void *L, const void *R,
+                     const void *fwd_workspace,
                      void *dx, float *dL, float *dR, int accumulate, int64_t tokens,
                      int32_t q, int32_t b1, int32_t b, int32_t r, int dtype,
                      void *workspace, size_t workspace_bytes, void *stream);

@@ -28,7 +28,7 @@ _SIGNATURES = {
     "monarch_mlp_bwd": (_int, [_vp] * 14 + [_int, _i64, _i32, _i32, _int, _vp, _sz, _vp]),
     "monarch_rect_fwd": (_int, [_vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32, _int, _vp, _sz, _vp]),
     "monarch_rect_workspace_bytes": (_sz, [_i64, _i32, _i32, _i32, _i32, _int]),
-    "monarch_rect_bwd": (_int, [_vp] * 7 + [_int, _i64, _i32, _i32, _i32, _i32, _int, _vp, _sz, _vp]),
+    "monarch_rect_bwd": (_int, [_vp] * 8 + [_int, _i64, _i32, _i32, _i32, _i32, _int, _vp, _sz, _vp]),
     "monarch_rect_bwd_workspace_bytes": (_sz, [_i64, _i32, _i32, _i32, _i32, _int]),
     "monarch_cplx_fwd": (_int, [_vp, _vp, _vp, _vp, _int, _i64, _i32, _i32, _int, _vp, _sz, _vp]),
     "monarch_dense": (_int, [_vp, _vp, _vp, _i32, _i32, _int, _vp]),
@@ -270,12 +270,15 @@ def monarch_rect_bwd_workspace_bytes(tokens: int, q: int, b1: int, b: int, r: in
     return int(lib().monarch_rect_bwd_workspace_bytes(tokens, q, b1, b, r, dtype))
 
 
-def monarch_rect_bwd(x, dy, L, R, dx, dL, dR, accumulate, tokens, q, b1, b, r, workspace, stream=None) -> None:
-    """Gradients of <dy, L R x> for the general class: dx like x; dL [b, r, q] and dR [q, b, b1] in float32."""
+def monarch_rect_bwd(x, dy, L, R, dx, dL, dR, accumulate, tokens, q, b1, b, r, workspace, fwd_workspace=None,
+                     stream=None) -> None:
+    """Gradients of <dy, L R x> for the general class: dx like x; dL [b, r, q] and dR [q, b, b1] in float32.
+    fwd_workspace = the Workspace monarch_rect_fwd used for the same x, R (its intermediate is then reused)."""
     import torch
     dt, f32 = x.dtype, torch.float32
     p, nb = _ws(workspace)
-    _check(lib().monarch_rect_bwd(_ptr(x, "x"), _ptr(dy, "dy", dt), _ptr(L, "L", dt), _ptr(R, "R", dt),
+    fp = _ws(fwd_workspace)[0] if fwd_workspace is not None else None
+    _check(lib().monarch_rect_bwd(_ptr(x, "x"), _ptr(dy, "dy", dt), _ptr(L, "L", dt), _ptr(R, "R", dt), fp,
                                   _ptr(dx, "dx", dt), _ptr(dL, "dL", f32), _ptr(dR, "dR", f32), int(accumulate),
                                   tokens, q, b1, b, r, _dtype_code(x), p, nb, _stream(stream)), "monarch_rect_bwd")
 

@@ -362,12 +362,14 @@ size_t monarch_rect_bwd_workspace_bytes(int64_t tokens, int32_t q, int32_t b1, i
     return MONARCH_STATUS_BYTES + 2 * round256((size_t)tokens * q * b * esize(dtype));      // [status][u][du]
 }
 
-int monarch_rect_bwd(const void *x, const void *dy, const void *L, const void *R, void *dx, float *dL, float *dR,
-                     int accumulate, int64_t tokens, int32_t q, int32_t b1, int32_t b, int32_t r, int dtype,
+int monarch_rect_bwd(const void *x, const void *dy, const void *L, const void *R, const void *fwd_workspace,
+                     void *dx, float *dL, float *dR, int accumulate, int64_t tokens, int32_t q, int32_t b1, int32_t b, int32_t r, int dtype,
                      void *workspace, size_t workspace_bytes, void *stream)
 {
     MONARCH_TRY(check_rect(tokens, q, b1, b, r, dtype));
     if (accumulate != 0 && accumulate != 1) return MONARCH_ERR_INVALID_ARG;
+    if (fwd_workspace != nullptr && (fwd_workspace == workspace || !aligned(fwd_workspace, 256)))
+        return MONARCH_ERR_INVALID_ARG;
     const size_t es = esize(dtype);
     const size_t lb = (size_t)b * r * q, rb = (size_t)q * b * b1;
     const Range in[] = {{x, (size_t)tokens * q * b1 * es}, {dy, (size_t)tokens * r * b * es}, {L, lb * es}, {R, rb * es}};
@@ -381,14 +383,17 @@ int monarch_rect_bwd(const void *x, const void *dy, const void *L, const void *R
     }
     if (tokens == 0) return MONARCH_OK;
     unsigned *status = (unsigned *)workspace;
-    char *u = (char *)workspace + MONARCH_STATUS_BYTES;
-    char *du = u + round256((size_t)tokens * q * b * es);
+    char *u_own = (char *)workspace + MONARCH_STATUS_BYTES;
+    char *du = u_own + round256((size_t)tokens * q * b * es);
     const bool fast = g_impl.load(std::memory_order_relaxed) != MONARCH_IMPL_STAGED;
-    // u = blockdiag(R) x (recomputed: the forward call keeps nothing)
-    if (fast && rect_stage1_tc_available(q, b1, b, dtype))
-        MONARCH_TRY(rect_stage1_tc(x, R, u, tokens, q, b1, b, status, s));
-    else
-        MONARCH_TRY(rect_stage1_simt(x, R, u, tokens, q, b1, b, dtype, 0, s));
+    // u = blockdiag(R) x: what the forward call left in its workspace ([status][u]), else recomputed
+    const char *u = fwd_workspace ? (const char *)fwd_workspace + MONARCH_STATUS_BYTES : u_own;
+    if (!fwd_workspace) {
+        if (fast && rect_stage1_tc_available(q, b1, b, dtype))
+            MONARCH_TRY(rect_stage1_tc(x, R, u_own, tokens, q, b1, b, status, s));
+        else
+            MONARCH_TRY(rect_stage1_simt(x, R, u_own, tokens, q, b1, b, dtype, 0, s));
+    }
     // du = L^T dy: stage 2 with the roles of q and r exchanged and the blocks read transposed
     if (fast && rect_stage2_stream_available(r, b, q, dtype))
         MONARCH_TRY(rect_stage2_stream(dy, L, du, tokens, r, b, q, 1, status, s));

@@ -470,8 +470,15 @@ def test_rect_bwd(P, q, b1, b, r, T, dtype):
     assert_close(_instances(to_host64(dR)), _instances(ref["dR"]), dtype, "rect dR")
     for flat, what in ((dxf, "dx"), (dLf, "dL"), (dRf, "dR")):
         _check_guard(flat, f"rect {what}")
-    P.monarch_rect_bwd(x, dy, L, R, dx, dL, dR, 1, T, q, b1, b, r, ws)
+    # second call: accumulate, with the intermediate a forward call left in its workspace
+    ws_f = P.Workspace(P.monarch_rect_workspace_bytes(T, q, b1, b, r, code))
+    y = torch.empty(T, r * b, dtype=_tdtype(dtype), device="cuda")
+    P.monarch_rect_fwd(x, L, R, y, T, q, b1, b, r, ws_f)
+    dx.fill_(float("nan"))
+    P.monarch_rect_bwd(x, dy, L, R, dx, dL, dR, 1, T, q, b1, b, r, ws, fwd_workspace=ws_f)
     torch.cuda.synchronize()
+    assert P.monarch_last_device_status(ws) == 0 and P.monarch_last_device_status(ws_f) == 0
+    assert_close(to_host64(dx), ref["dx"], dtype, "rect dx (saved u)")
     assert_close(_instances(to_host64(dL)), _instances(2 * ref["dL"]), dtype, "rect dL accumulate")
     assert_close(_instances(to_host64(dR)), _instances(2 * ref["dR"]), dtype, "rect dR accumulate")
 
