@@ -196,6 +196,217 @@ rect_stage1_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     if (warp == 0) tmem_dealloc(tmem_base, 2 * NT);
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// The same stage on CTA pairs (clusters of two, tcgen05 cta_group::2): one MMA instruction of 256 x 256 x 16 runs on
+// both SMs.  Each CTA loads the x rows of its own 128 tokens and HALF of the 256 weight rows of the tile (its
+// N/2 rows of the B operand), so the weight traffic from L2 to shared memory halves and the ring gets deeper; each
+// CTA ends up with the 128 x 256 accumulator of its own tokens in its own TMEM, laid out as for a single CTA, and
+// the epilogue is unchanged.  The even CTA's MMA thread issues for both; both CTAs' TMA loads count their bytes on
+// the even CTA's "stage full" barrier (a software relay of "my half has landed" through a release-arrive on the
+// peer's barrier cost about a microsecond per stage and made the kernel 2.5x slower).  Freed ring slots and finished
+// accumulators are announced to both CTAs by a multicast commit; drained accumulators are reported back to the
+// even CTA.
+constexpr int kPairStages = 6;
+constexpr int kPairStageBytes = 2 * kTokTile * kKChunk * 2;                // A 16 KB + this CTA's half of B 16 KB
+constexpr int kPairSmem = kPairStages * kPairStageBytes + 2 * (kTokTile * 128) + 1024;
+
+struct PairBars {
+    uint64_t full[kPairStages], empty[kPairStages];                     // full: used in the even CTA only
+    uint64_t acc_full[2], acc_empty[2];
+};
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+rect_stage1_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_R,
+                        const __grid_constant__ CUtensorMap tm_u, const RectParams p)
+{
+    constexpr int NT = 256;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) PairBars bars;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int dead_s;
+
+    const uint32_t ring0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t staging0 = ring0 + kPairStages * kPairStageBytes;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+    volatile int *dead = &dead_s;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kPairStages; ++s) {
+            mbar_init(smem_u32(&bars.full[s]), 1);                        // the even CTA's expect_tx arrival
+            mbar_init(smem_u32(&bars.empty[s]), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(smem_u32(&bars.acc_full[a]), 1);
+            mbar_init(smem_u32(&bars.acc_empty[a]), 8);                   // four epilogue warps of each CTA
+        }
+        fence_mbar_init();
+        dead_s = 0;
+        tma_prefetch_desc(&tm_x); tma_prefetch_desc(&tm_R); tma_prefetch_desc(&tm_u);
+    }
+    if (warp == 0) {
+        tmem_alloc_pair(smem_u32(&tmem_base_s), 2 * NT);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_arrive_release();                                             // both CTAs' barriers exist before any remote arrive
+    cluster_wait_acquire();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+
+    const int ntiles = p.q * p.ntiles_per_block;
+    const int mpairs = (p.mtiles + 1) / 2;                                // token tiles come in pairs, one per CTA
+    const long long total = (long long)mpairs * ntiles;
+    const int kchunks = p.kdim / kKChunk;
+    const uint32_t full0 = smem_u32(bars.full), empty0 = smem_u32(bars.empty);
+    const uint32_t accf0 = smem_u32(bars.acc_full), acce0 = smem_u32(bars.acc_empty);
+
+    if (warp == 4) {
+        // ------------------------------------------------------------ loader (both CTAs)
+        if (lane == 0) {
+            uint32_t n = 0;
+            bool ok = true;
+            for (long long tile = pair; ok && tile < total; tile += npairs) {
+                const int mt = (int)(tile / ntiles) * 2 + (int)rank, nt = (int)(tile % ntiles);
+                const int k = nt / p.ntiles_per_block, n0 = (nt % p.ntiles_per_block) * NT;
+                for (int c = 0; c < kchunks; ++c, ++n) {
+                    const uint32_t s = n % kPairStages;
+                    if (!mbar_wait(empty0 + s * 8, ((n / kPairStages) & 1) ^ 1, p.status, dead, kErrSlotWait)) { ok = false; break; }
+                    // the even CTA announces the bytes of both halves; either CTA's may land first
+                    if (rank == 0) mbar_expect_tx(full0 + s * 8, 2 * kPairStageBytes);
+                    tma_load_2d_pair(ring0 + s * kPairStageBytes, &tm_x, k * p.kdim + c * kKChunk, mt * kTokTile, full0 + s * 8);
+                    tma_load_2d_pair(ring0 + s * kPairStageBytes + kPairStageBytes / 2, &tm_R, c * kKChunk,
+                                     k * p.ndim + n0 + (int)rank * (NT / 2), full0 + s * 8);
+                }
+            }
+        }
+    } else if (warp == 5) {
+        if (lane == 0 && rank == 0) {
+            // ------------------------------------------------------------ even CTA: MMA issuer for the pair
+            constexpr uint32_t idesc = make_idesc_bf16(2 * kTokTile, NT, 0, 0);
+            uint32_t n = 0, it = 0;
+            bool ok = true;
+            for (long long tile = pair; ok && tile < total; tile += npairs, ++it) {
+                const uint32_t buf = it & 1;
+                if (!mbar_wait<true>(acce0 + buf * 8, ((it >> 1) & 1) ^ 1, p.status, dead, kErrTmemWait)) break;
+                tc_fence_after();
+                const uint32_t d = tmem_base + buf * NT;
+                for (int c = 0; c < kchunks; ++c, ++n) {
+                    const uint32_t s = n % kPairStages;
+                    if (!mbar_wait<true>(full0 + s * 8, (n / kPairStages) & 1, p.status, dead, kErrTmaWait)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = ring0 + s * kPairStageBytes;
+                    const uint64_t ad = make_smem_desc(a_addr, 16, 1024, kSwizzle128);
+                    const uint64_t bd = make_smem_desc(a_addr + kPairStageBytes / 2, 16, 1024, kSwizzle128);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        mma_f16_ss_pair(d, ad + 2 * kk, bd + 2 * kk, idesc, (c | kk) != 0);
+                    mma_commit_pair(empty0 + s * 8, 3);
+                }
+                if (!ok) break;
+                mma_commit_pair(accf0 + buf * 8, 3);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (both CTAs; own 128 tokens)
+        const int row = warp * 32 + lane;
+        const uint32_t acce_leader = map_to_cta(acce0, 0);
+        uint32_t it = 0, nchunk = 0;
+        for (long long tile = pair; tile < total; tile += npairs, ++it) {
+            const int mt = (int)(tile / ntiles) * 2 + (int)rank, nt = (int)(tile % ntiles);
+            const int k = nt / p.ntiles_per_block, n0 = (nt % p.ntiles_per_block) * NT;
+            const uint32_t buf = it & 1;
+            if (!mbar_wait(accf0 + buf * 8, (it >> 1) & 1, p.status, dead, kErrMmaWait)) break;
+            tc_fence_after();
+#pragma unroll 1
+            for (int h = 0; h < NT / 64; ++h, ++nchunk) {
+                const uint32_t stg = staging0 + (nchunk & 1) * (kTokTile * 128);
+                if (threadIdx.x == 0) tma_store_wait_read<1>();
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + buf * NT + h * 64;
+                uint32_t v[4][16];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) tmem_ld16(taddr + i * 16, v[i]);
+                tmem_ld_wait();
+                if (h == NT / 64 - 1) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(acce_leader + buf * 8);
+                }
+                const uint32_t dst = stg + row * 128;
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const uint32_t *w = &v[c >> 1][(c & 1) * 8];
+                    const uint32_t o0 = pack_bf16(__uint_as_float(w[0]), __uint_as_float(w[1]));
+                    const uint32_t o1 = pack_bf16(__uint_as_float(w[2]), __uint_as_float(w[3]));
+                    const uint32_t o2 = pack_bf16(__uint_as_float(w[4]), __uint_as_float(w[5]));
+                    const uint32_t o3 = pack_bf16(__uint_as_float(w[6]), __uint_as_float(w[7]));
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((c ^ (row & 7)) << 4)),
+                                 "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
+                }
+                fence_proxy_async_smem();
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (threadIdx.x == 0) {
+                    tma_store_2d(&tm_u, stg, k * p.ndim + n0 + h * 64, mt * kTokTile);
+                    tma_store_commit();
+                }
+            }
+        }
+        if (threadIdx.x == 0) tma_store_wait_all<0>();
+    }
+
+    // the even CTA's barriers receive arrivals from the odd CTA until it is done: leave together
+    tc_fence_before();
+    __syncthreads();
+    cluster_arrive_release();
+    cluster_wait_acquire();
+    if (warp == 0) tmem_dealloc_pair(tmem_base, 2 * NT);
+}
+
+int launch_pair(const void *in, const void *W, void *out, int64_t tokens, int q, int kdim, int ndim, unsigned *status,
+                cudaStream_t s, bool *used)
+{
+    *used = false;
+    CUtensorMap tm_x, tm_R, tm_u;
+    MONARCH_TRY(encode_tmap_2d(&tm_x, in, (uint64_t)tokens, (uint64_t)q * kdim, (uint64_t)q * kdim * 2, kTokTile, kKChunk, 128));
+    MONARCH_TRY(encode_tmap_2d(&tm_R, W, (uint64_t)q * ndim, (uint64_t)kdim, (uint64_t)kdim * 2, 128, kKChunk, 128));
+    MONARCH_TRY(encode_tmap_2d(&tm_u, out, (uint64_t)tokens, (uint64_t)q * ndim, (uint64_t)q * ndim * 2, kTokTile, 64, 128));
+    static int max_pairs = -1;
+    if (max_pairs < 0) {
+        MONARCH_CUDA_TRY(cudaFuncSetAttribute(rect_stage1_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmem));
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2, 1, 1);
+        cfg.blockDim = dim3(kThreads, 1, 1);
+        cfg.dynamicSmemBytes = kPairSmem;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, rect_stage1_pair_kernel, &cfg) != cudaSuccess) {
+            (void)cudaGetLastError();
+            n = 0;
+        }
+        max_pairs = n;
+    }
+    if (max_pairs < 1) return MONARCH_OK;                                 // the caller falls back to single CTAs
+    RectParams p;
+    p.status = status;
+    p.q = q; p.kdim = kdim; p.ndim = ndim;
+    p.mtiles = (int)((tokens + kTokTile - 1) / kTokTile);
+    p.ntiles_per_block = ndim / 256;
+    const long long total = (long long)((p.mtiles + 1) / 2) * q * p.ntiles_per_block;
+    const int pairs = (int)(total < max_pairs ? total : max_pairs);
+    rect_stage1_pair_kernel<<<2 * pairs, kThreads, kPairSmem, s>>>(tm_x, tm_R, tm_u, p);
+    note_launch();
+    MONARCH_CUDA_TRY(cudaGetLastError());
+    *used = true;
+    return MONARCH_OK;
+}
+
 // in: [tokens][q * kdim], W: [q][b][b1] (kdim = b1, ndim = b) or, with BT, contracted over its rows (kdim = b, ndim = b1)
 template <int NT, bool BT>
 int launch(const void *in, const void *W, void *out, int64_t tokens, int q, int kdim, int ndim, unsigned *status,
@@ -654,6 +865,12 @@ int rect_stage1_tc(const void *x, const void *R, void *u, int64_t tokens, int q,
                    cudaStream_t s)
 {
     if (tokens == 0) return MONARCH_OK;
+    if (b % 256 == 0 && tokens > 128) {
+        // two or more token tiles: CTA pairs (falls through where no cluster of two can be resident)
+        bool used = false;
+        MONARCH_TRY(tc::launch_pair(x, R, u, tokens, q, b1, b, status, s, &used));
+        if (used) return MONARCH_OK;
+    }
     if (b % 256 == 0) return tc::launch<256, false>(x, R, u, tokens, q, b1, b, status, s);
     return b % 128 == 0 ? tc::launch<128, false>(x, R, u, tokens, q, b1, b, status, s)
                         : tc::launch<64, false>(x, R, u, tokens, q, b1, b, status, s);
