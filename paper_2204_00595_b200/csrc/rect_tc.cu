@@ -215,6 +215,7 @@ struct PairBars {
     uint64_t acc_full[2], acc_empty[2];
 };
 
+template <bool BT>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 rect_stage1_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_R,
                         const __grid_constant__ CUtensorMap tm_u, const RectParams p)
@@ -277,15 +278,23 @@ rect_stage1_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_c
                     // the even CTA announces the bytes of both halves; either CTA's may land first
                     if (rank == 0) mbar_expect_tx(full0 + s * 8, 2 * kPairStageBytes);
                     tma_load_2d_pair(ring0 + s * kPairStageBytes, &tm_x, k * p.kdim + c * kKChunk, mt * kTokTile, full0 + s * 8);
-                    tma_load_2d_pair(ring0 + s * kPairStageBytes + kPairStageBytes / 2, &tm_R, c * kKChunk,
-                                     k * p.ndim + n0 + (int)rank * (NT / 2), full0 + s * 8);
+                    if constexpr (!BT) {
+                        tma_load_2d_pair(ring0 + s * kPairStageBytes + kPairStageBytes / 2, &tm_R, c * kKChunk,
+                                         k * p.ndim + n0 + (int)rank * (NT / 2), full0 + s * 8);
+                    } else {
+#pragma unroll
+                        for (int a = 0; a < 2; ++a)          // this CTA's 128 columns of R_k: two 64 x 64 boxes
+                            tma_load_2d_pair(ring0 + s * kPairStageBytes + kPairStageBytes / 2 + a * 8192, &tm_R,
+                                             n0 + (int)rank * (NT / 2) + a * 64, k * p.kdim + c * kKChunk, full0 + s * 8);
+                    }
                 }
             }
         }
     } else if (warp == 5) {
         if (lane == 0 && rank == 0) {
             // ------------------------------------------------------------ even CTA: MMA issuer for the pair
-            constexpr uint32_t idesc = make_idesc_bf16(2 * kTokTile, NT, 0, 0);
+            constexpr uint32_t idesc = make_idesc_bf16(2 * kTokTile, NT, 0, BT ? 1 : 0);
+            constexpr uint32_t bstep = BT ? 128 : 2;
             uint32_t n = 0, it = 0;
             bool ok = true;
             for (long long tile = pair; ok && tile < total; tile += npairs, ++it) {
@@ -299,10 +308,11 @@ rect_stage1_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_c
                     tc_fence_after();
                     const uint32_t a_addr = ring0 + s * kPairStageBytes;
                     const uint64_t ad = make_smem_desc(a_addr, 16, 1024, kSwizzle128);
-                    const uint64_t bd = make_smem_desc(a_addr + kPairStageBytes / 2, 16, 1024, kSwizzle128);
+                    const uint64_t bd = BT ? make_smem_desc(a_addr + kPairStageBytes / 2, 8192, 1024, kSwizzle128)
+                                           : make_smem_desc(a_addr + kPairStageBytes / 2, 16, 1024, kSwizzle128);
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
-                        mma_f16_ss_pair(d, ad + 2 * kk, bd + 2 * kk, idesc, (c | kk) != 0);
+                        mma_f16_ss_pair(d, ad + 2 * kk, bd + bstep * kk, idesc, (c | kk) != 0);
                     mma_commit_pair(empty0 + s * 8, 3);
                 }
                 if (!ok) break;
@@ -365,17 +375,21 @@ rect_stage1_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_c
     if (warp == 0) tmem_dealloc_pair(tmem_base, 2 * NT);
 }
 
+template <bool BT>
 int launch_pair(const void *in, const void *W, void *out, int64_t tokens, int q, int kdim, int ndim, unsigned *status,
                 cudaStream_t s, bool *used)
 {
     *used = false;
     CUtensorMap tm_x, tm_R, tm_u;
     MONARCH_TRY(encode_tmap_2d(&tm_x, in, (uint64_t)tokens, (uint64_t)q * kdim, (uint64_t)q * kdim * 2, kTokTile, kKChunk, 128));
-    MONARCH_TRY(encode_tmap_2d(&tm_R, W, (uint64_t)q * ndim, (uint64_t)kdim, (uint64_t)kdim * 2, 128, kKChunk, 128));
+    if (BT)
+        MONARCH_TRY(encode_tmap_2d(&tm_R, W, (uint64_t)q * kdim, (uint64_t)ndim, (uint64_t)ndim * 2, 64, 64, 128));
+    else
+        MONARCH_TRY(encode_tmap_2d(&tm_R, W, (uint64_t)q * ndim, (uint64_t)kdim, (uint64_t)kdim * 2, 128, kKChunk, 128));
     MONARCH_TRY(encode_tmap_2d(&tm_u, out, (uint64_t)tokens, (uint64_t)q * ndim, (uint64_t)q * ndim * 2, kTokTile, 64, 128));
     static int max_pairs = -1;
     if (max_pairs < 0) {
-        MONARCH_CUDA_TRY(cudaFuncSetAttribute(rect_stage1_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmem));
+        MONARCH_CUDA_TRY(cudaFuncSetAttribute(rect_stage1_pair_kernel<BT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmem));
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(2, 1, 1);
         cfg.blockDim = dim3(kThreads, 1, 1);
@@ -386,7 +400,7 @@ int launch_pair(const void *in, const void *W, void *out, int64_t tokens, int q,
         cfg.attrs = &attr;
         cfg.numAttrs = 1;
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, rect_stage1_pair_kernel, &cfg) != cudaSuccess) {
+        if (cudaOccupancyMaxActiveClusters(&n, rect_stage1_pair_kernel<BT>, &cfg) != cudaSuccess) {
             (void)cudaGetLastError();
             n = 0;
         }
@@ -400,7 +414,7 @@ int launch_pair(const void *in, const void *W, void *out, int64_t tokens, int q,
     p.ntiles_per_block = ndim / 256;
     const long long total = (long long)((p.mtiles + 1) / 2) * q * p.ntiles_per_block;
     const int pairs = (int)(total < max_pairs ? total : max_pairs);
-    rect_stage1_pair_kernel<<<2 * pairs, kThreads, kPairSmem, s>>>(tm_x, tm_R, tm_u, p);
+    rect_stage1_pair_kernel<BT><<<2 * pairs, kThreads, kPairSmem, s>>>(tm_x, tm_R, tm_u, p);
     note_launch();
     MONARCH_CUDA_TRY(cudaGetLastError());
     *used = true;
@@ -868,7 +882,7 @@ int rect_stage1_tc(const void *x, const void *R, void *u, int64_t tokens, int q,
     if (b % 256 == 0 && tokens > 128) {
         // two or more token tiles: CTA pairs (falls through where no cluster of two can be resident)
         bool used = false;
-        MONARCH_TRY(tc::launch_pair(x, R, u, tokens, q, b1, b, status, s, &used));
+        MONARCH_TRY(tc::launch_pair<false>(x, R, u, tokens, q, b1, b, status, s, &used));
         if (used) return MONARCH_OK;
     }
     if (b % 256 == 0) return tc::launch<256, false>(x, R, u, tokens, q, b1, b, status, s);
@@ -928,6 +942,11 @@ int rect_stage1_adjoint_tc(const void *du, const void *R, void *dx, int64_t toke
                            unsigned *status, cudaStream_t s)
 {
     if (tokens == 0) return MONARCH_OK;
+    if (b1 % 256 == 0 && tokens > 128) {
+        bool used = false;
+        MONARCH_TRY(tc::launch_pair<true>(du, R, dx, tokens, q, b, b1, status, s, &used));
+        if (used) return MONARCH_OK;
+    }
     if (b1 % 256 == 0) return tc::launch<256, true>(du, R, dx, tokens, q, b, b1, status, s);
     return b1 % 128 == 0 ? tc::launch<128, true>(du, R, dx, tokens, q, b, b1, status, s)
                          : tc::launch<64, true>(du, R, dx, tokens, q, b, b1, status, s);
