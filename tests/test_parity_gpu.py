@@ -525,6 +525,39 @@ def test_workload_rect(P, impl):
     assert_close(to_host64(y[torch.from_numpy(rows).cuda()]), ref.reshape(len(rows), q * b), "bf16", "rect identity L")
 
 
+def test_workload_rect_bwd(P, impl):
+    """Backward of the measured case at full size, in the configuration the benchmark times (the forward's
+    intermediate reused): dx on sampled token rows against the oracle; the weight gradients through the Euler
+    and adjoint identities <dL, L> = <dR, R> = <dx, x> = <dy, y> evaluated on the device results."""
+    import torch
+    from paper_2204_00595_b200.inputs import make_rect_inputs
+    d = make_rect_inputs()
+    q, b1, b, r, T = d["q"], d["b1"], d["b"], d["r"], d["tokens"]
+    rng = np.random.default_rng(606)
+    dy_h = round_to_storage(rng.standard_normal((T, r * b), dtype=np.float32), "bf16")
+    x, L, R, dy = (to_device(a, "bf16") for a in (d["x"], d["L"], d["R"], dy_h))
+    y = torch.empty(T, r * b, dtype=torch.bfloat16, device="cuda")
+    dx = torch.full((T, q * b1), float("nan"), dtype=torch.bfloat16, device="cuda")
+    dL = torch.full((b, r, q), float("nan"), dtype=torch.float32, device="cuda")
+    dR = torch.full((q, b, b1), float("nan"), dtype=torch.float32, device="cuda")
+    ws_f = P.Workspace(P.monarch_rect_workspace_bytes(T, q, b1, b, r, P.BF16))
+    ws_b = P.Workspace(P.monarch_rect_bwd_workspace_bytes(T, q, b1, b, r, P.BF16))
+    P.monarch_rect_fwd(x, L, R, y, T, q, b1, b, r, ws_f)
+    P.monarch_rect_bwd(x, dy, L, R, dx, dL, dR, 0, T, q, b1, b, r, ws_b, fwd_workspace=ws_f)
+    torch.cuda.synchronize()
+    assert P.monarch_last_device_status(ws_b) == 0 and P.monarch_last_device_status(ws_f) == 0
+    rows = _sample_tokens(T, 64, 66)
+    ref = O.rect_bwd(d["x"][rows], dy_h[rows], d["L"], d["R"])
+    dxh = to_host64(dx)
+    assert np.isfinite(dxh).all()
+    assert_close(dxh[rows], ref["dx"], "bf16", "rect workload dx")
+    s = float(np.sum(dy_h.astype(np.float64) * to_host64(y)))
+    tol = 2e-2 * float(np.sqrt(T * r * b))
+    assert abs(float(np.sum(dxh * d["x"])) - s) <= tol
+    assert abs(float(np.sum(to_host64(dL) * d["L"])) - s) <= tol
+    assert abs(float(np.sum(to_host64(dR) * d["R"])) - s) <= tol
+
+
 def test_rect_arguments(P):
     import torch
     x = torch.zeros(4, 64, device="cuda")
