@@ -343,7 +343,7 @@ rect_stage1_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_c
                 if (h == NT / 64 - 1) {
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(acce_leader + buf * 8);
+                    if (lane == 0) mbar_arrive_remote(acce_leader + buf * 8);
                 }
                 const uint32_t dst = stg + row * 128;
 #pragma unroll
