@@ -90,8 +90,11 @@ int gemm_permute_fwd_m128(const void *x, const void *L, const void *R, void *y, 
 
 // ---- backward as a chain of tensor-core launches (bf16; dx for m >= 32, dL/dR for m = 128), tc_bwd.cu ----
 size_t tc_staged_bwd_workspace_bytes(int64_t tokens, int m);
+// saved_up: for m = 128, u' = P blockdiag(R) x left by the forward call (gemm_permute_fwd_m128_saved_u), or null
 int tc_staged_bwd(const void *x, const void *dy, const void *L, const void *R, void *dx, float *dL, float *dR,
-                  int accumulate, int want_dx, int want_dw, int64_t tokens, int m, void *ws, cudaStream_t s);
+                  int accumulate, int want_dx, int want_dw, int64_t tokens, int m, void *ws, cudaStream_t s,
+                  const void *saved_up = nullptr);
+const void *gemm_permute_fwd_m128_saved_u(const void *fwd_ws, int64_t tokens);
 
 // ---- forward for m = 16 in one launch on the CUDA cores, both dtypes (fused_m16.cu); no workspace use ----
 int fused_fwd_m16(const void *x, const void *L, const void *R, void *y, int64_t tokens, int dtype, cudaStream_t s);

@@ -255,8 +255,11 @@ int monarch_bwd(const void *x, const void *dy, const void *L, const void *R, con
         return fused_bwd_m64(x, dy, L, R, saved ? fused_fwd_m64_saved_u(fwd_workspace) : nullptr, dx, dL,
                              dR, accumulate, tokens, workspace, s);
     }
-    if (which == kTcStaged)
-        return tc_staged_bwd(x, dy, L, R, dx, dL, dR, accumulate, 1, 1, tokens, m, workspace, s);
+    if (which == kTcStaged) {
+        const bool saved = fwd_workspace != nullptr && m == 128 && pick(MONARCH_OP_FWD, m, dtype) == kTcStaged;
+        return tc_staged_bwd(x, dy, L, R, dx, dL, dR, accumulate, 1, 1, tokens, m, workspace, s,
+                             saved ? gemm_permute_fwd_m128_saved_u(fwd_workspace, tokens) : nullptr);
+    }
     MONARCH_TRY(staged_bwd_dx(dy, L, R, dx, tokens, m, dtype, workspace, s));
     return staged_bwd_dw(x, dy, L, R, dL, dR, accumulate, tokens, m, dtype, workspace, s);
 }

@@ -297,7 +297,7 @@ size_t tc_staged_bwd_workspace_bytes(int64_t tokens, int m)
 // enough for 128-wide MMAs and the kernel runs at the HBM limit), the stride permutation a pass of its own:
 //   forward  u = blockdiag(R) x, u' = P u, w = blockdiag(L) u', y = P w
 //   backward z = P dy, du' = blockdiag(L)^T z, du = P du', dx = blockdiag(R)^T du,
-//            dR = sum_t du (x) x, dL = sum_t z (x) u'  (u' recomputed)
+//            dR = sum_t du (x) x, dL = sum_t z (x) u'  (u' recomputed, or read from the forward call's workspace)
 int gemm_permute_fwd_m128(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws, cudaStream_t s)
 {
     constexpr int m = 128;
@@ -310,8 +310,15 @@ int gemm_permute_fwd_m128(const void *x, const void *L, const void *R, void *y, 
     return tc::permute(a, y, m, tokens, s);
 }
 
-int gemm_permute_bwd_m128(const void *x, const void *dy, const void *L, const void *R, void *dx, float *dL, float *dR,
-                          int accumulate, int want_dx, int want_dw, int64_t tokens, void *ws, cudaStream_t s)
+// u' = P blockdiag(R) x as the forward call above leaves it in its workspace (the second token buffer)
+const void *gemm_permute_fwd_m128_saved_u(const void *fwd_ws, int64_t tokens)
+{
+    return (const char *)fwd_ws + MONARCH_STATUS_BYTES + tc::align256((size_t)tokens * 128 * 128 * 2);
+}
+
+int gemm_permute_bwd_m128(const void *x, const void *dy, const void *L, const void *R, const void *saved_up, void *dx,
+                          float *dL, float *dR, int accumulate, int want_dx, int want_dw, int64_t tokens, void *ws,
+                          cudaStream_t s)
 {
     constexpr int m = 128;
     unsigned *status = (unsigned *)ws;
@@ -328,21 +335,26 @@ int gemm_permute_bwd_m128(const void *x, const void *dy, const void *L, const vo
     MONARCH_TRY(tc::permute(dup, du, m, tokens, s));                                       // du[t][k][j]
     if (want_dx) MONARCH_TRY(rect_stage1_adjoint_tc(du, R, dx, tokens, m, m, m, status, s));
     if (want_dw) {
-        MONARCH_TRY(rect_stage1_tc(x, R, dup, tokens, m, m, m, status, s));                // u (du' is dead)
-        MONARCH_TRY(tc::permute(dup, up, m, tokens, s));                                   // u'[t][j][k]
+        if (saved_up == nullptr) {
+            MONARCH_TRY(rect_stage1_tc(x, R, dup, tokens, m, m, m, status, s));            // u (du' is dead)
+            MONARCH_TRY(tc::permute(dup, up, m, tokens, s));                               // u'[t][j][k]
+            saved_up = up;
+        }
         MONARCH_TRY(rect_wgrad_R_tc(du, x, dR, tokens, m, m, m, status, s));
-        MONARCH_TRY(rect_wgrad_R_tc(z, up, dL, tokens, m, m, m, status, s));
+        MONARCH_TRY(rect_wgrad_R_tc(z, saved_up, dL, tokens, m, m, m, status, s));
     }
     return MONARCH_OK;
 }
 
 // want_dx / want_dw select the outputs; dW needs m = 128 (the token-reduction kernel's block size)
 int tc_staged_bwd(const void *x, const void *dy, const void *L, const void *R, void *dx, float *dL, float *dR,
-                  int accumulate, int want_dx, int want_dw, int64_t tokens, int m, void *ws, cudaStream_t s)
+                  int accumulate, int want_dx, int want_dw, int64_t tokens, int m, void *ws, cudaStream_t s,
+                  const void *saved_up)
 {
     using namespace tc;
     if (want_dw && m != 128) return MONARCH_ERR_UNSUPPORTED;
-    if (m == 128) return gemm_permute_bwd_m128(x, dy, L, R, dx, dL, dR, accumulate, want_dx, want_dw, tokens, ws, s);
+    if (m == 128)
+        return gemm_permute_bwd_m128(x, dy, L, R, saved_up, dx, dL, dR, accumulate, want_dx, want_dw, tokens, ws, s);
     unsigned *status = (unsigned *)ws;
     const Layout l = carve(ws, tokens, m);
     if (want_dw && !accumulate) {
