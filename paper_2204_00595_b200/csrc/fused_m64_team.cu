@@ -324,23 +324,24 @@ fused_fwd_m64_team_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid
                 for (int c = sub; c < 8; c += 2, ++nchunk) {
                     const uint32_t k = nchunk & (kStagesPerHalf - 1);
                     const uint32_t sbuf = my_stage + k * kStageBytes;
-                    if (!wait_fast(stfree0 + k * 8, ((nchunk / kStagesPerHalf) & 1) ^ 1, p.status, dead, kErrSlotWait)) { ok = false; break; }
                     // chunk = 8 consecutive j; this lane holds blocks 4h..4h+3 of row `row`
                     uint32_t v[4][8];
 #pragma unroll
                     for (int kb = 0; kb < 4; ++kb) tmem_ld8(lane_base + kb * 64 + c * 8, v[kb]);
                     tmem_ld_wait();
+                    if (c + 2 >= 8) {
+                        // the accumulators are in registers: hand them back before waiting for a staging buffer
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(s1e);
+                    }
+                    if (!wait_fast(stfree0 + k * 8, ((nchunk / kStagesPerHalf) & 1) ^ 1, p.status, dead, kErrSlotWait)) { ok = false; break; }
 #pragma unroll
                     for (int q = 0; q < 8; ++q) {
                         const uint32_t o0 = pack_bf16(__uint_as_float(v[0][q]), __uint_as_float(v[1][q]));
                         const uint32_t o1 = pack_bf16(__uint_as_float(v[2][q]), __uint_as_float(v[3][q]));
                         // staging [j local 8][t 64][8 k]: the 1 KB slab of u'[tile][j][k/8 = grp]
                         asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(sbuf + q * 1024 + row * 16 + h * 8), "r"(o0), "r"(o1) : "memory");
-                    }
-                    if (c + 2 >= 8) {
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(s1e);
                     }
                     fence_proxy_async_smem();
                     __syncwarp();
@@ -354,12 +355,17 @@ fused_fwd_m64_team_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid
                 for (int c = sub; c < 8; c += 2, ++nchunk) {
                     const uint32_t k = nchunk & (kStagesPerHalf - 1);
                     const uint32_t sbuf = my_stage + k * kStageBytes;
-                    if (!wait_fast(stfree0 + k * 8, ((nchunk / kStagesPerHalf) & 1) ^ 1, p.status, dead, kErrSlotWait)) { ok = false; break; }
                     // chunk = 4 consecutive output rows l; lanes i and i+16 hold blocks 0-7 and 8-15
                     uint32_t v[8][4];
 #pragma unroll
                     for (int a = 0; a < 8; ++a) tmem_ld4(lane_base + 256 + a * 32 + c * 4, v[a]);
                     tmem_ld_wait();
+                    if (c + 2 >= 8) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(s2e);
+                    }
+                    if (!wait_fast(stfree0 + k * 8, ((nchunk / kStagesPerHalf) & 1) ^ 1, p.status, dead, kErrSlotWait)) { ok = false; break; }
                     if (p.bias != nullptr) {
                         // output element (l, j): l = 32 hl + 4c + q, j = 16 hj + 8h + a
 #pragma unroll
@@ -384,11 +390,6 @@ fused_fwd_m64_team_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid
                         // staging [l local 4][t 64][16 j]
                         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sbuf + q * 2048 + row * 32 + h * 16),
                                      "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
-                    }
-                    if (c + 2 >= 8) {
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(s2e);
                     }
                     fence_proxy_async_smem();
                     __syncwarp();
