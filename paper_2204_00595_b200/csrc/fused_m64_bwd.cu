@@ -59,6 +59,7 @@ struct BwdParams {
     int tiles;
     int b1, b2;                // CTAs per B1 group, per B2 group
     int b3;                    // all-in-one kernel: CTAs per group of the dL kind (0 elsewhere)
+    int want_dx;               // all-in-one kernel: 0 = weight gradients only (dx is neither formed nor stored)
     unsigned need, reset_at;   // a tile is ready at `need` arrivals; the consumer that brings it to `reset_at` clears it
     const __nv_bfloat16 *dy;   // natural dy (for L2 prefetch hints only; the data path goes through TMA)
     const __nv_bfloat16 *u;    // all-in-one kernel: u' = P R x, [tiles][64 j][8][64 t][8] (forward exchange layout)
@@ -715,30 +716,36 @@ __device__ __forceinline__ void b2r_body(const CUtensorMap &tm_R, const CUtensor
         const uint64_t b_dr = make_smem_desc(0, 16, 1024, kSwizzle128) | (uint64_t)((ring0 + 8192) >> 4);
         uint32_t nitem = 0;
         for (int tile = first; tile < p.tiles; tile += step, ++nitem) {
-            // dx of this tile: the single accumulator set must have been drained
-            if (!wait_fast(dxe, (nitem & 1) ^ 1, p.status, dead, kErrTmemWait)) return;
-            tc_fence_after();
-#pragma unroll
-            for (int g = 0; g < 4; ++g) {
-                if (!wait_fast(full0 + g * 8, nitem & 1, p.status, dead, kErrTmaWait)) return;
+            if (p.want_dx) {
+                // dx of this tile: the single accumulator set must have been drained
+                if (!wait_fast(dxe, (nitem & 1) ^ 1, p.status, dead, kErrTmemWait)) return;
                 tc_fence_after();
 #pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    const int b = g * 2 + i;
-                    const uint64_t ad = a_dx + (uint64_t)(b * (kRSlotBytes >> 4));
-                    const uint64_t bd = b_dx + b * 512;
-                    const uint32_t d = tmem_base + b * 64;
-                    mma_f16_ss(d, ad, bd, idesc_dx, 0);
-                    mma_f16_ss(d, ad + 128, bd + 128, idesc_dx, 1);
-                    mma_f16_ss(d, ad + 256, bd + 256, idesc_dx, 1);
-                    mma_f16_ss(d, ad + 384, bd + 384, idesc_dx, 1);
+                for (int g = 0; g < 4; ++g) {
+                    if (!wait_fast(full0 + g * 8, nitem & 1, p.status, dead, kErrTmaWait)) return;
+                    tc_fence_after();
+#pragma unroll
+                    for (int i = 0; i < 2; ++i) {
+                        const int b = g * 2 + i;
+                        const uint64_t ad = a_dx + (uint64_t)(b * (kRSlotBytes >> 4));
+                        const uint64_t bd = b_dx + b * 512;
+                        const uint32_t d = tmem_base + b * 64;
+                        mma_f16_ss(d, ad, bd, idesc_dx, 0);
+                        mma_f16_ss(d, ad + 128, bd + 128, idesc_dx, 1);
+                        mma_f16_ss(d, ad + 256, bd + 256, idesc_dx, 1);
+                        mma_f16_ss(d, ad + 384, bd + 384, idesc_dx, 1);
+                    }
                 }
+                mma_commit(dxf);
             }
-            mma_commit(dxf);
             // dR += du^T x while the epilogue drains dx; each pair of slots is released after its last use
             const uint32_t acc = nitem != 0;
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
+                if (!p.want_dx) {      // (with dx the operands of the pair were awaited above)
+                    if (!wait_fast(full0 + g * 8, nitem & 1, p.status, dead, kErrTmaWait)) return;
+                    tc_fence_after();
+                }
 #pragma unroll
                 for (int i = 0; i < 2; ++i) {
                     const int b = g * 2 + i;
@@ -763,7 +770,7 @@ __device__ __forceinline__ void b2r_body(const CUtensorMap &tm_R, const CUtensor
         const uint32_t stfree0 = smem_u32(bars->st_free) + sub * NST * 8;
         const bool mine = lane < 16;                                       // dx lives in the first 16 lanes of each quarter
         uint32_t nitem = 0, nchunk = 0;
-        for (int tile = first; tile < p.tiles; tile += step, ++nitem) {
+        for (int tile = first; p.want_dx && tile < p.tiles; tile += step, ++nitem) {
             if (!wait_fast(dxf, nitem & 1, p.status, dead, kErrMmaWait)) return;
             tc_fence_after();
 #pragma unroll 1
@@ -823,7 +830,7 @@ __device__ __forceinline__ void b2r_body(const CUtensorMap &tm_R, const CUtensor
             }
         }
     } else if (warp >= kStoreWarp0 && warp < kStoreWarp0 + 2) {
-        if (lane != 0) return;
+        if (lane != 0 || !p.want_dx) return;
         const int sub = warp - kStoreWarp0;
         store_thread<false, NST>(p, bars, stage0, sub, first, step, dead,
             [&](uint32_t sbuf, int tile, int c) { tma_store_2d(&tm_dx, sbuf, (grp * 8 + c) * kM, tile * 64); });
@@ -1058,6 +1065,7 @@ int launch_bwd_m64(const void *dy, const void *L, const void *R, void *dx, void 
     p.b1 = b1;
     p.b2 = b2;
     p.b3 = 0;
+    p.want_dx = 1;
     p.need = kB1Arrivals;
     p.reset_at = kB1Arrivals + kB2Groups;
     p.u = nullptr;
@@ -1093,7 +1101,8 @@ int fused_bwd_all_m64(const void *x, const void *dy, const void *L, const void *
     }
     MONARCH_TRY(encode_tmap_2d(&tm_Lt, L, kN, kM, kM * 2, 64, 64, 128));
     MONARCH_TRY(encode_tmap_2d(&tm_R, R, kN, kM, kM * 2, 64, 64, 128));
-    MONARCH_TRY(encode_tmap_2d(&tm_dx, dx, (uint64_t)tokens, kN, kN * 2, 64, 64, 128));
+    // dx == null: weight gradients only (the map is never used; it only has to be a valid one)
+    MONARCH_TRY(encode_tmap_2d(&tm_dx, dx ? dx : x, (uint64_t)tokens, kN, kN * 2, 64, 64, 128));
     MONARCH_TRY(encode_tmap_2d(&tm_x, x, (uint64_t)tokens, kN, kN * 2, 64, 64, 128));
     static int sms = 0;
     if (!sms) {
@@ -1112,11 +1121,14 @@ int fused_bwd_all_m64(const void *x, const void *dy, const void *L, const void *
     p.u = (const __nv_bfloat16 *)u;
     p.dL = dL;
     p.dR = dR;
+    p.want_dx = dx != nullptr;
     p.tokens = tokens;
     p.tiles = (int)tiles;
     // SM split: 8/7/6 CTAs per group (8 B1 groups, 8 B2R groups, 4 WL groups: 144 CTAs) was the best of a sweep
     // on 148 SMs; one CTA per group less of any kind costs 2-10 %
     int b1 = (sms * 8) / 144, b2 = (sms * 7) / 144, b3 = (sms * 6) / 144;
+    // weight gradients only: the B2R kind has half the work, 10/4/7 was the best of a sweep (132 against 140 us)
+    if (dx == nullptr) { b1 = (sms * 10) / 144; b2 = (sms * 4) / 144; b3 = (sms * 7) / 144; }
 #ifdef MONARCH_TRACE
     if (const char *e = getenv("MONARCH_BWD_SPLIT3")) sscanf(e, "%d,%d,%d", &b1, &b2, &b3);
 #endif

@@ -259,6 +259,12 @@ int fused_bwd_dw_m64(const void *x, const void *dy, const void *L, const void *R
     char *u = (char *)ws + MONARCH_STATUS_BYTES + kDwCounterBytes;
     char *du = u + ex, *dyp = du + ex;
     MONARCH_TRY(fused_fwd_m64_stage1(x, R, u, tokens, status, s));
+    // the one-launch backward with its dx part switched off: du and P dy are consumed from L2 as they appear
+    // instead of after a launch of their own (it declines, before launching anything, on a GPU too small to hold
+    // all of its CTAs at once; then the three-launch form below runs)
+    unsigned *counters = (unsigned *)((char *)ws + MONARCH_STATUS_BYTES);
+    const int rc = fused_bwd_all_m64(x, dy, L, R, u, nullptr, du, dyp, dL, dR, counters, status, tokens, s);
+    if (rc != MONARCH_ERR_UNSUPPORTED) return rc;
     MONARCH_TRY(fused_bwd_m64_stage1(dy, L, du, dyp, tokens, status, s));
     return launch_dw(x, u, du, dyp, dL, dR, status, tokens, s);
 }
