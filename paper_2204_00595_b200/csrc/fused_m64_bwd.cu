@@ -1124,9 +1124,9 @@ int fused_bwd_all_m64(const void *x, const void *dy, const void *L, const void *
     p.want_dx = dx != nullptr;
     p.tokens = tokens;
     p.tiles = (int)tiles;
-    // SM split: 8/7/6 CTAs per group (8 B1 groups, 8 B2R groups, 4 WL groups: 144 CTAs) was the best of a sweep
-    // on 148 SMs; one CTA per group less of any kind costs 2-10 %
-    int b1 = (sms * 8) / 144, b2 = (sms * 7) / 144, b3 = (sms * 6) / 144;
+    // SM split: 8/7/7 CTAs per group (8 B1 groups, 8 B2R groups, 4 WL groups: all 148 SMs) was the best of a sweep
+    // on 148 SMs; one CTA per group less of the first two kinds costs 2-10 %
+    int b1 = (sms * 8) / 144, b2 = (sms * 7) / 144, b3 = (sms * 7) / 144;
     // weight gradients only: the B2R kind has half the work, 10/4/7 was the best of a sweep (132 against 140 us)
     if (dx == nullptr) { b1 = (sms * 10) / 144; b2 = (sms * 4) / 144; b3 = (sms * 7) / 144; }
 #ifdef MONARCH_TRACE
