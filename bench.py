@@ -34,7 +34,9 @@ FALLBACK_BF16_TFLOPS = 1590.0
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--steps", type=int, default=None,
+                    help="timed steps (default: 1000, so that the timed region spans several clock samples; "
+                         "100 for workload 7; 30 for --impl reference)")
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=3, choices=[1, 2, 3, 4, 5, 6, 7, 8],
@@ -46,7 +48,10 @@ def parse_args():
                     "(profiling aid; the default step runs them all)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    return ap.parse_args()
+    args = ap.parse_args()
+    if args.steps is None:
+        args.steps = 30 if args.impl == "reference" else (100 if args.workload == 7 else 1000)
+    return args
 
 
 # ----------------------------------------------------------------------------- accounting
