@@ -50,9 +50,18 @@ static __device__ __forceinline__ float gelu_fast_exp(float a)               // 
     const float a2 = fminf(a * a, 64.0f);
     float t = fmaf(a2, 0.0010142630198970437f, -0.10677572339773178f);     // -2 log2(e) * (c2 a^2 + c1)
     t = fmaf(a2, t, -2.301121234893799f);
-    return exp2f(a * t);
+    // flush-to-zero forms: no range fix-up code around the two MUFU operations (the exponent is at most 40 for
+    // |a| <= 8; beyond that 2^x overflows to inf or flushes to 0 and the sigmoid saturates to 0 or 1, as it should)
+    float e;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(a * t));
+    return e;
 }
-static __device__ __forceinline__ float gelu_fast(float a) { return __fdividef(a, 1.0f + gelu_fast_exp(a)); }
+static __device__ __forceinline__ float gelu_fast(float a)
+{
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + gelu_fast_exp(a)));
+    return a * r;
+}
 
 // d/da GELU(a) = Phi(a) + a phi(a) with Phi from the same sigmoid (|Phi error| <= 5.1e-5) and the normal
 // density phi evaluated directly: |error| <= 5.1e-5, for results that are rounded to bf16.
