@@ -1,0 +1,555 @@
+// m = 128 (n = 16384), bf16: the Monarch multiply and its adjoints as chains of block GEMMs whose stride
+// permutations cost nothing on chip.
+//
+// The permutation between the two stages of Section 3.3 (steps 1-3) moves 2-byte elements: u'[t][j][k] = u[t][k][j].
+// With 128 x 128 blocks neither the accumulators of 16 blocks (for 32-byte pieces) nor a token tile of u (32 KB per
+// token) fit an SM, so the permuted intermediate cannot be assembled on chip.  What can be chosen freely is which
+// index of an intermediate is contiguous in memory: the tensor cores read an operand either with its contraction
+// index contiguous ("K-major") or with its row/column index contiguous ("MN-major").  All intermediates here are
+// stored TOKEN-INNERMOST in tiles of 128 tokens, as [tile][p][q][t]:
+//     u'  = [tile][j][k][t]    written by stage 1 block k as rows j of D_k[j][t]   (q = k fixed, 256-byte rows)
+//                              read by stage 2 block j as the 32 KB slab [k][t]    (p = j fixed), an MN-major operand
+//     w'  = [tile][l][j][t]    written by stage 2 block j as rows l of D_j[l][t]; a last pass transposes the
+//                              128 x 128 (j, t) planes into y[t][l*128 + j] - both sides in 256-byte rows.
+// So every global access of the whole chain is a 128- or 256-byte row, the inner permutation of Def. 3.1 is the
+// choice of a store box, and the outer one is a plane transpose through shared memory (ldmatrix.trans / stmatrix).
+// The adjoints reverse the chain (transpose dy into dw' = [tile][l][j][t], du'[k][t] = L_j^T dw'_j written as
+// [tile][k][j][t], dx = du'_k^T R_k), and because the token index is contiguous the same tiles are K-major operands
+// of the token reductions dL_j = dw'_j u'_j^T and dR_k = du'_k x_k, which ride along in the same kernels with their
+// accumulators resident in TMEM for all tiles of a block (one writer per block: deterministic sums).
+//
+// One kernel template serves all block products: persistent CTAs, the 32 KB weight block resident, token operands
+// through a TMA ring, tcgen05.mma 128 x 128 x 16 with two accumulator buffers in TMEM, epilogue through swizzled
+// staging tiles and TMA stores.
+#include "tc_common.cuh"
+
+namespace monarch {
+namespace tc {
+namespace {
+
+constexpr int kB = 128;                      // block size m
+constexpr int kOpBytes = 32768;              // one 128 x 128 bf16 operand: two boxes of [128 rows][64 columns]
+constexpr int kHalfBytes = 16384;
+constexpr int kThreads = 6 * 32;             // warps 0-3 epilogue, 4 loader, 5 MMA
+constexpr int kStagingBytes = 2 * kHalfBytes;
+
+enum { kLdX = 0, kLdP = 1, kLdQ = 2 };       // token-major tensor; [tile][p][q][t] with p fixed; with q fixed
+enum { kStX = 0, kStQ = 1 };
+
+struct ChainParams {
+    unsigned *status;
+    float *dW;                               // token-reduction output [block][128][128], added to
+    int ntiles;                              // 128-token tiles
+    int nblk;                                // blocks (128)
+};
+
+struct ChainBars {
+    uint64_t full[4], empty[4];
+    uint64_t acc_full[2], acc_empty[2];
+    uint64_t w_full[2], w_empty[2];
+    uint64_t wg_full, wg_empty;
+};
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *m, int c0, int c1, int c2, int c3, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(dst),
+        "l"(m), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap *m, uint32_t src, int c0, int c1, int c2, int c3)
+{
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(m), "r"(src),
+                 "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+                 : "memory");
+}
+
+// Load one 128 x 128 operand (two 64-column boxes) of block `blk`, tile `tile`.
+template <int KIND>
+__device__ __forceinline__ void load_operand(uint32_t dst, const CUtensorMap *m, int blk, int tile, uint32_t bar)
+{
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        if (KIND == kLdX) tma_load_2d(dst + h * kHalfBytes, m, blk * kB + h * 64, tile * 128, bar);
+        else if (KIND == kLdP) tma_load_4d(dst + h * kHalfBytes, m, h * 64, 0, blk, tile, bar);
+        else tma_load_4d(dst + h * kHalfBytes, m, h * 64, blk, 0, tile, bar);
+    }
+}
+
+// Descriptor of K-step s (16 of the contraction index) of an operand tile: with the contraction index along the
+// 128-byte rows (K-major: four steps per box) or down the rows (MN-major: 16 rows = 2 KB per step, the two boxes
+// side by side along the row/column index).
+__device__ __forceinline__ uint64_t op_desc(uint32_t base, bool mn, int s)
+{
+    return mn ? make_smem_desc(base + s * 2048, kHalfBytes, 1024, kSwizzle128)
+              : make_smem_desc(base + (s >> 2) * kHalfBytes + (s & 3) * 32, 16, 1024, kSwizzle128);
+}
+
+// D = A B^T per (block, tile).  W_IS_A: the weight block is the A operand (rows of D = weight rows or columns,
+// columns of D = tokens) else the token operand T0 is A (rows of D = tokens).  *_MN: operand read MN-major.
+// WG: additionally dW[blk] += T0 (rows as M, tokens as K) x T1 (T1_MN ? token-major natural tensor : [..][t]).
+// MAIN = false drops the main product (weight gradients only).
+template <int T0_LD, bool W_IS_A, bool W_MN, bool T0_MN, int ST, bool WG, int T1_LD, bool T1_MN, bool MAIN, int SLOTS>
+__global__ void __launch_bounds__(kThreads, 1)
+chain_gemm_kernel(const __grid_constant__ CUtensorMap tm_t0, const __grid_constant__ CUtensorMap tm_t1,
+                  const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_out, const ChainParams p)
+{
+    constexpr int kSlotBytes = WG ? 2 * kOpBytes : kOpBytes;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) ChainBars bars;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int dead_s;
+
+    const uint32_t w0 = (smem_u32(smem_raw) + 1023u) & ~1023u;          // two weight buffers
+    const uint32_t ring0 = w0 + 2 * kOpBytes;
+    const uint32_t staging0 = ring0 + SLOTS * kSlotBytes;                // two 16 KB staging tiles
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    volatile int *dead = &dead_s;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < SLOTS; ++s) {
+            mbar_init(smem_u32(&bars.full[s]), 1);
+            mbar_init(smem_u32(&bars.empty[s]), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(smem_u32(&bars.acc_full[a]), 1);
+            mbar_init(smem_u32(&bars.acc_empty[a]), 4);
+            mbar_init(smem_u32(&bars.w_full[a]), 1);
+            mbar_init(smem_u32(&bars.w_empty[a]), 1);
+        }
+        mbar_init(smem_u32(&bars.wg_full), 1);
+        mbar_init(smem_u32(&bars.wg_empty), 4);
+        fence_mbar_init();
+        dead_s = 0;
+        tma_prefetch_desc(&tm_t0); tma_prefetch_desc(&tm_w);
+        if (MAIN) tma_prefetch_desc(&tm_out);
+        if (WG) tma_prefetch_desc(&tm_t1);
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&tmem_base_s), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+
+    // items = (block, tile), block-major.  With a token reduction a CTA owns whole blocks (its accumulator lives in
+    // TMEM across the tiles of a block); otherwise the items are cut into equal contiguous runs.
+    long long i0, i1;
+    if (WG) {
+        i0 = (long long)p.nblk * blockIdx.x / gridDim.x * p.ntiles;
+        i1 = (long long)p.nblk * (blockIdx.x + 1) / gridDim.x * p.ntiles;
+    } else {
+        const long long total = (long long)p.nblk * p.ntiles;
+        i0 = total * blockIdx.x / gridDim.x;
+        i1 = total * (blockIdx.x + 1) / gridDim.x;
+    }
+    const uint32_t full0 = smem_u32(bars.full), empty0 = smem_u32(bars.empty);
+    const uint32_t accf0 = smem_u32(bars.acc_full), acce0 = smem_u32(bars.acc_empty);
+    const uint32_t wf0 = smem_u32(bars.w_full), we0 = smem_u32(bars.w_empty);
+    const uint32_t wgf = smem_u32(&bars.wg_full), wge = smem_u32(&bars.wg_empty);
+
+    if (warp == 4) {
+        // ------------------------------------------------------------ loader
+        if (lane == 0) {
+            uint32_t n = 0, wcount = 0;
+            int cur = -1;
+            for (long long i = i0; i < i1; ++i, ++n) {
+                const int blk = (int)(i / p.ntiles), tile = (int)(i % p.ntiles);
+                if (blk != cur) {
+                    const uint32_t wp = wcount & 1;
+                    if (!mbar_wait(we0 + wp * 8, ((wcount >> 1) & 1) ^ 1, p.status, dead, kErrSlotWait)) break;
+                    mbar_expect_tx(wf0 + wp * 8, kOpBytes);
+                    tma_load_2d(w0 + wp * kOpBytes, &tm_w, 0, blk * kB, wf0 + wp * 8);
+                    tma_load_2d(w0 + wp * kOpBytes + kHalfBytes, &tm_w, 64, blk * kB, wf0 + wp * 8);
+                    ++wcount;
+                    cur = blk;
+                }
+                const uint32_t s = n % SLOTS;
+                if (!mbar_wait(empty0 + s * 8, ((n / SLOTS) & 1) ^ 1, p.status, dead, kErrSlotWait)) break;
+                mbar_expect_tx(full0 + s * 8, kSlotBytes);
+                load_operand<T0_LD>(ring0 + s * kSlotBytes, &tm_t0, blk, tile, full0 + s * 8);
+                if (WG) load_operand<T1_LD>(ring0 + s * kSlotBytes + kOpBytes, &tm_t1, blk, tile, full0 + s * 8);
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc_main = W_IS_A ? make_idesc_bf16(128, 128, W_MN, T0_MN) : make_idesc_bf16(128, 128, T0_MN, W_MN);
+            constexpr uint32_t idesc_wg = make_idesc_bf16(128, 128, 0, T1_MN);
+            uint32_t n = 0, wcount = 0, wp = 0;
+            int cur = -1;
+            bool wg_first = true;
+            for (long long i = i0; i < i1; ++i, ++n) {
+                const int blk = (int)(i / p.ntiles);
+                if (blk != cur) {
+                    wp = wcount & 1;
+                    if (!mbar_wait(wf0 + wp * 8, (wcount >> 1) & 1, p.status, dead, kErrTmaWait)) break;
+                    if (WG) {
+                        // the previous block's sums have left TMEM
+                        if (!mbar_wait(wge, (wcount & 1) ^ 1, p.status, dead, kErrTmemWait)) break;
+                        wg_first = true;
+                    }
+                    ++wcount;
+                    cur = blk;
+                }
+                const uint32_t buf = n & 1, s = n % SLOTS;
+                if (MAIN) {
+                    if (!mbar_wait(acce0 + buf * 8, ((n >> 1) & 1) ^ 1, p.status, dead, kErrTmemWait)) break;
+                }
+                if (!mbar_wait(full0 + s * 8, (n / SLOTS) & 1, p.status, dead, kErrTmaWait)) break;
+                tc_fence_after();
+                const uint32_t t0 = ring0 + s * kSlotBytes, t1 = t0 + kOpBytes, w = w0 + wp * kOpBytes;
+                if (MAIN) {
+                    const uint32_t d = tmem_base + buf * 128;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint64_t dw = op_desc(w, W_MN, ks), dt = op_desc(t0, T0_MN, ks);
+                        mma_f16_ss(d, W_IS_A ? dw : dt, W_IS_A ? dt : dw, idesc_main, ks != 0);
+                    }
+                    mma_commit(accf0 + buf * 8);
+                }
+                if (WG) {
+                    const uint32_t d = tmem_base + 256;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)
+                        mma_f16_ss(d, op_desc(t0, false, ks), op_desc(t1, T1_MN, ks), idesc_wg, !(wg_first && ks == 0));
+                    wg_first = false;
+                }
+                mma_commit(empty0 + s * 8);
+                if (i + 1 == i1 || (int)((i + 1) / p.ntiles) != blk) {
+                    mma_commit(we0 + wp * 8);
+                    if (WG) mma_commit(wgf);
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 0-3 = TMEM lanes 32w..32w+31)
+        const int row = warp * 32 + lane;
+        const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+        uint32_t n = 0, nchunk = 0, nb = 0;
+        bool ok = true;
+        for (long long i = i0; ok && i < i1; ++i, ++n) {
+            const int blk = (int)(i / p.ntiles), tile = (int)(i % p.ntiles);
+            if (MAIN) {
+                const uint32_t buf = n & 1;
+                if (!mbar_wait(accf0 + buf * 8, (n >> 1) & 1, p.status, dead, kErrMmaWait)) break;
+                tc_fence_after();
+#pragma unroll 1
+                for (int h = 0; h < 2; ++h, ++nchunk) {
+                    const uint32_t stg = staging0 + (nchunk & 1) * kHalfBytes;
+                    // this staging tile is free once the store issued two chunks ago has read it
+                    if (threadIdx.x == 0) tma_store_wait_read<1>();
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    uint32_t v[4][16];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) tmem_ld16(lane_base + buf * 128 + h * 64 + q * 16, v[q]);
+                    tmem_ld_wait();
+                    if (h == 1) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(acce0 + buf * 8);
+                    }
+                    const uint32_t dst = stg + row * 128;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const uint32_t *w = &v[c >> 1][(c & 1) * 8];
+                        const uint32_t o0 = pack_bf16(__uint_as_float(w[0]), __uint_as_float(w[1]));
+                        const uint32_t o1 = pack_bf16(__uint_as_float(w[2]), __uint_as_float(w[3]));
+                        const uint32_t o2 = pack_bf16(__uint_as_float(w[4]), __uint_as_float(w[5]));
+                        const uint32_t o3 = pack_bf16(__uint_as_float(w[6]), __uint_as_float(w[7]));
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((c ^ (row & 7)) << 4)),
+                                     "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
+                    }
+                    fence_proxy_async_smem();
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    if (threadIdx.x == 0) {
+                        if (ST == kStX) tma_store_2d(&tm_out, stg, blk * kB + h * 64, tile * 128);
+                        else tma_store_4d(&tm_out, stg, h * 64, blk, 0, tile);
+                        tma_store_commit();
+                    }
+                }
+            }
+            if (WG && (i + 1 == i1 || (int)((i + 1) / p.ntiles) != blk)) {
+                // the block's token sums are complete: add them to dW[blk] (one writer per element)
+                if (!mbar_wait(wgf, nb & 1, p.status, dead, kErrMmaWait)) break;
+                tc_fence_after();
+                float *out = p.dW + ((size_t)blk * kB + row) * kB;
+#pragma unroll 1
+                for (int c = 0; c < kB; c += 16) {
+                    uint32_t v[16];
+                    tmem_ld16(lane_base + 256 + c, v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(out + c + e * 4),
+                                     "f"(__uint_as_float(v[e * 4])), "f"(__uint_as_float(v[e * 4 + 1])),
+                                     "f"(__uint_as_float(v[e * 4 + 2])), "f"(__uint_as_float(v[e * 4 + 3]))
+                                     : "memory");
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(wge);
+                ++nb;
+            }
+        }
+        if (MAIN && threadIdx.x == 0) tma_store_wait_all<0>();
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem_base, 512);
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// 128 x 128 plane transposes between a token-major tensor v[t][p*128 + c] and planes [tile][p][c][t]:
+// TO_PLANES = false: planes -> token-major (the outer P of step 3 of the forward pass), true: the reverse (first step
+// of the adjoint).  In and out are each two boxes of [128 rows][64 columns] with the 128-byte swizzle; four warps
+// move 8 x 8 tiles with ldmatrix.trans / stmatrix (conflict-free under the swizzle).
+constexpr int kTrIn = 3, kTrOut = 2;
+constexpr int kTrThreads = 5 * 32;
+constexpr int kTrSmem = (kTrIn + kTrOut) * kOpBytes + 1024;
+
+struct TransposeParams {
+    unsigned *status;
+    int ntiles, nplanes;                 // planes per tile (128)
+};
+
+template <bool TO_PLANES>
+__global__ void __launch_bounds__(kTrThreads, 1)
+plane_transpose_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_constant__ CUtensorMap tm_out,
+                       const TransposeParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full[kTrIn], empty[kTrIn];
+    __shared__ int dead_s;
+    const uint32_t in0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t out0 = in0 + kTrIn * kOpBytes;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    volatile int *dead = &dead_s;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kTrIn; ++s) {
+            mbar_init(smem_u32(&full[s]), 1);
+            mbar_init(smem_u32(&empty[s]), 4);
+        }
+        fence_mbar_init();
+        dead_s = 0;
+        tma_prefetch_desc(&tm_in); tma_prefetch_desc(&tm_out);
+    }
+    __syncthreads();
+    const long long total = (long long)p.ntiles * p.nplanes;
+    const long long i0 = total * blockIdx.x / gridDim.x, i1 = total * (blockIdx.x + 1) / gridDim.x;
+
+    if (warp == 4) {
+        if (lane == 0) {
+            uint32_t n = 0;
+            for (long long i = i0; i < i1; ++i, ++n) {
+                const int tile = (int)(i / p.nplanes), pl = (int)(i % p.nplanes);
+                const uint32_t s = n % kTrIn;
+                if (!mbar_wait(smem_u32(&empty[s]), ((n / kTrIn) & 1) ^ 1, p.status, dead, kErrSlotWait)) break;
+                mbar_expect_tx(smem_u32(&full[s]), kOpBytes);
+                load_operand<TO_PLANES ? kLdX : kLdP>(in0 + s * kOpBytes, &tm_in, pl, tile, smem_u32(&full[s]));
+            }
+        }
+    } else {
+        uint32_t n = 0;
+        for (long long i = i0; i < i1; ++i, ++n) {
+            const int tile = (int)(i / p.nplanes), pl = (int)(i % p.nplanes);
+            const uint32_t s = n % kTrIn, ob = out0 + (n & 1) * kOpBytes, ib = in0 + s * kOpBytes;
+            // the output buffer used two items ago has been read by its stores
+            if (threadIdx.x == 0) tma_store_wait_read<1>();
+            if (!mbar_wait(smem_u32(&full[s]), (n / kTrIn) & 1, p.status, dead, kErrTmaWait)) break;
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            // in[r][c] -> out[c][r]; warp w takes source rows 32w..32w+31 (four row octets), all 16 column octets
+#pragma unroll 1
+            for (int ro = 0; ro < 4; ++ro) {
+                const int r0 = warp * 32 + ro * 8;
+#pragma unroll
+                for (int cq = 0; cq < 4; ++cq) {
+                    // four 8 x 8 tiles: source rows r0..r0+7, column octets 4cq..4cq+3
+                    const int mi = lane >> 3, ri = lane & 7;
+                    const int co = cq * 4 + mi;                                  // column octet 0..15
+                    const int sr = r0 + ri;
+                    const uint32_t src = ib + (co >> 3) * kHalfBytes + sr * 128 + (((co & 7) ^ (sr & 7)) << 4);
+                    uint32_t a, b, c, d;
+                    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(a), "=r"(b), "=r"(c), "=r"(d) : "r"(src) : "memory");
+                    // destination tile of matrix mi: rows co*8..co*8+7 (source columns), column octet r0/8
+                    const int dr = co * 8 + ri, dco = r0 >> 3;
+                    const uint32_t dst = ob + (dco >> 3) * kHalfBytes + dr * 128 + (((dco & 7) ^ (dr & 7)) << 4);
+                    asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(a),
+                                 "r"(b), "r"(c), "r"(d) : "memory");
+                }
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&empty[s]));
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (threadIdx.x == 0) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    if (TO_PLANES) tma_store_4d(&tm_out, ob + h * kHalfBytes, h * 64, 0, pl, tile);
+                    else tma_store_2d(&tm_out, ob + h * kHalfBytes, pl * kB + h * 64, tile * 128);
+                }
+                tma_store_commit();
+            }
+        }
+        if (threadIdx.x == 0) tma_store_wait_all<0>();
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+struct Maps {
+    CUtensorMap x2d;       // token-major [tokens][n], box 128 rows x 64 columns
+    CUtensorMap p4d;       // planes [tile][p][q][t], box = rows q of one p
+    CUtensorMap q4d;       // planes, box = rows p of one q
+};
+
+int map_tokens(CUtensorMap *m, const void *v, int64_t tokens)
+{
+    return encode_tmap_2d(m, v, (uint64_t)tokens, (uint64_t)kB * kB, (uint64_t)kB * kB * 2, 128, 64, 128);
+}
+int map_weights(CUtensorMap *m, const void *W)
+{
+    return encode_tmap_2d(m, W, (uint64_t)kB * kB, kB, kB * 2, 128, 64, 128);
+}
+int map_planes(CUtensorMap *m, const void *v, int ntiles, bool fixed_p)
+{
+    const uint64_t dims[4] = {128, 128, 128, (uint64_t)ntiles}, strides[3] = {256, 32768, 4194304};
+    const uint32_t box_p[4] = {64, 128, 1, 1}, box_q[4] = {64, 1, 128, 1};
+    return encode_tmap_nd(m, v, 2, 4, dims, strides, fixed_p ? box_p : box_q, 128);
+}
+
+int device_sms(int *sms)
+{
+    int dev = 0;
+    MONARCH_CUDA_TRY(cudaGetDevice(&dev));
+    MONARCH_CUDA_TRY(cudaDeviceGetAttribute(sms, cudaDevAttrMultiProcessorCount, dev));
+    return MONARCH_OK;
+}
+
+template <int T0_LD, bool W_IS_A, bool W_MN, bool T0_MN, int ST, bool WG, int T1_LD, bool T1_MN, bool MAIN>
+int launch_gemm(const CUtensorMap &t0, const CUtensorMap &t1, const CUtensorMap &w, const CUtensorMap &out, float *dW,
+                int ntiles, unsigned *status, cudaStream_t s)
+{
+    constexpr int SLOTS = WG ? 2 : 3;
+    constexpr int smem = 2 * kOpBytes + SLOTS * (WG ? 2 : 1) * kOpBytes + kStagingBytes + 1024;
+    auto kern = chain_gemm_kernel<T0_LD, W_IS_A, W_MN, T0_MN, ST, WG, T1_LD, T1_MN, MAIN, SLOTS>;
+    int sms = 0;
+    MONARCH_TRY(device_sms(&sms));
+    MONARCH_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    ChainParams p;
+    p.status = status;
+    p.dW = dW;
+    p.ntiles = ntiles;
+    p.nblk = kB;
+    long long grid = WG ? kB : (long long)kB * ntiles;
+    if (grid > sms) grid = sms;
+    kern<<<(unsigned)grid, kThreads, smem, s>>>(t0, t1, w, out, p);
+    note_launch();
+    MONARCH_CUDA_TRY(cudaGetLastError());
+    return MONARCH_OK;
+}
+
+template <bool TO_PLANES>
+int launch_transpose(const CUtensorMap &in, const CUtensorMap &out, int ntiles, unsigned *status, cudaStream_t s)
+{
+    int sms = 0;
+    MONARCH_TRY(device_sms(&sms));
+    MONARCH_CUDA_TRY(cudaFuncSetAttribute(plane_transpose_kernel<TO_PLANES>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTrSmem));
+    TransposeParams p;
+    p.status = status;
+    p.ntiles = ntiles;
+    p.nplanes = kB;
+    long long grid = (long long)ntiles * kB;
+    if (grid > sms) grid = sms;
+    plane_transpose_kernel<TO_PLANES><<<(unsigned)grid, kTrThreads, kTrSmem, s>>>(in, out, p);
+    note_launch();
+    MONARCH_CUDA_TRY(cudaGetLastError());
+    return MONARCH_OK;
+}
+
+size_t planes_bytes(int64_t tokens) { return (size_t)((tokens + 127) / 128) * 128 * kB * kB * 2; }
+
+}  // namespace
+}  // namespace tc
+
+// Forward workspace: [status][u' planes][w' planes]; the backward call reads u' from it.
+size_t chain_fwd_m128_workspace_bytes(int64_t tokens) { return MONARCH_STATUS_BYTES + 2 * tc::planes_bytes(tokens); }
+const void *chain_fwd_m128_saved_u(const void *fwd_ws) { return (const char *)fwd_ws + MONARCH_STATUS_BYTES; }
+// Backward workspace: [status][dw' planes][du' planes][u' planes (when the forward call's are not passed)]
+size_t chain_bwd_m128_workspace_bytes(int64_t tokens) { return MONARCH_STATUS_BYTES + 3 * tc::planes_bytes(tokens); }
+
+// y = P L P^T R x (Def. 3.1; Section 3.3 steps 1-3) in three launches.
+int chain_fwd_m128(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws, cudaStream_t s)
+{
+    using namespace tc;
+    if (tokens == 0) return MONARCH_OK;
+    if (tokens > (int64_t)1 << 30) return MONARCH_ERR_UNSUPPORTED;
+    const int ntiles = (int)((tokens + 127) / 128);
+    unsigned *status = (unsigned *)ws;
+    char *up = (char *)ws + MONARCH_STATUS_BYTES, *wp = up + planes_bytes(tokens);
+    CUtensorMap mx, my, mR, mL, mu_q, mu_p, mw_q, mw_p;
+    MONARCH_TRY(map_tokens(&mx, x, tokens));
+    MONARCH_TRY(map_tokens(&my, y, tokens));
+    MONARCH_TRY(map_weights(&mR, R));
+    MONARCH_TRY(map_weights(&mL, L));
+    MONARCH_TRY(map_planes(&mu_q, up, ntiles, false));
+    MONARCH_TRY(map_planes(&mu_p, up, ntiles, true));
+    MONARCH_TRY(map_planes(&mw_q, wp, ntiles, false));
+    MONARCH_TRY(map_planes(&mw_p, wp, ntiles, true));
+    // step 1 + inner permutation: D_k[j][t] = sum_i R[k][j][i] x[t][k*128+i]  ->  u'[tile][j][k][t]
+    MONARCH_TRY((launch_gemm<kLdX, true, false, false, kStQ, false, kLdX, false, true>(mx, mx, mR, mu_q, nullptr, ntiles, status, s)));
+    // step 2: D_j[l][t] = sum_k L[j][l][k] u'[tile][j][k][t]  ->  w'[tile][l][j][t]
+    MONARCH_TRY((launch_gemm<kLdP, true, false, true, kStQ, false, kLdX, false, true>(mu_p, mu_p, mL, mw_q, nullptr, ntiles, status, s)));
+    // step 3 (outer permutation): y[t][l*128+j] = w'[tile][l][j][t]
+    return launch_transpose<false>(mw_p, my, ntiles, status, s);
+}
+
+// dx = M^T dy, dL, dR (the adjoints of steps 1-3); saved_up = u' planes of the forward call or null (recomputed).
+// dL and dR are added to: the caller zeroes them when they are not to accumulate.
+int chain_bwd_m128(const void *x, const void *dy, const void *L, const void *R, const void *saved_up, void *dx, float *dL,
+                   float *dR, int want_dx, int want_dw, int64_t tokens, void *ws, cudaStream_t s)
+{
+    using namespace tc;
+    if (tokens == 0) return MONARCH_OK;
+    if (tokens > (int64_t)1 << 30) return MONARCH_ERR_UNSUPPORTED;
+    const int ntiles = (int)((tokens + 127) / 128);
+    unsigned *status = (unsigned *)ws;
+    char *dwp = (char *)ws + MONARCH_STATUS_BYTES, *dup = dwp + planes_bytes(tokens), *up_own = dup + planes_bytes(tokens);
+    CUtensorMap mx, mdy, mdx, mR, mL, mdw_p, mdw_q, mdu_q, mdu_p, mu_q, mu_p;
+    MONARCH_TRY(map_tokens(&mdy, dy, tokens));
+    MONARCH_TRY(map_weights(&mR, R));
+    MONARCH_TRY(map_weights(&mL, L));
+    MONARCH_TRY(map_planes(&mdw_p, dwp, ntiles, true));
+    MONARCH_TRY(map_planes(&mdw_q, dwp, ntiles, false));
+    MONARCH_TRY(map_planes(&mdu_q, dup, ntiles, false));
+    MONARCH_TRY(map_planes(&mdu_p, dup, ntiles, true));
+    if (want_dx) MONARCH_TRY(map_tokens(&mdx, dx, tokens));
+    else mdx = mdy;
+    if (want_dw) {
+        MONARCH_TRY(map_tokens(&mx, x, tokens));
+        if (saved_up == nullptr) {
+            MONARCH_TRY(map_planes(&mu_q, up_own, ntiles, false));
+            MONARCH_TRY((launch_gemm<kLdX, true, false, false, kStQ, false, kLdX, false, true>(mx, mx, mR, mu_q, nullptr, ntiles, status, s)));
+            saved_up = up_own;
+        }
+        MONARCH_TRY(map_planes(&mu_p, saved_up, ntiles, true));
+    }
+    // dw'[tile][l][j][t] = dy[t][l*128+j]
+    MONARCH_TRY(launch_transpose<true>(mdy, mdw_p, ntiles, status, s));
+    // du'[tile][k][j][t] = sum_l L[j][l][k] dw'[tile][l][j][t]   (+ dL[j][l][k] += sum_t dw'[..][l][j][t] u'[..][j][k][t])
+    if (want_dw)
+        MONARCH_TRY((launch_gemm<kLdQ, true, true, true, kStQ, true, kLdP, false, true>(mdw_q, mu_p, mL, mdu_q, dL, ntiles, status, s)));
+    else
+        MONARCH_TRY((launch_gemm<kLdQ, true, true, true, kStQ, false, kLdP, false, true>(mdw_q, mdw_q, mL, mdu_q, nullptr, ntiles, status, s)));
+    // dx[t][k*128+i] = sum_j du'[tile][k][j][t] R[k][j][i]        (+ dR[k][j][i] += sum_t du'[..][k][j][t] x[t][k*128+i])
+    if (want_dw && want_dx)
+        return launch_gemm<kLdP, false, true, true, kStX, true, kLdX, true, true>(mdu_p, mx, mR, mdx, dR, ntiles, status, s);
+    if (want_dw)
+        return launch_gemm<kLdP, false, true, true, kStX, true, kLdX, true, false>(mdu_p, mx, mR, mdx, dR, ntiles, status, s);
+    return launch_gemm<kLdP, false, true, true, kStX, false, kLdX, true, true>(mdu_p, mdu_p, mR, mdx, nullptr, ntiles, status, s);
+}
+
+}  // namespace monarch

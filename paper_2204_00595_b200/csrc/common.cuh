@@ -94,16 +94,21 @@ int tc_staged_mlp_fwd(const void *x, const void *L1, const void *R1, const void 
                       cudaStream_t s);
 
 
-// m = 128 through the GEMM kernels of the general class plus permutation passes (tc_bwd.cu)
-int gemm_permute_fwd_m128(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws, cudaStream_t s);
+// m = 128 as chains of block GEMMs on token-innermost planes (chain_m128.cu)
+size_t chain_fwd_m128_workspace_bytes(int64_t tokens);
+size_t chain_bwd_m128_workspace_bytes(int64_t tokens);
+int chain_fwd_m128(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws, cudaStream_t s);
+// saved_up: the u' planes the forward call left in its workspace (chain_fwd_m128_saved_u), or null; dL, dR are added to
+int chain_bwd_m128(const void *x, const void *dy, const void *L, const void *R, const void *saved_up, void *dx, float *dL,
+                   float *dR, int want_dx, int want_dw, int64_t tokens, void *ws, cudaStream_t s);
+const void *chain_fwd_m128_saved_u(const void *fwd_ws);
 
 // ---- backward as a chain of tensor-core launches (bf16; dx for m >= 32, dL/dR for m = 128), tc_bwd.cu ----
 size_t tc_staged_bwd_workspace_bytes(int64_t tokens, int m);
-// saved_up: for m = 128, u' = P blockdiag(R) x left by the forward call (gemm_permute_fwd_m128_saved_u), or null
+// saved_up: for m = 128, the u' planes left by the forward call (chain_fwd_m128_saved_u), or null
 int tc_staged_bwd(const void *x, const void *dy, const void *L, const void *R, void *dx, float *dL, float *dR,
                   int accumulate, int want_dx, int want_dw, int64_t tokens, int m, void *ws, cudaStream_t s,
                   const void *saved_up = nullptr);
-const void *gemm_permute_fwd_m128_saved_u(const void *fwd_ws, int64_t tokens);
 
 // ---- forward for m = 16 in one launch on the CUDA cores, both dtypes (fused_m16.cu); no workspace use ----
 int fused_fwd_m16(const void *x, const void *L, const void *R, void *y, int64_t tokens, int dtype, cudaStream_t s);

@@ -153,8 +153,7 @@ size_t monarch_workspace_bytes(int op, int64_t tokens, int32_t n, int32_t m, int
     if (which < 0) return 0;
     if (which == kTcStaged && op != MONARCH_OP_FWD && op != MONARCH_OP_MLP_FWD)
         return tc_staged_bwd_workspace_bytes(tokens, m);
-    if (which == kTcStaged && op == MONARCH_OP_FWD && m == 128)       // GEMM and permutation passes alternate
-        return MONARCH_STATUS_BYTES + 2 * round256((size_t)tokens * n * esize(dtype));
+    if (which == kTcStaged && op == MONARCH_OP_FWD && m == 128) return chain_fwd_m128_workspace_bytes(tokens);
     if (op == MONARCH_OP_BWD) {
         if (which == kFused) return fused_bwd_m64_workspace_bytes(tokens);
         const size_t a = staged_workspace_bytes(MONARCH_OP_BWD_DX, tokens, n, m, dtype);
@@ -258,7 +257,7 @@ int monarch_bwd(const void *x, const void *dy, const void *L, const void *R, con
     if (which == kTcStaged) {
         const bool saved = fwd_workspace != nullptr && m == 128 && pick(MONARCH_OP_FWD, m, dtype) == kTcStaged;
         return tc_staged_bwd(x, dy, L, R, dx, dL, dR, accumulate, 1, 1, tokens, m, workspace, s,
-                             saved ? gemm_permute_fwd_m128_saved_u(fwd_workspace, tokens) : nullptr);
+                             saved ? chain_fwd_m128_saved_u(fwd_workspace) : nullptr);
     }
     MONARCH_TRY(staged_bwd_dx(dy, L, R, dx, tokens, m, dtype, workspace, s));
     return staged_bwd_dw(x, dy, L, R, dL, dR, accumulate, tokens, m, dtype, workspace, s);

@@ -286,64 +286,12 @@ Layout carve(void *ws, int64_t tokens, int m)
 }  // namespace
 }  // namespace tc
 
-// Workspace: [status][z][du][u'][L^T][R^T]; for m = 128 the two weight areas hold a fourth token buffer instead
+// Workspace: [status][z][du][u'][L^T][R^T]; m = 128 has its own layout (chain_m128.cu)
 size_t tc_staged_bwd_workspace_bytes(int64_t tokens, int m)
 {
+    if (m == 128) return chain_bwd_m128_workspace_bytes(tokens);
     const size_t act = tc::align256((size_t)tokens * m * m * 2), wb = tc::align256((size_t)m * m * m * 2);
-    return MONARCH_STATUS_BYTES + 3 * act + (m == 128 ? (act > 2 * wb ? act : 2 * wb) : 2 * wb);
-}
-
-// m = 128: every block product is a GEMM of the general class's kernels (rect_tc.cu: 128 x 128 blocks are large
-// enough for 128-wide MMAs and the kernel runs at the HBM limit), the stride permutation a pass of its own:
-//   forward  u = blockdiag(R) x, u' = P u, w = blockdiag(L) u', y = P w
-//   backward z = P dy, du' = blockdiag(L)^T z, du = P du', dx = blockdiag(R)^T du,
-//            dR = sum_t du (x) x, dL = sum_t z (x) u'  (u' recomputed, or read from the forward call's workspace)
-int gemm_permute_fwd_m128(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws, cudaStream_t s)
-{
-    constexpr int m = 128;
-    unsigned *status = (unsigned *)ws;
-    const size_t act = tc::align256((size_t)tokens * m * m * 2);
-    char *a = (char *)ws + MONARCH_STATUS_BYTES, *b = a + act;
-    MONARCH_TRY(rect_stage1_tc(x, R, a, tokens, m, m, m, status, s));
-    MONARCH_TRY(tc::permute(a, b, m, tokens, s));
-    MONARCH_TRY(rect_stage1_tc(b, L, a, tokens, m, m, m, status, s));
-    return tc::permute(a, y, m, tokens, s);
-}
-
-// u' = P blockdiag(R) x as the forward call above leaves it in its workspace (the second token buffer)
-const void *gemm_permute_fwd_m128_saved_u(const void *fwd_ws, int64_t tokens)
-{
-    return (const char *)fwd_ws + MONARCH_STATUS_BYTES + tc::align256((size_t)tokens * 128 * 128 * 2);
-}
-
-int gemm_permute_bwd_m128(const void *x, const void *dy, const void *L, const void *R, const void *saved_up, void *dx,
-                          float *dL, float *dR, int accumulate, int want_dx, int want_dw, int64_t tokens, void *ws,
-                          cudaStream_t s)
-{
-    constexpr int m = 128;
-    unsigned *status = (unsigned *)ws;
-    const size_t act = tc::align256((size_t)tokens * m * m * 2);
-    char *z = (char *)ws + MONARCH_STATUS_BYTES, *dup = z + act, *du = dup + act, *up = du + act;
-    if (want_dw && !accumulate) {
-        const size_t gb = (size_t)m * m * m * sizeof(float);
-        MONARCH_CUDA_TRY(cudaMemsetAsync(dL, 0, gb, s));
-        MONARCH_CUDA_TRY(cudaMemsetAsync(dR, 0, gb, s));
-    }
-    if (tokens == 0) return MONARCH_OK;
-    MONARCH_TRY(tc::permute(dy, z, m, tokens, s));
-    MONARCH_TRY(rect_stage1_adjoint_tc(z, L, dup, tokens, m, m, m, status, s));            // du'[t][j][k]
-    MONARCH_TRY(tc::permute(dup, du, m, tokens, s));                                       // du[t][k][j]
-    if (want_dx) MONARCH_TRY(rect_stage1_adjoint_tc(du, R, dx, tokens, m, m, m, status, s));
-    if (want_dw) {
-        if (saved_up == nullptr) {
-            MONARCH_TRY(rect_stage1_tc(x, R, dup, tokens, m, m, m, status, s));            // u (du' is dead)
-            MONARCH_TRY(tc::permute(dup, up, m, tokens, s));                               // u'[t][j][k]
-            saved_up = up;
-        }
-        MONARCH_TRY(rect_wgrad_R_tc(du, x, dR, tokens, m, m, m, status, s));
-        MONARCH_TRY(rect_wgrad_R_tc(z, saved_up, dL, tokens, m, m, m, status, s));
-    }
-    return MONARCH_OK;
+    return MONARCH_STATUS_BYTES + 3 * act + 2 * wb;
 }
 
 // want_dx / want_dw select the outputs; dW needs m = 128 (the token-reduction kernel's block size)
@@ -353,8 +301,15 @@ int tc_staged_bwd(const void *x, const void *dy, const void *L, const void *R, v
 {
     using namespace tc;
     if (want_dw && m != 128) return MONARCH_ERR_UNSUPPORTED;
-    if (m == 128)
-        return gemm_permute_bwd_m128(x, dy, L, R, saved_up, dx, dL, dR, accumulate, want_dx, want_dw, tokens, ws, s);
+    if (m == 128) {
+        // chain of block GEMMs on token-innermost planes (chain_m128.cu); dL, dR are added to
+        if (want_dw && !accumulate) {
+            const size_t gb = (size_t)m * m * m * sizeof(float);
+            MONARCH_CUDA_TRY(cudaMemsetAsync(dL, 0, gb, s));
+            MONARCH_CUDA_TRY(cudaMemsetAsync(dR, 0, gb, s));
+        }
+        return chain_bwd_m128(x, dy, L, R, saved_up, dx, dL, dR, want_dx, want_dw, tokens, ws, s);
+    }
     unsigned *status = (unsigned *)ws;
     const Layout l = carve(ws, tokens, m);
     if (want_dw && !accumulate) {

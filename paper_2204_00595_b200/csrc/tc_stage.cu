@@ -288,8 +288,10 @@ int encode_tmap_nd(CUtensorMap *out, const void *base, int elem_bytes, int rank,
                                                    : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     const CUresult r = fn(out, dt, (cuuint32_t)rank, const_cast<void *>(base), d, st, b, es,
                           CU_TENSOR_MAP_INTERLEAVE_NONE,
-                          swizzle_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE,
-                          CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                          swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                          : swizzle_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                          swizzle_bytes == 128 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B : CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? MONARCH_OK : MONARCH_ERR_CUDA;
 }
 
@@ -300,7 +302,7 @@ int encode_tmap_nd(CUtensorMap *out, const void *base, int elem_bytes, int rank,
 int tc_staged_fwd(const void *x, const void *L, const void *R, void *y, int64_t tokens, int m,
                   void *ws, cudaStream_t s)
 {
-    if (m == 128) return gemm_permute_fwd_m128(x, L, R, y, tokens, ws, s);   // workspace: two token buffers
+    if (m == 128) return chain_fwd_m128(x, L, R, y, tokens, ws, s);          // workspace: two plane buffers
     unsigned *status = (unsigned *)ws;
     void *u = (char *)ws + MONARCH_STATUS_BYTES;
     MONARCH_TRY(tc::tc_stage(m, x, R, u, nullptr, 0, tokens, status, s));

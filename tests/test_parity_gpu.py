@@ -604,7 +604,7 @@ def test_cplx_fwd(P, impl, m, T, dtype, adjoint):
     yh = to_host64(y)
     # a problem instance is a token's complex row: compare re and im side by side
     assert_close(np.concatenate([yh[0], yh[1]], axis=1), np.concatenate([ref.real, ref.imag], axis=1), dtype,
-                 f"complex y adjoint={adjoint}", scale=1.5 if dtype == "bf16" else 1.0)
+                 f"complex y adjoint={adjoint}")
     _check_guard(yf, "complex y")
 
 
@@ -628,7 +628,7 @@ def test_cplx_dft_closed_form(P):
     ref = np.fft.fft(xc, axis=1)
     yh = to_host64(y)
     assert_close(np.concatenate([yh[0], yh[1]], axis=1), np.concatenate([ref.real, ref.imag], axis=1), "f32",
-                 "DFT", scale=3.0)          # the factors themselves are rounded to fp32 (1e-7 each, n terms)
+                 "DFT")
 
 
 # ----------------------------------------------------------------- dense <-> factors (Eq. 2, Algorithm 1)
@@ -672,11 +672,11 @@ def test_project_recovers_monarch_and_planted(P, m, dtype):
     A = O.dense(d["L"], d["R"])
     A32 = round_to_storage(A.astype(np.float32), dtype)
     Lg, Rg = _project_gpu(P, A32, m, dtype)
-    assert_close(O.dense(Lg, Rg), A32.astype(np.float64), dtype, "project(monarch)", scale=2.0)
+    assert_close(O.dense(Lg, Rg), A32.astype(np.float64), dtype, "project(monarch)")
     noisy = round_to_storage((A + 0.02 / m * rng.standard_normal(A.shape)).astype(np.float32), dtype)
     Lg, Rg = _project_gpu(P, noisy, m, dtype)
     Lo, Ro = O.project(noisy.astype(np.float64), m)
-    assert_close(O.dense(Lg, Rg), O.dense(Lo, Ro), dtype, "project(planted)", scale=2.0)
+    assert_close(O.dense(Lg, Rg), O.dense(Lo, Ro), dtype, "project(planted)")
 
 
 @pytest.mark.parametrize("m", [16, 64])
@@ -718,9 +718,20 @@ def _sample_tokens(T, count, seed):
     return np.array(sorted(idx))
 
 
+def _tile_rows(T, seed, tile=64):
+    """Both edges and one random interior row of every 64-token tile (the finest token tiling any kernel uses;
+    coarser tiles and every CTA / team residue are unions of these)."""
+    rng = np.random.default_rng(seed)
+    idx = set()
+    for t0 in range(0, T, tile):
+        t1 = min(t0 + tile, T)
+        idx.update({t0, t1 - 1, int(rng.integers(t0, t1))})
+    return np.array(sorted(idx))
+
+
 @pytest.mark.parametrize("cfg", [1, 2, 3, 4])
 def test_workload_fwd_bwd(P, impl, cfg):
-    """Full-size workloads 1-4: y and dx on sampled token rows, dL and dR in full, plus the
+    """Full-size workloads 1-4: every row of y and dx and all of dL and dR against the oracle, plus the
     adjoint and Euler identities evaluated on the device results."""
     import torch
     c = CONFIGS[cfg]
@@ -734,11 +745,11 @@ def test_workload_fwd_bwd(P, impl, cfg):
     ws = P.Workspace(max(P.monarch_workspace_bytes(op, T, n, m, code) for op in ops))
     P.monarch_fwd(x, L, R, y, T, n, m, ws)
     torch.cuda.synchronize()
-    rows = _sample_tokens(T, 192, cfg)
-    ref_y = O.fwd(d["x"][rows], d["L"], d["R"])
+    rows = np.arange(T)
+    ref_y = O.fwd(d["x"], d["L"], d["R"])
     yh = to_host64(y)
     assert np.isfinite(yh).all()
-    assert_close(yh[rows], ref_y, c.dtype, f"cfg{cfg} y")
+    assert_close(yh, ref_y, c.dtype, f"cfg{cfg} y")
     if "bwd_dx" not in c.ops:
         assert P.monarch_last_device_status(ws) == 0
         return
@@ -788,7 +799,7 @@ def test_workload_mlp(P, impl):
     P.monarch_mlp_fwd(t["x"], t["L"], t["R"], t["b1"], t["L2"], t["R2"], t["b2"], y, T, n, m, ws)
     torch.cuda.synchronize()
     assert P.monarch_last_device_status(ws) == 0
-    rows = _sample_tokens(T, 256, 5)
+    rows = _tile_rows(T, 5)                      # 3 rows of each of the 512 tiles
     ref = O.mlp_fwd(d["x"][rows], d["L"], d["R"], d["b1"], d["L2"], d["R2"], d["b2"])
     yh = to_host64(y[torch.from_numpy(rows).cuda()])
     assert bool(torch.isfinite(y.float()).all())
@@ -822,7 +833,7 @@ def test_workload_mlp_bwd(P, impl):
     _call_mlp_bwd(P, t, bufs, 0, T, n, m, ws)
     torch.cuda.synchronize()
     assert P.monarch_last_device_status(ws) == 0
-    rows = _sample_tokens(T, 256, 55)
+    rows = _tile_rows(T, 55)
     ref = O.mlp_bwd(d["x"][rows], d["dy"][rows], d["L"], d["R"], d["b1"], d["L2"], d["R2"])
     dxh = to_host64(bufs["dx"][1])
     assert np.isfinite(dxh).all()

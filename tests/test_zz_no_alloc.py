@@ -3,14 +3,16 @@
 Some users of this library run where cudaMalloc is not an option (a serving loop whose
 device memory was fixed at start-up, a plug-in under a framework that owns the device heap).
 monarch_fwd_noalloc serves them from an array built into the library.  This file checks,
-through the C ABI, that it gives the same result as monarch_fwd on two calls in a row (the
-second call reuses the array the first one left dirty) and that it refuses what does not fit.
+through the C ABI, that it gives the same result as monarch_fwd - and as the CPU oracle - on
+two calls in a row (the second call reuses the array the first one left dirty) and that it
+refuses what does not fit.
 It is named to be collected last, so a failure here cannot hide another test's result.
 """
 import numpy as np
 import pytest
 
 import __graft_entry__ as entry
+from oracle import monarch_oracle as O
 from tests.helpers import assert_close, to_device, to_host64
 from paper_2204_00595_b200.inputs import round_to_storage
 
@@ -44,7 +46,8 @@ def test_noalloc_matches_fwd_on_two_calls_in_a_row(P, dtype):
         # scratch that still holds the first call's intermediate
         for m, T, seed in ((64, 300, 1), (32, 77, 2)):
             n = m * m
-            x, L, R = (to_device(a, dtype) for a in _inputs(m, T, dtype, seed))
+            host = _inputs(m, T, dtype, seed)
+            x, L, R = (to_device(a, dtype) for a in host)
             code = P.F32 if dtype == "f32" else P.BF16
             ws = P.Workspace(P.monarch_workspace_bytes(P.OP_FWD, T, n, m, code))
             y_ref = torch.full_like(x, float("nan"))
@@ -54,6 +57,7 @@ def test_noalloc_matches_fwd_on_two_calls_in_a_row(P, dtype):
             torch.cuda.synchronize()
             assert bool(torch.isfinite(y_new.float()).all())
             assert_close(to_host64(y_new), to_host64(y_ref), dtype, f"noalloc m={m}")
+            assert_close(to_host64(y_new), O.fwd(*host), dtype, f"noalloc m={m} against the oracle")
     finally:
         P.monarch_set_impl(prev)
 
