@@ -1,17 +1,20 @@
 #!/usr/bin/env python
 """Benchmark of the Monarch multiply hot path on B200.
 
-One step = one pass of the hot path over one batch of synthetic tokens of the chosen
-workload (default: workload 3, n=4096, m=64, 8192 tokens per GPU, bf16):
-    monarch_fwd (y) + monarch_bwd_dx (dx) + monarch_bwd_dw (dL, dR).
+One step = one pass of the hot path over one batch of synthetic tokens.  The headline is the largest
+forward + backward configuration, workload 4 (n = 16384, m = 128, 4096 tokens per GPU, bf16):
+    monarch_fwd (y), then monarch_bwd (dx, dL, dR in one call, reusing the intermediate the forward call left
+    in its workspace).
+The same JSON line carries, under "workloads", every other workload of the contract (1: fp32 forward, 2: m = 32
+forward, 3: m = 64 forward + backward, 5: feed-forward block) timed the same way with fewer steps.
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
-`--workload 5 --calls mlp_fwd,mlp_bwd` adds the backward of the feed-forward block; `--workload 6` times the
-forward of the general (rectangular) Monarch class.
+`--workload N` picks another headline; `--calls fwd,bwd_dx,bwd_dw` times the three separately exported calls;
+`--workload 5 --calls mlp_fwd,mlp_bwd` adds the backward of the feed-forward block; workloads 6-8 are the
+general (rectangular) class, the projection and the complex multiply.
 
-Launch for N > 1:  python -m torch.distributed.run --nnodes=1 --nproc-per-node N
-    --master-addr 127.0.0.1 --master-port P bench.py --gpus N --steps K --warmup W
-Tokens are sharded over ranks (fixed tokens per GPU: weak scaling); the only exchange is
-one all-reduce of the packed (dL, dR) gradients per step.
+`python bench.py --gpus N` starts N ranks itself (torch.distributed.run, one per GPU, NCCL); under an external
+launcher (WORLD_SIZE set) it is one of the ranks.  Tokens are sharded over ranks (fixed tokens per GPU: weak
+scaling); the only exchange is one all-reduce of the packed (dL, dR) gradients per step.
 """
 from __future__ import annotations
 
@@ -39,13 +42,16 @@ def parse_args():
                          "100 for workload 7; 30 for --impl reference)")
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=3, choices=[1, 2, 3, 4, 5, 6, 7, 8],
+    ap.add_argument("--workload", type=int, default=4, choices=[1, 2, 3, 4, 5, 6, 7, 8],
                     help="1-5: the square workloads; 6: the general (rectangular) class, forward only; "
                          "7: projection of a dense matrix onto the Monarch class + dense materialisation; "
                          "8: complex multiply (planar), y = M x then z = M^H y")
     ap.add_argument("--kernels", default="auto", choices=["auto", "staged", "fused"])
     ap.add_argument("--calls", default="", help="comma-separated subset of the workload's calls "
                     "(profiling aid; the default step runs them all)")
+    ap.add_argument("--no-side-workloads", dest="side_workloads", action="store_false",
+                    help="time only the headline workload (default: the other workloads of the contract are "
+                         "timed too, with fewer steps, and reported under \"workloads\")")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -192,19 +198,30 @@ def time_oracle(cfg, d, target_s=12.0, calls=None):
 # ----------------------------------------------------------------------------- main
 
 # Kernels behind each timed call, and the DRAM traffic one call generated under ncu (dram__bytes_read.sum +
-# dram__bytes_write.sum of the call's kernels, captured at workload 3's full size with this script).
+# dram__bytes_write.sum of the call's kernels; the note names the capture under profiles/ and says when the
+# value was scaled from a smaller token count).
 KERNELS_OF = {
+    (16, "f32", "fwd"): "fused_fwd_m16_kernel (1 launch)",
+    (32, "bf16", "fwd"): "fused_fwd_m32_kernel (1 launch)",
     (64, "bf16", "fwd"): "fused_fwd_m64_team_kernel (1 launch)",
     (64, "bf16", "bwd"): "fused_bwd_all_m64_kernel (1 launch, 2 memset nodes)",
+    (64, "bf16", "bwd_dx"): "fused_bwd_dx_m64_kernel (1 launch)",
+    (64, "bf16", "bwd_dw"): "fused_fwd_m64_kernel (stage 1 only) + fused_bwd_all_m64_kernel without dx "
+                            "(2 launches, 2 memset nodes)",
     (64, "bf16", "mlp_fwd"): "fused_fwd_m64_team_kernel (2 launches)",
     (64, "bf16", "mlp_bwd"): "fused_fwd_m64_team_kernel + mlp_act_kernel + fused_fwd_m64_kernel (stage 1 only) + "
                              "2 x fused_bwd_all_m64_kernel + mlp_dact_kernel + merge_status_kernel (7 launches)",
-    (32, "bf16", "fwd"): "fused_fwd_m32_kernel (1 launch)",
-    (64, "bf16", "bwd_dx"): "fused_bwd_dx_m64_kernel (1 launch)",
-    (64, "bf16", "bwd_dw"): "fused_fwd_m64_kernel (stage 1 only) + fused_bwd_dx_m64_kernel (stage 1 only) + "
-                            "fused_bwd_dw_m64_kernel (3 launches, 2 memset nodes)",
+    (128, "bf16", "fwd"): "chain_gemm_kernel x 2 + plane_transpose_kernel (3 launches)",
+    (128, "bf16", "bwd"): "plane_transpose_kernel + chain_gemm_kernel x 2 with the token reductions "
+                          "(3 launches, 2 memset nodes)",
+    (128, "bf16", "bwd_dx"): "plane_transpose_kernel + chain_gemm_kernel x 2 (3 launches)",
+    (128, "bf16", "bwd_dw"): "chain_gemm_kernel (stage 1) + plane_transpose_kernel + chain_gemm_kernel x 2 "
+                             "(4 launches, 2 memset nodes)",
 }
-NCU_TRAFFIC_MB = {(3, "fwd"): 150.0, (3, "bwd"): 365.6}
+NCU_TRAFFIC_MB = {
+    (3, "fwd"): (150.0, "profiles/fused_m64_step_workload3_ncu_full.md, full size"),
+    (3, "bwd"): (365.6, "profiles/fused_m64_step_workload3_ncu_full.md, full size"),
+}
 
 
 def main_rect(args):
@@ -258,7 +275,7 @@ def main_rect(args):
     import __graft_entry__ as entry
     entry.build()
     import paper_2204_00595_b200 as P
-    from tests.helpers import to_device
+    from paper_2204_00595_b200.inputs import to_device
     torch.cuda.set_device(local_rank)
     dist = None
     if world > 1:
@@ -504,7 +521,7 @@ def main_cplx(args):
     import __graft_entry__ as entry
     entry.build()
     import paper_2204_00595_b200 as P
-    from tests.helpers import to_device
+    from paper_2204_00595_b200.inputs import to_device
     torch.cuda.set_device(local_rank)
     dist = None
     if world > 1:
@@ -571,8 +588,154 @@ def main_cplx(args):
     return 0
 
 
+def launch_ranks(args):
+    """`python bench.py --gpus N` outside a launcher: start N ranks of this script under torch.distributed.run
+    (one per GPU, NCCL rendezvous on 127.0.0.1) and pass rank 0's JSON line through."""
+    import socket
+    import subprocess
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def default_calls(cfg, requested):
+    calls = list(cfg.ops)
+    if requested:
+        # the backward of the feed-forward block is an optional extra call of the workload that has the block
+        extra = ["mlp_bwd"] if "mlp_fwd" in calls else []
+        return [k for k in calls + extra if k in requested.split(",")]
+    if calls == ["fwd", "bwd_dx", "bwd_dw"]:
+        # default: the backward pass as one call (dx, dL, dR) that reuses the intermediate the forward
+        # call left in its workspace; --calls fwd,bwd_dx,bwd_dw times the three separate entry points
+        return ["fwd", "bwd"]
+    return calls
+
+
+def measure(P, torch, dist, cfg, calls, steps, warmup, rank, local_rank, sample_clocks):
+    """Time `steps` steps of `calls` on workload `cfg` (device-resident inputs, CUDA events on the launching
+    stream, rotating buffer sets).  Returns the step time, per-call figures and what the run needs to report."""
+    from paper_2204_00595_b200.inputs import make_inputs, to_device
+    n, m, T = cfg.n, cfg.m, cfg.tokens
+    code = P.F32 if cfg.dtype == "f32" else P.BF16
+    d = make_inputs(cfg.index, with_dy="mlp_bwd" in calls)   # every rank draws the same recipe, then offsets it
+    # Rotating sets of token tensors so that no launch finds its operands in L2 from the previous step: enough
+    # sets that together they hold at least 512 MB (each set of workloads 3-5 alone exceeds the 126 MB L2).
+    per_set = T * n * esize(cfg.dtype) * (4 if "dy" in d else 2)
+    SETS = max(2, min(8, -(-(512 << 20) // per_set))) if per_set < (1 << 30) else 1
+    sets = []
+    for s in range(SETS):
+        x = to_device(d["x"], cfg.dtype)
+        if s or rank:
+            x = torch.roll(x, shifts=17 * s + 5 * rank, dims=0).contiguous()
+        e = {"x": x, "y": torch.empty_like(x)}
+        if "dy" in d:
+            e["dy"] = torch.roll(to_device(d["dy"], cfg.dtype), shifts=3 * s + rank, dims=0).contiguous()
+            e["dx"] = torch.empty_like(x)
+        sets.append(e)
+    W = {k: to_device(d[k], cfg.dtype) for k in ("L", "R", "L2", "R2", "b1", "b2") if k in d}
+    grads = torch.zeros(2, m, m, m, dtype=torch.float32, device="cuda")   # packed (dL, dR)
+    mlp_grads = ([torch.zeros(m, m, m, dtype=torch.float32, device="cuda") for _ in range(4)] +
+                 [torch.zeros(n, dtype=torch.float32, device="cuda") for _ in range(2)]) if "mlp_bwd" in calls else []
+    op_of = {"fwd": P.OP_FWD, "bwd_dx": P.OP_BWD_DX, "bwd_dw": P.OP_BWD_DW, "mlp_fwd": P.OP_MLP_FWD,
+             "bwd": P.OP_BWD, "mlp_bwd": P.OP_MLP_BWD}
+    ws = P.Workspace(max([P.monarch_workspace_bytes(op_of[k], T, n, m, code) for k in calls if k != "bwd"]
+                         + [256]))
+    ws_b = P.Workspace(P.monarch_workspace_bytes(P.OP_BWD, T, n, m, code)) if "bwd" in calls else None
+    stream = torch.cuda.current_stream()
+
+    # One boundary event between consecutive calls (pre-created: nothing but the records sits between two
+    # launches): call k of a timed step runs between marks[j] and marks[j+1].
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(steps * len(calls) + 1)]
+    nmark = [0]
+
+    def step(i, timed):
+        e = sets[i % SETS]
+        for k in calls:
+            if k == "fwd":
+                P.monarch_fwd(e["x"], W["L"], W["R"], e["y"], T, n, m, ws)
+            elif k == "bwd_dx":
+                P.monarch_bwd_dx(e["dy"], W["L"], W["R"], e["dx"], T, n, m, ws)
+            elif k == "bwd_dw":
+                P.monarch_bwd_dw(e["x"], e["dy"], W["L"], W["R"], grads[0], grads[1], 0, T, n, m, ws)
+                if dist is not None:
+                    dist.all_reduce(grads)
+            elif k == "bwd":
+                P.monarch_bwd(e["x"], e["dy"], W["L"], W["R"], e["dx"], grads[0], grads[1], 0, T, n, m,
+                              ws_b, fwd_workspace=ws)
+                if dist is not None:
+                    dist.all_reduce(grads)
+            elif k == "mlp_fwd":
+                P.monarch_mlp_fwd(e["x"], W["L"], W["R"], W["b1"], W["L2"], W["R2"], W["b2"],
+                                  e["y"], T, n, m, ws)
+            elif k == "mlp_bwd":
+                g = mlp_grads
+                P.monarch_mlp_bwd(e["x"], e["dy"], W["L"], W["R"], W["b1"], W["L2"], W["R2"], e["dx"],
+                                  g[0], g[1], g[4], g[2], g[3], g[5], 0, T, n, m, ws)
+                if dist is not None:
+                    for t in g:
+                        dist.all_reduce(t)
+            if timed:
+                nmark[0] += 1
+                marks[nmark[0]].record(stream)
+
+    for i in range(warmup):
+        step(i, False)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    sampler = ClockSampler(local_rank) if sample_clocks else None
+    if sampler:
+        sampler.start()
+    launches0 = P.monarch_launch_count()
+    torch.cuda.synchronize()
+    t_start = torch.cuda.Event(enable_timing=True)
+    t_stop = torch.cuda.Event(enable_timing=True)
+    t_start.record(stream)
+    marks[0].record(stream)
+    for i in range(steps):
+        step(warmup + i, True)
+    t_stop.record(stream)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    total_ms = t_start.elapsed_time(t_stop)
+    clocks = sampler.stop() if sampler else None
+    launches = P.monarch_launch_count() - launches0
+    # a wait that ran out in any kernel of the timed region shows in the status word of the workspace it used
+    status = P.monarch_last_device_status(ws) | (P.monarch_last_device_status(ws_b) if ws_b is not None else 0)
+    if dist is not None:
+        tmax = torch.tensor([total_ms], device="cuda")
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        total_ms = float(tmax.item())
+    ms_per_step = total_ms / steps
+
+    peaks = load_peaks()
+    per_call = {}
+    for ci, k in enumerate(calls):
+        ts = [marks[st * len(calls) + ci].elapsed_time(marks[st * len(calls) + ci + 1]) for st in range(steps)]
+        ms = statistics.mean(ts)
+        by = call_bytes(k, n, m, T, cfg.dtype)
+        fl = call_flops(k, n, m, T)
+        roof_ms = max(by / (peaks["hbm_gbs"] * 1e9), fl / (peaks["bf16_tflops"] * 1e12)) * 1e3
+        tr = NCU_TRAFFIC_MB.get((cfg.index, k))
+        per_call[k] = {"ms": ms, "ms_min": min(ts), "gbs": by / ms / 1e6, "tflops": fl / ms / 1e9,
+                       "roofline_ms": roof_ms, "roofline_frac": roof_ms / ms,
+                       "impl": P.monarch_impl_name(op_of[k], m, code),
+                       "kernels": KERNELS_OF.get((m, cfg.dtype, k)),
+                       "algorithmic_mb": by / 1e6,
+                       "traffic_mb": tr[0] if tr else None, "traffic_note": tr[1] if tr else None}
+    return {"ms_per_step": ms_per_step, "calls": per_call, "clocks": clocks, "launches": int(launches),
+            "status": int(status), "sets": SETS, "inputs": d, "weights": W, "grads": grads}
+
+
 def main():
     args = parse_args()
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return launch_ranks(args)
     if args.workload == 8:
         return main_cplx(args)
     if args.workload == 6:
@@ -582,17 +745,8 @@ def main():
     from paper_2204_00595_b200.inputs import CONFIGS, make_inputs
     cfg = CONFIGS[args.workload]
     rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    calls = list(cfg.ops)
-    if args.calls:
-        # the backward of the feed-forward block is an optional extra call of the workload that has the block
-        extra = ["mlp_bwd"] if "mlp_fwd" in calls else []
-        calls = [k for k in calls + extra if k in args.calls.split(",")]
-    elif calls == ["fwd", "bwd_dx", "bwd_dw"]:
-        # default: the backward pass as one call (dx, dL, dR) that reuses the intermediate the forward
-        # call left in its workspace; --calls fwd,bwd_dx,bwd_dw times the three separate entry points
-        calls = ["fwd", "bwd"]
+    calls = default_calls(cfg, args.calls)
     n, m, T = cfg.n, cfg.m, cfg.tokens
     workload = (f"workload {cfg.index}: {'+'.join(calls)} {cfg.dtype} n={n} m={m} "
                 f"tokens/GPU={T}")
@@ -633,6 +787,7 @@ def main():
     import __graft_entry__ as entry
     entry.build()
     import paper_2204_00595_b200 as P
+    from paper_2204_00595_b200.inputs import to_device
 
     torch.cuda.set_device(local_rank)
     dist = None
@@ -640,122 +795,24 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     P.monarch_set_impl({"auto": P.IMPL_AUTO, "staged": P.IMPL_STAGED, "fused": P.IMPL_FUSED}[args.kernels])
-
     code = P.F32 if cfg.dtype == "f32" else P.BF16
-    tdt = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
-    d = make_inputs(cfg.index, with_dy="mlp_bwd" in calls)   # every rank draws the same recipe, then offsets it
-    from tests.helpers import to_device
 
-    # Two rotating sets of token tensors so that no launch finds its operands in L2 from the
-    # previous step (each set alone already exceeds the 126 MB L2 for workloads 3-5).
-    SETS = 2 if T * n * esize(cfg.dtype) * 4 < (1 << 30) else 1
-    sets = []
-    for s in range(SETS):
-        x = to_device(d["x"], cfg.dtype)
-        if s or rank:
-            x = torch.roll(x, shifts=17 * s + 5 * rank, dims=0).contiguous()
-        e = {"x": x, "y": torch.empty_like(x)}
-        if "dy" in d:
-            e["dy"] = torch.roll(to_device(d["dy"], cfg.dtype), shifts=3 * s + rank, dims=0).contiguous()
-            e["dx"] = torch.empty_like(x)
-        sets.append(e)
-    W = {k: to_device(d[k], cfg.dtype) for k in ("L", "R", "L2", "R2", "b1", "b2") if k in d}
-    grads = torch.zeros(2, m, m, m, dtype=torch.float32, device="cuda")   # packed (dL, dR)
-    mlp_grads = [torch.zeros(m, m, m, dtype=torch.float32, device="cuda") for _ in range(4)] + \
-                [torch.zeros(n, dtype=torch.float32, device="cuda") for _ in range(2)]   # dL1 dR1 dL2 dR2 db1 db2
-    op_of = {"fwd": P.OP_FWD, "bwd_dx": P.OP_BWD_DX, "bwd_dw": P.OP_BWD_DW, "mlp_fwd": P.OP_MLP_FWD,
-             "bwd": P.OP_BWD, "mlp_bwd": P.OP_MLP_BWD}
-    ws = P.Workspace(max([P.monarch_workspace_bytes(op_of[k], T, n, m, code) for k in calls if k != "bwd"]
-                         + [256]))
-    ws_b = P.Workspace(P.monarch_workspace_bytes(P.OP_BWD, T, n, m, code)) if "bwd" in calls else None
-    stream = torch.cuda.current_stream()
-
-    # One boundary event between consecutive calls (pre-created: nothing but the records sits between two
-    # launches): call k of a timed step runs between marks[j] and marks[j+1].
-    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps * len(calls) + 1)]
-    nmark = [0]
-
-    def step(i, timed):
-        e = sets[i % SETS]
-        for k in calls:
-            if k == "fwd":
-                P.monarch_fwd(e["x"], W["L"], W["R"], e["y"], T, n, m, ws)
-            elif k == "bwd_dx":
-                P.monarch_bwd_dx(e["dy"], W["L"], W["R"], e["dx"], T, n, m, ws)
-            elif k == "bwd_dw":
-                P.monarch_bwd_dw(e["x"], e["dy"], W["L"], W["R"], grads[0], grads[1], 0, T, n, m, ws)
-                if dist is not None:
-                    dist.all_reduce(grads)
-            elif k == "bwd":
-                P.monarch_bwd(e["x"], e["dy"], W["L"], W["R"], e["dx"], grads[0], grads[1], 0, T, n, m,
-                              ws_b, fwd_workspace=ws)
-                if dist is not None:
-                    dist.all_reduce(grads)
-            elif k == "mlp_fwd":
-                P.monarch_mlp_fwd(e["x"], W["L"], W["R"], W["b1"], W["L2"], W["R2"], W["b2"],
-                                  e["y"], T, n, m, ws)
-            elif k == "mlp_bwd":
-                g = mlp_grads
-                P.monarch_mlp_bwd(e["x"], e["dy"], W["L"], W["R"], W["b1"], W["L2"], W["R2"], e["dx"],
-                                  g[0], g[1], g[4], g[2], g[3], g[5], 0, T, n, m, ws)
-                if dist is not None:
-                    for t in g:
-                        dist.all_reduce(t)
-            if timed:
-                nmark[0] += 1
-                marks[nmark[0]].record(stream)
-
-    for i in range(args.warmup):
-        step(i, False)
-    torch.cuda.synchronize()
-    if dist is not None:
-        dist.barrier()
-    sampler = ClockSampler(local_rank)
-    sampler.start()
-    launches0 = P.monarch_launch_count()
-    torch.cuda.synchronize()
-    t_start = torch.cuda.Event(enable_timing=True)
-    t_stop = torch.cuda.Event(enable_timing=True)
-    t_start.record(stream)
-    marks[0].record(stream)
-    for i in range(args.steps):
-        step(args.warmup + i, True)
-    t_stop.record(stream)
-    torch.cuda.synchronize()
-    if dist is not None:
-        dist.barrier()
-    total_ms = t_start.elapsed_time(t_stop)
-    clocks = sampler.stop()
-    launches = P.monarch_launch_count() - launches0
-    status = P.monarch_last_device_status(ws)
-    if dist is not None:
-        tmax = torch.tensor([total_ms], device="cuda")
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        total_ms = float(tmax.item())
-    ms_per_step = total_ms / args.steps
+    res = measure(P, torch, dist, cfg, calls, args.steps, args.warmup, rank, local_rank, True)
+    d, W, grads = res.pop("inputs"), res.pop("weights"), res.pop("grads")
+    ms_per_step, per_call = res["ms_per_step"], res["calls"]
     value = step_flops * world / (ms_per_step * 1e-3) / 1e12
     tokens_per_s = T * world / (ms_per_step * 1e-3)
 
     peaks = load_peaks()
-    per_call = {}
-    for ci, k in enumerate(calls):
-        ts = [marks[st * len(calls) + ci].elapsed_time(marks[st * len(calls) + ci + 1]) for st in range(args.steps)]
-        ms = statistics.mean(ts)
-        by = call_bytes(k, n, m, T, cfg.dtype)
-        fl = call_flops(k, n, m, T)
-        roof_ms = max(by / (peaks["hbm_gbs"] * 1e9), fl / (peaks["bf16_tflops"] * 1e12)) * 1e3
-        per_call[k] = {"ms": ms, "ms_min": min(ts), "gbs": by / ms / 1e6, "tflops": fl / ms / 1e9,
-                       "roofline_ms": roof_ms, "roofline_frac": roof_ms / ms,
-                       "impl": P.monarch_impl_name(op_of[k], m, code)}
     dom = max(calls, key=lambda k: per_call[k]["ms"])
     roofline = {
-        "bound": "hbm", "kernel": f"{dom}: {KERNELS_OF.get((m, cfg.dtype, dom), per_call[dom]['impl'])}",
+        "bound": "hbm", "kernel": f"{dom}: {per_call[dom]['kernels'] or per_call[dom]['impl']}",
         "achieved": per_call[dom]["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
         "frac": per_call[dom]["gbs"] / peaks["hbm_gbs"], "peak_source": peaks["source"],
-        "traffic": NCU_TRAFFIC_MB.get((cfg.index, dom)),
+        "traffic": per_call[dom]["traffic_mb"],
         "traffic_unit": "MB per call (dram__bytes_read.sum + dram__bytes_write.sum, summed over the "
-                        "call's kernels, from an ncu capture of this workload at full size)",
-        "algorithmic_mb": call_bytes(dom, n, m, T, cfg.dtype) / 1e6,
+                        "call's kernels, from the ncu capture named in the call's traffic_note)",
+        "algorithmic_mb": per_call[dom]["algorithmic_mb"],
     }
 
     line = {
@@ -763,17 +820,39 @@ def main():
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
         "tokens_per_s": tokens_per_s,
-        "config": {"workload": workload, "l2": f"inputs larger than L2; {SETS} rotating buffer sets",
-                   "kernels": args.kernels, "device_status": status},
-        "clocks": clocks, "gpu_launches": int(launches), "roofline": roofline, "calls": per_call,
+        "config": {"workload": workload, "l2": f"inputs larger than L2; {res['sets']} rotating buffer sets",
+                   "kernels": args.kernels, "device_status": res["status"]},
+        "clocks": res["clocks"], "gpu_launches": res["launches"], "roofline": roofline, "calls": per_call,
     }
+
+    # The other workloads of the contract, timed the same way with fewer steps (per call: time, fraction of the
+    # roofline, kernels, algorithmic and measured DRAM megabytes).  The headline above is the largest
+    # forward + backward configuration; these entries carry the rest.
+    if args.side_workloads and not args.calls:
+        side = {str(cfg.index): {"calls": per_call, "ms_per_step": ms_per_step, "steps": args.steps}}
+        for idx in (1, 2, 3, 4, 5):
+            if idx == cfg.index:
+                continue
+            c2 = CONFIGS[idx]
+            k2 = default_calls(c2, "")
+            torch.cuda.empty_cache()
+            steps2 = max(20, min(args.steps, 200))
+            r2 = measure(P, torch, dist, c2, k2, steps2, max(args.warmup, 3), rank, local_rank, False)
+            for key in ("inputs", "weights", "grads"):
+                r2.pop(key)
+            side[str(idx)] = {"calls": r2["calls"], "ms_per_step": r2["ms_per_step"], "steps": steps2,
+                              "device_status": r2["status"], "gpu_launches": r2["launches"],
+                              "workload": f"{'+'.join(k2)} {c2.dtype} n={c2.n} m={c2.m} tokens/GPU={c2.tokens}"}
+            line["config"]["device_status"] |= r2["status"]
+        line["workloads"] = dict(sorted(side.items()))
+    if line["config"]["device_status"] != 0:
+        line["invalid"] = "a device-side wait ran out inside the timed region"
 
     if not args.no_e2e:
         e2e = None
         if "fwd" in calls and ("bwd" in calls or "bwd_dw" in calls):
             # the same step through the host-buffer entry point: pinned host tensors in, host tensors
             # out, uploads and downloads inside the timed region (wall clock around blocking calls)
-            del sets, ws, ws_b
             torch.cuda.empty_cache()
             hx = torch.roll(to_device(d["x"], cfg.dtype), 5 * rank, 0).cpu().pin_memory()
             hdy = torch.roll(to_device(d["dy"], cfg.dtype), rank, 0).cpu().pin_memory()

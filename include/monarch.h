@@ -234,6 +234,19 @@ int monarch_workspace_init(void *workspace, size_t workspace_bytes, void *stream
  * reusing it), or MONARCH_ERR_CUDA. */
 int monarch_last_device_status(void *workspace, void *stream);
 
+/* Test aids for the bounded waits (the paper has no counterpart; they exist so that the
+ * time-out path can be exercised without faulting or hanging a GPU).
+ * monarch_debug_set_wait_limit: kernels that use `workspace` from now on give up a wait after
+ * `microseconds` instead of about one second (0 restores the default; monarch_workspace_init
+ * also does).  Enqueued on `stream`.
+ * monarch_debug_skip_load: host-side fault injection.  The next m = 128 forward call leaves out
+ * one operand load of its last step (item = tile * 128 + output row block; -1 cancels), so the
+ * thread block that owns the item waits for data that never arrives, gives up after the wait
+ * limit, records MONARCH_ERR_TIMEOUT in the status word and returns; its outputs are undefined.
+ * Nothing faults and no wait is unbounded. */
+int monarch_debug_set_wait_limit(void *workspace, unsigned int microseconds, void *stream);
+int monarch_debug_skip_load(int64_t item);
+
 /* Select the kernel family for later calls (a monarch_impl_t).  Not
  * thread-safe against concurrent calls. Returns the previous value, or -1. */
 int monarch_set_impl(int impl);

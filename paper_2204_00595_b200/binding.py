@@ -36,6 +36,8 @@ _SIGNATURES = {
     "monarch_workspace_bytes": (_sz, [_int, _i64, _i32, _i32, _int]),
     "monarch_workspace_init": (_int, [_vp, _sz, _vp]),
     "monarch_last_device_status": (_int, [_vp, _vp]),
+    "monarch_debug_set_wait_limit": (_int, [_vp, ctypes.c_uint, _vp]),
+    "monarch_debug_skip_load": (_int, [_i64]),
     "monarch_set_impl": (_int, [_int]),
     "monarch_impl_name": (ctypes.c_char_p, [_int, _i32, _int]),
     "monarch_launch_count": (ctypes.c_uint64, []),
@@ -146,6 +148,15 @@ def monarch_workspace_init(workspace, stream=None) -> None:
 def monarch_last_device_status(workspace, stream=None) -> int:
     p, _ = _ws(workspace)
     return int(lib().monarch_last_device_status(p, _stream(stream)))
+
+
+def monarch_debug_set_wait_limit(workspace, microseconds: int, stream=None) -> None:
+    p, _ = _ws(workspace)
+    _check(lib().monarch_debug_set_wait_limit(p, int(microseconds), _stream(stream)), "monarch_debug_set_wait_limit")
+
+
+def monarch_debug_skip_load(item: int) -> None:
+    _check(lib().monarch_debug_skip_load(int(item)), "monarch_debug_skip_load")
 
 
 def monarch_set_impl(impl: int) -> int:

@@ -21,11 +21,24 @@
 // One kernel template serves all block products: persistent CTAs, the 32 KB weight block resident, token operands
 // through a TMA ring, tcgen05.mma 128 x 128 x 16 with two accumulator buffers in TMEM, epilogue through swizzled
 // staging tiles and TMA stores.
+#include <atomic>
+#include <cstdlib>
+
 #include "tc_common.cuh"
 
 namespace monarch {
 namespace tc {
 namespace {
+
+// Host-side fault injection for the test of the bounded waits: the next plane-transpose launch leaves out the load of
+// this item (neither announced nor copied), so its consumers wait for bytes that never come.  -1 = none.
+std::atomic<long long> g_skip_load{-1};
+// forward pass in one persistent launch (default) or in three launches (comparison runs: MONARCH_CHAIN_SPLIT set)
+bool chain_fused_enabled()
+{
+    static const bool on = getenv("MONARCH_CHAIN_SPLIT") == nullptr;
+    return on;
+}
 
 constexpr int kB = 128;                      // block size m
 constexpr int kOpBytes = 32768;              // one 128 x 128 bf16 operand: two boxes of [128 rows][64 columns]
@@ -314,6 +327,7 @@ constexpr int kTrSmem = (kTrIn + kTrOut) * kOpBytes + 1024;
 struct TransposeParams {
     unsigned *status;
     int ntiles, nplanes;                 // planes per tile (128)
+    long long skip_item;                 // injected fault (tests only), else -1
 };
 
 template <bool TO_PLANES>
@@ -344,12 +358,24 @@ plane_transpose_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_c
     if (warp == 4) {
         if (lane == 0) {
             uint32_t n = 0;
+            int last_fill[kTrIn];
+#pragma unroll
+            for (int s = 0; s < kTrIn; ++s) last_fill[s] = -1;
             for (long long i = i0; i < i1; ++i, ++n) {
                 const int tile = (int)(i / p.nplanes), pl = (int)(i % p.nplanes);
                 const uint32_t s = n % kTrIn;
                 if (!mbar_wait(smem_u32(&empty[s]), ((n / kTrIn) & 1) ^ 1, p.status, dead, kErrSlotWait)) break;
+                if (i == p.skip_item) continue;
                 mbar_expect_tx(smem_u32(&full[s]), kOpBytes);
                 load_operand<TO_PLANES ? kLdX : kLdP>(in0 + s * kOpBytes, &tm_in, pl, tile, smem_u32(&full[s]));
+                last_fill[s] = (int)(n / kTrIn);
+            }
+            if (*dead) {
+                // unwinding after a wait that ran out: no copy into this CTA's shared memory may outlive the CTA
+#pragma unroll
+                for (int s = 0; s < kTrIn; ++s)
+                    if (last_fill[s] >= 0)
+                        for (int spin = 0; spin < (1 << 22) && !mbar_try_wait(smem_u32(&full[s]), last_fill[s] & 1); ++spin) { }
             }
         }
     } else {
@@ -397,6 +423,314 @@ plane_transpose_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_c
         }
         if (threadIdx.x == 0) tma_store_wait_all<0>();
     }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// The whole forward pass in one persistent launch: CTA b (one per SM, 128 of them) owns block b of every step and
+// walks the token tiles; at step s it runs
+//     A: D_b[j][t] = R_b x_b(tile s)            -> u'[tile s][j][b][t]             (stage 1, rows to all j)
+//     B: D_b[l][t] = L_b u'_b(tile s - LAG)     -> w'[(tile s - LAG) % RING][l][b][t]   (stage 2)
+//     C: y[t][b*128 + j] = w'[tile s - 2 LAG][b][j][t]                              (plane b transposed)
+// B needs the rows that all 128 CTAs wrote in A two steps earlier, C those of B: one counter per tile and stage,
+// bumped by each CTA's store thread when its TMA stores have completed and polled (bounded) by the consumer's
+// loader.  Dependencies only point to earlier steps, every CTA is resident (the launch is refused otherwise), so
+// the waits cannot deadlock; the lag hides them.  x is read once and y written once; u' is also kept for the
+// backward call, w' lives in a ring of RING tiles that stays in L2.
+constexpr int kFusedLag = 2, kFusedRing = 2 * kFusedLag + 2;
+constexpr int kFusedThreads = 11 * 32;       // warps 0-3 epilogue, 4-7 transposers, 8 loader, 9 MMA, 10 store thread
+constexpr int kFusedSmem = 2 * kOpBytes /* R_b, L_b */ + 2 * kOpBytes /* operand ring */ + kStagingBytes +
+                           2 * kOpBytes /* plane in, out */ + 1024;
+constexpr unsigned kFusedCounters = 8192;    // tiles per counter array (two arrays in the 64 KB after the status word)
+
+struct FusedParams {
+    unsigned *status;
+    unsigned *cnt1, *cnt2;                   // per tile: CTAs whose stage-1 / stage-2 rows have landed; zero between calls
+    int ntiles;
+};
+
+struct FusedBars {
+    uint64_t w_full;
+    uint64_t full[2], empty[2];
+    uint64_t acc_full[2], acc_empty[2];
+    uint64_t st_full[2], st_free[2];
+    uint64_t tr_full, tr_empty;
+};
+
+__device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned *p)
+{
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void fence_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
+
+// Wait (bounded) until all `need` producers of a tile have published; the last of the `need` consumers to get here
+// puts the counter back to zero for the next call.
+__device__ __forceinline__ bool wait_counter(unsigned *ctr, unsigned need, unsigned *status, volatile int *dead)
+{
+    if (ld_acquire_gpu(ctr) < need) {
+        const unsigned long long t0 = global_timer_ns(), limit = wait_limit_ns(status);
+        while (ld_acquire_gpu(ctr) < need) {
+            if (*dead || global_timer_ns() - t0 > limit) {
+                *dead = 1;
+                atomicCAS(status, 0u, (unsigned)kErrPeerWait);
+                return false;
+            }
+        }
+    }
+    if (atomicAdd(ctr, 1u) + 1 == 2 * need) atomicExch(ctr, 0u);
+    fence_async_global();
+    return true;
+}
+
+__global__ void __launch_bounds__(kFusedThreads, 1)
+chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_R,
+                       const __grid_constant__ CUtensorMap tm_L, const __grid_constant__ CUtensorMap tm_u_st,
+                       const __grid_constant__ CUtensorMap tm_u_ld, const __grid_constant__ CUtensorMap tm_w_st,
+                       const __grid_constant__ CUtensorMap tm_w_ld, const __grid_constant__ CUtensorMap tm_y,
+                       const FusedParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) FusedBars bars;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int dead_s;
+
+    const uint32_t w0 = (smem_u32(smem_raw) + 1023u) & ~1023u;          // R_b, L_b
+    const uint32_t ring0 = w0 + 2 * kOpBytes;
+    const uint32_t staging0 = ring0 + 2 * kOpBytes;
+    const uint32_t trin = staging0 + kStagingBytes, trout = trin + kOpBytes;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int b = (int)blockIdx.x;
+    volatile int *dead = &dead_s;
+
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bars.w_full), 1);
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(smem_u32(&bars.full[a]), 1);
+            mbar_init(smem_u32(&bars.empty[a]), 1);
+            mbar_init(smem_u32(&bars.acc_full[a]), 1);
+            mbar_init(smem_u32(&bars.acc_empty[a]), 4);
+            mbar_init(smem_u32(&bars.st_full[a]), 4);
+            mbar_init(smem_u32(&bars.st_free[a]), 1);
+        }
+        mbar_init(smem_u32(&bars.tr_full), 1);
+        mbar_init(smem_u32(&bars.tr_empty), 4);
+        fence_mbar_init();
+        dead_s = 0;
+        tma_prefetch_desc(&tm_x); tma_prefetch_desc(&tm_R); tma_prefetch_desc(&tm_L); tma_prefetch_desc(&tm_u_st);
+        tma_prefetch_desc(&tm_u_ld); tma_prefetch_desc(&tm_w_st); tma_prefetch_desc(&tm_w_ld); tma_prefetch_desc(&tm_y);
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&tmem_base_s), 256);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+
+    const int nt = p.ntiles, nsteps = nt + 2 * kFusedLag;
+    const uint32_t full0 = smem_u32(bars.full), empty0 = smem_u32(bars.empty);
+    const uint32_t accf0 = smem_u32(bars.acc_full), acce0 = smem_u32(bars.acc_empty);
+    const uint32_t stf0 = smem_u32(bars.st_full), stfree0 = smem_u32(bars.st_free);
+    const uint32_t trf = smem_u32(&bars.tr_full), tre = smem_u32(&bars.tr_empty);
+
+    if (warp == 8) {
+        // ------------------------------------------------------------ loader
+        if (lane == 0) {
+            const uint32_t wbar = smem_u32(&bars.w_full);
+            mbar_expect_tx(wbar, 2 * kOpBytes);
+            tma_load_2d(w0, &tm_R, 0, b * kB, wbar);
+            tma_load_2d(w0 + kHalfBytes, &tm_R, 64, b * kB, wbar);
+            tma_load_2d(w0 + kOpBytes, &tm_L, 0, b * kB, wbar);
+            tma_load_2d(w0 + kOpBytes + kHalfBytes, &tm_L, 64, b * kB, wbar);
+            uint32_t g = 0, c = 0;                         // operand-ring items, planes loaded so far
+            bool ok = true;
+            for (int s = 0; ok && s < nsteps; ++s) {
+                if (s < nt) {
+                    const uint32_t sl = g & 1;
+                    if (!mbar_wait(empty0 + sl * 8, ((g >> 1) & 1) ^ 1, p.status, dead, kErrSlotWait)) break;
+                    mbar_expect_tx(full0 + sl * 8, kOpBytes);
+                    load_operand<kLdX>(ring0 + sl * kOpBytes, &tm_x, b, s, full0 + sl * 8);
+                    ++g;
+                }
+                const int tb = s - kFusedLag;
+                if (tb >= 0 && tb < nt) {
+                    if (!wait_counter(p.cnt1 + tb, kB, p.status, dead)) break;
+                    const uint32_t sl = g & 1;
+                    if (!mbar_wait(empty0 + sl * 8, ((g >> 1) & 1) ^ 1, p.status, dead, kErrSlotWait)) break;
+                    mbar_expect_tx(full0 + sl * 8, kOpBytes);
+                    load_operand<kLdP>(ring0 + sl * kOpBytes, &tm_u_ld, b, tb, full0 + sl * 8);
+                    ++g;
+                }
+                const int tc = s - 2 * kFusedLag;
+                if (tc >= 0) {
+                    if (!wait_counter(p.cnt2 + tc, kB, p.status, dead)) break;
+                    if (!mbar_wait(tre, (c & 1) ^ 1, p.status, dead, kErrSlotWait)) break;
+                    mbar_expect_tx(trf, kOpBytes);
+                    load_operand<kLdP>(trin, &tm_w_ld, b, tc % kFusedRing, trf);
+                    ++c;
+                }
+            }
+        }
+    } else if (warp == 9) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0 && mbar_wait(smem_u32(&bars.w_full), 0, p.status, dead, kErrTmaWait)) {
+            constexpr uint32_t idesc_a = make_idesc_bf16(128, 128, 0, 0), idesc_b = make_idesc_bf16(128, 128, 0, 1);
+            uint32_t g = 0;
+            bool ok = true;
+            for (int s = 0; ok && s < nsteps; ++s) {
+#pragma unroll
+                for (int kind = 0; kind < 2; ++kind) {
+                    const int tile = kind == 0 ? s : s - kFusedLag;
+                    if (tile < 0 || tile >= nt) continue;
+                    const uint32_t buf = g & 1;
+                    if (!mbar_wait(acce0 + buf * 8, ((g >> 1) & 1) ^ 1, p.status, dead, kErrTmemWait)) { ok = false; break; }
+                    if (!mbar_wait(full0 + buf * 8, (g >> 1) & 1, p.status, dead, kErrTmaWait)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t t0 = ring0 + buf * kOpBytes, w = w0 + kind * kOpBytes, d = tmem_base + buf * 128;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)
+                        mma_f16_ss(d, op_desc(w, false, ks), op_desc(t0, kind == 1, ks), kind == 0 ? idesc_a : idesc_b, ks != 0);
+                    mma_commit(empty0 + buf * 8);
+                    mma_commit(accf0 + buf * 8);
+                    ++g;
+                }
+            }
+        }
+    } else if (warp < 4) {
+        // ------------------------------------------------------------ epilogue: TMEM -> bf16 -> staging halves
+        const int row = warp * 32 + lane;
+        const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+        uint32_t g = 0;
+        bool ok = true;
+        for (int s = 0; ok && s < nsteps; ++s) {
+#pragma unroll 1
+            for (int kind = 0; kind < 2; ++kind) {
+                const int tile = kind == 0 ? s : s - kFusedLag;
+                if (tile < 0 || tile >= nt) continue;
+                const uint32_t buf = g & 1;
+                if (!mbar_wait(accf0 + buf * 8, (g >> 1) & 1, p.status, dead, kErrMmaWait)) { ok = false; break; }
+                tc_fence_after();
+#pragma unroll 1
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t v[4][16];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) tmem_ld16(lane_base + buf * 128 + h * 64 + q * 16, v[q]);
+                    tmem_ld_wait();
+                    if (h == 1) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(acce0 + buf * 8);
+                    }
+                    // staging half h is free once the store of the previous item's half h has read it
+                    if (!mbar_wait(stfree0 + h * 8, (g & 1) ^ 1, p.status, dead, kErrSlotWait)) { ok = false; break; }
+                    const uint32_t dst = staging0 + h * kHalfBytes + row * 128;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const uint32_t *w = &v[c >> 1][(c & 1) * 8];
+                        const uint32_t o0 = pack_bf16(__uint_as_float(w[0]), __uint_as_float(w[1]));
+                        const uint32_t o1 = pack_bf16(__uint_as_float(w[2]), __uint_as_float(w[3]));
+                        const uint32_t o2 = pack_bf16(__uint_as_float(w[4]), __uint_as_float(w[5]));
+                        const uint32_t o3 = pack_bf16(__uint_as_float(w[6]), __uint_as_float(w[7]));
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((c ^ (row & 7)) << 4)),
+                                     "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(stf0 + h * 8);
+                }
+                if (!ok) break;
+                ++g;
+            }
+        }
+    } else if (warp == 10) {
+        // ------------------------------------------------------------ store thread: staging -> u' / w', publish
+        if (lane == 0) {
+            uint32_t g = 0;
+            int prev_kind = -1, prev_tile = 0;
+            bool ok = true;
+            for (int s = 0; ok && s < nsteps; ++s) {
+#pragma unroll 1
+                for (int kind = 0; kind < 2; ++kind) {
+                    const int tile = kind == 0 ? s : s - kFusedLag;
+                    if (tile < 0 || tile >= nt) continue;
+#pragma unroll 1
+                    for (int h = 0; h < 2; ++h) {
+                        if (!mbar_wait(stf0 + h * 8, g & 1, p.status, dead, kErrMmaWait)) { ok = false; break; }
+                        if (kind == 0) tma_store_4d(&tm_u_st, staging0 + h * kHalfBytes, h * 64, b, 0, tile);
+                        else tma_store_4d(&tm_w_st, staging0 + h * kHalfBytes, h * 64, b, 0, tile % kFusedRing);
+                        tma_store_commit();
+                        // the store committed before this one has read its staging half
+                        if (g != 0 || h != 0) {
+                            tma_store_wait_read<1>();
+                            mbar_arrive(stfree0 + (h ^ 1) * 8);
+                        }
+                    }
+                    if (!ok) break;
+                    // all but the two stores just issued have completed: the previous item's rows are in memory
+                    if (prev_kind >= 0) {
+                        tma_store_wait_all<2>();
+                        fence_async_global();
+                        __threadfence();
+                        atomicAdd((prev_kind == 0 ? p.cnt1 : p.cnt2) + prev_tile, 1u);
+                    }
+                    prev_kind = kind;
+                    prev_tile = tile;
+                    ++g;
+                }
+            }
+            tma_store_wait_all<0>();
+            if (ok && prev_kind >= 0) {
+                fence_async_global();
+                __threadfence();
+                atomicAdd((prev_kind == 0 ? p.cnt1 : p.cnt2) + prev_tile, 1u);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ transposers (warps 4-7): plane b of w' -> y
+        const int tw = warp - 4;
+        const int tid = threadIdx.x - 128;
+        uint32_t c = 0;
+        for (int s = 2 * kFusedLag; s < nsteps; ++s, ++c) {
+            const int tile = s - 2 * kFusedLag;
+            if (!mbar_wait(trf, c & 1, p.status, dead, kErrTmaWait)) break;
+            // the stores of the previous plane have read the output buffer
+            if (tid == 0) tma_store_wait_read<0>();
+            asm volatile("bar.sync 2, 128;" ::: "memory");
+#pragma unroll 1
+            for (int ro = 0; ro < 4; ++ro) {
+                const int r0 = tw * 32 + ro * 8;
+#pragma unroll
+                for (int cq = 0; cq < 4; ++cq) {
+                    const int mi = lane >> 3, ri = lane & 7;
+                    const int co = cq * 4 + mi, sr = r0 + ri;
+                    const uint32_t src = trin + (co >> 3) * kHalfBytes + sr * 128 + (((co & 7) ^ (sr & 7)) << 4);
+                    uint32_t a, bq, cc, d;
+                    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(a), "=r"(bq), "=r"(cc), "=r"(d) : "r"(src) : "memory");
+                    const int dr = co * 8 + ri, dco = r0 >> 3;
+                    const uint32_t dst = trout + (dco >> 3) * kHalfBytes + dr * 128 + (((dco & 7) ^ (dr & 7)) << 4);
+                    asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(a),
+                                 "r"(bq), "r"(cc), "r"(d) : "memory");
+                }
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tre);
+            asm volatile("bar.sync 2, 128;" ::: "memory");
+            if (tid == 0) {
+                tma_store_2d(&tm_y, trout, b * kB, tile * 128);
+                tma_store_2d(&tm_y, trout + kHalfBytes, b * kB + 64, tile * 128);
+                tma_store_commit();
+            }
+        }
+        if (tid == 0) tma_store_wait_all<0>();
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem_base, 256);
 }
 
 // ---------------------------------------------------------------------------------------------------------
@@ -462,6 +796,7 @@ int launch_transpose(const CUtensorMap &in, const CUtensorMap &out, int ntiles, 
     p.status = status;
     p.ntiles = ntiles;
     p.nplanes = kB;
+    p.skip_item = g_skip_load.exchange(-1);
     long long grid = (long long)ntiles * kB;
     if (grid > sms) grid = sms;
     plane_transpose_kernel<TO_PLANES><<<(unsigned)grid, kTrThreads, kTrSmem, s>>>(in, out, p);
@@ -475,9 +810,18 @@ size_t planes_bytes(int64_t tokens) { return (size_t)((tokens + 127) / 128) * 12
 }  // namespace
 }  // namespace tc
 
-// Forward workspace: [status][u' planes][w' planes]; the backward call reads u' from it.
-size_t chain_fwd_m128_workspace_bytes(int64_t tokens) { return MONARCH_STATUS_BYTES + 2 * tc::planes_bytes(tokens); }
-const void *chain_fwd_m128_saved_u(const void *fwd_ws) { return (const char *)fwd_ws + MONARCH_STATUS_BYTES; }
+void debug_skip_next_plane_load(long long item) { tc::g_skip_load.store(item); }
+
+// Forward workspace: [status][tile counters 64 KB][u' planes][w' planes]; the backward call reads u' from it.
+constexpr size_t kChainCounterBytes = 65536;
+size_t chain_fwd_m128_workspace_bytes(int64_t tokens)
+{
+    return MONARCH_STATUS_BYTES + kChainCounterBytes + 2 * tc::planes_bytes(tokens);
+}
+const void *chain_fwd_m128_saved_u(const void *fwd_ws)
+{
+    return (const char *)fwd_ws + MONARCH_STATUS_BYTES + kChainCounterBytes;
+}
 // Backward workspace: [status][dw' planes][du' planes][u' planes (when the forward call's are not passed)]
 size_t chain_bwd_m128_workspace_bytes(int64_t tokens) { return MONARCH_STATUS_BYTES + 3 * tc::planes_bytes(tokens); }
 
@@ -489,7 +833,7 @@ int chain_fwd_m128(const void *x, const void *L, const void *R, void *y, int64_t
     if (tokens > (int64_t)1 << 30) return MONARCH_ERR_UNSUPPORTED;
     const int ntiles = (int)((tokens + 127) / 128);
     unsigned *status = (unsigned *)ws;
-    char *up = (char *)ws + MONARCH_STATUS_BYTES, *wp = up + planes_bytes(tokens);
+    char *up = (char *)ws + MONARCH_STATUS_BYTES + kChainCounterBytes, *wp = up + planes_bytes(tokens);
     CUtensorMap mx, my, mR, mL, mu_q, mu_p, mw_q, mw_p;
     MONARCH_TRY(map_tokens(&mx, x, tokens));
     MONARCH_TRY(map_tokens(&my, y, tokens));
@@ -499,6 +843,22 @@ int chain_fwd_m128(const void *x, const void *L, const void *R, void *y, int64_t
     MONARCH_TRY(map_planes(&mu_p, up, ntiles, true));
     MONARCH_TRY(map_planes(&mw_q, wp, ntiles, false));
     MONARCH_TRY(map_planes(&mw_p, wp, ntiles, true));
+    int sms = 0;
+    MONARCH_TRY(device_sms(&sms));
+    if (chain_fused_enabled() && sms >= kB && ntiles <= (int)kFusedCounters &&
+        g_skip_load.load(std::memory_order_relaxed) < 0) {
+        // one persistent launch; every CTA must be resident at once (one per SM)
+        MONARCH_CUDA_TRY(cudaFuncSetAttribute(chain_fused_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmem));
+        FusedParams fp;
+        fp.status = status;
+        fp.cnt1 = (unsigned *)((char *)ws + MONARCH_STATUS_BYTES);
+        fp.cnt2 = fp.cnt1 + kFusedCounters;
+        fp.ntiles = ntiles;
+        chain_fused_fwd_kernel<<<kB, kFusedThreads, kFusedSmem, s>>>(mx, mR, mL, mu_q, mu_p, mw_q, mw_p, my, fp);
+        note_launch();
+        MONARCH_CUDA_TRY(cudaGetLastError());
+        return MONARCH_OK;
+    }
     // step 1 + inner permutation: D_k[j][t] = sum_i R[k][j][i] x[t][k*128+i]  ->  u'[tile][j][k][t]
     MONARCH_TRY((launch_gemm<kLdX, true, false, false, kStQ, false, kLdX, false, true>(mx, mx, mR, mu_q, nullptr, ntiles, status, s)));
     // step 2: D_j[l][t] = sum_k L[j][l][k] u'[tile][j][k][t]  ->  w'[tile][l][j][t]

@@ -102,6 +102,8 @@ int chain_fwd_m128(const void *x, const void *L, const void *R, void *y, int64_t
 int chain_bwd_m128(const void *x, const void *dy, const void *L, const void *R, const void *saved_up, void *dx, float *dL,
                    float *dR, int want_dx, int want_dw, int64_t tokens, void *ws, cudaStream_t s);
 const void *chain_fwd_m128_saved_u(const void *fwd_ws);
+// test aid: the next plane-transpose launch (last step of the m = 128 forward) leaves out the load of this item
+void debug_skip_next_plane_load(long long item);
 
 // ---- backward as a chain of tensor-core launches (bf16; dx for m >= 32, dL/dR for m = 128), tc_bwd.cu ----
 size_t tc_staged_bwd_workspace_bytes(int64_t tokens, int m);

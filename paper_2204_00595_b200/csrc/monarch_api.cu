@@ -492,6 +492,21 @@ int monarch_last_device_status(void *workspace, void *stream)
     return MONARCH_OK;
 }
 
+int monarch_debug_set_wait_limit(void *workspace, unsigned int microseconds, void *stream)
+{
+    if (!workspace || ((uintptr_t)workspace & 255)) return MONARCH_ERR_WORKSPACE;
+    // pageable source: the copy is staged before the call returns
+    MONARCH_CUDA_TRY(cudaMemcpyAsync((char *)workspace + sizeof(unsigned int), &microseconds, sizeof(microseconds),
+                                     cudaMemcpyHostToDevice, (cudaStream_t)stream));
+    return MONARCH_OK;
+}
+
+int monarch_debug_skip_load(int64_t item)
+{
+    debug_skip_next_plane_load(item);
+    return MONARCH_OK;
+}
+
 int monarch_set_impl(int impl)
 {
     if (impl < MONARCH_IMPL_AUTO || impl > MONARCH_IMPL_FUSED) return -1;

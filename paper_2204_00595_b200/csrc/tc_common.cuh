@@ -23,6 +23,14 @@ enum : unsigned {
 
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // ~1 s
 
+// The word after the status word optionally holds a shorter limit in microseconds (0 = the default above);
+// monarch_debug_set_wait_limit writes it, monarch_workspace_init clears it.  Read on the slow path only.
+__device__ __forceinline__ unsigned long long wait_limit_ns(const unsigned *status)
+{
+    const unsigned us = reinterpret_cast<const volatile unsigned *>(status)[1];
+    return us ? (unsigned long long)us * 1000ull : kWaitLimitNs;
+}
+
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
 {
     return (uint32_t)__cvta_generic_to_shared(p);
@@ -101,14 +109,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigne
             return true;
     }
     if (*dead) return false;
-    const unsigned long long t0 = global_timer_ns();
+    const unsigned long long t0 = global_timer_ns(), limit = wait_limit_ns(status);
     while (true) {
         for (int i = 0; i < 32; ++i) {
             if (CLUSTER_ACQUIRE ? mbar_try_wait_cluster_acquire(bar, parity)
                                 : mbar_try_wait(bar, parity))
                 return true;
         }
-        if (*dead || global_timer_ns() - t0 > kWaitLimitNs) break;
+        if (*dead || global_timer_ns() - t0 > limit) break;
     }
     *dead = 1;
     atomicCAS(status, 0u, code);

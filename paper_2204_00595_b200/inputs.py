@@ -130,3 +130,16 @@ def make_rect_inputs(tokens: int | None = None, seed: int = 595006, **sizes) -> 
     out["R"] = draw((q, b, b1), 1.0 / math.sqrt(b1))
     out["L"] = draw((b, r, q), 1.0 / math.sqrt(q))
     return out
+
+
+def to_device(a: np.ndarray, dtype: str):
+    """float32 numpy array (already rounded to the storage dtype) -> torch CUDA tensor, exactly."""
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).cuda()
+    return t.to(torch.bfloat16) if dtype == "bf16" else t
+
+
+def to_host64(t) -> np.ndarray:
+    """torch tensor (any float dtype, any device) -> float64 numpy array, exactly."""
+    import torch
+    return t.detach().to(torch.float32).cpu().numpy().astype(np.float64)

@@ -40,13 +40,4 @@ def assert_close(got, ref, dtype: str, what: str = "", scale: float = 1.0):
     return emax, emean
 
 
-def to_device(a: np.ndarray, dtype: str):
-    """float32 numpy array (already rounded to storage dtype) -> torch CUDA tensor, exactly."""
-    import torch
-    t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).cuda()
-    return t.to(torch.bfloat16) if dtype == "bf16" else t
-
-
-def to_host64(t) -> np.ndarray:
-    import torch
-    return t.detach().to(torch.float32).cpu().numpy().astype(np.float64)
+from paper_2204_00595_b200.inputs import to_device, to_host64  # noqa: E402,F401  (re-exported for the tests)

@@ -853,3 +853,34 @@ def test_workload_mlp_bwd(P, impl):
     s1 = float(np.sum(dxh * d["x"]))
     assert abs(float(np.sum(g["dL1"] * d["L"])) - s1) <= tol
     assert abs(float(np.sum(g["dR1"] * d["R"])) - s1) <= tol
+
+
+# ----------------------------------------------------------------- a bounded wait that runs out
+
+def test_bounded_wait_runs_out_and_the_workspace_recovers(P):
+    """One operand load of the m = 128 forward is left out on the host side (nothing faults): the thread block
+    that waits for it gives up after the 5 ms limit set here, the call returns, the status word reads
+    MONARCH_ERR_TIMEOUT once, and after monarch_workspace_init the same workspace serves a correct call."""
+    import time
+    import torch
+    m, T, dtype = 128, 129, "bf16"
+    n = m * m
+    d = _small_inputs(m, T, dtype, seed=4242)
+    x, L, R = (to_device(d[k], dtype) for k in ("x", "L", "R"))
+    y = torch.full_like(x, float("nan"))
+    ws = P.Workspace(P.monarch_workspace_bytes(P.OP_FWD, T, n, m, P.BF16))
+    assert P.monarch_impl_name(P.OP_FWD, m, P.BF16) == "staged-tcgen05"
+    P.monarch_debug_set_wait_limit(ws, 5000)
+    P.monarch_debug_skip_load(0)
+    t0 = time.perf_counter()
+    P.monarch_fwd(x, L, R, y, T, n, m, ws)
+    torch.cuda.synchronize()
+    assert time.perf_counter() - t0 < 5.0          # the wait ended at its limit, not at the default second
+    assert P.monarch_last_device_status(ws) == 5   # MONARCH_ERR_TIMEOUT
+    assert P.monarch_last_device_status(ws) == 0   # cleared on read
+    P.monarch_workspace_init(ws)
+    y.fill_(float("nan"))
+    P.monarch_fwd(x, L, R, y, T, n, m, ws)
+    torch.cuda.synchronize()
+    assert P.monarch_last_device_status(ws) == 0
+    assert_close(to_host64(y), O.fwd(d["x"], d["L"], d["R"]), dtype, "y after recovery")
