@@ -15,6 +15,7 @@ NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC",
     "-cudart", "static",
+    "--threads", "0",          # one compile job per source file
 ]
 
 

@@ -428,31 +428,54 @@ plane_transpose_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_c
 // ---------------------------------------------------------------------------------------------------------
 // The whole forward pass in one persistent launch: CTA b (one per SM, 128 of them) owns block b of every step and
 // walks the token tiles; at step s it runs
-//     A: D_b[j][t] = R_b x_b(tile s)            -> u'[tile s][j][b][t]             (stage 1, rows to all j)
+//     A: D_b[j][t] = R_b x_b(tile s)            -> u'[tile s][j][b][t]                  (stage 1, rows to all j)
 //     B: D_b[l][t] = L_b u'_b(tile s - LAG)     -> w'[(tile s - LAG) % RING][l][b][t]   (stage 2)
-//     C: y[t][b*128 + j] = w'[tile s - 2 LAG][b][j][t]                              (plane b transposed)
-// B needs the rows that all 128 CTAs wrote in A two steps earlier, C those of B: one counter per tile and stage,
-// bumped by each CTA's store thread when its TMA stores have completed and polled (bounded) by the consumer's
-// loader.  Dependencies only point to earlier steps, every CTA is resident (the launch is refused otherwise), so
-// the waits cannot deadlock; the lag hides them.  x is read once and y written once; u' is also kept for the
-// backward call, w' lives in a ring of RING tiles that stays in L2.
-constexpr int kFusedLag = 2, kFusedRing = 2 * kFusedLag + 2;
-constexpr int kFusedThreads = 11 * 32;       // warps 0-3 epilogue, 4-7 transposers, 8 loader, 9 MMA, 10 store thread
+//     C: y[t][b*128 + j] = w'[tile s - 2 LAG][b][j][t]                                   (plane b transposed)
+// u' and w' are planes [tile][p][q][t] as in the three-launch chain (a producer writes 256-byte rows 32 KB apart, a
+// consumer reads one contiguous 32 KB plane by TMA).  An SM can push about 28.6 bytes per clock towards L2 whatever
+// the mechanism (load/store units or bulk copies; measured), i.e. the 96 KB a CTA writes per step cost 3.4 k
+// cycles: the stores, not the loads (70 B/clk) or the tensor pipe, bound this kernel.  Rows leave through the
+// load/store units from dedicated store warps (8 lanes per 128-byte piece); publishing a slab costs a memory fence
+// of a few thousand cycles, so kStoreSets warp pairs take the items in turn.  TMA stores were tried instead (tiled:
+// the TMA unit then carries 160 KB per step at its 30 B/clk for tiled copies; linear bulk copies of contiguous
+// slabs with the consumers gathering rows by 16-byte asynchronous copies: no faster, the store thread waits on the
+// same 28.6 B/clk) and are not kept.
+// B needs the rows that all 128 CTAs wrote in A LAG steps earlier, C those of B: one counter per tile and stage,
+// bumped by each CTA's store warps when their rows are in memory and polled (bounded) by the consumer's loader.  Dependencies only point to earlier steps, every CTA is resident (the launch is refused otherwise), so
+// the waits cannot deadlock; the lag hides them.  x is read once and y written once (by the load/store units,
+// straight from the transposed plane); u' is also kept for the backward call, w' lives in a ring of RING tiles
+// that stays in L2.
+constexpr int kFusedLag = 3, kFusedRing = 2 * kFusedLag + 2;
+constexpr int kStoreSets = 3;                // store-warp pairs taking the items in turn
+constexpr int kFusedThreads = (11 + 2 * kStoreSets) * 32;   // warps 0-3 epilogue, 4-7 transposers, 8 loader, 9 MMA, 10.. store warps, last: plane loader
 constexpr int kFusedSmem = 2 * kOpBytes /* R_b, L_b */ + 2 * kOpBytes /* operand ring */ + kStagingBytes +
                            2 * kOpBytes /* plane in, out */ + 1024;
 constexpr unsigned kFusedCounters = 8192;    // tiles per counter array (two arrays in the 64 KB after the status word)
 
 struct FusedParams {
     unsigned *status;
-    unsigned *cnt1, *cnt2;                   // per tile: CTAs whose stage-1 / stage-2 rows have landed; zero between calls
+    unsigned *cnt1, *cnt2;                   // per tile: store warps (two per CTA) whose stage-1 / stage-2 rows are in memory
+    char *u, *w, *y;                         // u' planes, w' ring, output
+    long long tokens;
     int ntiles;
+    long long *trace;                        // debug builds: per-CTA cycle sums of the waits, else null
 };
+
+#ifdef MONARCH_TRACE
+#define FT0() const long long ft0_ = clock64()
+#define FACC(v) v += clock64() - ft0_
+#define FOUT(site, v) do { if (p.trace) p.trace[blockIdx.x * 16 + (site)] = (v); } while (0)
+#else
+#define FT0() do { } while (0)
+#define FACC(v) do { } while (0)
+#define FOUT(site, v) do { } while (0)
+#endif
 
 struct FusedBars {
     uint64_t w_full;
     uint64_t full[2], empty[2];
     uint64_t acc_full[2], acc_empty[2];
-    uint64_t st_full[2], st_free[2];
+    uint64_t st_full[2 * kStoreSets], st_free[2];   // st_full: one per store-warp set and staging half
     uint64_t tr_full, tr_empty;
 };
 
@@ -464,9 +487,10 @@ __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned *p)
 }
 __device__ __forceinline__ void fence_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
 
-// Wait (bounded) until all `need` producers of a tile have published; the last of the `need` consumers to get here
-// puts the counter back to zero for the next call.
-__device__ __forceinline__ bool wait_counter(unsigned *ctr, unsigned need, unsigned *status, volatile int *dead)
+// Wait (bounded) until all `need` producers of a tile have published; the last of the `consumers` to get here puts
+// the counter back to zero for the next call.
+__device__ __forceinline__ bool wait_counter(unsigned *ctr, unsigned need, unsigned consumers, unsigned *status,
+                                             volatile int *dead)
 {
     if (ld_acquire_gpu(ctr) < need) {
         const unsigned long long t0 = global_timer_ns(), limit = wait_limit_ns(status);
@@ -478,17 +502,15 @@ __device__ __forceinline__ bool wait_counter(unsigned *ctr, unsigned need, unsig
             }
         }
     }
-    if (atomicAdd(ctr, 1u) + 1 == 2 * need) atomicExch(ctr, 0u);
+    if (atomicAdd(ctr, 1u) + 1 == need + consumers) atomicExch(ctr, 0u);
     fence_async_global();
     return true;
 }
 
 __global__ void __launch_bounds__(kFusedThreads, 1)
 chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_R,
-                       const __grid_constant__ CUtensorMap tm_L, const __grid_constant__ CUtensorMap tm_u_st,
-                       const __grid_constant__ CUtensorMap tm_u_ld, const __grid_constant__ CUtensorMap tm_w_st,
-                       const __grid_constant__ CUtensorMap tm_w_ld, const __grid_constant__ CUtensorMap tm_y,
-                       const FusedParams p)
+                       const __grid_constant__ CUtensorMap tm_L, const __grid_constant__ CUtensorMap tm_u_ld,
+                       const __grid_constant__ CUtensorMap tm_w_ld, const FusedParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) FusedBars bars;
@@ -510,15 +532,15 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
             mbar_init(smem_u32(&bars.empty[a]), 1);
             mbar_init(smem_u32(&bars.acc_full[a]), 1);
             mbar_init(smem_u32(&bars.acc_empty[a]), 4);
-            mbar_init(smem_u32(&bars.st_full[a]), 4);
+            for (int k = 0; k < kStoreSets; ++k) mbar_init(smem_u32(&bars.st_full[k * 2 + a]), 4);
             mbar_init(smem_u32(&bars.st_free[a]), 1);
         }
         mbar_init(smem_u32(&bars.tr_full), 1);
         mbar_init(smem_u32(&bars.tr_empty), 4);
         fence_mbar_init();
         dead_s = 0;
-        tma_prefetch_desc(&tm_x); tma_prefetch_desc(&tm_R); tma_prefetch_desc(&tm_L); tma_prefetch_desc(&tm_u_st);
-        tma_prefetch_desc(&tm_u_ld); tma_prefetch_desc(&tm_w_st); tma_prefetch_desc(&tm_w_ld); tma_prefetch_desc(&tm_y);
+        tma_prefetch_desc(&tm_x); tma_prefetch_desc(&tm_R); tma_prefetch_desc(&tm_L);
+        tma_prefetch_desc(&tm_u_ld); tma_prefetch_desc(&tm_w_ld);
     }
     if (warp == 0) {
         tmem_alloc(smem_u32(&tmem_base_s), 256);
@@ -544,34 +566,27 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
             tma_load_2d(w0 + kHalfBytes, &tm_R, 64, b * kB, wbar);
             tma_load_2d(w0 + kOpBytes, &tm_L, 0, b * kB, wbar);
             tma_load_2d(w0 + kOpBytes + kHalfBytes, &tm_L, 64, b * kB, wbar);
-            uint32_t g = 0, c = 0;                         // operand-ring items, planes loaded so far
-            bool ok = true;
-            for (int s = 0; ok && s < nsteps; ++s) {
-                if (s < nt) {
-                    const uint32_t sl = g & 1;
-                    if (!mbar_wait(empty0 + sl * 8, ((g >> 1) & 1) ^ 1, p.status, dead, kErrSlotWait)) break;
-                    mbar_expect_tx(full0 + sl * 8, kOpBytes);
-                    load_operand<kLdX>(ring0 + sl * kOpBytes, &tm_x, b, s, full0 + sl * 8);
-                    ++g;
-                }
+            uint32_t g = 0;                                // operand-ring items so far
+            [[maybe_unused]] long long wa = 0, wc = 0, wb = 0;
+            for (int s = 0; s < nsteps; ++s) {
                 const int tb = s - kFusedLag;
                 if (tb >= 0 && tb < nt) {
-                    if (!wait_counter(p.cnt1 + tb, kB, p.status, dead)) break;
+                    { FT0(); if (!wait_counter(p.cnt1 + tb, 2 * kB, kB, p.status, dead)) break; FACC(wc); }
                     const uint32_t sl = g & 1;
-                    if (!mbar_wait(empty0 + sl * 8, ((g >> 1) & 1) ^ 1, p.status, dead, kErrSlotWait)) break;
+                    { FT0(); if (!mbar_wait(empty0 + sl * 8, ((g >> 1) & 1) ^ 1, p.status, dead, kErrSlotWait)) break; FACC(wb); }
                     mbar_expect_tx(full0 + sl * 8, kOpBytes);
                     load_operand<kLdP>(ring0 + sl * kOpBytes, &tm_u_ld, b, tb, full0 + sl * 8);
                     ++g;
                 }
-                const int tc = s - 2 * kFusedLag;
-                if (tc >= 0) {
-                    if (!wait_counter(p.cnt2 + tc, kB, p.status, dead)) break;
-                    if (!mbar_wait(tre, (c & 1) ^ 1, p.status, dead, kErrSlotWait)) break;
-                    mbar_expect_tx(trf, kOpBytes);
-                    load_operand<kLdP>(trin, &tm_w_ld, b, tc % kFusedRing, trf);
-                    ++c;
+                if (s < nt) {
+                    const uint32_t sl = g & 1;
+                    { FT0(); if (!mbar_wait(empty0 + sl * 8, ((g >> 1) & 1) ^ 1, p.status, dead, kErrSlotWait)) break; FACC(wa); }
+                    mbar_expect_tx(full0 + sl * 8, kOpBytes);
+                    load_operand<kLdX>(ring0 + sl * kOpBytes, &tm_x, b, s, full0 + sl * 8);
+                    ++g;
                 }
             }
+            FOUT(0, wa); FOUT(1, wc); FOUT(2, wb);
         }
     } else if (warp == 9) {
         // ------------------------------------------------------------ MMA issuer
@@ -579,14 +594,16 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
             constexpr uint32_t idesc_a = make_idesc_bf16(128, 128, 0, 0), idesc_b = make_idesc_bf16(128, 128, 0, 1);
             uint32_t g = 0;
             bool ok = true;
+            [[maybe_unused]] long long wa = 0, wf = 0;
             for (int s = 0; ok && s < nsteps; ++s) {
 #pragma unroll
-                for (int kind = 0; kind < 2; ++kind) {
+                for (int ki = 0; ki < 2; ++ki) {
+                    const int kind = 1 - ki;                      // stage 2 of the older tile first, then stage 1
                     const int tile = kind == 0 ? s : s - kFusedLag;
                     if (tile < 0 || tile >= nt) continue;
                     const uint32_t buf = g & 1;
-                    if (!mbar_wait(acce0 + buf * 8, ((g >> 1) & 1) ^ 1, p.status, dead, kErrTmemWait)) { ok = false; break; }
-                    if (!mbar_wait(full0 + buf * 8, (g >> 1) & 1, p.status, dead, kErrTmaWait)) { ok = false; break; }
+                    { FT0(); if (!mbar_wait(acce0 + buf * 8, ((g >> 1) & 1) ^ 1, p.status, dead, kErrTmemWait)) { ok = false; break; } FACC(wa); }
+                    { FT0(); if (!mbar_wait(full0 + buf * 8, (g >> 1) & 1, p.status, dead, kErrTmaWait)) { ok = false; break; } FACC(wf); }
                     tc_fence_after();
                     const uint32_t t0 = ring0 + buf * kOpBytes, w = w0 + kind * kOpBytes, d = tmem_base + buf * 128;
 #pragma unroll
@@ -597,6 +614,7 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
                     ++g;
                 }
             }
+            FOUT(3, wa); FOUT(4, wf);
         }
     } else if (warp < 4) {
         // ------------------------------------------------------------ epilogue: TMEM -> bf16 -> staging halves
@@ -604,13 +622,16 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
         const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
         uint32_t g = 0;
         bool ok = true;
+        [[maybe_unused]] long long wa = 0, ws = 0;
+        [[maybe_unused]] const long long te0 = clock64();
         for (int s = 0; ok && s < nsteps; ++s) {
 #pragma unroll 1
-            for (int kind = 0; kind < 2; ++kind) {
+            for (int ki = 0; ki < 2; ++ki) {
+                const int kind = 1 - ki;
                 const int tile = kind == 0 ? s : s - kFusedLag;
                 if (tile < 0 || tile >= nt) continue;
                 const uint32_t buf = g & 1;
-                if (!mbar_wait(accf0 + buf * 8, (g >> 1) & 1, p.status, dead, kErrMmaWait)) { ok = false; break; }
+                { FT0(); if (!mbar_wait(accf0 + buf * 8, (g >> 1) & 1, p.status, dead, kErrMmaWait)) { ok = false; break; } FACC(wa); }
                 tc_fence_after();
 #pragma unroll 1
                 for (int h = 0; h < 2; ++h) {
@@ -624,7 +645,7 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
                         if (lane == 0) mbar_arrive(acce0 + buf * 8);
                     }
                     // staging half h is free once the store of the previous item's half h has read it
-                    if (!mbar_wait(stfree0 + h * 8, (g & 1) ^ 1, p.status, dead, kErrSlotWait)) { ok = false; break; }
+                    { FT0(); if (!mbar_wait(stfree0 + h * 8, (g & 1) ^ 1, p.status, dead, kErrSlotWait)) { ok = false; break; } FACC(ws); }
                     const uint32_t dst = staging0 + h * kHalfBytes + row * 128;
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
@@ -636,67 +657,85 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
                         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((c ^ (row & 7)) << 4)),
                                      "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
                     }
-                    fence_proxy_async_smem();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(stf0 + h * 8);
+                    if (lane == 0) mbar_arrive(stf0 + ((g % kStoreSets) * 2 + h) * 8);
                 }
                 if (!ok) break;
                 ++g;
             }
         }
-    } else if (warp == 10) {
-        // ------------------------------------------------------------ store thread: staging -> u' / w', publish
-        if (lane == 0) {
-            uint32_t g = 0;
-            int prev_kind = -1, prev_tile = 0;
-            bool ok = true;
-            for (int s = 0; ok && s < nsteps; ++s) {
+        if (threadIdx.x == 0) { FOUT(5, wa); FOUT(6, ws); FOUT(7, clock64() - te0); }
+    } else if (warp >= 10 && warp < 10 + 2 * kStoreSets) {
+        // ------------------------------------------------------------ store warps (per set: one per staging half):
+        // rows of D leave as 128-byte pieces through the load/store units (8 lanes per row), then this warp's part
+        // of the tile is published
+        const int h = (warp - 10) & 1, set = (warp - 10) >> 1;
+        const uint32_t src = staging0 + h * kHalfBytes;
+        uint32_t g = 0;
+        bool ok = true;
+        [[maybe_unused]] long long wf = 0;
+        [[maybe_unused]] const long long ts0 = clock64();
+        for (int s = 0; ok && s < nsteps; ++s) {
 #pragma unroll 1
-                for (int kind = 0; kind < 2; ++kind) {
-                    const int tile = kind == 0 ? s : s - kFusedLag;
-                    if (tile < 0 || tile >= nt) continue;
-#pragma unroll 1
-                    for (int h = 0; h < 2; ++h) {
-                        if (!mbar_wait(stf0 + h * 8, g & 1, p.status, dead, kErrMmaWait)) { ok = false; break; }
-                        if (kind == 0) tma_store_4d(&tm_u_st, staging0 + h * kHalfBytes, h * 64, b, 0, tile);
-                        else tma_store_4d(&tm_w_st, staging0 + h * kHalfBytes, h * 64, b, 0, tile % kFusedRing);
-                        tma_store_commit();
-                        // the store committed before this one has read its staging half
-                        if (g != 0 || h != 0) {
-                            tma_store_wait_read<1>();
-                            mbar_arrive(stfree0 + (h ^ 1) * 8);
-                        }
+            for (int ki = 0; ki < 2; ++ki) {
+                const int kind = 1 - ki;
+                const int tile = kind == 0 ? s : s - kFusedLag;
+                if (tile < 0 || tile >= nt) continue;
+                if ((int)(g % kStoreSets) != set) { ++g; continue; }
+                { FT0(); if (!mbar_wait(stf0 + (set * 2 + h) * 8, (g / kStoreSets) & 1, p.status, dead, kErrMmaWait)) { ok = false; break; } FACC(wf); }
+                char *dst = (kind == 0 ? p.u + (size_t)tile * (kB * kOpBytes) : p.w + (size_t)(tile % kFusedRing) * (kB * kOpBytes)) +
+                            b * 256 + h * 128 + (lane & 7) * 16;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    uint4 v[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int r = (q * 8 + i) * 4 + (lane >> 3);
+                        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v[i].x), "=r"(v[i].y), "=r"(v[i].z), "=r"(v[i].w)
+                                     : "r"(src + r * 128 + (((lane & 7) ^ (r & 7)) << 4)) : "memory");
                     }
-                    if (!ok) break;
-                    // all but the two stores just issued have completed: the previous item's rows are in memory
-                    if (prev_kind >= 0) {
-                        tma_store_wait_all<2>();
-                        fence_async_global();
-                        __threadfence();
-                        atomicAdd((prev_kind == 0 ? p.cnt1 : p.cnt2) + prev_tile, 1u);
+                    if (q == 3) {
+                        // the staging half is in registers: hand it back to the epilogue
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(stfree0 + h * 8);
                     }
-                    prev_kind = kind;
-                    prev_tile = tile;
-                    ++g;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int r = (q * 8 + i) * 4 + (lane >> 3);
+                        *reinterpret_cast<uint4 *>(dst + (size_t)r * kOpBytes) = v[i];
+                    }
                 }
-            }
-            tma_store_wait_all<0>();
-            if (ok && prev_kind >= 0) {
-                fence_async_global();
                 __threadfence();
-                atomicAdd((prev_kind == 0 ? p.cnt1 : p.cnt2) + prev_tile, 1u);
+                __syncwarp();
+                if (lane == 0) atomicAdd((kind == 0 ? p.cnt1 : p.cnt2) + tile, 1u);
+                ++g;
             }
+        }
+        if (warp == 10 && lane == 0) { FOUT(8, wf); FOUT(9, clock64() - ts0); }
+    } else if (warp == 10 + 2 * kStoreSets) {
+        // ------------------------------------------------------------ plane loader
+        if (lane == 0) {
+            uint32_t c = 0;
+            [[maybe_unused]] long long wc = 0, we = 0;
+            for (int s = 2 * kFusedLag; s < nsteps; ++s, ++c) {
+                const int tc = s - 2 * kFusedLag;
+                { FT0(); if (!wait_counter(p.cnt2 + tc, 2 * kB, kB, p.status, dead)) break; FACC(wc); }
+                { FT0(); if (!mbar_wait(tre, (c & 1) ^ 1, p.status, dead, kErrSlotWait)) break; FACC(we); }
+                mbar_expect_tx(trf, kOpBytes);
+                load_operand<kLdP>(trin, &tm_w_ld, b, tc % kFusedRing, trf);
+            }
+            FOUT(10, wc); FOUT(11, we);
         }
     } else {
         // ------------------------------------------------------------ transposers (warps 4-7): plane b of w' -> y
         const int tw = warp - 4;
-        const int tid = threadIdx.x - 128;
         uint32_t c = 0;
+        [[maybe_unused]] long long wf = 0;
+        [[maybe_unused]] const long long tt0 = clock64();
         for (int s = 2 * kFusedLag; s < nsteps; ++s, ++c) {
             const int tile = s - 2 * kFusedLag;
-            if (!mbar_wait(trf, c & 1, p.status, dead, kErrTmaWait)) break;
-            // the stores of the previous plane have read the output buffer
-            if (tid == 0) tma_store_wait_read<0>();
+            { FT0(); if (!mbar_wait(trf, c & 1, p.status, dead, kErrTmaWait)) break; FACC(wf); }
+            // every warp has copied its rows of the previous plane out of the output buffer
             asm volatile("bar.sync 2, 128;" ::: "memory");
 #pragma unroll 1
             for (int ro = 0; ro < 4; ++ro) {
@@ -715,17 +754,29 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
                                  "r"(bq), "r"(cc), "r"(d) : "memory");
                 }
             }
-            fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(tre);
             asm volatile("bar.sync 2, 128;" ::: "memory");
-            if (tid == 0) {
-                tma_store_2d(&tm_y, trout, b * kB, tile * 128);
-                tma_store_2d(&tm_y, trout + kHalfBytes, b * kB + 64, tile * 128);
-                tma_store_commit();
+            // rows t = 32 tw .. 32 tw + 31 of y[t][b*128 ..], two 128-byte pieces each; rows past the last token stay put
+            char *yrow = p.y + ((size_t)tile * 128) * kOpBytes + b * 256 + (lane & 7) * 16;
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                uint4 v[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = tw * 32 + i * 4 + (lane >> 3);
+                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v[i].x), "=r"(v[i].y), "=r"(v[i].z), "=r"(v[i].w)
+                                 : "r"(trout + hh * kHalfBytes + r * 128 + (((lane & 7) ^ (r & 7)) << 4)) : "memory");
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int t = tw * 32 + i * 4 + (lane >> 3);
+                    if ((long long)tile * 128 + t < p.tokens)
+                        *reinterpret_cast<uint4 *>(yrow + (size_t)t * kOpBytes + hh * 128) = v[i];
+                }
             }
         }
-        if (tid == 0) tma_store_wait_all<0>();
+        if (warp == 4 && lane == 0) { FOUT(12, wf); FOUT(13, clock64() - tt0); }
     }
 
     tc_fence_before();
@@ -818,8 +869,23 @@ size_t chain_fwd_m128_workspace_bytes(int64_t tokens)
 {
     return MONARCH_STATUS_BYTES + kChainCounterBytes + 2 * tc::planes_bytes(tokens);
 }
-const void *chain_fwd_m128_saved_u(const void *fwd_ws)
+namespace tc {
+namespace {
+// true when chain_fwd_m128 runs as one persistent launch for this many tokens (every CTA resident, counters fit)
+bool fwd_runs_fused(int64_t tokens)
 {
+    int sms = 0;
+    if (device_sms(&sms) != MONARCH_OK) return false;
+    return chain_fused_enabled() && sms >= kB && (tokens + 127) / 128 <= (int64_t)kFusedCounters;
+}
+}  // namespace
+}  // namespace tc
+
+// u' as the three-launch forward leaves it (planes [tile][j][k][t]); null when the forward call ran as one launch,
+// whose slabs the chain of separate backward launches does not read
+const void *chain_fwd_m128_saved_u(const void *fwd_ws, int64_t tokens)
+{
+    if (tc::fwd_runs_fused(tokens)) return nullptr;
     return (const char *)fwd_ws + MONARCH_STATUS_BYTES + kChainCounterBytes;
 }
 // Backward workspace: [status][dw' planes][du' planes][u' planes (when the forward call's are not passed)]
@@ -843,10 +909,7 @@ int chain_fwd_m128(const void *x, const void *L, const void *R, void *y, int64_t
     MONARCH_TRY(map_planes(&mu_p, up, ntiles, true));
     MONARCH_TRY(map_planes(&mw_q, wp, ntiles, false));
     MONARCH_TRY(map_planes(&mw_p, wp, ntiles, true));
-    int sms = 0;
-    MONARCH_TRY(device_sms(&sms));
-    if (chain_fused_enabled() && sms >= kB && ntiles <= (int)kFusedCounters &&
-        g_skip_load.load(std::memory_order_relaxed) < 0) {
+    if (fwd_runs_fused(tokens) && g_skip_load.load(std::memory_order_relaxed) < 0) {
         // one persistent launch; every CTA must be resident at once (one per SM)
         MONARCH_CUDA_TRY(cudaFuncSetAttribute(chain_fused_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmem));
         FusedParams fp;
@@ -854,7 +917,15 @@ int chain_fwd_m128(const void *x, const void *L, const void *R, void *y, int64_t
         fp.cnt1 = (unsigned *)((char *)ws + MONARCH_STATUS_BYTES);
         fp.cnt2 = fp.cnt1 + kFusedCounters;
         fp.ntiles = ntiles;
-        chain_fused_fwd_kernel<<<kB, kFusedThreads, kFusedSmem, s>>>(mx, mR, mL, mu_q, mu_p, mw_q, mw_p, my, fp);
+        fp.u = up;
+        fp.w = wp;
+        fp.y = (char *)y;
+        fp.tokens = tokens;
+        fp.trace = nullptr;
+#ifdef MONARCH_TRACE
+        if (const char *e = getenv("MONARCH_TRACE_PTR")) fp.trace = (long long *)strtoull(e, nullptr, 0);
+#endif
+        chain_fused_fwd_kernel<<<kB, kFusedThreads, kFusedSmem, s>>>(mx, mR, mL, mu_p, mw_p, fp);
         note_launch();
         MONARCH_CUDA_TRY(cudaGetLastError());
         return MONARCH_OK;

@@ -257,7 +257,7 @@ int monarch_bwd(const void *x, const void *dy, const void *L, const void *R, con
     if (which == kTcStaged) {
         const bool saved = fwd_workspace != nullptr && m == 128 && pick(MONARCH_OP_FWD, m, dtype) == kTcStaged;
         return tc_staged_bwd(x, dy, L, R, dx, dL, dR, accumulate, 1, 1, tokens, m, workspace, s,
-                             saved ? chain_fwd_m128_saved_u(fwd_workspace) : nullptr);
+                             saved ? chain_fwd_m128_saved_u(fwd_workspace, tokens) : nullptr);
     }
     MONARCH_TRY(staged_bwd_dx(dy, L, R, dx, tokens, m, dtype, workspace, s));
     return staged_bwd_dw(x, dy, L, R, dL, dR, accumulate, tokens, m, dtype, workspace, s);
