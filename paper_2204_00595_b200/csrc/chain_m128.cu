@@ -785,6 +785,273 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
 }
 
 // ---------------------------------------------------------------------------------------------------------
+// The two block products of the backward pass and both token reductions in one persistent launch (the plane
+// transpose of dy runs before it as a launch of its own).  CTA b owns block b: at step s it runs
+//     E: D[k][t] = L_b^T dw'_b(tile s)         -> du'[tile s % RING][k][b][t]      dL_b += dw'_b u'_b^T   (over t)
+//     F: D[t][i] = du'_b(tile s - LAG)^T R_b   -> dx[t][b*128 + i]                dR_b += du'_b x_b      (over t)
+// with du' in an L2-resident ring, one counter per tile (bumped by the store warps of E, polled by the loader of
+// F), the two 128 x 128 fp32 sums resident in TMEM from the first tile to the last (one writer per block: the sums
+// are deterministic) and added to dL, dR at the end.  A ring slot holds the two operands of an item (64 KB).
+constexpr int kBwdSlotBytes = 2 * kOpBytes;
+constexpr int kBwdThreads = (6 + 2 * kStoreSets) * 32;      // warps 0-3 epilogue, 4 loader, 5 MMA, 6.. store warps
+constexpr int kBwdSmem = 2 * kOpBytes + 2 * kBwdSlotBytes + kStagingBytes + 1024;
+
+struct FusedBwdParams {
+    unsigned *status;
+    unsigned *cnt;                           // per tile: store warps (two per CTA) whose du' rows are in memory
+    char *du, *dx;                           // du' ring, output
+    float *dL, *dR;                          // added to
+    long long tokens;
+    int ntiles;
+};
+
+struct FusedBwdBars {
+    uint64_t w_full;
+    uint64_t full[2], empty[2];
+    uint64_t acc_full[2], acc_empty[2];
+    uint64_t st_full[2 * kStoreSets], st_free[2];
+    uint64_t wg_full;
+};
+
+__global__ void __launch_bounds__(kBwdThreads, 1)
+chain_fused_bwd_kernel(const __grid_constant__ CUtensorMap tm_dw, const __grid_constant__ CUtensorMap tm_u,
+                       const __grid_constant__ CUtensorMap tm_du, const __grid_constant__ CUtensorMap tm_x,
+                       const __grid_constant__ CUtensorMap tm_R, const __grid_constant__ CUtensorMap tm_L,
+                       const FusedBwdParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) FusedBwdBars bars;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int dead_s;
+
+    const uint32_t w0 = (smem_u32(smem_raw) + 1023u) & ~1023u;          // L_b, R_b
+    const uint32_t ring0 = w0 + 2 * kOpBytes;
+    const uint32_t staging0 = ring0 + 2 * kBwdSlotBytes;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int b = (int)blockIdx.x;
+    volatile int *dead = &dead_s;
+
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bars.w_full), 1);
+        mbar_init(smem_u32(&bars.wg_full), 1);
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(smem_u32(&bars.full[a]), 1);
+            mbar_init(smem_u32(&bars.empty[a]), 1);
+            mbar_init(smem_u32(&bars.acc_full[a]), 1);
+            mbar_init(smem_u32(&bars.acc_empty[a]), 4);
+            for (int k = 0; k < kStoreSets; ++k) mbar_init(smem_u32(&bars.st_full[k * 2 + a]), 4);
+            mbar_init(smem_u32(&bars.st_free[a]), 1);
+        }
+        fence_mbar_init();
+        dead_s = 0;
+        tma_prefetch_desc(&tm_dw); tma_prefetch_desc(&tm_u); tma_prefetch_desc(&tm_du); tma_prefetch_desc(&tm_x);
+        tma_prefetch_desc(&tm_R); tma_prefetch_desc(&tm_L);
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&tmem_base_s), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+
+    const int nt = p.ntiles, nsteps = nt + kFusedLag;
+    const uint32_t full0 = smem_u32(bars.full), empty0 = smem_u32(bars.empty);
+    const uint32_t accf0 = smem_u32(bars.acc_full), acce0 = smem_u32(bars.acc_empty);
+    const uint32_t stf0 = smem_u32(bars.st_full), stfree0 = smem_u32(bars.st_free);
+    const uint32_t wgf = smem_u32(&bars.wg_full);
+
+    // item order within a step: F of the older tile first, then E
+    if (warp == 4) {
+        // ------------------------------------------------------------ loader
+        if (lane == 0) {
+            const uint32_t wbar = smem_u32(&bars.w_full);
+            mbar_expect_tx(wbar, 2 * kOpBytes);
+            tma_load_2d(w0, &tm_L, 0, b * kB, wbar);
+            tma_load_2d(w0 + kHalfBytes, &tm_L, 64, b * kB, wbar);
+            tma_load_2d(w0 + kOpBytes, &tm_R, 0, b * kB, wbar);
+            tma_load_2d(w0 + kOpBytes + kHalfBytes, &tm_R, 64, b * kB, wbar);
+            uint32_t g = 0;
+            for (int s = 0; s < nsteps; ++s) {
+                const int tf = s - kFusedLag;
+                if (tf >= 0) {
+                    if (!wait_counter(p.cnt + tf, 2 * kB, kB, p.status, dead)) break;
+                    const uint32_t sl = g & 1;
+                    if (!mbar_wait(empty0 + sl * 8, ((g >> 1) & 1) ^ 1, p.status, dead, kErrSlotWait)) break;
+                    mbar_expect_tx(full0 + sl * 8, kBwdSlotBytes);
+                    load_operand<kLdP>(ring0 + sl * kBwdSlotBytes, &tm_du, b, tf % kFusedRing, full0 + sl * 8);
+                    load_operand<kLdX>(ring0 + sl * kBwdSlotBytes + kOpBytes, &tm_x, b, tf, full0 + sl * 8);
+                    ++g;
+                }
+                if (s < nt) {
+                    const uint32_t sl = g & 1;
+                    if (!mbar_wait(empty0 + sl * 8, ((g >> 1) & 1) ^ 1, p.status, dead, kErrSlotWait)) break;
+                    mbar_expect_tx(full0 + sl * 8, kBwdSlotBytes);
+                    load_operand<kLdQ>(ring0 + sl * kBwdSlotBytes, &tm_dw, b, s, full0 + sl * 8);
+                    load_operand<kLdP>(ring0 + sl * kBwdSlotBytes + kOpBytes, &tm_u, b, s, full0 + sl * 8);
+                    ++g;
+                }
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0 && mbar_wait(smem_u32(&bars.w_full), 0, p.status, dead, kErrTmaWait)) {
+            constexpr uint32_t idesc_main = make_idesc_bf16(128, 128, 1, 1);
+            constexpr uint32_t idesc_dl = make_idesc_bf16(128, 128, 0, 0), idesc_dr = make_idesc_bf16(128, 128, 0, 1);
+            uint32_t g = 0;
+            bool ok = true, first_dl = true, first_dr = true;
+            for (int s = 0; ok && s < nsteps; ++s) {
+#pragma unroll
+                for (int ki = 0; ki < 2; ++ki) {
+                    const int kind = 1 - ki;                  // 1 = F, 0 = E
+                    const int tile = kind == 0 ? s : s - kFusedLag;
+                    if (tile < 0 || tile >= nt) continue;
+                    const uint32_t buf = g & 1;
+                    if (!mbar_wait(acce0 + buf * 8, ((g >> 1) & 1) ^ 1, p.status, dead, kErrTmemWait)) { ok = false; break; }
+                    if (!mbar_wait(full0 + buf * 8, (g >> 1) & 1, p.status, dead, kErrTmaWait)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t t0 = ring0 + buf * kBwdSlotBytes, t1 = t0 + kOpBytes, w = w0 + kind * kOpBytes;
+                    const uint32_t d = tmem_base + buf * 128;
+                    // E: A = L_b^T (weights, MN-major), B = dw' tile (MN-major); F: A = du' tile (MN-major), B = R_b (MN-major)
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint64_t dwt = op_desc(w, true, ks), dt = op_desc(t0, true, ks);
+                        mma_f16_ss(d, kind == 0 ? dwt : dt, kind == 0 ? dt : dwt, idesc_main, ks != 0);
+                    }
+                    mma_commit(accf0 + buf * 8);
+                    // token reductions: rows of T0 as M, tokens as K
+                    const uint32_t dsum = tmem_base + 256 + kind * 128;
+                    bool &first = kind == 0 ? first_dl : first_dr;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)
+                        mma_f16_ss(dsum, op_desc(t0, false, ks), op_desc(t1, kind == 1, ks), kind == 0 ? idesc_dl : idesc_dr,
+                                   !(first && ks == 0));
+                    first = false;
+                    mma_commit(empty0 + buf * 8);
+                    ++g;
+                }
+            }
+            if (ok) mma_commit(wgf);
+        }
+    } else if (warp < 4) {
+        // ------------------------------------------------------------ epilogue: TMEM -> bf16 -> staging halves
+        const int row = warp * 32 + lane;
+        const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+        uint32_t g = 0;
+        bool ok = true;
+        for (int s = 0; ok && s < nsteps; ++s) {
+#pragma unroll 1
+            for (int ki = 0; ki < 2; ++ki) {
+                const int kind = 1 - ki;
+                const int tile = kind == 0 ? s : s - kFusedLag;
+                if (tile < 0 || tile >= nt) continue;
+                const uint32_t buf = g & 1;
+                if (!mbar_wait(accf0 + buf * 8, (g >> 1) & 1, p.status, dead, kErrMmaWait)) { ok = false; break; }
+                tc_fence_after();
+#pragma unroll 1
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t v[4][16];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) tmem_ld16(lane_base + buf * 128 + h * 64 + q * 16, v[q]);
+                    tmem_ld_wait();
+                    if (h == 1) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(acce0 + buf * 8);
+                    }
+                    if (!mbar_wait(stfree0 + h * 8, (g & 1) ^ 1, p.status, dead, kErrSlotWait)) { ok = false; break; }
+                    const uint32_t dst = staging0 + h * kHalfBytes + row * 128;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const uint32_t *w = &v[c >> 1][(c & 1) * 8];
+                        const uint32_t o0 = pack_bf16(__uint_as_float(w[0]), __uint_as_float(w[1]));
+                        const uint32_t o1 = pack_bf16(__uint_as_float(w[2]), __uint_as_float(w[3]));
+                        const uint32_t o2 = pack_bf16(__uint_as_float(w[4]), __uint_as_float(w[5]));
+                        const uint32_t o3 = pack_bf16(__uint_as_float(w[6]), __uint_as_float(w[7]));
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((c ^ (row & 7)) << 4)),
+                                     "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(stf0 + ((g % kStoreSets) * 2 + h) * 8);
+                }
+                if (!ok) break;
+                ++g;
+            }
+        }
+        // the token sums of this block: dL_b (columns 256..383) and dR_b (384..511), one writer per element
+        if (ok && mbar_wait(wgf, 0, p.status, dead, kErrMmaWait)) {
+            tc_fence_after();
+#pragma unroll 1
+            for (int which = 0; which < 2; ++which) {
+                float *out = (which == 0 ? p.dL : p.dR) + ((size_t)b * kB + row) * kB;
+#pragma unroll 1
+                for (int c = 0; c < kB; c += 16) {
+                    uint32_t v[16];
+                    tmem_ld16(lane_base + 256 + which * 128 + c, v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(out + c + e * 4),
+                                     "f"(__uint_as_float(v[e * 4])), "f"(__uint_as_float(v[e * 4 + 1])),
+                                     "f"(__uint_as_float(v[e * 4 + 2])), "f"(__uint_as_float(v[e * 4 + 3]))
+                                     : "memory");
+                }
+            }
+        }
+    } else if (warp >= 6 && warp < 6 + 2 * kStoreSets) {
+        // ------------------------------------------------------------ store warps: rows of D leave as 128-byte pieces
+        const int h = (warp - 6) & 1, set = (warp - 6) >> 1;
+        const uint32_t src = staging0 + h * kHalfBytes;
+        uint32_t g = 0;
+        bool ok = true;
+        for (int s = 0; ok && s < nsteps; ++s) {
+#pragma unroll 1
+            for (int ki = 0; ki < 2; ++ki) {
+                const int kind = 1 - ki;
+                const int tile = kind == 0 ? s : s - kFusedLag;
+                if (tile < 0 || tile >= nt) continue;
+                if ((int)(g % kStoreSets) != set) { ++g; continue; }
+                if (!mbar_wait(stf0 + (set * 2 + h) * 8, (g / kStoreSets) & 1, p.status, dead, kErrMmaWait)) { ok = false; break; }
+                // E: row k of du'[ring][k][b][t]; F: token row t of dx[t][b*128 ..] (rows past the last token stay put)
+                char *dst = (kind == 0 ? p.du + (size_t)(tile % kFusedRing) * (kB * kOpBytes) : p.dx + (size_t)tile * (kB * kOpBytes)) +
+                            b * 256 + h * 128 + (lane & 7) * 16;
+                const int rows_ok = kind == 0 ? 128 : (int)((p.tokens - (long long)tile * 128) < 128 ? (p.tokens - (long long)tile * 128) : 128);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    uint4 v[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int r = (q * 8 + i) * 4 + (lane >> 3);
+                        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v[i].x), "=r"(v[i].y), "=r"(v[i].z), "=r"(v[i].w)
+                                     : "r"(src + r * 128 + (((lane & 7) ^ (r & 7)) << 4)) : "memory");
+                    }
+                    if (q == 3) {
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(stfree0 + h * 8);
+                    }
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int r = (q * 8 + i) * 4 + (lane >> 3);
+                        if (r < rows_ok) *reinterpret_cast<uint4 *>(dst + (size_t)r * kOpBytes) = v[i];
+                    }
+                }
+                if (kind == 0) {
+                    __threadfence();
+                    __syncwarp();
+                    if (lane == 0) atomicAdd(p.cnt + tile, 1u);
+                }
+                ++g;
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem_base, 512);
+}
+
+// ---------------------------------------------------------------------------------------------------------
 struct Maps {
     CUtensorMap x2d;       // token-major [tokens][n], box 128 rows x 64 columns
     CUtensorMap p4d;       // planes [tile][p][q][t], box = rows q of one p
@@ -881,15 +1148,17 @@ bool fwd_runs_fused(int64_t tokens)
 }  // namespace
 }  // namespace tc
 
-// u' as the three-launch forward leaves it (planes [tile][j][k][t]); null when the forward call ran as one launch,
-// whose slabs the chain of separate backward launches does not read
+// u' as either form of the forward pass leaves it: planes [tile][j][k][t]
 const void *chain_fwd_m128_saved_u(const void *fwd_ws, int64_t tokens)
 {
-    if (tc::fwd_runs_fused(tokens)) return nullptr;
+    (void)tokens;
     return (const char *)fwd_ws + MONARCH_STATUS_BYTES + kChainCounterBytes;
 }
-// Backward workspace: [status][dw' planes][du' planes][u' planes (when the forward call's are not passed)]
-size_t chain_bwd_m128_workspace_bytes(int64_t tokens) { return MONARCH_STATUS_BYTES + 3 * tc::planes_bytes(tokens); }
+// Backward workspace: [status][tile counters 64 KB][dw' planes][du' planes][u' planes (when the forward call's are not passed)]
+size_t chain_bwd_m128_workspace_bytes(int64_t tokens)
+{
+    return MONARCH_STATUS_BYTES + kChainCounterBytes + 3 * tc::planes_bytes(tokens);
+}
 
 // y = P L P^T R x (Def. 3.1; Section 3.3 steps 1-3) in three launches.
 int chain_fwd_m128(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws, cudaStream_t s)
@@ -948,7 +1217,8 @@ int chain_bwd_m128(const void *x, const void *dy, const void *L, const void *R, 
     if (tokens > (int64_t)1 << 30) return MONARCH_ERR_UNSUPPORTED;
     const int ntiles = (int)((tokens + 127) / 128);
     unsigned *status = (unsigned *)ws;
-    char *dwp = (char *)ws + MONARCH_STATUS_BYTES, *dup = dwp + planes_bytes(tokens), *up_own = dup + planes_bytes(tokens);
+    char *dwp = (char *)ws + MONARCH_STATUS_BYTES + kChainCounterBytes, *dup = dwp + planes_bytes(tokens),
+         *up_own = dup + planes_bytes(tokens);
     CUtensorMap mx, mdy, mdx, mR, mL, mdw_p, mdw_q, mdu_q, mdu_p, mu_q, mu_p;
     MONARCH_TRY(map_tokens(&mdy, dy, tokens));
     MONARCH_TRY(map_weights(&mR, R));
@@ -970,6 +1240,23 @@ int chain_bwd_m128(const void *x, const void *dy, const void *L, const void *R, 
     }
     // dw'[tile][l][j][t] = dy[t][l*128+j]
     MONARCH_TRY(launch_transpose<true>(mdy, mdw_p, ntiles, status, s));
+    if (want_dw && want_dx && fwd_runs_fused(tokens)) {
+        // both block products and both token reductions in one persistent launch (every CTA resident)
+        MONARCH_CUDA_TRY(cudaFuncSetAttribute(chain_fused_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmem));
+        FusedBwdParams bp;
+        bp.status = status;
+        bp.cnt = (unsigned *)((char *)ws + MONARCH_STATUS_BYTES);
+        bp.du = dup;
+        bp.dx = (char *)dx;
+        bp.dL = dL;
+        bp.dR = dR;
+        bp.tokens = tokens;
+        bp.ntiles = ntiles;
+        chain_fused_bwd_kernel<<<kB, kBwdThreads, kBwdSmem, s>>>(mdw_q, mu_p, mdu_p, mx, mR, mL, bp);
+        note_launch();
+        MONARCH_CUDA_TRY(cudaGetLastError());
+        return MONARCH_OK;
+    }
     // du'[tile][k][j][t] = sum_l L[j][l][k] dw'[tile][l][j][t]   (+ dL[j][l][k] += sum_t dw'[..][l][j][t] u'[..][j][k][t])
     if (want_dw)
         MONARCH_TRY((launch_gemm<kLdQ, true, true, true, kStQ, true, kLdP, false, true>(mdw_q, mu_p, mL, mdu_q, dL, ntiles, status, s)));
