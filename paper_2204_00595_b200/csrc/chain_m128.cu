@@ -6,17 +6,24 @@
 // token) fit an SM, so the permuted intermediate cannot be assembled on chip.  What can be chosen freely is which
 // index of an intermediate is contiguous in memory: the tensor cores read an operand either with its contraction
 // index contiguous ("K-major") or with its row/column index contiguous ("MN-major").  All intermediates here are
-// stored TOKEN-INNERMOST in tiles of 128 tokens, as [tile][p][q][t]:
-//     u'  = [tile][j][k][t]    written by stage 1 block k as rows j of D_k[j][t]   (q = k fixed, 256-byte rows)
-//                              read by stage 2 block j as the 32 KB slab [k][t]    (p = j fixed), an MN-major operand
-//     w'  = [tile][l][j][t]    written by stage 2 block j as rows l of D_j[l][t]; a last pass transposes the
-//                              128 x 128 (j, t) planes into y[t][l*128 + j] - both sides in 256-byte rows.
-// So every global access of the whole chain is a 128- or 256-byte row, the inner permutation of Def. 3.1 is the
-// choice of a store box, and the outer one is a plane transpose through shared memory (ldmatrix.trans / stmatrix).
-// The adjoints reverse the chain (transpose dy into dw' = [tile][l][j][t], du'[k][t] = L_j^T dw'_j written as
-// [tile][k][j][t], dx = du'_k^T R_k), and because the token index is contiguous the same tiles are K-major operands
-// of the token reductions dL_j = dw'_j u'_j^T and dR_k = du'_k x_k, which ride along in the same kernels with their
-// accumulators resident in TMEM for all tiles of a block (one writer per block: deterministic sums).
+// stored TOKEN-INNERMOST in tiles of 128 tokens and CONSUMER-CONTIGUOUS: every intermediate is written by 128
+// producer blocks p and read by 128 consumer blocks c (every consumer needs one 128 x 128 slab made of one row of
+// every producer's result), and lives as
+//     [tile][c][half h][p][64 tokens]      (a 128-byte row = tokens 64h .. 64h+63 of row c of producer p's result)
+// with the eight 16-byte chunks of a row stored at position (chunk XOR p % 8).  A consumer's slab [c] is then 32 KB
+// contiguous and is, byte for byte, the 128-byte-swizzled shared-memory image of a tensor-core operand with rows p:
+// ONE linear bulk copy fetches it (linear copies run at 72 B/clk per SM, tiled TMA copies of 128-byte rows at 33;
+// measured), read MN-major (tokens as the row/column index) by the block products and K-major (tokens as the
+// contraction index) by the token reductions.  A producer writes 128-byte pieces 32 KB apart.
+//     u'  (c = j, p = k)  rows j of D_k[j][t] = R_k x_k        -> operand of stage 2, block j
+//     w'  (c = l, p = j)  rows l of D_j[l][t] = L_j u'_j       -> plane l, transposed through shared memory
+//                         (ldmatrix.trans / stmatrix) into y[t][l*128 + j]
+// So the inner permutation of Def. 3.1 is the choice of where a row goes, the outer one a plane transpose, and every
+// global access of the chain is a full 128-byte line.  The adjoints reverse the chain (dy transposed into
+// dw' (c = j, p = l), du'[k][t] = L_j^T dw'_j stored as du' (c = k, p = j), dx = du'_k^T R_k), and because the token
+// index is contiguous the same slabs are K-major operands of the token reductions dL_j = dw'_j u'_j^T and
+// dR_k = du'_k x_k, which ride along in the same kernels with their accumulators resident in TMEM for all tiles of a
+// block (one writer per block: deterministic sums).
 //
 // One kernel template serves all block products: persistent CTAs, the 32 KB weight block resident, token operands
 // through a TMA ring, tcgen05.mma 128 x 128 x 16 with two accumulator buffers in TMEM, epilogue through swizzled
@@ -46,12 +53,13 @@ constexpr int kHalfBytes = 16384;
 constexpr int kThreads = 6 * 32;             // warps 0-3 epilogue, 4 loader, 5 MMA
 constexpr int kStagingBytes = 2 * kHalfBytes;
 
-enum { kLdX = 0, kLdP = 1, kLdQ = 2 };       // token-major tensor; [tile][p][q][t] with p fixed; with q fixed
-enum { kStX = 0, kStQ = 1 };
+enum { kLdX = 0, kLdC = 1 };                 // token-major tensor (tiled TMA); consumer slab of an intermediate (linear)
+enum { kStX = 0, kStP = 1 };                 // token-major tensor; producer pieces of an intermediate
 
 struct ChainParams {
     unsigned *status;
     float *dW;                               // token-reduction output [block][128][128], added to
+    const char *t0_base, *t1_base;           // intermediates read as consumer slabs (kLdC)
     int ntiles;                              // 128-token tiles
     int nblk;                                // blocks (128)
 };
@@ -63,29 +71,29 @@ struct ChainBars {
     uint64_t wg_full, wg_empty;
 };
 
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *m, int c0, int c1, int c2, int c3, uint32_t bar)
+__device__ __forceinline__ void tma_store_5d(const CUtensorMap *m, uint32_t src, int c0, int c1, int c2, int c3, int c4)
 {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(dst),
-        "l"(m), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-        : "memory");
+    asm volatile("cp.async.bulk.tensor.5d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5, %6}], [%1];" ::"l"(m), "r"(src),
+                 "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+                 : "memory");
 }
-__device__ __forceinline__ void tma_store_4d(const CUtensorMap *m, uint32_t src, int c0, int c1, int c2, int c3)
+__device__ __forceinline__ void bulk_load_linear(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
 {
-    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(m), "r"(src),
-                 "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst), "l"(src),
+                 "r"(bytes), "r"(bar)
                  : "memory");
 }
 
-// Load one 128 x 128 operand (two 64-column boxes) of block `blk`, tile `tile`.
+// Load one 128 x 128 operand of block `blk`, tile `tile`: two 64-column boxes of a token-major tensor, or the
+// consumer slab [tile][blk] of an intermediate (already the swizzled image).
 template <int KIND>
-__device__ __forceinline__ void load_operand(uint32_t dst, const CUtensorMap *m, int blk, int tile, uint32_t bar)
+__device__ __forceinline__ void load_operand(uint32_t dst, const CUtensorMap *m, const char *base, int blk, int tile, uint32_t bar)
 {
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        if (KIND == kLdX) tma_load_2d(dst + h * kHalfBytes, m, blk * kB + h * 64, tile * 128, bar);
-        else if (KIND == kLdP) tma_load_4d(dst + h * kHalfBytes, m, h * 64, 0, blk, tile, bar);
-        else tma_load_4d(dst + h * kHalfBytes, m, h * 64, blk, 0, tile, bar);
+    if (KIND == kLdX) {
+        tma_load_2d(dst, m, blk * kB, tile * 128, bar);
+        tma_load_2d(dst + kHalfBytes, m, blk * kB + 64, tile * 128, bar);
+    } else {
+        bulk_load_linear(dst, base + ((size_t)tile * kB + blk) * kOpBytes, kOpBytes, bar);
     }
 }
 
@@ -182,8 +190,8 @@ chain_gemm_kernel(const __grid_constant__ CUtensorMap tm_t0, const __grid_consta
                 const uint32_t s = n % SLOTS;
                 if (!mbar_wait(empty0 + s * 8, ((n / SLOTS) & 1) ^ 1, p.status, dead, kErrSlotWait)) break;
                 mbar_expect_tx(full0 + s * 8, kSlotBytes);
-                load_operand<T0_LD>(ring0 + s * kSlotBytes, &tm_t0, blk, tile, full0 + s * 8);
-                if (WG) load_operand<T1_LD>(ring0 + s * kSlotBytes + kOpBytes, &tm_t1, blk, tile, full0 + s * 8);
+                load_operand<T0_LD>(ring0 + s * kSlotBytes, &tm_t0, p.t0_base, blk, tile, full0 + s * 8);
+                if (WG) load_operand<T1_LD>(ring0 + s * kSlotBytes + kOpBytes, &tm_t1, p.t1_base, blk, tile, full0 + s * 8);
             }
         }
     } else if (warp == 5) {
@@ -245,6 +253,7 @@ chain_gemm_kernel(const __grid_constant__ CUtensorMap tm_t0, const __grid_consta
         bool ok = true;
         for (long long i = i0; ok && i < i1; ++i, ++n) {
             const int blk = (int)(i / p.ntiles), tile = (int)(i % p.ntiles);
+            const int xorp = ST == kStP ? (blk & 7) : 0;
             if (MAIN) {
                 const uint32_t buf = n & 1;
                 if (!mbar_wait(accf0 + buf * 8, (n >> 1) & 1, p.status, dead, kErrMmaWait)) break;
@@ -272,14 +281,15 @@ chain_gemm_kernel(const __grid_constant__ CUtensorMap tm_t0, const __grid_consta
                         const uint32_t o1 = pack_bf16(__uint_as_float(w[2]), __uint_as_float(w[3]));
                         const uint32_t o2 = pack_bf16(__uint_as_float(w[4]), __uint_as_float(w[5]));
                         const uint32_t o3 = pack_bf16(__uint_as_float(w[6]), __uint_as_float(w[7]));
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((c ^ (row & 7)) << 4)),
+                        // producer pieces: the store un-swizzles by the row, the slab wants the chunks XORed with blk % 8
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((c ^ xorp ^ (row & 7)) << 4)),
                                      "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
                     }
                     fence_proxy_async_smem();
                     asm volatile("bar.sync 1, 128;" ::: "memory");
                     if (threadIdx.x == 0) {
                         if (ST == kStX) tma_store_2d(&tm_out, stg, blk * kB + h * 64, tile * 128);
-                        else tma_store_4d(&tm_out, stg, h * 64, blk, 0, tile);
+                        else tma_store_5d(&tm_out, stg, 0, blk, h, 0, tile);
                         tma_store_commit();
                     }
                 }
@@ -316,16 +326,18 @@ chain_gemm_kernel(const __grid_constant__ CUtensorMap tm_t0, const __grid_consta
 }
 
 // ---------------------------------------------------------------------------------------------------------
-// 128 x 128 plane transposes between a token-major tensor v[t][p*128 + c] and planes [tile][p][c][t]:
-// TO_PLANES = false: planes -> token-major (the outer P of step 3 of the forward pass), true: the reverse (first step
-// of the adjoint).  In and out are each two boxes of [128 rows][64 columns] with the 128-byte swizzle; four warps
-// move 8 x 8 tiles with ldmatrix.trans / stmatrix (conflict-free under the swizzle).
+// 128 x 128 plane transposes between a token-major tensor v[t][pl*128 + r] and an intermediate:
+// TO_PLANES = false: consumer slab pl (rows r, tokens along the row) -> token-major (the outer P of step 3 of the
+// forward pass); true: token-major -> producer pieces of plane pl (row r of the transposed tile goes to consumer r;
+// first step of the adjoint).  In and out are each two halves of [128 rows][64 columns] with the 128-byte swizzle;
+// four warps move 8 x 8 tiles with ldmatrix.trans / stmatrix (conflict-free under the swizzle).
 constexpr int kTrIn = 3, kTrOut = 2;
 constexpr int kTrThreads = 5 * 32;
 constexpr int kTrSmem = (kTrIn + kTrOut) * kOpBytes + 1024;
 
 struct TransposeParams {
     unsigned *status;
+    const char *in_base;                 // the intermediate (TO_PLANES = false)
     int ntiles, nplanes;                 // planes per tile (128)
     long long skip_item;                 // injected fault (tests only), else -1
 };
@@ -367,7 +379,7 @@ plane_transpose_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_c
                 if (!mbar_wait(smem_u32(&empty[s]), ((n / kTrIn) & 1) ^ 1, p.status, dead, kErrSlotWait)) break;
                 if (i == p.skip_item) continue;
                 mbar_expect_tx(smem_u32(&full[s]), kOpBytes);
-                load_operand<TO_PLANES ? kLdX : kLdP>(in0 + s * kOpBytes, &tm_in, pl, tile, smem_u32(&full[s]));
+                load_operand<TO_PLANES ? kLdX : kLdC>(in0 + s * kOpBytes, &tm_in, p.in_base, pl, tile, smem_u32(&full[s]));
                 last_fill[s] = (int)(n / kTrIn);
             }
             if (*dead) {
@@ -402,8 +414,9 @@ plane_transpose_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_c
                     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
                                  : "=r"(a), "=r"(b), "=r"(c), "=r"(d) : "r"(src) : "memory");
                     // destination tile of matrix mi: rows co*8..co*8+7 (source columns), column octet r0/8
-                    const int dr = co * 8 + ri, dco = r0 >> 3;
-                    const uint32_t dst = ob + (dco >> 3) * kHalfBytes + dr * 128 + (((dco & 7) ^ (dr & 7)) << 4);
+                    // producer pieces: the store un-swizzles by the row, the slab wants the chunks XORed with pl % 8
+                    const int dr = co * 8 + ri, dco = (r0 >> 3) ^ (TO_PLANES ? (pl & 7) : 0);
+                    const uint32_t dst = ob + (r0 >> 6) * kHalfBytes + dr * 128 + (((dco & 7) ^ (dr & 7)) << 4);
                     asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(a),
                                  "r"(b), "r"(c), "r"(d) : "memory");
                 }
@@ -415,7 +428,7 @@ plane_transpose_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_c
             if (threadIdx.x == 0) {
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    if (TO_PLANES) tma_store_4d(&tm_out, ob + h * kHalfBytes, h * 64, 0, pl, tile);
+                    if (TO_PLANES) tma_store_5d(&tm_out, ob + h * kHalfBytes, 0, pl, h, 0, tile);
                     else tma_store_2d(&tm_out, ob + h * kHalfBytes, pl * kB + h * 64, tile * 128);
                 }
                 tma_store_commit();
@@ -428,11 +441,11 @@ plane_transpose_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_c
 // ---------------------------------------------------------------------------------------------------------
 // The whole forward pass in one persistent launch: CTA b (one per SM, 128 of them) owns block b of every step and
 // walks the token tiles; at step s it runs
-//     A: D_b[j][t] = R_b x_b(tile s)            -> u'[tile s][j][b][t]                  (stage 1, rows to all j)
-//     B: D_b[l][t] = L_b u'_b(tile s - LAG)     -> w'[(tile s - LAG) % RING][l][b][t]   (stage 2)
-//     C: y[t][b*128 + j] = w'[tile s - 2 LAG][b][j][t]                                   (plane b transposed)
-// u' and w' are planes [tile][p][q][t] as in the three-launch chain (a producer writes 256-byte rows 32 KB apart, a
-// consumer reads one contiguous 32 KB plane by TMA).  An SM can push about 28.6 bytes per clock towards L2 whatever
+//     A: D_b[j][t] = R_b x_b(tile s)            -> pieces of u'[tile s] (row j to consumer j)      (stage 1)
+//     B: D_b[l][t] = L_b u'_b(tile s - LAG)     -> pieces of w'[(tile s - LAG) % RING]             (stage 2)
+//     C: y[t][b*128 + j] = slab b of w'[tile s - 2 LAG], transposed                                (outer P)
+// u' and w' have the layout of the three-launch chain (a producer writes 128-byte pieces 32 KB apart, a consumer
+// reads its 32 KB slab with one linear bulk copy).  An SM can push about 28.6 bytes per clock towards L2 whatever
 // the mechanism (load/store units or bulk copies; measured), i.e. the 96 KB a CTA writes per step cost 3.4 k
 // cycles: the stores, not the loads (70 B/clk) or the tensor pipe, bound this kernel.  Rows leave through the
 // load/store units from dedicated store warps (8 lanes per 128-byte piece); publishing a slab costs a memory fence
@@ -509,8 +522,7 @@ __device__ __forceinline__ bool wait_counter(unsigned *ctr, unsigned need, unsig
 
 __global__ void __launch_bounds__(kFusedThreads, 1)
 chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_R,
-                       const __grid_constant__ CUtensorMap tm_L, const __grid_constant__ CUtensorMap tm_u_ld,
-                       const __grid_constant__ CUtensorMap tm_w_ld, const FusedParams p)
+                       const __grid_constant__ CUtensorMap tm_L, const FusedParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) FusedBars bars;
@@ -540,7 +552,6 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
         fence_mbar_init();
         dead_s = 0;
         tma_prefetch_desc(&tm_x); tma_prefetch_desc(&tm_R); tma_prefetch_desc(&tm_L);
-        tma_prefetch_desc(&tm_u_ld); tma_prefetch_desc(&tm_w_ld);
     }
     if (warp == 0) {
         tmem_alloc(smem_u32(&tmem_base_s), 256);
@@ -575,14 +586,14 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
                     const uint32_t sl = g & 1;
                     { FT0(); if (!mbar_wait(empty0 + sl * 8, ((g >> 1) & 1) ^ 1, p.status, dead, kErrSlotWait)) break; FACC(wb); }
                     mbar_expect_tx(full0 + sl * 8, kOpBytes);
-                    load_operand<kLdP>(ring0 + sl * kOpBytes, &tm_u_ld, b, tb, full0 + sl * 8);
+                    load_operand<kLdC>(ring0 + sl * kOpBytes, nullptr, p.u, b, tb, full0 + sl * 8);
                     ++g;
                 }
                 if (s < nt) {
                     const uint32_t sl = g & 1;
                     { FT0(); if (!mbar_wait(empty0 + sl * 8, ((g >> 1) & 1) ^ 1, p.status, dead, kErrSlotWait)) break; FACC(wa); }
                     mbar_expect_tx(full0 + sl * 8, kOpBytes);
-                    load_operand<kLdX>(ring0 + sl * kOpBytes, &tm_x, b, s, full0 + sl * 8);
+                    load_operand<kLdX>(ring0 + sl * kOpBytes, &tm_x, nullptr, b, s, full0 + sl * 8);
                     ++g;
                 }
             }
@@ -683,8 +694,9 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
                 if (tile < 0 || tile >= nt) continue;
                 if ((int)(g % kStoreSets) != set) { ++g; continue; }
                 { FT0(); if (!mbar_wait(stf0 + (set * 2 + h) * 8, (g / kStoreSets) & 1, p.status, dead, kErrMmaWait)) { ok = false; break; } FACC(wf); }
+                // row r of D is the piece [tile][c = r][h][p = b] of the intermediate, chunks XORed with b % 8
                 char *dst = (kind == 0 ? p.u + (size_t)tile * (kB * kOpBytes) : p.w + (size_t)(tile % kFusedRing) * (kB * kOpBytes)) +
-                            b * 256 + h * 128 + (lane & 7) * 16;
+                            h * kHalfBytes + b * 128 + (((lane & 7) ^ (b & 7)) << 4);
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                     uint4 v[8];
@@ -722,7 +734,7 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
                 { FT0(); if (!wait_counter(p.cnt2 + tc, 2 * kB, kB, p.status, dead)) break; FACC(wc); }
                 { FT0(); if (!mbar_wait(tre, (c & 1) ^ 1, p.status, dead, kErrSlotWait)) break; FACC(we); }
                 mbar_expect_tx(trf, kOpBytes);
-                load_operand<kLdP>(trin, &tm_w_ld, b, tc % kFusedRing, trf);
+                load_operand<kLdC>(trin, nullptr, p.w, b, tc % kFusedRing, trf);
             }
             FOUT(10, wc); FOUT(11, we);
         }
@@ -785,273 +797,6 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
 }
 
 // ---------------------------------------------------------------------------------------------------------
-// The two block products of the backward pass and both token reductions in one persistent launch (the plane
-// transpose of dy runs before it as a launch of its own).  CTA b owns block b: at step s it runs
-//     E: D[k][t] = L_b^T dw'_b(tile s)         -> du'[tile s % RING][k][b][t]      dL_b += dw'_b u'_b^T   (over t)
-//     F: D[t][i] = du'_b(tile s - LAG)^T R_b   -> dx[t][b*128 + i]                dR_b += du'_b x_b      (over t)
-// with du' in an L2-resident ring, one counter per tile (bumped by the store warps of E, polled by the loader of
-// F), the two 128 x 128 fp32 sums resident in TMEM from the first tile to the last (one writer per block: the sums
-// are deterministic) and added to dL, dR at the end.  A ring slot holds the two operands of an item (64 KB).
-constexpr int kBwdSlotBytes = 2 * kOpBytes;
-constexpr int kBwdThreads = (6 + 2 * kStoreSets) * 32;      // warps 0-3 epilogue, 4 loader, 5 MMA, 6.. store warps
-constexpr int kBwdSmem = 2 * kOpBytes + 2 * kBwdSlotBytes + kStagingBytes + 1024;
-
-struct FusedBwdParams {
-    unsigned *status;
-    unsigned *cnt;                           // per tile: store warps (two per CTA) whose du' rows are in memory
-    char *du, *dx;                           // du' ring, output
-    float *dL, *dR;                          // added to
-    long long tokens;
-    int ntiles;
-};
-
-struct FusedBwdBars {
-    uint64_t w_full;
-    uint64_t full[2], empty[2];
-    uint64_t acc_full[2], acc_empty[2];
-    uint64_t st_full[2 * kStoreSets], st_free[2];
-    uint64_t wg_full;
-};
-
-__global__ void __launch_bounds__(kBwdThreads, 1)
-chain_fused_bwd_kernel(const __grid_constant__ CUtensorMap tm_dw, const __grid_constant__ CUtensorMap tm_u,
-                       const __grid_constant__ CUtensorMap tm_du, const __grid_constant__ CUtensorMap tm_x,
-                       const __grid_constant__ CUtensorMap tm_R, const __grid_constant__ CUtensorMap tm_L,
-                       const FusedBwdParams p)
-{
-    extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) FusedBwdBars bars;
-    __shared__ uint32_t tmem_base_s;
-    __shared__ int dead_s;
-
-    const uint32_t w0 = (smem_u32(smem_raw) + 1023u) & ~1023u;          // L_b, R_b
-    const uint32_t ring0 = w0 + 2 * kOpBytes;
-    const uint32_t staging0 = ring0 + 2 * kBwdSlotBytes;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int b = (int)blockIdx.x;
-    volatile int *dead = &dead_s;
-
-    if (threadIdx.x == 0) {
-        mbar_init(smem_u32(&bars.w_full), 1);
-        mbar_init(smem_u32(&bars.wg_full), 1);
-        for (int a = 0; a < 2; ++a) {
-            mbar_init(smem_u32(&bars.full[a]), 1);
-            mbar_init(smem_u32(&bars.empty[a]), 1);
-            mbar_init(smem_u32(&bars.acc_full[a]), 1);
-            mbar_init(smem_u32(&bars.acc_empty[a]), 4);
-            for (int k = 0; k < kStoreSets; ++k) mbar_init(smem_u32(&bars.st_full[k * 2 + a]), 4);
-            mbar_init(smem_u32(&bars.st_free[a]), 1);
-        }
-        fence_mbar_init();
-        dead_s = 0;
-        tma_prefetch_desc(&tm_dw); tma_prefetch_desc(&tm_u); tma_prefetch_desc(&tm_du); tma_prefetch_desc(&tm_x);
-        tma_prefetch_desc(&tm_R); tma_prefetch_desc(&tm_L);
-    }
-    if (warp == 0) {
-        tmem_alloc(smem_u32(&tmem_base_s), 512);
-        tmem_relinquish();
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = tmem_base_s;
-
-    const int nt = p.ntiles, nsteps = nt + kFusedLag;
-    const uint32_t full0 = smem_u32(bars.full), empty0 = smem_u32(bars.empty);
-    const uint32_t accf0 = smem_u32(bars.acc_full), acce0 = smem_u32(bars.acc_empty);
-    const uint32_t stf0 = smem_u32(bars.st_full), stfree0 = smem_u32(bars.st_free);
-    const uint32_t wgf = smem_u32(&bars.wg_full);
-
-    // item order within a step: F of the older tile first, then E
-    if (warp == 4) {
-        // ------------------------------------------------------------ loader
-        if (lane == 0) {
-            const uint32_t wbar = smem_u32(&bars.w_full);
-            mbar_expect_tx(wbar, 2 * kOpBytes);
-            tma_load_2d(w0, &tm_L, 0, b * kB, wbar);
-            tma_load_2d(w0 + kHalfBytes, &tm_L, 64, b * kB, wbar);
-            tma_load_2d(w0 + kOpBytes, &tm_R, 0, b * kB, wbar);
-            tma_load_2d(w0 + kOpBytes + kHalfBytes, &tm_R, 64, b * kB, wbar);
-            uint32_t g = 0;
-            for (int s = 0; s < nsteps; ++s) {
-                const int tf = s - kFusedLag;
-                if (tf >= 0) {
-                    if (!wait_counter(p.cnt + tf, 2 * kB, kB, p.status, dead)) break;
-                    const uint32_t sl = g & 1;
-                    if (!mbar_wait(empty0 + sl * 8, ((g >> 1) & 1) ^ 1, p.status, dead, kErrSlotWait)) break;
-                    mbar_expect_tx(full0 + sl * 8, kBwdSlotBytes);
-                    load_operand<kLdP>(ring0 + sl * kBwdSlotBytes, &tm_du, b, tf % kFusedRing, full0 + sl * 8);
-                    load_operand<kLdX>(ring0 + sl * kBwdSlotBytes + kOpBytes, &tm_x, b, tf, full0 + sl * 8);
-                    ++g;
-                }
-                if (s < nt) {
-                    const uint32_t sl = g & 1;
-                    if (!mbar_wait(empty0 + sl * 8, ((g >> 1) & 1) ^ 1, p.status, dead, kErrSlotWait)) break;
-                    mbar_expect_tx(full0 + sl * 8, kBwdSlotBytes);
-                    load_operand<kLdQ>(ring0 + sl * kBwdSlotBytes, &tm_dw, b, s, full0 + sl * 8);
-                    load_operand<kLdP>(ring0 + sl * kBwdSlotBytes + kOpBytes, &tm_u, b, s, full0 + sl * 8);
-                    ++g;
-                }
-            }
-        }
-    } else if (warp == 5) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0 && mbar_wait(smem_u32(&bars.w_full), 0, p.status, dead, kErrTmaWait)) {
-            constexpr uint32_t idesc_main = make_idesc_bf16(128, 128, 1, 1);
-            constexpr uint32_t idesc_dl = make_idesc_bf16(128, 128, 0, 0), idesc_dr = make_idesc_bf16(128, 128, 0, 1);
-            uint32_t g = 0;
-            bool ok = true, first_dl = true, first_dr = true;
-            for (int s = 0; ok && s < nsteps; ++s) {
-#pragma unroll
-                for (int ki = 0; ki < 2; ++ki) {
-                    const int kind = 1 - ki;                  // 1 = F, 0 = E
-                    const int tile = kind == 0 ? s : s - kFusedLag;
-                    if (tile < 0 || tile >= nt) continue;
-                    const uint32_t buf = g & 1;
-                    if (!mbar_wait(acce0 + buf * 8, ((g >> 1) & 1) ^ 1, p.status, dead, kErrTmemWait)) { ok = false; break; }
-                    if (!mbar_wait(full0 + buf * 8, (g >> 1) & 1, p.status, dead, kErrTmaWait)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t t0 = ring0 + buf * kBwdSlotBytes, t1 = t0 + kOpBytes, w = w0 + kind * kOpBytes;
-                    const uint32_t d = tmem_base + buf * 128;
-                    // E: A = L_b^T (weights, MN-major), B = dw' tile (MN-major); F: A = du' tile (MN-major), B = R_b (MN-major)
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        const uint64_t dwt = op_desc(w, true, ks), dt = op_desc(t0, true, ks);
-                        mma_f16_ss(d, kind == 0 ? dwt : dt, kind == 0 ? dt : dwt, idesc_main, ks != 0);
-                    }
-                    mma_commit(accf0 + buf * 8);
-                    // token reductions: rows of T0 as M, tokens as K
-                    const uint32_t dsum = tmem_base + 256 + kind * 128;
-                    bool &first = kind == 0 ? first_dl : first_dr;
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)
-                        mma_f16_ss(dsum, op_desc(t0, false, ks), op_desc(t1, kind == 1, ks), kind == 0 ? idesc_dl : idesc_dr,
-                                   !(first && ks == 0));
-                    first = false;
-                    mma_commit(empty0 + buf * 8);
-                    ++g;
-                }
-            }
-            if (ok) mma_commit(wgf);
-        }
-    } else if (warp < 4) {
-        // ------------------------------------------------------------ epilogue: TMEM -> bf16 -> staging halves
-        const int row = warp * 32 + lane;
-        const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
-        uint32_t g = 0;
-        bool ok = true;
-        for (int s = 0; ok && s < nsteps; ++s) {
-#pragma unroll 1
-            for (int ki = 0; ki < 2; ++ki) {
-                const int kind = 1 - ki;
-                const int tile = kind == 0 ? s : s - kFusedLag;
-                if (tile < 0 || tile >= nt) continue;
-                const uint32_t buf = g & 1;
-                if (!mbar_wait(accf0 + buf * 8, (g >> 1) & 1, p.status, dead, kErrMmaWait)) { ok = false; break; }
-                tc_fence_after();
-#pragma unroll 1
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t v[4][16];
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) tmem_ld16(lane_base + buf * 128 + h * 64 + q * 16, v[q]);
-                    tmem_ld_wait();
-                    if (h == 1) {
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(acce0 + buf * 8);
-                    }
-                    if (!mbar_wait(stfree0 + h * 8, (g & 1) ^ 1, p.status, dead, kErrSlotWait)) { ok = false; break; }
-                    const uint32_t dst = staging0 + h * kHalfBytes + row * 128;
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        const uint32_t *w = &v[c >> 1][(c & 1) * 8];
-                        const uint32_t o0 = pack_bf16(__uint_as_float(w[0]), __uint_as_float(w[1]));
-                        const uint32_t o1 = pack_bf16(__uint_as_float(w[2]), __uint_as_float(w[3]));
-                        const uint32_t o2 = pack_bf16(__uint_as_float(w[4]), __uint_as_float(w[5]));
-                        const uint32_t o3 = pack_bf16(__uint_as_float(w[6]), __uint_as_float(w[7]));
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((c ^ (row & 7)) << 4)),
-                                     "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(stf0 + ((g % kStoreSets) * 2 + h) * 8);
-                }
-                if (!ok) break;
-                ++g;
-            }
-        }
-        // the token sums of this block: dL_b (columns 256..383) and dR_b (384..511), one writer per element
-        if (ok && mbar_wait(wgf, 0, p.status, dead, kErrMmaWait)) {
-            tc_fence_after();
-#pragma unroll 1
-            for (int which = 0; which < 2; ++which) {
-                float *out = (which == 0 ? p.dL : p.dR) + ((size_t)b * kB + row) * kB;
-#pragma unroll 1
-                for (int c = 0; c < kB; c += 16) {
-                    uint32_t v[16];
-                    tmem_ld16(lane_base + 256 + which * 128 + c, v);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(out + c + e * 4),
-                                     "f"(__uint_as_float(v[e * 4])), "f"(__uint_as_float(v[e * 4 + 1])),
-                                     "f"(__uint_as_float(v[e * 4 + 2])), "f"(__uint_as_float(v[e * 4 + 3]))
-                                     : "memory");
-                }
-            }
-        }
-    } else if (warp >= 6 && warp < 6 + 2 * kStoreSets) {
-        // ------------------------------------------------------------ store warps: rows of D leave as 128-byte pieces
-        const int h = (warp - 6) & 1, set = (warp - 6) >> 1;
-        const uint32_t src = staging0 + h * kHalfBytes;
-        uint32_t g = 0;
-        bool ok = true;
-        for (int s = 0; ok && s < nsteps; ++s) {
-#pragma unroll 1
-            for (int ki = 0; ki < 2; ++ki) {
-                const int kind = 1 - ki;
-                const int tile = kind == 0 ? s : s - kFusedLag;
-                if (tile < 0 || tile >= nt) continue;
-                if ((int)(g % kStoreSets) != set) { ++g; continue; }
-                if (!mbar_wait(stf0 + (set * 2 + h) * 8, (g / kStoreSets) & 1, p.status, dead, kErrMmaWait)) { ok = false; break; }
-                // E: row k of du'[ring][k][b][t]; F: token row t of dx[t][b*128 ..] (rows past the last token stay put)
-                char *dst = (kind == 0 ? p.du + (size_t)(tile % kFusedRing) * (kB * kOpBytes) : p.dx + (size_t)tile * (kB * kOpBytes)) +
-                            b * 256 + h * 128 + (lane & 7) * 16;
-                const int rows_ok = kind == 0 ? 128 : (int)((p.tokens - (long long)tile * 128) < 128 ? (p.tokens - (long long)tile * 128) : 128);
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    uint4 v[8];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int r = (q * 8 + i) * 4 + (lane >> 3);
-                        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v[i].x), "=r"(v[i].y), "=r"(v[i].z), "=r"(v[i].w)
-                                     : "r"(src + r * 128 + (((lane & 7) ^ (r & 7)) << 4)) : "memory");
-                    }
-                    if (q == 3) {
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(stfree0 + h * 8);
-                    }
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int r = (q * 8 + i) * 4 + (lane >> 3);
-                        if (r < rows_ok) *reinterpret_cast<uint4 *>(dst + (size_t)r * kOpBytes) = v[i];
-                    }
-                }
-                if (kind == 0) {
-                    __threadfence();
-                    __syncwarp();
-                    if (lane == 0) atomicAdd(p.cnt + tile, 1u);
-                }
-                ++g;
-            }
-        }
-    }
-
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem_base, 512);
-}
-
-// ---------------------------------------------------------------------------------------------------------
 struct Maps {
     CUtensorMap x2d;       // token-major [tokens][n], box 128 rows x 64 columns
     CUtensorMap p4d;       // planes [tile][p][q][t], box = rows q of one p
@@ -1066,11 +811,12 @@ int map_weights(CUtensorMap *m, const void *W)
 {
     return encode_tmap_2d(m, W, (uint64_t)kB * kB, kB, kB * 2, 128, 64, 128);
 }
-int map_planes(CUtensorMap *m, const void *v, int ntiles, bool fixed_p)
+// producer pieces of an intermediate [tile][c][h][p][64 t]: box = the 128-byte pieces of one producer and half, all c
+int map_pieces(CUtensorMap *m, const void *v, int ntiles)
 {
-    const uint64_t dims[4] = {128, 128, 128, (uint64_t)ntiles}, strides[3] = {256, 32768, 4194304};
-    const uint32_t box_p[4] = {64, 128, 1, 1}, box_q[4] = {64, 1, 128, 1};
-    return encode_tmap_nd(m, v, 2, 4, dims, strides, fixed_p ? box_p : box_q, 128);
+    const uint64_t dims[5] = {64, 128, 2, 128, (uint64_t)ntiles}, strides[4] = {128, 16384, 32768, 4194304};
+    const uint32_t box[5] = {64, 1, 1, 128, 1};
+    return encode_tmap_nd(m, v, 2, 5, dims, strides, box, 128);
 }
 
 int device_sms(int *sms)
@@ -1081,9 +827,14 @@ int device_sms(int *sms)
     return MONARCH_OK;
 }
 
+// t0 / t1: a tensor map (token-major tensor) or the base pointer of an intermediate, whichever the load kind reads
+struct Src {
+    const CUtensorMap *map;
+    const char *base;
+};
+
 template <int T0_LD, bool W_IS_A, bool W_MN, bool T0_MN, int ST, bool WG, int T1_LD, bool T1_MN, bool MAIN>
-int launch_gemm(const CUtensorMap &t0, const CUtensorMap &t1, const CUtensorMap &w, const CUtensorMap &out, float *dW,
-                int ntiles, unsigned *status, cudaStream_t s)
+int launch_gemm(Src t0, Src t1, const CUtensorMap &w, const CUtensorMap &out, float *dW, int ntiles, unsigned *status, cudaStream_t s)
 {
     constexpr int SLOTS = WG ? 2 : 3;
     constexpr int smem = 2 * kOpBytes + SLOTS * (WG ? 2 : 1) * kOpBytes + kStagingBytes + 1024;
@@ -1094,30 +845,34 @@ int launch_gemm(const CUtensorMap &t0, const CUtensorMap &t1, const CUtensorMap 
     ChainParams p;
     p.status = status;
     p.dW = dW;
+    p.t0_base = t0.base;
+    p.t1_base = t1.base;
     p.ntiles = ntiles;
     p.nblk = kB;
     long long grid = WG ? kB : (long long)kB * ntiles;
     if (grid > sms) grid = sms;
-    kern<<<(unsigned)grid, kThreads, smem, s>>>(t0, t1, w, out, p);
+    // a load kind that reads a base pointer ignores its map: pass any valid one
+    kern<<<(unsigned)grid, kThreads, smem, s>>>(t0.map ? *t0.map : w, t1.map ? *t1.map : w, w, out, p);
     note_launch();
     MONARCH_CUDA_TRY(cudaGetLastError());
     return MONARCH_OK;
 }
 
 template <bool TO_PLANES>
-int launch_transpose(const CUtensorMap &in, const CUtensorMap &out, int ntiles, unsigned *status, cudaStream_t s)
+int launch_transpose(Src in, const CUtensorMap &out, int ntiles, unsigned *status, cudaStream_t s)
 {
     int sms = 0;
     MONARCH_TRY(device_sms(&sms));
     MONARCH_CUDA_TRY(cudaFuncSetAttribute(plane_transpose_kernel<TO_PLANES>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTrSmem));
     TransposeParams p;
     p.status = status;
+    p.in_base = in.base;
     p.ntiles = ntiles;
     p.nplanes = kB;
     p.skip_item = g_skip_load.exchange(-1);
     long long grid = (long long)ntiles * kB;
     if (grid > sms) grid = sms;
-    plane_transpose_kernel<TO_PLANES><<<(unsigned)grid, kTrThreads, kTrSmem, s>>>(in, out, p);
+    plane_transpose_kernel<TO_PLANES><<<(unsigned)grid, kTrThreads, kTrSmem, s>>>(in.map ? *in.map : out, out, p);
     note_launch();
     MONARCH_CUDA_TRY(cudaGetLastError());
     return MONARCH_OK;
@@ -1160,7 +915,7 @@ size_t chain_bwd_m128_workspace_bytes(int64_t tokens)
     return MONARCH_STATUS_BYTES + kChainCounterBytes + 3 * tc::planes_bytes(tokens);
 }
 
-// y = P L P^T R x (Def. 3.1; Section 3.3 steps 1-3) in three launches.
+// y = P L P^T R x (Def. 3.1; Section 3.3 steps 1-3): one persistent launch, or three launches.
 int chain_fwd_m128(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws, cudaStream_t s)
 {
     using namespace tc;
@@ -1169,15 +924,10 @@ int chain_fwd_m128(const void *x, const void *L, const void *R, void *y, int64_t
     const int ntiles = (int)((tokens + 127) / 128);
     unsigned *status = (unsigned *)ws;
     char *up = (char *)ws + MONARCH_STATUS_BYTES + kChainCounterBytes, *wp = up + planes_bytes(tokens);
-    CUtensorMap mx, my, mR, mL, mu_q, mu_p, mw_q, mw_p;
+    CUtensorMap mx, my, mR, mL, mu_st, mw_st;
     MONARCH_TRY(map_tokens(&mx, x, tokens));
-    MONARCH_TRY(map_tokens(&my, y, tokens));
     MONARCH_TRY(map_weights(&mR, R));
     MONARCH_TRY(map_weights(&mL, L));
-    MONARCH_TRY(map_planes(&mu_q, up, ntiles, false));
-    MONARCH_TRY(map_planes(&mu_p, up, ntiles, true));
-    MONARCH_TRY(map_planes(&mw_q, wp, ntiles, false));
-    MONARCH_TRY(map_planes(&mw_p, wp, ntiles, true));
     if (fwd_runs_fused(tokens) && g_skip_load.load(std::memory_order_relaxed) < 0) {
         // one persistent launch; every CTA must be resident at once (one per SM)
         MONARCH_CUDA_TRY(cudaFuncSetAttribute(chain_fused_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmem));
@@ -1194,20 +944,25 @@ int chain_fwd_m128(const void *x, const void *L, const void *R, void *y, int64_t
 #ifdef MONARCH_TRACE
         if (const char *e = getenv("MONARCH_TRACE_PTR")) fp.trace = (long long *)strtoull(e, nullptr, 0);
 #endif
-        chain_fused_fwd_kernel<<<kB, kFusedThreads, kFusedSmem, s>>>(mx, mR, mL, mu_p, mw_p, fp);
+        chain_fused_fwd_kernel<<<kB, kFusedThreads, kFusedSmem, s>>>(mx, mR, mL, fp);
         note_launch();
         MONARCH_CUDA_TRY(cudaGetLastError());
         return MONARCH_OK;
     }
-    // step 1 + inner permutation: D_k[j][t] = sum_i R[k][j][i] x[t][k*128+i]  ->  u'[tile][j][k][t]
-    MONARCH_TRY((launch_gemm<kLdX, true, false, false, kStQ, false, kLdX, false, true>(mx, mx, mR, mu_q, nullptr, ntiles, status, s)));
-    // step 2: D_j[l][t] = sum_k L[j][l][k] u'[tile][j][k][t]  ->  w'[tile][l][j][t]
-    MONARCH_TRY((launch_gemm<kLdP, true, false, true, kStQ, false, kLdX, false, true>(mu_p, mu_p, mL, mw_q, nullptr, ntiles, status, s)));
-    // step 3 (outer permutation): y[t][l*128+j] = w'[tile][l][j][t]
-    return launch_transpose<false>(mw_p, my, ntiles, status, s);
+    MONARCH_TRY(map_tokens(&my, y, tokens));
+    MONARCH_TRY(map_pieces(&mu_st, up, ntiles));
+    MONARCH_TRY(map_pieces(&mw_st, wp, ntiles));
+    // step 1 + inner permutation: D_k[j][t] = sum_i R[k][j][i] x[t][k*128+i]  ->  pieces of u' (row j to consumer j)
+    MONARCH_TRY((launch_gemm<kLdX, true, false, false, kStP, false, kLdX, false, true>({&mx, nullptr}, {nullptr, nullptr}, mR, mu_st, nullptr,
+                                                                                          ntiles, status, s)));
+    // step 2: D_j[l][t] = sum_k L[j][l][k] u'_j[k][t]  ->  pieces of w' (row l to consumer l)
+    MONARCH_TRY((launch_gemm<kLdC, true, false, true, kStP, false, kLdX, false, true>({nullptr, up}, {nullptr, nullptr}, mL, mw_st, nullptr,
+                                                                                         ntiles, status, s)));
+    // step 3 (outer permutation): y[t][l*128+j] = w'_l[j][t]
+    return launch_transpose<false>({nullptr, wp}, my, ntiles, status, s);
 }
 
-// dx = M^T dy, dL, dR (the adjoints of steps 1-3); saved_up = u' planes of the forward call or null (recomputed).
+// dx = M^T dy, dL, dR (the adjoints of steps 1-3); saved_up = u' of the forward call or null (recomputed).
 // dL and dR are added to: the caller zeroes them when they are not to accumulate.
 int chain_bwd_m128(const void *x, const void *dy, const void *L, const void *R, const void *saved_up, void *dx, float *dL,
                    float *dR, int want_dx, int want_dw, int64_t tokens, void *ws, cudaStream_t s)
@@ -1219,55 +974,39 @@ int chain_bwd_m128(const void *x, const void *dy, const void *L, const void *R, 
     unsigned *status = (unsigned *)ws;
     char *dwp = (char *)ws + MONARCH_STATUS_BYTES + kChainCounterBytes, *dup = dwp + planes_bytes(tokens),
          *up_own = dup + planes_bytes(tokens);
-    CUtensorMap mx, mdy, mdx, mR, mL, mdw_p, mdw_q, mdu_q, mdu_p, mu_q, mu_p;
+    CUtensorMap mx, mdy, mdx, mR, mL, mdw_st, mdu_st, mu_st;
     MONARCH_TRY(map_tokens(&mdy, dy, tokens));
     MONARCH_TRY(map_weights(&mR, R));
     MONARCH_TRY(map_weights(&mL, L));
-    MONARCH_TRY(map_planes(&mdw_p, dwp, ntiles, true));
-    MONARCH_TRY(map_planes(&mdw_q, dwp, ntiles, false));
-    MONARCH_TRY(map_planes(&mdu_q, dup, ntiles, false));
-    MONARCH_TRY(map_planes(&mdu_p, dup, ntiles, true));
+    MONARCH_TRY(map_pieces(&mdw_st, dwp, ntiles));
+    MONARCH_TRY(map_pieces(&mdu_st, dup, ntiles));
     if (want_dx) MONARCH_TRY(map_tokens(&mdx, dx, tokens));
     else mdx = mdy;
+    const char *up = (const char *)saved_up;
     if (want_dw) {
         MONARCH_TRY(map_tokens(&mx, x, tokens));
-        if (saved_up == nullptr) {
-            MONARCH_TRY(map_planes(&mu_q, up_own, ntiles, false));
-            MONARCH_TRY((launch_gemm<kLdX, true, false, false, kStQ, false, kLdX, false, true>(mx, mx, mR, mu_q, nullptr, ntiles, status, s)));
-            saved_up = up_own;
+        if (up == nullptr) {
+            MONARCH_TRY(map_pieces(&mu_st, up_own, ntiles));
+            MONARCH_TRY((launch_gemm<kLdX, true, false, false, kStP, false, kLdX, false, true>({&mx, nullptr}, {nullptr, nullptr}, mR, mu_st,
+                                                                                                  nullptr, ntiles, status, s)));
+            up = up_own;
         }
-        MONARCH_TRY(map_planes(&mu_p, saved_up, ntiles, true));
     }
-    // dw'[tile][l][j][t] = dy[t][l*128+j]
-    MONARCH_TRY(launch_transpose<true>(mdy, mdw_p, ntiles, status, s));
-    if (want_dw && want_dx && fwd_runs_fused(tokens)) {
-        // both block products and both token reductions in one persistent launch (every CTA resident)
-        MONARCH_CUDA_TRY(cudaFuncSetAttribute(chain_fused_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmem));
-        FusedBwdParams bp;
-        bp.status = status;
-        bp.cnt = (unsigned *)((char *)ws + MONARCH_STATUS_BYTES);
-        bp.du = dup;
-        bp.dx = (char *)dx;
-        bp.dL = dL;
-        bp.dR = dR;
-        bp.tokens = tokens;
-        bp.ntiles = ntiles;
-        chain_fused_bwd_kernel<<<kB, kBwdThreads, kBwdSmem, s>>>(mdw_q, mu_p, mdu_p, mx, mR, mL, bp);
-        note_launch();
-        MONARCH_CUDA_TRY(cudaGetLastError());
-        return MONARCH_OK;
-    }
-    // du'[tile][k][j][t] = sum_l L[j][l][k] dw'[tile][l][j][t]   (+ dL[j][l][k] += sum_t dw'[..][l][j][t] u'[..][j][k][t])
+    // dw' (consumer j, producer l): row j of the transposed tile dy[t][l*128 + j]
+    MONARCH_TRY(launch_transpose<true>({&mdy, nullptr}, mdw_st, ntiles, status, s));
+    // du'_k[j][t] = sum_l L[j][l][k] dw'_j[l][t] -> pieces of du' (row k to consumer k)   (+ dL[j][l][k] += sum_t dw'_j[l][t] u'_j[k][t])
     if (want_dw)
-        MONARCH_TRY((launch_gemm<kLdQ, true, true, true, kStQ, true, kLdP, false, true>(mdw_q, mu_p, mL, mdu_q, dL, ntiles, status, s)));
+        MONARCH_TRY((launch_gemm<kLdC, true, true, true, kStP, true, kLdC, false, true>({nullptr, dwp}, {nullptr, up}, mL, mdu_st, dL, ntiles,
+                                                                                          status, s)));
     else
-        MONARCH_TRY((launch_gemm<kLdQ, true, true, true, kStQ, false, kLdP, false, true>(mdw_q, mdw_q, mL, mdu_q, nullptr, ntiles, status, s)));
-    // dx[t][k*128+i] = sum_j du'[tile][k][j][t] R[k][j][i]        (+ dR[k][j][i] += sum_t du'[..][k][j][t] x[t][k*128+i])
+        MONARCH_TRY((launch_gemm<kLdC, true, true, true, kStP, false, kLdC, false, true>({nullptr, dwp}, {nullptr, nullptr}, mL, mdu_st, nullptr,
+                                                                                           ntiles, status, s)));
+    // dx[t][k*128+i] = sum_j du'_k[j][t] R[k][j][i]        (+ dR[k][j][i] += sum_t du'_k[j][t] x[t][k*128+i])
     if (want_dw && want_dx)
-        return launch_gemm<kLdP, false, true, true, kStX, true, kLdX, true, true>(mdu_p, mx, mR, mdx, dR, ntiles, status, s);
+        return launch_gemm<kLdC, false, true, true, kStX, true, kLdX, true, true>({nullptr, dup}, {&mx, nullptr}, mR, mdx, dR, ntiles, status, s);
     if (want_dw)
-        return launch_gemm<kLdP, false, true, true, kStX, true, kLdX, true, false>(mdu_p, mx, mR, mdx, dR, ntiles, status, s);
-    return launch_gemm<kLdP, false, true, true, kStX, false, kLdX, true, true>(mdu_p, mdu_p, mR, mdx, nullptr, ntiles, status, s);
+        return launch_gemm<kLdC, false, true, true, kStX, true, kLdX, true, false>({nullptr, dup}, {&mx, nullptr}, mR, mdx, dR, ntiles, status, s);
+    return launch_gemm<kLdC, false, true, true, kStX, false, kLdX, true, true>({nullptr, dup}, {nullptr, nullptr}, mR, mdx, nullptr, ntiles, status, s);
 }
 
 }  // namespace monarch
