@@ -122,6 +122,10 @@ int fused_fwd_m32(const void *x, const void *L, const void *R, void *y, int64_t 
 size_t fused_fwd_m64_workspace_bytes(int64_t tokens);
 int fused_fwd_m64(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws,
                   cudaStream_t s);
+// the same on clusters of four CTAs with the intermediate in distributed shared memory (fused_m64_cluster.cu);
+// MONARCH_ERR_UNSUPPORTED when the device cannot host such a cluster
+int fused_fwd_m64_cluster(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws, cudaStream_t s);
+bool fused_fwd_m64_on_clusters();
 // the same with every CTA doing both stages (fused_m64_team.cu); same workspace layout
 int fused_fwd_m64_team(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws,
                        cudaStream_t s);

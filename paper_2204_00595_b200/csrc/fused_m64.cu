@@ -454,7 +454,8 @@ constexpr size_t kFusedCounterBytes = 65536;
 
 size_t fused_fwd_m64_workspace_bytes(int64_t tokens)
 {
-    const size_t tiles = (size_t)((tokens + 63) / 64);
+    // at least two tiles: the forward on clusters keeps its 1 MB of weight images where the exchange buffer starts
+    const size_t tiles = tokens < 128 ? 2 : (size_t)((tokens + 63) / 64);
     return MONARCH_STATUS_BYTES + kFusedCounterBytes + tc::align256(tiles * 64 * (size_t)tc::kN * 2);
 }
 
@@ -551,11 +552,25 @@ int fused_fwd_m64(const void *x, const void *L, const void *R, void *y, int64_t 
         return launch_fwd_m64(x, L, R, y, (char *)ws + MONARCH_STATUS_BYTES + kFusedCounterBytes,
                               (unsigned *)((char *)ws + MONARCH_STATUS_BYTES), (unsigned *)ws, tokens, s);
 #endif
+    if (fused_fwd_m64_on_clusters()) {
+        const int st = fused_fwd_m64_cluster(x, L, R, y, tokens, ws, s);
+        if (st != MONARCH_ERR_UNSUPPORTED) return st;
+    }
     return fused_fwd_m64_team(x, L, R, y, tokens, ws, s);
+}
+
+// The forward pass on clusters of four CTAs (the intermediate stays in distributed shared memory; nothing is left in
+// the workspace for the backward call) when MONARCH_M64_CLUSTER is set.  Not the default: measured 80 us against
+// 59 us (8192 tokens) and 273 against 180 us (32768 tokens) for the team schedule with its exchange through L2.
+bool fused_fwd_m64_on_clusters()
+{
+    static const bool on = getenv("MONARCH_M64_CLUSTER") != nullptr;
+    return on;
 }
 
 const void *fused_fwd_m64_saved_u(const void *fwd_ws)
 {
+    if (fused_fwd_m64_on_clusters()) return nullptr;
     return (const char *)fwd_ws + MONARCH_STATUS_BYTES + kFusedCounterBytes;
 }
 

@@ -884,3 +884,38 @@ def test_bounded_wait_runs_out_and_the_workspace_recovers(P):
     torch.cuda.synchronize()
     assert P.monarch_last_device_status(ws) == 0
     assert_close(to_host64(y), O.fwd(d["x"], d["L"], d["R"]), dtype, "y after recovery")
+
+
+# ----------------------------------------------------------------- the m = 64 forward on clusters of four CTAs
+
+@pytest.mark.parametrize("T", [1, 63, 130, 257, 2500])
+def test_fwd_m64_on_clusters(T):
+    """The variant that keeps the permuted intermediate in distributed shared memory (selected by an environment
+    variable read once per process, hence the child process) against the oracle."""
+    import os
+    import subprocess
+    import sys
+    code = f"""
+import sys, numpy as np, torch
+sys.path.insert(0, {os.path.dirname(os.path.dirname(os.path.abspath(__file__)))!r})
+import paper_2204_00595_b200 as P
+from oracle import monarch_oracle as O
+from paper_2204_00595_b200.inputs import round_to_storage, to_device, to_host64
+from tests.helpers import assert_close
+m, n, T = 64, 4096, {T}
+rng = np.random.default_rng(6400 + T)
+draw = lambda shape, std: round_to_storage(rng.standard_normal(shape, dtype=np.float32) * np.float32(std), "bf16")
+hx, hL, hR = draw((T, n), 1.0), draw((m, m, m), 0.125), draw((m, m, m), 0.125)
+x, L, R = (to_device(a, "bf16") for a in (hx, hL, hR))
+y = torch.full_like(x, float("nan"))
+ws = P.Workspace(P.monarch_workspace_bytes(P.OP_FWD, T, n, m, P.BF16))
+for _ in range(2):
+    P.monarch_fwd(x, L, R, y, T, n, m, ws)
+torch.cuda.synchronize()
+assert P.monarch_last_device_status(ws) == 0
+assert_close(to_host64(y), O.fwd(hx, hL, hR), "bf16", "y on clusters")
+print("ok")
+"""
+    env = dict(os.environ, MONARCH_M64_CLUSTER="1")
+    out = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0 and "ok" in out.stdout, out.stderr[-2000:]
