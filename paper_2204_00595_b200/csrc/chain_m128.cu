@@ -30,6 +30,7 @@
 // staging tiles and TMA stores.
 #include <atomic>
 #include <cstdlib>
+#include <utility>
 
 #include "tc_common.cuh"
 
@@ -58,7 +59,8 @@ enum { kStX = 0, kStP = 1 };                 // token-major tensor; producer pie
 
 struct ChainParams {
     unsigned *status;
-    float *dW;                               // token-reduction output [block][128][128], added to
+    float *dW;                               // token-reduction output [block][128][128]
+    int overwrite;                           // 1: dW = sums, 0: dW += sums
     const char *t0_base, *t1_base;           // intermediates read as consumer slabs (kLdC)
     int ntiles;                              // 128-token tiles
     int nblk;                                // blocks (128)
@@ -70,6 +72,12 @@ struct ChainBars {
     uint64_t w_full[2], w_empty[2];
     uint64_t wg_full, wg_empty;
 };
+
+// Programmatic dependent launch: a kernel of the chain lets its successor start as SMs become free (barrier set-up, TMEM
+// allocation and the weight load overlap this kernel's tail); the successor waits here, once per thread, before it
+// touches anything the chain wrote.  Both are no-ops in a launch without the attribute.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 __device__ __forceinline__ void tma_store_5d(const CUtensorMap *m, uint32_t src, int c0, int c1, int c2, int c3, int c4)
 {
@@ -150,10 +158,12 @@ chain_gemm_kernel(const __grid_constant__ CUtensorMap tm_t0, const __grid_consta
         tmem_alloc(smem_u32(&tmem_base_s), 512);
         tmem_relinquish();
     }
+    pdl_launch_dependents();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
+    if (!(warp == 4 && lane == 0)) pdl_wait();          // the loader waits after it has asked for its first weight block
 
     // items = (block, tile), block-major.  With a token reduction a CTA owns whole blocks (its accumulator lives in
     // TMEM across the tiles of a block); otherwise the items are cut into equal contiguous runs.
@@ -184,6 +194,7 @@ chain_gemm_kernel(const __grid_constant__ CUtensorMap tm_t0, const __grid_consta
                     mbar_expect_tx(wf0 + wp * 8, kOpBytes);
                     tma_load_2d(w0 + wp * kOpBytes, &tm_w, 0, blk * kB, wf0 + wp * 8);
                     tma_load_2d(w0 + wp * kOpBytes + kHalfBytes, &tm_w, 64, blk * kB, wf0 + wp * 8);
+                    if (wcount == 0) pdl_wait();
                     ++wcount;
                     cur = blk;
                 }
@@ -295,7 +306,7 @@ chain_gemm_kernel(const __grid_constant__ CUtensorMap tm_t0, const __grid_consta
                 }
             }
             if (WG && (i + 1 == i1 || (int)((i + 1) / p.ntiles) != blk)) {
-                // the block's token sums are complete: add them to dW[blk] (one writer per element)
+                // the block's token sums are complete: store them to dW[blk] or add them to it (one writer per element)
                 if (!mbar_wait(wgf, nb & 1, p.status, dead, kErrMmaWait)) break;
                 tc_fence_after();
                 float *out = p.dW + ((size_t)blk * kB + row) * kB;
@@ -305,11 +316,17 @@ chain_gemm_kernel(const __grid_constant__ CUtensorMap tm_t0, const __grid_consta
                     tmem_ld16(lane_base + 256 + c, v);
                     tmem_ld_wait();
 #pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(out + c + e * 4),
-                                     "f"(__uint_as_float(v[e * 4])), "f"(__uint_as_float(v[e * 4 + 1])),
-                                     "f"(__uint_as_float(v[e * 4 + 2])), "f"(__uint_as_float(v[e * 4 + 3]))
-                                     : "memory");
+                    for (int e = 0; e < 4; ++e) {
+                        if (p.overwrite)
+                            *reinterpret_cast<float4 *>(out + c + e * 4) =
+                                make_float4(__uint_as_float(v[e * 4]), __uint_as_float(v[e * 4 + 1]), __uint_as_float(v[e * 4 + 2]),
+                                            __uint_as_float(v[e * 4 + 3]));
+                        else
+                            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(out + c + e * 4),
+                                         "f"(__uint_as_float(v[e * 4])), "f"(__uint_as_float(v[e * 4 + 1])),
+                                         "f"(__uint_as_float(v[e * 4 + 2])), "f"(__uint_as_float(v[e * 4 + 3]))
+                                         : "memory");
+                    }
                 }
                 tc_fence_before();
                 __syncwarp();
@@ -363,7 +380,9 @@ plane_transpose_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_c
         dead_s = 0;
         tma_prefetch_desc(&tm_in); tma_prefetch_desc(&tm_out);
     }
+    pdl_launch_dependents();
     __syncthreads();
+    pdl_wait();
     const long long total = (long long)p.ntiles * p.nplanes;
     const long long i0 = total * blockIdx.x / gridDim.x, i1 = total * (blockIdx.x + 1) / gridDim.x;
 
@@ -557,10 +576,12 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
         tmem_alloc(smem_u32(&tmem_base_s), 256);
         tmem_relinquish();
     }
+    pdl_launch_dependents();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
+    if (!(warp == 8 && lane == 0)) pdl_wait();          // the loader waits after it has asked for the weights
 
     const int nt = p.ntiles, nsteps = nt + 2 * kFusedLag;
     const uint32_t full0 = smem_u32(bars.full), empty0 = smem_u32(bars.empty);
@@ -577,6 +598,7 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
             tma_load_2d(w0 + kHalfBytes, &tm_R, 64, b * kB, wbar);
             tma_load_2d(w0 + kOpBytes, &tm_L, 0, b * kB, wbar);
             tma_load_2d(w0 + kOpBytes + kHalfBytes, &tm_L, 64, b * kB, wbar);
+            pdl_wait();
             uint32_t g = 0;                                // operand-ring items so far
             [[maybe_unused]] long long wa = 0, wc = 0, wb = 0;
             for (int s = 0; s < nsteps; ++s) {
@@ -827,6 +849,23 @@ int device_sms(int *sms)
     return MONARCH_OK;
 }
 
+// Launch with programmatic stream serialization: the kernel may start while its predecessor in the stream drains.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kern)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t s, Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(block, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+
 // t0 / t1: a tensor map (token-major tensor) or the base pointer of an intermediate, whichever the load kind reads
 struct Src {
     const CUtensorMap *map;
@@ -834,7 +873,8 @@ struct Src {
 };
 
 template <int T0_LD, bool W_IS_A, bool W_MN, bool T0_MN, int ST, bool WG, int T1_LD, bool T1_MN, bool MAIN>
-int launch_gemm(Src t0, Src t1, const CUtensorMap &w, const CUtensorMap &out, float *dW, int ntiles, unsigned *status, cudaStream_t s)
+int launch_gemm(Src t0, Src t1, const CUtensorMap &w, const CUtensorMap &out, float *dW, int ntiles, unsigned *status, cudaStream_t s,
+                int overwrite = 0)
 {
     constexpr int SLOTS = WG ? 2 : 3;
     constexpr int smem = 2 * kOpBytes + SLOTS * (WG ? 2 : 1) * kOpBytes + kStagingBytes + 1024;
@@ -845,6 +885,7 @@ int launch_gemm(Src t0, Src t1, const CUtensorMap &w, const CUtensorMap &out, fl
     ChainParams p;
     p.status = status;
     p.dW = dW;
+    p.overwrite = overwrite;
     p.t0_base = t0.base;
     p.t1_base = t1.base;
     p.ntiles = ntiles;
@@ -852,9 +893,8 @@ int launch_gemm(Src t0, Src t1, const CUtensorMap &w, const CUtensorMap &out, fl
     long long grid = WG ? kB : (long long)kB * ntiles;
     if (grid > sms) grid = sms;
     // a load kind that reads a base pointer ignores its map: pass any valid one
-    kern<<<(unsigned)grid, kThreads, smem, s>>>(t0.map ? *t0.map : w, t1.map ? *t1.map : w, w, out, p);
+    MONARCH_CUDA_TRY(launch_chained(kern, (unsigned)grid, kThreads, smem, s, t0.map ? *t0.map : w, t1.map ? *t1.map : w, w, out, p));
     note_launch();
-    MONARCH_CUDA_TRY(cudaGetLastError());
     return MONARCH_OK;
 }
 
@@ -872,9 +912,8 @@ int launch_transpose(Src in, const CUtensorMap &out, int ntiles, unsigned *statu
     p.skip_item = g_skip_load.exchange(-1);
     long long grid = (long long)ntiles * kB;
     if (grid > sms) grid = sms;
-    plane_transpose_kernel<TO_PLANES><<<(unsigned)grid, kTrThreads, kTrSmem, s>>>(in.map ? *in.map : out, out, p);
+    MONARCH_CUDA_TRY(launch_chained(plane_transpose_kernel<TO_PLANES>, (unsigned)grid, kTrThreads, kTrSmem, s, in.map ? *in.map : out, out, p));
     note_launch();
-    MONARCH_CUDA_TRY(cudaGetLastError());
     return MONARCH_OK;
 }
 
@@ -944,9 +983,8 @@ int chain_fwd_m128(const void *x, const void *L, const void *R, void *y, int64_t
 #ifdef MONARCH_TRACE
         if (const char *e = getenv("MONARCH_TRACE_PTR")) fp.trace = (long long *)strtoull(e, nullptr, 0);
 #endif
-        chain_fused_fwd_kernel<<<kB, kFusedThreads, kFusedSmem, s>>>(mx, mR, mL, fp);
+        MONARCH_CUDA_TRY(launch_chained(chain_fused_fwd_kernel, kB, kFusedThreads, kFusedSmem, s, mx, mR, mL, fp));
         note_launch();
-        MONARCH_CUDA_TRY(cudaGetLastError());
         return MONARCH_OK;
     }
     MONARCH_TRY(map_tokens(&my, y, tokens));
@@ -963,9 +1001,9 @@ int chain_fwd_m128(const void *x, const void *L, const void *R, void *y, int64_t
 }
 
 // dx = M^T dy, dL, dR (the adjoints of steps 1-3); saved_up = u' of the forward call or null (recomputed).
-// dL and dR are added to: the caller zeroes them when they are not to accumulate.
+// accumulate = 0: dL and dR are overwritten (every block of them has one writing CTA), 1: added to.
 int chain_bwd_m128(const void *x, const void *dy, const void *L, const void *R, const void *saved_up, void *dx, float *dL,
-                   float *dR, int want_dx, int want_dw, int64_t tokens, void *ws, cudaStream_t s)
+                   float *dR, int accumulate, int want_dx, int want_dw, int64_t tokens, void *ws, cudaStream_t s)
 {
     using namespace tc;
     if (tokens == 0) return MONARCH_OK;
@@ -997,15 +1035,17 @@ int chain_bwd_m128(const void *x, const void *dy, const void *L, const void *R, 
     // du'_k[j][t] = sum_l L[j][l][k] dw'_j[l][t] -> pieces of du' (row k to consumer k)   (+ dL[j][l][k] += sum_t dw'_j[l][t] u'_j[k][t])
     if (want_dw)
         MONARCH_TRY((launch_gemm<kLdC, true, true, true, kStP, true, kLdC, false, true>({nullptr, dwp}, {nullptr, up}, mL, mdu_st, dL, ntiles,
-                                                                                          status, s)));
+                                                                                          status, s, !accumulate)));
     else
         MONARCH_TRY((launch_gemm<kLdC, true, true, true, kStP, false, kLdC, false, true>({nullptr, dwp}, {nullptr, nullptr}, mL, mdu_st, nullptr,
                                                                                            ntiles, status, s)));
     // dx[t][k*128+i] = sum_j du'_k[j][t] R[k][j][i]        (+ dR[k][j][i] += sum_t du'_k[j][t] x[t][k*128+i])
     if (want_dw && want_dx)
-        return launch_gemm<kLdC, false, true, true, kStX, true, kLdX, true, true>({nullptr, dup}, {&mx, nullptr}, mR, mdx, dR, ntiles, status, s);
+        return launch_gemm<kLdC, false, true, true, kStX, true, kLdX, true, true>({nullptr, dup}, {&mx, nullptr}, mR, mdx, dR, ntiles, status, s,
+                                                                                  !accumulate);
     if (want_dw)
-        return launch_gemm<kLdC, false, true, true, kStX, true, kLdX, true, false>({nullptr, dup}, {&mx, nullptr}, mR, mdx, dR, ntiles, status, s);
+        return launch_gemm<kLdC, false, true, true, kStX, true, kLdX, true, false>({nullptr, dup}, {&mx, nullptr}, mR, mdx, dR, ntiles, status, s,
+                                                                                   !accumulate);
     return launch_gemm<kLdC, false, true, true, kStX, false, kLdX, true, true>({nullptr, dup}, {nullptr, nullptr}, mR, mdx, nullptr, ntiles, status, s);
 }
 

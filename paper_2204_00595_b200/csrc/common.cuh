@@ -98,9 +98,9 @@ int tc_staged_mlp_fwd(const void *x, const void *L1, const void *R1, const void 
 size_t chain_fwd_m128_workspace_bytes(int64_t tokens);
 size_t chain_bwd_m128_workspace_bytes(int64_t tokens);
 int chain_fwd_m128(const void *x, const void *L, const void *R, void *y, int64_t tokens, void *ws, cudaStream_t s);
-// saved_up: the u' planes the forward call left in its workspace (chain_fwd_m128_saved_u), or null; dL, dR are added to
+// saved_up: the u' the forward call left in its workspace (chain_fwd_m128_saved_u), or null
 int chain_bwd_m128(const void *x, const void *dy, const void *L, const void *R, const void *saved_up, void *dx, float *dL,
-                   float *dR, int want_dx, int want_dw, int64_t tokens, void *ws, cudaStream_t s);
+                   float *dR, int accumulate, int want_dx, int want_dw, int64_t tokens, void *ws, cudaStream_t s);
 const void *chain_fwd_m128_saved_u(const void *fwd_ws, int64_t tokens);
 // test aid: the next plane-transpose launch (last step of the m = 128 forward) leaves out the load of this item
 void debug_skip_next_plane_load(long long item);

@@ -302,13 +302,13 @@ int tc_staged_bwd(const void *x, const void *dy, const void *L, const void *R, v
     using namespace tc;
     if (want_dw && m != 128) return MONARCH_ERR_UNSUPPORTED;
     if (m == 128) {
-        // chain of block GEMMs on token-innermost planes (chain_m128.cu); dL, dR are added to
-        if (want_dw && !accumulate) {
+        // chain of block GEMMs on token-innermost intermediates (chain_m128.cu)
+        if (tokens == 0 && want_dw && !accumulate) {
             const size_t gb = (size_t)m * m * m * sizeof(float);
             MONARCH_CUDA_TRY(cudaMemsetAsync(dL, 0, gb, s));
             MONARCH_CUDA_TRY(cudaMemsetAsync(dR, 0, gb, s));
         }
-        return chain_bwd_m128(x, dy, L, R, saved_up, dx, dL, dR, want_dx, want_dw, tokens, ws, s);
+        return chain_bwd_m128(x, dy, L, R, saved_up, dx, dL, dR, accumulate, want_dx, want_dw, tokens, ws, s);
     }
     unsigned *status = (unsigned *)ws;
     const Layout l = carve(ws, tokens, m);
