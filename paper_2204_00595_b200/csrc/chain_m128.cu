@@ -64,6 +64,8 @@ struct ChainParams {
     const char *t0_base, *t1_base;           // intermediates read as consumer slabs (kLdC)
     int ntiles;                              // 128-token tiles
     int nblk;                                // blocks (128)
+    int reverse;                             // walk the tiles from the last to the first: what the previous launch of
+                                             // the chain wrote last is still in L2
 };
 
 struct ChainBars {
@@ -187,7 +189,7 @@ chain_gemm_kernel(const __grid_constant__ CUtensorMap tm_t0, const __grid_consta
             uint32_t n = 0, wcount = 0;
             int cur = -1;
             for (long long i = i0; i < i1; ++i, ++n) {
-                const int blk = (int)(i / p.ntiles), tile = (int)(i % p.ntiles);
+                const int blk = (int)(i / p.ntiles), tile = p.reverse ? p.ntiles - 1 - (int)(i % p.ntiles) : (int)(i % p.ntiles);
                 if (blk != cur) {
                     const uint32_t wp = wcount & 1;
                     if (!mbar_wait(we0 + wp * 8, ((wcount >> 1) & 1) ^ 1, p.status, dead, kErrSlotWait)) break;
@@ -263,7 +265,7 @@ chain_gemm_kernel(const __grid_constant__ CUtensorMap tm_t0, const __grid_consta
         uint32_t n = 0, nchunk = 0, nb = 0;
         bool ok = true;
         for (long long i = i0; ok && i < i1; ++i, ++n) {
-            const int blk = (int)(i / p.ntiles), tile = (int)(i % p.ntiles);
+            const int blk = (int)(i / p.ntiles), tile = p.reverse ? p.ntiles - 1 - (int)(i % p.ntiles) : (int)(i % p.ntiles);
             const int xorp = ST == kStP ? (blk & 7) : 0;
             if (MAIN) {
                 const uint32_t buf = n & 1;
@@ -383,8 +385,10 @@ plane_transpose_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_c
     pdl_launch_dependents();
     __syncthreads();
     pdl_wait();
+    // items (tile, plane), tile-major, dealt out round robin: the whole grid moves through the tiles together, so the
+    // next launch of the chain can start with the tiles written last (still in L2)
     const long long total = (long long)p.ntiles * p.nplanes;
-    const long long i0 = total * blockIdx.x / gridDim.x, i1 = total * (blockIdx.x + 1) / gridDim.x;
+    const long long i0 = blockIdx.x, istep = gridDim.x;
 
     if (warp == 4) {
         if (lane == 0) {
@@ -392,7 +396,7 @@ plane_transpose_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_c
             int last_fill[kTrIn];
 #pragma unroll
             for (int s = 0; s < kTrIn; ++s) last_fill[s] = -1;
-            for (long long i = i0; i < i1; ++i, ++n) {
+            for (long long i = i0; i < total; i += istep, ++n) {
                 const int tile = (int)(i / p.nplanes), pl = (int)(i % p.nplanes);
                 const uint32_t s = n % kTrIn;
                 if (!mbar_wait(smem_u32(&empty[s]), ((n / kTrIn) & 1) ^ 1, p.status, dead, kErrSlotWait)) break;
@@ -411,7 +415,7 @@ plane_transpose_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_c
         }
     } else {
         uint32_t n = 0;
-        for (long long i = i0; i < i1; ++i, ++n) {
+        for (long long i = i0; i < total; i += istep, ++n) {
             const int tile = (int)(i / p.nplanes), pl = (int)(i % p.nplanes);
             const uint32_t s = n % kTrIn, ob = out0 + (n & 1) * kOpBytes, ib = in0 + s * kOpBytes;
             // the output buffer used two items ago has been read by its stores
@@ -841,13 +845,7 @@ int map_pieces(CUtensorMap *m, const void *v, int ntiles)
     return encode_tmap_nd(m, v, 2, 5, dims, strides, box, 128);
 }
 
-int device_sms(int *sms)
-{
-    int dev = 0;
-    MONARCH_CUDA_TRY(cudaGetDevice(&dev));
-    MONARCH_CUDA_TRY(cudaDeviceGetAttribute(sms, cudaDevAttrMultiProcessorCount, dev));
-    return MONARCH_OK;
-}
+int device_sms(int *sms) { return current_device_sms(sms); }
 
 // Launch with programmatic stream serialization: the kernel may start while its predecessor in the stream drains.
 template <typename... KArgs, typename... Args>
@@ -874,7 +872,7 @@ struct Src {
 
 template <int T0_LD, bool W_IS_A, bool W_MN, bool T0_MN, int ST, bool WG, int T1_LD, bool T1_MN, bool MAIN>
 int launch_gemm(Src t0, Src t1, const CUtensorMap &w, const CUtensorMap &out, float *dW, int ntiles, unsigned *status, cudaStream_t s,
-                int overwrite = 0)
+                int overwrite = 0, int reverse = 0)
 {
     constexpr int SLOTS = WG ? 2 : 3;
     constexpr int smem = 2 * kOpBytes + SLOTS * (WG ? 2 : 1) * kOpBytes + kStagingBytes + 1024;
@@ -886,6 +884,7 @@ int launch_gemm(Src t0, Src t1, const CUtensorMap &w, const CUtensorMap &out, fl
     p.status = status;
     p.dW = dW;
     p.overwrite = overwrite;
+    p.reverse = reverse;
     p.t0_base = t0.base;
     p.t1_base = t1.base;
     p.ntiles = ntiles;
@@ -995,7 +994,7 @@ int chain_fwd_m128(const void *x, const void *L, const void *R, void *y, int64_t
                                                                                           ntiles, status, s)));
     // step 2: D_j[l][t] = sum_k L[j][l][k] u'_j[k][t]  ->  pieces of w' (row l to consumer l)
     MONARCH_TRY((launch_gemm<kLdC, true, false, true, kStP, false, kLdX, false, true>({nullptr, up}, {nullptr, nullptr}, mL, mw_st, nullptr,
-                                                                                         ntiles, status, s)));
+                                                                                         ntiles, status, s, 0, 1)));
     // step 3 (outer permutation): y[t][l*128+j] = w'_l[j][t]
     return launch_transpose<false>({nullptr, wp}, my, ntiles, status, s);
 }
@@ -1030,15 +1029,17 @@ int chain_bwd_m128(const void *x, const void *dy, const void *L, const void *R, 
             up = up_own;
         }
     }
+    // Tile order: a launch walks the tiles in the opposite direction of the one before it, so that it starts with what
+    // is still in L2 (an intermediate is 134 MB at 4096 tokens, L2 holds 126).
     // dw' (consumer j, producer l): row j of the transposed tile dy[t][l*128 + j]
     MONARCH_TRY(launch_transpose<true>({&mdy, nullptr}, mdw_st, ntiles, status, s));
     // du'_k[j][t] = sum_l L[j][l][k] dw'_j[l][t] -> pieces of du' (row k to consumer k)   (+ dL[j][l][k] += sum_t dw'_j[l][t] u'_j[k][t])
     if (want_dw)
         MONARCH_TRY((launch_gemm<kLdC, true, true, true, kStP, true, kLdC, false, true>({nullptr, dwp}, {nullptr, up}, mL, mdu_st, dL, ntiles,
-                                                                                          status, s, !accumulate)));
+                                                                                          status, s, !accumulate, 1)));
     else
         MONARCH_TRY((launch_gemm<kLdC, true, true, true, kStP, false, kLdC, false, true>({nullptr, dwp}, {nullptr, nullptr}, mL, mdu_st, nullptr,
-                                                                                           ntiles, status, s)));
+                                                                                           ntiles, status, s, 0, 1)));
     // dx[t][k*128+i] = sum_j du'_k[j][t] R[k][j][i]        (+ dR[k][j][i] += sum_t du'_k[j][t] x[t][k*128+i])
     if (want_dw && want_dx)
         return launch_gemm<kLdC, false, true, true, kStX, true, kLdX, true, true>({nullptr, dup}, {&mx, nullptr}, mR, mdx, dR, ntiles, status, s,

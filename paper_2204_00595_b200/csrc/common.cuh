@@ -5,12 +5,34 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "monarch.h"
 
 namespace monarch {
 
 // Launch counter behind monarch_launch_count().
 void note_launch(int n = 1);
+
+// SM count of the current device (cached per device ordinal, safe against concurrent first calls).
+int current_device_sms(int *sms);
+
+// A value cached per device ordinal (an occupancy figure): get() returns -1 until set() has stored one for the current
+// device.  Two threads racing on a first call both compute and store the same value.
+struct PerDeviceCache {
+    std::atomic<int> v[64];                  // value + 1; zero-initialised as a static
+    int get() const
+    {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
+        return v[dev].load(std::memory_order_relaxed) - 1;
+    }
+    void set(int value)
+    {
+        int dev = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64) v[dev].store(value + 1, std::memory_order_relaxed);
+    }
+};
 
 #define MONARCH_CUDA_TRY(expr)                                   \
     do {                                                         \

@@ -385,14 +385,12 @@ int fused_fwd_m32(const void *x, const void *L, const void *R, void *y, int64_t 
         const uint32_t ybox[3] = {16, 64, 4};
         MONARCH_TRY(encode_tmap_nd(&tm_y, y, 2, 3, ydims, ystrides, ybox));
     }
-    static int sms = 0;
-    if (!sms) {
-        int dev = 0;
-        MONARCH_CUDA_TRY(cudaGetDevice(&dev));
-        MONARCH_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        MONARCH_CUDA_TRY(cudaFuncSetAttribute(fused_fwd_m32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              kSmemBytes));
-    }
+    // per call: the SM count and the shared-memory attribute belong to the current device, and a first-call
+    // cache would not be safe against two host threads
+    int sms = 0;
+    MONARCH_TRY(current_device_sms(&sms));
+    MONARCH_CUDA_TRY(cudaFuncSetAttribute(fused_fwd_m32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          kSmemBytes));
     P32 p;
     p.status = (unsigned *)ws;
     p.tiles = (int)tiles;

@@ -490,14 +490,12 @@ int launch_fwd_m64(const void *x, const void *L, const void *R, void *y, void *u
         tm_L = tm_R;
         tm_y = tm_u;
     }
-    static int sms = 0;
-    if (!sms) {
-        int dev = 0;
-        MONARCH_CUDA_TRY(cudaGetDevice(&dev));
-        MONARCH_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        MONARCH_CUDA_TRY(cudaFuncSetAttribute(fused_fwd_m64_kernel,
-                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-    }
+    // per call: the SM count and the shared-memory attribute belong to the current device, and a first-call
+    // cache would not be safe against two host threads
+    int sms = 0;
+    MONARCH_TRY(current_device_sms(&sms));
+    MONARCH_CUDA_TRY(cudaFuncSetAttribute(fused_fwd_m64_kernel,
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
     FwdParams p;
     p.status = status;
     p.counters = counters;

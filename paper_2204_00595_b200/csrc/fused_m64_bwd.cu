@@ -1035,14 +1035,12 @@ int launch_bwd_m64(const void *dy, const void *L, const void *R, void *dx, void 
         tm_R = tm_Lt;
         tm_dx = tm_du;
     }
-    static int sms = 0;
-    if (!sms) {
-        int dev = 0;
-        MONARCH_CUDA_TRY(cudaGetDevice(&dev));
-        MONARCH_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        MONARCH_CUDA_TRY(cudaFuncSetAttribute(fused_bwd_dx_m64_kernel,
-                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-    }
+    // per call: the SM count and the shared-memory attribute belong to the current device, and a first-call
+    // cache would not be safe against two host threads
+    int sms = 0;
+    MONARCH_TRY(current_device_sms(&sms));
+    MONARCH_CUDA_TRY(cudaFuncSetAttribute(fused_bwd_dx_m64_kernel,
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
     BwdParams p;
     p.status = status;
     p.counters = counters;
@@ -1104,14 +1102,12 @@ int fused_bwd_all_m64(const void *x, const void *dy, const void *L, const void *
     // dx == null: weight gradients only (the map is never used; it only has to be a valid one)
     MONARCH_TRY(encode_tmap_2d(&tm_dx, dx ? dx : x, (uint64_t)tokens, kN, kN * 2, 64, 64, 128));
     MONARCH_TRY(encode_tmap_2d(&tm_x, x, (uint64_t)tokens, kN, kN * 2, 64, 64, 128));
-    static int sms = 0;
-    if (!sms) {
-        int dev = 0;
-        MONARCH_CUDA_TRY(cudaGetDevice(&dev));
-        MONARCH_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        MONARCH_CUDA_TRY(cudaFuncSetAttribute(fused_bwd_all_m64_kernel,
-                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-    }
+    // per call: the SM count and the shared-memory attribute belong to the current device, and a first-call
+    // cache would not be safe against two host threads
+    int sms = 0;
+    MONARCH_TRY(current_device_sms(&sms));
+    MONARCH_CUDA_TRY(cudaFuncSetAttribute(fused_bwd_all_m64_kernel,
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
     BwdParams p;
     p.status = status;
     p.counters = counters;

@@ -208,14 +208,12 @@ int launch_dw(const void *x, const void *u, const void *du, const void *dyp, flo
     const long long tiles = (tokens + 63) / 64;
     CUtensorMap tm_x;
     MONARCH_TRY(encode_tmap_2d(&tm_x, x, (uint64_t)tokens, kN, kN * 2, 64, 64, 128));
-    static int sms = 0;
-    if (!sms) {
-        int dev = 0;
-        MONARCH_CUDA_TRY(cudaGetDevice(&dev));
-        MONARCH_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        MONARCH_CUDA_TRY(cudaFuncSetAttribute(fused_bwd_dw_m64_kernel,
-                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-    }
+    // per call: the SM count and the shared-memory attribute belong to the current device, and a first-call
+    // cache would not be safe against two host threads
+    int sms = 0;
+    MONARCH_TRY(current_device_sms(&sms));
+    MONARCH_CUDA_TRY(cudaFuncSetAttribute(fused_bwd_dw_m64_kernel,
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
     DwParams p;
     p.u = (const __nv_bfloat16 *)u;
     p.du = (const __nv_bfloat16 *)du;
@@ -299,7 +297,12 @@ int fused_bwd_m64(const void *x, const void *dy, const void *L, const void *R, c
         return launch_dw(x, u, du, dyp, dL, dR, status, tokens, s);
     }
 #endif
-    return fused_bwd_all_m64(x, dy, L, R, u, dx, du, dyp, dL, dR, counters, status, tokens, s);
+    // the one-launch form declines, before launching anything, on a GPU too small to hold all of its CTAs at once
+    // (or for more tiles than it has counters): then the backward kernel and the token reduction run as two launches
+    const int rc = fused_bwd_all_m64(x, dy, L, R, u, dx, du, dyp, dL, dR, counters, status, tokens, s);
+    if (rc != MONARCH_ERR_UNSUPPORTED) return rc;
+    MONARCH_TRY(fused_bwd_dx_m64_keep(dy, L, R, dx, du, dyp, counters, status, tokens, s));
+    return launch_dw(x, u, du, dyp, dL, dR, status, tokens, s);
 }
 
 }  // namespace monarch

@@ -374,7 +374,8 @@ int fused_fwd_m64_cluster(const void *x, const void *L, const void *R, void *y, 
     if (tokens == 0) return MONARCH_OK;
     const long long tiles = (tokens + kTile - 1) / kTile;
     if (tiles > (1 << 24)) return MONARCH_ERR_UNSUPPORTED;
-    static int max_clusters = -1;
+    static PerDeviceCache max_clusters_cache;
+    int max_clusters = max_clusters_cache.get();
     if (max_clusters < 0) {
         MONARCH_CUDA_TRY(cudaFuncSetAttribute(fused_fwd_m64_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem));
         cudaLaunchConfig_t cfg = {};
@@ -392,6 +393,7 @@ int fused_fwd_m64_cluster(const void *x, const void *L, const void *R, void *y, 
             n = 0;
         }
         max_clusters = n;
+        max_clusters_cache.set(n);
     }
     if (max_clusters < 1) return MONARCH_ERR_UNSUPPORTED;
     char *Rimg = (char *)ws + MONARCH_STATUS_BYTES + 65536, *Limg = Rimg + (size_t)kN * kM * 2;

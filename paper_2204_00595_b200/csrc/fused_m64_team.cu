@@ -505,14 +505,12 @@ int launch_team(const void *x, const void *L, const void *R, const void *bias, i
         const uint32_t ybox[3] = {16, 64, 4};
         MONARCH_TRY(encode_tmap_nd(&tm_y, y, 2, 3, ydims, ystrides, ybox));
     }
-    static int sms = 0;
-    if (!sms) {
-        int dev = 0;
-        MONARCH_CUDA_TRY(cudaGetDevice(&dev));
-        MONARCH_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        MONARCH_CUDA_TRY(cudaFuncSetAttribute(fused_fwd_m64_team_kernel,
-                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-    }
+    // per call: the SM count and the shared-memory attribute belong to the current device, and a first-call
+    // cache would not be safe against two host threads
+    int sms = 0;
+    MONARCH_TRY(current_device_sms(&sms));
+    MONARCH_CUDA_TRY(cudaFuncSetAttribute(fused_fwd_m64_team_kernel,
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
     TeamParams p;
     p.status = status;
     p.counters = counters;

@@ -11,6 +11,21 @@ static std::atomic<int> g_impl{MONARCH_IMPL_AUTO};
 
 void note_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
+int current_device_sms(int *sms)
+{
+    constexpr int kMaxDevices = 64;
+    static std::atomic<int> cache[kMaxDevices];          // zero-initialised: 0 = not yet queried
+    int dev = 0;
+    MONARCH_CUDA_TRY(cudaGetDevice(&dev));
+    int v = dev < kMaxDevices ? cache[dev].load(std::memory_order_relaxed) : 0;
+    if (v == 0) {
+        MONARCH_CUDA_TRY(cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev));
+        if (dev < kMaxDevices) cache[dev].store(v, std::memory_order_relaxed);
+    }
+    *sms = v;
+    return MONARCH_OK;
+}
+
 namespace {
 
 bool aligned(const void *p, size_t a) { return ((uintptr_t)p & (a - 1)) == 0; }
@@ -33,6 +48,7 @@ bool overlap(const Range &a, const Range &b)
 int check_shape(int64_t tokens, int32_t n, int32_t m, int dtype)
 {
     if (tokens < 0 || n <= 0 || m <= 0) return MONARCH_ERR_INVALID_ARG;
+    if (tokens > ((int64_t)1 << 40)) return MONARCH_ERR_INVALID_ARG;        // keeps tokens * n * 4 inside 64 bits
     if ((int64_t)m * m != (int64_t)n) return MONARCH_ERR_INVALID_ARG;
     if (dtype != MONARCH_F32 && dtype != MONARCH_BF16) return MONARCH_ERR_INVALID_ARG;
     if (m != 16 && m != 32 && m != 64 && m != 128) return MONARCH_ERR_UNSUPPORTED;
@@ -151,6 +167,9 @@ size_t monarch_workspace_bytes(int op, int64_t tokens, int32_t n, int32_t m, int
     }
     const int which = pick(op, m, dtype);
     if (which < 0) return 0;
+    // the fused m = 64 kernels keep one dependency counter per 64-token tile in 64 KB: beyond 2^20 tokens the calls
+    // refuse, and so does this query (shard the tokens)
+    if (which == kFused && m == 64 && tokens > ((int64_t)1 << 20)) return 0;
     if (which == kTcStaged && op != MONARCH_OP_FWD && op != MONARCH_OP_MLP_FWD)
         return tc_staged_bwd_workspace_bytes(tokens, m);
     if (which == kTcStaged && op == MONARCH_OP_FWD && m == 128) return chain_fwd_m128_workspace_bytes(tokens);

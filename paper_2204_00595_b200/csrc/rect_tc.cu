@@ -387,7 +387,8 @@ int launch_pair(const void *in, const void *W, void *out, int64_t tokens, int q,
     else
         MONARCH_TRY(encode_tmap_2d(&tm_R, W, (uint64_t)q * ndim, (uint64_t)kdim, (uint64_t)kdim * 2, 128, kKChunk, 128));
     MONARCH_TRY(encode_tmap_2d(&tm_u, out, (uint64_t)tokens, (uint64_t)q * ndim, (uint64_t)q * ndim * 2, kTokTile, 64, 128));
-    static int max_pairs = -1;
+    static PerDeviceCache max_pairs_cache;
+    int max_pairs = max_pairs_cache.get();
     if (max_pairs < 0) {
         MONARCH_CUDA_TRY(cudaFuncSetAttribute(rect_stage1_pair_kernel<BT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmem));
         cudaLaunchConfig_t cfg = {};
@@ -405,6 +406,7 @@ int launch_pair(const void *in, const void *W, void *out, int64_t tokens, int q,
             n = 0;
         }
         max_pairs = n;
+        max_pairs_cache.set(n);
     }
     if (max_pairs < 1) return MONARCH_OK;                                 // the caller falls back to single CTAs
     RectParams p;
@@ -434,12 +436,10 @@ int launch(const void *in, const void *W, void *out, int64_t tokens, int q, int 
     else
         MONARCH_TRY(encode_tmap_2d(&tm_R, W, (uint64_t)q * ndim, (uint64_t)kdim, (uint64_t)kdim * 2, NT, kKChunk, 128));
     MONARCH_TRY(encode_tmap_2d(&tm_u, out, (uint64_t)tokens, (uint64_t)q * ndim, (uint64_t)q * ndim * 2, kTokTile, 64, 128));
-    static int sms = 0;
-    if (!sms) {
-        int dev = 0;
-        MONARCH_CUDA_TRY(cudaGetDevice(&dev));
-        MONARCH_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    }
+    // per call: the SM count and the shared-memory attribute belong to the current device, and a first-call
+    // cache would not be safe against two host threads
+    int sms = 0;
+    MONARCH_TRY(current_device_sms(&sms));
     static bool attr = false;
     if (!attr) {
         MONARCH_CUDA_TRY(cudaFuncSetAttribute(rect_stage1_kernel<NT, BT>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kBytes));
@@ -806,13 +806,11 @@ int launch_wgrad(const void *du, const void *x, float *dR, int64_t tokens, int q
     CUtensorMap tm_du, tm_x;
     MONARCH_TRY(encode_tmap_2d(&tm_du, du, (uint64_t)tokens, (uint64_t)q * b, (uint64_t)q * b * 2, 64, 64, 128));
     MONARCH_TRY(encode_tmap_2d(&tm_x, x, (uint64_t)tokens, (uint64_t)q * b1, (uint64_t)q * b1 * 2, 64, 64, 128));
-    static int sms = 0;
-    if (!sms) {
-        int dev = 0;
-        MONARCH_CUDA_TRY(cudaGetDevice(&dev));
-        MONARCH_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        MONARCH_CUDA_TRY(cudaFuncSetAttribute(rect_wgrad_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    }
+    // per call: the SM count and the shared-memory attribute belong to the current device, and a first-call
+    // cache would not be safe against two host threads
+    int sms = 0;
+    MONARCH_TRY(current_device_sms(&sms));
+    MONARCH_CUDA_TRY(cudaFuncSetAttribute(rect_wgrad_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     WgParams p;
     p.out = dR;
     p.status = status;
@@ -853,14 +851,12 @@ int rect_stage2_stream(const void *u, const void *Lp, void *y, int64_t tokens, i
     if (tokens == 0) return MONARCH_OK;
     CUtensorMap tm_u;
     MONARCH_TRY(encode_tmap_2d(&tm_u, u, (uint64_t)tokens, (uint64_t)q * b, (uint64_t)q * b * 2, kS2Tok, kS2Cols, 0));
-    static int sms = 0;
-    if (!sms) {
-        int dev = 0;
-        MONARCH_CUDA_TRY(cudaGetDevice(&dev));
-        MONARCH_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        MONARCH_CUDA_TRY(cudaFuncSetAttribute(rect_stage2_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              kS2SmemBytes));
-    }
+    // per call: the SM count and the shared-memory attribute belong to the current device, and a first-call
+    // cache would not be safe against two host threads
+    int sms = 0;
+    MONARCH_TRY(current_device_sms(&sms));
+    MONARCH_CUDA_TRY(cudaFuncSetAttribute(rect_stage2_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          kS2SmemBytes));
     const int cx = (b + kS2Cols - 1) / kS2Cols;
     long long slabs = (2LL * sms + cx - 1) / cx;                     // two CTAs per SM, one wave
     if (slabs > (tokens + kS2Tok - 1) / kS2Tok) slabs = (tokens + kS2Tok - 1) / kS2Tok;
@@ -900,13 +896,11 @@ int rect_dl_stream(const void *dy, const void *u, float *dL, int64_t tokens, int
     MONARCH_TRY(encode_tmap_2d(&tm_dy, dy, (uint64_t)tokens, (uint64_t)r * b, (uint64_t)r * b * 2, kS2Tok, kS2Cols, 0));
     MONARCH_TRY(encode_tmap_2d(&tm_u, u, (uint64_t)tokens, (uint64_t)q * b, (uint64_t)q * b * 2, kS2Tok, kS2Cols, 0));
     constexpr int smem = kS2Stages * 8 * kS2SliceBytes + 128;
-    static int sms = 0;
-    if (!sms) {
-        int dev = 0;
-        MONARCH_CUDA_TRY(cudaGetDevice(&dev));
-        MONARCH_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        MONARCH_CUDA_TRY(cudaFuncSetAttribute(rect_dl_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    }
+    // per call: the SM count and the shared-memory attribute belong to the current device, and a first-call
+    // cache would not be safe against two host threads
+    int sms = 0;
+    MONARCH_TRY(current_device_sms(&sms));
+    MONARCH_CUDA_TRY(cudaFuncSetAttribute(rect_dl_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     const int cx = (b + kS2Cols - 1) / kS2Cols;
     long long slabs = (sms + cx - 1) / cx;                            // one CTA per SM, one wave
     if (slabs > (tokens + kS2Tok - 1) / kS2Tok) slabs = (tokens + kS2Tok - 1) / kS2Tok;

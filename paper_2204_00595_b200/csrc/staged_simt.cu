@@ -376,11 +376,13 @@ extern "C" int monarch_fwd_noalloc(const void *x, const void *L, const void *R, 
     const void *ptrs[] = {x, L, R, y};
     for (const void *p : ptrs)
         if (!p || ((uintptr_t)p & 15)) return MONARCH_ERR_INVALID_ARG;
-    const size_t act = (size_t)tokens * n * esize(dtype), wb = (size_t)n * m * esize(dtype);
+    // the intermediate needs one element per input element; it must fit the built-in array (compared by division:
+    // tokens * n * element size could wrap for absurd token counts)
+    const size_t row = (size_t)n * esize(dtype);
+    if ((uint64_t)tokens > (uint64_t)MONARCH_NOALLOC_SCRATCH_BYTES / row) return MONARCH_ERR_WORKSPACE;
+    const size_t act = (size_t)tokens * row, wb = (size_t)n * m * esize(dtype);
     if (ranges_overlap(y, act, x, act) || ranges_overlap(y, act, L, wb) || ranges_overlap(y, act, R, wb))
         return MONARCH_ERR_INVALID_ARG;
-    // the intermediate needs one element per input element; it must fit the built-in array
-    if (act > (size_t)MONARCH_NOALLOC_SCRATCH_BYTES) return MONARCH_ERR_WORKSPACE;
     if (tokens == 0) return MONARCH_OK;
     void *u = nullptr;
     MONARCH_TRY(noalloc_scratch_address(&u));

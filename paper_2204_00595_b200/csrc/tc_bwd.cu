@@ -215,13 +215,11 @@ int launch_wgrad128(const void *A, const void *B, float *out, int64_t tokens, un
     CUtensorMap tm_a, tm_b;
     MONARCH_TRY(encode_tmap_2d(&tm_a, A, (uint64_t)tokens, n, (uint64_t)n * 2, 64, 64, 128));
     MONARCH_TRY(encode_tmap_2d(&tm_b, B, (uint64_t)tokens, n, (uint64_t)n * 2, 64, 64, 128));
-    static int sms = 0;
-    if (!sms) {
-        int dev = 0;
-        MONARCH_CUDA_TRY(cudaGetDevice(&dev));
-        MONARCH_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        MONARCH_CUDA_TRY(cudaFuncSetAttribute(tc_wgrad128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmem));
-    }
+    // per call: the SM count and the shared-memory attribute belong to the current device, and a first-call
+    // cache would not be safe against two host threads
+    int sms = 0;
+    MONARCH_TRY(current_device_sms(&sms));
+    MONARCH_CUDA_TRY(cudaFuncSetAttribute(tc_wgrad128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmem));
     WgradParams p;
     p.out = out;
     p.status = status;
