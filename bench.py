@@ -211,16 +211,26 @@ KERNELS_OF = {
     (64, "bf16", "mlp_fwd"): "fused_fwd_m64_team_kernel (2 launches)",
     (64, "bf16", "mlp_bwd"): "fused_fwd_m64_team_kernel + mlp_act_kernel + fused_fwd_m64_kernel (stage 1 only) + "
                              "2 x fused_bwd_all_m64_kernel + mlp_dact_kernel + merge_status_kernel (7 launches)",
-    (128, "bf16", "fwd"): "chain_gemm_kernel x 2 + plane_transpose_kernel (3 launches)",
-    (128, "bf16", "bwd"): "plane_transpose_kernel + chain_gemm_kernel x 2 with the token reductions "
-                          "(3 launches, 2 memset nodes)",
+    (128, "bf16", "fwd"): "chain_fused_fwd_kernel (1 persistent launch; chain_gemm_kernel x 2 + plane_transpose_kernel "
+                          "beyond 8192 tiles)",
+    (128, "bf16", "bwd"): "plane_transpose_kernel + chain_gemm_kernel x 2 with the token reductions (3 launches)",
     (128, "bf16", "bwd_dx"): "plane_transpose_kernel + chain_gemm_kernel x 2 (3 launches)",
-    (128, "bf16", "bwd_dw"): "chain_gemm_kernel (stage 1) + plane_transpose_kernel + chain_gemm_kernel x 2 "
-                             "(4 launches, 2 memset nodes)",
+    (128, "bf16", "bwd_dw"): "chain_gemm_kernel (stage 1) + plane_transpose_kernel + chain_gemm_kernel x 2 (4 launches)",
 }
+_W3 = "profiles/fused_m64_workload3_ncu.md, full size"
+_W4 = "profiles/chain_m128_workload4_ncu.md, full size, cold L2 per launch (upper bound)"
 NCU_TRAFFIC_MB = {
-    (3, "fwd"): (150.0, "profiles/fused_m64_step_workload3_ncu_full.md, full size"),
-    (3, "bwd"): (365.6, "profiles/fused_m64_step_workload3_ncu_full.md, full size"),
+    (1, "fwd"): (0.1, "profiles/fused_fwd_m16_workload1_ncu.md, full size; the 65 KB output is still in L2 at kernel end"),
+    (2, "fwd"): (33.9, "profiles/fused_fwd_m32_workload2_ncu.md, full size; the 33.6 MB output is still in L2 at kernel end"),
+    (3, "fwd"): (146.9, _W3),
+    (3, "bwd"): (364.0, _W3),
+    (3, "bwd_dx"): (139.8, _W3),
+    (3, "bwd_dw"): (408.3, _W3),
+    (4, "fwd"): (480.4, _W4),
+    (4, "bwd"): (948.0, _W4),
+    (4, "bwd_dx"): (649.0, _W4),
+    (4, "bwd_dw"): (1070.0, _W4),
+    (5, "mlp_fwd"): (1511.0, "profiles/mlp_fwd_workload5_ncu.md, full size, both passes"),
 }
 
 
