@@ -34,10 +34,12 @@
  *    when one of their bounded waits runs out; zero it once with
  *    monarch_workspace_init and read it with monarch_last_device_status.
  *    Calls that overlap on the GPU must not share a workspace.
- *  - Weight gradients of the tensor-core families are summed with fp32
- *    reductions whose order across thread blocks is not fixed: dL, dR can
- *    differ in the last fp32 bits from run to run (the CUDA-core family,
- *    MONARCH_IMPL_STAGED, sums in a fixed order).
+ *  - Weight gradients of the fused tensor-core kernels (bf16, m = 64; the
+ *    general class) are summed with fp32 reductions whose order across thread
+ *    blocks is not fixed: dL, dR can differ in the last fp32 bits from run to
+ *    run.  The bf16 m = 128 kernels (one thread block sums all tokens of a
+ *    block, in a fixed order) and the CUDA-core family (MONARCH_IMPL_STAGED)
+ *    give the same bits every run.
  *  - Return value: a monarch_status_t.  Nothing throws.
  */
 #ifndef MONARCH_H_
