@@ -85,22 +85,6 @@ static __device__ __forceinline__ float gelu_fast(float a)
     return a * r;
 }
 
-// The same function with one MUFU operation instead of two: a sigmoid(2 z) = a/2 (1 + tanh z), z = a poly(a^2)
-// with the same fitted polynomial, tanh from the hardware approximation (relative error 2^-11, so the result
-// is off by at most 2.5e-4 |a|: a sixteenth of a bf16 ulp for a > 0, an absolute 1e-3 in the negative tail).
-// For epilogues in which the two MUFU operations per element of gelu_fast are the longest pipe (four warps,
-// one per scheduler, 16 MUFU lanes per SM).
-static __device__ __forceinline__ float gelu_fast_tanh(float a)
-{
-    const float a2 = fminf(a * a, 64.0f);
-    float t = fmaf(a2, -0.00035151677629392575f, 0.03700564581269318f);
-    t = fmaf(a2, t, 0.7975078480466281f);
-    float th;
-    asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(a * t));
-    const float ha = 0.5f * a;
-    return fmaf(ha, th, ha);
-}
-
 // d/da GELU(a) = Phi(a) + a phi(a) with Phi from the same sigmoid (|Phi error| <= 5.1e-5) and the normal
 // density phi evaluated directly: |error| <= 5.1e-5, for results that are rounded to bf16.
 static __device__ __forceinline__ float gelu_fast_grad(float a)

@@ -376,7 +376,7 @@ fused_fwd_m64_team_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid
                             for (int a = 0; a < 8; ++a) {
                                 const float b = __uint_as_float((a & 1) ? (bw[a >> 1] & 0xFFFF0000u) : (bw[a >> 1] << 16));
                                 float f = __uint_as_float(v[a][q]) + b;
-                                if (p.gelu) f = gelu_fast_tanh(f);
+                                if (p.gelu) f = gelu_fast(f);
                                 v[a][q] = __float_as_uint(f);
                             }
                         }
