@@ -253,6 +253,22 @@ int monarch_debug_skip_load(int64_t item);
  * thread-safe against concurrent calls. Returns the previous value, or -1. */
 int monarch_set_impl(int impl);
 
+/* Summation order of the weight gradients dL[j][l][k] = sum_t dy[t][l*m+j] u[t][k][j]
+ * and dR[k][j][i] = sum_t du[t][k][j] x[t][k*m+i] (the adjoints of Section 3.3,
+ * steps 1-2) in the fused bf16 m = 64 kernels behind monarch_bwd and
+ * monarch_bwd_dw.  on != 0: every thread block writes the partial sums of its
+ * (fixed) share of the token tiles to the workspace and a second small launch adds
+ * them in a fixed order - the same bits on every run, accumulate honoured by that
+ * launch; monarch_workspace_bytes for these two operations then reports 32 MiB
+ * more, and a device on which the one-launch backward cannot run gets
+ * MONARCH_ERR_UNSUPPORTED instead of the multi-launch form.  on == 0 (default):
+ * partial sums are added with fp32 atomics in whatever order they arrive.  Other
+ * sizes and dtypes already sum in a fixed order or are not affected (the
+ * feed-forward block and the general class keep their atomics).  Process-wide,
+ * affects later calls and later workspace-size queries; not thread-safe against
+ * concurrent calls.  Returns the previous setting. */
+int monarch_set_deterministic(int on);
+
 /* Name of the kernel family the next call with these arguments would use
  * ("staged-simt", "fused-simt", "staged-tcgen05", "fused-tcgen05"; "unsupported").  Static storage. */
 const char *monarch_impl_name(int op, int32_t m, int dtype);

@@ -39,6 +39,7 @@ _SIGNATURES = {
     "monarch_debug_set_wait_limit": (_int, [_vp, ctypes.c_uint, _vp]),
     "monarch_debug_skip_load": (_int, [_i64]),
     "monarch_set_impl": (_int, [_int]),
+    "monarch_set_deterministic": (_int, [_int]),
     "monarch_impl_name": (ctypes.c_char_p, [_int, _i32, _int]),
     "monarch_launch_count": (ctypes.c_uint64, []),
     "monarch_status_string": (ctypes.c_char_p, [_int]),
@@ -161,6 +162,11 @@ def monarch_debug_skip_load(item: int) -> None:
 
 def monarch_set_impl(impl: int) -> int:
     return int(lib().monarch_set_impl(impl))
+
+
+def monarch_set_deterministic(on: bool) -> bool:
+    """Fixed summation order for dL, dR of the fused bf16 m = 64 backward; returns the previous setting."""
+    return bool(lib().monarch_set_deterministic(1 if on else 0))
 
 
 def monarch_impl_name(op: int, m: int, dtype: int) -> str:

@@ -175,19 +175,25 @@ int fused_bwd_dx_m64_keep(const void *dy, const void *L, const void *R, void *dx
                           unsigned *counters, unsigned *status, int64_t tokens, cudaStream_t s);
 
 // dx, dL +=, dR += in one launch; u = P R x in the forward exchange layout, du / dyp = scratch exchange buffers
+// partials (optional, kBwdPartialBytes): per-CTA partial sums + a fixed-order reduction instead of atomic adds; dL, dR
+// are then overwritten (accumulate = 0) or added to (1) by that reduction
+constexpr int kBwdMaxPartials = 16;                                  // CTAs per group of a weight-gradient kind, at most
+constexpr size_t kBwdPartialBytes = (size_t)2 * kBwdMaxPartials * 64 * 64 * 64 * sizeof(float);
 int fused_bwd_all_m64(const void *x, const void *dy, const void *L, const void *R, const void *u, void *dx,
                       void *du, void *dyp, float *dL, float *dR, unsigned *counters, unsigned *status,
-                      int64_t tokens, cudaStream_t s);
+                      int64_t tokens, cudaStream_t s, float *partials = nullptr, int accumulate = 1);
 
 // ---- weight gradients for m = 64, bf16 (fused_m64_bwd_dw.cu) ----
-size_t fused_bwd_dw_m64_workspace_bytes(int64_t tokens);
+// fixed_order: the weight gradients are summed in a fixed order (partial sums in the workspace, which is then
+// kBwdPartialBytes larger); refused (MONARCH_ERR_UNSUPPORTED) where the one-launch backward cannot run
+size_t fused_bwd_dw_m64_workspace_bytes(int64_t tokens, bool fixed_order = false);
 int fused_bwd_dw_m64(const void *x, const void *dy, const void *L, const void *R, float *dL, float *dR,
-                     int accumulate, int64_t tokens, void *ws, cudaStream_t s);
+                     int accumulate, int64_t tokens, void *ws, cudaStream_t s, bool fixed_order = false);
 // dx, dL, dR in one pass; u_saved (optional) = the exchange buffer a fused forward call left behind
-size_t fused_bwd_m64_workspace_bytes(int64_t tokens);
+size_t fused_bwd_m64_workspace_bytes(int64_t tokens, bool fixed_order = false);
 int fused_bwd_m64(const void *x, const void *dy, const void *L, const void *R, const void *u_saved,
                   void *dx, float *dL, float *dR, int accumulate, int64_t tokens, void *ws,
-                  cudaStream_t s);
+                  cudaStream_t s, bool fixed_order = false);
 // where the fused forward keeps u inside its workspace
 const void *fused_fwd_m64_saved_u(const void *fwd_ws);
 

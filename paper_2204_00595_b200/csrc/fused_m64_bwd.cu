@@ -64,6 +64,8 @@ struct BwdParams {
     const __nv_bfloat16 *dy;   // natural dy (for L2 prefetch hints only; the data path goes through TMA)
     const __nv_bfloat16 *u;    // all-in-one kernel: u' = P R x, [tiles][64 j][8][64 t][8] (forward exchange layout)
     float *dL, *dR;            // all-in-one kernel: gradients (added to)
+    float *part_dL, *part_dR;  // all-in-one kernel, fixed summation order: every CTA stores its partial sums to slot
+                               // [index within its group][64 blocks][64][64] instead of adding them to dL / dR (else null)
     long long *trace;          // optional per-CTA timeline (debug builds), else null
 };
 
@@ -659,6 +661,11 @@ __device__ __forceinline__ void red_add_v4(float *p, uint32_t a, uint32_t b, uin
                  : "memory");
 }
 
+__device__ __forceinline__ void store_v4(float *p, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    *reinterpret_cast<uint4 *>(p) = make_uint4(a, b, c, d);
+}
+
 constexpr int kRSlotBytes = 16384;               // B2R / WL ring slot: two 8 KB operands of one block
 
 __device__ __forceinline__ void b2r_body(const CUtensorMap &tm_R, const CUtensorMap &tm_x, const CUtensorMap &tm_dx,
@@ -811,7 +818,8 @@ __device__ __forceinline__ void b2r_body(const CUtensorMap &tm_R, const CUtensor
         // dR partial sums of this CTA's tiles: lanes 16-31 of each quarter hold row 16 q4 + lane - 16 of block b
         if (!mbar_wait(drf, 0, p.status, dead, kErrMmaWait)) return;
         tc_fence_after();
-        float *out = p.dR + (long long)(grp * 8) * 4096 + row * 64;
+        const bool part = p.part_dR != nullptr;
+        float *out = (part ? p.part_dR + (size_t)first * (64 * 4096) : p.dR) + (long long)(grp * 8) * 4096 + row * 64;
 #pragma unroll 1
         for (int b = sub * 4; b < sub * 4 + 4; ++b) {
 #pragma unroll
@@ -824,7 +832,8 @@ __device__ __forceinline__ void b2r_body(const CUtensorMap &tm_R, const CUtensor
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
                         const uint32_t *w = &v[e >> 2][(e & 3) * 4];
-                        red_add_v4(out + b * 4096 + h * 32 + e * 4, w[0], w[1], w[2], w[3]);
+                        if (part) store_v4(out + b * 4096 + h * 32 + e * 4, w[0], w[1], w[2], w[3]);
+                        else red_add_v4(out + b * 4096 + h * 32 + e * 4, w[0], w[1], w[2], w[3]);
                     }
                 }
             }
@@ -910,7 +919,8 @@ __device__ __forceinline__ void wl_body(const BwdParams &p, uint32_t ring0, Bars
         tc_fence_after();
         const uint32_t lane_base = tmem_base + ((uint32_t)(q4 * 32) << 16);
         const int row = q4 * 16 + (lane & 15);
-        float *out = p.dL + (long long)(blk0 + (lane >> 4) * 8) * 4096 + row * 64;
+        const bool part = p.part_dL != nullptr;
+        float *out = (part ? p.part_dL + (size_t)first * (64 * 4096) : p.dL) + (long long)(blk0 + (lane >> 4) * 8) * 4096 + row * 64;
 #pragma unroll 1
         for (int b = sub * 4; b < sub * 4 + 4; ++b) {
 #pragma unroll
@@ -922,7 +932,8 @@ __device__ __forceinline__ void wl_body(const BwdParams &p, uint32_t ring0, Bars
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                     const uint32_t *w = &v[e >> 2][(e & 3) * 4];
-                    red_add_v4(out + b * 4096 + h * 32 + e * 4, w[0], w[1], w[2], w[3]);
+                    if (part) store_v4(out + b * 4096 + h * 32 + e * 4, w[0], w[1], w[2], w[3]);
+                    else red_add_v4(out + b * 4096 + h * 32 + e * 4, w[0], w[1], w[2], w[3]);
                 }
             }
         }
@@ -1079,10 +1090,28 @@ int launch_bwd_m64(const void *dy, const void *L, const void *R, void *dx, void 
 }
 }  // namespace
 
-// dx, dL += , dR += in one launch (see the all-in-one kernel); u = u' in the forward exchange layout
+namespace {
+// dW = (accumulate ? dW : 0) + part[0] + part[1] + ... in this order: the same bits every run
+__global__ void reduce_partials_kernel(float4 *__restrict__ dW, const float4 *__restrict__ part, int count, int accumulate,
+                                       int n4)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n4) return;
+    float4 acc = accumulate ? dW[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < count; ++s) {
+        const float4 v = part[(size_t)s * n4 + i];
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    dW[i] = acc;
+}
+}  // namespace
+
+// dx, dL += , dR += in one launch (see the all-in-one kernel); u = u' in the forward exchange layout.
+// partials != null (kBwdPartialBytes of scratch): the CTAs store their partial sums there and a second small launch adds
+// them in a fixed order: dL, dR = (accumulate ? old : 0) + sums, bit-identical from run to run.
 int fused_bwd_all_m64(const void *x, const void *dy, const void *L, const void *R, const void *u, void *dx,
                       void *du, void *dyp, float *dL, float *dR, unsigned *counters, unsigned *status,
-                      int64_t tokens, cudaStream_t s)
+                      int64_t tokens, cudaStream_t s, float *partials, int accumulate)
 {
     using namespace tc;
     if (tokens == 0) return MONARCH_OK;
@@ -1135,6 +1164,9 @@ int fused_bwd_all_m64(const void *x, const void *dy, const void *L, const void *
     if (b2 > tiles) b2 = (int)tiles;
     if (b3 > tiles) b3 = (int)tiles;
     if (8 * b1 + 8 * b2 + 4 * b3 > sms) return MONARCH_ERR_UNSUPPORTED;   // all CTAs must be co-resident
+    if (partials != nullptr && (b2 > kBwdMaxPartials || b3 > kBwdMaxPartials)) return MONARCH_ERR_UNSUPPORTED;
+    p.part_dR = partials;
+    p.part_dL = partials ? partials + (size_t)kBwdMaxPartials * (kN * kM) : nullptr;
     p.b1 = b1;
     p.b2 = b2;
     p.b3 = b3;
@@ -1148,6 +1180,14 @@ int fused_bwd_all_m64(const void *x, const void *dy, const void *L, const void *
                                                                                  tm_x, p);
     note_launch();
     MONARCH_CUDA_TRY(cudaGetLastError());
+    if (partials != nullptr) {
+        // a CTA of a group takes tiles first, first + step, ...: CTAs beyond the tile count have no partial sums
+        const int n4 = kN * kM / 4;
+        reduce_partials_kernel<<<(n4 + 255) / 256, 256, 0, s>>>((float4 *)dR, (const float4 *)p.part_dR, b2, accumulate, n4);
+        reduce_partials_kernel<<<(n4 + 255) / 256, 256, 0, s>>>((float4 *)dL, (const float4 *)p.part_dL, b3, accumulate, n4);
+        note_launch(2);
+        MONARCH_CUDA_TRY(cudaGetLastError());
+    }
     return MONARCH_OK;
 }
 

@@ -193,10 +193,11 @@ fused_bwd_dw_m64_kernel(const __grid_constant__ CUtensorMap tm_x, const DwParams
 constexpr size_t kDwCounterBytes = 65536;
 
 // Workspace: [status 256 B][reserved 64 KB][u][du][P dy], each tokens (rounded up to 64) x 4096 bf16.
-size_t fused_bwd_dw_m64_workspace_bytes(int64_t tokens)
+size_t fused_bwd_dw_m64_workspace_bytes(int64_t tokens, bool fixed_order)
 {
     const size_t tiles = (size_t)((tokens + 63) / 64);
-    return MONARCH_STATUS_BYTES + kDwCounterBytes + 3 * ((tiles * 64 * (size_t)tc::kN * 2 + 255) & ~(size_t)255);
+    return MONARCH_STATUS_BYTES + kDwCounterBytes + 3 * ((tiles * 64 * (size_t)tc::kN * 2 + 255) & ~(size_t)255) +
+           (fixed_order ? kBwdPartialBytes : 0);
 }
 
 namespace {
@@ -248,15 +249,18 @@ int zero_grads(float *dL, float *dR, cudaStream_t s)
 }  // namespace
 
 int fused_bwd_dw_m64(const void *x, const void *dy, const void *L, const void *R, float *dL, float *dR,
-                     int accumulate, int64_t tokens, void *ws, cudaStream_t s)
+                     int accumulate, int64_t tokens, void *ws, cudaStream_t s, bool fixed_order)
 {
-    if (!accumulate) MONARCH_TRY(zero_grads(dL, dR, s));
+    if (!accumulate && (!fixed_order || tokens == 0)) MONARCH_TRY(zero_grads(dL, dR, s));
     if (tokens == 0) return MONARCH_OK;
     const size_t ex = exchange_bytes(tokens);
     unsigned *status = (unsigned *)ws;
     char *u = (char *)ws + MONARCH_STATUS_BYTES + kDwCounterBytes;
     char *du = u + ex, *dyp = du + ex;
     MONARCH_TRY(fused_fwd_m64_stage1(x, R, u, tokens, status, s));
+    if (fixed_order)
+        return fused_bwd_all_m64(x, dy, L, R, u, nullptr, du, dyp, dL, dR, (unsigned *)((char *)ws + MONARCH_STATUS_BYTES), status,
+                                 tokens, s, (float *)(dyp + ex), accumulate);
     // the one-launch backward with its dx part switched off: du and P dy are consumed from L2 as they appear
     // instead of after a launch of their own (it declines, before launching anything, on a GPU too small to hold
     // all of its CTAs at once; then the three-launch form below runs)
@@ -268,16 +272,16 @@ int fused_bwd_dw_m64(const void *x, const void *dy, const void *L, const void *R
 }
 
 // Workspace: [status 256 B][tile counters 64 KB][du][P dy][u], each tokens (rounded up to 64) x 4096 bf16.
-size_t fused_bwd_m64_workspace_bytes(int64_t tokens)
+size_t fused_bwd_m64_workspace_bytes(int64_t tokens, bool fixed_order)
 {
-    return MONARCH_STATUS_BYTES + kDwCounterBytes + 3 * exchange_bytes(tokens);
+    return MONARCH_STATUS_BYTES + kDwCounterBytes + 3 * exchange_bytes(tokens) + (fixed_order ? kBwdPartialBytes : 0);
 }
 
 int fused_bwd_m64(const void *x, const void *dy, const void *L, const void *R, const void *u_saved,
                   void *dx, float *dL, float *dR, int accumulate, int64_t tokens, void *ws,
-                  cudaStream_t s)
+                  cudaStream_t s, bool fixed_order)
 {
-    if (!accumulate) MONARCH_TRY(zero_grads(dL, dR, s));
+    if (!accumulate && (!fixed_order || tokens == 0)) MONARCH_TRY(zero_grads(dL, dR, s));
     if (tokens == 0) return MONARCH_OK;
     const size_t ex = exchange_bytes(tokens);
     unsigned *status = (unsigned *)ws;
@@ -299,6 +303,9 @@ int fused_bwd_m64(const void *x, const void *dy, const void *L, const void *R, c
 #endif
     // the one-launch form declines, before launching anything, on a GPU too small to hold all of its CTAs at once
     // (or for more tiles than it has counters): then the backward kernel and the token reduction run as two launches
+    if (fixed_order)
+        return fused_bwd_all_m64(x, dy, L, R, u, dx, du, dyp, dL, dR, counters, status, tokens, s, (float *)(u_own + ex),
+                                 accumulate);
     const int rc = fused_bwd_all_m64(x, dy, L, R, u, dx, du, dyp, dL, dR, counters, status, tokens, s);
     if (rc != MONARCH_ERR_UNSUPPORTED) return rc;
     MONARCH_TRY(fused_bwd_dx_m64_keep(dy, L, R, dx, du, dyp, counters, status, tokens, s));

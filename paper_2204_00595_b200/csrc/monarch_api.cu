@@ -8,6 +8,7 @@ namespace monarch {
 
 static std::atomic<uint64_t> g_launches{0};
 static std::atomic<int> g_impl{MONARCH_IMPL_AUTO};
+static std::atomic<int> g_fixed_order{0};     // monarch_set_deterministic
 
 void note_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
@@ -174,7 +175,7 @@ size_t monarch_workspace_bytes(int op, int64_t tokens, int32_t n, int32_t m, int
         return tc_staged_bwd_workspace_bytes(tokens, m);
     if (which == kTcStaged && op == MONARCH_OP_FWD && m == 128) return chain_fwd_m128_workspace_bytes(tokens);
     if (op == MONARCH_OP_BWD) {
-        if (which == kFused) return fused_bwd_m64_workspace_bytes(tokens);
+        if (which == kFused) return fused_bwd_m64_workspace_bytes(tokens, g_fixed_order.load(std::memory_order_relaxed) != 0);
         const size_t a = staged_workspace_bytes(MONARCH_OP_BWD_DX, tokens, n, m, dtype);
         const size_t b = staged_workspace_bytes(MONARCH_OP_BWD_DW, tokens, n, m, dtype);
         return a > b ? a : b;
@@ -184,7 +185,7 @@ size_t monarch_workspace_bytes(int op, int64_t tokens, int32_t n, int32_t m, int
                : op == MONARCH_OP_MLP_FWD ? fused_mlp_fwd_m64_workspace_bytes(tokens)
                : op == MONARCH_OP_FWD    ? fused_fwd_m64_workspace_bytes(tokens)
                : op == MONARCH_OP_BWD_DX ? fused_bwd_dx_m64_workspace_bytes(tokens)
-                                         : fused_bwd_dw_m64_workspace_bytes(tokens);
+                                         : fused_bwd_dw_m64_workspace_bytes(tokens, g_fixed_order.load(std::memory_order_relaxed) != 0);
     return staged_workspace_bytes(op, tokens, n, m, dtype);
 }
 
@@ -244,7 +245,8 @@ int monarch_bwd_dw(const void *x, const void *dy, const void *L, const void *R, 
     MONARCH_TRY(check_buffers(in, 4, out, 2, workspace, workspace_bytes,
                               monarch_workspace_bytes(MONARCH_OP_BWD_DW, tokens, n, m, dtype)));
     if (which == kFused)
-        return fused_bwd_dw_m64(x, dy, L, R, dL, dR, accumulate, tokens, workspace, (cudaStream_t)stream);
+        return fused_bwd_dw_m64(x, dy, L, R, dL, dR, accumulate, tokens, workspace, (cudaStream_t)stream,
+                                g_fixed_order.load(std::memory_order_relaxed) != 0);
     if (which == kTcStaged)
         return tc_staged_bwd(x, dy, L, R, nullptr, dL, dR, accumulate, 0, 1, tokens, m, workspace,
                              (cudaStream_t)stream);
@@ -271,7 +273,7 @@ int monarch_bwd(const void *x, const void *dy, const void *L, const void *R, con
     if (which == kFused) {
         const bool saved = fwd_workspace != nullptr && pick(MONARCH_OP_FWD, m, dtype) == kFused;
         return fused_bwd_m64(x, dy, L, R, saved ? fused_fwd_m64_saved_u(fwd_workspace) : nullptr, dx, dL,
-                             dR, accumulate, tokens, workspace, s);
+                             dR, accumulate, tokens, workspace, s, g_fixed_order.load(std::memory_order_relaxed) != 0);
     }
     if (which == kTcStaged) {
         const bool saved = fwd_workspace != nullptr && m == 128 && pick(MONARCH_OP_FWD, m, dtype) == kTcStaged;
@@ -524,6 +526,11 @@ int monarch_debug_skip_load(int64_t item)
 {
     debug_skip_next_plane_load(item);
     return MONARCH_OK;
+}
+
+int monarch_set_deterministic(int on)
+{
+    return g_fixed_order.exchange(on != 0 ? 1 : 0);
 }
 
 int monarch_set_impl(int impl)

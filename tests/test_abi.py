@@ -88,6 +88,28 @@ def test_impl_selection(lib):
         B.monarch_set_impl(prev)
 
 
+def test_deterministic_switch_changes_only_the_m64_backward_workspaces(lib):
+    """monarch_set_deterministic: returns the previous setting; while on, the workspace of the two bf16 m = 64
+    calls that sum weight gradients grows by the 32 MiB of partial sums; every other query is unchanged."""
+    T = 1000
+    def sizes():
+        return {(op, m, dt): B.monarch_workspace_bytes(op, T, m * m, m, dt)
+                for op in (B.OP_FWD, B.OP_BWD_DX, B.OP_BWD_DW, B.OP_BWD, B.OP_MLP_FWD)
+                for m, dt in ((16, B.F32), (32, B.BF16), (64, B.BF16), (64, B.F32), (128, B.BF16))}
+    before = sizes()
+    assert B.monarch_set_deterministic(True) is False
+    try:
+        assert B.monarch_set_deterministic(True) is True
+        after = sizes()
+    finally:
+        B.monarch_set_deterministic(False)
+    grown = {k for k in before if after[k] != before[k]}
+    assert grown == {(B.OP_BWD_DW, 64, B.BF16), (B.OP_BWD, 64, B.BF16)}
+    for k in grown:
+        assert after[k] - before[k] == 2 * 16 * 64 ** 3 * 4
+    assert sizes() == before
+
+
 def test_missing_library_fails_loudly(tmp_path, monkeypatch):
     monkeypatch.setattr(B, "_lib", None)
     monkeypatch.setattr(B, "_LIB_PATH", str(tmp_path / "libmonarch.so"))

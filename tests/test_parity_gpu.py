@@ -147,6 +147,58 @@ def test_bwd_one_call(P, impl, m, T, dtype, saved):
     assert_close(to_host64(dR), 2 * ref["dR"], dtype, "dR accumulate")
 
 
+@pytest.mark.parametrize("T", [1, 130, 64 * 40 - 63, 8192])
+def test_bwd_m64_fixed_summation_order(P, T):
+    """monarch_set_deterministic(1): dL and dR of the fused m = 64 backward are sums in a fixed order - two runs
+    from different initial contents give the same bits, both calls (monarch_bwd, monarch_bwd_dw) agree with the
+    oracle, accumulate = 1 adds to what is there, and a workspace sized before the switch is refused."""
+    import torch
+    m, dtype, code = 64, "bf16", P.BF16
+    n = m * m
+    d = _small_inputs(m, T, dtype, seed=9100 + T)
+    x, dy, L, R = (to_device(d[k], dtype) for k in ("x", "dy", "L", "R"))
+    ref = O.bwd(d["x"], d["dy"], d["L"], d["R"])
+    small = P.monarch_workspace_bytes(P.OP_BWD, T, n, m, code)
+    prev = P.monarch_set_deterministic(True)
+    try:
+        assert P.monarch_impl_name(P.OP_BWD, m, code) == "fused-tcgen05"
+        nb = P.monarch_workspace_bytes(P.OP_BWD, T, n, m, code)
+        assert nb > small
+        ws_f = P.Workspace(P.monarch_workspace_bytes(P.OP_FWD, T, n, m, code))
+        ws_b = P.Workspace(nb)
+        ws_w = P.Workspace(P.monarch_workspace_bytes(P.OP_BWD_DW, T, n, m, code))
+        y = torch.empty_like(x)
+        dx = torch.empty_like(x)
+        P.monarch_fwd(x, L, R, y, T, n, m, ws_f)
+        runs = []
+        for fill, saved in ((float("nan"), True), (123.0, False), (-7.0, True)):
+            dL = torch.full((m, m, m), fill, device="cuda")
+            dR = torch.full((m, m, m), fill, device="cuda")
+            P.monarch_bwd(x, dy, L, R, dx, dL, dR, 0, T, n, m, ws_b, fwd_workspace=ws_f if saved else None)
+            torch.cuda.synchronize()
+            assert P.monarch_last_device_status(ws_b) == 0
+            runs.append((dL.clone(), dR.clone()))
+        for dL, dR in runs[1:]:
+            assert torch.equal(dL, runs[0][0]) and torch.equal(dR, runs[0][1])
+        assert_close(to_host64(dx), ref["dx"], dtype, "dx")
+        assert_close(to_host64(runs[0][0]), ref["dL"], dtype, "dL fixed order")
+        assert_close(to_host64(runs[0][1]), ref["dR"], dtype, "dR fixed order")
+        # weight gradients alone: same partial sums, same order
+        dL = torch.full((m, m, m), float("nan"), device="cuda")
+        dR = torch.full((m, m, m), float("nan"), device="cuda")
+        P.monarch_bwd_dw(x, dy, L, R, dL, dR, 0, T, n, m, ws_w)
+        P.monarch_bwd_dw(x, dy, L, R, dL, dR, 1, T, n, m, ws_w)
+        torch.cuda.synchronize()
+        assert P.monarch_last_device_status(ws_w) == 0
+        assert_close(to_host64(dL), 2 * ref["dL"], dtype, "dL accumulate, fixed order")
+        assert_close(to_host64(dR), 2 * ref["dR"], dtype, "dR accumulate, fixed order")
+        with pytest.raises(P.MonarchError):
+            P.monarch_bwd(x, dy, L, R, dx, dL, dR, 0, T, n, m, P.Workspace(small))
+    finally:
+        P.monarch_set_deterministic(prev)
+    assert P.monarch_workspace_bytes(P.OP_BWD, T, n, m, code) == small
+
+
 # Token counts around the persistent kernels' schedule boundaries: 18 teams of 8 CTAs (m = 64: one, two and
 # "two and a bit" tiles per team), 148 CTAs (m = 32), each with a ragged last tile.
 @pytest.mark.parametrize("m,T", [(64, 64 * 18 - 1), (64, 64 * 18 + 1), (64, 64 * 36 + 5), (64, 64 * 40 - 63),
