@@ -481,9 +481,13 @@ plane_transpose_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_c
 // the waits cannot deadlock; the lag hides them.  x is read once and y written once (by the load/store units,
 // straight from the transposed plane); u' is also kept for the backward call, w' lives in a ring of RING tiles
 // that stays in L2.
-constexpr int kFusedLag = 3, kFusedRing = 2 * kFusedLag + 2;
+#ifndef MONARCH_FUSED_LAG
+#define MONARCH_FUSED_LAG 3
+#endif
+constexpr int kFusedLag = MONARCH_FUSED_LAG, kFusedRing = 2 * kFusedLag + 2;
 constexpr int kStoreSets = 3;                // store-warp pairs taking the items in turn
-constexpr int kFusedThreads = (11 + 2 * kStoreSets) * 32;   // warps 0-3 epilogue, 4-7 transposers, 8 loader, 9 MMA, 10.. store warps, last: plane loader
+constexpr int kFusedThreads = (12 + 2 * kStoreSets) * 32;   // warps 0-3 epilogue, 4-7 transposers, 8 loader, 9 MMA, 10.. store warps, then plane loader, then L2 prefetch
+constexpr int kFusedPrefetch = 2;           // steps between the L2 prefetch of an x tile and its load
 constexpr int kFusedSmem = 2 * kOpBytes /* R_b, L_b */ + 2 * kOpBytes /* operand ring */ + kStagingBytes +
                            2 * kOpBytes /* plane in, out */ + 1024;
 constexpr unsigned kFusedCounters = 8192;    // tiles per counter array (two arrays in the 64 KB after the status word)
@@ -492,6 +496,7 @@ struct FusedParams {
     unsigned *status;
     unsigned *cnt1, *cnt2;                   // per tile: store warps (two per CTA) whose stage-1 / stage-2 rows are in memory
     char *u, *w, *y;                         // u' planes, w' ring, output
+    const char *x;                           // input, for the L2 prefetch hints only (the data path goes through TMA)
     long long tokens;
     int ntiles;
     long long *trace;                        // debug builds: per-CTA cycle sums of the waits, else null
@@ -551,6 +556,7 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
     __shared__ __align__(8) FusedBars bars;
     __shared__ uint32_t tmem_base_s;
     __shared__ int dead_s;
+    __shared__ int x_prog_s;                 // x tiles the loader has asked for
 
     const uint32_t w0 = (smem_u32(smem_raw) + 1023u) & ~1023u;          // R_b, L_b
     const uint32_t ring0 = w0 + 2 * kOpBytes;
@@ -574,6 +580,7 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
         mbar_init(smem_u32(&bars.tr_empty), 4);
         fence_mbar_init();
         dead_s = 0;
+        x_prog_s = 0;
         tma_prefetch_desc(&tm_x); tma_prefetch_desc(&tm_R); tma_prefetch_desc(&tm_L);
     }
     if (warp == 0) {
@@ -621,6 +628,7 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
                     mbar_expect_tx(full0 + sl * 8, kOpBytes);
                     load_operand<kLdX>(ring0 + sl * kOpBytes, &tm_x, nullptr, b, s, full0 + sl * 8);
                     ++g;
+                    *reinterpret_cast<volatile int *>(&x_prog_s) = s + 1;
                 }
             }
             FOUT(0, wa); FOUT(1, wc); FOUT(2, wb);
@@ -750,6 +758,24 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
             }
         }
         if (warp == 10 && lane == 0) { FOUT(8, wf); FOUT(9, clock64() - ts0); }
+    } else if (warp == 11 + 2 * kStoreSets) {
+        // ------------------------------------------------------------ L2 prefetch of x: the operand ring has two slots, so
+        // an x tile is asked for only when the MMAs two items back are done - one DRAM latency too late.  This warp asks
+        // L2 for the tile kFusedPrefetch steps ahead (256-byte rows, one token apart) through the load/store units.
+        volatile int *x_prog = &x_prog_s;
+        const unsigned long long limit = wait_limit_ns(p.status);
+        for (int s = 0; s < nt; ++s) {
+            if (s >= *x_prog + kFusedPrefetch) {
+                const unsigned long long t0 = global_timer_ns();
+                while (s >= *x_prog + kFusedPrefetch && !*dead && global_timer_ns() - t0 < limit) { }
+                if (s >= *x_prog + kFusedPrefetch) break;
+            }
+            const char *a = p.x + ((size_t)s * 128 + (lane >> 1)) * ((size_t)kB * kB * 2) + b * 256 + (lane & 1) * 128;
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if ((long long)s * 128 + i * 16 + (lane >> 1) < p.tokens)
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(a + (size_t)i * 16 * ((size_t)kB * kB * 2)));
+        }
     } else if (warp == 10 + 2 * kStoreSets) {
         // ------------------------------------------------------------ plane loader
         if (lane == 0) {
@@ -977,6 +1003,7 @@ int chain_fwd_m128(const void *x, const void *L, const void *R, void *y, int64_t
         fp.u = up;
         fp.w = wp;
         fp.y = (char *)y;
+        fp.x = (const char *)x;
         fp.tokens = tokens;
         fp.trace = nullptr;
 #ifdef MONARCH_TRACE
