@@ -109,7 +109,7 @@ bool tc_staged_available(int op, int m, int dtype)
 {
     if (dtype != MONARCH_BF16 || m < 32) return false;
     if (op == MONARCH_OP_FWD || op == MONARCH_OP_MLP_FWD || op == MONARCH_OP_BWD_DX) return true;
-    return m == 128;      // dL, dR: the token-reduction kernel is built for 128 x 128 blocks
+    return m == 32 || m == 64 || m == 128;      // dL, dR: the token-reduction kernel works on 128-column windows
 }
 
 // kernel family for a call under the current selection

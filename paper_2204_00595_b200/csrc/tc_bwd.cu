@@ -76,10 +76,12 @@ __global__ void __launch_bounds__(256) transpose_blocks_kernel(const __nv_bfloat
 }
 
 // ---------------------------------------------------------------------------------------------- token reduction
-// out[b][r][c] += sum_t A[t][b*128 + r] * B[t][b*128 + c] for 128 x 128 blocks: both operands are read
-// token-major (MN-major descriptors over 64-token x 64-column TMA boxes, 128B swizzle), a CTA owns 4 blocks
-// (4 accumulators of 128 lanes x 128 columns fill TMEM) and a slice of the token tiles, and adds its partial
-// sums to the output with vector reductions in L2 at the end.
+// out[g][r][c] += sum_t A[t][g*m + r] * B[t][g*m + c] for m x m blocks, m = 32, 64 or 128 (dR from du and x, dL from
+// P dy and u').  The kernel works on windows of 128 columns: D = A_w^T B_w (128 x 128, contraction over tokens) holds
+// the sums of the window's 128 / m blocks on its diagonal; the off-diagonal part pairs different blocks and is
+// dropped (the tensor pipe is idle anyway).  Both operands are read token-major (MN-major descriptors over 64-token x
+// 64-column TMA boxes, 128B swizzle), a CTA owns 4 windows (4 accumulators of 128 lanes x 128 columns fill TMEM) and
+// a slice of the token tiles, and adds its partial sums to the output with vector reductions in L2 at the end.
 constexpr int kWM = 128;
 constexpr int kWSlotBytes = 32768;             // A tile 16 KB + B tile 16 KB (two 64-column halves each)
 constexpr int kWSlots = 6;
@@ -90,6 +92,8 @@ struct WgradParams {
     float *out;
     unsigned *status;
     int tiles, slices;
+    int m;                 // block size: 128 (a window is one block), 64 or 32 (its 2 or 4 diagonal sub-blocks are blocks)
+    int windows;           // 128-column windows of a token row (n / 128)
 };
 
 __device__ __forceinline__ bool wait_fast(uint32_t bar, uint32_t parity, unsigned *status, volatile int *dead,
@@ -100,7 +104,7 @@ __device__ __forceinline__ bool wait_fast(uint32_t bar, uint32_t parity, unsigne
 }
 
 __global__ void __launch_bounds__(kWThreads, 1)
-tc_wgrad128_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const WgradParams p)
+tc_wgrad_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const WgradParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[kWSlots], bar_empty[kWSlots], bar_acc;
@@ -139,7 +143,7 @@ tc_wgrad128_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
                 uint32_t ph = 0;
                 for (int tile = first; tile < p.tiles && !dead; tile += step) {
 #pragma unroll 1
-                    for (int b = 0; b < 4; ++b) {
+                    for (int b = 0; b < 4 && blk0 + b < p.windows; ++b) {
                         if (!wait_fast(empty0 + slot * 8, ph ^ 1, p.status, &dead, kErrSlotWait)) break;
                         const uint32_t dst = ring0 + slot * kWSlotBytes, full = full0 + slot * 8;
                         const int col = (blk0 + b) * kWM;
@@ -163,7 +167,7 @@ tc_wgrad128_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
                 for (int tile = first; ok && tile < p.tiles; tile += step) {
                     const uint32_t accum = tile != first;
 #pragma unroll 1
-                    for (int b = 0; b < 4; ++b) {
+                    for (int b = 0; b < 4 && blk0 + b < p.windows; ++b) {
                         if (!wait_fast(full0 + slot * 8, ph, p.status, &dead, kErrTmaWait)) { ok = false; break; }
                         tc_fence_after();
                         const uint64_t ad = desc | (uint64_t)((ring0 + slot * kWSlotBytes) >> 4);
@@ -185,10 +189,13 @@ tc_wgrad128_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
                 const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
                 const int row = warp * 32 + lane;
 #pragma unroll 1
-                for (int b = 0; b < 4; ++b) {
-                    float *out = p.out + ((long long)(blk0 + b) * kWM + row) * kWM;
+                for (int b = 0; b < 4 && blk0 + b < p.windows; ++b) {
+                    // the window's diagonal m x m sub-blocks are the blocks' sums (the rest of the 128 x 128 product pairs
+                    // rows and columns of different blocks and is dropped); row `row` of the window is row g % m of block g / m
+                    const int g = (blk0 + b) * kWM + row, c0 = (row / p.m) * p.m;     // c0 is uniform over a warp: m >= 32
+                    float *out = p.out + ((long long)(g / p.m) * p.m + g % p.m) * p.m - c0;
 #pragma unroll 1
-                    for (int c = 0; c < kWM; c += 16) {
+                    for (int c = c0; c < c0 + p.m; c += 16) {
                         uint32_t v[16];
                         tmem_ld16(lane_base + b * 128 + c, v);
                         tmem_ld_wait();
@@ -208,10 +215,11 @@ tc_wgrad128_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
     if (warp == 0) tmem_dealloc(tmem_base, 512);
 }
 
-int launch_wgrad128(const void *A, const void *B, float *out, int64_t tokens, unsigned *status, cudaStream_t s)
+// out[g][r][c] += sum_t A[t][g*m + r] B[t][g*m + c] for every block g (m = 32, 64 or 128; A, B token-major [tokens][m*m])
+int launch_wgrad(const void *A, const void *B, float *out, int64_t tokens, int m, unsigned *status, cudaStream_t s)
 {
     if (tokens == 0) return MONARCH_OK;
-    const int n = kWM * kWM;
+    const int n = m * m;
     CUtensorMap tm_a, tm_b;
     MONARCH_TRY(encode_tmap_2d(&tm_a, A, (uint64_t)tokens, n, (uint64_t)n * 2, 64, 64, 128));
     MONARCH_TRY(encode_tmap_2d(&tm_b, B, (uint64_t)tokens, n, (uint64_t)n * 2, 64, 64, 128));
@@ -219,16 +227,19 @@ int launch_wgrad128(const void *A, const void *B, float *out, int64_t tokens, un
     // cache would not be safe against two host threads
     int sms = 0;
     MONARCH_TRY(current_device_sms(&sms));
-    MONARCH_CUDA_TRY(cudaFuncSetAttribute(tc_wgrad128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmem));
+    MONARCH_CUDA_TRY(cudaFuncSetAttribute(tc_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmem));
     WgradParams p;
     p.out = out;
     p.status = status;
     p.tiles = (int)((tokens + 63) / 64);
-    int slices = sms / 32;
+    p.m = m;
+    p.windows = n / kWM;
+    const int groups = (p.windows + 3) / 4;          // a CTA keeps the accumulators of four windows in TMEM
+    int slices = sms / groups;
     if (slices < 1) slices = 1;
     if (slices > p.tiles) slices = p.tiles;
     p.slices = slices;
-    tc_wgrad128_kernel<<<dim3(32, slices), kWThreads, kWSmem, s>>>(tm_a, tm_b, p);
+    tc_wgrad_kernel<<<dim3(groups, slices), kWThreads, kWSmem, s>>>(tm_a, tm_b, p);
     note_launch();
     MONARCH_CUDA_TRY(cudaGetLastError());
     return MONARCH_OK;
@@ -292,13 +303,13 @@ size_t tc_staged_bwd_workspace_bytes(int64_t tokens, int m)
     return MONARCH_STATUS_BYTES + 3 * act + 2 * wb;
 }
 
-// want_dx / want_dw select the outputs; dW needs m = 128 (the token-reduction kernel's block size)
+// want_dx / want_dw select the outputs
 int tc_staged_bwd(const void *x, const void *dy, const void *L, const void *R, void *dx, float *dL, float *dR,
                   int accumulate, int want_dx, int want_dw, int64_t tokens, int m, void *ws, cudaStream_t s,
                   const void *saved_up)
 {
     using namespace tc;
-    if (want_dw && m != 128) return MONARCH_ERR_UNSUPPORTED;
+    if (want_dw && m != 32 && m != 64 && m != 128) return MONARCH_ERR_UNSUPPORTED;
     if (m == 128) {
         // chain of block GEMMs on token-innermost intermediates (chain_m128.cu)
         if (tokens == 0 && want_dw && !accumulate) {
@@ -325,8 +336,8 @@ int tc_staged_bwd(const void *x, const void *dy, const void *L, const void *R, v
     }
     if (want_dw) {
         MONARCH_TRY(tc_stage(m, x, R, l.u, nullptr, 0, tokens, status, s));               // u'[t][j][k]
-        MONARCH_TRY(launch_wgrad128(l.du, x, dR, tokens, status, s));
-        MONARCH_TRY(launch_wgrad128(l.z, l.u, dL, tokens, status, s));
+        MONARCH_TRY(launch_wgrad(l.du, x, dR, tokens, m, status, s));
+        MONARCH_TRY(launch_wgrad(l.z, l.u, dL, tokens, m, status, s));
     }
     return MONARCH_OK;
 }

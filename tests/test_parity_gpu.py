@@ -114,8 +114,8 @@ def test_fwd_bwd_small(P, impl, m, T, dtype):
 
 
 @pytest.mark.parametrize("saved", [False, True])
-@pytest.mark.parametrize("m,T,dtype", [(16, 65, "f32"), (32, 129, "bf16"), (64, 1, "bf16"), (64, 130, "bf16"),
-                                       (64, 257, "bf16"), (128, 70, "bf16")])
+@pytest.mark.parametrize("m,T,dtype", [(16, 65, "f32"), (32, 129, "bf16"), (32, 64 * 150 + 7, "bf16"), (64, 1, "bf16"),
+                                       (64, 130, "bf16"), (64, 257, "bf16"), (128, 70, "bf16")])
 def test_bwd_one_call(P, impl, m, T, dtype, saved):
     """monarch_bwd = monarch_bwd_dx + monarch_bwd_dw, with or without the forward call's workspace."""
     import torch
@@ -197,6 +197,28 @@ def test_bwd_m64_fixed_summation_order(P, T):
     finally:
         P.monarch_set_deterministic(prev)
     assert P.monarch_workspace_bytes(P.OP_BWD, T, n, m, code) == small
+
+
+def test_m32_backward_runs_on_the_tensor_cores(P):
+    """bf16 m = 32: dL and dR come from the tcgen05 token-reduction kernel (128-column windows whose diagonal 32 x 32
+    sub-blocks are the blocks' sums), not from the CUDA-core kernel - by name and against the oracle, on a token count
+    with a ragged last tile."""
+    import torch
+    m, T, dtype, code = 32, 64 * 9 + 5, "bf16", P.BF16
+    n = m * m
+    for op in (P.OP_BWD, P.OP_BWD_DW, P.OP_BWD_DX):
+        assert P.monarch_impl_name(op, m, code) == "staged-tcgen05"
+    d = _small_inputs(m, T, dtype, seed=3232)
+    x, dy, L, R = (to_device(d[k], dtype) for k in ("x", "dy", "L", "R"))
+    dL = torch.full((m, m, m), float("nan"), device="cuda")
+    dR = torch.full((m, m, m), float("nan"), device="cuda")
+    ws = P.Workspace(P.monarch_workspace_bytes(P.OP_BWD_DW, T, n, m, code))
+    P.monarch_bwd_dw(x, dy, L, R, dL, dR, 0, T, n, m, ws)
+    torch.cuda.synchronize()
+    assert P.monarch_last_device_status(ws) == 0
+    ref = O.bwd(d["x"], d["dy"], d["L"], d["R"])
+    assert_close(to_host64(dL), ref["dL"], dtype, "m32 dL")
+    assert_close(to_host64(dR), ref["dR"], dtype, "m32 dR")
 
 
 # Token counts around the persistent kernels' schedule boundaries: 18 teams of 8 CTAs (m = 64: one, two and
