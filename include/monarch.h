@@ -294,7 +294,9 @@ const char *monarch_status_string(int status);
  * the outputs are complete and are not re-entrant on one context.
  *
  * monarch_host_create: max_tokens bounds later calls; chunk_tokens is the
- * staging granularity (a multiple of 64; 0 picks a default).  Allocates
+ * staging granularity (a multiple of 64; 0 picks max_tokens / 8 rounded up to
+ * 64 and clamped to [256, 2048], so that uploads and downloads of different
+ * chunks overlap for most of a call).  Allocates
  * device memory with cudaMalloc on the current device; MONARCH_ERR_CUDA if
  * that fails, MONARCH_ERR_UNSUPPORTED / MONARCH_ERR_INVALID_ARG for bad
  * shapes.  monarch_host_destroy frees everything (null is a no-op). */

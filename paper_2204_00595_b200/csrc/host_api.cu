@@ -106,7 +106,13 @@ int monarch_host_create(monarch_host_ctx **out, int64_t max_tokens, int32_t n, i
 {
     if (!out || max_tokens < 0 || chunk_tokens < 0) return MONARCH_ERR_INVALID_ARG;
     *out = nullptr;
-    if (chunk_tokens == 0) chunk_tokens = 2048;
+    if (chunk_tokens == 0) {
+        // default: about eight chunks, so that uploads and downloads overlap for most of the call (the first upload
+        // and the last download cannot), but no smaller than 256 tokens (the kernels' fill and drain) nor larger than 2048
+        chunk_tokens = (max_tokens / 8 + 63) / 64 * 64;
+        if (chunk_tokens < 256) chunk_tokens = 256;
+        if (chunk_tokens > 2048) chunk_tokens = 2048;
+    }
     if (chunk_tokens % 64) return MONARCH_ERR_INVALID_ARG;
     if (chunk_tokens > max_tokens && max_tokens > 0) chunk_tokens = (max_tokens + 63) / 64 * 64;
     const size_t wsb = monarch_workspace_bytes(MONARCH_OP_FWD, chunk_tokens, n, m, dtype);
