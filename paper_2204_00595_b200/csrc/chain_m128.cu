@@ -486,7 +486,7 @@ plane_transpose_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_c
 #endif
 constexpr int kFusedLag = MONARCH_FUSED_LAG, kFusedRing = 2 * kFusedLag + 2;
 constexpr int kStoreSets = 3;                // store-warp pairs taking the items in turn
-constexpr int kFusedThreads = (12 + 2 * kStoreSets) * 32;   // warps 0-3 epilogue, 4-7 transposers, 8 loader, 9 MMA, 10.. store warps, then plane loader, then L2 prefetch
+constexpr int kFusedThreads = (13 + 2 * kStoreSets) * 32;   // warps 0-3 epilogue, 4-7 transposers, 8 u' loader, 9 MMA, 10.. store warps, then plane loader, L2 prefetch, x loader
 constexpr int kFusedPrefetch = 2;           // steps between the L2 prefetch of an x tile and its load
 constexpr int kFusedSmem = 2 * kOpBytes /* R_b, L_b */ + 2 * kOpBytes /* operand ring */ + kStagingBytes +
                            2 * kOpBytes /* plane in, out */ + 1024;
@@ -610,28 +610,29 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
             tma_load_2d(w0 + kOpBytes, &tm_L, 0, b * kB, wbar);
             tma_load_2d(w0 + kOpBytes + kHalfBytes, &tm_L, 64, b * kB, wbar);
             pdl_wait();
-            uint32_t g = 0;                                // operand-ring items so far
-            [[maybe_unused]] long long wa = 0, wc = 0, wb = 0;
-            for (int s = 0; s < nsteps; ++s) {
-                const int tb = s - kFusedLag;
-                if (tb >= 0 && tb < nt) {
-                    { FT0(); if (!wait_counter(p.cnt1 + tb, 2 * kB, kB, p.status, dead)) break; FACC(wc); }
-                    const uint32_t sl = g & 1;
-                    { FT0(); if (!mbar_wait(empty0 + sl * 8, ((g >> 1) & 1) ^ 1, p.status, dead, kErrSlotWait)) break; FACC(wb); }
-                    mbar_expect_tx(full0 + sl * 8, kOpBytes);
-                    load_operand<kLdC>(ring0 + sl * kOpBytes, nullptr, p.u, b, tb, full0 + sl * 8);
-                    ++g;
-                }
-                if (s < nt) {
-                    const uint32_t sl = g & 1;
-                    { FT0(); if (!mbar_wait(empty0 + sl * 8, ((g >> 1) & 1) ^ 1, p.status, dead, kErrSlotWait)) break; FACC(wa); }
-                    mbar_expect_tx(full0 + sl * 8, kOpBytes);
-                    load_operand<kLdX>(ring0 + sl * kOpBytes, &tm_x, nullptr, b, s, full0 + sl * 8);
-                    ++g;
-                    *reinterpret_cast<volatile int *>(&x_prog_s) = s + 1;
-                }
+            // the u' slabs of stage 2 go through ring slot 1; the x tiles have their own loader and slot 0, so that a wait
+            // for the other CTAs here never holds back this CTA's own stage 1 (whose rows the others are waiting for)
+            [[maybe_unused]] long long wc = 0, wb = 0;
+            for (int tb = 0; tb < nt; ++tb) {
+                { FT0(); if (!wait_counter(p.cnt1 + tb, 2 * kB, kB, p.status, dead)) break; FACC(wc); }
+                { FT0(); if (!mbar_wait(empty0 + 8, (tb & 1) ^ 1, p.status, dead, kErrSlotWait)) break; FACC(wb); }
+                mbar_expect_tx(full0 + 8, kOpBytes);
+                load_operand<kLdC>(ring0 + kOpBytes, nullptr, p.u, b, tb, full0 + 8);
             }
-            FOUT(0, wa); FOUT(1, wc); FOUT(2, wb);
+            FOUT(1, wc); FOUT(2, wb);
+        }
+    } else if (warp == 12 + 2 * kStoreSets) {
+        // ------------------------------------------------------------ x loader (ring slot 0)
+        if (lane == 0) {
+            pdl_wait();
+            [[maybe_unused]] long long wa = 0;
+            for (int s = 0; s < nt; ++s) {
+                { FT0(); if (!mbar_wait(empty0, (s & 1) ^ 1, p.status, dead, kErrSlotWait)) break; FACC(wa); }
+                mbar_expect_tx(full0, kOpBytes);
+                load_operand<kLdX>(ring0, &tm_x, nullptr, b, s, full0);
+                *reinterpret_cast<volatile int *>(&x_prog_s) = s + 1;
+            }
+            FOUT(0, wa);
         }
     } else if (warp == 9) {
         // ------------------------------------------------------------ MMA issuer
@@ -646,15 +647,16 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
                     const int kind = 1 - ki;                      // stage 2 of the older tile first, then stage 1
                     const int tile = kind == 0 ? s : s - kFusedLag;
                     if (tile < 0 || tile >= nt) continue;
-                    const uint32_t buf = g & 1;
+                    // accumulators alternate item by item; the operand comes from the slot of its kind (slot use = tile)
+                    const uint32_t buf = g & 1, sl = kind;
                     { FT0(); if (!mbar_wait(acce0 + buf * 8, ((g >> 1) & 1) ^ 1, p.status, dead, kErrTmemWait)) { ok = false; break; } FACC(wa); }
-                    { FT0(); if (!mbar_wait(full0 + buf * 8, (g >> 1) & 1, p.status, dead, kErrTmaWait)) { ok = false; break; } FACC(wf); }
+                    { FT0(); if (!mbar_wait(full0 + sl * 8, tile & 1, p.status, dead, kErrTmaWait)) { ok = false; break; } FACC(wf); }
                     tc_fence_after();
-                    const uint32_t t0 = ring0 + buf * kOpBytes, w = w0 + kind * kOpBytes, d = tmem_base + buf * 128;
+                    const uint32_t t0 = ring0 + sl * kOpBytes, w = w0 + kind * kOpBytes, d = tmem_base + buf * 128;
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks)
                         mma_f16_ss(d, op_desc(w, false, ks), op_desc(t0, kind == 1, ks), kind == 0 ? idesc_a : idesc_b, ks != 0);
-                    mma_commit(empty0 + buf * 8);
+                    mma_commit(empty0 + sl * 8);
                     mma_commit(accf0 + buf * 8);
                     ++g;
                 }
