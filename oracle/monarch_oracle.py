@@ -277,6 +277,84 @@ def rect_factors_from_definition(Lp, R):
     return Ld, Rd
 
 
+# --------------------------------------------------------------------------
+# rectangular class with wrapped-diagonal blocks (appendix, rectangular definition with b2 != b3)
+# --------------------------------------------------------------------------
+
+def wrapped_positions(b2: int, b3: int):
+    """Where the stored entries of one wrapped-diagonal block S (b3 x b2) sit: entry e of the max(b2, b3) stored
+    values is S[i0[e], j0[e]].  For b2 <= b3 a row i0 holds its one non-zero in column i0 mod b2; for b2 > b3 the
+    definition is applied to the transpose: a column j0 holds its one non-zero in row j0 mod b3."""
+    e = np.arange(max(b2, b3))
+    return (e, e % b2) if b2 <= b3 else (e % b3, e)
+
+
+def rectw_factors_from_definition(Lw, R, b3: int):
+    """Dense factors of the rectangular definition: R = diag(R_k) (n2 x n1) and L (n3 x n2), an r x q grid of
+    wrapped-diagonal blocks, built entry by entry from the definition's rule for the zero pattern (every (i, j) is
+    visited and tested), with S_{l,k}'s stored values Lw[l, k, :]."""
+    Lw = np.asarray(Lw, dtype=np.float64); R = np.asarray(R, dtype=np.float64)
+    q, b2, b1 = R.shape
+    r = Lw.shape[0]
+    if Lw.shape != (r, q, max(b2, b3)):
+        raise ValueError("Lw must be [r, q, max(b2, b3)]")
+    Rd = np.zeros((q * b2, q * b1))
+    for k in range(q):
+        Rd[k * b2:(k + 1) * b2, k * b1:(k + 1) * b1] = R[k]
+    Ld = np.zeros((r * b3, q * b2))
+    for i in range(r * b3):
+        i1, i0 = divmod(i, b3)
+        for j in range(q * b2):
+            j1, j0 = divmod(j, b2)
+            if b2 <= b3:
+                if i0 % b2 == j0:
+                    Ld[i, j] = Lw[i1, j1, i0]
+            elif j0 % b3 == i0:
+                Ld[i, j] = Lw[i1, j1, j0]
+    return Ld, Rd
+
+
+def rectw_fwd(x, Lw, R, b3: int) -> np.ndarray:
+    """y = L R x for the rectangular class with wrapped-diagonal blocks, as two steps:
+    u[t, k, :] = R_k x[t, k, :], then every stored entry of L moves one element of u to one element of y:
+    y[t, l*b3 + i0(e)] += Lw[l, k, e] * u[t, k*b2 + j0(e)].   x: [T, q*b1] -> y: [T, r*b3]."""
+    Lw = _f64(Lw); R = _f64(R); x = _f64(x)
+    q, b2, b1 = R.shape
+    r = Lw.shape[0]
+    T = x.shape[0]
+    if Lw.shape != (r, q, max(b2, b3)) or x.shape != (T, q * b1):
+        raise ValueError("shape mismatch")
+    i0, j0 = wrapped_positions(b2, b3)
+    u = np.einsum("kji,tki->tkj", R, x.reshape(T, q, b1))
+    y = np.zeros((T, r, b3))
+    for l in range(r):
+        for k in range(q):
+            np.add.at(y[:, l, :], (slice(None), i0), Lw[l, k][None, :] * u[:, k, j0])
+    return y.reshape(T, r * b3)
+
+
+def rectw_bwd(x, dy, Lw, R, b3: int):
+    """Gradients of <dy, L R x> for the wrapped-diagonal rectangular class: dict with dx, dL (like Lw), dR."""
+    Lw = _f64(Lw); R = _f64(R); x = _f64(x); dy = _f64(dy)
+    q, b2, b1 = R.shape
+    r = Lw.shape[0]
+    T = x.shape[0]
+    if Lw.shape != (r, q, max(b2, b3)) or x.shape != (T, q * b1) or dy.shape != (T, r * b3):
+        raise ValueError("shape mismatch")
+    i0, j0 = wrapped_positions(b2, b3)
+    xk = x.reshape(T, q, b1)
+    u = np.einsum("kji,tki->tkj", R, xk)
+    dyl = dy.reshape(T, r, b3)
+    du = np.zeros((T, q, b2))
+    dL = np.empty_like(Lw)
+    for l in range(r):
+        for k in range(q):
+            np.add.at(du[:, k, :], (slice(None), j0), Lw[l, k][None, :] * dyl[:, l, i0])
+            dL[l, k] = np.einsum("te,te->e", dyl[:, l, i0], u[:, k, j0])
+    return {"dx": np.einsum("kji,tkj->tki", R, du).reshape(T, q * b1), "dL": dL,
+            "dR": np.einsum("tkj,tki->kji", du, xk)}
+
+
 def cplx_dense_from_definition(L, R) -> np.ndarray:
     """Definition 3.1 with complex factors: M = P L P^T R as a dense complex n x n matrix."""
     L = np.asarray(L, dtype=np.complex128); R = np.asarray(R, dtype=np.complex128)

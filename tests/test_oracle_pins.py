@@ -548,6 +548,65 @@ def test_rect_gradients(q, b1, b, r):
     assert np.isclose(np.sum(g["dx"] * x), s, rtol=1e-12)
 
 
+WRAPPED = [(3, 2, 2, 4, 2), (2, 3, 4, 2, 3), (2, 2, 3, 5, 2), (3, 1, 5, 3, 2), (2, 4, 2, 6, 1), (2, 2, 6, 2, 3),
+           (1, 3, 4, 4, 2)]
+
+
+@pytest.mark.parametrize("q,b1,b2,b3,r", WRAPPED)
+def test_wrapped_rect_matches_definition(q, b1, b2, b3, r):
+    """The two-step multiply against L R x with both factors materialised from the appendix's rectangular definition
+    (block-diagonal R; L a grid of wrapped-diagonal blocks, whose zero pattern is tested entry by entry), and the
+    number of stored entries against the count the paper states, n2 n3 / min(b2, b3)."""
+    rng = np.random.default_rng(q * 1000 + b1 * 100 + b2 * 10 + b3)
+    R = rng.standard_normal((q, b2, b1)); Lw = rng.standard_normal((r, q, max(b2, b3)))
+    x = rng.standard_normal((5, q * b1))
+    Ld, Rd = O.rectw_factors_from_definition(Lw, R, b3)
+    assert np.count_nonzero(Ld) == (q * b2) * (r * b3) // min(b2, b3) == Lw.size
+    assert np.allclose(O.rectw_fwd(x, Lw, R, b3), x @ (Ld @ Rd).T, atol=1e-12)
+
+
+@pytest.mark.parametrize("q,b1,b,r", [(3, 2, 4, 2), (2, 5, 3, 3)])
+def test_wrapped_rect_reduces_to_diagonal_blocks(q, b1, b, r):
+    """b2 = b3: a wrapped diagonal is a diagonal, and the multiply is the rectangular multiply pinned above with
+    Lp[j, l, k] = Lw[l, k, j]."""
+    rng = np.random.default_rng(77 + q + b)
+    R = rng.standard_normal((q, b, b1)); Lw = rng.standard_normal((r, q, b)); x = rng.standard_normal((4, q * b1))
+    Lp = np.ascontiguousarray(Lw.transpose(2, 0, 1))
+    assert np.allclose(O.rectw_fwd(x, Lw, R, b), O.rect_fwd(x, Lp, R), atol=1e-12)
+    dy = rng.standard_normal((4, r * b))
+    g, h = O.rectw_bwd(x, dy, Lw, R, b), O.rect_bwd(x, dy, Lp, R)
+    assert np.allclose(g["dx"], h["dx"], atol=1e-12) and np.allclose(g["dR"], h["dR"], atol=1e-12)
+    assert np.allclose(g["dL"], h["dL"].transpose(1, 2, 0), atol=1e-12)
+
+
+@pytest.mark.parametrize("q,b1,b2,b3,r", WRAPPED)
+def test_wrapped_rect_gradients(q, b1, b2, b3, r):
+    """dx, dL, dR against the dense chain rule through the factors of the definition (dM = dy^T x, dL = dM R^T and
+    dR = L^T dM restricted to the stored entries) and central differences of the pinned forward."""
+    rng = np.random.default_rng(5000 + q * 100 + b2 * 10 + b3)
+    R = rng.standard_normal((q, b2, b1)); Lw = rng.standard_normal((r, q, max(b2, b3)))
+    x = rng.standard_normal((6, q * b1)); dy = rng.standard_normal((6, r * b3))
+    g = O.rectw_bwd(x, dy, Lw, R, b3)
+    Ld, Rd = O.rectw_factors_from_definition(Lw, R, b3)
+    assert np.allclose(g["dx"], dy @ (Ld @ Rd), atol=1e-12)
+    dM = dy.T @ x
+    dLd, dRd = dM @ Rd.T, Ld.T @ dM
+    i0, j0 = O.wrapped_positions(b2, b3)
+    for l in range(r):
+        for k in range(q):
+            assert np.allclose(g["dL"][l, k], dLd[l * b3 + i0, k * b2 + j0], atol=1e-11)
+    for k in range(q):
+        assert np.allclose(g["dR"][k], dRd[k * b2:(k + 1) * b2, k * b1:(k + 1) * b1], atol=1e-11)
+    f = lambda Lw_, R_: float(np.sum(dy * O.rectw_fwd(x, Lw_, R_, b3)))
+    eps = 1e-6
+    for idx in [(0, 0, 0), (r - 1, q - 1, max(b2, b3) - 1)]:
+        d = np.zeros_like(Lw); d[idx] = eps
+        assert abs((f(Lw + d, R) - f(Lw - d, R)) / (2 * eps) - g["dL"][idx]) < 1e-6
+    for idx in [(0, 0, 0), (q - 1, b2 - 1, b1 - 1)]:
+        d = np.zeros_like(R); d[idx] = eps
+        assert abs((f(Lw, R + d) - f(Lw, R - d)) / (2 * eps) - g["dR"][idx]) < 1e-6
+
+
 def test_rect_gradients_reduce_to_square():
     rng = np.random.default_rng(36)
     m, T = 4, 5
