@@ -42,10 +42,11 @@ def parse_args():
                          "100 for workload 7; 30 for --impl reference)")
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=4, choices=[1, 2, 3, 4, 5, 6, 7, 8],
+    ap.add_argument("--workload", type=int, default=4, choices=[1, 2, 3, 4, 5, 6, 7, 8, 9],
                     help="1-5: the square workloads; 6: the general (rectangular) class, forward only; "
                          "7: projection of a dense matrix onto the Monarch class + dense materialisation; "
-                         "8: complex multiply (planar), y = M x then z = M^H y")
+                         "8: complex multiply (planar), y = M x then z = M^H y; 9: the rectangular class with "
+                         "wrapped-diagonal blocks (b2 != b3)")
     ap.add_argument("--kernels", default="auto", choices=["auto", "staged", "fused"])
     ap.add_argument("--calls", default="", help="comma-separated subset of the workload's calls "
                     "(profiling aid; the default step runs them all)")
@@ -237,26 +238,33 @@ NCU_TRAFFIC_MB = {
 def main_rect(args):
     """Workload 6: forward of the general Monarch class (appendix), q = 4 blocks of 1024 x 1024, one GPU or
     token-sharded replicas; bound by the tensor pipe (stage 1 holds nearly all the FLOPs)."""
-    from paper_2204_00595_b200.inputs import RECT_WORKLOAD, make_rect_inputs
+    from paper_2204_00595_b200.inputs import RECT_WORKLOAD, RECTW_WORKLOAD, make_rect_inputs, make_rectw_inputs
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    c = RECT_WORKLOAD
-    q, b1, b, r, T = c["q"], c["b1"], c["b"], c["r"], c["tokens"]
+    wrapped = args.workload == 9                          # wrapped-diagonal blocks: b is R's block height b2, b3 that of L's blocks
+    c = RECTW_WORKLOAD if wrapped else RECT_WORKLOAD
+    q, b1, b, r, T = c["q"], c["b1"], c["b2" if wrapped else "b"], c["r"], c["tokens"]
+    b3 = c["b3"] if wrapped else b
+    nL = r * q * max(b, b3)                               # stored entries of L
     with_bwd = "rect_bwd" in args.calls.split(",")
-    fwd_flops = 2 * T * (q * b * b1 + b * r * q)
+    fwd_flops = 2 * T * (q * b * b1 + nL)
     flops = fwd_flops * (3 if with_bwd else 1)           # backward: dx and the two weight gradients, 2x the forward
-    nbytes = T * (q * b1 + r * b) * 2 + (q * b * b1 + b * r * q) * 2
-    workload = (f"workload 6: rect_fwd{'+rect_bwd' if with_bwd else ''} bf16 q={q} b1={b1} b={b} r={r} "
-                f"tokens/GPU={T}")
+    nbytes = T * (q * b1 + r * b3) * 2 + (q * b * b1 + nL) * 2
+    workload = (f"workload {args.workload}: rect_fwd{'+rect_bwd' if with_bwd else ''} bf16 q={q} b1={b1} "
+                + (f"b2={b} b3={b3}" if wrapped else f"b={b}") + f" r={r} tokens/GPU={T}")
     metric, unit = "monarch_rect_fwd_tflops", "TFLOP/s"
+    make_inputs_ = make_rectw_inputs if wrapped else make_rect_inputs
 
     def time_oracle_rect(d, target_s):
         from oracle import monarch_oracle as O
         Ts, dt = 8, 0.0
         while True:
             t0 = time.perf_counter()
-            O.rect_fwd(d["x"][:Ts], d["L"], d["R"])
+            if wrapped:
+                O.rectw_fwd(d["x"][:Ts], d["L"], d["R"], b3)
+            else:
+                O.rect_fwd(d["x"][:Ts], d["L"], d["R"])
             dt = time.perf_counter() - t0
             if dt >= target_s / 4 or Ts >= T:
                 break
@@ -268,7 +276,7 @@ def main_rect(args):
             return 0
         from oracle import monarch_oracle as O
         O.build()
-        d = make_rect_inputs()
+        d = make_inputs_()
         rs = [time_oracle_rect(d, 8.0) for _ in range(args.warmup + args.steps)][args.warmup:]
         tfl = statistics.mean(x["tflops"] for x in rs)
         print(json.dumps({
@@ -292,19 +300,23 @@ def main_rect(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     P.monarch_set_impl({"auto": P.IMPL_AUTO, "staged": P.IMPL_STAGED, "fused": P.IMPL_AUTO}[args.kernels])
-    d = make_rect_inputs()
+    d = make_inputs_()
     R, L = to_device(d["R"], "bf16"), to_device(d["L"], "bf16")
     sets = []
     for s in range(2):                          # two rotating sets, each larger than L2 with its output
         x = torch.roll(to_device(d["x"], "bf16"), shifts=17 * s + 5 * rank, dims=0).contiguous()
-        sets.append((x, torch.empty(T, r * b, dtype=torch.bfloat16, device="cuda")))
-    ws = P.Workspace(P.monarch_rect_workspace_bytes(T, q, b1, b, r, P.BF16))
-    ws_b = P.Workspace(P.monarch_rect_bwd_workspace_bytes(T, q, b1, b, r, P.BF16))
+        sets.append((x, torch.empty(T, r * b3, dtype=torch.bfloat16, device="cuda")))
+    if wrapped:
+        ws = P.Workspace(P.monarch_rectw_workspace_bytes(T, q, b1, b, b3, r, P.BF16))
+        ws_b = P.Workspace(P.monarch_rectw_bwd_workspace_bytes(T, q, b1, b, b3, r, P.BF16))
+    else:
+        ws = P.Workspace(P.monarch_rect_workspace_bytes(T, q, b1, b, r, P.BF16))
+        ws_b = P.Workspace(P.monarch_rect_bwd_workspace_bytes(T, q, b1, b, r, P.BF16))
     stream = torch.cuda.current_stream()
     if with_bwd:
-        dy = torch.randn(T, r * b, device="cuda", generator=torch.Generator("cuda").manual_seed(595006)).bfloat16()
+        dy = torch.randn(T, r * b3, device="cuda", generator=torch.Generator("cuda").manual_seed(595006)).bfloat16()
         dxs = [torch.empty_like(sets[0][0]) for _ in range(2)]
-        gL = torch.zeros(b, r, q, dtype=torch.float32, device="cuda")
+        gL = torch.zeros(L.shape, dtype=torch.float32, device="cuda")
         gR = torch.zeros(q, b, b1, dtype=torch.float32, device="cuda")
     mid = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
@@ -312,11 +324,16 @@ def main_rect(args):
 
     def step(i, timed=False):
         x, y = sets[i % 2]
-        P.monarch_rect_fwd(x, L, R, y, T, q, b1, b, r, ws)
+        if wrapped:
+            P.monarch_rectw_fwd(x, L, R, y, T, q, b1, b, b3, r, ws)
+        else:
+            P.monarch_rect_fwd(x, L, R, y, T, q, b1, b, r, ws)
         if timed and with_bwd:                   # boundary between the two calls of a step
             mid[nmid[0]].record(stream)
             nmid[0] += 1
-        if with_bwd:
+        if with_bwd and wrapped:
+            P.monarch_rectw_bwd(x, dy, L, R, dxs[i % 2], gL, gR, 0, T, q, b1, b, b3, r, ws_b)
+        elif with_bwd:
             P.monarch_rect_bwd(x, dy, L, R, dxs[i % 2], gL, gR, 0, T, q, b1, b, r, ws_b, fwd_workspace=ws)
             if dist is not None:
                 dist.all_reduce(gL)
@@ -363,7 +380,8 @@ def main_rect(args):
         "calls": {"rect_fwd": {"ms": fwd_ms, "tflops": fwd_flops / fwd_ms / 1e9},
                   **({"rect_bwd": {"ms": ms - fwd_ms, "tflops": 2 * fwd_flops / (ms - fwd_ms) / 1e9}} if with_bwd else {})},
         "roofline": {"bound": "tensor", "kernel": "rect_fwd: rect_stage1_kernel<256> (tcgen05) + "
-                                                  "rect_stage2_stream_kernel (2 launches)"
+                                                  + ("relabel_kernel + " if wrapped else "") +
+                                                  "rect_stage2_stream_kernel (%d launches)" % (3 if wrapped else 2)
                                                   + ("; rect_bwd: stage 1, adjoint stage 2, adjoint stage 1 (tcgen05), "
                                                      "rect_wgrad_kernel (tcgen05), dl_small4_kernel" if with_bwd else ""),
                      "achieved": tfl, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
@@ -748,7 +766,7 @@ def main():
         return launch_ranks(args)
     if args.workload == 8:
         return main_cplx(args)
-    if args.workload == 6:
+    if args.workload in (6, 9):
         return main_rect(args)
     if args.workload == 7:
         return main_project(args)

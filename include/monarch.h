@@ -187,6 +187,40 @@ int monarch_rect_bwd(const void *x, const void *dy, const void *L, const void *R
 size_t monarch_rect_bwd_workspace_bytes(int64_t tokens, int32_t q, int32_t b1, int32_t b,
                                         int32_t r, int dtype);
 
+/* The rectangular class with WRAPPED-DIAGONAL blocks (appendix "General Monarch
+ * Matrix Parametrization", rectangular definition with b2 != b3):  y = L R x,
+ *   R = diag(R_0 .. R_{q-1}), R_k of size b2 x b1  (n1 = q*b1 inputs, n2 = q*b2),
+ *   L of size n3 x n2 (n3 = r*b3): an r x q grid of blocks S_{l,k} of size b3 x b2,
+ *   each a wrapped diagonal with max(b2, b3) entries: for b2 <= b3 row i0 has its
+ *   one non-zero in column i0 mod b2; for b2 > b3 column j0 has its one non-zero
+ *   in row j0 mod b3 (the definition applied to the transpose).
+ * Stored entry e of a block sits at (i0, j0) = (e, e mod b2) if b2 <= b3, else
+ * (e mod b3, e).  Steps:
+ *   u[t][k*b2 + j] = sum_i R[k][j][i] x[t][k*b1 + i]
+ *   y[t][l*b3 + i0(e)] += L[l][k][e] u[t][k*b2 + j0(e)]    over all k and e.
+ * x: [tokens][q*b1], y: [tokens][r*b3], storage dtype; R: [q][b2][b1];
+ * L: [r][q][max(b2, b3)].  b2 == b3 is monarch_rect_fwd with L[l][k][j] there
+ * stored as L[j][l][k].  Where one of b2, b3 divides the other the product is a
+ * diagonal-block product of other sizes and runs on those kernels after the
+ * weights are re-labelled in the workspace; other sizes run on plain CUDA-core
+ * kernels.  u is rounded to the storage dtype once.  Size limits and errors as
+ * for monarch_rect_fwd.  The backward call returns dx, dL (float32, laid out like
+ * L) and dR (float32 [q][b2][b1]) of f = <dy, L R x>; accumulate == 0 overwrites
+ * the two weight gradients, 1 adds to them; the sums over tokens use atomic adds.
+ * Workspaces: monarch_rectw_workspace_bytes, monarch_rectw_bwd_workspace_bytes
+ * (0 for invalid arguments). */
+int monarch_rectw_fwd(const void *x, const void *L, const void *R, void *y, int64_t tokens,
+                      int32_t q, int32_t b1, int32_t b2, int32_t b3, int32_t r, int dtype,
+                      void *workspace, size_t workspace_bytes, void *stream);
+size_t monarch_rectw_workspace_bytes(int64_t tokens, int32_t q, int32_t b1, int32_t b2, int32_t b3,
+                                     int32_t r, int dtype);
+int monarch_rectw_bwd(const void *x, const void *dy, const void *L, const void *R,
+                      void *dx, float *dL, float *dR, int accumulate, int64_t tokens,
+                      int32_t q, int32_t b1, int32_t b2, int32_t b3, int32_t r, int dtype,
+                      void *workspace, size_t workspace_bytes, void *stream);
+size_t monarch_rectw_bwd_workspace_bytes(int64_t tokens, int32_t q, int32_t b1, int32_t b2,
+                                         int32_t b3, int32_t r, int dtype);
+
 /* Complex Monarch multiply (Section 3.2: the DFT and the MM* products need
  * complex factors):  y = M x  (adjoint == 0)  or  y = M^H x  (adjoint == 1),
  * M = P L P^T R with complex blocks, M^H = R^H P L^H P.  An MM* product

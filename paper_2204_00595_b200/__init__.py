@@ -10,6 +10,7 @@ from .binding import (  # noqa: F401
     HostContext, MonarchError, Workspace, lib, monarch_bwd, monarch_bwd_dw, monarch_bwd_dx, monarch_fwd, monarch_fwd_noalloc, monarch_impl_name,
     monarch_last_device_status, monarch_launch_count, monarch_cplx_fwd, monarch_dense, monarch_mlp_bwd, monarch_mlp_fwd, monarch_project, monarch_rect_bwd, monarch_rect_bwd_workspace_bytes,
     monarch_rect_fwd, monarch_rect_workspace_bytes,
+    monarch_rectw_fwd, monarch_rectw_bwd, monarch_rectw_workspace_bytes, monarch_rectw_bwd_workspace_bytes,
     monarch_set_impl, monarch_set_deterministic, monarch_debug_set_wait_limit, monarch_debug_skip_load,
     monarch_status_string, monarch_workspace_bytes, monarch_workspace_init,
 )

@@ -30,6 +30,11 @@ _SIGNATURES = {
     "monarch_rect_workspace_bytes": (_sz, [_i64, _i32, _i32, _i32, _i32, _int]),
     "monarch_rect_bwd": (_int, [_vp] * 8 + [_int, _i64, _i32, _i32, _i32, _i32, _int, _vp, _sz, _vp]),
     "monarch_rect_bwd_workspace_bytes": (_sz, [_i64, _i32, _i32, _i32, _i32, _int]),
+    "monarch_rectw_fwd": (_int, [_vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32, _i32, _int, _vp, _sz, _vp]),
+    "monarch_rectw_workspace_bytes": (_sz, [_i64, _i32, _i32, _i32, _i32, _i32, _int]),
+    "monarch_rectw_bwd": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _int, _i64, _i32, _i32, _i32, _i32, _i32, _int, _vp, _sz,
+                                 _vp]),
+    "monarch_rectw_bwd_workspace_bytes": (_sz, [_i64, _i32, _i32, _i32, _i32, _i32, _int]),
     "monarch_cplx_fwd": (_int, [_vp, _vp, _vp, _vp, _int, _i64, _i32, _i32, _int, _vp, _sz, _vp]),
     "monarch_dense": (_int, [_vp, _vp, _vp, _i32, _i32, _int, _vp]),
     "monarch_project": (_int, [_vp, _vp, _vp, _i32, _i32, _int, _vp, _vp]),
@@ -298,6 +303,32 @@ def monarch_rect_bwd(x, dy, L, R, dx, dL, dR, accumulate, tokens, q, b1, b, r, w
     _check(lib().monarch_rect_bwd(_ptr(x, "x"), _ptr(dy, "dy", dt), _ptr(L, "L", dt), _ptr(R, "R", dt), fp,
                                   _ptr(dx, "dx", dt), _ptr(dL, "dL", f32), _ptr(dR, "dR", f32), int(accumulate),
                                   tokens, q, b1, b, r, _dtype_code(x), p, nb, _stream(stream)), "monarch_rect_bwd")
+
+
+def monarch_rectw_workspace_bytes(tokens: int, q: int, b1: int, b2: int, b3: int, r: int, dtype: int) -> int:
+    return int(lib().monarch_rectw_workspace_bytes(tokens, q, b1, b2, b3, r, dtype))
+
+
+def monarch_rectw_bwd_workspace_bytes(tokens: int, q: int, b1: int, b2: int, b3: int, r: int, dtype: int) -> int:
+    return int(lib().monarch_rectw_bwd_workspace_bytes(tokens, q, b1, b2, b3, r, dtype))
+
+
+def monarch_rectw_fwd(x, L, R, y, tokens, q, b1, b2, b3, r, workspace, stream=None) -> None:
+    """y = L R x for the rectangular class with wrapped-diagonal blocks: R [q, b2, b1], L [r, q, max(b2, b3)]."""
+    dt = x.dtype
+    p, nb = _ws(workspace)
+    _check(lib().monarch_rectw_fwd(_ptr(x, "x"), _ptr(L, "L", dt), _ptr(R, "R", dt), _ptr(y, "y", dt), tokens, q, b1, b2,
+                                   b3, r, _dtype_code(x), p, nb, _stream(stream)), "monarch_rectw_fwd")
+
+
+def monarch_rectw_bwd(x, dy, L, R, dx, dL, dR, accumulate, tokens, q, b1, b2, b3, r, workspace, stream=None) -> None:
+    """Gradients of <dy, L R x> for the wrapped-diagonal class: dx like x; dL like L and dR like R, in float32."""
+    import torch
+    dt, f32 = x.dtype, torch.float32
+    p, nb = _ws(workspace)
+    _check(lib().monarch_rectw_bwd(_ptr(x, "x"), _ptr(dy, "dy", dt), _ptr(L, "L", dt), _ptr(R, "R", dt),
+                                   _ptr(dx, "dx", dt), _ptr(dL, "dL", f32), _ptr(dR, "dR", f32), int(accumulate),
+                                   tokens, q, b1, b2, b3, r, _dtype_code(x), p, nb, _stream(stream)), "monarch_rectw_bwd")
 
 
 NOALLOC_SCRATCH_BYTES = 8 << 20

@@ -224,6 +224,14 @@ bool rect_stage2_stream_available(int q, int b, int r, int dtype);
 int rect_stage2_stream(const void *u, const void *Lp, void *y, int64_t tokens, int q, int b, int r, int wt,
                        unsigned *status, cudaStream_t s);
 
+// ---- rectangular class with wrapped-diagonal blocks, b2 != b3 (rect_wrapped.cu) ----
+size_t rectw_workspace_bytes(int64_t tokens, int q, int b2, int b3, int r, int dtype);
+size_t rectw_bwd_workspace_bytes(int64_t tokens, int q, int b2, int b3, int r, int dtype);
+int rectw_fwd(const void *x, const void *Lw, const void *R, void *y, int64_t tokens, int q, int b1, int b2, int b3, int r,
+              int dtype, bool fast, void *ws, cudaStream_t s);
+int rectw_bwd(const void *x, const void *dy, const void *Lw, const void *R, void *dx, float *dLw, float *dR, int accumulate,
+              int64_t tokens, int q, int b1, int b2, int b3, int r, int dtype, bool fast, void *ws, cudaStream_t s);
+
 // ---- dense <-> Monarch factors (project.cu): Eq. (2) and Algorithm 1 ----
 int dense_from_factors(const void *L, const void *R, void *M, int m, int dtype, cudaStream_t s);
 int project_to_factors(const void *A, void *L, void *R, int m, int dtype, unsigned long long *rotations, cudaStream_t s);

@@ -379,6 +379,48 @@ int monarch_rect_fwd(const void *x, const void *L, const void *R, void *y, int64
     return rect_stage2_simt(u, L, y, tokens, q, b, r, dtype, 0, s);
 }
 
+size_t monarch_rectw_workspace_bytes(int64_t tokens, int32_t q, int32_t b1, int32_t b2, int32_t b3, int32_t r, int dtype)
+{
+    if (check_rect(tokens, q, b1, b2, 1, dtype) != MONARCH_OK || check_rect(tokens, q, 1, b3, r, dtype) != MONARCH_OK) return 0;
+    return rectw_workspace_bytes(tokens, q, b2, b3, r, dtype);
+}
+
+size_t monarch_rectw_bwd_workspace_bytes(int64_t tokens, int32_t q, int32_t b1, int32_t b2, int32_t b3, int32_t r, int dtype)
+{
+    if (check_rect(tokens, q, b1, b2, 1, dtype) != MONARCH_OK || check_rect(tokens, q, 1, b3, r, dtype) != MONARCH_OK) return 0;
+    return rectw_bwd_workspace_bytes(tokens, q, b2, b3, r, dtype);
+}
+
+int monarch_rectw_fwd(const void *x, const void *L, const void *R, void *y, int64_t tokens, int32_t q, int32_t b1,
+                      int32_t b2, int32_t b3, int32_t r, int dtype, void *workspace, size_t workspace_bytes, void *stream)
+{
+    MONARCH_TRY(check_rect(tokens, q, b1, b2, 1, dtype));
+    MONARCH_TRY(check_rect(tokens, q, 1, b3, r, dtype));
+    const size_t es = esize(dtype), bmax = b2 > b3 ? b2 : b3;
+    const Range in[] = {{x, (size_t)tokens * q * b1 * es}, {L, (size_t)r * q * bmax * es}, {R, (size_t)q * b2 * b1 * es}};
+    const Range out[] = {{y, (size_t)tokens * r * b3 * es}};
+    MONARCH_TRY(check_buffers(in, 3, out, 1, workspace, workspace_bytes, rectw_workspace_bytes(tokens, q, b2, b3, r, dtype)));
+    const bool fast = g_impl.load(std::memory_order_relaxed) != MONARCH_IMPL_STAGED;
+    return rectw_fwd(x, L, R, y, tokens, q, b1, b2, b3, r, dtype, fast, workspace, (cudaStream_t)stream);
+}
+
+int monarch_rectw_bwd(const void *x, const void *dy, const void *L, const void *R, void *dx, float *dL, float *dR,
+                      int accumulate, int64_t tokens, int32_t q, int32_t b1, int32_t b2, int32_t b3, int32_t r, int dtype,
+                      void *workspace, size_t workspace_bytes, void *stream)
+{
+    MONARCH_TRY(check_rect(tokens, q, b1, b2, 1, dtype));
+    MONARCH_TRY(check_rect(tokens, q, 1, b3, r, dtype));
+    if (accumulate != 0 && accumulate != 1) return MONARCH_ERR_INVALID_ARG;
+    const size_t es = esize(dtype), bmax = b2 > b3 ? b2 : b3;
+    const size_t lb = (size_t)r * q * bmax, rb = (size_t)q * b2 * b1;
+    const Range in[] = {{x, (size_t)tokens * q * b1 * es}, {dy, (size_t)tokens * r * b3 * es}, {L, lb * es}, {R, rb * es}};
+    const Range out[] = {{dx, (size_t)tokens * q * b1 * es}, {dL, lb * sizeof(float)}, {dR, rb * sizeof(float)}};
+    MONARCH_TRY(check_buffers(in, 4, out, 3, workspace, workspace_bytes,
+                              rectw_bwd_workspace_bytes(tokens, q, b2, b3, r, dtype)));
+    const bool fast = g_impl.load(std::memory_order_relaxed) != MONARCH_IMPL_STAGED;
+    return rectw_bwd(x, dy, L, R, dx, dL, dR, accumulate, tokens, q, b1, b2, b3, r, dtype, fast, workspace, (cudaStream_t)stream);
+}
+
 size_t monarch_rect_bwd_workspace_bytes(int64_t tokens, int32_t q, int32_t b1, int32_t b, int32_t r, int dtype)
 {
     if (check_rect(tokens, q, b1, b, r, dtype) != MONARCH_OK) return 0;

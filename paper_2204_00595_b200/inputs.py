@@ -132,6 +132,32 @@ def make_rect_inputs(tokens: int | None = None, seed: int = 595006, **sizes) -> 
     return out
 
 
+# The same class with wrapped-diagonal blocks (b2 != b3): R has q blocks of b2 x b1, L an r x q grid of b3 x b2 blocks
+# with max(b2, b3) stored entries each.  One measured case beside the diagonal one: the same 4096 x 4096 product with
+# blocks of L twice as tall as wide.
+RECTW_WORKLOAD = {"q": 4, "b1": 1024, "b2": 1024, "b3": 2048, "r": 2, "tokens": 8192, "dtype": "bf16"}
+
+
+def make_rectw_inputs(tokens: int | None = None, seed: int = 595009, **sizes) -> dict:
+    """Seeded tensors x [T, q*b1], R [q, b2, b1], L [r, q, max(b2, b3)] of the wrapped-diagonal class (weights scaled
+    so that u and y keep unit variance), rounded to the storage dtype."""
+    cfg = dict(RECTW_WORKLOAD)
+    cfg.update(sizes)
+    if tokens is not None:
+        cfg["tokens"] = int(tokens)
+    q, b1, b2, b3, r, T, dt = cfg["q"], cfg["b1"], cfg["b2"], cfg["b3"], cfg["r"], cfg["tokens"], cfg["dtype"]
+    rng = np.random.default_rng(seed)
+
+    def draw(shape, std):
+        return round_to_storage(rng.standard_normal(shape, dtype=np.float32) * np.float32(std), dt)
+
+    out = dict(cfg)
+    out["x"] = draw((T, q * b1), 1.0)
+    out["R"] = draw((q, b2, b1), 1.0 / math.sqrt(b1))
+    out["L"] = draw((r, q, max(b2, b3)), 1.0 / math.sqrt(q * max(1, b2 // b3)))
+    return out
+
+
 def to_device(a: np.ndarray, dtype: str):
     """float32 numpy array (already rounded to the storage dtype) -> torch CUDA tensor, exactly."""
     import torch

@@ -557,6 +557,83 @@ def test_rect_bwd(P, q, b1, b, r, T, dtype):
     assert_close(_instances(to_host64(dR)), _instances(2 * ref["dR"]), dtype, "rect dR accumulate")
 
 
+# (q, b1, b2, b3, r, T): b3 a multiple of b2, b2 a multiple of b3, neither; tiny, ragged and tensor-core sizes
+RECTW_CASES = [
+    (3, 2, 2, 4, 2, 7), (2, 3, 4, 2, 3, 65), (2, 2, 3, 5, 2, 130), (3, 1, 5, 3, 2, 70), (2, 4, 2, 6, 1, 33),
+    (4, 64, 64, 256, 2, 257), (4, 128, 512, 256, 4, 300), (3, 20, 17, 34, 6, 129), (5, 24, 40, 8, 3, 200),
+    (4, 64, 96, 160, 2, 140), (2, 48, 80, 48, 5, 90), (4, 256, 256, 256, 4, 200), (4, 1024, 512, 1024, 2, 150),
+    (4, 64, 1024, 256, 3, 131),
+]
+
+
+def _rectw_inputs(q, b1, b2, b3, r, T, dtype, seed):
+    rng = np.random.default_rng(seed)
+
+    def draw(shape, std):
+        return round_to_storage(rng.standard_normal(shape, dtype=np.float32) * np.float32(std), dtype)
+
+    terms = q * max(1, b2 // b3)                          # entries that meet in one output element
+    return {"x": draw((T, q * b1), 1.0), "R": draw((q, b2, b1), 1.0 / np.sqrt(b1)),
+            "L": draw((r, q, max(b2, b3)), 1.0 / np.sqrt(terms)), "dy": draw((T, r * b3), 1.0)}
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("q,b1,b2,b3,r,T", RECTW_CASES)
+def test_rect_wrapped_fwd_bwd(P, q, b1, b2, b3, r, T, dtype):
+    """The rectangular class with wrapped-diagonal blocks (b2 != b3): forward, then dx, dL, dR (overwrite, then
+    accumulate) against the oracle, over sizes that take the re-labelled fast path in both directions and sizes that
+    take the general kernels."""
+    import torch
+    code = _code(P, dtype)
+    if dtype == "bf16" and min(q * b1, r * b3) < 64:
+        pytest.skip("token rows of fewer than 64 elements make the normwise bf16 comparison a componentwise one; "
+                    "these index-arithmetic cases run in fp32, at 1e-5")
+    d = _rectw_inputs(q, b1, b2, b3, r, T, dtype, seed=11 + q * 1000003 + b1 * 1009 + b2 * 31 + b3)
+    x, dy, L, R = (to_device(d[k], dtype) for k in ("x", "dy", "L", "R"))
+    bmax = max(b2, b3)
+    yf, y = _guarded((T, r * b3), _tdtype(dtype))
+    ws = P.Workspace(P.monarch_rectw_workspace_bytes(T, q, b1, b2, b3, r, code))
+    P.monarch_rectw_fwd(x, L, R, y, T, q, b1, b2, b3, r, ws)
+    torch.cuda.synchronize()
+    assert P.monarch_last_device_status(ws) == 0
+    assert_close(to_host64(y), O.rectw_fwd(d["x"], d["L"], d["R"], b3), dtype, "wrapped y")
+    _check_guard(yf, "wrapped y")
+    dxf, dx = _guarded((T, q * b1), _tdtype(dtype))
+    dLf, dL = _guarded((r, q, bmax), torch.float32)
+    dRf, dR = _guarded((q, b2, b1), torch.float32)
+    wsb = P.Workspace(P.monarch_rectw_bwd_workspace_bytes(T, q, b1, b2, b3, r, code))
+    P.monarch_rectw_bwd(x, dy, L, R, dx, dL, dR, 0, T, q, b1, b2, b3, r, wsb)
+    torch.cuda.synchronize()
+    assert P.monarch_last_device_status(wsb) == 0
+    ref = O.rectw_bwd(d["x"], d["dy"], d["L"], d["R"], b3)
+    assert_close(to_host64(dx), ref["dx"], dtype, "wrapped dx")
+    # a block of L has max(b2, b3) entries; all of dL is one instance when that is small (reading S13)
+    assert_close(_instances(to_host64(dL).reshape(r * q, bmax)), _instances(ref["dL"].reshape(r * q, bmax)), dtype, "wrapped dL")
+    assert_close(_instances(to_host64(dR)), _instances(ref["dR"]), dtype, "wrapped dR")
+    for flat, what in ((dxf, "dx"), (dLf, "dL"), (dRf, "dR")):
+        _check_guard(flat, f"wrapped {what}")
+    P.monarch_rectw_bwd(x, dy, L, R, dx, dL, dR, 1, T, q, b1, b2, b3, r, wsb)
+    torch.cuda.synchronize()
+    assert_close(_instances(to_host64(dL).reshape(r * q, bmax)), _instances(2 * ref["dL"].reshape(r * q, bmax)), dtype,
+                 "wrapped dL accumulate")
+    assert_close(_instances(to_host64(dR)), _instances(2 * ref["dR"]), dtype, "wrapped dR accumulate")
+
+
+def test_rect_wrapped_equal_sizes_is_the_diagonal_case(P):
+    """b2 = b3: the wrapped call equals monarch_rect_fwd on the transposed weight layout, bit for bit."""
+    import torch
+    q, b1, b, r, T, dtype = 4, 128, 256, 3, 300, "bf16"
+    d = _rectw_inputs(q, b1, b, b, r, T, dtype, seed=99)
+    x, L, R = (to_device(d[k], dtype) for k in ("x", "L", "R"))
+    Lp = L.permute(2, 0, 1).contiguous()
+    y1 = torch.empty(T, r * b, dtype=torch.bfloat16, device="cuda")
+    y2 = torch.empty_like(y1)
+    P.monarch_rectw_fwd(x, L, R, y1, T, q, b1, b, b, r, P.Workspace(P.monarch_rectw_workspace_bytes(T, q, b1, b, b, r, P.BF16)))
+    P.monarch_rect_fwd(x, Lp, R, y2, T, q, b1, b, r, P.Workspace(P.monarch_rect_workspace_bytes(T, q, b1, b, r, P.BF16)))
+    torch.cuda.synchronize()
+    assert torch.equal(y1, y2)
+
+
 def test_rect_square_case_equals_monarch_fwd(P):
     """q = b1 = b = r = m is Definition 3.1: both entry points see the same tensors."""
     import torch
@@ -572,6 +649,42 @@ def test_rect_square_case_equals_monarch_fwd(P):
     torch.cuda.synchronize()
     assert_close(to_host64(y2), to_host64(y1), "f32", "rect vs square")
     assert_close(to_host64(y2), O.fwd(d["x"], d["L"], d["R"]), "f32", "rect vs oracle")
+
+
+def test_workload_rect_wrapped(P):
+    """The measured case of the wrapped-diagonal class (workload 9: R four 1024 x 1024 blocks, L a 2 x 4 grid of
+    2048 x 1024 wrapped diagonals, 8192 tokens) at full size, in the configuration the benchmark times: both edge rows
+    and a random interior row of every 64-token tile against the oracle, finiteness of the whole output, and the
+    adjoint identity <dy, y> = <dx, x> with the Euler identities <dL, L> = <dR, R> = <dy, y> on the device results."""
+    import torch
+    from paper_2204_00595_b200.inputs import make_rectw_inputs
+    d = make_rectw_inputs()
+    q, b1, b2, b3, r, T = d["q"], d["b1"], d["b2"], d["b3"], d["r"], d["tokens"]
+    x, L, R = (to_device(d[k], "bf16") for k in ("x", "L", "R"))
+    y = torch.full((T, r * b3), float("nan"), dtype=torch.bfloat16, device="cuda")
+    ws = P.Workspace(P.monarch_rectw_workspace_bytes(T, q, b1, b2, b3, r, P.BF16))
+    P.monarch_rectw_fwd(x, L, R, y, T, q, b1, b2, b3, r, ws)
+    torch.cuda.synchronize()
+    assert P.monarch_last_device_status(ws) == 0
+    assert bool(torch.isfinite(y.float()).all())
+    rows = _tile_rows(T, 9)
+    ref = O.rectw_fwd(d["x"][rows], d["L"], d["R"], b3)
+    assert_close(to_host64(y[torch.from_numpy(rows).cuda()]), ref, "bf16", "wrapped workload y")
+    dy = torch.randn(T, r * b3, device="cuda", generator=torch.Generator("cuda").manual_seed(9)).bfloat16()
+    dx = torch.empty_like(x)
+    dL = torch.empty(L.shape, dtype=torch.float32, device="cuda")
+    dR = torch.empty(R.shape, dtype=torch.float32, device="cuda")
+    wsb = P.Workspace(P.monarch_rectw_bwd_workspace_bytes(T, q, b1, b2, b3, r, P.BF16))
+    P.monarch_rectw_bwd(x, dy, L, R, dx, dL, dR, 0, T, q, b1, b2, b3, r, wsb)
+    torch.cuda.synchronize()
+    assert P.monarch_last_device_status(wsb) == 0
+    refb = O.rectw_bwd(d["x"][rows], to_host64(dy)[rows], d["L"], d["R"], b3)
+    assert_close(to_host64(dx[torch.from_numpy(rows).cuda()]), refb["dx"], "bf16", "wrapped workload dx")
+    dot = lambda a, b: float((a.double() * b.double()).sum())
+    # sums of T*r*b3 products of unit-variance factors: the identities hold to the bf16 rounding of y, dx and u
+    s_y, tol = dot(dy, y), 2e-2 * float(np.sqrt(T * r * b3))
+    for what, v in (("<dx, x>", dot(dx, x)), ("<dL, L>", dot(dL, L)), ("<dR, R>", dot(dR, R))):
+        assert abs(v - s_y) <= tol, (what, v, s_y)
 
 
 def test_workload_rect(P, impl):
