@@ -361,7 +361,8 @@ def main_rect(args):
     total_ms = t_start.elapsed_time(t_stop)
     clocks = sampler.stop()
     launches = P.monarch_launch_count() - launches0
-    status = P.monarch_last_device_status(ws)
+    # a wait that ran out in any kernel of the timed region shows in the status word of the workspace it used
+    status = P.monarch_last_device_status(ws) | (P.monarch_last_device_status(ws_b) if with_bwd else 0)
     if dist is not None:
         tmax = torch.tensor([total_ms], device="cuda")
         dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
@@ -390,6 +391,8 @@ def main_rect(args):
                      "hbm_time_ms": nbytes / (peaks["hbm_gbs"] * 1e9) * 1e3},
         "e2e": None,
     }
+    if status != 0:
+        line["invalid"] = "a device-side wait ran out inside the timed region"
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         rr = time_oracle_rect(d, 12.0)
         line["cpu_baseline"] = {"value": rr["tflops"], "unit": unit, "cores": rr["cores"], "kind": "oracle",
