@@ -1106,3 +1106,77 @@ print("ok")
     env = dict(os.environ, MONARCH_M64_CLUSTER="1")
     out = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=600)
     assert out.returncode == 0 and "ok" in out.stdout, out.stderr[-2000:]
+
+
+# ----------------------------------------------------------------- m = 128: the three-launch forward, and run-to-run bits
+
+@pytest.mark.parametrize("T", [1, 130, 700])
+def test_fwd_m128_as_three_launches(T):
+    """The forward of the m = 128 chain in its three-launch form (what a device too small for the persistent launch,
+    or a batch of more than 8192 tiles, gets; selected by an environment variable read once per process, hence the
+    child process), and the backward reading the u' that form left behind, against the oracle."""
+    import os
+    import subprocess
+    import sys
+    code = f"""
+import sys, numpy as np, torch
+sys.path.insert(0, {os.path.dirname(os.path.dirname(os.path.abspath(__file__)))!r})
+import paper_2204_00595_b200 as P
+from oracle import monarch_oracle as O
+from paper_2204_00595_b200.inputs import round_to_storage, to_device, to_host64
+from tests.helpers import assert_close
+m, n, T = 128, 16384, {T}
+rng = np.random.default_rng(12800 + T)
+draw = lambda shape, std: round_to_storage(rng.standard_normal(shape, dtype=np.float32) * np.float32(std), "bf16")
+hx, hdy, hL, hR = draw((T, n), 1.0), draw((T, n), 1.0), draw((m, m, m), 0.088), draw((m, m, m), 0.088)
+x, dy, L, R = (to_device(a, "bf16") for a in (hx, hdy, hL, hR))
+y = torch.full_like(x, float("nan")); dx = torch.full_like(x, float("nan"))
+dL = torch.full((m, m, m), float("nan"), device="cuda"); dR = torch.full((m, m, m), float("nan"), device="cuda")
+ws = P.Workspace(P.monarch_workspace_bytes(P.OP_FWD, T, n, m, P.BF16))
+wsb = P.Workspace(P.monarch_workspace_bytes(P.OP_BWD, T, n, m, P.BF16))
+n0 = P.monarch_launch_count()
+P.monarch_fwd(x, L, R, y, T, n, m, ws)
+assert P.monarch_launch_count() - n0 == 3
+P.monarch_bwd(x, dy, L, R, dx, dL, dR, 0, T, n, m, wsb, fwd_workspace=ws)
+torch.cuda.synchronize()
+assert P.monarch_last_device_status(ws) == 0 and P.monarch_last_device_status(wsb) == 0
+ref = O.bwd(hx, hdy, hL, hR)
+assert_close(to_host64(y), O.fwd(hx, hL, hR), "bf16", "y, three launches")
+assert_close(to_host64(dx), ref["dx"], "bf16", "dx")
+assert_close(to_host64(dL), ref["dL"], "bf16", "dL")
+assert_close(to_host64(dR), ref["dR"], "bf16", "dR")
+print("ok")
+"""
+    env = dict(os.environ, MONARCH_CHAIN_SPLIT="1")
+    out = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0 and "ok" in out.stdout, out.stderr[-2000:]
+
+
+def test_m128_weight_gradients_have_the_same_bits_every_run(P):
+    """bf16 m = 128: one thread block sums all tokens of a weight block in a fixed order, so dL and dR do not depend on
+    timing - three runs from different initial contents (overwrite mode), with and without the saved u', agree bit
+    for bit; accumulate = 1 from equal contents does too."""
+    import torch
+    m, T, dtype = 128, 700, "bf16"
+    n = m * m
+    d = _small_inputs(m, T, dtype, seed=128700)
+    x, dy, L, R = (to_device(d[k], dtype) for k in ("x", "dy", "L", "R"))
+    y = torch.empty_like(x)
+    dx = torch.empty_like(x)
+    ws_f = P.Workspace(P.monarch_workspace_bytes(P.OP_FWD, T, n, m, P.BF16))
+    ws_b = P.Workspace(P.monarch_workspace_bytes(P.OP_BWD, T, n, m, P.BF16))
+    P.monarch_fwd(x, L, R, y, T, n, m, ws_f)
+    runs = []
+    for fill, saved, acc in ((float("nan"), True, 0), (3.0, False, 0), (-1.0, True, 0), (0.5, True, 1), (0.5, False, 1)):
+        dL = torch.full((m, m, m), fill, device="cuda")
+        dR = torch.full((m, m, m), fill, device="cuda")
+        P.monarch_bwd(x, dy, L, R, dx, dL, dR, acc, T, n, m, ws_b, fwd_workspace=ws_f if saved else None)
+        torch.cuda.synchronize()
+        assert P.monarch_last_device_status(ws_b) == 0
+        runs.append((dL, dR))
+    for k in (1, 2):
+        assert torch.equal(runs[k][0], runs[0][0]) and torch.equal(runs[k][1], runs[0][1])
+    assert torch.equal(runs[3][0], runs[4][0]) and torch.equal(runs[3][1], runs[4][1])
+    ref = O.bwd(d["x"], d["dy"], d["L"], d["R"])
+    assert_close(to_host64(runs[0][0]), ref["dL"], dtype, "dL")
+    assert_close(to_host64(runs[3][1] - 0.5), ref["dR"], dtype, "dR accumulated onto 0.5")
