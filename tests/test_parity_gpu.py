@@ -1180,3 +1180,35 @@ def test_m128_weight_gradients_have_the_same_bits_every_run(P):
     ref = O.bwd(d["x"], d["dy"], d["L"], d["R"])
     assert_close(to_host64(runs[0][0]), ref["dL"], dtype, "dL")
     assert_close(to_host64(runs[3][1] - 0.5), ref["dR"], dtype, "dR accumulated onto 0.5")
+
+
+def test_zero_tokens_m128_and_wrapped(P):
+    """An empty batch: outputs untouched, weight gradients zeroed (overwrite) or left alone (accumulate)."""
+    import torch
+    m = 128
+    n = m * m
+    x = torch.zeros(1, n, dtype=torch.bfloat16, device="cuda")
+    W = torch.zeros(m, m, m, dtype=torch.bfloat16, device="cuda")
+    y = torch.full((1, n), 3.0, dtype=torch.bfloat16, device="cuda")
+    g = torch.full((2, m, m, m), 5.0, dtype=torch.float32, device="cuda")
+    ws = P.Workspace(max(P.monarch_workspace_bytes(P.OP_FWD, 0, n, m, P.BF16), 256))
+    wsb = P.Workspace(max(P.monarch_workspace_bytes(P.OP_BWD, 0, n, m, P.BF16), 256))
+    P.monarch_fwd(x, W, W.clone(), y, 0, n, m, ws)
+    P.monarch_bwd(x, x.clone(), W, W.clone(), y.clone(), g[0], g[1], 1, 0, n, m, wsb)
+    torch.cuda.synchronize()
+    assert float(y.float().min()) == 3.0 and float(g.min()) == 5.0
+    P.monarch_bwd(x, x.clone(), W, W.clone(), y.clone(), g[0], g[1], 0, 0, n, m, wsb)
+    torch.cuda.synchronize()
+    assert float(g.abs().max()) == 0.0
+    q, b1, b2, b3, r = 2, 8, 4, 8, 3
+    xr = torch.zeros(1, q * b1, device="cuda")
+    R = torch.zeros(q, b2, b1, device="cuda")
+    L = torch.zeros(r, q, max(b2, b3), device="cuda")
+    yr = torch.full((1, r * b3), 3.0, device="cuda")
+    gL, gR = torch.full(L.shape, 5.0, device="cuda"), torch.full(R.shape, 5.0, device="cuda")
+    w1 = P.Workspace(max(P.monarch_rectw_workspace_bytes(0, q, b1, b2, b3, r, P.F32), 256))
+    w2 = P.Workspace(max(P.monarch_rectw_bwd_workspace_bytes(0, q, b1, b2, b3, r, P.F32), 256))
+    P.monarch_rectw_fwd(xr, L, R, yr, 0, q, b1, b2, b3, r, w1)
+    P.monarch_rectw_bwd(xr, yr.clone(), L, R, xr.clone(), gL, gR, 0, 0, q, b1, b2, b3, r, w2)
+    torch.cuda.synchronize()
+    assert float(yr.min()) == 3.0 and float(gL.abs().max()) == 0.0 and float(gR.abs().max()) == 0.0
