@@ -94,6 +94,29 @@ __device__ __forceinline__ void bulk_load_linear(uint32_t dst, const void *src, 
                  : "memory");
 }
 
+// Data with no further use in this launch (an intermediate's slab at its one read, the input, the output) is marked
+// evict-first in L2, so that it does not push out the rows that are read back a few steps after they were written.
+__device__ __forceinline__ uint64_t l2_evict_first_policy()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void tma_load_2d_last_use(uint32_t dst, const CUtensorMap *m, int x, int y, uint32_t bar, uint64_t pol)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%3, %4}], [%2], %5;" ::"r"(dst),
+        "l"(m), "r"(bar), "r"(x), "r"(y), "l"(pol)
+        : "memory");
+}
+__device__ __forceinline__ void bulk_load_linear_last_use(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar, uint64_t pol)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar), "l"(pol)
+                 : "memory");
+}
+
 // Load one 128 x 128 operand of block `blk`, tile `tile`: two 64-column boxes of a token-major tensor, or the
 // consumer slab [tile][blk] of an intermediate (already the swizzled image).
 template <int KIND>
@@ -613,11 +636,12 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
             // the u' slabs of stage 2 go through ring slot 1; the x tiles have their own loader and slot 0, so that a wait
             // for the other CTAs here never holds back this CTA's own stage 1 (whose rows the others are waiting for)
             [[maybe_unused]] long long wc = 0, wb = 0;
+            const uint64_t pol = l2_evict_first_policy();
             for (int tb = 0; tb < nt; ++tb) {
                 { FT0(); if (!wait_counter(p.cnt1 + tb, 2 * kB, kB, p.status, dead)) break; FACC(wc); }
                 { FT0(); if (!mbar_wait(empty0 + 8, (tb & 1) ^ 1, p.status, dead, kErrSlotWait)) break; FACC(wb); }
                 mbar_expect_tx(full0 + 8, kOpBytes);
-                load_operand<kLdC>(ring0 + kOpBytes, nullptr, p.u, b, tb, full0 + 8);
+                bulk_load_linear_last_use(ring0 + kOpBytes, p.u + ((size_t)tb * kB + b) * kOpBytes, kOpBytes, full0 + 8, pol);
             }
             FOUT(1, wc); FOUT(2, wb);
         }
@@ -625,11 +649,13 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
         // ------------------------------------------------------------ x loader (ring slot 0)
         if (lane == 0) {
             pdl_wait();
+            const uint64_t pol = l2_evict_first_policy();
             [[maybe_unused]] long long wa = 0;
             for (int s = 0; s < nt; ++s) {
                 { FT0(); if (!mbar_wait(empty0, (s & 1) ^ 1, p.status, dead, kErrSlotWait)) break; FACC(wa); }
                 mbar_expect_tx(full0, kOpBytes);
-                load_operand<kLdX>(ring0, &tm_x, nullptr, b, s, full0);
+                tma_load_2d_last_use(ring0, &tm_x, b * kB, s * 128, full0, pol);
+                tma_load_2d_last_use(ring0 + kHalfBytes, &tm_x, b * kB + 64, s * 128, full0, pol);
                 *reinterpret_cast<volatile int *>(&x_prog_s) = s + 1;
             }
             FOUT(0, wa);
@@ -783,12 +809,13 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
         if (lane == 0) {
             uint32_t c = 0;
             [[maybe_unused]] long long wc = 0, we = 0;
+            const uint64_t pol = l2_evict_first_policy();
             for (int s = 2 * kFusedLag; s < nsteps; ++s, ++c) {
                 const int tc = s - 2 * kFusedLag;
                 { FT0(); if (!wait_counter(p.cnt2 + tc, 2 * kB, kB, p.status, dead)) break; FACC(wc); }
                 { FT0(); if (!mbar_wait(tre, (c & 1) ^ 1, p.status, dead, kErrSlotWait)) break; FACC(we); }
                 mbar_expect_tx(trf, kOpBytes);
-                load_operand<kLdC>(trin, nullptr, p.w, b, tc % kFusedRing, trf);
+                bulk_load_linear_last_use(trin, p.w + ((size_t)(tc % kFusedRing) * kB + b) * kOpBytes, kOpBytes, trf, pol);
             }
             FOUT(10, wc); FOUT(11, we);
         }
@@ -838,7 +865,8 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
                 for (int i = 0; i < 8; ++i) {
                     const int t = tw * 32 + i * 4 + (lane >> 3);
                     if ((long long)tile * 128 + t < p.tokens)
-                        *reinterpret_cast<uint4 *>(yrow + (size_t)t * kOpBytes + hh * 128) = v[i];
+                        asm volatile("st.global.cs.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(yrow + (size_t)t * kOpBytes + hh * 128),
+                                     "r"(v[i].x), "r"(v[i].y), "r"(v[i].z), "r"(v[i].w) : "memory");
                 }
             }
         }
