@@ -129,6 +129,18 @@ __device__ __forceinline__ void load_operand(uint32_t dst, const CUtensorMap *m,
         bulk_load_linear(dst, base + ((size_t)tile * kB + blk) * kOpBytes, kOpBytes, bar);
     }
 }
+// the same for an operand that is not read again by this launch or the next ones of the chain
+template <int KIND>
+__device__ __forceinline__ void load_operand_last_use(uint32_t dst, const CUtensorMap *m, const char *base, int blk, int tile,
+                                                      uint32_t bar, uint64_t pol)
+{
+    if (KIND == kLdX) {
+        tma_load_2d_last_use(dst, m, blk * kB, tile * 128, bar, pol);
+        tma_load_2d_last_use(dst + kHalfBytes, m, blk * kB + 64, tile * 128, bar, pol);
+    } else {
+        bulk_load_linear_last_use(dst, base + ((size_t)tile * kB + blk) * kOpBytes, kOpBytes, bar, pol);
+    }
+}
 
 // Descriptor of K-step s (16 of the contraction index) of an operand tile: with the contraction index along the
 // 128-byte rows (K-major: four steps per box) or down the rows (MN-major: 16 rows = 2 KB per step, the two boxes
@@ -211,6 +223,7 @@ chain_gemm_kernel(const __grid_constant__ CUtensorMap tm_t0, const __grid_consta
         if (lane == 0) {
             uint32_t n = 0, wcount = 0;
             int cur = -1;
+            const uint64_t pol = l2_evict_first_policy();
             for (long long i = i0; i < i1; ++i, ++n) {
                 const int blk = (int)(i / p.ntiles), tile = p.reverse ? p.ntiles - 1 - (int)(i % p.ntiles) : (int)(i % p.ntiles);
                 if (blk != cur) {
@@ -226,8 +239,8 @@ chain_gemm_kernel(const __grid_constant__ CUtensorMap tm_t0, const __grid_consta
                 const uint32_t s = n % SLOTS;
                 if (!mbar_wait(empty0 + s * 8, ((n / SLOTS) & 1) ^ 1, p.status, dead, kErrSlotWait)) break;
                 mbar_expect_tx(full0 + s * 8, kSlotBytes);
-                load_operand<T0_LD>(ring0 + s * kSlotBytes, &tm_t0, p.t0_base, blk, tile, full0 + s * 8);
-                if (WG) load_operand<T1_LD>(ring0 + s * kSlotBytes + kOpBytes, &tm_t1, p.t1_base, blk, tile, full0 + s * 8);
+                load_operand_last_use<T0_LD>(ring0 + s * kSlotBytes, &tm_t0, p.t0_base, blk, tile, full0 + s * 8, pol);
+                if (WG) load_operand_last_use<T1_LD>(ring0 + s * kSlotBytes + kOpBytes, &tm_t1, p.t1_base, blk, tile, full0 + s * 8, pol);
             }
         }
     } else if (warp == 5) {
@@ -416,6 +429,7 @@ plane_transpose_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_c
     if (warp == 4) {
         if (lane == 0) {
             uint32_t n = 0;
+            const uint64_t pol = l2_evict_first_policy();
             int last_fill[kTrIn];
 #pragma unroll
             for (int s = 0; s < kTrIn; ++s) last_fill[s] = -1;
@@ -425,7 +439,7 @@ plane_transpose_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_c
                 if (!mbar_wait(smem_u32(&empty[s]), ((n / kTrIn) & 1) ^ 1, p.status, dead, kErrSlotWait)) break;
                 if (i == p.skip_item) continue;
                 mbar_expect_tx(smem_u32(&full[s]), kOpBytes);
-                load_operand<TO_PLANES ? kLdX : kLdC>(in0 + s * kOpBytes, &tm_in, p.in_base, pl, tile, smem_u32(&full[s]));
+                load_operand_last_use<TO_PLANES ? kLdX : kLdC>(in0 + s * kOpBytes, &tm_in, p.in_base, pl, tile, smem_u32(&full[s]), pol);
                 last_fill[s] = (int)(n / kTrIn);
             }
             if (*dead) {
