@@ -51,7 +51,7 @@ bool chain_fused_enabled()
 constexpr int kB = 128;                      // block size m
 constexpr int kOpBytes = 32768;              // one 128 x 128 bf16 operand: two boxes of [128 rows][64 columns]
 constexpr int kHalfBytes = 16384;
-constexpr int kThreads = 6 * 32;             // warps 0-3 epilogue, 4 loader, 5 MMA
+constexpr int kThreads = 7 * 32;             // warps 0-3 epilogue, 4 loader, 5 MMA, 6 drops consumed slabs from L2
 constexpr int kStagingBytes = 2 * kHalfBytes;
 
 enum { kLdX = 0, kLdC = 1 };                 // token-major tensor (tiled TMA); consumer slab of an intermediate (linear)
@@ -66,6 +66,7 @@ struct ChainParams {
     int nblk;                                // blocks (128)
     int reverse;                             // walk the tiles from the last to the first: what the previous launch of
                                              // the chain wrote last is still in L2
+    int discard_t0;                          // the T0 slabs are dead once read (dw', du'; not u', which the backward call reads)
 };
 
 struct ChainBars {
@@ -115,6 +116,15 @@ __device__ __forceinline__ void bulk_load_linear_last_use(uint32_t dst, const vo
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst),
                  "l"(src), "r"(bytes), "r"(bar), "l"(pol)
                  : "memory");
+}
+
+// An intermediate's slab is read exactly once, by one CTA.  Once its copy has landed in shared memory the 256 lines are
+// dropped from L2 without a write-back (what is still dirty there would otherwise go to DRAM for nothing); the values
+// at those addresses are undefined until the next call writes them again.  One warp: 8 lines per lane.
+__device__ __forceinline__ void discard_slab(const char *slab, int lane)
+{
+#pragma unroll
+    for (int i = 0; i < 8; ++i) asm volatile("discard.global.L2 [%0], 128;" ::"l"(slab + (i * 32 + lane) * 128) : "memory");
 }
 
 // Load one 128 x 128 operand of block `blk`, tile `tile`: two 64-column boxes of a token-major tensor, or the
@@ -175,7 +185,7 @@ chain_gemm_kernel(const __grid_constant__ CUtensorMap tm_t0, const __grid_consta
     if (threadIdx.x == 0) {
         for (int s = 0; s < SLOTS; ++s) {
             mbar_init(smem_u32(&bars.full[s]), 1);
-            mbar_init(smem_u32(&bars.empty[s]), 1);
+            mbar_init(smem_u32(&bars.empty[s]), T0_LD == kLdC ? 2 : 1);      // the MMAs, and the warp that drops the slab
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&bars.acc_full[a]), 1);
@@ -243,6 +253,19 @@ chain_gemm_kernel(const __grid_constant__ CUtensorMap tm_t0, const __grid_consta
                 if (WG) load_operand_last_use<T1_LD>(ring0 + s * kSlotBytes + kOpBytes, &tm_t1, p.t1_base, blk, tile, full0 + s * 8, pol);
             }
         }
+    } else if (warp == 6) {
+        // ------------------------------------------------------------ the consumed slab of the intermediate leaves L2
+        if (T0_LD == kLdC) {
+            uint32_t n = 0;
+            for (long long i = i0; i < i1; ++i, ++n) {
+                const int blk = (int)(i / p.ntiles), tile = p.reverse ? p.ntiles - 1 - (int)(i % p.ntiles) : (int)(i % p.ntiles);
+                const uint32_t s = n % SLOTS;
+                if (!mbar_wait(full0 + s * 8, (n / SLOTS) & 1, p.status, dead, kErrTmaWait)) break;
+                if (p.discard_t0) discard_slab(p.t0_base + ((size_t)tile * kB + blk) * kOpBytes, lane);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty0 + s * 8);
+            }
+        }
     } else if (warp == 5) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
@@ -294,7 +317,7 @@ chain_gemm_kernel(const __grid_constant__ CUtensorMap tm_t0, const __grid_consta
                 }
             }
         }
-    } else {
+    } else if (warp < 4) {
         // ------------------------------------------------------------ epilogue (warps 0-3 = TMEM lanes 32w..32w+31)
         const int row = warp * 32 + lane;
         const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
@@ -942,7 +965,7 @@ struct Src {
 
 template <int T0_LD, bool W_IS_A, bool W_MN, bool T0_MN, int ST, bool WG, int T1_LD, bool T1_MN, bool MAIN>
 int launch_gemm(Src t0, Src t1, const CUtensorMap &w, const CUtensorMap &out, float *dW, int ntiles, unsigned *status, cudaStream_t s,
-                int overwrite = 0, int reverse = 0)
+                int overwrite = 0, int reverse = 0, int discard_t0 = 0)
 {
     constexpr int SLOTS = WG ? 2 : 3;
     constexpr int smem = 2 * kOpBytes + SLOTS * (WG ? 2 : 1) * kOpBytes + kStagingBytes + 1024;
@@ -955,6 +978,7 @@ int launch_gemm(Src t0, Src t1, const CUtensorMap &w, const CUtensorMap &out, fl
     p.dW = dW;
     p.overwrite = overwrite;
     p.reverse = reverse;
+    p.discard_t0 = discard_t0;
     p.t0_base = t0.base;
     p.t1_base = t1.base;
     p.ntiles = ntiles;
@@ -1107,18 +1131,19 @@ int chain_bwd_m128(const void *x, const void *dy, const void *L, const void *R, 
     // du'_k[j][t] = sum_l L[j][l][k] dw'_j[l][t] -> pieces of du' (row k to consumer k)   (+ dL[j][l][k] += sum_t dw'_j[l][t] u'_j[k][t])
     if (want_dw)
         MONARCH_TRY((launch_gemm<kLdC, true, true, true, kStP, true, kLdC, false, true>({nullptr, dwp}, {nullptr, up}, mL, mdu_st, dL, ntiles,
-                                                                                          status, s, !accumulate, 1)));
+                                                                                          status, s, !accumulate, 1, 1)));
     else
         MONARCH_TRY((launch_gemm<kLdC, true, true, true, kStP, false, kLdC, false, true>({nullptr, dwp}, {nullptr, nullptr}, mL, mdu_st, nullptr,
-                                                                                           ntiles, status, s, 0, 1)));
+                                                                                           ntiles, status, s, 0, 1, 1)));
     // dx[t][k*128+i] = sum_j du'_k[j][t] R[k][j][i]        (+ dR[k][j][i] += sum_t du'_k[j][t] x[t][k*128+i])
     if (want_dw && want_dx)
         return launch_gemm<kLdC, false, true, true, kStX, true, kLdX, true, true>({nullptr, dup}, {&mx, nullptr}, mR, mdx, dR, ntiles, status, s,
-                                                                                  !accumulate);
+                                                                                  !accumulate, 0, 1);
     if (want_dw)
         return launch_gemm<kLdC, false, true, true, kStX, true, kLdX, true, false>({nullptr, dup}, {&mx, nullptr}, mR, mdx, dR, ntiles, status, s,
-                                                                                   !accumulate);
-    return launch_gemm<kLdC, false, true, true, kStX, false, kLdX, true, true>({nullptr, dup}, {nullptr, nullptr}, mR, mdx, nullptr, ntiles, status, s);
+                                                                                   !accumulate, 0, 1);
+    return launch_gemm<kLdC, false, true, true, kStX, false, kLdX, true, true>({nullptr, dup}, {nullptr, nullptr}, mR, mdx, nullptr, ntiles, status, s,
+                                                                               0, 0, 1);
 }
 
 }  // namespace monarch
