@@ -227,10 +227,10 @@ NCU_TRAFFIC_MB = {
     (3, "bwd"): (364.0, _W3),
     (3, "bwd_dx"): (139.8, _W3),
     (3, "bwd_dw"): (408.3, _W3),
-    (4, "fwd"): (480.4, _W4),
-    (4, "bwd"): (948.0, _W4),
-    (4, "bwd_dx"): (649.0, _W4),
-    (4, "bwd_dw"): (1070.0, _W4),
+    (4, "fwd"): (460.8, _W4),
+    (4, "bwd"): (924.8, _W4),
+    (4, "bwd_dx"): (637.8, _W4),
+    (4, "bwd_dw"): (1055.3, _W4),
     (5, "mlp_fwd"): (1511.0, "profiles/mlp_fwd_workload5_ncu.md, full size, both passes"),
 }
 
