@@ -601,6 +601,7 @@ __device__ __forceinline__ bool wait_counter(unsigned *ctr, unsigned need, unsig
                 atomicCAS(status, 0u, (unsigned)kErrPeerWait);
                 return false;
             }
+            __nanosleep(64);                     // 128 CTAs poll this word; a hot loop only costs power
         }
     }
     if (atomicAdd(ctr, 1u) + 1 == need + consumers) atomicExch(ctr, 0u);
@@ -832,7 +833,7 @@ chain_fused_fwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
         for (int s = 0; s < nt; ++s) {
             if (s >= *x_prog + kFusedPrefetch) {
                 const unsigned long long t0 = global_timer_ns();
-                while (s >= *x_prog + kFusedPrefetch && !*dead && global_timer_ns() - t0 < limit) { }
+                while (s >= *x_prog + kFusedPrefetch && !*dead && global_timer_ns() - t0 < limit) __nanosleep(256);
                 if (s >= *x_prog + kFusedPrefetch) break;
             }
             const char *a = p.x + ((size_t)s * 128 + (lane >> 1)) * ((size_t)kB * kB * 2) + b * 256 + (lane & 1) * 128;
