@@ -111,6 +111,24 @@ __device__ __forceinline__ void tma_load_2d_last_use(uint32_t dst, const CUtenso
         "l"(m), "r"(bar), "r"(x), "r"(y), "l"(pol)
         : "memory");
 }
+__device__ __forceinline__ uint64_t l2_evict_last_policy()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void tma_store_5d_keep(const CUtensorMap *m, uint32_t src, int c0, int c1, int c2, int c3, int c4, uint64_t pol)
+{
+    asm volatile("cp.async.bulk.tensor.5d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3, %4, %5, %6}], [%1], %7;" ::"l"(m),
+                 "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "l"(pol)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_store_2d_stream(const CUtensorMap *m, uint32_t src, int x, int y, uint64_t pol)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;" ::"l"(m),
+                 "r"(src), "r"(x), "r"(y), "l"(pol)
+                 : "memory");
+}
 __device__ __forceinline__ void bulk_load_linear_last_use(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar, uint64_t pol)
 {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst),
@@ -360,8 +378,9 @@ chain_gemm_kernel(const __grid_constant__ CUtensorMap tm_t0, const __grid_consta
                     fence_proxy_async_smem();
                     asm volatile("bar.sync 1, 128;" ::: "memory");
                     if (threadIdx.x == 0) {
-                        if (ST == kStX) tma_store_2d(&tm_out, stg, blk * kB + h * 64, tile * 128);
-                        else tma_store_5d(&tm_out, stg, 0, blk, h, 0, tile);
+                        // a token-major output is final (written once, not read by this chain): evict-first
+                        if (ST == kStX) tma_store_2d_stream(&tm_out, stg, blk * kB + h * 64, tile * 128, l2_evict_first_policy());
+                        else tma_store_5d_keep(&tm_out, stg, 0, blk, h, 0, tile, l2_evict_last_policy());
                         tma_store_commit();
                     }
                 }
@@ -511,7 +530,7 @@ plane_transpose_kernel(const __grid_constant__ CUtensorMap tm_in, const __grid_c
             if (threadIdx.x == 0) {
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    if (TO_PLANES) tma_store_5d(&tm_out, ob + h * kHalfBytes, 0, pl, h, 0, tile);
+                    if (TO_PLANES) tma_store_5d_keep(&tm_out, ob + h * kHalfBytes, 0, pl, h, 0, tile, l2_evict_last_policy());
                     else tma_store_2d(&tm_out, ob + h * kHalfBytes, pl * kB + h * 64, tile * 128);
                 }
                 tma_store_commit();
