@@ -25,6 +25,11 @@
 // dR_k = du'_k x_k, which ride along in the same kernels with their accumulators resident in TMEM for all tiles of a
 // block (one writer per block: deterministic sums).
 //
+// L2 management: an intermediate (134 MB at 4096 tokens) is larger than what L2 keeps, and the backward launches are
+// bound by DRAM, so (i) every load of data that nothing reads again carries an evict-first policy, (ii) the pieces of an
+// intermediate are stored evict-last and the next launch walks the tiles in the opposite direction, (iii) a consumed
+// slab is dropped from L2 without a write-back (discard.global.L2) - dead dirty lines never reach DRAM.
+//
 // One kernel template serves all block products: persistent CTAs, the 32 KB weight block resident, token operands
 // through a TMA ring, tcgen05.mma 128 x 128 x 16 with two accumulator buffers in TMEM, epilogue through swizzled
 // staging tiles and TMA stores.
