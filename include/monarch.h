@@ -35,9 +35,9 @@
  *    monarch_workspace_init and read it with monarch_last_device_status.
  *    Calls that overlap on the GPU must not share a workspace.
  *  - Weight gradients of the fused tensor-core kernels (bf16, m = 64; the
- *    general class) are summed with fp32 reductions whose order across thread
- *    blocks is not fixed: dL, dR can differ in the last fp32 bits from run to
- *    run.  The bf16 m = 128 kernels (one thread block sums all tokens of a
+ *    general class) and of the staged tensor-core kernels (bf16, m = 32) are
+ *    summed with fp32 reductions whose order across thread blocks is not
+ *    fixed: dL, dR can differ in the last fp32 bits from run to run.  The bf16 m = 128 kernels (one thread block sums all tokens of a
  *    block, in a fixed order) and the CUDA-core family (MONARCH_IMPL_STAGED)
  *    give the same bits every run.
  *  - Return value: a monarch_status_t.  Nothing throws.
@@ -297,8 +297,9 @@ int monarch_set_impl(int impl);
  * more, and a device on which the one-launch backward cannot run gets
  * MONARCH_ERR_UNSUPPORTED instead of the multi-launch form.  on == 0 (default):
  * partial sums are added with fp32 atomics in whatever order they arrive.  Other
- * sizes and dtypes already sum in a fixed order or are not affected (the
- * feed-forward block and the general class keep their atomics).  Process-wide,
+ * sizes and dtypes already sum in a fixed order (bf16 m = 128, every fp32 call) or
+ * are not affected (bf16 m = 32, the feed-forward block and the general class keep
+ * their atomics).  Process-wide,
  * affects later calls and later workspace-size queries; not thread-safe against
  * concurrent calls.  Returns the previous setting. */
 int monarch_set_deterministic(int on);

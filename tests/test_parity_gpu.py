@@ -1182,6 +1182,37 @@ def test_m128_weight_gradients_have_the_same_bits_every_run(P):
     assert_close(to_host64(runs[3][1] - 0.5), ref["dR"], dtype, "dR accumulated onto 0.5")
 
 
+@pytest.mark.parametrize("m", [16, 32, 64])
+def test_fp32_weight_gradients_have_the_same_bits_every_run(P, m):
+    """fp32 runs on the CUDA-core family, whose token sums are taken slab by slab and added in slab order: dL and dR
+    from different initial contents (overwrite mode) agree bit for bit, through monarch_bwd and monarch_bwd_dw."""
+    import torch
+    T, dtype = 333, "f32"
+    n = m * m
+    d = _small_inputs(m, T, dtype, seed=3300 + m)
+    x, dy, L, R = (to_device(d[k], dtype) for k in ("x", "dy", "L", "R"))
+    dx = torch.empty_like(x)
+    ws = P.Workspace(max(P.monarch_workspace_bytes(P.OP_BWD, T, n, m, P.F32),
+                         P.monarch_workspace_bytes(P.OP_BWD_DW, T, n, m, P.F32)))
+    runs = []
+    for fill, one_call in ((float("nan"), True), (7.0, True), (-2.0, False), (0.25, False)):
+        dL = torch.full((m, m, m), fill, device="cuda")
+        dR = torch.full((m, m, m), fill, device="cuda")
+        if one_call:
+            P.monarch_bwd(x, dy, L, R, dx, dL, dR, 0, T, n, m, ws)
+        else:
+            P.monarch_bwd_dw(x, dy, L, R, dL, dR, 0, T, n, m, ws)
+        torch.cuda.synchronize()
+        assert P.monarch_last_device_status(ws) == 0
+        runs.append((dL, dR))
+    assert torch.equal(runs[0][0], runs[1][0]) and torch.equal(runs[0][1], runs[1][1])
+    assert torch.equal(runs[2][0], runs[3][0]) and torch.equal(runs[2][1], runs[3][1])
+    ref = O.bwd(d["x"], d["dy"], d["L"], d["R"])
+    for k in (0, 2):
+        assert_close(to_host64(runs[k][0]), ref["dL"], dtype, "dL")
+        assert_close(to_host64(runs[k][1]), ref["dR"], dtype, "dR")
+
+
 def test_zero_tokens_m128_and_wrapped(P):
     """An empty batch: outputs untouched, weight gradients zeroed (overwrite) or left alone (accumulate)."""
     import torch
