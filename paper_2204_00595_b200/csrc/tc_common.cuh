@@ -335,7 +335,7 @@ int encode_tmap_2d(CUtensorMap *out, const void *base, uint64_t rows, uint64_t c
                    uint64_t row_stride_bytes, uint32_t box_rows, uint32_t box_cols,
                    uint32_t swizzle_bytes);
 
-// General form: `rank` dimensions (innermost first) of `elem_bytes`-wide elements (2 = bf16,
+// General form: `rank` dimensions (innermost first) of `elem_bytes`-wide elements (2 = bf16, 4 = fp32,
 // 8 = opaque 64-bit words), strides in bytes for dimensions 1..rank-1; swizzle_bytes in {0, 32, 128}.
 int encode_tmap_nd(CUtensorMap *out, const void *base, int elem_bytes, int rank, const uint64_t *dims,
                    const uint64_t *strides_bytes, const uint32_t *box, uint32_t swizzle_bytes = 0);

@@ -284,7 +284,7 @@ int encode_tmap_nd(CUtensorMap *out, const void *base, int elem_bytes, int rank,
     for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; es[i] = 1; }
     for (int i = 0; i + 1 < rank; ++i) st[i] = strides_bytes[i];
     const CUtensorMapDataType dt = elem_bytes == 8 ? CU_TENSOR_MAP_DATA_TYPE_UINT64
-                                 : elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_UINT32
+                                 : elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
                                                    : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     const CUresult r = fn(out, dt, (cuuint32_t)rank, const_cast<void *>(base), d, st, b, es,
                           CU_TENSOR_MAP_INTERLEAVE_NONE,
