@@ -37,7 +37,8 @@
  *  - Weight gradients of the fused tensor-core kernels (bf16, m = 64; the
  *    general class) and of the staged tensor-core kernels (bf16, m = 32) are
  *    summed with fp32 reductions whose order across thread blocks is not
- *    fixed: dL, dR can differ in the last fp32 bits from run to run.  The bf16 m = 128 kernels (one thread block sums all tokens of a
+ *    fixed: dL, dR can differ in the last fp32 bits from run to run
+ *    (monarch_set_deterministic switches m = 32 and m = 64 to a fixed order).  The bf16 m = 128 kernels (one thread block sums all tokens of a
  *    block, in a fixed order) and the CUDA-core family (MONARCH_IMPL_STAGED)
  *    give the same bits every run.
  *  - Return value: a monarch_status_t.  Nothing throws.
@@ -289,19 +290,19 @@ int monarch_set_impl(int impl);
 
 /* Summation order of the weight gradients dL[j][l][k] = sum_t dy[t][l*m+j] u[t][k][j]
  * and dR[k][j][i] = sum_t du[t][k][j] x[t][k*m+i] (the adjoints of Section 3.3,
- * steps 1-2) in the fused bf16 m = 64 kernels behind monarch_bwd and
+ * steps 1-2) in the bf16 kernels that split the tokens over thread blocks: m = 64
+ * (fused family) and m = 32 (staged tensor-core family), behind monarch_bwd and
  * monarch_bwd_dw.  on != 0: every thread block writes the partial sums of its
  * (fixed) share of the token tiles to the workspace and a second small launch adds
  * them in a fixed order - the same bits on every run, accumulate honoured by that
  * launch; monarch_workspace_bytes for these two operations then reports 32 MiB
- * more, and a device on which the one-launch backward cannot run gets
+ * more, and at m = 64 a device on which the one-launch backward cannot run gets
  * MONARCH_ERR_UNSUPPORTED instead of the multi-launch form.  on == 0 (default):
  * partial sums are added with fp32 atomics in whatever order they arrive.  Other
  * sizes and dtypes already sum in a fixed order (bf16 m = 128, every fp32 call) or
- * are not affected (bf16 m = 32, the feed-forward block and the general class keep
- * their atomics).  Process-wide,
- * affects later calls and later workspace-size queries; not thread-safe against
- * concurrent calls.  Returns the previous setting. */
+ * are not affected (the feed-forward block and the general class keep their
+ * atomics).  Process-wide, affects later calls and later workspace-size queries;
+ * not thread-safe against concurrent calls.  Returns the previous setting. */
 int monarch_set_deterministic(int on);
 
 /* Name of the kernel family the next call with these arguments would use

@@ -128,11 +128,14 @@ const void *chain_fwd_m128_saved_u(const void *fwd_ws, int64_t tokens);
 void debug_skip_next_plane_load(long long item);
 
 // ---- backward as a chain of tensor-core launches (bf16; dx for m >= 32, dL/dR for m = 128), tc_bwd.cu ----
-size_t tc_staged_bwd_workspace_bytes(int64_t tokens, int m);
+// fixed_order (m = 32, 64): kTcPartialBytes more; the token slices of the weight-gradient launches store their sums there and a
+// small launch adds them in slice order (same bits on every run) instead of reductions in L2
+constexpr size_t kTcPartialBytes = (size_t)32 << 20;
+size_t tc_staged_bwd_workspace_bytes(int64_t tokens, int m, bool fixed_order = false);
 // saved_up: for m = 128, the u' planes left by the forward call (chain_fwd_m128_saved_u), or null
 int tc_staged_bwd(const void *x, const void *dy, const void *L, const void *R, void *dx, float *dL, float *dR,
                   int accumulate, int want_dx, int want_dw, int64_t tokens, int m, void *ws, cudaStream_t s,
-                  const void *saved_up = nullptr);
+                  const void *saved_up = nullptr, bool fixed_order = false);
 
 // ---- forward for m = 16 in one launch on the CUDA cores, both dtypes (fused_m16.cu); no workspace use ----
 int fused_fwd_m16(const void *x, const void *L, const void *R, void *y, int64_t tokens, int dtype, cudaStream_t s);

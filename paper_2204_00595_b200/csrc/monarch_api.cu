@@ -172,7 +172,7 @@ size_t monarch_workspace_bytes(int op, int64_t tokens, int32_t n, int32_t m, int
     // refuse, and so does this query (shard the tokens)
     if (which == kFused && m == 64 && tokens > ((int64_t)1 << 20)) return 0;
     if (which == kTcStaged && op != MONARCH_OP_FWD && op != MONARCH_OP_MLP_FWD)
-        return tc_staged_bwd_workspace_bytes(tokens, m);
+        return tc_staged_bwd_workspace_bytes(tokens, m, op != MONARCH_OP_BWD_DX && g_fixed_order.load(std::memory_order_relaxed) != 0);
     if (which == kTcStaged && op == MONARCH_OP_FWD && m == 128) return chain_fwd_m128_workspace_bytes(tokens);
     if (op == MONARCH_OP_BWD) {
         if (which == kFused) return fused_bwd_m64_workspace_bytes(tokens, g_fixed_order.load(std::memory_order_relaxed) != 0);
@@ -249,7 +249,7 @@ int monarch_bwd_dw(const void *x, const void *dy, const void *L, const void *R, 
                                 g_fixed_order.load(std::memory_order_relaxed) != 0);
     if (which == kTcStaged)
         return tc_staged_bwd(x, dy, L, R, nullptr, dL, dR, accumulate, 0, 1, tokens, m, workspace,
-                             (cudaStream_t)stream);
+                             (cudaStream_t)stream, nullptr, g_fixed_order.load(std::memory_order_relaxed) != 0);
     return staged_bwd_dw(x, dy, L, R, dL, dR, accumulate, tokens, m, dtype, workspace,
                          (cudaStream_t)stream);
 }
@@ -278,7 +278,8 @@ int monarch_bwd(const void *x, const void *dy, const void *L, const void *R, con
     if (which == kTcStaged) {
         const bool saved = fwd_workspace != nullptr && m == 128 && pick(MONARCH_OP_FWD, m, dtype) == kTcStaged;
         return tc_staged_bwd(x, dy, L, R, dx, dL, dR, accumulate, 1, 1, tokens, m, workspace, s,
-                             saved ? chain_fwd_m128_saved_u(fwd_workspace, tokens) : nullptr);
+                             saved ? chain_fwd_m128_saved_u(fwd_workspace, tokens) : nullptr,
+                             g_fixed_order.load(std::memory_order_relaxed) != 0);
     }
     MONARCH_TRY(staged_bwd_dx(dy, L, R, dx, tokens, m, dtype, workspace, s));
     return staged_bwd_dw(x, dy, L, R, dL, dR, accumulate, tokens, m, dtype, workspace, s);

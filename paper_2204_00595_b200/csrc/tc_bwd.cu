@@ -90,6 +90,7 @@ constexpr int kWThreads = 6 * 32;              // warps 0-3 epilogue, 4 loader, 
 
 struct WgradParams {
     float *out;
+    float *part;           // fixed summation order: slice y stores its sums to part[y][block][m][m] instead of adding them to out
     unsigned *status;
     int tiles, slices;
     int m;                 // block size: 128 (a window is one block), 64 or 32 (its 2 or 4 diagonal sub-blocks are blocks)
@@ -193,18 +194,25 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                     // the window's diagonal m x m sub-blocks are the blocks' sums (the rest of the 128 x 128 product pairs
                     // rows and columns of different blocks and is dropped); row `row` of the window is row g % m of block g / m
                     const int g = (blk0 + b) * kWM + row, c0 = (row / p.m) * p.m;     // c0 is uniform over a warp: m >= 32
-                    float *out = p.out + ((long long)(g / p.m) * p.m + g % p.m) * p.m - c0;
+                    float *out = (p.part ? p.part + (size_t)blockIdx.y * p.windows * kWM * p.m : p.out) +
+                                 ((long long)(g / p.m) * p.m + g % p.m) * p.m - c0;
 #pragma unroll 1
                     for (int c = c0; c < c0 + p.m; c += 16) {
                         uint32_t v[16];
                         tmem_ld16(lane_base + b * 128 + c, v);
                         tmem_ld_wait();
 #pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(out + c + e * 4),
-                                         "f"(__uint_as_float(v[e * 4])), "f"(__uint_as_float(v[e * 4 + 1])),
-                                         "f"(__uint_as_float(v[e * 4 + 2])), "f"(__uint_as_float(v[e * 4 + 3]))
-                                         : "memory");
+                        for (int e = 0; e < 4; ++e) {
+                            if (p.part)
+                                *reinterpret_cast<float4 *>(out + c + e * 4) =
+                                    make_float4(__uint_as_float(v[e * 4]), __uint_as_float(v[e * 4 + 1]),
+                                                __uint_as_float(v[e * 4 + 2]), __uint_as_float(v[e * 4 + 3]));
+                            else
+                                asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(out + c + e * 4),
+                                             "f"(__uint_as_float(v[e * 4])), "f"(__uint_as_float(v[e * 4 + 1])),
+                                             "f"(__uint_as_float(v[e * 4 + 2])), "f"(__uint_as_float(v[e * 4 + 3]))
+                                             : "memory");
+                        }
                     }
                 }
             }
@@ -215,8 +223,30 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     if (warp == 0) tmem_dealloc(tmem_base, 512);
 }
 
-// out[g][r][c] += sum_t A[t][g*m + r] B[t][g*m + c] for every block g (m = 32, 64 or 128; A, B token-major [tokens][m*m])
-int launch_wgrad(const void *A, const void *B, float *out, int64_t tokens, int m, unsigned *status, cudaStream_t s)
+// out[i] += part[0][i] + part[1][i] + ... in slice order, for the n*m elements of a weight gradient
+__global__ void __launch_bounds__(256) add_slices_kernel(float *__restrict__ out, const float *__restrict__ part, int slices,
+                                                         int elems)
+{
+    const int i = (blockIdx.x * 256 + threadIdx.x) * 4;
+    if (i >= elems) return;
+    float4 acc = *reinterpret_cast<const float4 *>(part + i);
+    for (int s = 1; s < slices; ++s) {
+        const float4 v = *reinterpret_cast<const float4 *>(part + (size_t)s * elems + i);
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    float4 o = *reinterpret_cast<float4 *>(out + i);
+    o.x += acc.x; o.y += acc.y; o.z += acc.z; o.w += acc.w;
+    *reinterpret_cast<float4 *>(out + i) = o;
+}
+
+// slices of the token tiles that fit the scratch for one gradient's partial sums
+int max_wgrad_slices(int m) { return (int)(kTcPartialBytes / 2 / ((size_t)m * m * m * sizeof(float))); }
+
+// out[g][r][c] += sum_t A[t][g*m + r] B[t][g*m + c] for every block g (m = 32, 64 or 128; A, B token-major [tokens][m*m]).
+// part != null (kTcPartialBytes / 2 of scratch): every slice of the tokens stores its sums there and a second launch adds
+// them to out in slice order - the same bits on every run; else the slices add to out with reductions in L2.
+int launch_wgrad(const void *A, const void *B, float *out, int64_t tokens, int m, unsigned *status, cudaStream_t s,
+                 float *part = nullptr)
 {
     if (tokens == 0) return MONARCH_OK;
     const int n = m * m;
@@ -230,6 +260,7 @@ int launch_wgrad(const void *A, const void *B, float *out, int64_t tokens, int m
     MONARCH_CUDA_TRY(cudaFuncSetAttribute(tc_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmem));
     WgradParams p;
     p.out = out;
+    p.part = part;
     p.status = status;
     p.tiles = (int)((tokens + 63) / 64);
     p.m = m;
@@ -238,9 +269,15 @@ int launch_wgrad(const void *A, const void *B, float *out, int64_t tokens, int m
     int slices = sms / groups;
     if (slices < 1) slices = 1;
     if (slices > p.tiles) slices = p.tiles;
+    if (part != nullptr && slices > max_wgrad_slices(m)) slices = max_wgrad_slices(m);
     p.slices = slices;
     tc_wgrad_kernel<<<dim3(groups, slices), kWThreads, kWSmem, s>>>(tm_a, tm_b, p);
     note_launch();
+    if (part != nullptr) {
+        const int elems = n * m;
+        add_slices_kernel<<<(elems / 4 + 255) / 256, 256, 0, s>>>(out, part, slices, elems);
+        note_launch();
+    }
     MONARCH_CUDA_TRY(cudaGetLastError());
     return MONARCH_OK;
 }
@@ -296,17 +333,17 @@ Layout carve(void *ws, int64_t tokens, int m)
 }  // namespace tc
 
 // Workspace: [status][z][du][u'][L^T][R^T]; m = 128 has its own layout (chain_m128.cu)
-size_t tc_staged_bwd_workspace_bytes(int64_t tokens, int m)
+size_t tc_staged_bwd_workspace_bytes(int64_t tokens, int m, bool fixed_order)
 {
     if (m == 128) return chain_bwd_m128_workspace_bytes(tokens);
     const size_t act = tc::align256((size_t)tokens * m * m * 2), wb = tc::align256((size_t)m * m * m * 2);
-    return MONARCH_STATUS_BYTES + 3 * act + 2 * wb;
+    return MONARCH_STATUS_BYTES + 3 * act + 2 * wb + (fixed_order ? kTcPartialBytes : 0);
 }
 
 // want_dx / want_dw select the outputs
 int tc_staged_bwd(const void *x, const void *dy, const void *L, const void *R, void *dx, float *dL, float *dR,
                   int accumulate, int want_dx, int want_dw, int64_t tokens, int m, void *ws, cudaStream_t s,
-                  const void *saved_up)
+                  const void *saved_up, bool fixed_order)
 {
     using namespace tc;
     if (want_dw && m != 32 && m != 64 && m != 128) return MONARCH_ERR_UNSUPPORTED;
@@ -336,8 +373,10 @@ int tc_staged_bwd(const void *x, const void *dy, const void *L, const void *R, v
     }
     if (want_dw) {
         MONARCH_TRY(tc_stage(m, x, R, l.u, nullptr, 0, tokens, status, s));               // u'[t][j][k]
-        MONARCH_TRY(launch_wgrad(l.du, x, dR, tokens, m, status, s));
-        MONARCH_TRY(launch_wgrad(l.z, l.u, dL, tokens, m, status, s));
+        // fixed summation order on request: the slices' sums go through the scratch behind R^T (one half per gradient)
+        float *part = fixed_order ? (float *)(l.Rt + align256((size_t)m * m * m * 2)) : nullptr;
+        MONARCH_TRY(launch_wgrad(l.du, x, dR, tokens, m, status, s, part));
+        MONARCH_TRY(launch_wgrad(l.z, l.u, dL, tokens, m, status, s, part ? part + kTcPartialBytes / 2 / sizeof(float) : nullptr));
     }
     return MONARCH_OK;
 }

@@ -88,9 +88,10 @@ def test_impl_selection(lib):
         B.monarch_set_impl(prev)
 
 
-def test_deterministic_switch_changes_only_the_m64_backward_workspaces(lib):
-    """monarch_set_deterministic: returns the previous setting; while on, the workspace of the two bf16 m = 64
-    calls that sum weight gradients grows by the 32 MiB of partial sums; every other query is unchanged."""
+def test_deterministic_switch_changes_only_the_split_token_backward_workspaces(lib):
+    """monarch_set_deterministic: returns the previous setting; while on, the workspace of the bf16 m = 32 and m = 64
+    calls that sum weight gradients over token slices grows by the 32 MiB of partial sums; every other query
+    (fp32, m = 128, forward, dx) is unchanged."""
     T = 1000
     def sizes():
         return {(op, m, dt): B.monarch_workspace_bytes(op, T, m * m, m, dt)
@@ -104,9 +105,9 @@ def test_deterministic_switch_changes_only_the_m64_backward_workspaces(lib):
     finally:
         B.monarch_set_deterministic(False)
     grown = {k for k in before if after[k] != before[k]}
-    assert grown == {(B.OP_BWD_DW, 64, B.BF16), (B.OP_BWD, 64, B.BF16)}
+    assert grown == {(B.OP_BWD_DW, 64, B.BF16), (B.OP_BWD, 64, B.BF16), (B.OP_BWD_DW, 32, B.BF16), (B.OP_BWD, 32, B.BF16)}
     for k in grown:
-        assert after[k] - before[k] == 2 * 16 * 64 ** 3 * 4
+        assert after[k] - before[k] == 32 << 20
     assert sizes() == before
 
 

@@ -1182,6 +1182,53 @@ def test_m128_weight_gradients_have_the_same_bits_every_run(P):
     assert_close(to_host64(runs[3][1] - 0.5), ref["dR"], dtype, "dR accumulated onto 0.5")
 
 
+@pytest.mark.parametrize("T", [1, 129, 64 * 150 + 7])
+def test_bwd_m32_fixed_summation_order(P, T):
+    """monarch_set_deterministic(1) at bf16 m = 32 (token reductions on the tensor cores, split over token slices):
+    runs from different initial contents give the same bits through monarch_bwd and monarch_bwd_dw, both match the
+    oracle, accumulate = 1 adds to what is there, and a workspace sized before the switch is refused."""
+    import torch
+    m, dtype, code = 32, "bf16", P.BF16
+    n = m * m
+    d = _small_inputs(m, T, dtype, seed=3200 + T)
+    x, dy, L, R = (to_device(d[k], dtype) for k in ("x", "dy", "L", "R"))
+    ref = O.bwd(d["x"], d["dy"], d["L"], d["R"])
+    small = P.monarch_workspace_bytes(P.OP_BWD, T, n, m, code)
+    prev = P.monarch_set_deterministic(True)
+    try:
+        assert P.monarch_impl_name(P.OP_BWD, m, code) == "staged-tcgen05"
+        nb = P.monarch_workspace_bytes(P.OP_BWD, T, n, m, code)
+        assert nb == small + (32 << 20)
+        ws = P.Workspace(max(nb, P.monarch_workspace_bytes(P.OP_BWD_DW, T, n, m, code)))
+        dx = torch.empty_like(x)
+        runs = []
+        for fill, one_call in ((float("nan"), True), (11.0, True), (-3.0, False), (0.5, False)):
+            dL = torch.full((m, m, m), fill, device="cuda")
+            dR = torch.full((m, m, m), fill, device="cuda")
+            if one_call:
+                P.monarch_bwd(x, dy, L, R, dx, dL, dR, 0, T, n, m, ws)
+            else:
+                P.monarch_bwd_dw(x, dy, L, R, dL, dR, 0, T, n, m, ws)
+            torch.cuda.synchronize()
+            assert P.monarch_last_device_status(ws) == 0
+            runs.append((dL, dR))
+        for dL, dR in runs[1:]:
+            assert torch.equal(dL, runs[0][0]) and torch.equal(dR, runs[0][1])
+        assert_close(to_host64(dx), ref["dx"], dtype, "dx")
+        assert_close(to_host64(runs[0][0]), ref["dL"], dtype, "dL fixed order")
+        assert_close(to_host64(runs[0][1]), ref["dR"], dtype, "dR fixed order")
+        dL, dR = runs[0][0].clone(), runs[0][1].clone()
+        P.monarch_bwd_dw(x, dy, L, R, dL, dR, 1, T, n, m, ws)
+        torch.cuda.synchronize()
+        assert_close(to_host64(dL), 2 * ref["dL"], dtype, "dL accumulate, fixed order")
+        assert_close(to_host64(dR), 2 * ref["dR"], dtype, "dR accumulate, fixed order")
+        with pytest.raises(P.MonarchError):
+            P.monarch_bwd(x, dy, L, R, dx, dL, dR, 0, T, n, m, P.Workspace(small))
+    finally:
+        P.monarch_set_deterministic(prev)
+    assert P.monarch_workspace_bytes(P.OP_BWD, T, n, m, code) == small
+
+
 @pytest.mark.parametrize("m", [16, 32, 64])
 def test_fp32_weight_gradients_have_the_same_bits_every_run(P, m):
     """fp32 runs on the CUDA-core family, whose token sums are taken slab by slab and added in slab order: dL and dR
