@@ -170,7 +170,8 @@ def monarch_set_impl(impl: int) -> int:
 
 
 def monarch_set_deterministic(on: bool) -> bool:
-    """Fixed summation order for dL, dR of the fused bf16 m = 64 backward; returns the previous setting."""
+    """Fixed summation order for dL, dR of the bf16 m = 32 and m = 64 backward (the calls that split the tokens
+    over thread blocks; their workspaces grow by 32 MiB while it is on); returns the previous setting."""
     return bool(lib().monarch_set_deterministic(1 if on else 0))
 
 
