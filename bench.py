@@ -161,8 +161,9 @@ class ClockSampler:
 
 # ----------------------------------------------------------------------------- CPU oracle timing
 
-def time_oracle(cfg, d, target_s=12.0, calls=None):
-    """Time the oracle (as it stands) on a bounded token sample of the workload."""
+def time_oracle(cfg, d, target_s=12.0, calls=None, tokens=None):
+    """Time the oracle (as it stands) on a bounded token sample of the workload: `tokens` of them, or (None) as many
+    as a short calibration says take about target_s seconds."""
     from oracle import monarch_oracle as O
     c = cfg
     calls = list(c.ops) if calls is None else [k for k in calls if k != "bwd"] + (
@@ -182,15 +183,19 @@ def time_oracle(cfg, d, target_s=12.0, calls=None):
             O.mlp_bwd(d["x"][:T], d["dy"][:T], d["L"], d["R"], d["b1"], d["L2"], d["R2"])
         return time.perf_counter() - t0
 
-    T = min(32, c.tokens)
-    dt = run(T)
-    while dt < 0.5 and T < c.tokens:
-        T = min(T * 4, c.tokens)
+    if tokens is not None:
+        T = int(min(c.tokens, max(1, tokens)))
         dt = run(T)
-    Ts = int(min(c.tokens, max(T, T * target_s / max(dt, 1e-9))))
-    if Ts != T:
-        dt = run(Ts)
-        T = Ts
+    else:
+        T = min(32, c.tokens)
+        dt = run(T)
+        while dt < min(0.5, target_s) and T < c.tokens:
+            T = min(T * 4, c.tokens)
+            dt = run(T)
+        Ts = int(min(c.tokens, max(8, T * target_s / max(dt, 1e-9))))
+        if Ts != T:
+            dt = run(Ts)
+            T = Ts
     flops = sum(call_flops(k, c.n, c.m, T) for k in calls)
     return {"tflops": flops / dt / 1e12, "tokens": T, "seconds": dt, "cores": O.num_threads(),
             "tokens_per_s": T / dt}
@@ -791,10 +796,12 @@ def main():
         from oracle import monarch_oracle as O
         O.build()
         d = make_inputs(cfg.index, with_dy="mlp_bwd" in calls)
+        # every step runs the oracle on the same bounded sample: sized once (first step) so that warm-up plus timed
+        # steps take about two minutes, whatever --steps is
         times, sample = [], None
+        per_step = max(0.05, min(8.0, 120.0 / (args.warmup + args.steps)))
         for i in range(args.warmup + args.steps):
-            r = time_oracle(cfg, d, target_s=max(1.0, min(8.0, 120.0 / (args.warmup + args.steps))),
-                            calls=calls)
+            r = time_oracle(cfg, d, target_s=per_step, calls=calls, tokens=sample["tokens"] if sample else None)
             sample = r
             if i >= args.warmup:
                 times.append(r)
