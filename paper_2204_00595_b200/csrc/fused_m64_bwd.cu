@@ -654,22 +654,35 @@ __device__ __forceinline__ bool wait_tile(const BwdParams &p, int tile, volatile
     return true;
 }
 
-__device__ __forceinline__ void red_add_v4(float *p, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+// A weight gradient's sums leave TMEM through shared memory and tiled TMA copies (boxes of 16 rows x 32 fp32 columns,
+// 128-byte rows, swizzled): added to the gradient in L2, or stored to this CTA's slot of the partial sums.  Plain
+// 16-byte reductions from the epilogue threads, each to its own 256-byte row, took 8 us of the call.
+__device__ __forceinline__ void grad_box_out(const CUtensorMap *m, uint32_t src, int x, int y, bool store)
 {
-    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(__uint_as_float(a)),
-                 "f"(__uint_as_float(b)), "f"(__uint_as_float(c)), "f"(__uint_as_float(d))
-                 : "memory");
+    if (store)
+        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(m), "r"(src), "r"(x), "r"(y)
+                     : "memory");
+    else
+        asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];" ::"l"(m),
+                     "r"(src), "r"(x), "r"(y)
+                     : "memory");
 }
-
-__device__ __forceinline__ void store_v4(float *p, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+// One warp, one block iteration: lanes with `active` hold 32 columns (v) of row r16 (0..15) of their block; `box` is
+// this lane's 2 KB box in the warp's staging area.
+__device__ __forceinline__ void grad_stage_row(uint32_t box, int r16, const uint32_t (&v)[2][16])
 {
-    *reinterpret_cast<uint4 *>(p) = make_uint4(a, b, c, d);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        const uint32_t *w = &v[e >> 2][(e & 3) * 4];
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(box + r16 * 128 + ((e ^ (r16 & 7)) << 4)), "r"(w[0]), "r"(w[1]),
+                     "r"(w[2]), "r"(w[3]) : "memory");
+    }
 }
 
 constexpr int kRSlotBytes = 16384;               // B2R / WL ring slot: two 8 KB operands of one block
 
 __device__ __forceinline__ void b2r_body(const CUtensorMap &tm_R, const CUtensorMap &tm_x, const CUtensorMap &tm_dx,
-                                         const BwdParams &p, uint32_t smem0, Bars *bars, volatile int *dep_items,
+                                         const CUtensorMap &tm_gR, const BwdParams &p, uint32_t smem0, Bars *bars, volatile int *dep_items,
                                          uint32_t tmem_base, volatile int *dead, int grp, int first)
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -815,29 +828,39 @@ __device__ __forceinline__ void b2r_body(const CUtensorMap &tm_R, const CUtensor
                 if (lane == 0) mbar_arrive(stf0 + k * 8);
             }
         }
-        // dR partial sums of this CTA's tiles: lanes 16-31 of each quarter hold row 16 q4 + lane - 16 of block b
+        // dR partial sums of this CTA's tiles: lanes 16-31 of each quarter hold row 16 q4 + lane - 16 of block b.  The
+        // operand ring is idle by now: every warp stages its 16 rows of a block there (two boxes of 32 columns, two
+        // buffers in turn) and its lane 0 sends them off
         if (!mbar_wait(drf, 0, p.status, dead, kErrMmaWait)) return;
         tc_fence_after();
         const bool part = p.part_dR != nullptr;
-        float *out = (part ? p.part_dR + (size_t)first * (64 * 4096) : p.dR) + (long long)(grp * 8) * 4096 + row * 64;
+        const uint32_t wst = ring0 + warp * 8192;
+        const int row0 = (part ? first * 4096 : 0) + (grp * 8) * 64 + q4 * 16;
+        int it = 0;
 #pragma unroll 1
-        for (int b = sub * 4; b < sub * 4 + 4; ++b) {
+        for (int b = sub * 4; b < sub * 4 + 4; ++b, ++it) {
+            const uint32_t buf = wst + (it & 1) * 4096;
+            if (it >= 2) {
+                if (lane == 0) tma_store_wait_read<1>();
+                __syncwarp();
+            }
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 uint32_t v[2][16];
                 tmem_ld16(lane_base + b * 64 + h * 32, v[0]);
                 tmem_ld16(lane_base + b * 64 + h * 32 + 16, v[1]);
                 tmem_ld_wait();
-                if (!mine) {
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const uint32_t *w = &v[e >> 2][(e & 3) * 4];
-                        if (part) store_v4(out + b * 4096 + h * 32 + e * 4, w[0], w[1], w[2], w[3]);
-                        else red_add_v4(out + b * 4096 + h * 32 + e * 4, w[0], w[1], w[2], w[3]);
-                    }
-                }
+                if (!mine) grad_stage_row(buf + h * 2048, lane & 15, v);
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                grad_box_out(&tm_gR, buf, 0, row0 + b * 64, part);
+                grad_box_out(&tm_gR, buf + 2048, 32, row0 + b * 64, part);
+                tma_store_commit();
             }
         }
+        if (lane == 0) tma_store_wait_all<0>();
     } else if (warp >= kStoreWarp0 && warp < kStoreWarp0 + 2) {
         if (lane != 0 || !p.want_dx) return;
         const int sub = warp - kStoreWarp0;
@@ -846,7 +869,7 @@ __device__ __forceinline__ void b2r_body(const CUtensorMap &tm_R, const CUtensor
     }
 }
 
-__device__ __forceinline__ void wl_body(const BwdParams &p, uint32_t ring0, Bars *bars, volatile int *dep_items,
+__device__ __forceinline__ void wl_body(const CUtensorMap &tm_gL, const BwdParams &p, uint32_t ring0, Bars *bars, volatile int *dep_items,
                                         uint32_t tmem_base, volatile int *dead, int grp, int first)
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -918,25 +941,38 @@ __device__ __forceinline__ void wl_body(const BwdParams &p, uint32_t ring0, Bars
         if (!mbar_wait(accf, 0, p.status, dead, kErrMmaWait)) return;
         tc_fence_after();
         const uint32_t lane_base = tmem_base + ((uint32_t)(q4 * 32) << 16);
-        const int row = q4 * 16 + (lane & 15);
+        // lanes 0-15 hold rows 16 q4 + lane of block blk0 + b, lanes 16-31 the same rows of block blk0 + 8 + b; staging
+        // in the idle operand ring as in the dR flush: four boxes (two blocks x two halves of the columns) per step
         const bool part = p.part_dL != nullptr;
-        float *out = (part ? p.part_dL + (size_t)first * (64 * 4096) : p.dL) + (long long)(blk0 + (lane >> 4) * 8) * 4096 + row * 64;
+        const uint32_t wst = ring0 + warp * 16384;
+        const int sel = lane >> 4;
+        const int row0 = (part ? first * 4096 : 0) + blk0 * 64 + q4 * 16;
+        int it = 0;
 #pragma unroll 1
-        for (int b = sub * 4; b < sub * 4 + 4; ++b) {
+        for (int b = sub * 4; b < sub * 4 + 4; ++b, ++it) {
+            const uint32_t buf = wst + (it & 1) * 8192;
+            if (it >= 2) {
+                if (lane == 0) tma_store_wait_read<1>();
+                __syncwarp();
+            }
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 uint32_t v[2][16];
                 tmem_ld16(lane_base + b * 64 + h * 32, v[0]);
                 tmem_ld16(lane_base + b * 64 + h * 32 + 16, v[1]);
                 tmem_ld_wait();
+                grad_stage_row(buf + (sel * 2 + h) * 2048, lane & 15, v);
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const uint32_t *w = &v[e >> 2][(e & 3) * 4];
-                    if (part) store_v4(out + b * 4096 + h * 32 + e * 4, w[0], w[1], w[2], w[3]);
-                    else red_add_v4(out + b * 4096 + h * 32 + e * 4, w[0], w[1], w[2], w[3]);
-                }
+                for (int k = 0; k < 4; ++k)
+                    grad_box_out(&tm_gL, buf + k * 2048, (k & 1) * 32, row0 + ((k >> 1) * 8 + b) * 64, part);
+                tma_store_commit();
             }
         }
+        if (lane == 0) tma_store_wait_all<0>();
     }
 }
 
@@ -944,6 +980,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 fused_bwd_all_m64_kernel(const __grid_constant__ CUtensorMap tm_dy3, const __grid_constant__ CUtensorMap tm_Lt,
                          const __grid_constant__ CUtensorMap tm_R, const __grid_constant__ CUtensorMap tm_du,
                          const __grid_constant__ CUtensorMap tm_dx, const __grid_constant__ CUtensorMap tm_x,
+                         const __grid_constant__ CUtensorMap tm_gL, const __grid_constant__ CUtensorMap tm_gR,
                          const BwdParams p)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -985,7 +1022,8 @@ fused_bwd_all_m64_kernel(const __grid_constant__ CUtensorMap tm_dy3, const __gri
         dead = 0;
         dep_items = 0;
         if (kind == 0) { tma_prefetch_desc(&tm_dy3); tma_prefetch_desc(&tm_Lt); }
-        else if (kind == 1) { tma_prefetch_desc(&tm_R); tma_prefetch_desc(&tm_dx); tma_prefetch_desc(&tm_x); }
+        else if (kind == 1) { tma_prefetch_desc(&tm_R); tma_prefetch_desc(&tm_dx); tma_prefetch_desc(&tm_x); tma_prefetch_desc(&tm_gR); }
+        else tma_prefetch_desc(&tm_gL);
     }
     if (warp == 0) {
         tmem_alloc(smem_u32(&tmem_base_s), 512);
@@ -997,8 +1035,8 @@ fused_bwd_all_m64_kernel(const __grid_constant__ CUtensorMap tm_dy3, const __gri
     const uint32_t tmem_base = tmem_base_s;
 
     if (kind == 0) b1_body(tm_dy3, tm_Lt, p, smem0, &bars, tmem_base, &dead, grp, first);
-    else if (kind == 1) b2r_body(tm_R, tm_x, tm_dx, p, smem0, &bars, &dep_items, tmem_base, &dead, grp, first);
-    else wl_body(p, smem0, &bars, &dep_items, tmem_base, &dead, grp, first);
+    else if (kind == 1) b2r_body(tm_R, tm_x, tm_dx, tm_gR, p, smem0, &bars, &dep_items, tmem_base, &dead, grp, first);
+    else wl_body(tm_gL, p, smem0, &bars, &dep_items, tmem_base, &dead, grp, first);
 
     tc_fence_before();
     __syncthreads();
@@ -1167,6 +1205,15 @@ int fused_bwd_all_m64(const void *x, const void *dy, const void *L, const void *
     if (partials != nullptr && (b2 > kBwdMaxPartials || b3 > kBwdMaxPartials)) return MONARCH_ERR_UNSUPPORTED;
     p.part_dR = partials;
     p.part_dL = partials ? partials + (size_t)kBwdMaxPartials * (kN * kM) : nullptr;
+    // the gradients (or the slots of the partial sums) as [rows of 64 fp32] in boxes of 16 rows x 32 columns
+    CUtensorMap tm_gL, tm_gR;
+    {
+        const uint64_t rows = (uint64_t)(partials ? kBwdMaxPartials : 1) * kN;
+        const uint64_t dims[2] = {(uint64_t)kM, rows}, strides[1] = {(uint64_t)kM * sizeof(float)};
+        const uint32_t box[2] = {32, 16};
+        MONARCH_TRY(encode_tmap_nd(&tm_gL, partials ? p.part_dL : dL, 4, 2, dims, strides, box, 128));
+        MONARCH_TRY(encode_tmap_nd(&tm_gR, partials ? p.part_dR : dR, 4, 2, dims, strides, box, 128));
+    }
     p.b1 = b1;
     p.b2 = b2;
     p.b3 = b3;
@@ -1177,7 +1224,7 @@ int fused_bwd_all_m64(const void *x, const void *dy, const void *L, const void *
     if (const char *e = getenv("MONARCH_TRACE_PTR_BWD")) p.trace = (long long *)strtoull(e, nullptr, 0);
 #endif
     fused_bwd_all_m64_kernel<<<8 * b1 + 8 * b2 + 4 * b3, kThreads, kSmemBytes, s>>>(tm_dy3, tm_Lt, tm_R, tm_du, tm_dx,
-                                                                                 tm_x, p);
+                                                                                 tm_x, tm_gL, tm_gR, p);
     note_launch();
     MONARCH_CUDA_TRY(cudaGetLastError());
     if (partials != nullptr) {
